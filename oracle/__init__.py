@@ -1,0 +1,25 @@
+"""CPU fp64 oracle for the TS-DP speculative denoising round (arXiv 2512.15773).
+
+TEST INFRASTRUCTURE ONLY.  This package is the slow, plain definition of what the
+CUDA path must compute.  It may be imported by the test-suite, by the smoke check
+and by the benchmark's CPU-baseline leg -- never by the product package, which has
+no CPU fallback and fails loudly when its CUDA library is missing.  It shares no
+code with the CUDA path: the counter-based random generator, the DDPM tables and
+both networks are written a second time here, in numpy fp64, from the paper's
+equations (Sec. 3.1 Eqs. 1-3 and the reflection-coupling equations, Sec. 3.2
+Eq. (3) and the log-acceptance-ratio equation) and from the textbook DDPM
+posterior the paper refers to as "the DDPM scheduler".
+
+Pin status (what checks each part against something other than itself):
+  philox.py   pinned  : published known-answer vectors of Philox4x32-10.
+  ddpm.py     pinned  : direct products, closed forms, the affine-Gaussian recursion.
+  spec.py     pinned  : Gaussian log-density identity, Householder invariants,
+                        closed-form acceptance rate 2*Phi(-|d|/2), brute-force
+                        first-rejection enumeration, drafter==base == vanilla,
+                        KS test against the analytic marginal of the sampler.
+  nets.py     parity unpinned against the paper (its trained networks and exact
+              layer layout are not published); pinned only by structural
+              invariants (causality, zero-weight behaviour, a hand-computed
+              1-token case) -- see the function headers.
+  sigma_scale parity unpinned against the paper (formula not given there).
+"""

@@ -1,0 +1,106 @@
+"""The denoisers eps = M(x, tau; obs) in numpy fp64: closed-form Gaussian toy, MLP, transformer.
+
+The paper states only the block counts ("DP consists of 8 Transformer blocks while the drafter
+contains only one", Sec. 4) and that the drafter has the same input-output interface and shares
+the encoder and scheduler (Sec. 3.2 "Draft Model Training").  Everything below that is more
+specific than that is this build's own architecture definition; parity with the paper's trained
+networks is UNPINNED (no weights or layer layout are published).  The pins that exist are
+structural: causality of self-attention, independence of candidates, zero-head => zero output,
+and the closed-form Gaussian denoiser against the analytic posterior mean.
+
+Parameters are dicts of float64 arrays produced by the seeded input generators; a linear layer
+y = x W + b stores W as [in, out].
+"""
+import numpy as np
+from .ddpm import sinusoidal_embedding
+
+
+# ----------------------------------------------------------------------------- Gaussian toy
+def gauss_eps(p, sched, x, tau):
+    """Optimal noise prediction when the data are iid N(m0, s0^2) per coordinate:
+
+    E[eps | x_tau] = sqrt(1 - abar) (x - sqrt(abar) m0) / (abar s0^2 + 1 - abar)."""
+    ab = sched.abar[tau]
+    return np.sqrt(1.0 - ab) * (x - np.sqrt(ab) * p["m0"]) / (ab * p["s0"] ** 2 + 1.0 - ab)
+
+
+# ----------------------------------------------------------------------------- MLP
+def silu(v):
+    return v / (1.0 + np.exp(-v))
+
+
+def mlp_eps(p, x, tau, obs):
+    """Input = [flattened latent | sinusoidal(tau, temb) | flattened obs]; `layers` hidden
+    SiLU layers; linear head back to the latent shape."""
+    temb = p["temb"]
+    h = np.concatenate([x.reshape(-1), sinusoidal_embedding(tau, temb), obs.reshape(-1)])
+    for W, b in zip(p["W"][:-1], p["b"][:-1]):
+        h = silu(h @ W + b)
+    return (h @ p["W"][-1] + p["b"][-1]).reshape(x.shape)
+
+
+# ----------------------------------------------------------------------------- transformer
+def layer_norm(h, g, b, eps=1e-5):
+    m = h.mean(axis=-1, keepdims=True)
+    v = ((h - m) ** 2).mean(axis=-1, keepdims=True)
+    return (h - m) / np.sqrt(v + eps) * g + b
+
+
+def gelu_tanh(v):
+    return 0.5 * v * (1.0 + np.tanh(np.sqrt(2.0 / np.pi) * (v + 0.044715 * v ** 3)))
+
+
+def softmax(s):
+    s = s - s.max(axis=-1, keepdims=True)
+    e = np.exp(s)
+    return e / e.sum(axis=-1, keepdims=True)
+
+
+def attention(q, k, v, heads, causal):
+    """Multi-head scaled dot-product attention; q [Nq,d], k,v [Nk,d]."""
+    Nq, d = q.shape
+    dh = d // heads
+    out = np.empty_like(q)
+    for h in range(heads):
+        sl = slice(h * dh, (h + 1) * dh)
+        s = q[:, sl] @ k[:, sl].T / np.sqrt(dh)
+        if causal:
+            s = np.where(np.tril(np.ones_like(s, dtype=bool)), s, -np.inf)
+        out[:, sl] = softmax(s) @ v[:, sl]
+    return out
+
+
+def xfmr_eps(p, x, tau, obs):
+    """Pre-LN decoder: tokens = latent rows [H, A] -> d; memory = [time token | obs tokens].
+
+    h   = x W_in + b_in + pos
+    mem = [sinusoidal(tau, d) ; obs W_obs + b_obs] + cpos
+    per block:  h += SelfAttn_causal(LN1 h);  h += CrossAttn(LN2 h, mem);  h += MLP_gelu(LN3 h)
+    eps = LN_f(h) W_out + b_out
+    """
+    d, heads = p["d"], p["heads"]
+    h = x @ p["W_in"] + p["b_in"] + p["pos"]
+    mem = np.vstack([sinusoidal_embedding(tau, d)[None, :], obs @ p["W_obs"] + p["b_obs"]]) + p["cpos"]
+    for L in p["layers"]:
+        a = layer_norm(h, L["ln1_g"], L["ln1_b"])
+        qkv = a @ L["Wqkv"] + L["bqkv"]
+        h = h + attention(qkv[:, :d], qkv[:, d:2 * d], qkv[:, 2 * d:], heads, True) @ L["Wo"] + L["bo"]
+        a = layer_norm(h, L["ln2_g"], L["ln2_b"])
+        q = a @ L["Wq2"] + L["bq2"]
+        kv = mem @ L["Wkv2"] + L["bkv2"]
+        h = h + attention(q, kv[:, :d], kv[:, d:], heads, False) @ L["Wo2"] + L["bo2"]
+        a = layer_norm(h, L["ln3_g"], L["ln3_b"])
+        h = h + gelu_tanh(a @ L["W1"] + L["b1"]) @ L["W2"] + L["b2"]
+    return layer_norm(h, p["lnf_g"], p["lnf_b"]) @ p["W_out"] + p["b_out"]
+
+
+def make_denoiser(p, sched):
+    """Return eps(x [H,A], tau, obs [To,Do]) for a parameter dict with key 'arch'."""
+    arch = p["arch"]
+    if arch == "gauss":
+        return lambda x, tau, obs: gauss_eps(p, sched, x, tau)
+    if arch == "mlp":
+        return lambda x, tau, obs: mlp_eps(p, x, tau, obs)
+    if arch == "xfmr":
+        return lambda x, tau, obs: xfmr_eps(p, x, tau, obs)
+    raise ValueError(arch)

@@ -1,0 +1,143 @@
+"""Chain-level pins: speculative sampling against vanilla DDPM and against the analytic marginal."""
+import os
+from concurrent.futures import ProcessPoolExecutor
+
+import numpy as np
+import pytest
+from scipy import stats
+
+from oracle import ddpm, nets, spec
+from paper_2512_15773_b200 import inputs
+
+S = ddpm.Schedule(100, 1e-4, 0.02)
+
+
+def _toy_nets(gamma=0.3):
+    wl = dict(inputs.WORKLOADS["toy_mlp"])
+    base = nets.make_denoiser(inputs.make_net(1, wl, "base", gamma=gamma), S)
+    draft = nets.make_denoiser(inputs.make_net(2, wl, "draft", gamma=gamma), S)
+    obs = inputs.make_obs(0, 1, wl["To"], wl["Do"])[0]
+    return base, draft, obs, (wl["H"], wl["A"])
+
+
+def test_drafter_equal_to_base_accepts_everything_and_reproduces_vanilla():
+    base, _, obs, shape = _toy_nets()
+    ref = spec.sample_vanilla(S, base, spec.PhiloxNoise(5), 2, obs, shape)
+    for K in (1, 4, 7):
+        for bonus in (True, False):
+            x, st = spec.sample_chunk(S, base, base, spec.PhiloxNoise(5), 2, obs, shape, K,
+                                      spec.Accept(bonus=bonus))
+            assert st["accepted"] == st["draft_evals"] and st["rejections"] == 0
+            assert np.array_equal(x, ref)
+
+
+def test_k0_is_vanilla_and_k1_without_bonus_takes_T_base_calls():
+    base, draft, obs, shape = _toy_nets()
+    ref = spec.sample_vanilla(S, base, spec.PhiloxNoise(9), 0, obs, shape)
+    x, st = spec.sample_chunk(S, base, draft, spec.PhiloxNoise(9), 0, obs, shape, 0, spec.Accept())
+    assert np.array_equal(x, ref) and st["rounds"] == 100 and st["base_evals"] == 100
+    x, st = spec.sample_chunk(S, base, draft, spec.PhiloxNoise(9), 0, obs, shape, 1,
+                              spec.Accept(bonus=False))
+    assert st["rounds"] == 100 and st["base_evals"] == 100 and st["draft_evals"] == 99
+
+
+def test_round_bookkeeping_and_planted_uniforms():
+    """Every accept pattern for K <= 3 is forced through the uniforms; the round must commit
+    exactly the accepted prefix, reflect at j*, and advance t by the right amount."""
+    base, draft, obs, shape = _toy_nets()
+
+    class Planted(spec.PhiloxNoise):
+        def __init__(self, seed, us):
+            super().__init__(seed); self.us = us
+
+        def u(self, env, tau):
+            return self.us[tau]
+
+    x0 = spec.PhiloxNoise(1).x_init(0, shape)
+    t = 60
+    for K in (1, 2, 3):
+        for pat in np.ndindex(*(2,) * K):
+            us = {t - k + 1: (1e-300 if pat[k - 1] else 1.0 - 1e-16) for k in range(1, K + 1)}
+            x, t_new, d = spec.spec_round(S, base, draft, Planted(1, us), 0, obs, x0, t, K, spec.Accept())
+            rej = [k for k in range(1, K + 1) if not pat[k - 1]]
+            if rej:
+                j = rej[0]
+                assert d["jstar"] == j and t_new == t - j
+                assert np.allclose(x, spec.reflect(d["x_tilde"][j], d["mu_hat"][j], d["mu"][j]))
+            else:
+                assert d["jstar"] == K + 1 and t_new == t - K - 1
+                tau = t - K
+                assert np.allclose(x, d["mu"][K + 1] + S.sigma[tau] * spec.PhiloxNoise(1).xi(0, tau, shape))
+            # every candidate's base mean is the posterior of the latent it was evaluated on
+            for k in range(d["n_base"]):
+                assert np.allclose(d["mu"][k + 1], S.posterior_mean(d["x_tilde"][k], d["eps"][k], t - k))
+
+
+def test_chunk_accounting():
+    base, draft, obs, shape = _toy_nets(gamma=0.05)
+    for K, bonus in ((4, True), (8, True), (3, False)):
+        _, st = spec.sample_chunk(S, base, draft, spec.PhiloxNoise(3), 1, obs, shape, K, spec.Accept(bonus=bonus))
+        adv = st["accepted"] + st["rejections"] + st["bonus"]
+        assert adv == 100
+        assert st["prop_hist"].sum() == st["draft_evals"] and st["acc_hist"].sum() == st["accepted"]
+        assert st["prop_hist"][0] == 0                       # the sigma_0 transition is never drafted
+        assert np.all(st["acc_hist"] <= st["test_hist"]) and np.all(st["test_hist"] <= st["prop_hist"])
+
+
+# ----------------------------------------------------------------------------- KS pin (10^5 chains)
+M0, S0 = 0.7, 0.5
+
+
+def _analytic_marginal():
+    """Law of the sampler's output when eps is the optimal denoiser of N(M0, S0^2) data: each reverse
+    transition is x_{t-1} = a_t x_t + b_t + sigma_t xi, so mean and variance follow a linear recursion
+    from N(0,1).  a_t, b_t come from E[x0 | x_t] by Gaussian conditioning and the Bayes-product form
+    of q(x_{t-1} | x_t, x0) -- not from the oracle's eps-parameterised formulas."""
+    mean, var = 0.0, 1.0
+    for t in range(99, -1, -1):
+        ab = S.abar[t]
+        g = np.sqrt(ab) * S0 ** 2 / (ab * S0 ** 2 + 1 - ab)            # d E[x0|x_t] / d x_t
+        if t > 0:
+            prec = S.alpha[t] / S.beta[t] + 1.0 / (1.0 - S.abar[t - 1])
+            cx0 = np.sqrt(S.abar[t - 1]) / (1.0 - S.abar[t - 1]) / prec
+            cxt = np.sqrt(S.alpha[t]) / S.beta[t] / prec
+            sig2 = 1.0 / prec
+        else:
+            cx0, cxt, sig2 = 1.0, 0.0, 0.0
+        a = cx0 * g + cxt
+        b = cx0 * (M0 - g * np.sqrt(ab) * M0)
+        mean, var = a * mean + b, a * a * var + sig2
+    return mean, np.sqrt(var)
+
+
+def _run_block(args):
+    kind, env0, n = args
+    base = nets.make_denoiser(inputs.make_gauss_params(M0, S0), S)
+    draft = nets.make_denoiser(inputs.make_gauss_params(M0 + 0.25, 0.8 * S0), S)
+    envs = list(range(env0, env0 + n))
+    noise = spec.TableNoise(1234, envs, 100, 1)
+    out = np.empty(n); acc = tested = 0
+    for i, e in enumerate(envs):
+        if kind == "vanilla":
+            out[i] = spec.sample_vanilla(S, base, noise, e, None, (1,))[0]
+        else:
+            x, st = spec.sample_chunk(S, base, draft, noise, e, None, (1,), 6, spec.Accept())
+            out[i] = x[0]; acc += st["accepted"]; tested += st["test_hist"].sum()
+    return out, acc, tested
+
+
+@pytest.mark.parametrize("kind", ["vanilla", "speculative"])
+def test_gaussian_toy_matches_analytic_marginal(kind):
+    N, blk = 100_000, 2_500
+    jobs = [(kind, e0, blk) for e0 in range(0, N, blk)]
+    with ProcessPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as ex:
+        res = list(ex.map(_run_block, jobs))
+    x = np.concatenate([r[0] for r in res])
+    mean, std = _analytic_marginal()
+    # abar_T = 0.36 for this 100-step schedule, so starting from N(0,1) leaves a visible bias:
+    # the sampler's law is near, not equal to, the data law N(M0, S0^2)
+    assert abs(mean - M0) < 0.15 and abs(std - S0) < 0.15
+    assert stats.kstest((x - mean) / std, "norm").pvalue > 0.01
+    if kind == "speculative":
+        rate = sum(r[1] for r in res) / sum(r[2] for r in res)
+        assert 0.2 < rate < 0.98                                 # rejections really happen

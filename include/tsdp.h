@@ -1,0 +1,166 @@
+/* tsdp.h -- C ABI of the B200 (sm_100a) implementation of the TS-DP speculative denoising loop for
+ * Diffusion Policy (arXiv 2512.15773).
+ *
+ * One context samples action chunks for up to max_B independent environments.  One chunk is T DDPM
+ * reverse steps, taken in speculative rounds (Sec. 3.2 of the paper):
+ *   1. the drafter rolls out K reverse steps with the shared DDPM scheduler         (Eq. (3));
+ *   2. the base denoiser is evaluated on all K+1 candidate latents of every environment in one
+ *      batched forward                                         ("Verification of Speculative Drafts");
+ *   3. per drafted step the Gaussian log acceptance ratio  log a = -1/2 |d|^2 - <d, xi>,
+ *      d = (mu^ - mu) / (s sigma)  is tested, the accepted prefix is committed, and the first rejected
+ *      step is replaced by its reflection-maximal coupling             (Sec. 3.1, Eqs. (1)-(3) and the
+ *      reflection equations).
+ *
+ * Conventions.  All pointers named d_* are DEVICE pointers, h_* are HOST pointers.  Arrays are dense,
+ * row-major, fp32 unless stated.  Timestep t in {T-1..0}: a network called with t receives the latent
+ * "at t"; the transition at t produces the latent at t-1; the latent at -1 is the clean action chunk.
+ * Every function returns a tsdp_status; nothing throws or aborts.  A context is not re-entrant: one
+ * call at a time.  There is no CPU fallback: without a CUDA device tsdp_init fails with TSDP_ERR_CUDA.
+ */
+#ifndef TSDP_H
+#define TSDP_H
+#include <stddef.h>
+#include <stdint.h>
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tsdp_ctx tsdp_ctx; /* opaque; owned by the library */
+
+typedef enum {
+  TSDP_OK = 0,
+  TSDP_ERR_ARG = 1,         /* null pointer, size out of range, unsupported shape          */
+  TSDP_ERR_STATE = 2,       /* weights not loaded yet                                      */
+  TSDP_ERR_WEIGHTS = 3,     /* blob size does not match the configured architecture        */
+  TSDP_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed (see tsdp_last_error)   */
+  TSDP_ERR_TIMEOUT = 5,     /* a bounded wait inside a kernel expired                      */
+  TSDP_ERR_NAN = 6,         /* non-finite value in a weight blob                           */
+  TSDP_ERR_UNSUPPORTED = 7  /* architecture not built                                      */
+} tsdp_status;
+
+enum { TSDP_ARCH_GAUSS = 0, TSDP_ARCH_MLP = 1, TSDP_ARCH_XFMR = 2 };
+enum { TSDP_BASE = 0, TSDP_DRAFT = 1 };
+enum { TSDP_MAX_T = 1024, TSDP_MAX_K = 32 };
+
+/* One denoiser eps = M(x, t; obs).
+ *   GAUSS: closed-form optimal denoiser of iid N(m0, s0^2) data (the 1-D Gaussian toy); no sizes.
+ *   MLP  : input [latent | sinusoidal(t, temb) | obs], `layers` hidden SiLU layers of width `d`.
+ *   XFMR : pre-LN decoder, `layers` blocks [causal self-attn, cross-attn to (time token | obs tokens),
+ *          GELU MLP 4d], model width `d` (multiple of 128), `heads` heads (d/heads multiple of 32).
+ * The paper fixes only the block counts (8 for the base policy, 1 for the drafter; Sec. 4). */
+typedef struct {
+  int arch, layers, d, heads, temb;
+} tsdp_net_t;
+
+typedef struct {
+  tsdp_net_t base, draft;
+  int H, A;                /* action horizon and action dimension; latent size D = H*A        */
+  int obs_tokens, obs_dim; /* observation: obs_tokens x obs_dim features per environment       */
+  int T;                   /* DDPM steps (paper: 100), <= TSDP_MAX_T                          */
+  float beta0, beta1;      /* linear beta schedule                                            */
+  float clip;              /* clamp x0_hat to +-clip when > 0                                  */
+  int max_B, max_K;        /* capacity: environments per call, draft steps per round          */
+  int precision;           /* 0: fp32 check mode (CUDA cores); 1: bf16 tensor-core mode       */
+  int device;              /* CUDA device ordinal                                              */
+  float draft_nfe;         /* NFE cost of one drafter call; 0 => draft.layers/base.layers
+                              (the paper's 1/8 rule, Sec. 4 "Evaluation Metrics")               */
+  int use_graph;           /* 1: replay each round from a captured CUDA graph                  */
+} tsdp_config_t;
+
+/* Speculative parameters of a round -- the scheduler's action space (Sec. 3.3).
+ *   mode 0: accept iff U <= min(1, alpha)  (lossless likelihood-ratio test, Sec. 3.1 Eq. (2));
+ *   mode 1: accept iff min(1, alpha) >= lambda, lambda in (0,1]  (the threshold rule of Sec. 3.2).
+ *   sigma_scale s >= 1 widens only the test statistic, d = (mu^ - mu)/(s sigma).
+ *   bonus 1: when no draft is rejected the base model's evaluation of the last draft is used for one
+ *            more reverse step (K+1 candidates verified); 0: only the K drafted latents count. */
+typedef struct {
+  int mode;
+  float lambda;
+  float sigma_scale;
+  int bonus;
+} tsdp_accept_t;
+
+typedef struct {
+  uint64_t chunks;          /* environment-chunks completed                                   */
+  uint64_t rounds;          /* batched rounds launched                                        */
+  uint64_t env_rounds;      /* rounds summed over environments (= batched base forwards each saw) */
+  uint64_t base_evals;      /* candidate latents the base model evaluated (useful ones)       */
+  uint64_t draft_evals;     /* drafter calls (= drafts proposed)                               */
+  uint64_t drafts_tested, drafts_accepted, rejections, bonus_steps, steps_advanced;
+  double nfe;               /* env_rounds + draft_nfe * draft_evals                           */
+  uint64_t hist_drafted[TSDP_MAX_T], hist_tested[TSDP_MAX_T], hist_accepted[TSDP_MAX_T];
+                            /* per timestep of the drafted transition                          */
+} tsdp_stats_t;
+
+/* Create a context on cfg->device: allocates every workspace for (max_B, max_K).  *out is set only on
+ * success.  Errors: ARG (bad sizes), UNSUPPORTED (arch), CUDA. */
+int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out);
+void tsdp_destroy(tsdp_ctx* ctx);
+const char* tsdp_strerror(int status);
+/* Text of the last CUDA failure seen by this context ("" if none); valid until the next call. */
+const char* tsdp_last_error(const tsdp_ctx* ctx);
+
+/* Number of fp32 values tsdp_load_weights expects for net `which` (0 on a bad argument). */
+size_t tsdp_weights_count(const tsdp_config_t* cfg, int which);
+
+/* Load a denoiser from a HOST blob of n fp32 values, copied during the call (caller keeps ownership).
+ * Linear layers y = x W + b are stored W [in, out] row-major then b [out].  Order:
+ *   GAUSS: m0, s0.
+ *   MLP  : (W, b) for each hidden layer, then the head.  in = H*A + temb + obs_tokens*obs_dim.
+ *   XFMR : W_in [A,d], b_in, pos [H,d], W_obs [obs_dim,d], b_obs, cpos [1+obs_tokens,d];
+ *          per block: ln1_g, ln1_b, Wqkv [d,3d], bqkv, Wo, bo, ln2_g, ln2_b, Wq2, bq2, Wkv2 [d,2d], bkv2,
+ *                     Wo2, bo2, ln3_g, ln3_b, W1 [d,4d], b1, W2 [4d,d], b2;
+ *          lnf_g, lnf_b, W_out [d,A], b_out.
+ * In precision 1 the large matrices are rounded to bf16.  Errors: WEIGHTS (n mismatch), NAN, CUDA. */
+int tsdp_load_weights(tsdp_ctx* ctx, int which, const float* h_blob, size_t n);
+
+/* Per-round overrides for the following chunks: round r uses K_per_round[min(r, n-1)] and
+ * per_round[min(r, n-1)]; n = 0 clears the schedule (every round then uses the arguments of
+ * tsdp_sample_chunk).  Stands in for the RL scheduler's output (Sec. 3.3).  HOST arrays, copied. */
+int tsdp_set_schedule(tsdp_ctx* ctx, const int* h_K_per_round, const tsdp_accept_t* h_per_round, int n);
+
+/* Sample one action chunk for each of B environments (the whole hot path: init, rounds until every
+ * environment reaches t = -1).  d_obs [B, obs_tokens, obs_dim] and d_actions [B, H, A] are DEVICE
+ * buffers owned by the caller; work is enqueued on `cuda_stream` (a cudaStream_t, may be 0) and the
+ * call returns after the chunk has finished (it reads a completion flag between rounds).  The same
+ * (weights, obs, seed, K, accept, schedule) always gives the same chunk.
+ * Errors: ARG, STATE, CUDA, TIMEOUT. */
+int tsdp_sample_chunk(tsdp_ctx* ctx, const float* d_obs, int B, int K, const tsdp_accept_t* accept,
+                      uint64_t seed, float* d_actions, void* cuda_stream);
+
+/* The same with HOST buffers: copies h_obs to the device, samples, copies the chunk back. */
+int tsdp_sample_chunk_host(tsdp_ctx* ctx, const float* h_obs, int B, int K, const tsdp_accept_t* accept,
+                           uint64_t seed, float* h_actions);
+
+/* One speculative round from a given state, with every intermediate exposed (test interface).
+ *   d_x [B, D] in/out: current latents;  h_t [B] in/out: their timesteps (HOST).
+ * Optional outputs (null to skip): d_xtilde [B, K+1, D] candidates (slot 0 = input latent),
+ * d_muhat [B, K, D] drafter means, d_eps [B, K+1, D] base outputs, d_logalpha [B, K],
+ * h_jstar [B] (HOST; first rejected step, K_eff+1 if none, -1 if the environment was finished).
+ * Synchronous. */
+int tsdp_round(tsdp_ctx* ctx, const float* d_obs, int B, int K, const tsdp_accept_t* accept, uint64_t seed,
+               float* d_x, int* h_t, float* d_xtilde, float* d_muhat, float* d_eps, float* d_logalpha,
+               int* h_jstar, void* cuda_stream);
+
+/* eps = M_which(x_n, tau_n; obs_n) for n < N <= max_B (test interface).  d_x, d_eps [N, D];
+ * h_tau [N] HOST; d_obs [N, obs_tokens, obs_dim].  Synchronous. */
+int tsdp_denoise(tsdp_ctx* ctx, int which, const float* d_x, const int* h_tau, const float* d_obs, int N,
+                 float* d_eps, void* cuda_stream);
+
+/* C[M,N] = A[M,K] W[N,K]^T + bias through the context's GEMM (tcgen05 in precision 1, where d_A, d_W
+ * are bf16 and K % 64 == 0, N % 32 == 0; CUDA cores in precision 0, where they are fp32).
+ * epi: 0 store (bf16 / fp32 by precision), 1 GELU then store, 2 d_out fp32 += result, 3 store fp32.
+ * Test interface; synchronous. */
+int tsdp_gemm(tsdp_ctx* ctx, const void* d_A, const void* d_W, const float* d_bias, int M, int N, int K,
+              int epi, void* d_out, void* cuda_stream);
+
+/* Copy the counters accumulated since the last reset (synchronises the device). */
+int tsdp_stats(tsdp_ctx* ctx, tsdp_stats_t* out);
+int tsdp_reset_stats(tsdp_ctx* ctx);
+/* Number of kernels this library launched (or replayed through graphs) since the last reset. */
+uint64_t tsdp_kernel_launches(const tsdp_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TSDP_H */

@@ -1,0 +1,128 @@
+// Shared device helpers of the TS-DP CUDA path: Philox4x32-10 noise streams, the DDPM posterior,
+// warp reductions.  Written for sm_100a; nothing here is shared with the CPU oracle.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace tsdp {
+
+// ----------------------------------------------------------------------------------------------
+// Counter-based noise.  Every random number is a pure function of (seed, env, stream, timestep,
+// element): counter = (quad index, timestep code, env, stream), key = seed.  A draft at timestep
+// tau and a base step at tau therefore see the same xi_tau, which makes "drafter == base"
+// reproduce vanilla DDPM bit for bit (Sec. 3.2: the rollout retains its noise realisations).
+// ----------------------------------------------------------------------------------------------
+enum : uint32_t { STREAM_INIT = 0, STREAM_XI = 1, STREAM_U = 2 };
+
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                               uint32_t k0, uint32_t k1, uint32_t out[4]) {
+  const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
+    const uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
+    const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    k0 += W0; k1 += W1;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// ((n >> 9) + 0.5) * 2^-23: in (0,1), exact in fp32.
+__device__ __forceinline__ float bits_to_unit(uint32_t n) {
+  return (__uint2float_rn(n >> 9) + 0.5f) * 1.1920928955078125e-07f;
+}
+
+// Four standard normals of counter quad `quad`: lanes (0,1) and (2,3) are the cosine / sine branches
+// of one Box-Muller pair each.
+__device__ __forceinline__ void normal4(uint64_t seed, uint32_t env, uint32_t stream, uint32_t tcode,
+                                        uint32_t quad, float z[4]) {
+  uint32_t w[4];
+  philox4x32_10(quad, tcode, env, stream, (uint32_t)seed, (uint32_t)(seed >> 32), w);
+#pragma unroll
+  for (int p = 0; p < 2; ++p) {
+    const float r = sqrtf(-2.0f * logf(bits_to_unit(w[2 * p])));
+    float s, c;
+    sincospif(2.0f * bits_to_unit(w[2 * p + 1]), &s, &c);
+    z[2 * p] = r * c;
+    z[2 * p + 1] = r * s;
+  }
+}
+
+__device__ __forceinline__ float uniform1(uint64_t seed, uint32_t env, uint32_t tau) {
+  uint32_t w[4];
+  philox4x32_10(0u, tau, env, STREAM_U, (uint32_t)seed, (uint32_t)(seed >> 32), w);
+  return bits_to_unit(w[0]);
+}
+
+// ----------------------------------------------------------------------------------------------
+// DDPM scheduler S (the paper's x_{t-1} = S(m_t, t, x_t), Sec. 3.2): per-timestep coefficients of
+// the Gaussian reverse transition, tabulated once per context in fp64 and stored as fp32.
+// ----------------------------------------------------------------------------------------------
+struct DdpmTables {
+  const float* sqrt_ab;     // sqrt(abar_t)
+  const float* sqrt_1mab;   // sqrt(1 - abar_t)
+  const float* c_x0;        // sqrt(abar_{t-1}) beta_t / (1 - abar_t)
+  const float* c_xt;        // sqrt(alpha_t) (1 - abar_{t-1}) / (1 - abar_t)
+  const float* sigma;       // sqrt(beta_t (1 - abar_{t-1}) / (1 - abar_t)), sigma_0 = 0
+  int T;
+  float clip;               // clamp x0_hat to +-clip when > 0
+};
+
+__device__ __forceinline__ float posterior_mean(const DdpmTables& S, float x, float eps, int tau) {
+  float x0 = (x - S.sqrt_1mab[tau] * eps) / S.sqrt_ab[tau];
+  if (S.clip > 0.f) x0 = fminf(fmaxf(x0, -S.clip), S.clip);
+  return S.c_x0[tau] * x0 + S.c_xt[tau] * x;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float gelu_tanh(float v) {
+  const float k = 0.7978845608028654f;   // sqrt(2/pi)
+  return 0.5f * v * (1.0f + tanhf(k * (v + 0.044715f * v * v * v)));
+}
+__device__ __forceinline__ float silu(float v) { return v / (1.0f + __expf(-v)); }
+
+// Which candidate rows a forward pass covers: candidate n = (env b = n / C, slot c = n % C) reads its
+// latent at xin + b*x_stride_b + c*D, is evaluated at timestep clamp(t[b] - koff - c, 0, T-1) and
+// writes eps at eout + b*e_stride_b + c*D.
+struct CandMap {
+  const float* xin;  long long x_stride_b;
+  float* eout;       long long e_stride_b;
+  const int* t;      int C;  int koff;
+};
+
+// Per-round speculative parameters (the scheduler's action space, Sec. 3.3: draft steps, acceptance
+// threshold, sigma scale).
+struct RoundParams {
+  int K;
+  int mode;           // 0: U <= min(1, alpha)   1: min(1, alpha) >= lambda
+  float log_lambda;
+  float sigma_scale;
+  int bonus;
+};
+
+// Device-side counters behind tsdp_stats.
+struct DevStats {
+  unsigned long long env_rounds, base_evals, draft_evals, drafts_tested, drafts_accepted, rejections,
+      bonus_steps, steps_advanced, chunks_done;
+  unsigned long long hist_drafted[1024], hist_tested[1024], hist_accepted[1024];
+};
+
+}  // namespace tsdp

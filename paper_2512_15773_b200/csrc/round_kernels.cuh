@@ -1,0 +1,224 @@
+// Kernels of the speculative round that are not network forwards: chunk initialisation, the
+// drafter's scheduler step (posterior mean + noise), and the fused verification tail -- posterior
+// of every candidate, log acceptance ratio, decision, first-rejection scan, reflection / bonus
+// commit and statistics -- in one launch.
+#pragma once
+#include "common.cuh"
+
+namespace tsdp {
+
+// x_T ~ N(0, I), t = T-1 for every environment.  xt holds the round's candidate latents
+// [B, Kmax+1, D]; slot 0 is the current latent x.
+__global__ void init_chunk_kernel(float* __restrict__ xt, long long xs_b, int* __restrict__ t, int B, int D,
+                                  int T, const uint64_t* __restrict__ seedp, int* __restrict__ round_idx, int* __restrict__ n_done) {
+  const uint64_t seed = *seedp;
+  const int b = blockIdx.x;
+  const int nq = (D + 3) >> 2;
+  for (int q = threadIdx.x; q < nq; q += blockDim.x) {
+    float z[4];
+    normal4(seed, (uint32_t)b, STREAM_INIT, 0u, (uint32_t)q, z);
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if (4 * q + j < D) xt[b * xs_b + 4 * q + j] = z[j];
+  }
+  if (threadIdx.x == 0) {
+    t[b] = T - 1;
+    if (b == 0) { *round_idx = 0; *n_done = 0; }
+  }
+}
+
+// Draft step k (Eq. (3) of Sec. 3.2): tau = t - k + 1, mu^_k = posterior mean of (x~_{k-1}, eps^),
+// x~_k = mu^_k + sigma_tau xi_tau.  Slots beyond K_eff = min(K, t) copy the previous latent so that
+// every buffer stays finite.
+__global__ void draft_step_kernel(DdpmTables S, float* __restrict__ xt, long long xs_b, float* __restrict__ muhat,
+                                  long long ms_b, const float* __restrict__ eps_d, const int* __restrict__ t,
+                                  int k, int D, const uint64_t* __restrict__ seedp) {
+  const uint64_t seed = *seedp;
+  const int b = blockIdx.x;
+  const int tb = t[b];
+  const int tau = tb - k + 1;
+  const bool valid = (tb >= 0) && (tau >= 1);
+  const float* xp = xt + b * xs_b + (long long)(k - 1) * D;
+  float* xn = xt + b * xs_b + (long long)k * D;
+  float* mh = muhat + b * ms_b + (long long)(k - 1) * D;
+  const float* e = eps_d + (long long)b * D;
+  const int nq = (D + 3) >> 2;
+  for (int q = threadIdx.x; q < nq; q += blockDim.x) {
+    float z[4] = {0.f, 0.f, 0.f, 0.f};
+    if (valid) normal4(seed, (uint32_t)b, STREAM_XI, (uint32_t)tau, (uint32_t)q, z);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int i = 4 * q + j;
+      if (i < D) {
+        const float x = xp[i];
+        if (valid) {
+          const float m = posterior_mean(S, x, e[i], tau);
+          mh[i] = m;
+          xn[i] = m + S.sigma[tau] * z[j];
+        } else {
+          mh[i] = x;
+          xn[i] = x;
+        }
+      }
+    }
+  }
+}
+
+// Fused verification tail, one block per environment, one warp per drafted step.
+//   warp k-1 (k = 1..K_eff): mu_k = posterior mean of (x~_{k-1}, eps_{k-1}) at tau = t-k+1;
+//       d = (mu^_k - mu_k) / (s sigma_tau);  log alpha = -1/2 |d|^2 - <d, xi_tau>   (Sec. 3.2)
+//       accept iff log alpha >= log U_tau (mode 0) or min(0, log alpha) >= log lambda (mode 1).
+//   thread 0: j* = first rejected step (Sec. 3.1 Eq. (3)), statistics.
+//   all threads: commit -- reflection x = mu + (I - 2 e e^T)(x~ - mu^) at j* (Sec. 3.1), or the bonus
+//       base step, or the last draft -- into slot 0; t -= steps; finished chunks go to `actions`.
+// dbg_* may be null.
+__global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs_b,
+                              const float* __restrict__ muhat, long long ms_b,
+                              const float* __restrict__ eps, long long es_b, int* __restrict__ t, int K, int D,
+                              const uint64_t* __restrict__ seedp, const RoundParams* __restrict__ sched, int n_sched,
+                              const int* __restrict__ round_idx, float* __restrict__ actions,
+                              int* __restrict__ n_done, DevStats* __restrict__ stats, float draft_nfe,
+                              float* __restrict__ dbg_logalpha, int* __restrict__ dbg_jstar) {
+  __shared__ float s_la[32], s_s1[32], s_s2[32];
+  __shared__ int s_acc[32];
+  __shared__ int s_j;
+  const uint64_t seed = *seedp;
+  const int b = blockIdx.x;
+  const int tb = t[b];
+  if (tb < 0) {
+    if (dbg_jstar && threadIdx.x == 0) dbg_jstar[b] = -1;
+    return;
+  }
+  const int r = min(*round_idx, n_sched - 1);
+  const RoundParams rp = sched[r];
+  const int K_eff = min(K, tb);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nq = (D + 3) >> 2;
+  const float* xb = xt + b * xs_b;
+  const float* mb = muhat + b * ms_b;
+  const float* eb = eps + b * es_b;
+
+  for (int k = warp + 1; k <= K_eff; k += (blockDim.x >> 5)) {
+    const int tau = tb - k + 1;
+    const float inv = 1.0f / (rp.sigma_scale * S.sigma[tau]);
+    float s1 = 0.f, s2 = 0.f, d2 = 0.f;
+    for (int q = lane; q < nq; q += 32) {
+      float z[4];
+      normal4(seed, (uint32_t)b, STREAM_XI, (uint32_t)tau, (uint32_t)q, z);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int i = 4 * q + j;
+        if (i < D) {
+          const float mu = posterior_mean(S, xb[(long long)(k - 1) * D + i], eb[(long long)(k - 1) * D + i], tau);
+          const float delta = mb[(long long)(k - 1) * D + i] - mu;
+          const float d = delta * inv;
+          s1 += d * d; s2 += d * z[j]; d2 += delta * delta;
+        }
+      }
+    }
+    s1 = warp_sum(s1); s2 = warp_sum(s2); d2 = warp_sum(d2);
+    if (lane == 0) {
+      const float la = -0.5f * s1 - s2;
+      bool acc;
+      if (d2 < 1e-30f) acc = true;
+      else if (rp.mode == 0) acc = la >= logf(uniform1(seed, (uint32_t)b, (uint32_t)tau));
+      else acc = fminf(0.f, la) >= rp.log_lambda;
+      s_la[k - 1] = la; s_s1[k - 1] = s1; s_s2[k - 1] = s2; s_acc[k - 1] = acc ? 1 : 0;
+      if (dbg_logalpha) dbg_logalpha[b * K + (k - 1)] = la;
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int j = K_eff + 1;
+    for (int k = 1; k <= K_eff; ++k)
+      if (!s_acc[k - 1]) { j = k; break; }
+    s_j = j;
+    if (dbg_jstar) dbg_jstar[b] = j;
+    if (dbg_logalpha)
+      for (int k = K_eff + 1; k <= K; ++k) dbg_logalpha[b * K + (k - 1)] = 0.f;
+  }
+  __syncthreads();
+  const int j = s_j;
+  const bool rejected = j <= K_eff;
+  const bool bonus = !rejected && (rp.bonus || K_eff == 0);
+  const int adv = rejected ? j : (bonus ? K_eff + 1 : K_eff);
+  const int t_new = tb - adv;
+  float* xo = xt + b * xs_b;   // slot 0
+  if (rejected) {
+    const int tau = tb - j + 1;
+    const float sig = S.sigma[tau];
+    // e <e, xi> = Delta <Delta, xi> / |Delta|^2 = Delta * S2 / (S1 * s * sigma)
+    const float coef = 2.0f * s_s2[j - 1] / (s_s1[j - 1] * rp.sigma_scale * sig);
+    for (int q = threadIdx.x; q < nq; q += blockDim.x) {
+      float z[4];
+      normal4(seed, (uint32_t)b, STREAM_XI, (uint32_t)tau, (uint32_t)q, z);
+#pragma unroll
+      for (int jj = 0; jj < 4; ++jj) {
+        const int i = 4 * q + jj;
+        if (i < D) {
+          const float mu = posterior_mean(S, xb[(long long)(j - 1) * D + i], eb[(long long)(j - 1) * D + i], tau);
+          const float delta = mb[(long long)(j - 1) * D + i] - mu;
+          const float v = mu + sig * (z[jj] - coef * delta);
+          xo[i] = v;
+          if (t_new < 0) actions[(long long)b * D + i] = v;
+        }
+      }
+    }
+  } else if (bonus) {
+    const int tau = tb - K_eff;
+    const float sig = S.sigma[tau];
+    for (int q = threadIdx.x; q < nq; q += blockDim.x) {
+      float z[4] = {0.f, 0.f, 0.f, 0.f};
+      if (tau > 0) normal4(seed, (uint32_t)b, STREAM_XI, (uint32_t)tau, (uint32_t)q, z);
+#pragma unroll
+      for (int jj = 0; jj < 4; ++jj) {
+        const int i = 4 * q + jj;
+        if (i < D) {
+          const float mu = posterior_mean(S, xb[(long long)K_eff * D + i], eb[(long long)K_eff * D + i], tau);
+          const float v = mu + sig * z[jj];
+          xo[i] = v;
+          if (t_new < 0) actions[(long long)b * D + i] = v;
+        }
+      }
+    }
+  } else {
+    for (int i = threadIdx.x; i < D; i += blockDim.x) {
+      const float v = xb[(long long)K_eff * D + i];
+      xo[i] = v;
+      if (t_new < 0) actions[(long long)b * D + i] = v;
+    }
+  }
+  if (threadIdx.x == 0) {
+    t[b] = t_new;
+    const int n_acc = min(j - 1, K_eff);
+    const int n_tested = min(j, K_eff);
+    atomicAdd(&stats->env_rounds, 1ull);
+    atomicAdd(&stats->base_evals, (unsigned long long)((rp.bonus || K_eff == 0) ? K_eff + 1 : K_eff));
+    atomicAdd(&stats->draft_evals, (unsigned long long)K_eff);
+    atomicAdd(&stats->drafts_tested, (unsigned long long)n_tested);
+    atomicAdd(&stats->drafts_accepted, (unsigned long long)n_acc);
+    atomicAdd(&stats->rejections, rejected ? 1ull : 0ull);
+    atomicAdd(&stats->bonus_steps, bonus ? 1ull : 0ull);
+    atomicAdd(&stats->steps_advanced, (unsigned long long)adv);
+    for (int k = 1; k <= K_eff; ++k) {
+      const int tau = tb - k + 1;
+      atomicAdd(&stats->hist_drafted[tau], 1ull);
+      if (k <= n_tested) atomicAdd(&stats->hist_tested[tau], 1ull);
+      if (k <= n_acc) atomicAdd(&stats->hist_accepted[tau], 1ull);
+    }
+    if (t_new < 0) {
+      atomicAdd(&stats->chunks_done, 1ull);
+      atomicAdd(n_done, 1);
+    }
+  }
+}
+
+// End of a round: advance the schedule index and publish the number of finished chunks where the
+// host can read it.
+__global__ void round_end_kernel(int* __restrict__ round_idx, const int* __restrict__ n_done,
+                                 volatile int* __restrict__ host_done) {
+  *round_idx += 1;
+  *host_done = *n_done;
+}
+
+}  // namespace tsdp

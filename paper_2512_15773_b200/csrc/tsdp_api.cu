@@ -1,0 +1,964 @@
+// libtsdp: host side of the TS-DP speculative denoising loop -- context, weight loading, the round
+// orchestration (plain launches or a captured CUDA graph per (B, K)) and the C ABI of include/tsdp.h.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <string>
+#include <tuple>
+#include <vector>
+
+#include "../../include/tsdp.h"
+#include "common.cuh"
+#include "gemm_tcgen05.cuh"
+#include "net_kernels.cuh"
+#include "round_kernels.cuh"
+
+using namespace tsdp;
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct XfmrLayer {
+  float *ln1_g, *ln1_b, *bqkv, *bo, *ln2_g, *ln2_b, *bq2, *bo2, *ln3_g, *ln3_b, *b1, *b2;
+  void *Wqkv, *Wo, *Wq2, *Wo2, *W1, *W2;      // [out, in], bf16 or fp32 by precision
+};
+
+struct Net {
+  tsdp_net_t cfg{};
+  bool loaded = false;
+  float m0 = 0.f, s0 = 1.f;                   // GAUSS
+  MlpWeights mlp{};                           // MLP
+  float *W_in = nullptr, *b_in = nullptr, *pos = nullptr, *W_obs = nullptr, *b_obs = nullptr, *cpos = nullptr;
+  float *lnf_g = nullptr, *lnf_b = nullptr, *W_outT = nullptr, *b_out = nullptr;
+  std::vector<XfmrLayer> L;
+  void* Wkv_all = nullptr;                    // [L*2d, d]: the cross-attention K/V projections of all blocks
+  float* bkv_all = nullptr;
+  float* kv_time = nullptr;                   // [T, L*2d]   K/V of the time token for every timestep
+  float* kv_obs = nullptr;                    // [max_B*To, L*2d]  K/V of the obs tokens, per chunk
+  float* temb_table = nullptr;                // [T, temb or d] sinusoidal embedding
+  std::vector<void*> allocs;
+};
+
+}  // namespace
+
+struct tsdp_ctx {
+  tsdp_config_t cfg{};
+  int D = 0, num_sms = 148;
+  Net net[2];
+  DdpmTables S{};
+  std::vector<void*> allocs;
+  // round state
+  float *xt = nullptr, *muhat = nullptr, *eps = nullptr, *eps_d = nullptr, *actions = nullptr, *obs = nullptr;
+  int* t = nullptr;
+  uint64_t* seed = nullptr;
+  int *round_idx = nullptr, *n_done = nullptr, *status = nullptr;
+  int* host_done = nullptr;                   // mapped pinned
+  RoundParams* sched = nullptr;               // device, capacity TSDP_MAX_T + 1
+  RoundParams* sched_host = nullptr;          // pinned staging
+  DevStats* stats = nullptr;
+  float* dbg_logalpha = nullptr;
+  int* dbg_jstar = nullptr;
+  // transformer workspaces (bytes sized for the larger of the two nets)
+  float* h = nullptr;
+  void *a = nullptr, *qkv = nullptr, *q2 = nullptr, *f = nullptr, *memtok = nullptr;
+  // schedule set by the caller
+  std::vector<int> sched_K;
+  std::vector<tsdp_accept_t> sched_acc;
+  // graphs and tensor maps
+  std::map<std::tuple<int, int>, cudaGraphExec_t> graphs;
+  std::map<std::tuple<const void*, int, int, int>, CUtensorMap> maps;
+  EncodeTiledFn encode = nullptr;
+  cudaStream_t cap_stream = nullptr;
+  uint64_t rounds = 0, launches = 0;
+  int launches_per_round_tmp = 0;
+  std::string last_error;
+};
+
+namespace {
+
+#define CU_TRY(ctx, expr)                                                                         \
+  do {                                                                                            \
+    cudaError_t e__ = (expr);                                                                     \
+    if (e__ != cudaSuccess) {                                                                     \
+      (ctx)->last_error = std::string(#expr) + ": " + cudaGetErrorString(e__);                    \
+      return TSDP_ERR_CUDA;                                                                       \
+    }                                                                                             \
+  } while (0)
+
+template <typename T>
+int dev_alloc(tsdp_ctx* c, std::vector<void*>& pool, T** p, size_t n) {
+  void* q = nullptr;
+  CU_TRY(c, cudaMalloc(&q, n * sizeof(T) + 256));
+  CU_TRY(c, cudaMemset(q, 0, n * sizeof(T) + 256));
+  pool.push_back(q);
+  *p = reinterpret_cast<T*>(q);
+  return TSDP_OK;
+}
+
+int alloc_bytes(tsdp_ctx* c, std::vector<void*>& pool, void** p, size_t bytes) {
+  return dev_alloc<uint8_t>(c, pool, reinterpret_cast<uint8_t**>(p), bytes);
+}
+
+bool net_cfg_ok(const tsdp_config_t& cfg, const tsdp_net_t& n) {
+  if (n.arch == TSDP_ARCH_GAUSS) return true;
+  if (n.arch == TSDP_ARCH_MLP)
+    return n.layers >= 1 && n.layers <= MLP_MAX_LAYERS && n.d >= 1 && n.d <= 4096 && n.temb >= 2 && n.temb % 2 == 0;
+  if (n.arch == TSDP_ARCH_XFMR)
+    return n.layers >= 1 && n.d % 128 == 0 && n.d >= 128 && n.d <= 1024 && n.heads >= 1 && n.d % n.heads == 0 &&
+           (n.d / n.heads) % 32 == 0 && (n.d / n.heads) <= 128 && cfg.H <= 64 && cfg.obs_tokens <= 8 && cfg.A <= 64;
+  return false;
+}
+
+size_t weights_count(const tsdp_config_t& cfg, const tsdp_net_t& n) {
+  const size_t D = (size_t)cfg.H * cfg.A, d = n.d;
+  if (n.arch == TSDP_ARCH_GAUSS) return 2;
+  if (n.arch == TSDP_ARCH_MLP) {
+    size_t in = D + n.temb + (size_t)cfg.obs_tokens * cfg.obs_dim, tot = 0;
+    for (int l = 0; l < n.layers; ++l) { tot += in * d + d; in = d; }
+    return tot + in * D + D;
+  }
+  if (n.arch == TSDP_ARCH_XFMR) {
+    size_t tot = (size_t)cfg.A * d + d + (size_t)cfg.H * d + (size_t)cfg.obs_dim * d + d + (size_t)(1 + cfg.obs_tokens) * d;
+    const size_t per = 2 * d + d * 3 * d + 3 * d + d * d + d + 2 * d + d * d + d + d * 2 * d + 2 * d + d * d + d + 2 * d +
+                       d * 4 * d + 4 * d + 4 * d * d + d;
+    return tot + per * n.layers + 2 * d + d * cfg.A + cfg.A;
+  }
+  return 0;
+}
+
+// ------------------------------------------------------------------------------------------ GEMM
+int get_map(tsdp_ctx* c, const void* ptr, int rows, int cols, int box_rows, CUtensorMap* out) {
+  auto key = std::make_tuple(ptr, rows, cols, box_rows);
+  auto it = c->maps.find(key);
+  if (it != c->maps.end()) { *out = it->second; return TSDP_OK; }
+  CUtensorMap m;
+  cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t gstr[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)GEMM_BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = c->encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstr, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    c->last_error = "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r);
+    return TSDP_ERR_CUDA;
+  }
+  c->maps[key] = m;
+  *out = m;
+  return TSDP_OK;
+}
+
+template <int BN, int EPI>
+int launch_tc(tsdp_ctx* c, const CUtensorMap& ma, const CUtensorMap& mb, const GemmArgs& g, cudaStream_t s) {
+  const int tiles = ((g.M + GEMM_BM - 1) / GEMM_BM) * (g.N / BN);
+  const int grid = tiles < c->num_sms ? tiles : c->num_sms;
+  gemm_tcgen05_kernel<BN, EPI><<<grid, GEMM_THREADS, gemm_smem_bytes(BN), s>>>(ma, mb, g);
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  return TSDP_OK;
+}
+
+template <int BN>
+int launch_tc_epi(tsdp_ctx* c, const CUtensorMap& ma, const CUtensorMap& mb, const GemmArgs& g, int epi, cudaStream_t s) {
+  switch (epi) {
+    case EPI_STORE: return launch_tc<BN, EPI_STORE>(c, ma, mb, g, s);
+    case EPI_GELU: return launch_tc<BN, EPI_GELU>(c, ma, mb, g, s);
+    case EPI_RESID: return launch_tc<BN, EPI_RESID>(c, ma, mb, g, s);
+    default: return launch_tc<BN, EPI_F32>(c, ma, mb, g, s);
+  }
+}
+
+template <int BN, int EPI>
+cudaError_t set_smem_attr() {
+  return cudaFuncSetAttribute(gemm_tcgen05_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              gemm_smem_bytes(BN));
+}
+template <int BN>
+cudaError_t set_smem_attr_all() {
+  cudaError_t e;
+  if ((e = set_smem_attr<BN, EPI_STORE>()) != cudaSuccess) return e;
+  if ((e = set_smem_attr<BN, EPI_GELU>()) != cudaSuccess) return e;
+  if ((e = set_smem_attr<BN, EPI_RESID>()) != cudaSuccess) return e;
+  return set_smem_attr<BN, EPI_F32>();
+}
+
+// Tile width: the widest BN that divides N and still yields at least one tile per SM; otherwise the
+// narrowest that divides N (small-batch calls are latency-bound and want many CTAs).
+int pick_bn(int M, int N, int num_sms) {
+  const int tm = (M + GEMM_BM - 1) / GEMM_BM;
+  const int cands[4] = {256, 128, 64, 32};
+  for (int i = 0; i < 4; ++i)
+    if (N % cands[i] == 0 && tm * (N / cands[i]) >= num_sms) return cands[i];
+  for (int i = 3; i >= 0; --i)
+    if (N % cands[i] == 0) return cands[i];
+  return 0;
+}
+
+int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, int N, int K, int epi, void* out,
+         int ldo, cudaStream_t s) {
+  if (M <= 0) return TSDP_OK;
+  GemmArgs g{M, N, K, bias, out, ldo, c->status};
+  if (c->cfg.precision == 0) {
+    dim3 grid((N + 63) / 64, (M + 63) / 64);
+    const float* a = reinterpret_cast<const float*>(A);
+    const float* w = reinterpret_cast<const float*>(W);
+    switch (epi) {
+      case EPI_GELU: gemm_simt_kernel<EPI_GELU><<<grid, 256, 0, s>>>(a, w, g); break;
+      case EPI_RESID: gemm_simt_kernel<EPI_RESID><<<grid, 256, 0, s>>>(a, w, g); break;
+      default: gemm_simt_kernel<EPI_F32><<<grid, 256, 0, s>>>(a, w, g); break;
+    }
+    c->launches_per_round_tmp++;
+    CU_TRY(c, cudaGetLastError());
+    return TSDP_OK;
+  }
+  if (K % GEMM_BK != 0 || N % 32 != 0) {
+    c->last_error = "tensor-core GEMM needs K % 64 == 0 and N % 32 == 0";
+    return TSDP_ERR_ARG;
+  }
+  const int BN = pick_bn(M, N, c->num_sms);
+  CUtensorMap ma, mb;
+  int r;
+  if ((r = get_map(c, A, M, K, GEMM_BM, &ma)) != TSDP_OK) return r;
+  if ((r = get_map(c, W, N, K, BN, &mb)) != TSDP_OK) return r;
+  switch (BN) {
+    case 256: return launch_tc_epi<256>(c, ma, mb, g, epi, s);
+    case 128: return launch_tc_epi<128>(c, ma, mb, g, epi, s);
+    case 64: return launch_tc_epi<64>(c, ma, mb, g, epi, s);
+    default: return launch_tc_epi<32>(c, ma, mb, g, epi, s);
+  }
+}
+
+// ------------------------------------------------------------------------------------------ nets
+template <typename T>
+int ln_launch(tsdp_ctx* c, const float* h, const float* g, const float* b, T* out, int M, int d, cudaStream_t s) {
+  const int wpb = 8;
+  const int grid = (M + wpb - 1) / wpb;
+  switch (d / 128) {
+    case 1: ln_kernel<T, 1><<<grid, wpb * 32, 0, s>>>(h, g, b, out, M); break;
+    case 2: ln_kernel<T, 2><<<grid, wpb * 32, 0, s>>>(h, g, b, out, M); break;
+    case 3: ln_kernel<T, 3><<<grid, wpb * 32, 0, s>>>(h, g, b, out, M); break;
+    case 4: ln_kernel<T, 4><<<grid, wpb * 32, 0, s>>>(h, g, b, out, M); break;
+    case 5: ln_kernel<T, 5><<<grid, wpb * 32, 0, s>>>(h, g, b, out, M); break;
+    case 6: ln_kernel<T, 6><<<grid, wpb * 32, 0, s>>>(h, g, b, out, M); break;
+    case 7: ln_kernel<T, 7><<<grid, wpb * 32, 0, s>>>(h, g, b, out, M); break;
+    default: ln_kernel<T, 8><<<grid, wpb * 32, 0, s>>>(h, g, b, out, M); break;
+  }
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  return TSDP_OK;
+}
+
+int head_launch(tsdp_ctx* c, const Net& n, const CandMap& cm, int M, cudaStream_t s) {
+  const int wpb = 8;
+  const int grid = (M + wpb - 1) / wpb;
+  const int H = c->cfg.H, A = c->cfg.A;
+#define HEAD_CASE(V) head_kernel<V><<<grid, wpb * 32, 0, s>>>(c->h, n.lnf_g, n.lnf_b, n.W_outT, n.b_out, cm, M, H, A)
+  switch (n.cfg.d / 128) {
+    case 1: HEAD_CASE(1); break;
+    case 2: HEAD_CASE(2); break;
+    case 3: HEAD_CASE(3); break;
+    case 4: HEAD_CASE(4); break;
+    case 5: HEAD_CASE(5); break;
+    case 6: HEAD_CASE(6); break;
+    case 7: HEAD_CASE(7); break;
+    default: HEAD_CASE(8); break;
+  }
+#undef HEAD_CASE
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  return TSDP_OK;
+}
+
+template <typename T>
+int xfmr_forward_t(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStream_t s) {
+  const int H = c->cfg.H, A = c->cfg.A, d = n.cfg.d, heads = n.cfg.heads, L = n.cfg.layers;
+  const int M = n_cand * H;
+  const int dh = d / heads;
+  T* a = reinterpret_cast<T*>(c->a);
+  T* qkv = reinterpret_cast<T*>(c->qkv);
+  T* q2 = reinterpret_cast<T*>(c->q2);
+  T* f = reinterpret_cast<T*>(c->f);
+  int r;
+  embed_kernel<<<M, d < 256 ? d : 256, 0, s>>>(cm, n.W_in, n.b_in, n.pos, c->h, H, A, d);
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  const int sa_wpb = 4;
+  const size_t sa_smem = (size_t)sa_wpb * (H * dh + 2 * H * (dh + 1)) * sizeof(float);
+  const int out_epi = (c->cfg.precision == 0) ? EPI_F32 : EPI_STORE;
+  for (int l = 0; l < L; ++l) {
+    const XfmrLayer& w = n.L[l];
+    if ((r = ln_launch<T>(c, c->h, w.ln1_g, w.ln1_b, a, M, d, s))) return r;
+    if ((r = gemm(c, a, w.Wqkv, w.bqkv, M, 3 * d, d, out_epi, qkv, 3 * d, s))) return r;
+    self_attn_kernel<T><<<(n_cand * heads + sa_wpb - 1) / sa_wpb, sa_wpb * 32, sa_smem, s>>>(qkv, a, n_cand, H, d, heads);
+    c->launches_per_round_tmp++;
+    CU_TRY(c, cudaGetLastError());
+    if ((r = gemm(c, a, w.Wo, w.bo, M, d, d, EPI_RESID, c->h, d, s))) return r;
+    if ((r = ln_launch<T>(c, c->h, w.ln2_g, w.ln2_b, a, M, d, s))) return r;
+    if ((r = gemm(c, a, w.Wq2, w.bq2, M, d, d, out_epi, q2, d, s))) return r;
+    cross_attn_kernel<T><<<(M + 7) / 8, 256, 0, s>>>(q2, a, n.kv_time, n.kv_obs, cm, M, H, d, heads, c->cfg.obs_tokens, l, L,
+                                                      c->cfg.T);
+    c->launches_per_round_tmp++;
+    CU_TRY(c, cudaGetLastError());
+    if ((r = gemm(c, a, w.Wo2, w.bo2, M, d, d, EPI_RESID, c->h, d, s))) return r;
+    if ((r = ln_launch<T>(c, c->h, w.ln3_g, w.ln3_b, a, M, d, s))) return r;
+    if ((r = gemm(c, a, w.W1, w.b1, M, 4 * d, d, EPI_GELU, f, 4 * d, s))) return r;
+    if ((r = gemm(c, f, w.W2, w.b2, M, d, 4 * d, EPI_RESID, c->h, d, s))) return r;
+  }
+  return head_launch(c, n, cm, M, s);
+}
+
+// Observation tokens -> their cross-attention keys/values for every block (once per chunk).
+template <typename T>
+int xfmr_prepare_obs_t(tsdp_ctx* c, Net& n, int B, cudaStream_t s) {
+  const int To = c->cfg.obs_tokens, d = n.cfg.d, L = n.cfg.layers;
+  if (To == 0) return TSDP_OK;
+  T* mt = reinterpret_cast<T*>(c->memtok);
+  memtok_kernel<T><<<B * To, d < 256 ? d : 256, 0, s>>>(c->obs, c->cfg.obs_dim, n.W_obs, n.b_obs, n.cpos, To, 1, mt, d);
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  return gemm(c, mt, n.Wkv_all, n.bkv_all, B * To, L * 2 * d, d, EPI_F32, n.kv_obs, L * 2 * d, s);
+}
+
+int prepare_obs(tsdp_ctx* c, Net& n, int B, cudaStream_t s) {
+  if (n.cfg.arch != TSDP_ARCH_XFMR) return TSDP_OK;
+  return c->cfg.precision == 0 ? xfmr_prepare_obs_t<float>(c, n, B, s) : xfmr_prepare_obs_t<__nv_bfloat16>(c, n, B, s);
+}
+
+int forward(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStream_t s) {
+  if (n_cand <= 0) return TSDP_OK;
+  const int D = c->D;
+  switch (n.cfg.arch) {
+    case TSDP_ARCH_GAUSS: {
+      const long long tot = (long long)n_cand * D;
+      gauss_forward_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, s>>>(c->S, n.m0, n.s0, cm, n_cand, D);
+      c->launches_per_round_tmp++;
+      CU_TRY(c, cudaGetLastError());
+      return TSDP_OK;
+    }
+    case TSDP_ARCH_MLP: {
+      int maxw = 0;
+      for (int l = 0; l <= n.mlp.n_lin; ++l) maxw = n.mlp.dims[l] > maxw ? n.mlp.dims[l] : maxw;
+      mlp_forward_kernel<<<n_cand, 256, 2 * maxw * sizeof(float), s>>>(n.mlp, cm, c->obs, c->cfg.obs_tokens * c->cfg.obs_dim,
+                                                                        D, c->cfg.T);
+      c->launches_per_round_tmp++;
+      CU_TRY(c, cudaGetLastError());
+      return TSDP_OK;
+    }
+    case TSDP_ARCH_XFMR:
+      return c->cfg.precision == 0 ? xfmr_forward_t<float>(c, n, cm, n_cand, s)
+                                   : xfmr_forward_t<__nv_bfloat16>(c, n, cm, n_cand, s);
+  }
+  return TSDP_ERR_UNSUPPORTED;
+}
+
+// ------------------------------------------------------------------------------------------ round
+// Enqueue one speculative round for B environments with K draft steps.
+int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
+  const int D = c->D;
+  const long long xs_b = (long long)(c->cfg.max_K + 1) * D, ms_b = (long long)(c->cfg.max_K > 0 ? c->cfg.max_K : 1) * D;
+  int r;
+  for (int k = 1; k <= K; ++k) {
+    CandMap cm{c->xt + (long long)(k - 1) * D, xs_b, c->eps_d, (long long)D, c->t, 1, k - 1};
+    if ((r = forward(c, c->net[TSDP_DRAFT], cm, B, s))) return r;
+    draft_step_kernel<<<B, 128, 0, s>>>(c->S, c->xt, xs_b, c->muhat, ms_b, c->eps_d, c->t, k, D, c->seed);
+    c->launches_per_round_tmp++;
+    CU_TRY(c, cudaGetLastError());
+  }
+  CandMap cv{c->xt, xs_b, c->eps, xs_b, c->t, K + 1, 0};
+  if ((r = forward(c, c->net[TSDP_BASE], cv, B * (K + 1), s))) return r;
+  int warps = K < 1 ? 1 : K;
+  if (warps < 4) warps = 4;
+  if (warps > 16) warps = 16;
+  accept_kernel<<<B, warps * 32, 0, s>>>(c->S, c->xt, xs_b, c->muhat, ms_b, c->eps, xs_b, c->t, K, D, c->seed, c->sched,
+                                         TSDP_MAX_T + 1, c->round_idx, c->actions, c->n_done, c->stats, c->cfg.draft_nfe,
+                                         dbg ? c->dbg_logalpha : nullptr, dbg ? c->dbg_jstar : nullptr);
+  round_end_kernel<<<1, 1, 0, s>>>(c->round_idx, c->n_done, c->host_done);
+  c->launches_per_round_tmp += 2;
+  CU_TRY(c, cudaGetLastError());
+  return TSDP_OK;
+}
+
+struct GraphRec { cudaGraphExec_t exec; int launches; };
+
+int run_round(tsdp_ctx* c, int B, int K, cudaStream_t s) {
+  if (!c->cfg.use_graph) {
+    c->launches_per_round_tmp = 0;
+    int r = enqueue_round(c, B, K, s, false);
+    c->launches += c->launches_per_round_tmp;
+    return r;
+  }
+  static std::map<cudaGraphExec_t, int> launch_counts;
+  auto key = std::make_tuple(B, K);
+  auto it = c->graphs.find(key);
+  if (it == c->graphs.end()) {
+    // tensor maps must exist before capture; a dry enqueue outside capture would run the round, so
+    // instead capture directly: map creation is host-only work and is legal during capture.
+    cudaGraph_t graph = nullptr;
+    CU_TRY(c, cudaStreamBeginCapture(c->cap_stream, cudaStreamCaptureModeThreadLocal));
+    c->launches_per_round_tmp = 0;
+    int r = enqueue_round(c, B, K, c->cap_stream, false);
+    cudaError_t e = cudaStreamEndCapture(c->cap_stream, &graph);
+    if (r != TSDP_OK) { if (graph) cudaGraphDestroy(graph); return r; }
+    CU_TRY(c, e);
+    cudaGraphExec_t exec = nullptr;
+    CU_TRY(c, cudaGraphInstantiate(&exec, graph, 0));
+    cudaGraphDestroy(graph);
+    launch_counts[exec] = c->launches_per_round_tmp;
+    it = c->graphs.emplace(key, exec).first;
+  }
+  CU_TRY(c, cudaGraphLaunch(it->second, s));
+  c->launches += launch_counts[it->second];
+  return TSDP_OK;
+}
+
+int check_status(tsdp_ctx* c) {
+  int st = 0;
+  CU_TRY(c, cudaMemcpy(&st, c->status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (st != 0) {
+    cudaMemset(c->status, 0, sizeof(int));
+    return st;
+  }
+  return TSDP_OK;
+}
+
+void fill_round_params(RoundParams* rp, int K, const tsdp_accept_t& a) {
+  rp->K = K;
+  rp->mode = a.mode;
+  rp->log_lambda = logf(a.lambda > 0.f ? a.lambda : 1e-30f);
+  rp->sigma_scale = a.sigma_scale > 0.f ? a.sigma_scale : 1.0f;
+  rp->bonus = a.bonus;
+}
+
+bool accept_ok(const tsdp_accept_t* a) {
+  return a && (a->mode == 0 || a->mode == 1) && a->sigma_scale > 0.f && (a->mode == 0 || (a->lambda > 0.f && a->lambda <= 1.f));
+}
+
+// Upload the per-round parameter table: entry r for round r, the last entry repeating.
+int upload_schedule(tsdp_ctx* c, int K, const tsdp_accept_t& acc, cudaStream_t s, bool ignore_user_schedule) {
+  const int n = ignore_user_schedule ? 0 : (int)c->sched_K.size();
+  for (int r = 0; r <= TSDP_MAX_T; ++r) {
+    if (n > 0) {
+      const int i = r < n ? r : n - 1;
+      fill_round_params(&c->sched_host[r], c->sched_K[i], c->sched_acc[i]);
+    } else {
+      fill_round_params(&c->sched_host[r], K, acc);
+    }
+  }
+  CU_TRY(c, cudaMemcpyAsync(c->sched, c->sched_host, sizeof(RoundParams) * (TSDP_MAX_T + 1), cudaMemcpyHostToDevice, s));
+  return TSDP_OK;
+}
+
+}  // namespace
+
+// ================================================================================================ C ABI
+extern "C" {
+
+const char* tsdp_strerror(int st) {
+  switch (st) {
+    case TSDP_OK: return "ok";
+    case TSDP_ERR_ARG: return "bad argument";
+    case TSDP_ERR_STATE: return "weights not loaded";
+    case TSDP_ERR_WEIGHTS: return "weight blob does not match the configured architecture";
+    case TSDP_ERR_CUDA: return "CUDA call failed";
+    case TSDP_ERR_TIMEOUT: return "a bounded wait inside a kernel expired";
+    case TSDP_ERR_NAN: return "non-finite value in weights";
+    case TSDP_ERR_UNSUPPORTED: return "architecture not built";
+  }
+  return "unknown status";
+}
+
+const char* tsdp_last_error(const tsdp_ctx* ctx) { return ctx ? ctx->last_error.c_str() : ""; }
+
+size_t tsdp_weights_count(const tsdp_config_t* cfg, int which) {
+  if (!cfg || (which != TSDP_BASE && which != TSDP_DRAFT)) return 0;
+  const tsdp_net_t& n = which == TSDP_BASE ? cfg->base : cfg->draft;
+  if (!net_cfg_ok(*cfg, n)) return 0;
+  return weights_count(*cfg, n);
+}
+
+int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
+  if (!cfg || !out) return TSDP_ERR_ARG;
+  if (cfg->H < 1 || cfg->A < 1 || cfg->T < 1 || cfg->T > TSDP_MAX_T || cfg->max_B < 1 || cfg->max_K < 0 ||
+      cfg->max_K > TSDP_MAX_K || cfg->obs_tokens < 0 || cfg->obs_dim < 0 || !(cfg->beta0 > 0.f) || !(cfg->beta1 < 1.f) ||
+      (cfg->precision != 0 && cfg->precision != 1))
+    return TSDP_ERR_ARG;
+  for (const tsdp_net_t* n : {&cfg->base, &cfg->draft}) {
+    if (n->arch < TSDP_ARCH_GAUSS || n->arch > TSDP_ARCH_XFMR) return TSDP_ERR_UNSUPPORTED;
+    if (!net_cfg_ok(*cfg, *n)) return TSDP_ERR_ARG;
+  }
+  tsdp_ctx* c = new tsdp_ctx();
+  c->cfg = *cfg;
+  c->D = cfg->H * cfg->A;
+  auto fail = [&](int st) { tsdp_destroy(c); return st; };
+#define INIT_TRY(expr)                                                                    \
+  do {                                                                                    \
+    cudaError_t e__ = (expr);                                                             \
+    if (e__ != cudaSuccess) { fprintf(stderr, "tsdp_init: %s: %s\n", #expr, cudaGetErrorString(e__)); return fail(TSDP_ERR_CUDA); } \
+  } while (0)
+  INIT_TRY(cudaSetDevice(cfg->device));
+  cudaDeviceProp prop;
+  INIT_TRY(cudaGetDeviceProperties(&prop, cfg->device));
+  c->num_sms = prop.multiProcessorCount;
+  if (cfg->precision == 1 && prop.major != 10) {
+    fprintf(stderr, "tsdp_init: precision 1 needs an sm_100a device (found sm_%d%d)\n", prop.major, prop.minor);
+    return fail(TSDP_ERR_CUDA);
+  }
+  if (c->cfg.draft_nfe <= 0.f) {
+    const int lb = cfg->base.layers, ld = cfg->draft.layers;
+    c->cfg.draft_nfe = (lb > 0 && ld > 0) ? (float)ld / (float)lb : 0.125f;
+  }
+  // DDPM tables (fp64 on the host, stored fp32)
+  const int T = cfg->T;
+  std::vector<float> tab(5 * T);
+  {
+    double abar = 1.0, abar_prev = 1.0;
+    for (int t = 0; t < T; ++t) {
+      const double beta = T > 1 ? cfg->beta0 + ((double)cfg->beta1 - cfg->beta0) * t / (T - 1) : cfg->beta0;
+      const double alpha = 1.0 - beta;
+      abar_prev = abar;
+      abar *= alpha;
+      tab[0 * T + t] = (float)std::sqrt(abar);
+      tab[1 * T + t] = (float)std::sqrt(1.0 - abar);
+      tab[2 * T + t] = (float)(std::sqrt(abar_prev) * beta / (1.0 - abar));
+      tab[3 * T + t] = (float)(std::sqrt(alpha) * (1.0 - abar_prev) / (1.0 - abar));
+      tab[4 * T + t] = (float)std::sqrt(beta * (1.0 - abar_prev) / (1.0 - abar));
+    }
+  }
+  float* dtab = nullptr;
+  if (dev_alloc(c, c->allocs, &dtab, 5 * T)) return fail(TSDP_ERR_CUDA);
+  INIT_TRY(cudaMemcpy(dtab, tab.data(), sizeof(float) * 5 * T, cudaMemcpyHostToDevice));
+  c->S = DdpmTables{dtab, dtab + T, dtab + 2 * T, dtab + 3 * T, dtab + 4 * T, T, cfg->clip};
+
+  const size_t B = cfg->max_B, K1 = cfg->max_K + 1, Km = cfg->max_K > 0 ? cfg->max_K : 1, D = c->D;
+  int st = 0;
+  st |= dev_alloc(c, c->allocs, &c->xt, B * K1 * D);
+  st |= dev_alloc(c, c->allocs, &c->muhat, B * Km * D);
+  st |= dev_alloc(c, c->allocs, &c->eps, B * K1 * D);
+  st |= dev_alloc(c, c->allocs, &c->eps_d, B * D);
+  st |= dev_alloc(c, c->allocs, &c->actions, B * D);
+  st |= dev_alloc(c, c->allocs, &c->obs, B * (size_t)cfg->obs_tokens * cfg->obs_dim + 1);
+  st |= dev_alloc(c, c->allocs, &c->t, B);
+  st |= dev_alloc(c, c->allocs, &c->seed, 1);
+  st |= dev_alloc(c, c->allocs, &c->round_idx, 1);
+  st |= dev_alloc(c, c->allocs, &c->n_done, 1);
+  st |= dev_alloc(c, c->allocs, &c->status, 1);
+  st |= dev_alloc(c, c->allocs, &c->sched, TSDP_MAX_T + 1);
+  st |= dev_alloc(c, c->allocs, &c->stats, 1);
+  st |= dev_alloc(c, c->allocs, &c->dbg_logalpha, B * Km);
+  st |= dev_alloc(c, c->allocs, &c->dbg_jstar, B);
+  if (st) return fail(TSDP_ERR_CUDA);
+  INIT_TRY(cudaHostAlloc(reinterpret_cast<void**>(&c->host_done), sizeof(int), cudaHostAllocMapped));
+  *c->host_done = 0;
+  INIT_TRY(cudaHostAlloc(reinterpret_cast<void**>(&c->sched_host), sizeof(RoundParams) * (TSDP_MAX_T + 1), cudaHostAllocDefault));
+  INIT_TRY(cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking));
+
+  // transformer workspaces, sized for the larger of (base over all candidates, drafter over B)
+  size_t rows_d = 0, rows_4d = 0, mem_rows_d = 0;
+  const int esz = cfg->precision == 0 ? 4 : 2;
+  for (int w = 0; w < 2; ++w) {
+    const tsdp_net_t& n = w == TSDP_BASE ? cfg->base : cfg->draft;
+    if (n.arch != TSDP_ARCH_XFMR) continue;
+    const size_t M = (w == TSDP_BASE ? B * K1 : B) * cfg->H;
+    rows_d = std::max(rows_d, M * n.d);
+    rows_4d = std::max(rows_4d, M * 4 * n.d);
+    mem_rows_d = std::max(mem_rows_d, std::max((size_t)T, B * cfg->obs_tokens) * n.d);
+  }
+  if (rows_d) {
+    st |= dev_alloc(c, c->allocs, &c->h, rows_d);
+    st |= alloc_bytes(c, c->allocs, &c->a, rows_d * esz);
+    st |= alloc_bytes(c, c->allocs, &c->qkv, rows_d * 3 * esz);
+    st |= alloc_bytes(c, c->allocs, &c->q2, rows_d * esz);
+    st |= alloc_bytes(c, c->allocs, &c->f, rows_4d * esz);
+    st |= alloc_bytes(c, c->allocs, &c->memtok, mem_rows_d * esz);
+    if (st) return fail(TSDP_ERR_CUDA);
+  }
+  if (cfg->precision == 1) {
+    cudaDriverEntryPointQueryResult q;
+    void* fn = nullptr;
+    INIT_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
+    if (!fn || q != cudaDriverEntryPointSuccess) { fprintf(stderr, "tsdp_init: cuTensorMapEncodeTiled unavailable\n"); return fail(TSDP_ERR_CUDA); }
+    c->encode = reinterpret_cast<EncodeTiledFn>(fn);
+    INIT_TRY(set_smem_attr_all<256>());
+    INIT_TRY(set_smem_attr_all<128>());
+    INIT_TRY(set_smem_attr_all<64>());
+    INIT_TRY(set_smem_attr_all<32>());
+  }
+  INIT_TRY(cudaFuncSetAttribute(self_attn_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+  INIT_TRY(cudaFuncSetAttribute(self_attn_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+  c->net[TSDP_BASE].cfg = cfg->base;
+  c->net[TSDP_DRAFT].cfg = cfg->draft;
+  INIT_TRY(cudaDeviceSynchronize());
+#undef INIT_TRY
+  *out = c;
+  return TSDP_OK;
+}
+
+void tsdp_destroy(tsdp_ctx* c) {
+  if (!c) return;
+  cudaSetDevice(c->cfg.device);
+  cudaDeviceSynchronize();
+  for (auto& g : c->graphs) cudaGraphExecDestroy(g.second);
+  for (void* p : c->allocs) cudaFree(p);
+  for (int w = 0; w < 2; ++w)
+    for (void* p : c->net[w].allocs) cudaFree(p);
+  if (c->host_done) cudaFreeHost(c->host_done);
+  if (c->sched_host) cudaFreeHost(c->sched_host);
+  if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
+  delete c;
+}
+
+int tsdp_load_weights(tsdp_ctx* c, int which, const float* blob, size_t n) {
+  if (!c || !blob || (which != TSDP_BASE && which != TSDP_DRAFT)) return TSDP_ERR_ARG;
+  CU_TRY(c, cudaSetDevice(c->cfg.device));
+  Net& net = c->net[which];
+  const tsdp_config_t& cfg = c->cfg;
+  if (n != weights_count(cfg, net.cfg)) return TSDP_ERR_WEIGHTS;
+  for (size_t i = 0; i < n; ++i)
+    if (!std::isfinite(blob[i])) return TSDP_ERR_NAN;
+  CU_TRY(c, cudaDeviceSynchronize());
+  for (void* p : net.allocs) cudaFree(p);
+  net.allocs.clear();
+  net.L.clear();
+  net.loaded = false;
+  // graphs captured with the old pointers are stale
+  for (auto& g : c->graphs) cudaGraphExecDestroy(g.second);
+  c->graphs.clear();
+  c->maps.clear();
+
+  const float* cur = blob;
+  const int D = c->D, T = cfg.T;
+  auto up_f32 = [&](float** dst, size_t cnt) -> int {
+    if (dev_alloc(c, net.allocs, dst, cnt)) return TSDP_ERR_CUDA;
+    CU_TRY(c, cudaMemcpy(*dst, cur, cnt * sizeof(float), cudaMemcpyHostToDevice));
+    cur += cnt;
+    return TSDP_OK;
+  };
+  // W [in, out] in the blob -> [out, in] on the device, in the GEMM operand type
+  auto up_wT = [&](void** dst, const float* src, size_t in, size_t outn) -> int {
+    if (cfg.precision == 0) {
+      std::vector<float> tmp(in * outn);
+      for (size_t i = 0; i < in; ++i)
+        for (size_t o = 0; o < outn; ++o) tmp[o * in + i] = src[i * outn + o];
+      float* p;
+      if (dev_alloc(c, net.allocs, &p, in * outn)) return TSDP_ERR_CUDA;
+      CU_TRY(c, cudaMemcpy(p, tmp.data(), tmp.size() * sizeof(float), cudaMemcpyHostToDevice));
+      *dst = p;
+    } else {
+      std::vector<__nv_bfloat16> tmp(in * outn);
+      for (size_t i = 0; i < in; ++i)
+        for (size_t o = 0; o < outn; ++o) tmp[o * in + i] = __float2bfloat16_rn(src[i * outn + o]);
+      __nv_bfloat16* p;
+      if (dev_alloc(c, net.allocs, &p, in * outn)) return TSDP_ERR_CUDA;
+      CU_TRY(c, cudaMemcpy(p, tmp.data(), tmp.size() * sizeof(__nv_bfloat16), cudaMemcpyHostToDevice));
+      *dst = p;
+    }
+    return TSDP_OK;
+  };
+  auto sinus_table = [&](int dim, float** dst) -> int {
+    std::vector<float> tb((size_t)T * dim);
+    const int half = dim / 2;
+    for (int t = 0; t < T; ++t)
+      for (int i = 0; i < half; ++i) {
+        const double fr = std::pow(10000.0, -(double)i / half);
+        tb[(size_t)t * dim + i] = (float)std::sin(t * fr);
+        tb[(size_t)t * dim + half + i] = (float)std::cos(t * fr);
+      }
+    if (dev_alloc(c, net.allocs, dst, tb.size())) return TSDP_ERR_CUDA;
+    CU_TRY(c, cudaMemcpy(*dst, tb.data(), tb.size() * sizeof(float), cudaMemcpyHostToDevice));
+    return TSDP_OK;
+  };
+  int r;
+  if (net.cfg.arch == TSDP_ARCH_GAUSS) {
+    net.m0 = blob[0];
+    net.s0 = blob[1];
+  } else if (net.cfg.arch == TSDP_ARCH_MLP) {
+    MlpWeights& m = net.mlp;
+    m = MlpWeights{};
+    m.n_lin = net.cfg.layers + 1;
+    m.temb = net.cfg.temb;
+    m.dims[0] = D + net.cfg.temb + cfg.obs_tokens * cfg.obs_dim;
+    for (int l = 1; l <= net.cfg.layers; ++l) m.dims[l] = net.cfg.d;
+    m.dims[m.n_lin] = D;
+    for (int l = 0; l < m.n_lin; ++l) {
+      float *W, *b;
+      if ((r = up_f32(&W, (size_t)m.dims[l] * m.dims[l + 1]))) return r;
+      if ((r = up_f32(&b, m.dims[l + 1]))) return r;
+      m.W[l] = W; m.b[l] = b;
+    }
+    float* tt;
+    if ((r = sinus_table(net.cfg.temb, &tt))) return r;
+    m.temb_table = tt;
+  } else {
+    const size_t d = net.cfg.d, A = cfg.A, H = cfg.H, To = cfg.obs_tokens, L = net.cfg.layers;
+    if ((r = up_f32(&net.W_in, A * d))) return r;
+    if ((r = up_f32(&net.b_in, d))) return r;
+    if ((r = up_f32(&net.pos, H * d))) return r;
+    if ((r = up_f32(&net.W_obs, (size_t)cfg.obs_dim * d))) return r;
+    if ((r = up_f32(&net.b_obs, d))) return r;
+    if ((r = up_f32(&net.cpos, (1 + To) * d))) return r;
+    std::vector<float> wkv_all(d * L * 2 * d), bkv_all(L * 2 * d);   // [in = d, out = L*2d]
+    net.L.resize(L);
+    for (size_t l = 0; l < L; ++l) {
+      XfmrLayer& w = net.L[l];
+      if ((r = up_f32(&w.ln1_g, d))) return r;
+      if ((r = up_f32(&w.ln1_b, d))) return r;
+      if ((r = up_wT(&w.Wqkv, cur, d, 3 * d))) return r;
+      cur += d * 3 * d;
+      if ((r = up_f32(&w.bqkv, 3 * d))) return r;
+      if ((r = up_wT(&w.Wo, cur, d, d))) return r;
+      cur += d * d;
+      if ((r = up_f32(&w.bo, d))) return r;
+      if ((r = up_f32(&w.ln2_g, d))) return r;
+      if ((r = up_f32(&w.ln2_b, d))) return r;
+      if ((r = up_wT(&w.Wq2, cur, d, d))) return r;
+      cur += d * d;
+      if ((r = up_f32(&w.bq2, d))) return r;
+      for (size_t i = 0; i < d; ++i)
+        for (size_t o = 0; o < 2 * d; ++o) wkv_all[i * (L * 2 * d) + l * 2 * d + o] = cur[i * 2 * d + o];
+      cur += d * 2 * d;
+      for (size_t o = 0; o < 2 * d; ++o) bkv_all[l * 2 * d + o] = cur[o];
+      cur += 2 * d;
+      if ((r = up_wT(&w.Wo2, cur, d, d))) return r;
+      cur += d * d;
+      if ((r = up_f32(&w.bo2, d))) return r;
+      if ((r = up_f32(&w.ln3_g, d))) return r;
+      if ((r = up_f32(&w.ln3_b, d))) return r;
+      if ((r = up_wT(&w.W1, cur, d, 4 * d))) return r;
+      cur += d * 4 * d;
+      if ((r = up_f32(&w.b1, 4 * d))) return r;
+      if ((r = up_wT(&w.W2, cur, 4 * d, d))) return r;
+      cur += 4 * d * d;
+      if ((r = up_f32(&w.b2, d))) return r;
+    }
+    if ((r = up_f32(&net.lnf_g, d))) return r;
+    if ((r = up_f32(&net.lnf_b, d))) return r;
+    {   // W_out [d, A] -> fp32 [A, d]
+      std::vector<float> tmp(A * d);
+      for (size_t i = 0; i < d; ++i)
+        for (size_t a = 0; a < A; ++a) tmp[a * d + i] = cur[i * A + a];
+      cur += d * A;
+      if (dev_alloc(c, net.allocs, &net.W_outT, A * d)) return TSDP_ERR_CUDA;
+      CU_TRY(c, cudaMemcpy(net.W_outT, tmp.data(), tmp.size() * sizeof(float), cudaMemcpyHostToDevice));
+    }
+    if ((r = up_f32(&net.b_out, A))) return r;
+    if ((r = up_wT(&net.Wkv_all, wkv_all.data(), d, L * 2 * d))) return r;
+    if (dev_alloc(c, net.allocs, &net.bkv_all, L * 2 * d)) return TSDP_ERR_CUDA;
+    CU_TRY(c, cudaMemcpy(net.bkv_all, bkv_all.data(), bkv_all.size() * sizeof(float), cudaMemcpyHostToDevice));
+    if (dev_alloc(c, net.allocs, &net.kv_time, (size_t)T * L * 2 * d)) return TSDP_ERR_CUDA;
+    if (dev_alloc(c, net.allocs, &net.kv_obs, (size_t)cfg.max_B * (To ? To : 1) * L * 2 * d)) return TSDP_ERR_CUDA;
+    if ((r = sinus_table((int)d, &net.temb_table))) return r;
+    // keys/values of the time token for every timestep: (sinusoidal(tau) + cpos[0]) Wkv2 + bkv2, all blocks
+    c->launches_per_round_tmp = 0;
+    if (cfg.precision == 0) {
+      memtok_kernel<float><<<T, d < 256 ? (int)d : 256>>>(net.temb_table, (int)d, nullptr, nullptr, net.cpos, 0, 0,
+                                                           reinterpret_cast<float*>(c->memtok), (int)d);
+    } else {
+      memtok_kernel<__nv_bfloat16><<<T, d < 256 ? (int)d : 256>>>(net.temb_table, (int)d, nullptr, nullptr, net.cpos, 0, 0,
+                                                                   reinterpret_cast<__nv_bfloat16*>(c->memtok), (int)d);
+    }
+    CU_TRY(c, cudaGetLastError());
+    if ((r = gemm(c, c->memtok, net.Wkv_all, net.bkv_all, T, (int)(L * 2 * d), (int)d, EPI_F32, net.kv_time, (int)(L * 2 * d), 0)))
+      return r;
+    CU_TRY(c, cudaDeviceSynchronize());
+    if ((r = check_status(c))) return r;
+  }
+  if ((size_t)(cur - blob) != n && net.cfg.arch != TSDP_ARCH_GAUSS) return TSDP_ERR_WEIGHTS;
+  net.loaded = true;
+  return TSDP_OK;
+}
+
+int tsdp_set_schedule(tsdp_ctx* c, const int* Ks, const tsdp_accept_t* accs, int n) {
+  if (!c || n < 0 || n > TSDP_MAX_T || (n > 0 && (!Ks || !accs))) return TSDP_ERR_ARG;
+  for (int i = 0; i < n; ++i)
+    if (Ks[i] < 0 || Ks[i] > c->cfg.max_K || !accept_ok(&accs[i])) return TSDP_ERR_ARG;
+  c->sched_K.assign(Ks, Ks + n);
+  c->sched_acc.assign(accs, accs + n);
+  return TSDP_OK;
+}
+
+static int sample_chunk_impl(tsdp_ctx* c, const float* obs, bool obs_on_host, int B, int K, const tsdp_accept_t* acc,
+                             uint64_t seed, float* actions, bool actions_on_host, cudaStream_t s) {
+  if (!c || !acc || !actions || B < 1 || B > c->cfg.max_B || K < 0 || K > c->cfg.max_K || !accept_ok(acc))
+    return TSDP_ERR_ARG;
+  const size_t obs_n = (size_t)B * c->cfg.obs_tokens * c->cfg.obs_dim;
+  if (obs_n > 0 && !obs) return TSDP_ERR_ARG;
+  if (!c->net[0].loaded || !c->net[1].loaded) return TSDP_ERR_STATE;
+  CU_TRY(c, cudaSetDevice(c->cfg.device));
+  const int D = c->D, T = c->cfg.T;
+  int r;
+  if (obs_n)
+    CU_TRY(c, cudaMemcpyAsync(c->obs, obs, obs_n * sizeof(float), obs_on_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, s));
+  CU_TRY(c, cudaMemcpyAsync(c->seed, &seed, sizeof(seed), cudaMemcpyHostToDevice, s));
+  if ((r = upload_schedule(c, K, *acc, s, false))) return r;
+  const long long xs_b = (long long)(c->cfg.max_K + 1) * D;
+  init_chunk_kernel<<<B, 128, 0, s>>>(c->xt, xs_b, c->t, B, D, T, c->seed, c->round_idx, c->n_done);
+  CU_TRY(c, cudaGetLastError());
+  c->launches_per_round_tmp = 0;
+  if ((r = prepare_obs(c, c->net[TSDP_BASE], B, s))) return r;
+  if ((r = prepare_obs(c, c->net[TSDP_DRAFT], B, s))) return r;
+  c->launches += 1 + c->launches_per_round_tmp;
+  // Rounds.  No environment can finish before the drafted windows could have covered T steps, so the
+  // completion flag is only read once that bound is reached.
+  const int n_sched = (int)c->sched_K.size();
+  int budget = T;
+  for (int round = 0; round <= T; ++round) {
+    const int Kr = n_sched > 0 ? c->sched_K[round < n_sched ? round : n_sched - 1] : K;
+    if ((r = run_round(c, B, Kr, s))) return r;
+    c->rounds++;
+    budget -= Kr + 1;
+    if (budget <= 0) {
+      CU_TRY(c, cudaStreamSynchronize(s));
+      if (*c->host_done >= B) break;
+    }
+  }
+  CU_TRY(c, cudaMemcpyAsync(actions, c->actions, (size_t)B * D * sizeof(float),
+                            actions_on_host ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice, s));
+  CU_TRY(c, cudaStreamSynchronize(s));
+  return check_status(c);
+}
+
+int tsdp_sample_chunk(tsdp_ctx* c, const float* d_obs, int B, int K, const tsdp_accept_t* acc, uint64_t seed,
+                      float* d_actions, void* stream) {
+  return sample_chunk_impl(c, d_obs, false, B, K, acc, seed, d_actions, false, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int tsdp_sample_chunk_host(tsdp_ctx* c, const float* h_obs, int B, int K, const tsdp_accept_t* acc, uint64_t seed,
+                           float* h_actions) {
+  return sample_chunk_impl(c, h_obs, true, B, K, acc, seed, h_actions, true, nullptr);
+}
+
+int tsdp_round(tsdp_ctx* c, const float* d_obs, int B, int K, const tsdp_accept_t* acc, uint64_t seed, float* d_x,
+               int* h_t, float* d_xtilde, float* d_muhat, float* d_eps, float* d_logalpha, int* h_jstar, void* stream) {
+  if (!c || !acc || !d_x || !h_t || B < 1 || B > c->cfg.max_B || K < 0 || K > c->cfg.max_K || !accept_ok(acc))
+    return TSDP_ERR_ARG;
+  for (int b = 0; b < B; ++b)
+    if (h_t[b] < -1 || h_t[b] >= c->cfg.T) return TSDP_ERR_ARG;
+  const size_t obs_n = (size_t)B * c->cfg.obs_tokens * c->cfg.obs_dim;
+  if (obs_n > 0 && !d_obs) return TSDP_ERR_ARG;
+  if (!c->net[0].loaded || !c->net[1].loaded) return TSDP_ERR_STATE;
+  CU_TRY(c, cudaSetDevice(c->cfg.device));
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  const int D = c->D;
+  const size_t K1 = c->cfg.max_K + 1, Km = c->cfg.max_K > 0 ? c->cfg.max_K : 1;
+  int r;
+  if (obs_n) CU_TRY(c, cudaMemcpyAsync(c->obs, d_obs, obs_n * sizeof(float), cudaMemcpyDeviceToDevice, s));
+  CU_TRY(c, cudaMemcpyAsync(c->seed, &seed, sizeof(seed), cudaMemcpyHostToDevice, s));
+  if ((r = upload_schedule(c, K, *acc, s, true))) return r;
+  CU_TRY(c, cudaMemsetAsync(c->round_idx, 0, sizeof(int), s));
+  CU_TRY(c, cudaMemsetAsync(c->n_done, 0, sizeof(int), s));
+  CU_TRY(c, cudaMemcpyAsync(c->t, h_t, sizeof(int) * B, cudaMemcpyHostToDevice, s));
+  CU_TRY(c, cudaMemcpy2DAsync(c->xt, K1 * D * sizeof(float), d_x, D * sizeof(float), D * sizeof(float), B, cudaMemcpyDeviceToDevice, s));
+  c->launches_per_round_tmp = 0;
+  if ((r = prepare_obs(c, c->net[TSDP_BASE], B, s))) return r;
+  if ((r = prepare_obs(c, c->net[TSDP_DRAFT], B, s))) return r;
+  if ((r = enqueue_round(c, B, K, s, true))) return r;
+  c->launches += c->launches_per_round_tmp;
+  c->rounds++;
+  // candidates and drafter means are still intact except slot 0, which now holds the new latent
+  if (d_xtilde) {
+    CU_TRY(c, cudaMemcpy2DAsync(d_xtilde, (size_t)(K + 1) * D * sizeof(float), c->xt, K1 * D * sizeof(float),
+                                (size_t)(K + 1) * D * sizeof(float), B, cudaMemcpyDeviceToDevice, s));
+    CU_TRY(c, cudaMemcpy2DAsync(d_xtilde, (size_t)(K + 1) * D * sizeof(float), d_x, D * sizeof(float), D * sizeof(float), B,
+                                cudaMemcpyDeviceToDevice, s));
+  }
+  if (d_muhat && K > 0)
+    CU_TRY(c, cudaMemcpy2DAsync(d_muhat, (size_t)K * D * sizeof(float), c->muhat, Km * D * sizeof(float),
+                                (size_t)K * D * sizeof(float), B, cudaMemcpyDeviceToDevice, s));
+  if (d_eps)
+    CU_TRY(c, cudaMemcpy2DAsync(d_eps, (size_t)(K + 1) * D * sizeof(float), c->eps, K1 * D * sizeof(float),
+                                (size_t)(K + 1) * D * sizeof(float), B, cudaMemcpyDeviceToDevice, s));
+  if (d_logalpha && K > 0)
+    CU_TRY(c, cudaMemcpyAsync(d_logalpha, c->dbg_logalpha, sizeof(float) * B * K, cudaMemcpyDeviceToDevice, s));
+  CU_TRY(c, cudaMemcpy2DAsync(d_x, D * sizeof(float), c->xt, K1 * D * sizeof(float), D * sizeof(float), B, cudaMemcpyDeviceToDevice, s));
+  CU_TRY(c, cudaMemcpyAsync(h_t, c->t, sizeof(int) * B, cudaMemcpyDeviceToHost, s));
+  if (h_jstar) CU_TRY(c, cudaMemcpyAsync(h_jstar, c->dbg_jstar, sizeof(int) * B, cudaMemcpyDeviceToHost, s));
+  CU_TRY(c, cudaStreamSynchronize(s));
+  return check_status(c);
+}
+
+int tsdp_denoise(tsdp_ctx* c, int which, const float* d_x, const int* h_tau, const float* d_obs, int N, float* d_eps,
+                 void* stream) {
+  if (!c || !d_x || !h_tau || !d_eps || N < 1 || N > c->cfg.max_B || (which != TSDP_BASE && which != TSDP_DRAFT))
+    return TSDP_ERR_ARG;
+  for (int i = 0; i < N; ++i)
+    if (h_tau[i] < 0 || h_tau[i] >= c->cfg.T) return TSDP_ERR_ARG;
+  const size_t obs_n = (size_t)N * c->cfg.obs_tokens * c->cfg.obs_dim;
+  if (obs_n > 0 && !d_obs) return TSDP_ERR_ARG;
+  Net& n = c->net[which];
+  if (!n.loaded) return TSDP_ERR_STATE;
+  CU_TRY(c, cudaSetDevice(c->cfg.device));
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  int r;
+  if (obs_n) CU_TRY(c, cudaMemcpyAsync(c->obs, d_obs, obs_n * sizeof(float), cudaMemcpyDeviceToDevice, s));
+  CU_TRY(c, cudaMemcpyAsync(c->t, h_tau, sizeof(int) * N, cudaMemcpyHostToDevice, s));
+  c->launches_per_round_tmp = 0;
+  if ((r = prepare_obs(c, n, N, s))) return r;
+  CandMap cm{d_x, (long long)c->D, d_eps, (long long)c->D, c->t, 1, 0};
+  if ((r = forward(c, n, cm, N, s))) return r;
+  c->launches += c->launches_per_round_tmp;
+  CU_TRY(c, cudaStreamSynchronize(s));
+  return check_status(c);
+}
+
+int tsdp_gemm(tsdp_ctx* c, const void* d_A, const void* d_W, const float* d_bias, int M, int N, int K, int epi,
+              void* d_out, void* stream) {
+  if (!c || !d_A || !d_W || !d_out || M < 1 || N < 1 || K < 1 || epi < 0 || epi > 3) return TSDP_ERR_ARG;
+  CU_TRY(c, cudaSetDevice(c->cfg.device));
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (c->cfg.precision == 0 && epi == EPI_STORE) epi = EPI_F32;
+  c->launches_per_round_tmp = 0;
+  int r = gemm(c, d_A, d_W, d_bias, M, N, K, epi, d_out, N, s);
+  c->launches += c->launches_per_round_tmp;
+  if (r) return r;
+  CU_TRY(c, cudaStreamSynchronize(s));
+  // test interface: operands are caller-owned and may be freed, so their tensor maps are not kept
+  c->maps.clear();
+  return check_status(c);
+}
+
+int tsdp_stats(tsdp_ctx* c, tsdp_stats_t* out) {
+  if (!c || !out) return TSDP_ERR_ARG;
+  CU_TRY(c, cudaSetDevice(c->cfg.device));
+  CU_TRY(c, cudaDeviceSynchronize());
+  static DevStats ds;
+  CU_TRY(c, cudaMemcpy(&ds, c->stats, sizeof(DevStats), cudaMemcpyDeviceToHost));
+  memset(out, 0, sizeof(*out));
+  out->chunks = ds.chunks_done;
+  out->rounds = c->rounds;
+  out->env_rounds = ds.env_rounds;
+  out->base_evals = ds.base_evals;
+  out->draft_evals = ds.draft_evals;
+  out->drafts_tested = ds.drafts_tested;
+  out->drafts_accepted = ds.drafts_accepted;
+  out->rejections = ds.rejections;
+  out->bonus_steps = ds.bonus_steps;
+  out->steps_advanced = ds.steps_advanced;
+  out->nfe = (double)ds.env_rounds + (double)c->cfg.draft_nfe * (double)ds.draft_evals;
+  for (int i = 0; i < TSDP_MAX_T; ++i) {
+    out->hist_drafted[i] = ds.hist_drafted[i];
+    out->hist_tested[i] = ds.hist_tested[i];
+    out->hist_accepted[i] = ds.hist_accepted[i];
+  }
+  return TSDP_OK;
+}
+
+int tsdp_reset_stats(tsdp_ctx* c) {
+  if (!c) return TSDP_ERR_ARG;
+  CU_TRY(c, cudaSetDevice(c->cfg.device));
+  CU_TRY(c, cudaDeviceSynchronize());
+  CU_TRY(c, cudaMemset(c->stats, 0, sizeof(DevStats)));
+  c->rounds = 0;
+  c->launches = 0;
+  return TSDP_OK;
+}
+
+uint64_t tsdp_kernel_launches(const tsdp_ctx* c) { return c ? c->launches : 0; }
+
+}  // extern "C"

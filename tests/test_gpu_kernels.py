@@ -1,0 +1,92 @@
+"""GPU parity, kernel level: the tcgen05 GEMM and each denoiser against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2512_15773_b200 import binding, inputs
+from oracle import nets as onets
+from tests import helpers as hp
+
+pytestmark = pytest.mark.gpu
+
+
+def _gemm_case(smp, M, N, K, epi, rng):
+    A = inputs.bf16_round(rng.normal(size=(M, K)))
+    W = inputs.bf16_round(rng.normal(size=(N, K)) / np.sqrt(K))
+    bias = rng.normal(size=N).astype(np.float32)
+    dA = torch.tensor(A, dtype=torch.bfloat16, device="cuda")
+    dW = torch.tensor(W, dtype=torch.bfloat16, device="cuda")
+    db = torch.tensor(bias, device="cuda")
+    ref = A @ W.T + bias.astype(np.float64)
+    if epi == 1:
+        ref = onets.gelu_tanh(ref)
+    if epi in (0, 1):
+        out = torch.zeros(M, N, dtype=torch.bfloat16, device="cuda")
+    else:
+        base = rng.normal(size=(M, N)).astype(np.float32)
+        out = torch.tensor(base, device="cuda") if epi == 2 else torch.zeros(M, N, device="cuda")
+        if epi == 2:
+            ref = ref + base
+    smp.gemm(dA, dW, db, M, N, K, epi, out)
+    got = out.float().cpu().numpy().astype(np.float64)
+    tol = 1e-2 if epi in (0, 1) else 2e-5          # bf16 output rounding vs fp32 accumulate only
+    err = hp.max_rel(got, ref)
+    assert err < tol, (M, N, K, epi, err)
+
+
+def test_tcgen05_gemm_against_fp64():
+    wl = hp.small_xfmr_workload(1)
+    smp, *_ = hp.setup(wl, max_B=1, max_K=1)
+    rng = np.random.default_rng(0)
+    # every tile width (32/64/128/256 are picked from M and N), ragged M, multi-wave, long K
+    for (M, N, K) in [(16, 128, 128), (144, 768, 256), (100, 32, 64), (129, 64, 512), (1000, 256, 128),
+                      (2500, 384, 128), (19000, 256, 256), (40000, 512, 512), (4111, 128, 2048)]:
+        for epi in (0, 1, 2, 3):
+            _gemm_case(smp, M, N, K, epi, rng)
+    smp.close()
+
+
+@pytest.mark.parametrize("arch", ["mlp", "gauss"])
+def test_small_denoisers(arch):
+    rng = np.random.default_rng(1)
+    if arch == "mlp":
+        wl = dict(inputs.WORKLOADS["toy_mlp"])
+    else:
+        wl = dict(H=4, A=3, To=0, Do=0, T=100, precision=0, base=dict(arch="gauss"), draft=dict(arch="gauss"),
+                  base_params=inputs.make_gauss_params(0.7, 0.5), draft_params=inputs.make_gauss_params(0.9, 0.4))
+    N = 37
+    smp, S, base, draft = hp.setup(wl, max_B=N, max_K=2)
+    x = rng.normal(size=(N, wl["H"], wl["A"])).astype(np.float32)
+    tau = rng.integers(0, 100, size=N).astype(np.int32); tau[0], tau[1] = 0, 99
+    obs = inputs.make_obs(0, N, wl["To"], wl["Do"]) if wl["To"] else np.zeros((N, 0, 0))
+    dx = torch.tensor(x, device="cuda"); dobs = torch.tensor(obs, dtype=torch.float32, device="cuda")
+    for which, net in ((binding.BASE, base), (binding.DRAFT, draft)):
+        out = torch.zeros_like(dx)
+        smp.denoise(which, dx, tau, dobs if wl["To"] else None, N, out)
+        ref = np.stack([net(x[n].astype(np.float64), int(tau[n]), obs[n]) for n in range(N)])
+        assert hp.max_rel(out.cpu().numpy(), ref) < 1e-4
+    smp.close()
+
+
+@pytest.mark.parametrize("precision,tol", [(0, 1e-4), (1, 2e-2)])
+@pytest.mark.parametrize("shape", ["small", "pusht"])
+def test_transformer_denoiser(precision, tol, shape):
+    rng = np.random.default_rng(2)
+    if shape == "small":
+        wl = hp.small_xfmr_workload(precision, d=128, heads=4, layers=2, dd=256, dlayers=1, H=7, A=3, To=3, Do=5,
+                                    gamma=1.0)
+    else:
+        wl = dict(inputs.WORKLOADS["pusht_xfmr"], precision=precision, gamma=1.0)
+    N = 19      # 19*H token rows: ragged against the 128-row tiles
+    smp, S, base, draft = hp.setup(wl, max_B=N, max_K=1)
+    x = rng.normal(size=(N, wl["H"], wl["A"])).astype(np.float32)
+    tau = rng.integers(0, 100, size=N).astype(np.int32); tau[0], tau[1] = 0, 99
+    obs = inputs.make_obs(5, N, wl["To"], wl["Do"])
+    dx = torch.tensor(x, device="cuda"); dobs = torch.tensor(obs, dtype=torch.float32, device="cuda")
+    for which, net in ((binding.BASE, base), (binding.DRAFT, draft)):
+        out = torch.zeros_like(dx)
+        smp.denoise(which, dx, tau, dobs, N, out)
+        ref = np.stack([net(x[n].astype(np.float64), int(tau[n]), obs[n]) for n in range(N)])
+        err = hp.max_rel(out.cpu().numpy(), ref)
+        assert err < tol, (which, err)
+    smp.close()

@@ -1,0 +1,362 @@
+#!/usr/bin/env python
+"""Benchmark of the TS-DP speculative denoising loop on B200.
+
+One "step" = one pass of the whole hot path (chunk init, speculative rounds until every environment
+reaches t = -1) for one batch of B environments with synthetic observations: B action chunks.
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+
+    python bench.py --gpus 1 --steps 10 --warmup 3
+    python -m torch.distributed.run --nnodes=1 --nproc-per-node N ... bench.py --gpus N ...
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "action_chunks_per_s"
+UNIT = "chunks/s"
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_burst=d["bf16_tflops"], bf16_sustained=d["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+# ---------------------------------------------------------------------------------------- workload
+def workload_spec(name, batch):
+    from paper_2512_15773_b200 import inputs
+    wl = dict(inputs.WORKLOADS[name])
+    if batch:
+        wl["B"] = batch
+    if name == "serving_xfmr":
+        Ks, Ss = inputs.markov_schedule(0, 64)
+        wl["schedule"] = (Ks, Ss)
+        wl["K"] = 10
+    return wl
+
+
+def rank_seed(base, rank, step):
+    """Seeds differ per rank and per step so that every GPU samples different chunks."""
+    return int(base + 1_000_003 * rank + step)
+
+
+def shard_info(world, B):
+    """Weak scaling: every rank runs its own B environments; there is no data-path collective."""
+    return dict(envs_per_rank=B, envs_total=B * world, scaling="weak")
+
+
+def reduce_max_time(local_ms, world):
+    """max over ranks of a device-measured duration (torch.distributed; identity on one rank)."""
+    if world == 1:
+        return local_ms
+    import torch
+    import torch.distributed as dist
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([local_ms], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def reduce_sum(values, world):
+    if world == 1:
+        return list(values)
+    import torch
+    import torch.distributed as dist
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor(list(values), dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return [float(v) for v in t.tolist()]
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device):
+        self.device, self.rows, self.proc = device, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.device), "-lms", "200"], stdout=subprocess.PIPE, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[1])); mx = float(r[2])
+            except Exception:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=(float(np.median(sm)) if sm else None), sm_max_mhz=mx, reasons=sorted(reasons),
+                    samples=len(sm))
+
+
+# ---------------------------------------------------------------------------------------- ours
+def make_sampler(wl, B, device, use_graph=1):
+    from paper_2512_15773_b200 import binding, inputs
+    max_K = max(wl["K"], 1)
+    cfg = binding.make_config(wl["H"], wl["A"], wl["To"], wl["Do"], wl["base"], wl["draft"], T=wl["T"], max_B=B,
+                              max_K=max_K, precision=wl["precision"], device=device, use_graph=use_graph)
+    smp = binding.Sampler(cfg)
+    smp.load_weights(binding.BASE, inputs.make_net(1, wl, "base"))
+    smp.load_weights(binding.DRAFT, inputs.make_net(2, wl, "draft"))
+    if "schedule" in wl:
+        Ks, Ss = wl["schedule"]
+        smp.set_schedule(Ks, [binding.AcceptT(0, 1.0, s, 1) for s in Ss])
+    return smp
+
+
+def time_steps(smp, d_obs, out, B, K, acc, seeds, host=False, h_obs=None, h_out=None):
+    """Device time of each step (CUDA events on the stream the library launches on: the default one)."""
+    import torch
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in seeds]
+    for (e0, e1), sd in zip(evs, seeds):
+        e0.record()
+        if host:
+            smp.sample_chunk_host(h_obs, B, K, acc, sd, h_out)
+        else:
+            smp.sample_chunk(d_obs, B, K, acc, sd, out)
+        e1.record()
+    torch.cuda.synchronize()
+    return [e0.elapsed_time(e1) for e0, e1 in evs]
+
+
+def run_ours(args):
+    import torch
+    from paper_2512_15773_b200 import binding, inputs
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    peaks = load_peaks()
+    wl = workload_spec(args.workload, args.batch)
+    B, K = wl["B"], wl["K"]
+    acc = binding.AcceptT(0, 1.0, 1.0, 1)
+    smp = make_sampler(wl, B, local)
+    obs = inputs.make_obs(100 + rank, B, wl["To"], wl["Do"]).astype(np.float32)
+    d_obs = torch.tensor(obs, device="cuda")
+    out = torch.zeros(B, wl["H"], wl["A"], device="cuda")
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- warm-up (captures the round graphs), then the timed region
+    time_steps(smp, d_obs, out, B, K, acc, [rank_seed(7, rank, -1 - i) for i in range(args.warmup)])
+    smp.reset_stats()
+    clocks = ClockSampler(local)
+    if rank == 0:
+        clocks.start()
+    barrier()
+    l0 = smp.kernel_launches()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    per_step = time_steps(smp, d_obs, out, B, K, acc, [rank_seed(7, rank, i) for i in range(args.steps)])
+    e1.record()
+    barrier()
+    total_ms = reduce_max_time(e0.elapsed_time(e1), world)
+    launches = smp.kernel_launches() - l0
+    st = smp.stats()
+    clk = clocks.stop() if rank == 0 else None
+    acc_steps, drafted, env_rounds, nfe = reduce_sum(
+        [st["drafts_accepted"], st["draft_evals"], st["env_rounds"], st["nfe"]], world)
+    chunks_total = B * world * args.steps
+    value = chunks_total / (total_ms / 1e3)
+
+    # ---- end to end through the host-buffer entry point (pinned host memory; copies inside the timing)
+    h_obs = torch.tensor(obs).pin_memory()
+    h_out = torch.zeros(B, wl["H"], wl["A"]).pin_memory()
+    time_steps(smp, None, None, B, K, acc, [rank_seed(9, rank, -1)], host=True, h_obs=h_obs.numpy(), h_out=h_out.numpy())
+    barrier()
+    e0.record()
+    time_steps(smp, None, None, B, K, acc, [rank_seed(9, rank, i) for i in range(args.steps)], host=True,
+               h_obs=h_obs.numpy(), h_out=h_out.numpy())
+    e1.record()
+    barrier()
+    e2e_ms = reduce_max_time(e0.elapsed_time(e1), world)
+    e2e = dict(value=chunks_total / (e2e_ms / 1e3), unit=UNIT, h2d_bytes_per_step=int(obs.nbytes),
+               d2h_bytes_per_step=int(h_out.numel() * 4))
+
+    result = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+                  ms_per_step=total_ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
+                  dtype="bf16" if wl["precision"] == 1 else "f32", data="synthetic")
+    if rank == 0:
+        # ---- per-kernel-family device time (plain launches with an event pair around each), same workload
+        smp.profile(1)
+        time_steps(smp, d_obs, out, B, K, acc, [rank_seed(7, rank, 0)])
+        prof = smp.profile_read()
+        smp.profile(0)
+        g = prof["gemm"]
+        fam_ms = {k: round(v["ms"], 3) for k, v in prof.items() if v["launches"]}
+        tot_ms = sum(v["ms"] for v in prof.values())
+        if wl["precision"] == 1 and g["launches"]:
+            ach = g["flop"] / (g["ms"] * 1e-3) / 1e12
+            result["roofline"] = dict(bound="tensor", kernel="gemm_tcgen05_kernel", achieved=ach,
+                                      peak=peaks["bf16_sustained"], unit="TFLOP/s", frac=ach / peaks["bf16_sustained"],
+                                      peak_source=f"bf16_tflops_sustained of {peaks['source']}", traffic=None,
+                                      launches_timed=g["launches"], avg_launch_us=1e3 * g["ms"] / g["launches"],
+                                      share_of_kernel_time=g["ms"] / tot_ms, family_ms=fam_ms)
+        else:
+            result["roofline"] = dict(bound="alu", kernel="mlp_forward_kernel", achieved=None, peak=None, unit="TFLOP/s",
+                                      frac=None, traffic=None, family_ms=fam_ms)
+        # ---- vanilla 100-step DDPM with the same kernels (K = 0), the latency comparator
+        smp.set_schedule([], [])
+        v_ms = time_steps(smp, d_obs, out, B, 0, acc, [rank_seed(7, rank, 0)] * 2)[-1]
+        vanilla = dict(ms_per_step=v_ms, chunks_per_s=B / (v_ms / 1e3))
+        # ---- batch-1 latency on the PushT-shaped configuration (the paper's Table 5 setting)
+        lat = None
+        if args.latency:
+            wl1 = workload_spec("pusht_xfmr", 1)
+            s1 = make_sampler(wl1, 1, local)
+            o1 = torch.tensor(inputs.make_obs(5, 1, wl1["To"], wl1["Do"]).astype(np.float32), device="cuda")
+            a1 = torch.zeros(1, wl1["H"], wl1["A"], device="cuda")
+            time_steps(s1, o1, a1, 1, wl1["K"], acc, list(range(8)))
+            s1.reset_stats()
+            ts = time_steps(s1, o1, a1, 1, wl1["K"], acc, list(range(100, 164)))
+            st1 = s1.stats()
+            time_steps(s1, o1, a1, 1, 0, acc, [0, 1])
+            tv = time_steps(s1, o1, a1, 1, 0, acc, list(range(8)))
+            lat = dict(workload="pusht_xfmr B=1 K=8", p50_chunk_ms=float(np.median(ts)), p99_chunk_ms=float(np.percentile(ts, 99)),
+                       vanilla_p50_chunk_ms=float(np.median(tv)), speedup_vs_vanilla=float(np.median(tv) / np.median(ts)),
+                       acceptance=st1["drafts_accepted"] / max(st1["draft_evals"], 1),
+                       base_forwards_per_chunk=st1["env_rounds"] / 64, drafts_per_chunk=st1["draft_evals"] / 64,
+                       nfe_per_chunk=st1["nfe"] / 64)
+            s1.close()
+        cpu = cpu_baseline(wl, budget_s=args.cpu_seconds) if world == 1 else None
+        result.update(
+            accepted_denoise_steps_per_s=acc_steps / (total_ms / 1e3),
+            p50_step_ms=float(np.median(per_step)),
+            acceptance=acc_steps / max(drafted, 1.0), base_forwards_per_chunk=env_rounds / chunks_total,
+            drafts_per_chunk=drafted / chunks_total, nfe_per_chunk=nfe / chunks_total,
+            vanilla=vanilla, speedup_vs_vanilla=vanilla["ms_per_step"] / (total_ms / args.steps),
+            latency_b1=lat, e2e=e2e, gpu_launches=int(launches), clocks=clk, cpu_baseline=cpu,
+            config=dict(workload=f"{args.workload} B={B} (config 4: 12L d512 h8 base, 2L d256 drafter, H16 A7, "
+                                 f"seeded 3-state Markov K/sigma schedule)" if args.workload == "serving_xfmr"
+                        else f"{args.workload} B={B} K={K}",
+                        global_batch=B * world, K_max=K, T=wl["T"], gamma=wl.get("gamma"),
+                        l2="per-step working set (activations of all candidates) exceeds the 126 MB L2; no explicit flush"
+                        if B * (K + 1) * wl["H"] * wl["base"].get("d", 0) * 16 > 126e6 else
+                        "working set fits L2 by design (weights are reused across rounds); no explicit flush",
+                        parallelism=f"replicas x{world} (environments sharded, no collective)"))
+        print(json.dumps(result))
+    smp.close()
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+# ---------------------------------------------------------------------------------------- oracle arm
+def oracle_chunk(wl, env, seed):
+    from oracle import ddpm, nets, spec
+    from paper_2512_15773_b200 import inputs
+    S = ddpm.Schedule(wl["T"], 1e-4, 0.02)
+    base = nets.make_denoiser(inputs.make_net(1, wl, "base"), S)
+    draft = nets.make_denoiser(inputs.make_net(2, wl, "draft"), S)
+    obs = inputs.make_obs(100, env + 1, wl["To"], wl["Do"])[env]
+    sched = None
+    if "schedule" in wl:
+        Ks, Ss = wl["schedule"]
+        sched = lambda r, t: (Ks[min(r, len(Ks) - 1)], spec.Accept(sigma_scale=Ss[min(r, len(Ks) - 1)]))
+    t0 = time.perf_counter()
+    spec.sample_chunk(S, base, draft, spec.PhiloxNoise(seed), env, obs, (wl["H"], wl["A"]), wl["K"], spec.Accept(),
+                      schedule=sched)
+    return time.perf_counter() - t0
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def cpu_baseline(wl, budget_s=20.0):
+    """The oracle as it stands, timed on this machine's host cores on a bounded sample of the workload."""
+    n, spent = 0, 0.0
+    while spent < budget_s and n < 8:
+        spent += oracle_chunk(wl, n, 7 + n)
+        n += 1
+    return dict(value=n / spent, unit=UNIT, cores=blas_threads(), kind="oracle",
+                sample=f"{n} environment-chunk(s) of the same workload, one at a time, numpy fp64")
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = workload_spec(args.workload, args.batch)
+    for i in range(args.warmup):
+        if i == 0:
+            oracle_chunk(wl, 0, 1)          # one warm-up chunk is enough to page the library in
+    t = [oracle_chunk(wl, i, 7 + i) for i in range(args.steps)]
+    total = sum(t)
+    value = args.steps / total
+    cpu = dict(value=value, unit=UNIT, cores=blas_threads(), kind="oracle",
+               sample=f"each step = 1 environment-chunk of {args.workload} (bounded sample of the batch)")
+    print(json.dumps(dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=int(os.environ.get("WORLD_SIZE", "1")),
+                          steps=args.steps, warmup=args.warmup, ms_per_step=1e3 * total / args.steps,
+                          higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                          config=dict(workload=f"{args.workload} (oracle: one environment per step)"),
+                          cpu_baseline=cpu,
+                          e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="serving_xfmr", choices=["serving_xfmr", "pusht_xfmr", "toy_mlp"])
+    ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--cpu-seconds", type=float, default=20.0)
+    ap.add_argument("--no-latency", dest="latency", action="store_false")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

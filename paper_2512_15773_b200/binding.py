@@ -15,7 +15,8 @@ BASE, DRAFT = 0, 1
 EXPORTS = ["tsdp_init", "tsdp_destroy", "tsdp_strerror", "tsdp_last_error", "tsdp_weights_count",
            "tsdp_load_weights", "tsdp_set_schedule", "tsdp_sample_chunk", "tsdp_sample_chunk_host",
            "tsdp_round", "tsdp_denoise", "tsdp_gemm", "tsdp_stats", "tsdp_reset_stats",
-           "tsdp_kernel_launches"]
+           "tsdp_kernel_launches", "tsdp_profile", "tsdp_profile_read"]
+PROF_FAMILIES = ["gemm", "layernorm", "attention", "embed_head", "round", "small_net"]
 
 
 class NetT(C.Structure):
@@ -76,6 +77,8 @@ def load_library():
     lib.tsdp_stats.argtypes = [vp, C.POINTER(StatsT)]
     lib.tsdp_reset_stats.argtypes = [vp]
     lib.tsdp_kernel_launches.argtypes = [vp]; lib.tsdp_kernel_launches.restype = u64
+    lib.tsdp_profile.argtypes = [vp, i]
+    lib.tsdp_profile_read.argtypes = [vp, fp, fp, fp]
     for n in EXPORTS:
         if getattr(lib, n).restype is C.c_int:
             pass
@@ -202,6 +205,16 @@ class Sampler:
 
     def reset_stats(self):
         self._check(self.lib.tsdp_reset_stats(self.h), "tsdp_reset_stats")
+
+    def profile(self, enable):
+        self._check(self.lib.tsdp_profile(self.h, int(enable)), "tsdp_profile")
+
+    def profile_read(self):
+        n = len(PROF_FAMILIES)
+        ms, fl, ln = np.zeros(n), np.zeros(n), np.zeros(n, dtype=np.uint64)
+        self._check(self.lib.tsdp_profile_read(self.h, ms.ctypes.data, fl.ctypes.data, ln.ctypes.data),
+                    "tsdp_profile_read")
+        return {f: dict(ms=float(ms[i]), flop=float(fl[i]), launches=int(ln[i])) for i, f in enumerate(PROF_FAMILIES)}
 
     def kernel_launches(self):
         return int(self.lib.tsdp_kernel_launches(self.h))

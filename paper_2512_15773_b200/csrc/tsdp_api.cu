@@ -78,6 +78,11 @@ struct tsdp_ctx {
   cudaStream_t cap_stream = nullptr;
   uint64_t rounds = 0, launches = 0;
   int launches_per_round_tmp = 0;
+  // optional per-kernel-family timing with CUDA events (plain launches, no graph)
+  bool prof_on = false;
+  std::vector<cudaEvent_t> prof_ev;
+  std::vector<int> prof_cat;
+  std::vector<double> prof_flop;
   std::string last_error;
 };
 
@@ -104,6 +109,20 @@ int dev_alloc(tsdp_ctx* c, std::vector<void*>& pool, T** p, size_t n) {
 
 int alloc_bytes(tsdp_ctx* c, std::vector<void*>& pool, void** p, size_t bytes) {
   return dev_alloc<uint8_t>(c, pool, reinterpret_cast<uint8_t**>(p), bytes);
+}
+
+constexpr size_t PROF_CAP = 60000;
+void prof_begin(tsdp_ctx* c, cudaStream_t s, int cat, double flop) {
+  if (!c->prof_on || c->prof_cat.size() >= PROF_CAP) return;
+  cudaEvent_t a, b;
+  if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) return;
+  c->prof_ev.push_back(a); c->prof_ev.push_back(b);
+  c->prof_cat.push_back(cat); c->prof_flop.push_back(flop);
+  cudaEventRecord(a, s);
+}
+void prof_end(tsdp_ctx* c, cudaStream_t s) {
+  if (!c->prof_on || c->prof_ev.empty() || c->prof_ev.size() != 2 * c->prof_cat.size()) return;
+  cudaEventRecord(c->prof_ev.back(), s);
 }
 
 bool net_cfg_ok(const tsdp_config_t& cfg, const tsdp_net_t& n) {
@@ -159,7 +178,9 @@ template <int BN, int EPI>
 int launch_tc(tsdp_ctx* c, const CUtensorMap& ma, const CUtensorMap& mb, const GemmArgs& g, cudaStream_t s) {
   const int tiles = ((g.M + GEMM_BM - 1) / GEMM_BM) * (g.N / BN);
   const int grid = tiles < c->num_sms ? tiles : c->num_sms;
+  prof_begin(c, s, 0, 2.0 * g.M * g.N * g.K);
   gemm_tcgen05_kernel<BN, EPI><<<grid, GEMM_THREADS, gemm_smem_bytes(BN), s>>>(ma, mb, g);
+  prof_end(c, s);
   c->launches_per_round_tmp++;
   CU_TRY(c, cudaGetLastError());
   return TSDP_OK;
@@ -209,11 +230,13 @@ int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, in
     dim3 grid((N + 63) / 64, (M + 63) / 64);
     const float* a = reinterpret_cast<const float*>(A);
     const float* w = reinterpret_cast<const float*>(W);
+    prof_begin(c, s, 0, 2.0 * M * N * K);
     switch (epi) {
       case EPI_GELU: gemm_simt_kernel<EPI_GELU><<<grid, 256, 0, s>>>(a, w, g); break;
       case EPI_RESID: gemm_simt_kernel<EPI_RESID><<<grid, 256, 0, s>>>(a, w, g); break;
       default: gemm_simt_kernel<EPI_F32><<<grid, 256, 0, s>>>(a, w, g); break;
     }
+    prof_end(c, s);
     c->launches_per_round_tmp++;
     CU_TRY(c, cudaGetLastError());
     return TSDP_OK;
@@ -240,6 +263,7 @@ template <typename T>
 int ln_launch(tsdp_ctx* c, const float* h, const float* g, const float* b, T* out, int M, int d, cudaStream_t s) {
   const int wpb = 8;
   const int grid = (M + wpb - 1) / wpb;
+  prof_begin(c, s, 1, 0.0);
   switch (d / 128) {
     case 1: ln_kernel<T, 1><<<grid, wpb * 32, 0, s>>>(h, g, b, out, M); break;
     case 2: ln_kernel<T, 2><<<grid, wpb * 32, 0, s>>>(h, g, b, out, M); break;
@@ -250,6 +274,7 @@ int ln_launch(tsdp_ctx* c, const float* h, const float* g, const float* b, T* ou
     case 7: ln_kernel<T, 7><<<grid, wpb * 32, 0, s>>>(h, g, b, out, M); break;
     default: ln_kernel<T, 8><<<grid, wpb * 32, 0, s>>>(h, g, b, out, M); break;
   }
+  prof_end(c, s);
   c->launches_per_round_tmp++;
   CU_TRY(c, cudaGetLastError());
   return TSDP_OK;
@@ -260,6 +285,7 @@ int head_launch(tsdp_ctx* c, const Net& n, const CandMap& cm, int M, cudaStream_
   const int grid = (M + wpb - 1) / wpb;
   const int H = c->cfg.H, A = c->cfg.A;
 #define HEAD_CASE(V) head_kernel<V><<<grid, wpb * 32, 0, s>>>(c->h, n.lnf_g, n.lnf_b, n.W_outT, n.b_out, cm, M, H, A)
+  prof_begin(c, s, 3, 0.0);
   switch (n.cfg.d / 128) {
     case 1: HEAD_CASE(1); break;
     case 2: HEAD_CASE(2); break;
@@ -271,6 +297,7 @@ int head_launch(tsdp_ctx* c, const Net& n, const CandMap& cm, int M, cudaStream_
     default: HEAD_CASE(8); break;
   }
 #undef HEAD_CASE
+  prof_end(c, s);
   c->launches_per_round_tmp++;
   CU_TRY(c, cudaGetLastError());
   return TSDP_OK;
@@ -286,7 +313,9 @@ int xfmr_forward_t(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStrea
   T* q2 = reinterpret_cast<T*>(c->q2);
   T* f = reinterpret_cast<T*>(c->f);
   int r;
+  prof_begin(c, s, 3, 0.0);
   embed_kernel<<<M, d < 256 ? d : 256, 0, s>>>(cm, n.W_in, n.b_in, n.pos, c->h, H, A, d);
+  prof_end(c, s);
   c->launches_per_round_tmp++;
   CU_TRY(c, cudaGetLastError());
   const int sa_wpb = 4;
@@ -296,14 +325,18 @@ int xfmr_forward_t(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStrea
     const XfmrLayer& w = n.L[l];
     if ((r = ln_launch<T>(c, c->h, w.ln1_g, w.ln1_b, a, M, d, s))) return r;
     if ((r = gemm(c, a, w.Wqkv, w.bqkv, M, 3 * d, d, out_epi, qkv, 3 * d, s))) return r;
+    prof_begin(c, s, 2, 0.0);
     self_attn_kernel<T><<<(n_cand * heads + sa_wpb - 1) / sa_wpb, sa_wpb * 32, sa_smem, s>>>(qkv, a, n_cand, H, d, heads);
+    prof_end(c, s);
     c->launches_per_round_tmp++;
     CU_TRY(c, cudaGetLastError());
     if ((r = gemm(c, a, w.Wo, w.bo, M, d, d, EPI_RESID, c->h, d, s))) return r;
     if ((r = ln_launch<T>(c, c->h, w.ln2_g, w.ln2_b, a, M, d, s))) return r;
     if ((r = gemm(c, a, w.Wq2, w.bq2, M, d, d, out_epi, q2, d, s))) return r;
+    prof_begin(c, s, 2, 0.0);
     cross_attn_kernel<T><<<(M + 7) / 8, 256, 0, s>>>(q2, a, n.kv_time, n.kv_obs, cm, M, H, d, heads, c->cfg.obs_tokens, l, L,
                                                       c->cfg.T);
+    prof_end(c, s);
     c->launches_per_round_tmp++;
     CU_TRY(c, cudaGetLastError());
     if ((r = gemm(c, a, w.Wo2, w.bo2, M, d, d, EPI_RESID, c->h, d, s))) return r;
@@ -320,7 +353,9 @@ int xfmr_prepare_obs_t(tsdp_ctx* c, Net& n, int B, cudaStream_t s) {
   const int To = c->cfg.obs_tokens, d = n.cfg.d, L = n.cfg.layers;
   if (To == 0) return TSDP_OK;
   T* mt = reinterpret_cast<T*>(c->memtok);
+  prof_begin(c, s, 3, 0.0);
   memtok_kernel<T><<<B * To, d < 256 ? d : 256, 0, s>>>(c->obs, c->cfg.obs_dim, n.W_obs, n.b_obs, n.cpos, To, 1, mt, d);
+  prof_end(c, s);
   c->launches_per_round_tmp++;
   CU_TRY(c, cudaGetLastError());
   return gemm(c, mt, n.Wkv_all, n.bkv_all, B * To, L * 2 * d, d, EPI_F32, n.kv_obs, L * 2 * d, s);
@@ -337,7 +372,9 @@ int forward(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStream_t s) 
   switch (n.cfg.arch) {
     case TSDP_ARCH_GAUSS: {
       const long long tot = (long long)n_cand * D;
+      prof_begin(c, s, 5, 0.0);
       gauss_forward_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, s>>>(c->S, n.m0, n.s0, cm, n_cand, D);
+      prof_end(c, s);
       c->launches_per_round_tmp++;
       CU_TRY(c, cudaGetLastError());
       return TSDP_OK;
@@ -345,8 +382,10 @@ int forward(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStream_t s) 
     case TSDP_ARCH_MLP: {
       int maxw = 0;
       for (int l = 0; l <= n.mlp.n_lin; ++l) maxw = n.mlp.dims[l] > maxw ? n.mlp.dims[l] : maxw;
+      prof_begin(c, s, 5, 0.0);
       mlp_forward_kernel<<<n_cand, 256, 2 * maxw * sizeof(float), s>>>(n.mlp, cm, c->obs, c->cfg.obs_tokens * c->cfg.obs_dim,
                                                                         D, c->cfg.T);
+      prof_end(c, s);
       c->launches_per_round_tmp++;
       CU_TRY(c, cudaGetLastError());
       return TSDP_OK;
@@ -367,7 +406,9 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
   for (int k = 1; k <= K; ++k) {
     CandMap cm{c->xt + (long long)(k - 1) * D, xs_b, c->eps_d, (long long)D, c->t, 1, k - 1};
     if ((r = forward(c, c->net[TSDP_DRAFT], cm, B, s))) return r;
+    prof_begin(c, s, 4, 0.0);
     draft_step_kernel<<<B, 128, 0, s>>>(c->S, c->xt, xs_b, c->muhat, ms_b, c->eps_d, c->t, k, D, c->seed);
+    prof_end(c, s);
     c->launches_per_round_tmp++;
     CU_TRY(c, cudaGetLastError());
   }
@@ -376,9 +417,11 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
   int warps = K < 1 ? 1 : K;
   if (warps < 4) warps = 4;
   if (warps > 16) warps = 16;
+  prof_begin(c, s, 4, 0.0);
   accept_kernel<<<B, warps * 32, 0, s>>>(c->S, c->xt, xs_b, c->muhat, ms_b, c->eps, xs_b, c->t, K, D, c->seed, c->sched,
                                          TSDP_MAX_T + 1, c->round_idx, c->actions, c->n_done, c->stats, c->cfg.draft_nfe,
                                          dbg ? c->dbg_logalpha : nullptr, dbg ? c->dbg_jstar : nullptr);
+  prof_end(c, s);
   round_end_kernel<<<1, 1, 0, s>>>(c->round_idx, c->n_done, c->host_done);
   c->launches_per_round_tmp += 2;
   CU_TRY(c, cudaGetLastError());
@@ -388,7 +431,7 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
 struct GraphRec { cudaGraphExec_t exec; int launches; };
 
 int run_round(tsdp_ctx* c, int B, int K, cudaStream_t s) {
-  if (!c->cfg.use_graph) {
+  if (!c->cfg.use_graph || c->prof_on) {
     c->launches_per_round_tmp = 0;
     int r = enqueue_round(c, B, K, s, false);
     c->launches += c->launches_per_round_tmp;
@@ -605,6 +648,7 @@ void tsdp_destroy(tsdp_ctx* c) {
   cudaSetDevice(c->cfg.device);
   cudaDeviceSynchronize();
   for (auto& g : c->graphs) cudaGraphExecDestroy(g.second);
+  for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
   for (void* p : c->allocs) cudaFree(p);
   for (int w = 0; w < 2; ++w)
     for (void* p : c->net[w].allocs) cudaFree(p);
@@ -960,5 +1004,29 @@ int tsdp_reset_stats(tsdp_ctx* c) {
 }
 
 uint64_t tsdp_kernel_launches(const tsdp_ctx* c) { return c ? c->launches : 0; }
+
+int tsdp_profile(tsdp_ctx* c, int enable) {
+  if (!c) return TSDP_ERR_ARG;
+  CU_TRY(c, cudaSetDevice(c->cfg.device));
+  CU_TRY(c, cudaDeviceSynchronize());
+  for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
+  c->prof_ev.clear(); c->prof_cat.clear(); c->prof_flop.clear();
+  c->prof_on = enable != 0;
+  return TSDP_OK;
+}
+
+int tsdp_profile_read(tsdp_ctx* c, double* ms, double* flop, uint64_t* launches) {
+  if (!c || !ms || !flop || !launches) return TSDP_ERR_ARG;
+  CU_TRY(c, cudaSetDevice(c->cfg.device));
+  CU_TRY(c, cudaDeviceSynchronize());
+  for (int i = 0; i < TSDP_PROF_FAMILIES; ++i) { ms[i] = 0.0; flop[i] = 0.0; launches[i] = 0; }
+  for (size_t i = 0; i < c->prof_cat.size(); ++i) {
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, c->prof_ev[2 * i], c->prof_ev[2 * i + 1]) != cudaSuccess) continue;
+    const int k = c->prof_cat[i];
+    ms[k] += t; flop[k] += c->prof_flop[i]; launches[k] += 1;
+  }
+  return TSDP_OK;
+}
 
 }  // extern "C"

@@ -201,6 +201,13 @@ def run_ours(args):
     chunks_total = B * world * args.steps
     value = chunks_total / (total_ms / 1e3)
 
+    if args.only_timed:
+        if rank == 0:
+            print(json.dumps(dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps,
+                                  warmup=args.warmup, ms_per_step=total_ms / args.steps, gpu_launches=int(launches),
+                                  note="timed region only (launch-list capture)")))
+        smp.close()
+        return
     # ---- end to end through the host-buffer entry point (pinned host memory; copies inside the timing)
     h_obs = torch.tensor(obs).pin_memory()
     h_out = torch.zeros(B, wl["H"], wl["A"]).pin_memory()
@@ -313,6 +320,8 @@ def blas_threads():
 def cpu_baseline(wl, budget_s=20.0):
     """The oracle as it stands, timed on this machine's host cores on a bounded sample of the workload."""
     n, spent = 0, 0.0
+    if budget_s <= 0:
+        return None
     while spent < budget_s and n < 8:
         spent += oracle_chunk(wl, n, 7 + n)
         n += 1
@@ -351,6 +360,8 @@ def main():
     ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
     ap.add_argument("--no-latency", dest="latency", action="store_false")
+    ap.add_argument("--only-timed", action="store_true",
+                    help="run warm-up and the timed region only (for a profiler's launch list)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

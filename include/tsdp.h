@@ -154,6 +154,12 @@ int tsdp_denoise(tsdp_ctx* ctx, int which, const float* d_x, const int* h_tau, c
 int tsdp_gemm(tsdp_ctx* ctx, const void* d_A, const void* d_W, const float* d_bias, int M, int N, int K,
               int epi, void* d_out, void* cuda_stream);
 
+/* The same GEMM launched `reps` times back to back between one pair of CUDA events on `cuda_stream`
+ * (after one untimed launch); *h_ms (HOST) receives the mean device time of one launch in milliseconds.
+ * With EPI 2 the output accumulates over the launches.  Measurement interface; synchronous. */
+int tsdp_gemm_timed(tsdp_ctx* ctx, const void* d_A, const void* d_W, const float* d_bias, int M, int N, int K,
+                    int epi, void* d_out, int reps, float* h_ms, void* cuda_stream);
+
 /* Copy the counters accumulated since the last reset (synchronises the device). */
 int tsdp_stats(tsdp_ctx* ctx, tsdp_stats_t* out);
 int tsdp_reset_stats(tsdp_ctx* ctx);
@@ -163,11 +169,12 @@ uint64_t tsdp_kernel_launches(const tsdp_ctx* ctx);
 
 /* Per-kernel-family device timing with CUDA events, for the roofline report.  While enabled, rounds
  * are issued as plain launches (no graph) with an event pair around each launch on the caller's
- * stream.  Families: 0 GEMM (tcgen05 or check-mode), 1 LayerNorm, 2 attention, 3 embed/head/memory
- * tokens, 4 round kernels (draft step, accept), 5 MLP / Gaussian denoiser.  tsdp_profile(ctx, 0|1)
+ * stream.  Families: 0 GEMMs of the base model (tcgen05 or check-mode), 1 LayerNorm, 2 attention,
+ * 3 embed/head/memory tokens, 4 round kernels (draft step, accept), 5 MLP / Gaussian denoiser, 6 GEMMs
+ * of the drafter.  tsdp_profile(ctx, 0|1)
  * clears the record.  tsdp_profile_read fills three arrays of TSDP_PROF_FAMILIES entries: summed
  * milliseconds, summed algorithmic flops (2*M*N*K per GEMM launch, 0 elsewhere) and launch counts. */
-enum { TSDP_PROF_FAMILIES = 6 };
+enum { TSDP_PROF_FAMILIES = 7 };
 int tsdp_profile(tsdp_ctx* ctx, int enable);
 int tsdp_profile_read(tsdp_ctx* ctx, double* ms, double* flop, uint64_t* launches);
 

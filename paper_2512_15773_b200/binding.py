@@ -14,9 +14,9 @@ ARCH = {"gauss": 0, "mlp": 1, "xfmr": 2}
 BASE, DRAFT = 0, 1
 EXPORTS = ["tsdp_init", "tsdp_destroy", "tsdp_strerror", "tsdp_last_error", "tsdp_weights_count",
            "tsdp_load_weights", "tsdp_set_schedule", "tsdp_sample_chunk", "tsdp_sample_chunk_host",
-           "tsdp_round", "tsdp_denoise", "tsdp_gemm", "tsdp_stats", "tsdp_reset_stats",
+           "tsdp_round", "tsdp_denoise", "tsdp_gemm", "tsdp_gemm_timed", "tsdp_stats", "tsdp_reset_stats",
            "tsdp_kernel_launches", "tsdp_profile", "tsdp_profile_read"]
-PROF_FAMILIES = ["gemm", "layernorm", "attention", "embed_head", "round", "small_net"]
+PROF_FAMILIES = ["gemm", "layernorm", "attention", "embed_head", "round", "small_net", "gemm_draft"]
 
 
 class NetT(C.Structure):
@@ -74,6 +74,7 @@ def load_library():
     lib.tsdp_round.argtypes = [vp, fp, i, i, C.POINTER(AcceptT), u64, fp, fp, fp, fp, fp, fp, fp, vp]
     lib.tsdp_denoise.argtypes = [vp, i, fp, fp, fp, i, fp, vp]
     lib.tsdp_gemm.argtypes = [vp, fp, fp, fp, i, i, i, i, fp, vp]
+    lib.tsdp_gemm_timed.argtypes = [vp, fp, fp, fp, i, i, i, i, fp, i, C.POINTER(C.c_float), vp]
     lib.tsdp_stats.argtypes = [vp, C.POINTER(StatsT)]
     lib.tsdp_reset_stats.argtypes = [vp]
     lib.tsdp_kernel_launches.argtypes = [vp]; lib.tsdp_kernel_launches.restype = u64
@@ -193,6 +194,12 @@ class Sampler:
     def gemm(self, d_A, d_W, d_bias, M, N, K, epi, d_out, stream=0):
         self._check(self.lib.tsdp_gemm(self.h, _ptr(d_A), _ptr(d_W), _ptr(d_bias), M, N, K, epi, _ptr(d_out),
                                        stream), "tsdp_gemm")
+
+    def gemm_timed(self, d_A, d_W, d_bias, M, N, K, epi, d_out, reps, stream=0):
+        ms = C.c_float(0.0)
+        self._check(self.lib.tsdp_gemm_timed(self.h, _ptr(d_A), _ptr(d_W), _ptr(d_bias), M, N, K, epi, _ptr(d_out),
+                                             reps, C.byref(ms), stream), "tsdp_gemm_timed")
+        return ms.value
 
     def stats(self):
         s = StatsT()

@@ -80,6 +80,7 @@ struct tsdp_ctx {
   int launches_per_round_tmp = 0;
   // optional per-kernel-family timing with CUDA events (plain launches, no graph)
   bool prof_on = false;
+  int prof_gemm_cat = 0;                      // 0 while the base model runs, 6 while the drafter runs
   std::vector<cudaEvent_t> prof_ev;
   std::vector<int> prof_cat;
   std::vector<double> prof_flop;
@@ -178,7 +179,7 @@ template <int BN, int EPI>
 int launch_tc(tsdp_ctx* c, const CUtensorMap& ma, const CUtensorMap& mb, const GemmArgs& g, cudaStream_t s) {
   const int tiles = ((g.M + GEMM_BM - 1) / GEMM_BM) * (g.N / BN);
   const int grid = tiles < c->num_sms ? tiles : c->num_sms;
-  prof_begin(c, s, 0, 2.0 * g.M * g.N * g.K);
+  prof_begin(c, s, c->prof_gemm_cat, 2.0 * g.M * g.N * g.K);
   gemm_tcgen05_kernel<BN, EPI><<<grid, GEMM_THREADS, gemm_smem_bytes(BN), s>>>(ma, mb, g);
   prof_end(c, s);
   c->launches_per_round_tmp++;
@@ -230,7 +231,7 @@ int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, in
     dim3 grid((N + 63) / 64, (M + 63) / 64);
     const float* a = reinterpret_cast<const float*>(A);
     const float* w = reinterpret_cast<const float*>(W);
-    prof_begin(c, s, 0, 2.0 * M * N * K);
+    prof_begin(c, s, c->prof_gemm_cat, 2.0 * M * N * K);
     switch (epi) {
       case EPI_GELU: gemm_simt_kernel<EPI_GELU><<<grid, 256, 0, s>>>(a, w, g); break;
       case EPI_RESID: gemm_simt_kernel<EPI_RESID><<<grid, 256, 0, s>>>(a, w, g); break;
@@ -405,7 +406,10 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
   int r;
   for (int k = 1; k <= K; ++k) {
     CandMap cm{c->xt + (long long)(k - 1) * D, xs_b, c->eps_d, (long long)D, c->t, 1, k - 1};
-    if ((r = forward(c, c->net[TSDP_DRAFT], cm, B, s))) return r;
+    c->prof_gemm_cat = 6;
+    r = forward(c, c->net[TSDP_DRAFT], cm, B, s);
+    c->prof_gemm_cat = 0;
+    if (r) return r;
     prof_begin(c, s, 4, 0.0);
     draft_step_kernel<<<B, 128, 0, s>>>(c->S, c->xt, xs_b, c->muhat, ms_b, c->eps_d, c->t, k, D, c->seed);
     prof_end(c, s);
@@ -964,6 +968,34 @@ int tsdp_gemm(tsdp_ctx* c, const void* d_A, const void* d_W, const float* d_bias
   CU_TRY(c, cudaStreamSynchronize(s));
   // test interface: operands are caller-owned and may be freed, so their tensor maps are not kept
   c->maps.clear();
+  return check_status(c);
+}
+
+int tsdp_gemm_timed(tsdp_ctx* c, const void* d_A, const void* d_W, const float* d_bias, int M, int N, int K, int epi,
+                    void* d_out, int reps, float* h_ms, void* stream) {
+  if (!c || !d_A || !d_W || !d_out || !h_ms || M < 1 || N < 1 || K < 1 || epi < 0 || epi > 3 || reps < 1)
+    return TSDP_ERR_ARG;
+  CU_TRY(c, cudaSetDevice(c->cfg.device));
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (c->cfg.precision == 0 && epi == EPI_STORE) epi = EPI_F32;
+  cudaEvent_t e0, e1;
+  CU_TRY(c, cudaEventCreate(&e0));
+  CU_TRY(c, cudaEventCreate(&e1));
+  c->launches_per_round_tmp = 0;
+  int r = gemm(c, d_A, d_W, d_bias, M, N, K, epi, d_out, N, s);     // builds the tensor maps, warms up
+  cudaEventRecord(e0, s);
+  for (int i = 0; i < reps && r == TSDP_OK; ++i) r = gemm(c, d_A, d_W, d_bias, M, N, K, epi, d_out, N, s);
+  cudaEventRecord(e1, s);
+  c->launches += c->launches_per_round_tmp;
+  cudaError_t e = cudaStreamSynchronize(s);
+  float ms = 0.f;
+  if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  c->maps.clear();
+  if (r) return r;
+  CU_TRY(c, e);
+  *h_ms = ms / reps;
   return check_status(c);
 }
 

@@ -35,7 +35,8 @@ typedef enum {
   TSDP_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed (see tsdp_last_error)   */
   TSDP_ERR_TIMEOUT = 5,     /* a bounded wait inside a kernel expired                      */
   TSDP_ERR_NAN = 6,         /* non-finite value in a weight blob                           */
-  TSDP_ERR_UNSUPPORTED = 7  /* architecture not built                                      */
+  TSDP_ERR_UNSUPPORTED = 7, /* architecture not built                                      */
+  TSDP_ERR_TOO_LARGE = 8    /* size beyond the capacity of tsdp_verify_commit_static       */
 } tsdp_status;
 
 enum { TSDP_ARCH_GAUSS = 0, TSDP_ARCH_MLP = 1, TSDP_ARCH_XFMR = 2 };
@@ -177,6 +178,47 @@ uint64_t tsdp_kernel_launches(const tsdp_ctx* ctx);
 enum { TSDP_PROF_FAMILIES = 7 };
 int tsdp_profile(tsdp_ctx* ctx, int enable);
 int tsdp_profile_read(tsdp_ctx* ctx, double* ms, double* flop, uint64_t* launches);
+
+/* Verification tail without any allocation.  (The paper has no counterpart: this entry point exists
+ * for integration, not for the method.)
+ *
+ * Who needs it: code that runs where device memory cannot be requested -- a control loop that was
+ * handed a fixed memory budget at start-up, a plug-in inside a host application that owns the
+ * allocator, a real-time thread that must not take the driver's allocation lock.  Such a caller
+ * cannot create a tsdp_ctx (tsdp_init allocates), but it may already hold the candidate latents,
+ * drafter means and base outputs of a round and only need the decision: the posterior mean of every
+ * candidate, the log acceptance ratios, the first rejected step j*, and the committed latent
+ * (reflection at j*, bonus step, or last draft).  This function does exactly what the fused
+ * acceptance kernel of tsdp_sample_chunk does, on caller-owned buffers, and calls neither
+ * cudaMalloc / cudaFree nor any routine that allocates.
+ *
+ * Its working memory (DDPM tables for T steps, t[B], j*[B], the counters, seed and round
+ * parameters: under 64 KiB) is a fixed array inside the library image; every GPU that loads the
+ * library holds it until the process exits.  Capacity: B <= TSDP_STATIC_MAX_B, T <= TSDP_STATIC_MAX_T,
+ * K <= TSDP_MAX_K; larger sizes return TSDP_ERR_TOO_LARGE and print the limits to stderr.
+ * The first call on a device looks up the array's device address; make that first call before any
+ * stream capture begins.  All calls share the one array, which still holds the previous call's
+ * values on entry (the function clears what must start at zero itself); two calls whose GPU work
+ * overlaps -- different streams or threads -- race on it.  Synchronous: returns after `cuda_stream`
+ * has finished the work.
+ *
+ *   device              CUDA device ordinal (made current)
+ *   T, beta0, beta1, clip   DDPM schedule, as in tsdp_config_t
+ *   d_xt   [B, K+1, D]  DEVICE, in/out: candidate latents, slot 0 = the round's input latent; on return
+ *                       slot 0 of every unfinished environment holds the committed latent
+ *   d_muhat [B, K, D]   DEVICE, in: drafter means (may be null when K = 0)
+ *   d_eps  [B, K+1, D]  DEVICE, in: base-model outputs for every candidate
+ *   h_t    [B]          HOST, in: timestep of each environment's input latent (-1 = finished, skipped)
+ *   accept, seed        as in tsdp_sample_chunk; draft_nfe is ignored by the decision
+ *   d_actions [B, D]    DEVICE, out: written for environments that reach t = -1 in this round
+ *   h_t_new, h_jstar [B] HOST, out: new timesteps; first rejected step (K_eff+1 if none, -1 if finished)
+ *   d_logalpha [B, K]   DEVICE, out, may be null
+ * Errors: ARG, TOO_LARGE, CUDA (text on stderr). */
+enum { TSDP_STATIC_MAX_B = 1024, TSDP_STATIC_MAX_T = 1024 };
+int tsdp_verify_commit_static(int device, int T, float beta0, float beta1, float clip, float* d_xt,
+                              const float* d_muhat, const float* d_eps, const int* h_t, int B, int K, int D,
+                              const tsdp_accept_t* accept, uint64_t seed, float draft_nfe, float* d_actions,
+                              int* h_t_new, int* h_jstar, float* d_logalpha, void* cuda_stream);
 
 #ifdef __cplusplus
 }

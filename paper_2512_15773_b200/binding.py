@@ -15,7 +15,7 @@ BASE, DRAFT = 0, 1
 EXPORTS = ["tsdp_init", "tsdp_destroy", "tsdp_strerror", "tsdp_last_error", "tsdp_weights_count",
            "tsdp_load_weights", "tsdp_set_schedule", "tsdp_sample_chunk", "tsdp_sample_chunk_host",
            "tsdp_round", "tsdp_denoise", "tsdp_gemm", "tsdp_gemm_timed", "tsdp_stats", "tsdp_reset_stats",
-           "tsdp_kernel_launches", "tsdp_profile", "tsdp_profile_read"]
+           "tsdp_kernel_launches", "tsdp_profile", "tsdp_profile_read", "tsdp_verify_commit_static"]
 PROF_FAMILIES = ["gemm", "layernorm", "attention", "embed_head", "round", "small_net", "gemm_draft"]
 
 
@@ -75,6 +75,8 @@ def load_library():
     lib.tsdp_denoise.argtypes = [vp, i, fp, fp, fp, i, fp, vp]
     lib.tsdp_gemm.argtypes = [vp, fp, fp, fp, i, i, i, i, fp, vp]
     lib.tsdp_gemm_timed.argtypes = [vp, fp, fp, fp, i, i, i, i, fp, i, C.POINTER(C.c_float), vp]
+    lib.tsdp_verify_commit_static.argtypes = [i, i, C.c_float, C.c_float, C.c_float, fp, fp, fp, fp, i, i, i,
+                                              C.POINTER(AcceptT), u64, C.c_float, fp, fp, fp, fp, vp]
     lib.tsdp_stats.argtypes = [vp, C.POINTER(StatsT)]
     lib.tsdp_reset_stats.argtypes = [vp]
     lib.tsdp_kernel_launches.argtypes = [vp]; lib.tsdp_kernel_launches.restype = u64
@@ -124,6 +126,18 @@ def _ptr(t):
     if isinstance(t, np.ndarray):
         return t.ctypes.data
     return t.data_ptr()
+
+
+def verify_commit_static(d_xt, d_muhat, d_eps, h_t, B, K, D, accept, seed, d_actions, h_t_new, h_jstar,
+                         d_logalpha=None, T=100, beta0=1e-4, beta1=0.02, clip=0.0, device=0, stream=0):
+    """tsdp_verify_commit_static: the fused acceptance / commit step on caller-owned buffers, for
+    callers that may not allocate device memory (no context, no workspace; see tsdp.h)."""
+    lib = load_library()
+    st = lib.tsdp_verify_commit_static(device, T, beta0, beta1, clip, _ptr(d_xt), _ptr(d_muhat), _ptr(d_eps),
+                                       _ptr(h_t), B, K, D, C.byref(accept), seed, 0.0, _ptr(d_actions),
+                                       _ptr(h_t_new), _ptr(h_jstar), _ptr(d_logalpha), stream)
+    if st != 0:
+        raise TsdpError(st, "tsdp_verify_commit_static", lib.tsdp_strerror(st).decode())
 
 
 class Sampler:

@@ -517,6 +517,7 @@ const char* tsdp_strerror(int st) {
     case TSDP_ERR_TIMEOUT: return "a bounded wait inside a kernel expired";
     case TSDP_ERR_NAN: return "non-finite value in weights";
     case TSDP_ERR_UNSUPPORTED: return "architecture not built";
+    case TSDP_ERR_TOO_LARGE: return "size exceeds the capacity of the built-in scratch array";
   }
   return "unknown status";
 }
@@ -1058,6 +1059,112 @@ int tsdp_profile_read(tsdp_ctx* c, double* ms, double* flop, uint64_t* launches)
     const int k = c->prof_cat[i];
     ms[k] += t; flop[k] += c->prof_flop[i]; launches[k] += 1;
   }
+  return TSDP_OK;
+}
+
+
+// ------------------------------------------------------------------------------------------------
+// Allocation-free verification tail.
+//
+// The working memory of this entry point is a file-scope device array: it is part of the library
+// image on every GPU that loads it and lives until the process exits.  Host code never passes the
+// array's name to a kernel (on the host that name is only a stand-in); its device address is looked
+// up once per device with cudaGetSymbolAddress and kept in g_static_addr.
+// ------------------------------------------------------------------------------------------------
+namespace {
+constexpr size_t ST_OFF_STATS = 0;                                            // DevStats
+constexpr size_t ST_OFF_TAB = 24832;                                          // 5 x TSDP_STATIC_MAX_T floats
+constexpr size_t ST_OFF_T = ST_OFF_TAB + 5 * TSDP_STATIC_MAX_T * 4;           // t[B]
+constexpr size_t ST_OFF_J = ST_OFF_T + TSDP_STATIC_MAX_B * 4;                 // j*[B]
+constexpr size_t ST_OFF_MISC = ST_OFF_J + TSDP_STATIC_MAX_B * 4;              // seed, round index, done count, round parameters
+constexpr size_t ST_BYTES = ST_OFF_MISC + 256;
+static_assert(sizeof(DevStats) <= ST_OFF_TAB, "statistics block overlaps the tables");
+static_assert(ST_OFF_TAB % 256 == 0 && ST_OFF_T % 256 == 0 && ST_OFF_J % 256 == 0 && ST_OFF_MISC % 256 == 0, "alignment");
+static_assert(ST_BYTES <= 64 * 1024, "static scratch is meant to stay small");
+}  // namespace
+
+static __device__ __align__(256) unsigned char g_static_scratch[ST_BYTES];
+
+namespace {
+constexpr int ST_MAX_DEVICES = 64;
+unsigned char* g_static_addr[ST_MAX_DEVICES] = {};
+}  // namespace
+
+int tsdp_verify_commit_static(int device, int T, float beta0, float beta1, float clip, float* d_xt,
+                              const float* d_muhat, const float* d_eps, const int* h_t, int B, int K, int D,
+                              const tsdp_accept_t* acc, uint64_t seed, float draft_nfe, float* d_actions,
+                              int* h_t_new, int* h_jstar, float* d_logalpha, void* stream) {
+  if (!d_xt || !d_eps || !h_t || !acc || !d_actions || !h_t_new || !h_jstar || (K > 0 && !d_muhat) || B < 1 || K < 0 ||
+      D < 1 || T < 1 || device < 0 || device >= ST_MAX_DEVICES || !(beta0 > 0.f) || !(beta1 < 1.f) || !accept_ok(acc))
+    return TSDP_ERR_ARG;
+  if (B > TSDP_STATIC_MAX_B || T > TSDP_STATIC_MAX_T || K > TSDP_MAX_K) {
+    fprintf(stderr, "tsdp_verify_commit_static: B = %d, T = %d, K = %d exceed the built-in capacity (B <= %d, T <= %d, K <= %d)\n",
+            B, T, K, (int)TSDP_STATIC_MAX_B, (int)TSDP_STATIC_MAX_T, (int)TSDP_MAX_K);
+    return TSDP_ERR_TOO_LARGE;
+  }
+  for (int b = 0; b < B; ++b)
+    if (h_t[b] < -1 || h_t[b] >= T) return TSDP_ERR_ARG;
+#define ST_TRY(expr)                                                                              \
+  do {                                                                                            \
+    cudaError_t e__ = (expr);                                                                     \
+    if (e__ != cudaSuccess) {                                                                     \
+      fprintf(stderr, "tsdp_verify_commit_static: %s: %s\n", #expr, cudaGetErrorString(e__));    \
+      return TSDP_ERR_CUDA;                                                                       \
+    }                                                                                             \
+  } while (0)
+  ST_TRY(cudaSetDevice(device));
+  if (!g_static_addr[device]) {   // first call on this device: resolve the array's device address
+    void* p = nullptr;
+    ST_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
+    g_static_addr[device] = reinterpret_cast<unsigned char*>(p);
+  }
+  unsigned char* base = g_static_addr[device];
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  DevStats* st = reinterpret_cast<DevStats*>(base + ST_OFF_STATS);
+  float* dtab = reinterpret_cast<float*>(base + ST_OFF_TAB);
+  int* dt = reinterpret_cast<int*>(base + ST_OFF_T);
+  int* dj = reinterpret_cast<int*>(base + ST_OFF_J);
+  uint64_t* dseed = reinterpret_cast<uint64_t*>(base + ST_OFF_MISC);
+  int* dround = reinterpret_cast<int*>(base + ST_OFF_MISC + 8);
+  int* ddone = reinterpret_cast<int*>(base + ST_OFF_MISC + 12);
+  RoundParams* drp = reinterpret_cast<RoundParams*>(base + ST_OFF_MISC + 16);
+
+  float tab[5 * TSDP_STATIC_MAX_T];
+  {
+    double abar = 1.0, abar_prev = 1.0;
+    for (int t = 0; t < T; ++t) {
+      const double beta = T > 1 ? beta0 + ((double)beta1 - beta0) * t / (T - 1) : beta0;
+      const double alpha = 1.0 - beta;
+      abar_prev = abar;
+      abar *= alpha;
+      tab[0 * T + t] = (float)std::sqrt(abar);
+      tab[1 * T + t] = (float)std::sqrt(1.0 - abar);
+      tab[2 * T + t] = (float)(std::sqrt(abar_prev) * beta / (1.0 - abar));
+      tab[3 * T + t] = (float)(std::sqrt(alpha) * (1.0 - abar_prev) / (1.0 - abar));
+      tab[4 * T + t] = (float)std::sqrt(beta * (1.0 - abar_prev) / (1.0 - abar));
+    }
+  }
+  RoundParams rp;
+  fill_round_params(&rp, K, *acc);
+  // the array keeps whatever the previous call left: counters and indices start from zero again
+  ST_TRY(cudaMemsetAsync(base + ST_OFF_STATS, 0, sizeof(DevStats), s));
+  ST_TRY(cudaMemsetAsync(base + ST_OFF_MISC, 0, 256, s));
+  ST_TRY(cudaMemcpyAsync(dtab, tab, sizeof(float) * 5 * T, cudaMemcpyHostToDevice, s));
+  ST_TRY(cudaMemcpyAsync(dt, h_t, sizeof(int) * B, cudaMemcpyHostToDevice, s));
+  ST_TRY(cudaMemcpyAsync(dseed, &seed, sizeof(seed), cudaMemcpyHostToDevice, s));
+  ST_TRY(cudaMemcpyAsync(drp, &rp, sizeof(rp), cudaMemcpyHostToDevice, s));
+  const DdpmTables S{dtab, dtab + T, dtab + 2 * T, dtab + 3 * T, dtab + 4 * T, T, clip};
+  const long long xs_b = (long long)(K + 1) * D, ms_b = (long long)(K > 0 ? K : 1) * D;
+  int warps = K < 1 ? 1 : K;
+  if (warps < 4) warps = 4;
+  if (warps > 16) warps = 16;
+  accept_kernel<<<B, warps * 32, 0, s>>>(S, d_xt, xs_b, d_muhat, ms_b, d_eps, xs_b, dt, K, D, dseed, drp, 1, dround,
+                                         d_actions, ddone, st, draft_nfe, d_logalpha, dj);
+  ST_TRY(cudaGetLastError());
+  ST_TRY(cudaMemcpyAsync(h_t_new, dt, sizeof(int) * B, cudaMemcpyDeviceToHost, s));
+  ST_TRY(cudaMemcpyAsync(h_jstar, dj, sizeof(int) * B, cudaMemcpyDeviceToHost, s));
+  ST_TRY(cudaStreamSynchronize(s));
+#undef ST_TRY
   return TSDP_OK;
 }
 

@@ -91,6 +91,16 @@ __global__ void memtok_kernel(const float* __restrict__ in, int Din, const float
 // ------------------------------------------------------------------------------------------------
 // LayerNorm over d (multiple of 128), one warp per row, fp32 in, T out.
 // ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void store4(float* o, float a, float b, float c, float e) {
+  *reinterpret_cast<float4*>(o) = make_float4(a, b, c, e);
+}
+__device__ __forceinline__ void store4(__nv_bfloat16* o, float a, float b, float c, float e) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, e);
+  uint2 p;
+  p.x = *reinterpret_cast<uint32_t*>(&lo); p.y = *reinterpret_cast<uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(o) = p;
+}
+
 template <typename T, int VEC>
 __global__ void ln_kernel(const float* __restrict__ h, const float* __restrict__ gam, const float* __restrict__ bet,
                           T* __restrict__ out, int M) {
@@ -118,11 +128,8 @@ __global__ void ln_kernel(const float* __restrict__ h, const float* __restrict__
     const int c = (j * 32 + lane) * 4;
     const float4 gg = reinterpret_cast<const float4*>(gam)[j * 32 + lane];
     const float4 bb = reinterpret_cast<const float4*>(bet)[j * 32 + lane];
-    T* o = out + (size_t)row * d + c;
-    o[0] = from_f<T>(v[j].x * rstd * gg.x + bb.x);
-    o[1] = from_f<T>(v[j].y * rstd * gg.y + bb.y);
-    o[2] = from_f<T>(v[j].z * rstd * gg.z + bb.z);
-    o[3] = from_f<T>(v[j].w * rstd * gg.w + bb.w);
+    store4(out + (size_t)row * d + c, v[j].x * rstd * gg.x + bb.x, v[j].y * rstd * gg.y + bb.y,
+           v[j].z * rstd * gg.z + bb.z, v[j].w * rstd * gg.w + bb.w);
   }
 }
 
@@ -223,6 +230,223 @@ __global__ void cross_attn_kernel(const T* __restrict__ q, T* __restrict__ out, 
       }
       out[(size_t)row * d + hd * dh + i] = from_f<T>(o * inv);
     }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Tensor-core causal self-attention for bf16 activations: one warp per (candidate, head, 16-query
+// tile).  S = Q K^T and O = P V run on mma.sync m16n8k16 (the sequence has at most 64 tokens, so
+// one warp-level tile covers it; a tcgen05 tile would be 8x too tall).  Operand fragments are read
+// straight from qkv [M, 3d]; the softmax lives in the accumulator registers; the output tile is
+// staged in shared memory so that every lane stores 16 contiguous bytes.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void mma_bf16_16816(float c[4], const uint32_t a[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 h2 = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&h2);
+}
+
+constexpr int SA_WARPS = 4;
+
+template <int DH>
+__global__ void __launch_bounds__(SA_WARPS * 32)
+self_attn_mma_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ out, int n_cand, int H, int d,
+                     int heads) {
+  constexpr int KS = DH / 16;        // k-steps of Q K^T
+  constexpr int NO = DH / 8;         // n-tiles of the output
+  constexpr int LDS = DH + 8;        // staging row pitch (elements); keeps 16-byte alignment
+  __shared__ __align__(16) __nv_bfloat16 stage[SA_WARPS][16 * LDS];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int QT = (H + 15) >> 4;
+  const int wg = blockIdx.x * SA_WARPS + warp;
+  if (wg >= n_cand * heads * QT) return;
+  const int qt = wg % QT, hd = (wg / QT) % heads, n = wg / (QT * heads);
+  const int g = lane >> 2, tg = lane & 3;
+  const size_t ld = (size_t)3 * d;
+  const __nv_bfloat16* base = qkv + (size_t)n * H * ld + (size_t)hd * DH;
+  const int r0 = qt * 16 + g, r1 = r0 + 8;
+  auto ld32 = [&](int row, int col) -> uint32_t {
+    return row < H ? __ldg(reinterpret_cast<const uint32_t*>(base + (size_t)row * ld + col)) : 0u;
+  };
+  uint32_t qa[KS][4];
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks) {
+    const int c = ks * 16 + 2 * tg;
+    qa[ks][0] = ld32(r0, c); qa[ks][1] = ld32(r1, c); qa[ks][2] = ld32(r0, c + 8); qa[ks][3] = ld32(r1, c + 8);
+  }
+  // keys 0 .. 16 (qt+1) - 1 are the only ones a causal query of this tile can see
+  const int nkt = 2 * (qt + 1);
+  float s[8][4];
+#pragma unroll
+  for (int nt = 0; nt < 8; ++nt) {
+    s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+    if (nt < nkt) {
+      const int key = nt * 8 + g;
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+        const int c = d + ks * 16 + 2 * tg;
+        mma_bf16_16816(s[nt], qa[ks], ld32(key, c), ld32(key, c + 8));
+      }
+    }
+  }
+  const float scale = rsqrtf((float)DH);
+  float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+  for (int nt = 0; nt < 8; ++nt) {
+    if (nt < nkt) {
+      const int col = nt * 8 + 2 * tg;
+      s[nt][0] = (col <= r0 && col < H) ? s[nt][0] * scale : -INFINITY;
+      s[nt][1] = (col + 1 <= r0 && col + 1 < H) ? s[nt][1] * scale : -INFINITY;
+      s[nt][2] = (col <= r1 && col < H) ? s[nt][2] * scale : -INFINITY;
+      s[nt][3] = (col + 1 <= r1 && col + 1 < H) ? s[nt][3] * scale : -INFINITY;
+      m0 = fmaxf(m0, fmaxf(s[nt][0], s[nt][1]));
+      m1 = fmaxf(m1, fmaxf(s[nt][2], s[nt][3]));
+    }
+  }
+  m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 1)); m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 2));
+  m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 1)); m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 2));
+  // rows beyond H have no visible key: keep the arithmetic finite, their output is never stored
+  if (m0 == -INFINITY) m0 = 0.f;
+  if (m1 == -INFINITY) m1 = 0.f;
+  float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+  for (int nt = 0; nt < 8; ++nt) {
+    if (nt < nkt) {
+      s[nt][0] = __expf(s[nt][0] - m0); s[nt][1] = __expf(s[nt][1] - m0);
+      s[nt][2] = __expf(s[nt][2] - m1); s[nt][3] = __expf(s[nt][3] - m1);
+      l0 += s[nt][0] + s[nt][1]; l1 += s[nt][2] + s[nt][3];
+    }
+  }
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+  l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+  const float inv0 = l0 > 0.f ? 1.0f / l0 : 0.f, inv1 = l1 > 0.f ? 1.0f / l1 : 0.f;
+  // O = P V; the accumulator layout of two adjacent key tiles is the A-operand layout of one k-step
+  float o[NO][4];
+#pragma unroll
+  for (int no = 0; no < NO; ++no) o[no][0] = o[no][1] = o[no][2] = o[no][3] = 0.f;
+  const __nv_bfloat16* vbase = base + 2 * d;
+  const unsigned short* vraw = reinterpret_cast<const unsigned short*>(vbase);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    if (j <= qt) {
+      uint32_t pa[4];
+      pa[0] = pack_bf16(s[2 * j][0], s[2 * j][1]); pa[1] = pack_bf16(s[2 * j][2], s[2 * j][3]);
+      pa[2] = pack_bf16(s[2 * j + 1][0], s[2 * j + 1][1]); pa[3] = pack_bf16(s[2 * j + 1][2], s[2 * j + 1][3]);
+      const int k0 = 16 * j + 2 * tg;
+#pragma unroll
+      for (int no = 0; no < NO; ++no) {
+        const int col = no * 8 + g;
+        auto v16 = [&](int key) -> uint32_t {
+          return key < H ? (uint32_t)__ldg(vraw + (size_t)key * ld + col) : 0u;
+        };
+        const uint32_t b0 = v16(k0) | (v16(k0 + 1) << 16);
+        const uint32_t b1 = v16(k0 + 8) | (v16(k0 + 9) << 16);
+        mma_bf16_16816(o[no], pa, b0, b1);
+      }
+    }
+  }
+  __nv_bfloat16* st = stage[warp];
+#pragma unroll
+  for (int no = 0; no < NO; ++no) {
+    const int col = no * 8 + 2 * tg;
+    *reinterpret_cast<uint32_t*>(st + g * LDS + col) = pack_bf16(o[no][0] * inv0, o[no][1] * inv0);
+    *reinterpret_cast<uint32_t*>(st + (g + 8) * LDS + col) = pack_bf16(o[no][2] * inv1, o[no][3] * inv1);
+  }
+  __syncwarp();
+  constexpr int VPR = DH / 8;        // 16-byte vectors per row
+  for (int i = lane; i < 16 * VPR; i += 32) {
+    const int r = i / VPR, v = i % VPR;
+    const int row = qt * 16 + r;
+    if (row < H)
+      *reinterpret_cast<uint4*>(out + ((size_t)n * H + row) * d + (size_t)hd * DH + v * 8) =
+          *reinterpret_cast<const uint4*>(st + r * LDS + v * 8);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Cross-attention for bf16 activations with at most 4 memory tokens: DH/8 lanes own one (candidate,
+// head); they load that head's keys and values once into registers (they are the same for all H
+// query rows of the candidate) and then stream the H query rows, 16 bytes per lane per row.
+// ------------------------------------------------------------------------------------------------
+constexpr int CA_MAXNK = 4;
+
+template <int DH>
+__global__ void __launch_bounds__(256)
+cross_attn_group_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out,
+                        const float* __restrict__ kv_time, const float* __restrict__ kv_obs, CandMap cm, int n_cand,
+                        int H, int d, int heads, int To, int layer, int L, int Tsteps) {
+  constexpr int LG = DH / 8;
+  const int gid_raw = (blockIdx.x * blockDim.x + threadIdx.x) / LG;
+  const int sub = threadIdx.x % LG;
+  const bool live = gid_raw < n_cand * heads;
+  const int gid = live ? gid_raw : n_cand * heads - 1;
+  const int n = gid / heads, hd = gid % heads;
+  const int b = n / cm.C, c = n % cm.C;
+  int tau = cm.t[b] - cm.koff - c;
+  tau = max(0, min(Tsteps - 1, tau));
+  const size_t ldkv = (size_t)L * 2 * d;
+  const int NK = 1 + To;
+  float kreg[CA_MAXNK][8], vreg[CA_MAXNK][8];
+#pragma unroll
+  for (int kx = 0; kx < CA_MAXNK; ++kx) {
+    if (kx < NK) {
+      const float* kp = (kx == 0 ? kv_time + (size_t)tau * ldkv : kv_obs + ((size_t)b * To + (kx - 1)) * ldkv) +
+                        (size_t)layer * 2 * d + hd * DH + sub * 8;
+      const float4 k0 = __ldg(reinterpret_cast<const float4*>(kp)), k1 = __ldg(reinterpret_cast<const float4*>(kp) + 1);
+      const float4 v0 = __ldg(reinterpret_cast<const float4*>(kp + d)), v1 = __ldg(reinterpret_cast<const float4*>(kp + d) + 1);
+      kreg[kx][0] = k0.x; kreg[kx][1] = k0.y; kreg[kx][2] = k0.z; kreg[kx][3] = k0.w;
+      kreg[kx][4] = k1.x; kreg[kx][5] = k1.y; kreg[kx][6] = k1.z; kreg[kx][7] = k1.w;
+      vreg[kx][0] = v0.x; vreg[kx][1] = v0.y; vreg[kx][2] = v0.z; vreg[kx][3] = v0.w;
+      vreg[kx][4] = v1.x; vreg[kx][5] = v1.y; vreg[kx][6] = v1.z; vreg[kx][7] = v1.w;
+    }
+  }
+  const float scale = rsqrtf((float)DH);
+  const __nv_bfloat16* qp = q + (size_t)n * H * d + (size_t)hd * DH + sub * 8;
+  __nv_bfloat16* op = out + (size_t)n * H * d + (size_t)hd * DH + sub * 8;
+#pragma unroll 2
+  for (int r = 0; r < H; ++r) {
+    const uint4 qv = *reinterpret_cast<const uint4*>(qp + (size_t)r * d);
+    const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&qv);
+    float qf[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { const float2 f = __bfloat1622float2(q2[i]); qf[2 * i] = f.x; qf[2 * i + 1] = f.y; }
+    float sc[CA_MAXNK];
+    float m = -INFINITY;
+#pragma unroll
+    for (int kx = 0; kx < CA_MAXNK; ++kx) {
+      if (kx < NK) {
+        float a = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) a += qf[i] * kreg[kx][i];
+#pragma unroll
+        for (int o = LG / 2; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        sc[kx] = a * scale;
+        m = fmaxf(m, sc[kx]);
+      }
+    }
+    float l = 0.f;
+#pragma unroll
+    for (int kx = 0; kx < CA_MAXNK; ++kx)
+      if (kx < NK) { sc[kx] = __expf(sc[kx] - m); l += sc[kx]; }
+    const float inv = 1.0f / l;
+    float o8[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) o8[i] = 0.f;
+#pragma unroll
+    for (int kx = 0; kx < CA_MAXNK; ++kx)
+      if (kx < NK) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o8[i] += sc[kx] * vreg[kx][i];
+      }
+    uint4 ov;
+    ov.x = pack_bf16(o8[0] * inv, o8[1] * inv); ov.y = pack_bf16(o8[2] * inv, o8[3] * inv);
+    ov.z = pack_bf16(o8[4] * inv, o8[5] * inv); ov.w = pack_bf16(o8[6] * inv, o8[7] * inv);
+    if (live) *reinterpret_cast<uint4*>(op + (size_t)r * d) = ov;
   }
 }
 

@@ -9,6 +9,7 @@
 #include <map>
 #include <string>
 #include <tuple>
+#include <type_traits>
 #include <vector>
 
 #include "../../include/tsdp.h"
@@ -304,6 +305,60 @@ int head_launch(tsdp_ctx* c, const Net& n, const CandMap& cm, int M, cudaStream_
   return TSDP_OK;
 }
 
+// Causal self-attention: tensor-core kernel for bf16 activations, the scalar kernel in check mode.
+template <typename T>
+int self_attn_launch(tsdp_ctx* c, const T* qkv, T* out, int n_cand, int H, int d, int heads, cudaStream_t s) {
+  const int dh = d / heads;
+  prof_begin(c, s, 2, 0.0);
+  if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+    const int QT = (H + 15) / 16;
+    const int grid = (n_cand * heads * QT + SA_WARPS - 1) / SA_WARPS;
+    switch (dh) {
+      case 32: self_attn_mma_kernel<32><<<grid, SA_WARPS * 32, 0, s>>>(qkv, out, n_cand, H, d, heads); break;
+      case 64: self_attn_mma_kernel<64><<<grid, SA_WARPS * 32, 0, s>>>(qkv, out, n_cand, H, d, heads); break;
+      case 96: self_attn_mma_kernel<96><<<grid, SA_WARPS * 32, 0, s>>>(qkv, out, n_cand, H, d, heads); break;
+      default: self_attn_mma_kernel<128><<<grid, SA_WARPS * 32, 0, s>>>(qkv, out, n_cand, H, d, heads); break;
+    }
+  } else {
+    const size_t per_warp = (size_t)(H * dh + 2 * H * (dh + 1)) * sizeof(float);
+    int wpb = (int)((200 * 1024) / per_warp);      // the opt-in shared-memory limit set at init
+    wpb = wpb > 4 ? 4 : (wpb < 1 ? 1 : wpb);
+    const size_t smem = (size_t)wpb * per_warp;
+    self_attn_kernel<T><<<(n_cand * heads + wpb - 1) / wpb, wpb * 32, smem, s>>>(qkv, out, n_cand, H, d, heads);
+  }
+  prof_end(c, s);
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  return TSDP_OK;
+}
+
+// Cross-attention to [time token | obs tokens]: register-resident keys/values when there are at most
+// CA_MAXNK memory tokens and the head width is a power of two, the one-warp-per-row kernel otherwise.
+template <typename T>
+int cross_attn_launch(tsdp_ctx* c, const Net& n, const T* q2, T* out, const CandMap& cm, int n_cand, int layer,
+                      cudaStream_t s) {
+  const int H = c->cfg.H, d = n.cfg.d, heads = n.cfg.heads, L = n.cfg.layers, To = c->cfg.obs_tokens;
+  const int dh = d / heads, M = n_cand * H;
+  prof_begin(c, s, 2, 0.0);
+  bool done = false;
+  if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+    if (1 + To <= CA_MAXNK && (dh == 32 || dh == 64 || dh == 128)) {
+      const long long threads = (long long)n_cand * heads * (dh / 8);
+      const int grid = (int)((threads + 255) / 256);
+#define CA_CASE(DH) cross_attn_group_kernel<DH><<<grid, 256, 0, s>>>(q2, out, n.kv_time, n.kv_obs, cm, n_cand, H, d, heads, To, layer, L, c->cfg.T)
+      if (dh == 32) CA_CASE(32); else if (dh == 64) CA_CASE(64); else CA_CASE(128);
+#undef CA_CASE
+      done = true;
+    }
+  }
+  if (!done)
+    cross_attn_kernel<T><<<(M + 7) / 8, 256, 0, s>>>(q2, out, n.kv_time, n.kv_obs, cm, M, H, d, heads, To, layer, L, c->cfg.T);
+  prof_end(c, s);
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  return TSDP_OK;
+}
+
 template <typename T>
 int xfmr_forward_t(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStream_t s) {
   const int H = c->cfg.H, A = c->cfg.A, d = n.cfg.d, heads = n.cfg.heads, L = n.cfg.layers;
@@ -319,27 +374,16 @@ int xfmr_forward_t(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStrea
   prof_end(c, s);
   c->launches_per_round_tmp++;
   CU_TRY(c, cudaGetLastError());
-  const int sa_wpb = 4;
-  const size_t sa_smem = (size_t)sa_wpb * (H * dh + 2 * H * (dh + 1)) * sizeof(float);
   const int out_epi = (c->cfg.precision == 0) ? EPI_F32 : EPI_STORE;
   for (int l = 0; l < L; ++l) {
     const XfmrLayer& w = n.L[l];
     if ((r = ln_launch<T>(c, c->h, w.ln1_g, w.ln1_b, a, M, d, s))) return r;
     if ((r = gemm(c, a, w.Wqkv, w.bqkv, M, 3 * d, d, out_epi, qkv, 3 * d, s))) return r;
-    prof_begin(c, s, 2, 0.0);
-    self_attn_kernel<T><<<(n_cand * heads + sa_wpb - 1) / sa_wpb, sa_wpb * 32, sa_smem, s>>>(qkv, a, n_cand, H, d, heads);
-    prof_end(c, s);
-    c->launches_per_round_tmp++;
-    CU_TRY(c, cudaGetLastError());
+    if ((r = self_attn_launch<T>(c, qkv, a, n_cand, H, d, heads, s))) return r;
     if ((r = gemm(c, a, w.Wo, w.bo, M, d, d, EPI_RESID, c->h, d, s))) return r;
     if ((r = ln_launch<T>(c, c->h, w.ln2_g, w.ln2_b, a, M, d, s))) return r;
     if ((r = gemm(c, a, w.Wq2, w.bq2, M, d, d, out_epi, q2, d, s))) return r;
-    prof_begin(c, s, 2, 0.0);
-    cross_attn_kernel<T><<<(M + 7) / 8, 256, 0, s>>>(q2, a, n.kv_time, n.kv_obs, cm, M, H, d, heads, c->cfg.obs_tokens, l, L,
-                                                      c->cfg.T);
-    prof_end(c, s);
-    c->launches_per_round_tmp++;
-    CU_TRY(c, cudaGetLastError());
+    if ((r = cross_attn_launch<T>(c, n, q2, a, cm, n_cand, l, s))) return r;
     if ((r = gemm(c, a, w.Wo2, w.bo2, M, d, d, EPI_RESID, c->h, d, s))) return r;
     if ((r = ln_launch<T>(c, c->h, w.ln3_g, w.ln3_b, a, M, d, s))) return r;
     if ((r = gemm(c, a, w.W1, w.b1, M, 4 * d, d, EPI_GELU, f, 4 * d, s))) return r;

@@ -69,12 +69,17 @@ def test_small_denoisers(arch):
 
 
 @pytest.mark.parametrize("precision,tol", [(0, 1e-4), (1, 2e-2)])
-@pytest.mark.parametrize("shape", ["small", "pusht"])
+@pytest.mark.parametrize("shape", ["small", "pusht", "long"])
 def test_transformer_denoiser(precision, tol, shape):
     rng = np.random.default_rng(2)
     if shape == "small":
         wl = hp.small_xfmr_workload(precision, d=128, heads=4, layers=2, dd=256, dlayers=1, H=7, A=3, To=3, Do=5,
                                     gamma=1.0)
+    elif shape == "long":
+        # 50 tokens: four 16-query tiles with a ragged last one; head widths 128 and 96 (the latter takes the one-warp-per-row cross-attention)
+        wl = hp.small_xfmr_workload(precision, d=256, heads=2, layers=2, dd=384, dlayers=1, H=50, A=3, To=3, Do=6,
+                                    gamma=1.0)
+        wl["draft"]["heads"] = 4
     else:
         wl = dict(inputs.WORKLOADS["pusht_xfmr"], precision=precision, gamma=1.0)
     N = 19      # 19*H token rows: ragged against the 128-row tiles

@@ -11,8 +11,12 @@
 //               inputs) into one of two TMEM accumulator buffers; tcgen05.commit releases smem
 //               stages and publishes finished accumulators.
 //   warps 2..9  epilogue: tcgen05.ld the accumulator (each warp owns one 32-lane TMEM quadrant and
-//               half of the columns), fuse bias / GELU / residual, store.  The second accumulator
-//               buffer lets the next tile's MMAs overlap this tile's epilogue.
+//               half of the columns), fuse bias / GELU, and hand the tile back through shared
+//               memory: 128-row x 128-byte chunks in the 128-byte-swizzled layout, written to global
+//               memory by TMA (cp.async.bulk.tensor store; for the fp32 residual stream the TMA
+//               reduce-add, so the residual is never read into the SM).  Tiles narrower than 128
+//               columns store straight from registers.  The second accumulator buffer lets the
+//               next tile's MMAs overlap this tile's epilogue.
 // Every mbarrier wait is bounded: on expiry the kernel records TSDP_ERR_TIMEOUT in `status`, drains,
 // frees its TMEM and returns.  No cluster launch, no multicast.
 #pragma once
@@ -31,7 +35,11 @@ constexpr long long GEMM_WAIT_CYCLES = 2000000000ll;   // about one second of SM
 
 __host__ __device__ constexpr int gemm_stages(int BN) { return BN >= 256 ? 4 : (BN >= 128 ? 6 : 8); }
 __host__ __device__ constexpr int gemm_stage_bytes(int BN) { return GEMM_BM * GEMM_BK * 2 + BN * GEMM_BK * 2; }
-__host__ __device__ constexpr int gemm_smem_bytes(int BN) { return gemm_stages(BN) * gemm_stage_bytes(BN) + 1024 + 256; }
+constexpr int GEMM_STAGING_BYTES = 2 * 128 * 128;   // one 128-row x 128-byte chunk per column half
+__host__ __device__ constexpr bool gemm_tma_epilogue(int BN) { return BN >= 128; }
+__host__ __device__ constexpr int gemm_smem_bytes(int BN) {
+  return gemm_stages(BN) * gemm_stage_bytes(BN) + (gemm_tma_epilogue(BN) ? GEMM_STAGING_BYTES : 0) + 1024 + 256;
+}
 
 namespace ptx {
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -101,6 +109,50 @@ __device__ __forceinline__ void tmem_ld16(uint32_t addr, uint32_t v[16]) {
         "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
       : "r"(addr) : "memory");
 }
+__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t v[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(addr) : "memory");
+}
+// TMA store / reduce-add of one shared-memory box into a tiled global tensor (bulk async-group).
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(x), "r"(y), "r"(src) : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(x), "r"(y), "r"(src) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+// Barrier over `nthreads` threads that also ANDs a predicate across them.
+__device__ __forceinline__ bool named_bar_and(int id, int nthreads, bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.and.pred p, %2, %3, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r) : "r"(pred ? 1u : 0u), "r"(id), "r"(nthreads) : "memory");
+  return r != 0;
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ float tanh_fast(float x) {
+  float y;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 }  // namespace ptx
 
@@ -119,6 +171,11 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
 // Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M = 128, N = BN.
 __host__ __device__ constexpr uint32_t umma_idesc_bf16(int BN) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(GEMM_BM >> 4) << 24);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 h2 = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&h2);
 }
 
 struct GemmArgs {
@@ -165,7 +222,8 @@ __device__ __forceinline__ void epilogue_store16(const GemmArgs& g, int row, int
 
 template <int BN, int EPI>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmArgs g) {
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                    const __grid_constant__ CUtensorMap tmC, GemmArgs g) {
   constexpr int STAGES = gemm_stages(BN);
   constexpr int A_BYTES = GEMM_BM * GEMM_BK * 2;
   constexpr int STAGE_BYTES = gemm_stage_bytes(BN);
@@ -175,7 +233,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bar0 = base + STAGES * STAGE_BYTES;       // full[STAGES], empty[STAGES], tfull[2], tempty[2]
+  constexpr bool TMA_EPI = gemm_tma_epilogue(BN);
+  const uint32_t staging = base + STAGES * STAGE_BYTES;    // 1024-byte aligned: every stage is a multiple of 1 KB
+  const uint32_t bar0 = staging + (TMA_EPI ? GEMM_STAGING_BYTES : 0);   // full[STAGES], empty[STAGES], tfull[2], tempty[2]
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
   auto tfull_bar = [&](int s) { return bar0 + 8u * (2 * STAGES + s); };
@@ -250,23 +310,105 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const int half = ew >> 2;                // which half of the tile's columns
     constexpr int COLS = BN / 2;
     int it = 0;
-    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
-      const int tm = tile / tiles_n, tn = tile % tiles_n;
-      const int as = it & 1; const uint32_t aphase = (it >> 1) & 1;
-      if (!ptx::mbar_wait_warp(tfull_bar(as), aphase)) { ok = false; break; }
-      ptx::tc_fence_after();
-      const int row = tm * GEMM_BM + quad * 32 + lane;
-      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * BN + half * COLS);
+    if constexpr (TMA_EPI) {
+      // Output element size, columns per 128-byte chunk, chunks per half tile.
+      constexpr int ESZ = (EPI == EPI_STORE || EPI == EPI_GELU) ? 2 : 4;
+      constexpr int CW = 128 / ESZ;
+      constexpr int NCH = COLS / CW;
+      const uint32_t stg = staging + (uint32_t)half * (GEMM_STAGING_BYTES / 2);
+      const int r = quad * 32 + lane;        // row of the tile this thread owns
+      const uint32_t row_addr = stg + (uint32_t)r * 128u;
+      const uint32_t sw = (uint32_t)(r & 7);
+      const bool issuer = (quad == 0 && lane == 0);
+      const int bar_id = 1 + half;
+      for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
+        const int tm = tile / tiles_n, tn = tile % tiles_n;
+        const int as = it & 1; const uint32_t aphase = (it >> 1) & 1;
+        // all four warps of this half agree on the outcome, so none is left alone at a named barrier
+        ok = ptx::named_bar_and(bar_id, 128, ptx::mbar_wait_warp(tfull_bar(as), aphase));
+        if (!ok) break;
+        ptx::tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * BN + half * COLS);
 #pragma unroll 1
-      for (int c = 0; c < COLS; c += 16) {
-        uint32_t v[16];
-        ptx::tmem_ld16(taddr + (uint32_t)c, v);
-        ptx::tmem_ld_wait();
-        if (row < g.M) epilogue_store16<EPI>(g, row, tn * BN + half * COLS + c, v);
+        for (int ch = 0; ch < NCH; ++ch) {
+#pragma unroll
+          for (int part = 0; part < CW / 32; ++part) {
+            uint32_t v[32];
+            const int col_t = ch * CW + part * 32;                 // column inside this half
+            ptx::tmem_ld32(taddr + (uint32_t)col_t, v);
+            ptx::tmem_ld_wait();
+            if (ch == NCH - 1 && part == CW / 32 - 1) {            // accumulator fully read: hand it back
+              ptx::tc_fence_before();
+              __syncwarp();
+              if (lane == 0) ptx::mbar_arrive(tempty_bar(as));
+            }
+            const int col = tn * BN + half * COLS + col_t;
+            float f[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]);
+            if (g.bias) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const float4 bb = __ldg(reinterpret_cast<const float4*>(g.bias + col) + i);
+                f[4 * i] += bb.x; f[4 * i + 1] += bb.y; f[4 * i + 2] += bb.z; f[4 * i + 3] += bb.w;
+              }
+            }
+            if (EPI == EPI_GELU) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) {
+                const float x = f[i];
+                f[i] = 0.5f * x * (1.0f + ptx::tanh_fast(0.7978845608028654f * (x + 0.044715f * x * x * x)));
+              }
+            }
+            if (part == 0) {   // the previous chunk's TMA store must have drained the staging buffer
+              if (issuer) ptx::bulk_wait_read0();
+              ptx::named_bar_sync(bar_id, 128);
+            }
+            if (ESZ == 2) {
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const uint32_t c16 = (uint32_t)(part * 4 + j);
+                ptx::st_shared_v4(row_addr + ((c16 ^ sw) << 4),
+                                  pack_bf16x2(f[8 * j], f[8 * j + 1]), pack_bf16x2(f[8 * j + 2], f[8 * j + 3]),
+                                  pack_bf16x2(f[8 * j + 4], f[8 * j + 5]), pack_bf16x2(f[8 * j + 6], f[8 * j + 7]));
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                ptx::st_shared_v4(row_addr + (((uint32_t)j ^ sw) << 4), __float_as_uint(f[4 * j]),
+                                  __float_as_uint(f[4 * j + 1]), __float_as_uint(f[4 * j + 2]), __float_as_uint(f[4 * j + 3]));
+            }
+          }
+          ptx::fence_async_smem();
+          ptx::named_bar_sync(bar_id, 128);
+          if (issuer) {
+            const int x = tn * BN + half * COLS + ch * CW, y = tm * GEMM_BM;
+            if (EPI == EPI_RESID) ptx::tma_reduce_add_2d(&tmC, x, y, stg);
+            else ptx::tma_store_2d(&tmC, x, y, stg);
+            ptx::bulk_commit();
+          }
+        }
       }
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(tempty_bar(as));
+      if (issuer) ptx::bulk_wait_read0();
+    } else {
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
+        const int tm = tile / tiles_n, tn = tile % tiles_n;
+        const int as = it & 1; const uint32_t aphase = (it >> 1) & 1;
+        if (!ptx::mbar_wait_warp(tfull_bar(as), aphase)) { ok = false; break; }
+        ptx::tc_fence_after();
+        const int row = tm * GEMM_BM + quad * 32 + lane;
+        const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * BN + half * COLS);
+#pragma unroll 1
+        for (int c = 0; c < COLS; c += 16) {
+          uint32_t v[16];
+          ptx::tmem_ld16(taddr + (uint32_t)c, v);
+          ptx::tmem_ld_wait();
+          if (row < g.M) epilogue_store16<EPI>(g, row, tn * BN + half * COLS + c, v);
+        }
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(tempty_bar(as));
+      }
     }
   }
   if (!ok) {

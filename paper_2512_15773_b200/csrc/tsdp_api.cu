@@ -74,7 +74,7 @@ struct tsdp_ctx {
   std::vector<tsdp_accept_t> sched_acc;
   // graphs and tensor maps
   std::map<std::tuple<int, int>, cudaGraphExec_t> graphs;
-  std::map<std::tuple<const void*, int, int, int>, CUtensorMap> maps;
+  std::map<std::tuple<const void*, int, int, int, int, int, int>, CUtensorMap> maps;
   EncodeTiledFn encode = nullptr;
   cudaStream_t cap_stream = nullptr;
   uint64_t rounds = 0, launches = 0;
@@ -155,18 +155,21 @@ size_t weights_count(const tsdp_config_t& cfg, const tsdp_net_t& n) {
 }
 
 // ------------------------------------------------------------------------------------------ GEMM
-int get_map(tsdp_ctx* c, const void* ptr, int rows, int cols, int box_rows, CUtensorMap* out) {
-  auto key = std::make_tuple(ptr, rows, cols, box_rows);
+// Tiled 2-D tensor map with the 128-byte swizzle over a row-major [rows, cols] matrix whose rows are
+// `ld` elements apart; esz = 2 (bf16) or 4 (fp32).  The box is box_cols x box_rows (box_cols * esz = 128).
+int get_map(tsdp_ctx* c, const void* ptr, int esz, int rows, int cols, int ld, int box_cols, int box_rows,
+            CUtensorMap* out) {
+  auto key = std::make_tuple(ptr, esz, rows, cols, ld, box_cols, box_rows);
   auto it = c->maps.find(key);
   if (it != c->maps.end()) { *out = it->second; return TSDP_OK; }
   CUtensorMap m;
   cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  cuuint64_t gstr[1] = {(cuuint64_t)cols * 2};
-  cuuint32_t box[2] = {(cuuint32_t)GEMM_BK, (cuuint32_t)box_rows};
+  cuuint64_t gstr[1] = {(cuuint64_t)ld * esz};
+  cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = c->encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstr, box, estr,
-                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r = c->encode(&m, esz == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                         const_cast<void*>(ptr), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     c->last_error = "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r);
     return TSDP_ERR_CUDA;
@@ -177,11 +180,12 @@ int get_map(tsdp_ctx* c, const void* ptr, int rows, int cols, int box_rows, CUte
 }
 
 template <int BN, int EPI>
-int launch_tc(tsdp_ctx* c, const CUtensorMap& ma, const CUtensorMap& mb, const GemmArgs& g, cudaStream_t s) {
+int launch_tc(tsdp_ctx* c, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const GemmArgs& g,
+              cudaStream_t s) {
   const int tiles = ((g.M + GEMM_BM - 1) / GEMM_BM) * (g.N / BN);
   const int grid = tiles < c->num_sms ? tiles : c->num_sms;
   prof_begin(c, s, c->prof_gemm_cat, 2.0 * g.M * g.N * g.K);
-  gemm_tcgen05_kernel<BN, EPI><<<grid, GEMM_THREADS, gemm_smem_bytes(BN), s>>>(ma, mb, g);
+  gemm_tcgen05_kernel<BN, EPI><<<grid, GEMM_THREADS, gemm_smem_bytes(BN), s>>>(ma, mb, mc, g);
   prof_end(c, s);
   c->launches_per_round_tmp++;
   CU_TRY(c, cudaGetLastError());
@@ -189,12 +193,13 @@ int launch_tc(tsdp_ctx* c, const CUtensorMap& ma, const CUtensorMap& mb, const G
 }
 
 template <int BN>
-int launch_tc_epi(tsdp_ctx* c, const CUtensorMap& ma, const CUtensorMap& mb, const GemmArgs& g, int epi, cudaStream_t s) {
+int launch_tc_epi(tsdp_ctx* c, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const GemmArgs& g,
+                  int epi, cudaStream_t s) {
   switch (epi) {
-    case EPI_STORE: return launch_tc<BN, EPI_STORE>(c, ma, mb, g, s);
-    case EPI_GELU: return launch_tc<BN, EPI_GELU>(c, ma, mb, g, s);
-    case EPI_RESID: return launch_tc<BN, EPI_RESID>(c, ma, mb, g, s);
-    default: return launch_tc<BN, EPI_F32>(c, ma, mb, g, s);
+    case EPI_STORE: return launch_tc<BN, EPI_STORE>(c, ma, mb, mc, g, s);
+    case EPI_GELU: return launch_tc<BN, EPI_GELU>(c, ma, mb, mc, g, s);
+    case EPI_RESID: return launch_tc<BN, EPI_RESID>(c, ma, mb, mc, g, s);
+    default: return launch_tc<BN, EPI_F32>(c, ma, mb, mc, g, s);
   }
 }
 
@@ -248,15 +253,24 @@ int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, in
     return TSDP_ERR_ARG;
   }
   const int BN = pick_bn(M, N, c->num_sms);
-  CUtensorMap ma, mb;
+  CUtensorMap ma, mb, mc;
   int r;
-  if ((r = get_map(c, A, M, K, GEMM_BM, &ma)) != TSDP_OK) return r;
-  if ((r = get_map(c, W, N, K, BN, &mb)) != TSDP_OK) return r;
+  if ((r = get_map(c, A, 2, M, K, K, GEMM_BK, GEMM_BM, &ma)) != TSDP_OK) return r;
+  if ((r = get_map(c, W, 2, N, K, K, GEMM_BK, BN, &mb)) != TSDP_OK) return r;
+  mc = ma;
+  if (gemm_tma_epilogue(BN)) {   // the epilogue hands 128-row x 128-byte chunks to TMA
+    const int esz = (epi == EPI_STORE || epi == EPI_GELU) ? 2 : 4;
+    if (ldo % (16 / esz) != 0 || (reinterpret_cast<uintptr_t>(out) & 15) != 0) {
+      c->last_error = "GEMM output must be 16-byte aligned with a row pitch that is a multiple of 16 bytes";
+      return TSDP_ERR_ARG;
+    }
+    if ((r = get_map(c, out, esz, M, N, ldo, 128 / esz, GEMM_BM, &mc)) != TSDP_OK) return r;
+  }
   switch (BN) {
-    case 256: return launch_tc_epi<256>(c, ma, mb, g, epi, s);
-    case 128: return launch_tc_epi<128>(c, ma, mb, g, epi, s);
-    case 64: return launch_tc_epi<64>(c, ma, mb, g, epi, s);
-    default: return launch_tc_epi<32>(c, ma, mb, g, epi, s);
+    case 256: return launch_tc_epi<256>(c, ma, mb, mc, g, epi, s);
+    case 128: return launch_tc_epi<128>(c, ma, mb, mc, g, epi, s);
+    case 64: return launch_tc_epi<64>(c, ma, mb, mc, g, epi, s);
+    default: return launch_tc_epi<32>(c, ma, mb, mc, g, epi, s);
   }
 }
 

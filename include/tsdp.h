@@ -66,6 +66,12 @@ typedef struct {
   float draft_nfe;         /* NFE cost of one drafter call; 0 => draft.layers/base.layers
                               (the paper's 1/8 rule, Sec. 4 "Evaluation Metrics")               */
   int use_graph;           /* 1: replay each round from a captured CUDA graph                  */
+  int drafter;             /* how the K draft steps run.  0: chosen from the batch size; 1: layer
+                              by layer (batched tensor-core kernels, one drafter forward per step);
+                              2: one persistent thread-block-cluster kernel per round with the
+                              drafter's weights resident in shared memory (transformer drafter,
+                              precision 1, d = 128 or 256, H <= 16, obs_tokens <= 3, weights of a
+                              1/8 slice fitting one SM; otherwise tsdp_init returns UNSUPPORTED)  */
 } tsdp_config_t;
 
 /* Speculative parameters of a round -- the scheduler's action space (Sec. 3.3).
@@ -172,10 +178,10 @@ uint64_t tsdp_kernel_launches(const tsdp_ctx* ctx);
  * are issued as plain launches (no graph) with an event pair around each launch on the caller's
  * stream.  Families: 0 GEMMs of the base model (tcgen05 or check-mode), 1 LayerNorm, 2 attention,
  * 3 embed/head/memory tokens, 4 round kernels (draft step, accept), 5 MLP / Gaussian denoiser, 6 GEMMs
- * of the drafter.  tsdp_profile(ctx, 0|1)
+ * of the drafter, 7 the persistent cluster drafter.  tsdp_profile(ctx, 0|1)
  * clears the record.  tsdp_profile_read fills three arrays of TSDP_PROF_FAMILIES entries: summed
  * milliseconds, summed algorithmic flops (2*M*N*K per GEMM launch, 0 elsewhere) and launch counts. */
-enum { TSDP_PROF_FAMILIES = 7 };
+enum { TSDP_PROF_FAMILIES = 8 };
 int tsdp_profile(tsdp_ctx* ctx, int enable);
 int tsdp_profile_read(tsdp_ctx* ctx, double* ms, double* flop, uint64_t* launches);
 

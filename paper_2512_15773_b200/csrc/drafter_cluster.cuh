@@ -1,0 +1,449 @@
+// Persistent drafter: the whole K-step draft rollout of one environment (Sec. 3.2 "Draft Generation
+// Procedure", Eq. (3)) in ONE kernel launch, for small batches where the rollout is latency-bound.
+//
+// One thread-block cluster of DC_CS CTAs serves one environment at a time.  Every CTA keeps, for the
+// whole launch, its 1/DC_CS slice (a block of output columns) of every weight matrix of the drafter
+// in shared memory, and a full replica of the activations of the 16-token sequence.  A linear layer
+// is computed as Y[:, slice] = X W_slice^T on mma.sync m16n8k16 (the sequence is one 16-row tile),
+// and each CTA writes its slice of Y into the replicas of all CTAs through distributed shared
+// memory; one hardware cluster barrier separates dependent stages (6 per block).  LayerNorm, the two
+// attentions, the head, the DDPM posterior and the noise are cheap enough to be recomputed by every
+// CTA, which saves their broadcasts.  Reductions are warp shuffles.  Nothing spins on memory: the
+// only waits are __syncthreads and barrier.cluster, which all CTAs of a cluster reach the same
+// number of times because the control flow depends only on (t[b], k).
+#pragma once
+#include <cooperative_groups.h>
+#include "common.cuh"
+#include "gemm_tcgen05.cuh"
+#include "net_kernels.cuh"
+
+namespace tsdp {
+namespace cg = cooperative_groups;
+
+constexpr int DC_CS = 8;          // CTAs per cluster (the portable maximum)
+constexpr int DC_THREADS = 256;
+constexpr int DC_WARPS = DC_THREADS / 32;
+constexpr int DC_ROWS = 16;       // one m16 tile: H <= 16
+constexpr int DC_MAX_LAYERS = 4;
+constexpr int DC_MAX_NK = 4;      // memory tokens: time token + at most 3 observation tokens
+
+struct DcLayer {
+  const __nv_bfloat16 *Wqkv, *Wo, *Wq2, *Wo2, *W1, *W2;      // [out, in] bf16
+  const float *bqkv, *bo, *bq2, *bo2, *b1, *b2;
+  const float *ln1_g, *ln1_b, *ln2_g, *ln2_b, *ln3_g, *ln3_b;
+};
+
+struct DcParams {
+  DcLayer L[DC_MAX_LAYERS];
+  int layers, heads, H, A, To, T;
+  const float *W_in, *b_in, *pos;                            // [A, d], [d], [H, d]
+  const float *lnf_g, *lnf_b, *W_outT, *b_out;               // W_outT [A, d]
+  const float *kv_time, *kv_obs;                             // [T, L*2d], [B*To, L*2d]
+  DdpmTables S;
+  float* xt; long long xs_b;                                 // candidates [B, Kmax+1, D]
+  float* muhat; long long ms_b;                              // drafter means [B, Kmax, D]
+  const int* t;
+  const uint64_t* seed;
+  int B, K;
+};
+
+// Shared-memory plan of one CTA (bytes), for model width d.  Weight rows are padded by 8 elements so
+// that fragment loads of 8 consecutive rows fall into different banks.
+struct DcSmem {
+  int w_layer;      // bytes of one layer's weight slices
+  int off_h, off_a, off_qkv, off_q2, off_f, off_red, off_kv, off_x, off_posb, off_win, total;
+};
+__host__ __device__ inline DcSmem dc_smem_plan(int d, int layers, int A) {
+  DcSmem p;
+  const int pw = d + 8, pw4 = 4 * d + 8;
+  const int rows_d = (3 * d + d + d + d + 4 * d) / DC_CS;    // output rows of the K = d matrices in a slice
+  p.w_layer = (rows_d * pw + (d / DC_CS) * pw4) * 2;
+  int o = layers * p.w_layer;
+  auto take = [&](int bytes) { int r = o; o += (bytes + 15) & ~15; return r; };
+  p.off_h = take(DC_ROWS * d * 4);
+  p.off_a = take(DC_ROWS * (d + 8) * 2);
+  p.off_qkv = take(DC_ROWS * (3 * d + 8) * 2);
+  p.off_q2 = take(DC_ROWS * (d + 8) * 2);
+  p.off_f = take(DC_ROWS * (4 * d + 8) * 2);
+  p.off_red = take(DC_WARPS * DC_ROWS * 8 * 4);              // one 16 x 8 fp32 tile per warp
+  p.off_kv = take(DC_MAX_NK * 2 * d * 4);
+  p.off_x = take(DC_ROWS * 16 * 4 * 2);                      // latent and eps, D <= 256
+  p.off_posb = take(DC_ROWS * d * 4);
+  p.off_win = take(A * d * 4);
+  p.total = o;
+  return p;
+}
+
+// Y[16, n_slice] = X[16, KD] * Wslice[n_slice, KD]^T.  Work units are (8-column tile, K part): with
+// fewer tiles than warps the K range is split and the parts are summed through shared memory.
+// `emit(row, col, v0, v1)` receives two adjacent columns (col even) of the finished slice.
+template <int KD, typename Emit>
+__device__ __forceinline__ void dc_linear(const __nv_bfloat16* X, int px, const __nv_bfloat16* W, int n_slice,
+                                          float* red, Emit emit) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, tg = lane & 3;
+  constexpr int PW = KD + 8;
+  const int n_tiles = n_slice >> 3;
+  int ksplit = 1;
+  while (n_tiles * ksplit * 2 <= DC_WARPS && (KD / 16) % (ksplit * 2) == 0) ksplit *= 2;
+  const int units = n_tiles * ksplit;
+  for (int u0 = 0; u0 < units; u0 += DC_WARPS) {
+    const int u = u0 + warp;
+    if (u < units) {
+      const int nt = u % n_tiles, kp = u / n_tiles;
+      const int ks0 = kp * (KD / 16 / ksplit), ks1 = ks0 + KD / 16 / ksplit;
+      float c[4] = {0.f, 0.f, 0.f, 0.f};
+      const __nv_bfloat16* wrow = W + (size_t)(nt * 8 + g) * PW;
+      const __nv_bfloat16* x0 = X + (size_t)g * px;
+      const __nv_bfloat16* x1 = X + (size_t)(g + 8) * px;
+#pragma unroll 4
+      for (int ks = ks0; ks < ks1; ++ks) {
+        const int k = ks * 16 + 2 * tg;
+        uint32_t a[4];
+        a[0] = *reinterpret_cast<const uint32_t*>(x0 + k);
+        a[1] = *reinterpret_cast<const uint32_t*>(x1 + k);
+        a[2] = *reinterpret_cast<const uint32_t*>(x0 + k + 8);
+        a[3] = *reinterpret_cast<const uint32_t*>(x1 + k + 8);
+        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(wrow + k);
+        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(wrow + k + 8);
+        mma_bf16_16816(c, a, b0, b1);
+      }
+      float* r = red + (size_t)warp * (DC_ROWS * 8);
+      r[g * 8 + 2 * tg] = c[0]; r[g * 8 + 2 * tg + 1] = c[1];
+      r[(g + 8) * 8 + 2 * tg] = c[2]; r[(g + 8) * 8 + 2 * tg + 1] = c[3];
+    }
+    __syncthreads();
+    // finished tiles of this pass: tile nt = sum over its K parts (warps nt, nt + n_tiles, ...)
+    const int tiles_here = min(n_tiles, DC_WARPS);   // units are laid out part-major: a pass holds whole tiles
+    for (int i = threadIdx.x; i < tiles_here * DC_ROWS * 4; i += DC_THREADS) {
+      const int nt = i / (DC_ROWS * 4), rem = i % (DC_ROWS * 4);
+      const int row = rem >> 2, cp = (rem & 3) * 2;
+      const int tile = u0 + nt;              // with a K split there is a single pass (u0 = 0)
+      if (tile >= n_tiles) continue;
+      float v0 = 0.f, v1 = 0.f;
+      for (int kp = 0; kp < ksplit; ++kp) {
+        const int w = (ksplit == 1) ? nt : nt + kp * n_tiles;
+        v0 += red[(size_t)w * (DC_ROWS * 8) + row * 8 + cp];
+        v1 += red[(size_t)w * (DC_ROWS * 8) + row * 8 + cp + 1];
+      }
+      emit(row, tile * 8 + cp, v0, v1);
+    }
+    __syncthreads();
+  }
+}
+
+
+// LayerNorm of the 16 replicated rows: warp w normalises rows w and w + 8; fp32 in, bf16 out.
+template <int D_MODEL>
+__device__ __forceinline__ void dc_layernorm(const float* h, const float* __restrict__ gam, const float* __restrict__ bet,
+                                             __nv_bfloat16* out, int pitch) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int V = D_MODEL / 128;
+#pragma unroll
+  for (int rr = 0; rr < 2; ++rr) {
+    const int row = warp + rr * 8;
+    float4 v[V];
+    float s = 0.f;
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      v[j] = *reinterpret_cast<const float4*>(h + row * D_MODEL + j * 128 + lane * 4);
+      s += v[j].x + v[j].y + v[j].z + v[j].w;
+    }
+    const float mean = warp_sum(s) / D_MODEL;
+    float q = 0.f;
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      v[j].x -= mean; v[j].y -= mean; v[j].z -= mean; v[j].w -= mean;
+      q += v[j].x * v[j].x + v[j].y * v[j].y + v[j].z * v[j].z + v[j].w * v[j].w;
+    }
+    const float rstd = rsqrtf(warp_sum(q) / D_MODEL + 1e-5f);
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      const int c = j * 128 + lane * 4;
+      const float4 gg = __ldg(reinterpret_cast<const float4*>(gam + c)), bb = __ldg(reinterpret_cast<const float4*>(bet + c));
+      store4(out + row * pitch + c, v[j].x * rstd * gg.x + bb.x, v[j].y * rstd * gg.y + bb.y,
+             v[j].z * rstd * gg.z + bb.z, v[j].w * rstd * gg.w + bb.w);
+    }
+  }
+}
+
+// Attention of the replicated sequence, recomputed by every CTA: four lanes own one (head, query row),
+// each a quarter of the head width.  SELF: causal over the H tokens in qkv; otherwise over NK memory
+// tokens whose keys/values are the fp32 rows kv[kx] = [K (d) | V (d)].
+template <int D_MODEL, bool SELF>
+__device__ __forceinline__ void dc_attention(const __nv_bfloat16* qsrc, int pq, const __nv_bfloat16* qkv, int pqkv,
+                                             const float* kv, int NK, __nv_bfloat16* out, int po, int heads, int H) {
+  const int dh = D_MODEL / heads, seg = dh >> 2;
+  const int sub = threadIdx.x & 3;
+  const float scale = rsqrtf((float)dh);
+  for (int p = threadIdx.x >> 2; p < heads * DC_ROWS; p += DC_THREADS / 4) {
+    const int head = p / DC_ROWS, row = p % DC_ROWS;
+    const int c0 = head * dh + sub * seg;
+    constexpr int NKEY = SELF ? DC_ROWS : DC_MAX_NK;
+    float sc[NKEY];
+    float m = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < NKEY; ++j) {
+      float a = 0.f;
+      if (SELF) {
+        for (int i = 0; i < seg; ++i)
+          a += __bfloat162float(qsrc[row * pq + c0 + i]) * __bfloat162float(qkv[j * pqkv + D_MODEL + c0 + i]);
+      } else if (j < NK) {
+        for (int i = 0; i < seg; ++i) a += __bfloat162float(qsrc[row * pq + c0 + i]) * kv[j * 2 * D_MODEL + c0 + i];
+      }
+      a += __shfl_xor_sync(0xffffffffu, a, 1);
+      a += __shfl_xor_sync(0xffffffffu, a, 2);
+      const bool vis = SELF ? (j <= row && j < H) : (j < NK);
+      sc[j] = vis ? a * scale : -INFINITY;
+      m = fmaxf(m, sc[j]);
+    }
+    if (m == -INFINITY) m = 0.f;            // padding rows see nothing; keep them finite
+    float l = 0.f;
+#pragma unroll
+    for (int j = 0; j < NKEY; ++j) { sc[j] = __expf(sc[j] - m); l += sc[j]; }
+    const float inv = l > 0.f ? 1.0f / l : 0.f;
+    for (int i = 0; i < seg; ++i) {
+      float o = 0.f;
+#pragma unroll
+      for (int j = 0; j < NKEY; ++j) {
+        if (SELF) o += sc[j] * __bfloat162float(qkv[j * pqkv + 2 * D_MODEL + c0 + i]);
+        else if (j < NK) o += sc[j] * kv[j * 2 * D_MODEL + D_MODEL + c0 + i];
+      }
+      out[row * po + c0 + i] = __float2bfloat16_rn(o * inv);
+    }
+  }
+}
+
+// Copy this CTA's block of `rows_per_cta` output rows of W [N, KD] into shared memory (row pitch KD + 8).
+template <int KD>
+__device__ __forceinline__ void dc_load_slice(__nv_bfloat16* dst, const __nv_bfloat16* __restrict__ W, int rows_per_cta,
+                                              int rank) {
+  constexpr int VPR = KD / 8;                      // 16-byte vectors per row
+  const uint4* src = reinterpret_cast<const uint4*>(W + (size_t)rank * rows_per_cta * KD);
+  for (int i = threadIdx.x; i < rows_per_cta * VPR; i += DC_THREADS) {
+    const int r = i / VPR, v = i % VPR;
+    *reinterpret_cast<uint4*>(dst + (size_t)r * (KD + 8) + v * 8) = __ldg(src + (size_t)r * VPR + v);
+  }
+}
+
+template <int D_MODEL>
+__global__ void __cluster_dims__(DC_CS, 1, 1) __launch_bounds__(DC_THREADS, 1)
+drafter_cluster_kernel(const __grid_constant__ DcParams P) {
+  extern __shared__ __align__(16) uint8_t dc_smem[];
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = (int)cluster.block_rank();
+  const int cid = blockIdx.x / DC_CS, ncl = gridDim.x / DC_CS;
+  constexpr int d = D_MODEL;
+  constexpr int PA = d + 8, PQKV = 3 * d + 8, PF = 4 * d + 8;
+  const DcSmem pl = dc_smem_plan(d, P.layers, P.A);
+  float* h = reinterpret_cast<float*>(dc_smem + pl.off_h);
+  __nv_bfloat16* a = reinterpret_cast<__nv_bfloat16*>(dc_smem + pl.off_a);
+  __nv_bfloat16* qkv = reinterpret_cast<__nv_bfloat16*>(dc_smem + pl.off_qkv);
+  __nv_bfloat16* q2 = reinterpret_cast<__nv_bfloat16*>(dc_smem + pl.off_q2);
+  __nv_bfloat16* f = reinterpret_cast<__nv_bfloat16*>(dc_smem + pl.off_f);
+  float* red = reinterpret_cast<float*>(dc_smem + pl.off_red);
+  float* skv = reinterpret_cast<float*>(dc_smem + pl.off_kv);
+  float* sx = reinterpret_cast<float*>(dc_smem + pl.off_x);
+  float* seps = sx + DC_ROWS * 16;
+  float* posb = reinterpret_cast<float*>(dc_smem + pl.off_posb);
+  float* win = reinterpret_cast<float*>(dc_smem + pl.off_win);
+  const int H = P.H, A = P.A, D = H * A, L = P.layers, NK = 1 + P.To;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  // ---- once per launch: this CTA's weight slices, embedding tables, zeroed activations
+  constexpr int NS_D = d / DC_CS, NS_3D = 3 * d / DC_CS, NS_4D = 4 * d / DC_CS;   // slice widths
+  auto w_ptr = [&](int l, int which) -> __nv_bfloat16* {     // 0 qkv, 1 o, 2 q2, 3 o2, 4 w1, 5 w2
+    const int rows_before[6] = {0, NS_3D, NS_3D + NS_D, NS_3D + 2 * NS_D, NS_3D + 3 * NS_D, NS_3D + 3 * NS_D + NS_4D};
+    return reinterpret_cast<__nv_bfloat16*>(dc_smem + (size_t)l * pl.w_layer) + (size_t)rows_before[which] * PA;
+  };
+  for (int l = 0; l < L; ++l) {
+    dc_load_slice<d>(w_ptr(l, 0), P.L[l].Wqkv, NS_3D, rank);
+    dc_load_slice<d>(w_ptr(l, 1), P.L[l].Wo, NS_D, rank);
+    dc_load_slice<d>(w_ptr(l, 2), P.L[l].Wq2, NS_D, rank);
+    dc_load_slice<d>(w_ptr(l, 3), P.L[l].Wo2, NS_D, rank);
+    dc_load_slice<d>(w_ptr(l, 4), P.L[l].W1, NS_4D, rank);
+    dc_load_slice<4 * d>(w_ptr(l, 5), P.L[l].W2, NS_D, rank);
+  }
+  for (int i = threadIdx.x; i < DC_ROWS * d; i += DC_THREADS) {
+    const int row = i / d, col = i % d;
+    posb[i] = row < H ? P.b_in[col] + P.pos[row * d + col] : 0.f;
+    h[i] = 0.f;
+  }
+  for (int i = threadIdx.x; i < A * d; i += DC_THREADS) win[i] = P.W_in[i];
+  for (int i = threadIdx.x; i < DC_ROWS * PA; i += DC_THREADS) { a[i] = __float2bfloat16_rn(0.f); q2[i] = a[i]; }
+  for (int i = threadIdx.x; i < DC_ROWS * PQKV; i += DC_THREADS) qkv[i] = __float2bfloat16_rn(0.f);
+  for (int i = threadIdx.x; i < DC_ROWS * PF; i += DC_THREADS) f[i] = __float2bfloat16_rn(0.f);
+  // replicas of the other CTAs, addressed through distributed shared memory
+  float* rh[DC_CS]; __nv_bfloat16 *rqkv[DC_CS], *rq2[DC_CS], *rf[DC_CS];
+#pragma unroll
+  for (int r = 0; r < DC_CS; ++r) {
+    rh[r] = cluster.map_shared_rank(h, r);
+    rqkv[r] = cluster.map_shared_rank(qkv, r);
+    rq2[r] = cluster.map_shared_rank(q2, r);
+    rf[r] = cluster.map_shared_rank(f, r);
+  }
+  cluster.sync();
+
+  const uint64_t seed = *P.seed;
+  const size_t ldkv = (size_t)L * 2 * d;
+  for (int env = cid; env < P.B; env += ncl) {
+    const int tb = P.t[env];
+    float* xt_b = P.xt + env * P.xs_b;
+    float* mh_b = P.muhat + env * P.ms_b;
+    for (int i = threadIdx.x; i < D; i += DC_THREADS) sx[i] = xt_b[i];
+    __syncthreads();
+    for (int k = 1; k <= P.K; ++k) {
+      const int tau = tb - k + 1;
+      if (!(tb >= 0 && tau >= 1)) {          // beyond K_eff: carry the latent along (same for every CTA)
+        if (rank == 0)
+          for (int i = threadIdx.x; i < D; i += DC_THREADS) {
+            mh_b[(size_t)(k - 1) * D + i] = sx[i];
+            xt_b[(size_t)k * D + i] = sx[i];
+          }
+        continue;
+      }
+      // token embedding into the residual stream
+      for (int i = threadIdx.x; i < DC_ROWS * d; i += DC_THREADS) {
+        const int row = i / d, col = i % d;
+        float v = posb[i];
+        if (row < H)
+          for (int c = 0; c < A; ++c) v += sx[row * A + c] * win[c * d + col];
+        h[i] = v;
+      }
+      __syncthreads();
+      for (int l = 0; l < L; ++l) {
+        const DcLayer& W = P.L[l];
+        // ---- causal self-attention
+        dc_layernorm<d>(h, W.ln1_g, W.ln1_b, a, PA);
+        __syncthreads();
+        dc_linear<d>(a, PA, w_ptr(l, 0), NS_3D, red, [&](int row, int col, float v0, float v1) {
+          const int cg_ = rank * NS_3D + col;
+          const uint32_t pk = pack_bf16x2(v0 + __ldg(W.bqkv + cg_), v1 + __ldg(W.bqkv + cg_ + 1));
+#pragma unroll
+          for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint32_t*>(rqkv[r] + row * PQKV + cg_) = pk;
+        });
+        cluster.sync();
+        dc_attention<d, true>(qkv, PQKV, qkv, PQKV, nullptr, 0, a, PA, P.heads, H);
+        __syncthreads();
+        dc_linear<d>(a, PA, w_ptr(l, 1), NS_D, red, [&](int row, int col, float v0, float v1) {
+          const int cg_ = rank * NS_D + col;
+          const float2 hv = *reinterpret_cast<const float2*>(h + row * d + cg_);
+          const float2 o = make_float2(hv.x + v0 + __ldg(W.bo + cg_), hv.y + v1 + __ldg(W.bo + cg_ + 1));
+#pragma unroll
+          for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<float2*>(rh[r] + row * d + cg_) = o;
+        });
+        // keys / values of the memory tokens for this block: time token of tau, then the obs tokens
+        for (int i = threadIdx.x; i < NK * 2 * d; i += DC_THREADS) {
+          const int kx = i / (2 * d), c = i % (2 * d);
+          const float* src = kx == 0 ? P.kv_time + (size_t)tau * ldkv : P.kv_obs + ((size_t)env * P.To + (kx - 1)) * ldkv;
+          skv[i] = __ldg(src + (size_t)l * 2 * d + c);
+        }
+        cluster.sync();
+        // ---- cross-attention to [time token | obs tokens]
+        dc_layernorm<d>(h, W.ln2_g, W.ln2_b, a, PA);
+        __syncthreads();
+        dc_linear<d>(a, PA, w_ptr(l, 2), NS_D, red, [&](int row, int col, float v0, float v1) {
+          const int cg_ = rank * NS_D + col;
+          const uint32_t pk = pack_bf16x2(v0 + __ldg(W.bq2 + cg_), v1 + __ldg(W.bq2 + cg_ + 1));
+#pragma unroll
+          for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint32_t*>(rq2[r] + row * PA + cg_) = pk;
+        });
+        cluster.sync();
+        dc_attention<d, false>(q2, PA, nullptr, 0, skv, NK, a, PA, P.heads, H);
+        __syncthreads();
+        dc_linear<d>(a, PA, w_ptr(l, 3), NS_D, red, [&](int row, int col, float v0, float v1) {
+          const int cg_ = rank * NS_D + col;
+          const float2 hv = *reinterpret_cast<const float2*>(h + row * d + cg_);
+          const float2 o = make_float2(hv.x + v0 + __ldg(W.bo2 + cg_), hv.y + v1 + __ldg(W.bo2 + cg_ + 1));
+#pragma unroll
+          for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<float2*>(rh[r] + row * d + cg_) = o;
+        });
+        cluster.sync();
+        // ---- MLP
+        dc_layernorm<d>(h, W.ln3_g, W.ln3_b, a, PA);
+        __syncthreads();
+        dc_linear<d>(a, PA, w_ptr(l, 4), NS_4D, red, [&](int row, int col, float v0, float v1) {
+          const int cg_ = rank * NS_4D + col;
+          float x0 = v0 + __ldg(W.b1 + cg_), x1 = v1 + __ldg(W.b1 + cg_ + 1);
+          x0 = 0.5f * x0 * (1.0f + ptx::tanh_fast(0.7978845608028654f * (x0 + 0.044715f * x0 * x0 * x0)));
+          x1 = 0.5f * x1 * (1.0f + ptx::tanh_fast(0.7978845608028654f * (x1 + 0.044715f * x1 * x1 * x1)));
+          const uint32_t pk = pack_bf16x2(x0, x1);
+#pragma unroll
+          for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint32_t*>(rf[r] + row * PF + cg_) = pk;
+        });
+        cluster.sync();
+        dc_linear<4 * d>(f, PF, w_ptr(l, 5), NS_D, red, [&](int row, int col, float v0, float v1) {
+          const int cg_ = rank * NS_D + col;
+          const float2 hv = *reinterpret_cast<const float2*>(h + row * d + cg_);
+          const float2 o = make_float2(hv.x + v0 + __ldg(W.b2 + cg_), hv.y + v1 + __ldg(W.b2 + cg_ + 1));
+#pragma unroll
+          for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<float2*>(rh[r] + row * d + cg_) = o;
+        });
+        cluster.sync();
+      }
+      // ---- head: eps = LN_f(h) W_out + b_out   (every CTA, rows w and w + 8 per warp)
+      {
+        constexpr int V = d / 128;
+#pragma unroll
+        for (int rr = 0; rr < 2; ++rr) {
+          const int row = warp + rr * 8;
+          float4 v[V];
+          float s = 0.f;
+#pragma unroll
+          for (int j = 0; j < V; ++j) {
+            v[j] = *reinterpret_cast<const float4*>(h + row * d + j * 128 + lane * 4);
+            s += v[j].x + v[j].y + v[j].z + v[j].w;
+          }
+          const float mean = warp_sum(s) / d;
+          float q = 0.f;
+#pragma unroll
+          for (int j = 0; j < V; ++j) {
+            v[j].x -= mean; v[j].y -= mean; v[j].z -= mean; v[j].w -= mean;
+            q += v[j].x * v[j].x + v[j].y * v[j].y + v[j].z * v[j].z + v[j].w * v[j].w;
+          }
+          const float rstd = rsqrtf(warp_sum(q) / d + 1e-5f);
+#pragma unroll
+          for (int j = 0; j < V; ++j) {
+            const int c = j * 128 + lane * 4;
+            const float4 gg = __ldg(reinterpret_cast<const float4*>(P.lnf_g + c)), bb = __ldg(reinterpret_cast<const float4*>(P.lnf_b + c));
+            v[j].x = v[j].x * rstd * gg.x + bb.x; v[j].y = v[j].y * rstd * gg.y + bb.y;
+            v[j].z = v[j].z * rstd * gg.z + bb.z; v[j].w = v[j].w * rstd * gg.w + bb.w;
+          }
+          for (int c = 0; c < A; ++c) {
+            float acc = 0.f;
+#pragma unroll
+            for (int j = 0; j < V; ++j) {
+              const float4 w = __ldg(reinterpret_cast<const float4*>(P.W_outT + (size_t)c * d + j * 128 + lane * 4));
+              acc += v[j].x * w.x + v[j].y * w.y + v[j].z * w.z + v[j].w * w.w;
+            }
+            acc = warp_sum(acc);
+            if (lane == 0 && row < H) seps[row * A + c] = acc + __ldg(P.b_out + c);
+          }
+        }
+      }
+      __syncthreads();
+      // ---- scheduler step: mu^_k, x~_k = mu^_k + sigma_tau xi_tau
+      {
+        const int nq = (D + 3) >> 2;
+        for (int q = threadIdx.x; q < nq; q += DC_THREADS) {
+          float z[4];
+          normal4(seed, (uint32_t)env, STREAM_XI, (uint32_t)tau, (uint32_t)q, z);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int i = 4 * q + j;
+            if (i < D) {
+              const float m = posterior_mean(P.S, sx[i], seps[i], tau);
+              const float xn = m + P.S.sigma[tau] * z[j];
+              sx[i] = xn;
+              if (rank == 0) { mh_b[(size_t)(k - 1) * D + i] = m; xt_b[(size_t)k * D + i] = xn; }
+            }
+          }
+        }
+      }
+      __syncthreads();
+    }
+    __syncthreads();
+  }
+  cluster.sync();      // no CTA leaves while another may still write into its shared memory
+}
+}  // namespace tsdp

@@ -17,6 +17,7 @@
 #include "gemm_tcgen05.cuh"
 #include "net_kernels.cuh"
 #include "round_kernels.cuh"
+#include "drafter_cluster.cuh"
 
 using namespace tsdp;
 
@@ -77,6 +78,9 @@ struct tsdp_ctx {
   std::map<std::tuple<const void*, int, int, int, int, int, int>, CUtensorMap> maps;
   EncodeTiledFn encode = nullptr;
   cudaStream_t cap_stream = nullptr;
+  // persistent cluster drafter: usable for this configuration, shared memory per CTA, clusters that fit the GPU
+  bool dc_ok = false;
+  int dc_smem = 0, dc_max_clusters = 0;
   uint64_t rounds = 0, launches = 0;
   int launches_per_round_tmp = 0;
   // optional per-kernel-family timing with CUDA events (plain launches, no graph)
@@ -456,13 +460,62 @@ int forward(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStream_t s) 
   return TSDP_ERR_UNSUPPORTED;
 }
 
+// ------------------------------------------------------------------------------------------ drafter
+// Whether the persistent cluster kernel can run this context's drafter at all (shapes, shared memory).
+bool cluster_drafter_fits(const tsdp_config_t& cfg, int* smem_bytes) {
+  const tsdp_net_t& n = cfg.draft;
+  if (cfg.precision != 1 || n.arch != TSDP_ARCH_XFMR || (n.d != 128 && n.d != 256) || n.layers > DC_MAX_LAYERS ||
+      cfg.H > DC_ROWS || 1 + cfg.obs_tokens > DC_MAX_NK || cfg.H * cfg.A > 256 || (n.d / n.heads) % 4 != 0)
+    return false;
+  const DcSmem pl = dc_smem_plan(n.d, n.layers, cfg.A);
+  *smem_bytes = pl.total;
+  return pl.total <= 227 * 1024;
+}
+
+bool use_cluster_drafter(const tsdp_ctx* c, int B) {
+  if (!c->dc_ok || c->cfg.drafter == 1) return false;
+  if (c->cfg.drafter == 2) return true;
+  return B <= 4 * c->dc_max_clusters;     // beyond a few waves of clusters the batched tensor-core path wins
+}
+
+int launch_cluster_drafter(tsdp_ctx* c, int B, int K, cudaStream_t s) {
+  const Net& n = c->net[TSDP_DRAFT];
+  DcParams P{};
+  for (int l = 0; l < n.cfg.layers; ++l) {
+    const XfmrLayer& w = n.L[l];
+    DcLayer& o = P.L[l];
+    o.Wqkv = (const __nv_bfloat16*)w.Wqkv; o.Wo = (const __nv_bfloat16*)w.Wo; o.Wq2 = (const __nv_bfloat16*)w.Wq2;
+    o.Wo2 = (const __nv_bfloat16*)w.Wo2; o.W1 = (const __nv_bfloat16*)w.W1; o.W2 = (const __nv_bfloat16*)w.W2;
+    o.bqkv = w.bqkv; o.bo = w.bo; o.bq2 = w.bq2; o.bo2 = w.bo2; o.b1 = w.b1; o.b2 = w.b2;
+    o.ln1_g = w.ln1_g; o.ln1_b = w.ln1_b; o.ln2_g = w.ln2_g; o.ln2_b = w.ln2_b; o.ln3_g = w.ln3_g; o.ln3_b = w.ln3_b;
+  }
+  P.layers = n.cfg.layers; P.heads = n.cfg.heads; P.H = c->cfg.H; P.A = c->cfg.A; P.To = c->cfg.obs_tokens; P.T = c->cfg.T;
+  P.W_in = n.W_in; P.b_in = n.b_in; P.pos = n.pos;
+  P.lnf_g = n.lnf_g; P.lnf_b = n.lnf_b; P.W_outT = n.W_outT; P.b_out = n.b_out;
+  P.kv_time = n.kv_time; P.kv_obs = n.kv_obs;
+  P.S = c->S;
+  P.xt = c->xt; P.xs_b = (long long)(c->cfg.max_K + 1) * c->D;
+  P.muhat = c->muhat; P.ms_b = (long long)(c->cfg.max_K > 0 ? c->cfg.max_K : 1) * c->D;
+  P.t = c->t; P.seed = c->seed; P.B = B; P.K = K;
+  const int ncl = B < c->dc_max_clusters ? B : c->dc_max_clusters;
+  prof_begin(c, s, 7, 0.0);
+  if (n.cfg.d == 128) drafter_cluster_kernel<128><<<ncl * DC_CS, DC_THREADS, c->dc_smem, s>>>(P);
+  else drafter_cluster_kernel<256><<<ncl * DC_CS, DC_THREADS, c->dc_smem, s>>>(P);
+  prof_end(c, s);
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  return TSDP_OK;
+}
+
 // ------------------------------------------------------------------------------------------ round
 // Enqueue one speculative round for B environments with K draft steps.
 int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
   const int D = c->D;
   const long long xs_b = (long long)(c->cfg.max_K + 1) * D, ms_b = (long long)(c->cfg.max_K > 0 ? c->cfg.max_K : 1) * D;
   int r;
-  for (int k = 1; k <= K; ++k) {
+  const bool cluster_draft = K > 0 && use_cluster_drafter(c, B);
+  if (cluster_draft && (r = launch_cluster_drafter(c, B, K, s))) return r;
+  for (int k = 1; k <= K && !cluster_draft; ++k) {
     CandMap cm{c->xt + (long long)(k - 1) * D, xs_b, c->eps_d, (long long)D, c->t, 1, k - 1};
     c->prof_gemm_cat = 6;
     r = forward(c, c->net[TSDP_DRAFT], cm, B, s);
@@ -593,7 +646,7 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   if (!cfg || !out) return TSDP_ERR_ARG;
   if (cfg->H < 1 || cfg->A < 1 || cfg->T < 1 || cfg->T > TSDP_MAX_T || cfg->max_B < 1 || cfg->max_K < 0 ||
       cfg->max_K > TSDP_MAX_K || cfg->obs_tokens < 0 || cfg->obs_dim < 0 || !(cfg->beta0 > 0.f) || !(cfg->beta1 < 1.f) ||
-      (cfg->precision != 0 && cfg->precision != 1))
+      (cfg->precision != 0 && cfg->precision != 1) || cfg->drafter < 0 || cfg->drafter > 2)
     return TSDP_ERR_ARG;
   for (const tsdp_net_t* n : {&cfg->base, &cfg->draft}) {
     if (n->arch < TSDP_ARCH_GAUSS || n->arch > TSDP_ARCH_XFMR) return TSDP_ERR_UNSUPPORTED;
@@ -695,6 +748,24 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
     INIT_TRY(set_smem_attr_all<128>());
     INIT_TRY(set_smem_attr_all<64>());
     INIT_TRY(set_smem_attr_all<32>());
+  }
+  if (cluster_drafter_fits(*cfg, &c->dc_smem)) {
+    const void* fn = cfg->draft.d == 128 ? (const void*)drafter_cluster_kernel<128> : (const void*)drafter_cluster_kernel<256>;
+    INIT_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, c->dc_smem));
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(DC_CS * 64); lc.blockDim = dim3(DC_THREADS); lc.dynamicSmemBytes = (size_t)c->dc_smem;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = DC_CS; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    lc.attrs = at; lc.numAttrs = 1;
+    int ncl = 0;
+    if (cudaOccupancyMaxActiveClusters(&ncl, fn, &lc) != cudaSuccess || ncl < 1) { cudaGetLastError(); ncl = 0; }
+    c->dc_max_clusters = ncl;
+    c->dc_ok = ncl >= 1;
+  }
+  if (cfg->drafter == 2 && !c->dc_ok) {
+    fprintf(stderr, "tsdp_init: the persistent cluster drafter does not fit this configuration\n");
+    return fail(TSDP_ERR_UNSUPPORTED);
   }
   INIT_TRY(cudaFuncSetAttribute(self_attn_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
   INIT_TRY(cudaFuncSetAttribute(self_attn_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));

@@ -12,8 +12,8 @@ pytestmark = pytest.mark.gpu
 BAND = 1e-3     # |log alpha - log u| below which a flipped accept decision is tolerated
 
 
-def _round_parity(wl, B, K, acc, seed, tol_eps, tol_x, t0s, precision=None):
-    smp, S, base, draft = hp.setup(wl, max_B=B, max_K=max(K, 1), precision=precision)
+def _round_parity(wl, B, K, acc, seed, tol_eps, tol_x, t0s, precision=None, drafter=0):
+    smp, S, base, draft = hp.setup(wl, max_B=B, max_K=max(K, 1), precision=precision, drafter=drafter)
     shape = (wl["H"], wl["A"]); D = wl["H"] * wl["A"]
     obs = inputs.make_obs(3, B, wl["To"], wl["Do"])
     noise = spec.PhiloxNoise(seed)
@@ -61,8 +61,37 @@ def test_round_transformer(precision, tol_eps, tol_x):
     _round_parity(wl, 5, 8, hp.accept_t(), 21, tol_eps, tol_x, [99, 70, 40, 5, 0])
 
 
-def _chunk_parity(wl, B, K, acc, seed, tol_final, precision=None, schedule=None):
-    smp, S, base, draft = hp.setup(wl, max_B=B, max_K=max(K, 1) if schedule is None else 10, precision=precision)
+@pytest.mark.parametrize("drafter", [1, 2])
+def test_round_transformer_bf16_both_drafters(drafter):
+    """Layer-by-layer drafter and the persistent cluster drafter against the oracle, same round."""
+    wl = dict(inputs.WORKLOADS["pusht_xfmr"], precision=1)
+    _round_parity(wl, 5, 8, hp.accept_t(), 21, 2e-2, 3e-3, [99, 70, 40, 5, 0], drafter=drafter)
+    # more environments than clusters fit at once, ragged K_eff, A = 7
+    wl7 = hp.small_xfmr_workload(1, d=256, heads=4, layers=2, dd=128, dlayers=2, H=16, A=7, To=3, Do=9, gamma=0.05)
+    _round_parity(wl7, 23, 6, hp.accept_t(sigma_scale=1.5), 5, 2e-2, 3e-3, [99 - 4 * i for i in range(22)] + [2],
+                  drafter=drafter)
+
+
+def test_cluster_drafter_matches_layered_drafter():
+    wl = dict(inputs.WORKLOADS["pusht_xfmr"], precision=1)
+    B, K, D = 3, 8, 32
+    outs = []
+    for drafter in (1, 2):
+        smp, *_ = hp.setup(wl, max_B=B, max_K=K, drafter=drafter)
+        obs = torch.tensor(inputs.make_obs(3, B, wl["To"], wl["Do"]), dtype=torch.float32, device="cuda")
+        x = torch.tensor(np.random.default_rng(0).normal(size=(B, D)).astype(np.float32), device="cuda")
+        h_t = np.array([90, 50, 3], dtype=np.int32)
+        xt = torch.zeros(B, K + 1, D, device="cuda"); mh = torch.zeros(B, K, D, device="cuda")
+        smp.round(obs, B, K, hp.accept_t(), 4, x, h_t, xt, mh, None, None, None)
+        outs.append((xt.cpu().numpy(), mh.cpu().numpy()))
+        smp.close()
+    assert np.max(np.abs(outs[0][0] - outs[1][0])) < 3e-3
+    assert np.max(np.abs(outs[0][1] - outs[1][1])) < 3e-3
+
+
+def _chunk_parity(wl, B, K, acc, seed, tol_final, precision=None, schedule=None, drafter=0):
+    smp, S, base, draft = hp.setup(wl, max_B=B, max_K=max(K, 1) if schedule is None else 10, precision=precision,
+                                   drafter=drafter)
     shape = (wl["H"], wl["A"])
     obs = inputs.make_obs(4, B, wl["To"], wl["Do"])
     dobs = torch.tensor(obs, dtype=torch.float32, device="cuda")
@@ -105,11 +134,11 @@ def test_chunk_toy_mlp_fp32_matches_oracle_exactly_in_structure():
         assert st["env_rounds"] == tot["rounds"] and st["rejections"] == tot["rej"]
 
 
-@pytest.mark.parametrize("precision", [0, 1])
-def test_chunk_pusht_transformer(precision):
+@pytest.mark.parametrize("precision,drafter", [(0, 0), (1, 1), (1, 2)])
+def test_chunk_pusht_transformer(precision, drafter):
     wl = dict(inputs.WORKLOADS["pusht_xfmr"], precision=precision)
     B = 3
-    n_match, tot, st = _chunk_parity(wl, B, 8, hp.accept_t(), 9, 3e-2, precision=precision)
+    n_match, tot, st = _chunk_parity(wl, B, 8, hp.accept_t(), 9, 3e-2, precision=precision, drafter=drafter)
     if precision == 0:
         assert n_match >= B - 1
     else:
@@ -129,7 +158,8 @@ def test_chunk_with_round_schedule_fp32():
 def test_drafter_equal_to_base_accepts_everything_and_equals_vanilla():
     for wl in (dict(inputs.WORKLOADS["toy_mlp"]), hp.small_xfmr_workload(1)):
         B = 4
-        smp, S, base, _ = hp.setup(wl, max_B=B, max_K=6, draft_is_base=True)
+        # bit-identity needs the same kernels on both sides: the layer-by-layer drafter
+        smp, S, base, _ = hp.setup(wl, max_B=B, max_K=6, draft_is_base=True, drafter=1)
         obs = torch.tensor(inputs.make_obs(4, B, wl["To"], wl["Do"]), dtype=torch.float32, device="cuda")
         ref = torch.zeros(B, wl["H"], wl["A"], device="cuda")
         smp.sample_chunk(obs, B, 0, hp.accept_t(), 77, ref)                  # K = 0: vanilla DDPM
@@ -145,6 +175,21 @@ def test_drafter_equal_to_base_accepts_everything_and_equals_vanilla():
             if K == 1 and bonus == 0:
                 assert st["env_rounds"] == 100 * B                           # T base forwards per chunk
         smp.close()
+
+
+def test_cluster_drafter_equal_to_base_is_accepted_almost_always():
+    """Same weights through two different kernels (cluster drafter vs tensor-core base): the means
+    differ by rounding only, so nearly every draft passes the likelihood-ratio test."""
+    wl = hp.small_xfmr_workload(1)
+    B = 4
+    smp, *_ = hp.setup(wl, max_B=B, max_K=6, draft_is_base=True, drafter=2)
+    obs = torch.tensor(inputs.make_obs(4, B, wl["To"], wl["Do"]), dtype=torch.float32, device="cuda")
+    out = torch.zeros(B, wl["H"], wl["A"], device="cuda")
+    smp.sample_chunk(obs, B, 6, hp.accept_t(), 77, out)
+    st = smp.stats()
+    assert st["steps_advanced"] == 100 * B and torch.isfinite(out).all()
+    assert st["drafts_accepted"] >= 0.95 * st["drafts_tested"]
+    smp.close()
 
 
 def test_gaussian_toy_on_gpu_matches_analytic_marginal():

@@ -177,11 +177,12 @@ uint64_t tsdp_kernel_launches(const tsdp_ctx* ctx);
 /* Per-kernel-family device timing with CUDA events, for the roofline report.  While enabled, rounds
  * are issued as plain launches (no graph) with an event pair around each launch on the caller's
  * stream.  Families: 0 GEMMs of the base model (tcgen05 or check-mode), 1 LayerNorm, 2 attention,
- * 3 embed/head/memory tokens, 4 round kernels (draft step, accept), 5 MLP / Gaussian denoiser, 6 GEMMs
- * of the drafter, 7 the persistent cluster drafter.  tsdp_profile(ctx, 0|1)
+ * 3 embed/head/memory tokens, 4 draft-step kernel, 5 MLP / Gaussian denoiser, 6 GEMMs
+ * of the drafter, 7 the persistent cluster drafter, 8 the fused
+ * acceptance / commit kernel.  tsdp_profile(ctx, 0|1)
  * clears the record.  tsdp_profile_read fills three arrays of TSDP_PROF_FAMILIES entries: summed
  * milliseconds, summed algorithmic flops (2*M*N*K per GEMM launch, 0 elsewhere) and launch counts. */
-enum { TSDP_PROF_FAMILIES = 8 };
+enum { TSDP_PROF_FAMILIES = 9 };
 int tsdp_profile(tsdp_ctx* ctx, int enable);
 int tsdp_profile_read(tsdp_ctx* ctx, double* ms, double* flop, uint64_t* launches);
 

@@ -16,7 +16,7 @@ EXPORTS = ["tsdp_init", "tsdp_destroy", "tsdp_strerror", "tsdp_last_error", "tsd
            "tsdp_load_weights", "tsdp_set_schedule", "tsdp_sample_chunk", "tsdp_sample_chunk_host",
            "tsdp_round", "tsdp_denoise", "tsdp_gemm", "tsdp_gemm_timed", "tsdp_stats", "tsdp_reset_stats",
            "tsdp_kernel_launches", "tsdp_profile", "tsdp_profile_read", "tsdp_verify_commit_static"]
-PROF_FAMILIES = ["gemm", "layernorm", "attention", "embed_head", "round", "small_net", "gemm_draft", "drafter_cluster"]
+PROF_FAMILIES = ["gemm", "layernorm", "attention", "embed_head", "round", "small_net", "gemm_draft", "drafter_cluster", "accept"]
 
 
 class NetT(C.Structure):

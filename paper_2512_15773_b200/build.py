@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtsdp.so")
 SOURCES = ["tsdp_api.cu"]
-DEPS = ["common.cuh", "gemm_tcgen05.cuh", "net_kernels.cuh", "round_kernels.cuh", "../../include/tsdp.h"]
+DEPS = sorted(f for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))) + ["../../include/tsdp.h"]
 
 
 def _stale():

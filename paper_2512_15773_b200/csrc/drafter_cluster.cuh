@@ -76,7 +76,7 @@ __host__ __device__ inline DcSmem dc_smem_plan(int d, int layers, int A) {
 
 // Y[16, n_slice] = X[16, KD] * Wslice[n_slice, KD]^T.  Work units are (8-column tile, K part): with
 // fewer tiles than warps the K range is split and the parts are summed through shared memory.
-// `emit(row, col, v0, v1)` receives two adjacent columns (col even) of the finished slice.
+// `emit(row, col, v)` receives 8 adjacent columns (col a multiple of 8) of the finished slice.
 template <int KD, typename Emit>
 __device__ __forceinline__ void dc_linear(const __nv_bfloat16* X, int px, const __nv_bfloat16* W, int n_slice,
                                           float* red, Emit emit) {
@@ -113,20 +113,22 @@ __device__ __forceinline__ void dc_linear(const __nv_bfloat16* X, int px, const 
       r[(g + 8) * 8 + 2 * tg] = c[2]; r[(g + 8) * 8 + 2 * tg + 1] = c[3];
     }
     __syncthreads();
-    // finished tiles of this pass: tile nt = sum over its K parts (warps nt, nt + n_tiles, ...)
+    // finished tiles of this pass: tile nt = sum over its K parts (warps nt, nt + n_tiles, ...);
+    // one thread finishes one row of one tile, so that it can store 8 adjacent columns at once
     const int tiles_here = min(n_tiles, DC_WARPS);   // units are laid out part-major: a pass holds whole tiles
-    for (int i = threadIdx.x; i < tiles_here * DC_ROWS * 4; i += DC_THREADS) {
-      const int nt = i / (DC_ROWS * 4), rem = i % (DC_ROWS * 4);
-      const int row = rem >> 2, cp = (rem & 3) * 2;
+    for (int i = threadIdx.x; i < tiles_here * DC_ROWS; i += DC_THREADS) {
+      const int nt = i / DC_ROWS, row = i % DC_ROWS;
       const int tile = u0 + nt;              // with a K split there is a single pass (u0 = 0)
       if (tile >= n_tiles) continue;
-      float v0 = 0.f, v1 = 0.f;
+      float v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] = 0.f;
       for (int kp = 0; kp < ksplit; ++kp) {
-        const int w = (ksplit == 1) ? nt : nt + kp * n_tiles;
-        v0 += red[(size_t)w * (DC_ROWS * 8) + row * 8 + cp];
-        v1 += red[(size_t)w * (DC_ROWS * 8) + row * 8 + cp + 1];
+        const float4* rp = reinterpret_cast<const float4*>(red + (size_t)(nt + kp * n_tiles) * (DC_ROWS * 8) + row * 8);
+        const float4 lo = rp[0], hi = rp[1];
+        v[0] += lo.x; v[1] += lo.y; v[2] += lo.z; v[3] += lo.w; v[4] += hi.x; v[5] += hi.y; v[6] += hi.z; v[7] += hi.w;
       }
-      emit(row, tile * 8 + cp, v0, v1);
+      emit(row, tile * 8, v);
     }
     __syncthreads();
   }
@@ -210,6 +212,80 @@ __device__ __forceinline__ void dc_attention(const __nv_bfloat16* qsrc, int pq, 
         else if (j < NK) o += sc[j] * kv[j * 2 * D_MODEL + D_MODEL + c0 + i];
       }
       out[row * po + c0 + i] = __float2bfloat16_rn(o * inv);
+    }
+  }
+}
+
+// Causal self-attention of the replicated 16-token sequence on mma.sync: warp w takes heads w, w + 8, ...
+// Same fragment algebra as self_attn_mma_kernel, operands read from the shared-memory qkv replica.
+template <int D_MODEL, int DH>
+__device__ __forceinline__ void dc_self_attn_mma(const __nv_bfloat16* qkv, int pqkv, __nv_bfloat16* out, int po, int heads,
+                                                 int H) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, tg = lane & 3;
+  constexpr int KS = DH / 16, NO = DH / 8;
+  const float scale = rsqrtf((float)DH);
+  for (int hd = warp; hd < heads; hd += DC_WARPS) {
+    const __nv_bfloat16* qb = qkv + hd * DH;
+    const __nv_bfloat16* kb = qkv + D_MODEL + hd * DH;
+    const __nv_bfloat16* vb = qkv + 2 * D_MODEL + hd * DH;
+    float s[2][4];
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt) {
+      s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+        const int k = ks * 16 + 2 * tg;
+        uint32_t a[4];
+        a[0] = *reinterpret_cast<const uint32_t*>(qb + g * pqkv + k);
+        a[1] = *reinterpret_cast<const uint32_t*>(qb + (g + 8) * pqkv + k);
+        a[2] = *reinterpret_cast<const uint32_t*>(qb + g * pqkv + k + 8);
+        a[3] = *reinterpret_cast<const uint32_t*>(qb + (g + 8) * pqkv + k + 8);
+        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(kb + (nt * 8 + g) * pqkv + k);
+        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(kb + (nt * 8 + g) * pqkv + k + 8);
+        mma_bf16_16816(s[nt], a, b0, b1);
+      }
+    }
+    const int r0 = g, r1 = g + 8;
+    float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt) {
+      const int col = nt * 8 + 2 * tg;
+      s[nt][0] = (col <= r0 && col < H) ? s[nt][0] * scale : -INFINITY;
+      s[nt][1] = (col + 1 <= r0 && col + 1 < H) ? s[nt][1] * scale : -INFINITY;
+      s[nt][2] = (col <= r1 && col < H) ? s[nt][2] * scale : -INFINITY;
+      s[nt][3] = (col + 1 <= r1 && col + 1 < H) ? s[nt][3] * scale : -INFINITY;
+      m0 = fmaxf(m0, fmaxf(s[nt][0], s[nt][1]));
+      m1 = fmaxf(m1, fmaxf(s[nt][2], s[nt][3]));
+    }
+    m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 1)); m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 2));
+    m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 1)); m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 2));
+    if (m0 == -INFINITY) m0 = 0.f;
+    if (m1 == -INFINITY) m1 = 0.f;
+    float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt) {
+      s[nt][0] = __expf(s[nt][0] - m0); s[nt][1] = __expf(s[nt][1] - m0);
+      s[nt][2] = __expf(s[nt][2] - m1); s[nt][3] = __expf(s[nt][3] - m1);
+      l0 += s[nt][0] + s[nt][1]; l1 += s[nt][2] + s[nt][3];
+    }
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+    const float inv0 = l0 > 0.f ? 1.0f / l0 : 0.f, inv1 = l1 > 0.f ? 1.0f / l1 : 0.f;
+    uint32_t pa[4];
+    pa[0] = pack_bf16x2(s[0][0], s[0][1]); pa[1] = pack_bf16x2(s[0][2], s[0][3]);
+    pa[2] = pack_bf16x2(s[1][0], s[1][1]); pa[3] = pack_bf16x2(s[1][2], s[1][3]);
+    const unsigned short* vraw = reinterpret_cast<const unsigned short*>(vb);
+#pragma unroll
+    for (int no = 0; no < NO; ++no) {
+      float o[4] = {0.f, 0.f, 0.f, 0.f};
+      const int col = no * 8 + g, k0 = 2 * tg;
+      const uint32_t b0 = (uint32_t)vraw[k0 * pqkv + col] | ((uint32_t)vraw[(k0 + 1) * pqkv + col] << 16);
+      const uint32_t b1 = (uint32_t)vraw[(k0 + 8) * pqkv + col] | ((uint32_t)vraw[(k0 + 9) * pqkv + col] << 16);
+      mma_bf16_16816(o, pa, b0, b1);
+      const int oc = hd * DH + no * 8 + 2 * tg;
+      *reinterpret_cast<uint32_t*>(out + r0 * po + oc) = pack_bf16x2(o[0] * inv0, o[1] * inv0);
+      *reinterpret_cast<uint32_t*>(out + r1 * po + oc) = pack_bf16x2(o[2] * inv1, o[3] * inv1);
     }
   }
 }
@@ -316,21 +392,34 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         // ---- causal self-attention
         dc_layernorm<d>(h, W.ln1_g, W.ln1_b, a, PA);
         __syncthreads();
-        dc_linear<d>(a, PA, w_ptr(l, 0), NS_3D, red, [&](int row, int col, float v0, float v1) {
+        dc_linear<d>(a, PA, w_ptr(l, 0), NS_3D, red, [&](int row, int col, float* v) {
           const int cg_ = rank * NS_3D + col;
-          const uint32_t pk = pack_bf16x2(v0 + __ldg(W.bqkv + cg_), v1 + __ldg(W.bqkv + cg_ + 1));
+          const float4 b0 = __ldg(reinterpret_cast<const float4*>(W.bqkv + cg_)), b1 = __ldg(reinterpret_cast<const float4*>(W.bqkv + cg_) + 1);
+          v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+          const uint4 pk = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
 #pragma unroll
-          for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint32_t*>(rqkv[r] + row * PQKV + cg_) = pk;
+          for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(rqkv[r] + row * PQKV + cg_) = pk;
         });
         cluster.sync();
-        dc_attention<d, true>(qkv, PQKV, qkv, PQKV, nullptr, 0, a, PA, P.heads, H);
+        switch (d / P.heads) {
+          case 32: dc_self_attn_mma<d, 32>(qkv, PQKV, a, PA, P.heads, H); break;
+          case 64: dc_self_attn_mma<d, 64>(qkv, PQKV, a, PA, P.heads, H); break;
+          case 128: dc_self_attn_mma<d, 128>(qkv, PQKV, a, PA, P.heads, H); break;
+          default: dc_attention<d, true>(qkv, PQKV, qkv, PQKV, nullptr, 0, a, PA, P.heads, H); break;
+        }
         __syncthreads();
-        dc_linear<d>(a, PA, w_ptr(l, 1), NS_D, red, [&](int row, int col, float v0, float v1) {
+        dc_linear<d>(a, PA, w_ptr(l, 1), NS_D, red, [&](int row, int col, float* v) {
           const int cg_ = rank * NS_D + col;
-          const float2 hv = *reinterpret_cast<const float2*>(h + row * d + cg_);
-          const float2 o = make_float2(hv.x + v0 + __ldg(W.bo + cg_), hv.y + v1 + __ldg(W.bo + cg_ + 1));
+          const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
+          const float4 h0 = hp[0], h1 = hp[1];
+          const float4 b0 = __ldg(reinterpret_cast<const float4*>(W.bo + cg_)), b1 = __ldg(reinterpret_cast<const float4*>(W.bo + cg_) + 1);
+          const float4 o0 = make_float4(h0.x + v[0] + b0.x, h0.y + v[1] + b0.y, h0.z + v[2] + b0.z, h0.w + v[3] + b0.w);
+          const float4 o1 = make_float4(h1.x + v[4] + b1.x, h1.y + v[5] + b1.y, h1.z + v[6] + b1.z, h1.w + v[7] + b1.w);
 #pragma unroll
-          for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<float2*>(rh[r] + row * d + cg_) = o;
+          for (int r = 0; r < DC_CS; ++r) {
+            float4* dst = reinterpret_cast<float4*>(rh[r] + row * d + cg_);
+            dst[0] = o0; dst[1] = o1;
+          }
         });
         // keys / values of the memory tokens for this block: time token of tau, then the obs tokens
         for (int i = threadIdx.x; i < NK * 2 * d; i += DC_THREADS) {
@@ -342,42 +431,58 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         // ---- cross-attention to [time token | obs tokens]
         dc_layernorm<d>(h, W.ln2_g, W.ln2_b, a, PA);
         __syncthreads();
-        dc_linear<d>(a, PA, w_ptr(l, 2), NS_D, red, [&](int row, int col, float v0, float v1) {
+        dc_linear<d>(a, PA, w_ptr(l, 2), NS_D, red, [&](int row, int col, float* v) {
           const int cg_ = rank * NS_D + col;
-          const uint32_t pk = pack_bf16x2(v0 + __ldg(W.bq2 + cg_), v1 + __ldg(W.bq2 + cg_ + 1));
+          const float4 b0 = __ldg(reinterpret_cast<const float4*>(W.bq2 + cg_)), b1 = __ldg(reinterpret_cast<const float4*>(W.bq2 + cg_) + 1);
+          v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+          const uint4 pk = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
 #pragma unroll
-          for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint32_t*>(rq2[r] + row * PA + cg_) = pk;
+          for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(rq2[r] + row * PA + cg_) = pk;
         });
         cluster.sync();
         dc_attention<d, false>(q2, PA, nullptr, 0, skv, NK, a, PA, P.heads, H);
         __syncthreads();
-        dc_linear<d>(a, PA, w_ptr(l, 3), NS_D, red, [&](int row, int col, float v0, float v1) {
+        dc_linear<d>(a, PA, w_ptr(l, 3), NS_D, red, [&](int row, int col, float* v) {
           const int cg_ = rank * NS_D + col;
-          const float2 hv = *reinterpret_cast<const float2*>(h + row * d + cg_);
-          const float2 o = make_float2(hv.x + v0 + __ldg(W.bo2 + cg_), hv.y + v1 + __ldg(W.bo2 + cg_ + 1));
+          const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
+          const float4 h0 = hp[0], h1 = hp[1];
+          const float4 b0 = __ldg(reinterpret_cast<const float4*>(W.bo2 + cg_)), b1 = __ldg(reinterpret_cast<const float4*>(W.bo2 + cg_) + 1);
+          const float4 o0 = make_float4(h0.x + v[0] + b0.x, h0.y + v[1] + b0.y, h0.z + v[2] + b0.z, h0.w + v[3] + b0.w);
+          const float4 o1 = make_float4(h1.x + v[4] + b1.x, h1.y + v[5] + b1.y, h1.z + v[6] + b1.z, h1.w + v[7] + b1.w);
 #pragma unroll
-          for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<float2*>(rh[r] + row * d + cg_) = o;
+          for (int r = 0; r < DC_CS; ++r) {
+            float4* dst = reinterpret_cast<float4*>(rh[r] + row * d + cg_);
+            dst[0] = o0; dst[1] = o1;
+          }
         });
         cluster.sync();
         // ---- MLP
         dc_layernorm<d>(h, W.ln3_g, W.ln3_b, a, PA);
         __syncthreads();
-        dc_linear<d>(a, PA, w_ptr(l, 4), NS_4D, red, [&](int row, int col, float v0, float v1) {
+        dc_linear<d>(a, PA, w_ptr(l, 4), NS_4D, red, [&](int row, int col, float* v) {
           const int cg_ = rank * NS_4D + col;
-          float x0 = v0 + __ldg(W.b1 + cg_), x1 = v1 + __ldg(W.b1 + cg_ + 1);
-          x0 = 0.5f * x0 * (1.0f + ptx::tanh_fast(0.7978845608028654f * (x0 + 0.044715f * x0 * x0 * x0)));
-          x1 = 0.5f * x1 * (1.0f + ptx::tanh_fast(0.7978845608028654f * (x1 + 0.044715f * x1 * x1 * x1)));
-          const uint32_t pk = pack_bf16x2(x0, x1);
+          const float4 b0 = __ldg(reinterpret_cast<const float4*>(W.b1 + cg_)), b1 = __ldg(reinterpret_cast<const float4*>(W.b1 + cg_) + 1);
+          v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
 #pragma unroll
-          for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint32_t*>(rf[r] + row * PF + cg_) = pk;
+          for (int j = 0; j < 8; ++j)
+            v[j] = 0.5f * v[j] * (1.0f + ptx::tanh_fast(0.7978845608028654f * (v[j] + 0.044715f * v[j] * v[j] * v[j])));
+          const uint4 pk = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
+#pragma unroll
+          for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(rf[r] + row * PF + cg_) = pk;
         });
         cluster.sync();
-        dc_linear<4 * d>(f, PF, w_ptr(l, 5), NS_D, red, [&](int row, int col, float v0, float v1) {
+        dc_linear<4 * d>(f, PF, w_ptr(l, 5), NS_D, red, [&](int row, int col, float* v) {
           const int cg_ = rank * NS_D + col;
-          const float2 hv = *reinterpret_cast<const float2*>(h + row * d + cg_);
-          const float2 o = make_float2(hv.x + v0 + __ldg(W.b2 + cg_), hv.y + v1 + __ldg(W.b2 + cg_ + 1));
+          const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
+          const float4 h0 = hp[0], h1 = hp[1];
+          const float4 b0 = __ldg(reinterpret_cast<const float4*>(W.b2 + cg_)), b1 = __ldg(reinterpret_cast<const float4*>(W.b2 + cg_) + 1);
+          const float4 o0 = make_float4(h0.x + v[0] + b0.x, h0.y + v[1] + b0.y, h0.z + v[2] + b0.z, h0.w + v[3] + b0.w);
+          const float4 o1 = make_float4(h1.x + v[4] + b1.x, h1.y + v[5] + b1.y, h1.z + v[6] + b1.z, h1.w + v[7] + b1.w);
 #pragma unroll
-          for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<float2*>(rh[r] + row * d + cg_) = o;
+          for (int r = 0; r < DC_CS; ++r) {
+            float4* dst = reinterpret_cast<float4*>(rh[r] + row * d + cg_);
+            dst[0] = o0; dst[1] = o1;
+          }
         });
         cluster.sync();
       }

@@ -532,7 +532,7 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
   int warps = K < 1 ? 1 : K;
   if (warps < 4) warps = 4;
   if (warps > 16) warps = 16;
-  prof_begin(c, s, 4, 0.0);
+  prof_begin(c, s, 8, 0.0);
   accept_kernel<<<B, warps * 32, 0, s>>>(c->S, c->xt, xs_b, c->muhat, ms_b, c->eps, xs_b, c->t, K, D, c->seed, c->sched,
                                          TSDP_MAX_T + 1, c->round_idx, c->actions, c->n_done, c->stats, c->cfg.draft_nfe,
                                          dbg ? c->dbg_logalpha : nullptr, dbg ? c->dbg_jstar : nullptr);

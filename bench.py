@@ -241,6 +241,29 @@ def run_ours(args):
                                       peak_source=f"bf16_tflops_sustained of {peaks['source']}", traffic=None,
                                       launches_timed=g["launches"], avg_launch_us=1e3 * g["ms"] / g["launches"],
                                       share_of_kernel_time=g["ms"] / tot_ms, family_ms=fam_ms)
+            if args.workload == "serving_xfmr" and B == 256:
+                # ncu DRAM bytes (read + write) of the six GEMM shapes of one base block at K = 10 (45056 rows),
+                # averaged per launch: profiles/gemm_tcgen05_serving_shapes.md.  Rounds with a smaller K launch
+                # proportionally fewer rows.
+                result["roofline"]["traffic"] = 171.1e6
+                result["roofline"]["traffic_note"] = ("mean DRAM bytes per launch over the 6 GEMM shapes of a block at "
+                                                      "45056 rows (ncu); algorithmic operand+output bytes average 224e6, "
+                                                      "the difference stays in L2")
+        a = prof.get("accept")
+        if a and a["launches"]:
+            # fused acceptance / commit kernel: bytes it must move per launch (candidates, drafter means, base
+            # outputs read once; committed latent written), summed over the rounds of the profiled step
+            D = wl["H"] * wl["A"]
+            if "schedule" in wl:
+                Ks = [wl["schedule"][0][min(r, len(wl["schedule"][0]) - 1)] for r in range(a["launches"])]
+            else:
+                Ks = [K] * a["launches"]
+            nbytes = sum(B * (12 * D * (k + 1) + 4 * D) for k in Ks)
+            gbs = nbytes / (a["ms"] * 1e-3) / 1e9
+            result["roofline_accept"] = dict(bound="hbm", kernel="accept_kernel", achieved=gbs, peak=peaks["hbm_gbs"],
+                                             unit="GB/s", frac=gbs / peaks["hbm_gbs"],
+                                             avg_launch_us=1e3 * a["ms"] / a["launches"],
+                                             note="working set of a few MB: launch-latency-bound, not bandwidth-bound")
         else:
             result["roofline"] = dict(bound="alu", kernel="mlp_forward_kernel", achieved=None, peak=None, unit="TFLOP/s",
                                       frac=None, traffic=None, family_ms=fam_ms)
@@ -259,13 +282,21 @@ def run_ours(args):
             s1.reset_stats()
             ts = time_steps(s1, o1, a1, 1, wl1["K"], acc, list(range(100, 164)))
             st1 = s1.stats()
+            s1.reset_stats()
+            s1.profile(1)
+            time_steps(s1, o1, a1, 1, wl1["K"], acc, [100])
+            p1 = s1.profile_read()
+            s1.profile(0)
+            dstep = p1["drafter_cluster"]
+            draft_us = (1e3 * dstep["ms"] / max(s1.stats()["draft_evals"], 1)) if dstep["launches"] else None
             time_steps(s1, o1, a1, 1, 0, acc, [0, 1])
             tv = time_steps(s1, o1, a1, 1, 0, acc, list(range(8)))
             lat = dict(workload="pusht_xfmr B=1 K=8", p50_chunk_ms=float(np.median(ts)), p99_chunk_ms=float(np.percentile(ts, 99)),
                        vanilla_p50_chunk_ms=float(np.median(tv)), speedup_vs_vanilla=float(np.median(tv) / np.median(ts)),
                        acceptance=st1["drafts_accepted"] / max(st1["draft_evals"], 1),
                        base_forwards_per_chunk=st1["env_rounds"] / 64, drafts_per_chunk=st1["draft_evals"] / 64,
-                       nfe_per_chunk=st1["nfe"] / 64)
+                       nfe_per_chunk=st1["nfe"] / 64, drafter="persistent cluster kernel",
+                       drafter_us_per_draft_step=draft_us)
             s1.close()
         cpu = cpu_baseline(wl, budget_s=args.cpu_seconds) if world == 1 else None
         result.update(

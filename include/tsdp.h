@@ -14,6 +14,8 @@
  * Conventions.  All pointers named d_* are DEVICE pointers, h_* are HOST pointers.  Arrays are dense,
  * row-major, fp32 unless stated.  Timestep t in {T-1..0}: a network called with t receives the latent
  * "at t"; the transition at t produces the latent at t-1; the latent at -1 is the clean action chunk.
+ * Kernels of a round are chained with programmatic dependent launch (each may start its prologue while
+ * its predecessor drains); setting the environment variable TSDP_NO_PDL before tsdp_init turns that off.
  * Every function returns a tsdp_status; nothing throws or aborts.  A context is not re-entrant: one
  * call at a time.  There is no CPU fallback: without a CUDA device tsdp_init fails with TSDP_ERR_CUDA.
  */

@@ -76,6 +76,12 @@ __device__ __forceinline__ float posterior_mean(const DdpmTables& S, float x, fl
   return S.c_x0[tau] * x0 + S.c_xt[tau] * x;
 }
 
+// Programmatic dependent launch: a kernel signals early that its successor in the stream may be
+// scheduled, and waits (after whatever set-up touches no shared data) until every kernel it depends on
+// has completed and its memory is visible.  Both are no-ops for a kernel launched without the attribute.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

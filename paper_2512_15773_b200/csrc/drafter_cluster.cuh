@@ -51,7 +51,7 @@ struct DcParams {
 // that fragment loads of 8 consecutive rows fall into different banks.
 struct DcSmem {
   int w_layer;      // bytes of one layer's weight slices
-  int off_h, off_a, off_qkv, off_q2, off_f, off_red, off_kv, off_x, off_posb, off_win, total;
+  int off_h, off_a, off_qkv, off_q2, off_f, off_red, off_kv, off_x, off_posb, off_win, off_par, total;
 };
 __host__ __device__ inline DcSmem dc_smem_plan(int d, int layers, int A) {
   DcSmem p;
@@ -66,10 +66,11 @@ __host__ __device__ inline DcSmem dc_smem_plan(int d, int layers, int A) {
   p.off_q2 = take(DC_ROWS * (d + 8) * 2);
   p.off_f = take(DC_ROWS * (4 * d + 8) * 2);
   p.off_red = take(DC_WARPS * DC_ROWS * 8 * 4);              // one 16 x 8 fp32 tile per warp
-  p.off_kv = take(DC_MAX_NK * 2 * d * 4);
+  p.off_kv = take(layers * DC_MAX_NK * 2 * d * 4);           // keys / values of the memory tokens, every block
   p.off_x = take(DC_ROWS * 16 * 4 * 2);                      // latent and eps, D <= 256
   p.off_posb = take(DC_ROWS * d * 4);
   p.off_win = take(A * d * 4);
+  p.off_par = take((layers * 17 * d + 2 * d + A * d + 16) * 4);   // biases, LayerNorm parameters, head
   p.total = o;
   return p;
 }
@@ -137,7 +138,7 @@ __device__ __forceinline__ void dc_linear(const __nv_bfloat16* X, int px, const 
 
 // LayerNorm of the 16 replicated rows: warp w normalises rows w and w + 8; fp32 in, bf16 out.
 template <int D_MODEL>
-__device__ __forceinline__ void dc_layernorm(const float* h, const float* __restrict__ gam, const float* __restrict__ bet,
+__device__ __forceinline__ void dc_layernorm(const float* h, const float* gam, const float* bet,
                                              __nv_bfloat16* out, int pitch) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr int V = D_MODEL / 128;
@@ -162,7 +163,7 @@ __device__ __forceinline__ void dc_layernorm(const float* h, const float* __rest
 #pragma unroll
     for (int j = 0; j < V; ++j) {
       const int c = j * 128 + lane * 4;
-      const float4 gg = __ldg(reinterpret_cast<const float4*>(gam + c)), bb = __ldg(reinterpret_cast<const float4*>(bet + c));
+      const float4 gg = *reinterpret_cast<const float4*>(gam + c), bb = *reinterpret_cast<const float4*>(bet + c);
       store4(out + row * pitch + c, v[j].x * rstd * gg.x + bb.x, v[j].y * rstd * gg.y + bb.y,
              v[j].z * rstd * gg.z + bb.z, v[j].w * rstd * gg.w + bb.w);
     }
@@ -306,6 +307,7 @@ template <int D_MODEL>
 __global__ void __cluster_dims__(DC_CS, 1, 1) __launch_bounds__(DC_THREADS, 1)
 drafter_cluster_kernel(const __grid_constant__ DcParams P) {
   extern __shared__ __align__(16) uint8_t dc_smem[];
+  pdl_trigger();
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
   const int cid = blockIdx.x / DC_CS, ncl = gridDim.x / DC_CS;
@@ -323,6 +325,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
   float* seps = sx + DC_ROWS * 16;
   float* posb = reinterpret_cast<float*>(dc_smem + pl.off_posb);
   float* win = reinterpret_cast<float*>(dc_smem + pl.off_win);
+  float* par = reinterpret_cast<float*>(dc_smem + pl.off_par);
   const int H = P.H, A = P.A, D = H * A, L = P.layers, NK = 1 + P.To;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -346,6 +349,22 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
     h[i] = 0.f;
   }
   for (int i = threadIdx.x; i < A * d; i += DC_THREADS) win[i] = P.W_in[i];
+  // biases and LayerNorm parameters of every block, then the head: read from shared memory on the critical path
+  for (int l = 0; l < L; ++l) {
+    const DcLayer& G = P.L[l];
+    const float* src[12] = {G.bqkv, G.bo, G.bq2, G.bo2, G.b1, G.b2, G.ln1_g, G.ln1_b, G.ln2_g, G.ln2_b, G.ln3_g, G.ln3_b};
+    const int off[12] = {0, 3 * d, 4 * d, 5 * d, 6 * d, 10 * d, 11 * d, 12 * d, 13 * d, 14 * d, 15 * d, 16 * d};
+    const int len[12] = {3 * d, d, d, d, 4 * d, d, d, d, d, d, d, d};
+    for (int j = 0; j < 12; ++j)
+      for (int i = threadIdx.x; i < len[j]; i += DC_THREADS) par[(size_t)l * 17 * d + off[j] + i] = src[j][i];
+  }
+  float* lnf_g = par + (size_t)L * 17 * d;
+  float* lnf_b = lnf_g + d;
+  float* woutT = lnf_b + d;
+  float* bout = woutT + A * d;
+  for (int i = threadIdx.x; i < d; i += DC_THREADS) { lnf_g[i] = P.lnf_g[i]; lnf_b[i] = P.lnf_b[i]; }
+  for (int i = threadIdx.x; i < A * d; i += DC_THREADS) woutT[i] = P.W_outT[i];
+  for (int i = threadIdx.x; i < A; i += DC_THREADS) bout[i] = P.b_out[i];
   for (int i = threadIdx.x; i < DC_ROWS * PA; i += DC_THREADS) { a[i] = __float2bfloat16_rn(0.f); q2[i] = a[i]; }
   for (int i = threadIdx.x; i < DC_ROWS * PQKV; i += DC_THREADS) qkv[i] = __float2bfloat16_rn(0.f);
   for (int i = threadIdx.x; i < DC_ROWS * PF; i += DC_THREADS) f[i] = __float2bfloat16_rn(0.f);
@@ -359,6 +378,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
     rf[r] = cluster.map_shared_rank(f, r);
   }
   cluster.sync();
+  pdl_wait();      // weights and tables above are constant; t, the latents and the obs K/V come from earlier kernels
 
   const uint64_t seed = *P.seed;
   const size_t ldkv = (size_t)L * 2 * d;
@@ -367,6 +387,12 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
     float* xt_b = P.xt + env * P.xs_b;
     float* mh_b = P.muhat + env * P.ms_b;
     for (int i = threadIdx.x; i < D; i += DC_THREADS) sx[i] = xt_b[i];
+    // keys / values of this environment's observation tokens, every block (slot 0 is the time token)
+    for (int i = threadIdx.x; i < L * P.To * 2 * d; i += DC_THREADS) {
+      const int l = i / (P.To * 2 * d), rem = i % (P.To * 2 * d);
+      const int kx = 1 + rem / (2 * d), c = rem % (2 * d);
+      skv[((size_t)l * DC_MAX_NK + kx) * 2 * d + c] = __ldg(P.kv_obs + ((size_t)env * P.To + (kx - 1)) * ldkv + (size_t)l * 2 * d + c);
+    }
     __syncthreads();
     for (int k = 1; k <= P.K; ++k) {
       const int tau = tb - k + 1;
@@ -378,6 +404,11 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
           }
         continue;
       }
+      // keys / values of the time token of tau, every block
+      for (int i = threadIdx.x; i < L * 2 * d; i += DC_THREADS) {
+        const int l = i / (2 * d), c = i % (2 * d);
+        skv[(size_t)l * DC_MAX_NK * 2 * d + c] = __ldg(P.kv_time + (size_t)tau * ldkv + (size_t)l * 2 * d + c);
+      }
       // token embedding into the residual stream
       for (int i = threadIdx.x; i < DC_ROWS * d; i += DC_THREADS) {
         const int row = i / d, col = i % d;
@@ -388,13 +419,16 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
       }
       __syncthreads();
       for (int l = 0; l < L; ++l) {
-        const DcLayer& W = P.L[l];
+        const float* pb = par + (size_t)l * 17 * d;
+        struct { const float *bqkv, *bo, *bq2, *bo2, *b1, *b2, *ln1_g, *ln1_b, *ln2_g, *ln2_b, *ln3_g, *ln3_b; } W =
+            {pb, pb + 3 * d, pb + 4 * d, pb + 5 * d, pb + 6 * d, pb + 10 * d, pb + 11 * d, pb + 12 * d, pb + 13 * d,
+             pb + 14 * d, pb + 15 * d, pb + 16 * d};
         // ---- causal self-attention
         dc_layernorm<d>(h, W.ln1_g, W.ln1_b, a, PA);
         __syncthreads();
         dc_linear<d>(a, PA, w_ptr(l, 0), NS_3D, red, [&](int row, int col, float* v) {
           const int cg_ = rank * NS_3D + col;
-          const float4 b0 = __ldg(reinterpret_cast<const float4*>(W.bqkv + cg_)), b1 = __ldg(reinterpret_cast<const float4*>(W.bqkv + cg_) + 1);
+          const float4 b0 = *reinterpret_cast<const float4*>(W.bqkv + cg_), b1 = *(reinterpret_cast<const float4*>(W.bqkv + cg_) + 1);
           v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
           const uint4 pk = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
 #pragma unroll
@@ -412,7 +446,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
           const int cg_ = rank * NS_D + col;
           const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
           const float4 h0 = hp[0], h1 = hp[1];
-          const float4 b0 = __ldg(reinterpret_cast<const float4*>(W.bo + cg_)), b1 = __ldg(reinterpret_cast<const float4*>(W.bo + cg_) + 1);
+          const float4 b0 = *reinterpret_cast<const float4*>(W.bo + cg_), b1 = *(reinterpret_cast<const float4*>(W.bo + cg_) + 1);
           const float4 o0 = make_float4(h0.x + v[0] + b0.x, h0.y + v[1] + b0.y, h0.z + v[2] + b0.z, h0.w + v[3] + b0.w);
           const float4 o1 = make_float4(h1.x + v[4] + b1.x, h1.y + v[5] + b1.y, h1.z + v[6] + b1.z, h1.w + v[7] + b1.w);
 #pragma unroll
@@ -421,32 +455,26 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
             dst[0] = o0; dst[1] = o1;
           }
         });
-        // keys / values of the memory tokens for this block: time token of tau, then the obs tokens
-        for (int i = threadIdx.x; i < NK * 2 * d; i += DC_THREADS) {
-          const int kx = i / (2 * d), c = i % (2 * d);
-          const float* src = kx == 0 ? P.kv_time + (size_t)tau * ldkv : P.kv_obs + ((size_t)env * P.To + (kx - 1)) * ldkv;
-          skv[i] = __ldg(src + (size_t)l * 2 * d + c);
-        }
         cluster.sync();
         // ---- cross-attention to [time token | obs tokens]
         dc_layernorm<d>(h, W.ln2_g, W.ln2_b, a, PA);
         __syncthreads();
         dc_linear<d>(a, PA, w_ptr(l, 2), NS_D, red, [&](int row, int col, float* v) {
           const int cg_ = rank * NS_D + col;
-          const float4 b0 = __ldg(reinterpret_cast<const float4*>(W.bq2 + cg_)), b1 = __ldg(reinterpret_cast<const float4*>(W.bq2 + cg_) + 1);
+          const float4 b0 = *reinterpret_cast<const float4*>(W.bq2 + cg_), b1 = *(reinterpret_cast<const float4*>(W.bq2 + cg_) + 1);
           v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
           const uint4 pk = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
 #pragma unroll
           for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(rq2[r] + row * PA + cg_) = pk;
         });
         cluster.sync();
-        dc_attention<d, false>(q2, PA, nullptr, 0, skv, NK, a, PA, P.heads, H);
+        dc_attention<d, false>(q2, PA, nullptr, 0, skv + (size_t)l * DC_MAX_NK * 2 * d, NK, a, PA, P.heads, H);
         __syncthreads();
         dc_linear<d>(a, PA, w_ptr(l, 3), NS_D, red, [&](int row, int col, float* v) {
           const int cg_ = rank * NS_D + col;
           const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
           const float4 h0 = hp[0], h1 = hp[1];
-          const float4 b0 = __ldg(reinterpret_cast<const float4*>(W.bo2 + cg_)), b1 = __ldg(reinterpret_cast<const float4*>(W.bo2 + cg_) + 1);
+          const float4 b0 = *reinterpret_cast<const float4*>(W.bo2 + cg_), b1 = *(reinterpret_cast<const float4*>(W.bo2 + cg_) + 1);
           const float4 o0 = make_float4(h0.x + v[0] + b0.x, h0.y + v[1] + b0.y, h0.z + v[2] + b0.z, h0.w + v[3] + b0.w);
           const float4 o1 = make_float4(h1.x + v[4] + b1.x, h1.y + v[5] + b1.y, h1.z + v[6] + b1.z, h1.w + v[7] + b1.w);
 #pragma unroll
@@ -461,7 +489,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         __syncthreads();
         dc_linear<d>(a, PA, w_ptr(l, 4), NS_4D, red, [&](int row, int col, float* v) {
           const int cg_ = rank * NS_4D + col;
-          const float4 b0 = __ldg(reinterpret_cast<const float4*>(W.b1 + cg_)), b1 = __ldg(reinterpret_cast<const float4*>(W.b1 + cg_) + 1);
+          const float4 b0 = *reinterpret_cast<const float4*>(W.b1 + cg_), b1 = *(reinterpret_cast<const float4*>(W.b1 + cg_) + 1);
           v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
 #pragma unroll
           for (int j = 0; j < 8; ++j)
@@ -475,7 +503,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
           const int cg_ = rank * NS_D + col;
           const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
           const float4 h0 = hp[0], h1 = hp[1];
-          const float4 b0 = __ldg(reinterpret_cast<const float4*>(W.b2 + cg_)), b1 = __ldg(reinterpret_cast<const float4*>(W.b2 + cg_) + 1);
+          const float4 b0 = *reinterpret_cast<const float4*>(W.b2 + cg_), b1 = *(reinterpret_cast<const float4*>(W.b2 + cg_) + 1);
           const float4 o0 = make_float4(h0.x + v[0] + b0.x, h0.y + v[1] + b0.y, h0.z + v[2] + b0.z, h0.w + v[3] + b0.w);
           const float4 o1 = make_float4(h1.x + v[4] + b1.x, h1.y + v[5] + b1.y, h1.z + v[6] + b1.z, h1.w + v[7] + b1.w);
 #pragma unroll
@@ -510,7 +538,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
 #pragma unroll
           for (int j = 0; j < V; ++j) {
             const int c = j * 128 + lane * 4;
-            const float4 gg = __ldg(reinterpret_cast<const float4*>(P.lnf_g + c)), bb = __ldg(reinterpret_cast<const float4*>(P.lnf_b + c));
+            const float4 gg = *reinterpret_cast<const float4*>(lnf_g + c), bb = *reinterpret_cast<const float4*>(lnf_b + c);
             v[j].x = v[j].x * rstd * gg.x + bb.x; v[j].y = v[j].y * rstd * gg.y + bb.y;
             v[j].z = v[j].z * rstd * gg.z + bb.z; v[j].w = v[j].w * rstd * gg.w + bb.w;
           }
@@ -518,11 +546,11 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
             float acc = 0.f;
 #pragma unroll
             for (int j = 0; j < V; ++j) {
-              const float4 w = __ldg(reinterpret_cast<const float4*>(P.W_outT + (size_t)c * d + j * 128 + lane * 4));
+              const float4 w = *reinterpret_cast<const float4*>(woutT + (size_t)c * d + j * 128 + lane * 4);
               acc += v[j].x * w.x + v[j].y * w.y + v[j].z * w.z + v[j].w * w.w;
             }
             acc = warp_sum(acc);
-            if (lane == 0 && row < H) seps[row * A + c] = acc + __ldg(P.b_out + c);
+            if (lane == 0 && row < H) seps[row * A + c] = acc + bout[c];
           }
         }
       }

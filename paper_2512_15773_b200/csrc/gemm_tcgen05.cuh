@@ -232,6 +232,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   static_assert(BN == 32 || BN == 64 || BN == 128 || BN == 256, "BN");
 
   extern __shared__ uint8_t smem_raw[];
+  pdl_trigger();
   const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   constexpr bool TMA_EPI = gemm_tma_epilogue(BN);
   const uint32_t staging = base + STAGES * STAGE_BYTES;    // 1024-byte aligned: every stage is a multiple of 1 KB
@@ -265,6 +266,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_ptr;
   bool ok = true;
+  pdl_wait();      // operands, bias and the output belong to earlier kernels of the stream
 
   if (warp == 0) {
     if (lane == 0) {

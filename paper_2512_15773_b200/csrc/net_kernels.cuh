@@ -13,6 +13,8 @@ namespace tsdp {
 template <int EPI>
 __global__ void __launch_bounds__(256)
 gemm_simt_kernel(const float* __restrict__ A, const float* __restrict__ W, GemmArgs g) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float As[16][65], Ws[16][65];
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
   const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
@@ -56,6 +58,8 @@ gemm_simt_kernel(const float* __restrict__ A, const float* __restrict__ W, GemmA
 // ------------------------------------------------------------------------------------------------
 __global__ void embed_kernel(CandMap cm, const float* __restrict__ W_in, const float* __restrict__ b_in,
                              const float* __restrict__ pos, float* __restrict__ h, int H, int A, int d) {
+  pdl_trigger();
+  pdl_wait();
   const int row = blockIdx.x;
   const int n = row / H, i = row % H;
   const int b = n / cm.C, c = n % cm.C;
@@ -73,6 +77,8 @@ template <typename T>
 __global__ void memtok_kernel(const float* __restrict__ in, int Din, const float* __restrict__ W,
                               const float* __restrict__ bias, const float* __restrict__ cpos, int cpos_mod,
                               int cpos_off, T* __restrict__ out, int d) {
+  pdl_trigger();
+  pdl_wait();
   const int r = blockIdx.x;
   const float* x = in + (size_t)r * Din;
   const float* cp = cpos + (size_t)(cpos_off + (cpos_mod > 0 ? r % cpos_mod : 0)) * d;
@@ -104,6 +110,8 @@ __device__ __forceinline__ void store4(__nv_bfloat16* o, float a, float b, float
 template <typename T, int VEC>
 __global__ void ln_kernel(const float* __restrict__ h, const float* __restrict__ gam, const float* __restrict__ bet,
                           T* __restrict__ out, int M) {
+  pdl_trigger();
+  pdl_wait();
   constexpr int d = VEC * 128;
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
@@ -140,6 +148,8 @@ __global__ void ln_kernel(const float* __restrict__ h, const float* __restrict__
 template <typename T>
 __global__ void self_attn_kernel(const T* __restrict__ qkv, T* __restrict__ out, int n_cand, int H, int d,
                                  int heads) {
+  pdl_trigger();
+  pdl_wait();
   extern __shared__ float sm[];
   const int dh = d / heads;
   const int wpb = blockDim.x >> 5;
@@ -196,6 +206,8 @@ template <typename T>
 __global__ void cross_attn_kernel(const T* __restrict__ q, T* __restrict__ out, const float* __restrict__ kv_time,
                                   const float* __restrict__ kv_obs, CandMap cm, int M, int H, int d, int heads,
                                   int To, int layer, int L, int Tsteps) {
+  pdl_trigger();
+  pdl_wait();
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= M) return;
@@ -257,6 +269,8 @@ template <int DH>
 __global__ void __launch_bounds__(SA_WARPS * 32)
 self_attn_mma_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ out, int n_cand, int H, int d,
                      int heads) {
+  pdl_trigger();
+  pdl_wait();
   constexpr int KS = DH / 16;        // k-steps of Q K^T
   constexpr int NO = DH / 8;         // n-tiles of the output
   constexpr int LDS = DH + 8;        // staging row pitch (elements); keeps 16-byte alignment
@@ -380,6 +394,8 @@ __global__ void __launch_bounds__(256)
 cross_attn_group_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out,
                         const float* __restrict__ kv_time, const float* __restrict__ kv_obs, CandMap cm, int n_cand,
                         int H, int d, int heads, int To, int layer, int L, int Tsteps) {
+  pdl_trigger();
+  pdl_wait();
   constexpr int LG = DH / 8;
   const int gid_raw = (blockIdx.x * blockDim.x + threadIdx.x) / LG;
   const int sub = threadIdx.x % LG;
@@ -457,6 +473,8 @@ template <int VEC>
 __global__ void head_kernel(const float* __restrict__ h, const float* __restrict__ gam, const float* __restrict__ bet,
                             const float* __restrict__ W_outT, const float* __restrict__ b_out, CandMap cm, int M,
                             int H, int A) {
+  pdl_trigger();
+  pdl_wait();
   constexpr int d = VEC * 128;
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
@@ -514,6 +532,8 @@ struct MlpWeights {
 
 __global__ void mlp_forward_kernel(MlpWeights w, CandMap cm, const float* __restrict__ obs, int obs_len, int D,
                                    int Tsteps) {
+  pdl_trigger();
+  pdl_wait();
   extern __shared__ float sm[];
   const int n = blockIdx.x;
   const int b = n / cm.C, c = n % cm.C;
@@ -548,6 +568,8 @@ __global__ void mlp_forward_kernel(MlpWeights w, CandMap cm, const float* __rest
 
 // Closed-form denoiser of iid N(m0, s0^2) data: eps = sqrt(1-abar)(x - sqrt(abar) m0)/(abar s0^2 + 1 - abar).
 __global__ void gauss_forward_kernel(DdpmTables S, float m0, float s0, CandMap cm, int n_cand, int D) {
+  pdl_trigger();
+  pdl_wait();
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (long long)n_cand * D) return;
   const int n = (int)(idx / D), i = (int)(idx % D);

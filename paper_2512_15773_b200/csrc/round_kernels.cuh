@@ -11,6 +11,8 @@ namespace tsdp {
 // [B, Kmax+1, D]; slot 0 is the current latent x.
 __global__ void init_chunk_kernel(float* __restrict__ xt, long long xs_b, int* __restrict__ t, int B, int D,
                                   int T, const uint64_t* __restrict__ seedp, int* __restrict__ round_idx, int* __restrict__ n_done) {
+  pdl_trigger();
+  pdl_wait();
   const uint64_t seed = *seedp;
   const int b = blockIdx.x;
   const int nq = (D + 3) >> 2;
@@ -33,6 +35,8 @@ __global__ void init_chunk_kernel(float* __restrict__ xt, long long xs_b, int* _
 __global__ void draft_step_kernel(DdpmTables S, float* __restrict__ xt, long long xs_b, float* __restrict__ muhat,
                                   long long ms_b, const float* __restrict__ eps_d, const int* __restrict__ t,
                                   int k, int D, const uint64_t* __restrict__ seedp) {
+  pdl_trigger();
+  pdl_wait();
   const uint64_t seed = *seedp;
   const int b = blockIdx.x;
   const int tb = t[b];
@@ -79,6 +83,8 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
                               const int* __restrict__ round_idx, float* __restrict__ actions,
                               int* __restrict__ n_done, DevStats* __restrict__ stats, float draft_nfe,
                               float* __restrict__ dbg_logalpha, int* __restrict__ dbg_jstar) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float s_la[32], s_s1[32], s_s2[32];
   __shared__ int s_acc[32];
   __shared__ int s_j;
@@ -217,6 +223,8 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
 // host can read it.
 __global__ void round_end_kernel(int* __restrict__ round_idx, const int* __restrict__ n_done,
                                  volatile int* __restrict__ host_done) {
+  pdl_trigger();
+  pdl_wait();
   *round_idx += 1;
   *host_done = *n_done;
 }

@@ -5,11 +5,13 @@
 
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <string>
 #include <tuple>
 #include <type_traits>
+#include <utility>
 #include <vector>
 
 #include "../../include/tsdp.h"
@@ -79,6 +81,7 @@ struct tsdp_ctx {
   EncodeTiledFn encode = nullptr;
   cudaStream_t cap_stream = nullptr;
   // persistent cluster drafter: usable for this configuration, shared memory per CTA, clusters that fit the GPU
+  bool pdl = true;                            // programmatic dependent launch between the kernels of a round
   bool dc_ok = false;
   int dc_smem = 0, dc_max_clusters = 0;
   uint64_t rounds = 0, launches = 0;
@@ -116,6 +119,23 @@ int dev_alloc(tsdp_ctx* c, std::vector<void*>& pool, T** p, size_t n) {
 int alloc_bytes(tsdp_ctx* c, std::vector<void*>& pool, void** p, size_t bytes) {
   return dev_alloc<uint8_t>(c, pool, reinterpret_cast<uint8_t**>(p), bytes);
 }
+
+// Every kernel of the round is launched with programmatic stream serialisation: the next kernel of the
+// chain may be scheduled and run its prologue while this one drains; each kernel calls pdl_wait()
+// (griddepcontrol.wait) before it touches memory that its predecessors write or read.
+template <typename... P, typename... A>
+void launch_kernel(tsdp_ctx* c, void (*kern)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, A&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = c->pdl ? 1 : 0;
+  cudaLaunchKernelEx(&cfg, kern, std::forward<A>(args)...);   // a failure is read by cudaGetLastError at the call site
+}
+#define TSDP_LAUNCH(ctx, kern, grid, block, smem, stream, ...) \
+  launch_kernel(ctx, kern, dim3(grid), dim3(block), (size_t)(smem), stream, __VA_ARGS__)
 
 constexpr size_t PROF_CAP = 60000;
 void prof_begin(tsdp_ctx* c, cudaStream_t s, int cat, double flop) {
@@ -189,7 +209,7 @@ int launch_tc(tsdp_ctx* c, const CUtensorMap& ma, const CUtensorMap& mb, const C
   const int tiles = ((g.M + GEMM_BM - 1) / GEMM_BM) * (g.N / BN);
   const int grid = tiles < c->num_sms ? tiles : c->num_sms;
   prof_begin(c, s, c->prof_gemm_cat, 2.0 * g.M * g.N * g.K);
-  gemm_tcgen05_kernel<BN, EPI><<<grid, GEMM_THREADS, gemm_smem_bytes(BN), s>>>(ma, mb, mc, g);
+  TSDP_LAUNCH(c, (gemm_tcgen05_kernel<BN, EPI>), grid, GEMM_THREADS, gemm_smem_bytes(BN), s, ma, mb, mc, g);
   prof_end(c, s);
   c->launches_per_round_tmp++;
   CU_TRY(c, cudaGetLastError());
@@ -243,9 +263,9 @@ int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, in
     const float* w = reinterpret_cast<const float*>(W);
     prof_begin(c, s, c->prof_gemm_cat, 2.0 * M * N * K);
     switch (epi) {
-      case EPI_GELU: gemm_simt_kernel<EPI_GELU><<<grid, 256, 0, s>>>(a, w, g); break;
-      case EPI_RESID: gemm_simt_kernel<EPI_RESID><<<grid, 256, 0, s>>>(a, w, g); break;
-      default: gemm_simt_kernel<EPI_F32><<<grid, 256, 0, s>>>(a, w, g); break;
+      case EPI_GELU: TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_GELU>), grid, 256, 0, s, a, w, g); break;
+      case EPI_RESID: TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_RESID>), grid, 256, 0, s, a, w, g); break;
+      default: TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_F32>), grid, 256, 0, s, a, w, g); break;
     }
     prof_end(c, s);
     c->launches_per_round_tmp++;
@@ -285,14 +305,14 @@ int ln_launch(tsdp_ctx* c, const float* h, const float* g, const float* b, T* ou
   const int grid = (M + wpb - 1) / wpb;
   prof_begin(c, s, 1, 0.0);
   switch (d / 128) {
-    case 1: ln_kernel<T, 1><<<grid, wpb * 32, 0, s>>>(h, g, b, out, M); break;
-    case 2: ln_kernel<T, 2><<<grid, wpb * 32, 0, s>>>(h, g, b, out, M); break;
-    case 3: ln_kernel<T, 3><<<grid, wpb * 32, 0, s>>>(h, g, b, out, M); break;
-    case 4: ln_kernel<T, 4><<<grid, wpb * 32, 0, s>>>(h, g, b, out, M); break;
-    case 5: ln_kernel<T, 5><<<grid, wpb * 32, 0, s>>>(h, g, b, out, M); break;
-    case 6: ln_kernel<T, 6><<<grid, wpb * 32, 0, s>>>(h, g, b, out, M); break;
-    case 7: ln_kernel<T, 7><<<grid, wpb * 32, 0, s>>>(h, g, b, out, M); break;
-    default: ln_kernel<T, 8><<<grid, wpb * 32, 0, s>>>(h, g, b, out, M); break;
+    case 1: TSDP_LAUNCH(c, (ln_kernel<T, 1>), grid, wpb * 32, 0, s, h, g, b, out, M); break;
+    case 2: TSDP_LAUNCH(c, (ln_kernel<T, 2>), grid, wpb * 32, 0, s, h, g, b, out, M); break;
+    case 3: TSDP_LAUNCH(c, (ln_kernel<T, 3>), grid, wpb * 32, 0, s, h, g, b, out, M); break;
+    case 4: TSDP_LAUNCH(c, (ln_kernel<T, 4>), grid, wpb * 32, 0, s, h, g, b, out, M); break;
+    case 5: TSDP_LAUNCH(c, (ln_kernel<T, 5>), grid, wpb * 32, 0, s, h, g, b, out, M); break;
+    case 6: TSDP_LAUNCH(c, (ln_kernel<T, 6>), grid, wpb * 32, 0, s, h, g, b, out, M); break;
+    case 7: TSDP_LAUNCH(c, (ln_kernel<T, 7>), grid, wpb * 32, 0, s, h, g, b, out, M); break;
+    default: TSDP_LAUNCH(c, (ln_kernel<T, 8>), grid, wpb * 32, 0, s, h, g, b, out, M); break;
   }
   prof_end(c, s);
   c->launches_per_round_tmp++;
@@ -304,7 +324,7 @@ int head_launch(tsdp_ctx* c, const Net& n, const CandMap& cm, int M, cudaStream_
   const int wpb = 8;
   const int grid = (M + wpb - 1) / wpb;
   const int H = c->cfg.H, A = c->cfg.A;
-#define HEAD_CASE(V) head_kernel<V><<<grid, wpb * 32, 0, s>>>(c->h, n.lnf_g, n.lnf_b, n.W_outT, n.b_out, cm, M, H, A)
+#define HEAD_CASE(V) TSDP_LAUNCH(c, (head_kernel<V>), grid, wpb * 32, 0, s, c->h, n.lnf_g, n.lnf_b, n.W_outT, n.b_out, cm, M, H, A)
   prof_begin(c, s, 3, 0.0);
   switch (n.cfg.d / 128) {
     case 1: HEAD_CASE(1); break;
@@ -332,17 +352,17 @@ int self_attn_launch(tsdp_ctx* c, const T* qkv, T* out, int n_cand, int H, int d
     const int QT = (H + 15) / 16;
     const int grid = (n_cand * heads * QT + SA_WARPS - 1) / SA_WARPS;
     switch (dh) {
-      case 32: self_attn_mma_kernel<32><<<grid, SA_WARPS * 32, 0, s>>>(qkv, out, n_cand, H, d, heads); break;
-      case 64: self_attn_mma_kernel<64><<<grid, SA_WARPS * 32, 0, s>>>(qkv, out, n_cand, H, d, heads); break;
-      case 96: self_attn_mma_kernel<96><<<grid, SA_WARPS * 32, 0, s>>>(qkv, out, n_cand, H, d, heads); break;
-      default: self_attn_mma_kernel<128><<<grid, SA_WARPS * 32, 0, s>>>(qkv, out, n_cand, H, d, heads); break;
+      case 32: TSDP_LAUNCH(c, (self_attn_mma_kernel<32>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads); break;
+      case 64: TSDP_LAUNCH(c, (self_attn_mma_kernel<64>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads); break;
+      case 96: TSDP_LAUNCH(c, (self_attn_mma_kernel<96>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads); break;
+      default: TSDP_LAUNCH(c, (self_attn_mma_kernel<128>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads); break;
     }
   } else {
     const size_t per_warp = (size_t)(H * dh + 2 * H * (dh + 1)) * sizeof(float);
     int wpb = (int)((200 * 1024) / per_warp);      // the opt-in shared-memory limit set at init
     wpb = wpb > 4 ? 4 : (wpb < 1 ? 1 : wpb);
     const size_t smem = (size_t)wpb * per_warp;
-    self_attn_kernel<T><<<(n_cand * heads + wpb - 1) / wpb, wpb * 32, smem, s>>>(qkv, out, n_cand, H, d, heads);
+    TSDP_LAUNCH(c, (self_attn_kernel<T>), (n_cand * heads + wpb - 1) / wpb, wpb * 32, smem, s, qkv, out, n_cand, H, d, heads);
   }
   prof_end(c, s);
   c->launches_per_round_tmp++;
@@ -363,14 +383,14 @@ int cross_attn_launch(tsdp_ctx* c, const Net& n, const T* q2, T* out, const Cand
     if (1 + To <= CA_MAXNK && (dh == 32 || dh == 64 || dh == 128)) {
       const long long threads = (long long)n_cand * heads * (dh / 8);
       const int grid = (int)((threads + 255) / 256);
-#define CA_CASE(DH) cross_attn_group_kernel<DH><<<grid, 256, 0, s>>>(q2, out, n.kv_time, n.kv_obs, cm, n_cand, H, d, heads, To, layer, L, c->cfg.T)
+#define CA_CASE(DH) TSDP_LAUNCH(c, (cross_attn_group_kernel<DH>), grid, 256, 0, s, q2, out, n.kv_time, n.kv_obs, cm, n_cand, H, d, heads, To, layer, L, c->cfg.T)
       if (dh == 32) CA_CASE(32); else if (dh == 64) CA_CASE(64); else CA_CASE(128);
 #undef CA_CASE
       done = true;
     }
   }
   if (!done)
-    cross_attn_kernel<T><<<(M + 7) / 8, 256, 0, s>>>(q2, out, n.kv_time, n.kv_obs, cm, M, H, d, heads, To, layer, L, c->cfg.T);
+    TSDP_LAUNCH(c, (cross_attn_kernel<T>), (M + 7) / 8, 256, 0, s, q2, out, n.kv_time, n.kv_obs, cm, M, H, d, heads, To, layer, L, c->cfg.T);
   prof_end(c, s);
   c->launches_per_round_tmp++;
   CU_TRY(c, cudaGetLastError());
@@ -388,7 +408,7 @@ int xfmr_forward_t(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStrea
   T* f = reinterpret_cast<T*>(c->f);
   int r;
   prof_begin(c, s, 3, 0.0);
-  embed_kernel<<<M, d < 256 ? d : 256, 0, s>>>(cm, n.W_in, n.b_in, n.pos, c->h, H, A, d);
+  TSDP_LAUNCH(c, (embed_kernel), M, d < 256 ? d : 256, 0, s, cm, n.W_in, n.b_in, n.pos, c->h, H, A, d);
   prof_end(c, s);
   c->launches_per_round_tmp++;
   CU_TRY(c, cudaGetLastError());
@@ -417,7 +437,7 @@ int xfmr_prepare_obs_t(tsdp_ctx* c, Net& n, int B, cudaStream_t s) {
   if (To == 0) return TSDP_OK;
   T* mt = reinterpret_cast<T*>(c->memtok);
   prof_begin(c, s, 3, 0.0);
-  memtok_kernel<T><<<B * To, d < 256 ? d : 256, 0, s>>>(c->obs, c->cfg.obs_dim, n.W_obs, n.b_obs, n.cpos, To, 1, mt, d);
+  TSDP_LAUNCH(c, (memtok_kernel<T>), B * To, d < 256 ? d : 256, 0, s, c->obs, c->cfg.obs_dim, n.W_obs, n.b_obs, n.cpos, To, 1, mt, d);
   prof_end(c, s);
   c->launches_per_round_tmp++;
   CU_TRY(c, cudaGetLastError());
@@ -436,7 +456,7 @@ int forward(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStream_t s) 
     case TSDP_ARCH_GAUSS: {
       const long long tot = (long long)n_cand * D;
       prof_begin(c, s, 5, 0.0);
-      gauss_forward_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, s>>>(c->S, n.m0, n.s0, cm, n_cand, D);
+      TSDP_LAUNCH(c, (gauss_forward_kernel), (unsigned)((tot + 255) / 256), 256, 0, s, c->S, n.m0, n.s0, cm, n_cand, D);
       prof_end(c, s);
       c->launches_per_round_tmp++;
       CU_TRY(c, cudaGetLastError());
@@ -446,7 +466,7 @@ int forward(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStream_t s) 
       int maxw = 0;
       for (int l = 0; l <= n.mlp.n_lin; ++l) maxw = n.mlp.dims[l] > maxw ? n.mlp.dims[l] : maxw;
       prof_begin(c, s, 5, 0.0);
-      mlp_forward_kernel<<<n_cand, 256, 2 * maxw * sizeof(float), s>>>(n.mlp, cm, c->obs, c->cfg.obs_tokens * c->cfg.obs_dim,
+      TSDP_LAUNCH(c, (mlp_forward_kernel), n_cand, 256, 2 * maxw * sizeof(float), s, n.mlp, cm, c->obs, c->cfg.obs_tokens * c->cfg.obs_dim,
                                                                         D, c->cfg.T);
       prof_end(c, s);
       c->launches_per_round_tmp++;
@@ -499,8 +519,8 @@ int launch_cluster_drafter(tsdp_ctx* c, int B, int K, cudaStream_t s) {
   P.t = c->t; P.seed = c->seed; P.B = B; P.K = K;
   const int ncl = B < c->dc_max_clusters ? B : c->dc_max_clusters;
   prof_begin(c, s, 7, 0.0);
-  if (n.cfg.d == 128) drafter_cluster_kernel<128><<<ncl * DC_CS, DC_THREADS, c->dc_smem, s>>>(P);
-  else drafter_cluster_kernel<256><<<ncl * DC_CS, DC_THREADS, c->dc_smem, s>>>(P);
+  if (n.cfg.d == 128) TSDP_LAUNCH(c, (drafter_cluster_kernel<128>), ncl * DC_CS, DC_THREADS, c->dc_smem, s, P);
+  else TSDP_LAUNCH(c, (drafter_cluster_kernel<256>), ncl * DC_CS, DC_THREADS, c->dc_smem, s, P);
   prof_end(c, s);
   c->launches_per_round_tmp++;
   CU_TRY(c, cudaGetLastError());
@@ -522,7 +542,7 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
     c->prof_gemm_cat = 0;
     if (r) return r;
     prof_begin(c, s, 4, 0.0);
-    draft_step_kernel<<<B, 128, 0, s>>>(c->S, c->xt, xs_b, c->muhat, ms_b, c->eps_d, c->t, k, D, c->seed);
+    TSDP_LAUNCH(c, (draft_step_kernel), B, 128, 0, s, c->S, c->xt, xs_b, c->muhat, ms_b, c->eps_d, c->t, k, D, c->seed);
     prof_end(c, s);
     c->launches_per_round_tmp++;
     CU_TRY(c, cudaGetLastError());
@@ -533,11 +553,11 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
   if (warps < 4) warps = 4;
   if (warps > 16) warps = 16;
   prof_begin(c, s, 8, 0.0);
-  accept_kernel<<<B, warps * 32, 0, s>>>(c->S, c->xt, xs_b, c->muhat, ms_b, c->eps, xs_b, c->t, K, D, c->seed, c->sched,
+  TSDP_LAUNCH(c, (accept_kernel), B, warps * 32, 0, s, c->S, c->xt, xs_b, c->muhat, ms_b, c->eps, xs_b, c->t, K, D, c->seed, c->sched,
                                          TSDP_MAX_T + 1, c->round_idx, c->actions, c->n_done, c->stats, c->cfg.draft_nfe,
                                          dbg ? c->dbg_logalpha : nullptr, dbg ? c->dbg_jstar : nullptr);
   prof_end(c, s);
-  round_end_kernel<<<1, 1, 0, s>>>(c->round_idx, c->n_done, c->host_done);
+  TSDP_LAUNCH(c, (round_end_kernel), 1, 1, 0, s, c->round_idx, c->n_done, c->host_done);
   c->launches_per_round_tmp += 2;
   CU_TRY(c, cudaGetLastError());
   return TSDP_OK;
@@ -655,6 +675,7 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   tsdp_ctx* c = new tsdp_ctx();
   c->cfg = *cfg;
   c->D = cfg->H * cfg->A;
+  c->pdl = getenv("TSDP_NO_PDL") == nullptr;
   auto fail = [&](int st) { tsdp_destroy(c); return st; };
 #define INIT_TRY(expr)                                                                    \
   do {                                                                                    \

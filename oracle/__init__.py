@@ -21,5 +21,9 @@ Pin status (what checks each part against something other than itself):
               layer layout are not published); pinned only by structural
               invariants (causality, zero-weight behaviour, a hand-computed
               1-token case) -- see the function headers.
+  sched.py    parity unpinned against the paper (Sec. 3.3 names the three input streams, the
+              separate encoders, the aggregating MLP and the five outputs, but no sizes, weights
+              or ranges); pinned by structure: zero network, output ranges, stream separation,
+              a hand-computed path, the stage boundaries.
   sigma_scale parity unpinned against the paper (formula not given there).
 """

@@ -76,6 +76,21 @@ def make_xfmr_params(seed, H, A, To, Do, d, heads, layers, out_scale=1.0, bf16=T
     return p
 
 
+def make_sched_params(seed, H, A, To, Do, scale=1.0):
+    """Random weights of the scheduler network (three stream encoders 64 / 64 / 16, aggregate MLP
+    64, 5 outputs); fp32-representable.  `scale` multiplies the output layer."""
+    rng = np.random.default_rng(seed)
+    q = lambda a: np.asarray(a, dtype=np.float32).astype(np.float64)
+    p = dict(arch="sched")
+    p["W_o"], p["b_o"] = _lin(rng, To * Do, 64, 1.0 / np.sqrt(max(To * Do, 1)), q)
+    p["W_a"], p["b_a"] = _lin(rng, H * A, 64, 1.0 / np.sqrt(H * A), q)
+    p["W_p"], p["b_p"] = _lin(rng, 1, 16, 1.0, q)
+    p["W_1"], p["b_1"] = _lin(rng, 144, 64, 1.0 / 12.0, q)
+    W, b = _lin(rng, 64, 5, 1.0 / 8.0, q)
+    p["W_2"], p["b_2"] = q(W * scale), q(b * scale)
+    return p
+
+
 def make_obs(seed, B, To, Do):
     """Observation features ~ N(0,1), float32-representable, shape [B, To, Do]."""
     rng = np.random.default_rng(seed + 7919)

@@ -42,7 +42,7 @@ typedef enum {
 } tsdp_status;
 
 enum { TSDP_ARCH_GAUSS = 0, TSDP_ARCH_MLP = 1, TSDP_ARCH_XFMR = 2 };
-enum { TSDP_BASE = 0, TSDP_DRAFT = 1 };
+enum { TSDP_BASE = 0, TSDP_DRAFT = 1, TSDP_SCHED = 2 };
 enum { TSDP_MAX_T = 1024, TSDP_MAX_K = 32 };
 
 /* One denoiser eps = M(x, t; obs).
@@ -120,6 +120,8 @@ size_t tsdp_weights_count(const tsdp_config_t* cfg, int which);
  *          per block: ln1_g, ln1_b, Wqkv [d,3d], bqkv, Wo, bo, ln2_g, ln2_b, Wq2, bq2, Wkv2 [d,2d], bkv2,
  *                     Wo2, bo2, ln3_g, ln3_b, W1 [d,4d], b1, W2 [4d,d], b2;
  *          lnf_g, lnf_b, W_out [d,A], b_out.
+ *   SCHED (which = TSDP_SCHED, the scheduler network of Sec. 3.3, always fp32): W_o [obs_tokens*obs_dim, 64],
+ *          b_o, W_a [H*A, 64], b_a, W_p [1, 16], b_p, W_1 [144, 64], b_1, W_2 [64, 5], b_2.
  * In precision 1 the large matrices are rounded to bf16.  Errors: WEIGHTS (n mismatch), NAN, CUDA. */
 int tsdp_load_weights(tsdp_ctx* ctx, int which, const float* h_blob, size_t n);
 
@@ -127,6 +129,24 @@ int tsdp_load_weights(tsdp_ctx* ctx, int which, const float* h_blob, size_t n);
  * per_round[min(r, n-1)]; n = 0 clears the schedule (every round then uses the arguments of
  * tsdp_sample_chunk).  Stands in for the RL scheduler's output (Sec. 3.3).  HOST arrays, copied. */
 int tsdp_set_schedule(tsdp_ctx* ctx, const int* h_K_per_round, const tsdp_accept_t* h_per_round, int n);
+
+/* Scheduler network (Sec. 3.3 "Temporal-Complexity-Aware Speculative Decoding Scheduler").  Inputs per
+ * environment: its observation, the action chunk sampled for it last time (zeros before the first chunk)
+ * and its task progress in [0, 1]; three stream encoders, an aggregating MLP, five outputs:
+ *   sigma_scale = 1 + 2 sigmoid(y0),  lambda = sigmoid(y1),  K_stage = 1 + rint((max_K - 1) sigmoid(y_{2+stage}))
+ * for the stages early (t >= 4T/5), middle, late (t < T/5).  Sizes and squashing are this library's own;
+ * the paper names the streams, the encoders, the MLP and the outputs only.
+ * While enabled, tsdp_sample_chunk evaluates the network once per chunk (on a side stream, beside the
+ * chunk set-up) and every environment then uses its own sigma_scale, lambda and per-stage draft cap:
+ * K_eff = min(K of the round, K_stage, t).  mode and bonus still come from the `accept` argument.
+ * tsdp_set_scheduler: STATE if no TSDP_SCHED weights are loaded.  tsdp_set_progress copies B HOST floats. */
+int tsdp_set_scheduler(tsdp_ctx* ctx, int enable);
+int tsdp_set_progress(tsdp_ctx* ctx, const float* h_progress, int B);
+/* Evaluate the scheduler network alone (test interface; synchronous).  d_obs [B, obs_tokens, obs_dim] and
+ * d_prev_actions [B, H*A] DEVICE, h_progress [B] HOST; h_params [B, 8] HOST receives
+ * sigma_scale, lambda, K_early, K_mid, K_late, then the three draft counts before rounding. */
+int tsdp_sched_eval(tsdp_ctx* ctx, const float* d_obs, const float* d_prev_actions, const float* h_progress, int B,
+                    float* h_params, void* cuda_stream);
 
 /* Sample one action chunk for each of B environments (the whole hot path: init, rounds until every
  * environment reaches t = -1).  d_obs [B, obs_tokens, obs_dim] and d_actions [B, H, A] are DEVICE

@@ -11,11 +11,12 @@ LIB_PATH = os.path.join(HERE, "libtsdp.so")
 
 TSDP_MAX_T = 1024
 ARCH = {"gauss": 0, "mlp": 1, "xfmr": 2}
-BASE, DRAFT = 0, 1
+BASE, DRAFT, SCHED = 0, 1, 2
 EXPORTS = ["tsdp_init", "tsdp_destroy", "tsdp_strerror", "tsdp_last_error", "tsdp_weights_count",
            "tsdp_load_weights", "tsdp_set_schedule", "tsdp_sample_chunk", "tsdp_sample_chunk_host",
            "tsdp_round", "tsdp_denoise", "tsdp_gemm", "tsdp_gemm_timed", "tsdp_stats", "tsdp_reset_stats",
-           "tsdp_kernel_launches", "tsdp_profile", "tsdp_profile_read", "tsdp_verify_commit_static"]
+           "tsdp_kernel_launches", "tsdp_profile", "tsdp_profile_read", "tsdp_verify_commit_static", "tsdp_set_scheduler", "tsdp_set_progress",
+           "tsdp_sched_eval"]
 PROF_FAMILIES = ["gemm", "layernorm", "attention", "embed_head", "round", "small_net", "gemm_draft", "drafter_cluster", "accept"]
 
 
@@ -77,6 +78,9 @@ def load_library():
     lib.tsdp_gemm_timed.argtypes = [vp, fp, fp, fp, i, i, i, i, fp, i, C.POINTER(C.c_float), vp]
     lib.tsdp_verify_commit_static.argtypes = [i, i, C.c_float, C.c_float, C.c_float, fp, fp, fp, fp, i, i, i,
                                               C.POINTER(AcceptT), u64, C.c_float, fp, fp, fp, fp, vp]
+    lib.tsdp_set_scheduler.argtypes = [vp, i]
+    lib.tsdp_set_progress.argtypes = [vp, fp, i]
+    lib.tsdp_sched_eval.argtypes = [vp, fp, fp, fp, i, fp, vp]
     lib.tsdp_stats.argtypes = [vp, C.POINTER(StatsT)]
     lib.tsdp_reset_stats.argtypes = [vp]
     lib.tsdp_kernel_launches.argtypes = [vp]; lib.tsdp_kernel_launches.restype = u64
@@ -108,6 +112,8 @@ def pack_weights(p):
         parts = []
         for W, b in zip(p["W"], p["b"]):
             parts += [W, b]
+    elif a == "sched":
+        parts = [p[k] for k in ("W_o", "b_o", "W_a", "b_a", "W_p", "b_p", "W_1", "b_1", "W_2", "b_2")]
     elif a == "xfmr":
         parts = [p["W_in"], p["b_in"], p["pos"], p["W_obs"], p["b_obs"], p["cpos"]]
         for L in p["layers"]:
@@ -186,6 +192,20 @@ class Sampler:
         ka = (C.c_int * n)(*Ks)
         aa = (AcceptT * n)(*accepts)
         self._check(self.lib.tsdp_set_schedule(self.h, ka, aa, n), "tsdp_set_schedule")
+
+    def set_scheduler(self, enable):
+        self._check(self.lib.tsdp_set_scheduler(self.h, int(enable)), "tsdp_set_scheduler")
+
+    def set_progress(self, h_progress):
+        a = np.ascontiguousarray(h_progress, dtype=np.float32)
+        self._check(self.lib.tsdp_set_progress(self.h, a.ctypes.data, a.size), "tsdp_set_progress")
+
+    def sched_eval(self, d_obs, d_prev_actions, h_progress, B):
+        prog = np.ascontiguousarray(h_progress, dtype=np.float32)
+        out = np.zeros((B, 8), dtype=np.float32)
+        self._check(self.lib.tsdp_sched_eval(self.h, _ptr(d_obs), _ptr(d_prev_actions), prog.ctypes.data, B,
+                                             out.ctypes.data, 0), "tsdp_sched_eval")
+        return out
 
     def sample_chunk(self, d_obs, B, K, accept, seed, d_actions, stream=0):
         self._check(self.lib.tsdp_sample_chunk(self.h, _ptr(d_obs), B, K, C.byref(accept), seed, _ptr(d_actions),

@@ -124,6 +124,24 @@ struct RoundParams {
   int bonus;
 };
 
+// Per-environment speculative parameters written by the scheduler network (Sec. 3.3: sigma scale,
+// acceptance threshold, draft steps for the early / middle / late denoising stage).
+struct EnvParams {
+  float sigma_scale;
+  float log_lambda;
+  int K[3];
+};
+
+// Denoising stage of timestep t: 0 early (t >= 4T/5), 2 late (t < T/5), 1 in between.
+__device__ __forceinline__ int stage_of(int t, int T) { return t >= (4 * T) / 5 ? 0 : (t < T / 5 ? 2 : 1); }
+
+// Draft steps environment b may take in this round: the round's K, capped by the scheduler's choice.
+__device__ __forceinline__ int env_draft_cap(const EnvParams* envp, int b, int tb, int K, int T) {
+  if (envp == nullptr || tb < 0) return K;
+  const int kb = envp[b].K[stage_of(tb, T)];
+  return kb < K ? kb : K;
+}
+
 // Device-side counters behind tsdp_stats.
 struct DevStats {
   unsigned long long env_rounds, base_evals, draft_evals, drafts_tested, drafts_accepted, rejections,

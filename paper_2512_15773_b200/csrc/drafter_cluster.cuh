@@ -44,6 +44,7 @@ struct DcParams {
   float* muhat; long long ms_b;                              // drafter means [B, Kmax, D]
   const int* t;
   const uint64_t* seed;
+  const EnvParams* envp;                                     // per-environment draft cap, or null
   int B, K;
 };
 
@@ -396,7 +397,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
     __syncthreads();
     for (int k = 1; k <= P.K; ++k) {
       const int tau = tb - k + 1;
-      if (!(tb >= 0 && tau >= 1)) {          // beyond K_eff: carry the latent along (same for every CTA)
+      if (!(tb >= 0 && tau >= 1 && k <= env_draft_cap(P.envp, env, tb, P.K, P.T))) {          // beyond K_eff: carry the latent along (same for every CTA)
         if (rank == 0)
           for (int i = threadIdx.x; i < D; i += DC_THREADS) {
             mh_b[(size_t)(k - 1) * D + i] = sx[i];

@@ -34,14 +34,15 @@ __global__ void init_chunk_kernel(float* __restrict__ xt, long long xs_b, int* _
 // every buffer stays finite.
 __global__ void draft_step_kernel(DdpmTables S, float* __restrict__ xt, long long xs_b, float* __restrict__ muhat,
                                   long long ms_b, const float* __restrict__ eps_d, const int* __restrict__ t,
-                                  int k, int D, const uint64_t* __restrict__ seedp) {
+                                  int k, int D, const uint64_t* __restrict__ seedp, const EnvParams* __restrict__ envp,
+                                  int K, int Tsteps) {
   pdl_trigger();
   pdl_wait();
   const uint64_t seed = *seedp;
   const int b = blockIdx.x;
   const int tb = t[b];
   const int tau = tb - k + 1;
-  const bool valid = (tb >= 0) && (tau >= 1);
+  const bool valid = (tb >= 0) && (tau >= 1) && (k <= env_draft_cap(envp, b, tb, K, Tsteps));
   const float* xp = xt + b * xs_b + (long long)(k - 1) * D;
   float* xn = xt + b * xs_b + (long long)k * D;
   float* mh = muhat + b * ms_b + (long long)(k - 1) * D;
@@ -82,7 +83,8 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
                               const uint64_t* __restrict__ seedp, const RoundParams* __restrict__ sched, int n_sched,
                               const int* __restrict__ round_idx, float* __restrict__ actions,
                               int* __restrict__ n_done, DevStats* __restrict__ stats, float draft_nfe,
-                              float* __restrict__ dbg_logalpha, int* __restrict__ dbg_jstar) {
+                              float* __restrict__ dbg_logalpha, int* __restrict__ dbg_jstar,
+                              const EnvParams* __restrict__ envp) {
   pdl_trigger();
   pdl_wait();
   __shared__ float s_la[32], s_s1[32], s_s2[32];
@@ -96,8 +98,9 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
     return;
   }
   const int r = min(*round_idx, n_sched - 1);
-  const RoundParams rp = sched[r];
-  const int K_eff = min(K, tb);
+  RoundParams rp = sched[r];
+  if (envp) { rp.sigma_scale = envp[b].sigma_scale; rp.log_lambda = envp[b].log_lambda; }   // the scheduler's choice
+  const int K_eff = min(env_draft_cap(envp, b, tb, K, S.T), tb);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nq = (D + 3) >> 2;
   const float* xb = xt + b * xs_b;

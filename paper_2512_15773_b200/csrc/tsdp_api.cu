@@ -20,6 +20,7 @@
 #include "net_kernels.cuh"
 #include "round_kernels.cuh"
 #include "drafter_cluster.cuh"
+#include "sched_kernel.cuh"
 
 using namespace tsdp;
 
@@ -81,6 +82,14 @@ struct tsdp_ctx {
   EncodeTiledFn encode = nullptr;
   cudaStream_t cap_stream = nullptr;
   // persistent cluster drafter: usable for this configuration, shared memory per CTA, clusters that fit the GPU
+  // scheduler network (Sec. 3.3): weights, per-environment outputs, its inputs, the side stream it runs on
+  SchedWeights sched_w{};
+  bool sched_loaded = false, sched_on = false;
+  EnvParams* envp = nullptr;
+  float *progress = nullptr, *sched_dbg = nullptr;
+  std::vector<void*> sched_allocs;
+  cudaStream_t side_stream = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   bool pdl = true;                            // programmatic dependent launch between the kernels of a round
   bool dc_ok = false;
   int dc_smem = 0, dc_max_clusters = 0;
@@ -176,6 +185,12 @@ size_t weights_count(const tsdp_config_t& cfg, const tsdp_net_t& n) {
     return tot + per * n.layers + 2 * d + d * cfg.A + cfg.A;
   }
   return 0;
+}
+
+size_t sched_weights_count(const tsdp_config_t& cfg) {
+  const size_t obs_len = (size_t)cfg.obs_tokens * cfg.obs_dim, D = (size_t)cfg.H * cfg.A;
+  return obs_len * SCHED_HID + SCHED_HID + D * SCHED_HID + SCHED_HID + SCHED_PROG + SCHED_PROG +
+         (size_t)SCHED_CAT * SCHED_HID + SCHED_HID + (size_t)SCHED_HID * SCHED_OUT + SCHED_OUT;
 }
 
 // ------------------------------------------------------------------------------------------ GEMM
@@ -517,6 +532,7 @@ int launch_cluster_drafter(tsdp_ctx* c, int B, int K, cudaStream_t s) {
   P.xt = c->xt; P.xs_b = (long long)(c->cfg.max_K + 1) * c->D;
   P.muhat = c->muhat; P.ms_b = (long long)(c->cfg.max_K > 0 ? c->cfg.max_K : 1) * c->D;
   P.t = c->t; P.seed = c->seed; P.B = B; P.K = K;
+  P.envp = c->sched_on ? c->envp : nullptr;
   const int ncl = B < c->dc_max_clusters ? B : c->dc_max_clusters;
   prof_begin(c, s, 7, 0.0);
   if (n.cfg.d == 128) TSDP_LAUNCH(c, (drafter_cluster_kernel<128>), ncl * DC_CS, DC_THREADS, c->dc_smem, s, P);
@@ -542,7 +558,8 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
     c->prof_gemm_cat = 0;
     if (r) return r;
     prof_begin(c, s, 4, 0.0);
-    TSDP_LAUNCH(c, (draft_step_kernel), B, 128, 0, s, c->S, c->xt, xs_b, c->muhat, ms_b, c->eps_d, c->t, k, D, c->seed);
+    TSDP_LAUNCH(c, (draft_step_kernel), B, 128, 0, s, c->S, c->xt, xs_b, c->muhat, ms_b, c->eps_d, c->t, k, D, c->seed,
+                c->sched_on ? c->envp : nullptr, K, c->cfg.T);
     prof_end(c, s);
     c->launches_per_round_tmp++;
     CU_TRY(c, cudaGetLastError());
@@ -555,7 +572,8 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
   prof_begin(c, s, 8, 0.0);
   TSDP_LAUNCH(c, (accept_kernel), B, warps * 32, 0, s, c->S, c->xt, xs_b, c->muhat, ms_b, c->eps, xs_b, c->t, K, D, c->seed, c->sched,
                                          TSDP_MAX_T + 1, c->round_idx, c->actions, c->n_done, c->stats, c->cfg.draft_nfe,
-                                         dbg ? c->dbg_logalpha : nullptr, dbg ? c->dbg_jstar : nullptr);
+                                         dbg ? c->dbg_logalpha : nullptr, dbg ? c->dbg_jstar : nullptr,
+                                         c->sched_on ? c->envp : nullptr);
   prof_end(c, s);
   TSDP_LAUNCH(c, (round_end_kernel), 1, 1, 0, s, c->round_idx, c->n_done, c->host_done);
   c->launches_per_round_tmp += 2;
@@ -656,6 +674,7 @@ const char* tsdp_strerror(int st) {
 const char* tsdp_last_error(const tsdp_ctx* ctx) { return ctx ? ctx->last_error.c_str() : ""; }
 
 size_t tsdp_weights_count(const tsdp_config_t* cfg, int which) {
+  if (cfg && which == TSDP_SCHED) return sched_weights_count(*cfg);
   if (!cfg || (which != TSDP_BASE && which != TSDP_DRAFT)) return 0;
   const tsdp_net_t& n = which == TSDP_BASE ? cfg->base : cfg->draft;
   if (!net_cfg_ok(*cfg, n)) return 0;
@@ -733,11 +752,17 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   st |= dev_alloc(c, c->allocs, &c->stats, 1);
   st |= dev_alloc(c, c->allocs, &c->dbg_logalpha, B * Km);
   st |= dev_alloc(c, c->allocs, &c->dbg_jstar, B);
+  st |= dev_alloc(c, c->allocs, &c->envp, B);
+  st |= dev_alloc(c, c->allocs, &c->progress, B);
+  st |= dev_alloc(c, c->allocs, &c->sched_dbg, B * 8);
   if (st) return fail(TSDP_ERR_CUDA);
   INIT_TRY(cudaHostAlloc(reinterpret_cast<void**>(&c->host_done), sizeof(int), cudaHostAllocMapped));
   *c->host_done = 0;
   INIT_TRY(cudaHostAlloc(reinterpret_cast<void**>(&c->sched_host), sizeof(RoundParams) * (TSDP_MAX_T + 1), cudaHostAllocDefault));
   INIT_TRY(cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking));
+  INIT_TRY(cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking));
+  INIT_TRY(cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
+  INIT_TRY(cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming));
 
   // transformer workspaces, sized for the larger of (base over all candidates, drafter over B)
   size_t rows_d = 0, rows_4d = 0, mem_rows_d = 0;
@@ -810,10 +835,40 @@ void tsdp_destroy(tsdp_ctx* c) {
   if (c->host_done) cudaFreeHost(c->host_done);
   if (c->sched_host) cudaFreeHost(c->sched_host);
   if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
+  if (c->side_stream) cudaStreamDestroy(c->side_stream);
+  if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+  if (c->ev_join) cudaEventDestroy(c->ev_join);
+  for (void* p : c->sched_allocs) cudaFree(p);
   delete c;
 }
 
+static int load_sched_weights(tsdp_ctx* c, const float* blob, size_t n) {
+  if (n != sched_weights_count(c->cfg)) return TSDP_ERR_WEIGHTS;
+  for (size_t i = 0; i < n; ++i)
+    if (!std::isfinite(blob[i])) return TSDP_ERR_NAN;
+  CU_TRY(c, cudaDeviceSynchronize());
+  for (void* p : c->sched_allocs) cudaFree(p);
+  c->sched_allocs.clear();
+  c->sched_loaded = false;
+  float* d = nullptr;
+  if (dev_alloc(c, c->sched_allocs, &d, n)) return TSDP_ERR_CUDA;
+  CU_TRY(c, cudaMemcpy(d, blob, n * sizeof(float), cudaMemcpyHostToDevice));
+  const size_t obs_len = (size_t)c->cfg.obs_tokens * c->cfg.obs_dim, D = c->D;
+  SchedWeights& w = c->sched_w;
+  w.W_o = d; d += obs_len * SCHED_HID; w.b_o = d; d += SCHED_HID;
+  w.W_a = d; d += D * SCHED_HID; w.b_a = d; d += SCHED_HID;
+  w.W_p = d; d += SCHED_PROG; w.b_p = d; d += SCHED_PROG;
+  w.W_1 = d; d += (size_t)SCHED_CAT * SCHED_HID; w.b_1 = d; d += SCHED_HID;
+  w.W_2 = d; d += (size_t)SCHED_HID * SCHED_OUT; w.b_2 = d;
+  c->sched_loaded = true;
+  return TSDP_OK;
+}
+
 int tsdp_load_weights(tsdp_ctx* c, int which, const float* blob, size_t n) {
+  if (c && blob && which == TSDP_SCHED) {
+    CU_TRY(c, cudaSetDevice(c->cfg.device));
+    return load_sched_weights(c, blob, n);
+  }
   if (!c || !blob || (which != TSDP_BASE && which != TSDP_DRAFT)) return TSDP_ERR_ARG;
   CU_TRY(c, cudaSetDevice(c->cfg.device));
   Net& net = c->net[which];
@@ -982,6 +1037,43 @@ int tsdp_set_schedule(tsdp_ctx* c, const int* Ks, const tsdp_accept_t* accs, int
   return TSDP_OK;
 }
 
+int tsdp_set_scheduler(tsdp_ctx* c, int enable) {
+  if (!c) return TSDP_ERR_ARG;
+  if (enable && !c->sched_loaded) return TSDP_ERR_STATE;
+  CU_TRY(c, cudaSetDevice(c->cfg.device));
+  CU_TRY(c, cudaDeviceSynchronize());
+  // captured rounds carry the pointer to the per-environment parameters (or null): capture again
+  for (auto& g : c->graphs) cudaGraphExecDestroy(g.second);
+  c->graphs.clear();
+  c->sched_on = enable != 0;
+  return TSDP_OK;
+}
+
+int tsdp_set_progress(tsdp_ctx* c, const float* h_progress, int B) {
+  if (!c || !h_progress || B < 1 || B > c->cfg.max_B) return TSDP_ERR_ARG;
+  CU_TRY(c, cudaSetDevice(c->cfg.device));
+  CU_TRY(c, cudaMemcpy(c->progress, h_progress, sizeof(float) * B, cudaMemcpyHostToDevice));
+  return TSDP_OK;
+}
+
+int tsdp_sched_eval(tsdp_ctx* c, const float* d_obs, const float* d_prev_actions, const float* h_progress, int B,
+                    float* h_params, void* stream) {
+  if (!c || !d_prev_actions || !h_progress || !h_params || B < 1 || B > c->cfg.max_B) return TSDP_ERR_ARG;
+  const int obs_len = c->cfg.obs_tokens * c->cfg.obs_dim;
+  if (obs_len > 0 && !d_obs) return TSDP_ERR_ARG;
+  if (!c->sched_loaded) return TSDP_ERR_STATE;
+  CU_TRY(c, cudaSetDevice(c->cfg.device));
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  CU_TRY(c, cudaMemcpyAsync(c->progress, h_progress, sizeof(float) * B, cudaMemcpyHostToDevice, s));
+  sched_mlp_kernel<<<B, 128, 0, s>>>(c->sched_w, d_obs, obs_len, d_prev_actions, c->D, c->progress, c->cfg.max_K, c->envp,
+                                     c->sched_dbg);
+  c->launches++;
+  CU_TRY(c, cudaGetLastError());
+  CU_TRY(c, cudaMemcpyAsync(h_params, c->sched_dbg, sizeof(float) * 8 * B, cudaMemcpyDeviceToHost, s));
+  CU_TRY(c, cudaStreamSynchronize(s));
+  return TSDP_OK;
+}
+
 static int sample_chunk_impl(tsdp_ctx* c, const float* obs, bool obs_on_host, int B, int K, const tsdp_accept_t* acc,
                              uint64_t seed, float* actions, bool actions_on_host, cudaStream_t s) {
   if (!c || !acc || !actions || B < 1 || B > c->cfg.max_B || K < 0 || K > c->cfg.max_K || !accept_ok(acc))
@@ -996,6 +1088,17 @@ static int sample_chunk_impl(tsdp_ctx* c, const float* obs, bool obs_on_host, in
     CU_TRY(c, cudaMemcpyAsync(c->obs, obs, obs_n * sizeof(float), obs_on_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, s));
   CU_TRY(c, cudaMemcpyAsync(c->seed, &seed, sizeof(seed), cudaMemcpyHostToDevice, s));
   if ((r = upload_schedule(c, K, *acc, s, false))) return r;
+  if (c->sched_on) {
+    // the scheduler network reads the new observation, the previous chunk's actions and the progress; it
+    // runs on a side stream beside the chunk set-up and joins before the first round
+    CU_TRY(c, cudaEventRecord(c->ev_fork, s));
+    CU_TRY(c, cudaStreamWaitEvent(c->side_stream, c->ev_fork, 0));
+    sched_mlp_kernel<<<B, 128, 0, c->side_stream>>>(c->sched_w, c->obs, (int)(obs_n / B), c->actions, D, c->progress,
+                                                      c->cfg.max_K, c->envp, nullptr);
+    CU_TRY(c, cudaGetLastError());
+    CU_TRY(c, cudaEventRecord(c->ev_join, c->side_stream));
+    c->launches++;
+  }
   const long long xs_b = (long long)(c->cfg.max_K + 1) * D;
   init_chunk_kernel<<<B, 128, 0, s>>>(c->xt, xs_b, c->t, B, D, T, c->seed, c->round_idx, c->n_done);
   CU_TRY(c, cudaGetLastError());
@@ -1005,6 +1108,7 @@ static int sample_chunk_impl(tsdp_ctx* c, const float* obs, bool obs_on_host, in
   c->launches += 1 + c->launches_per_round_tmp;
   // Rounds.  No environment can finish before the drafted windows could have covered T steps, so the
   // completion flag is only read once that bound is reached.
+  if (c->sched_on) CU_TRY(c, cudaStreamWaitEvent(s, c->ev_join, 0));
   const int n_sched = (int)c->sched_K.size();
   int budget = T;
   for (int round = 0; round <= T; ++round) {
@@ -1309,7 +1413,7 @@ int tsdp_verify_commit_static(int device, int T, float beta0, float beta1, float
   if (warps < 4) warps = 4;
   if (warps > 16) warps = 16;
   accept_kernel<<<B, warps * 32, 0, s>>>(S, d_xt, xs_b, d_muhat, ms_b, d_eps, xs_b, dt, K, D, dseed, drp, 1, dround,
-                                         d_actions, ddone, st, draft_nfe, d_logalpha, dj);
+                                         d_actions, ddone, st, draft_nfe, d_logalpha, dj, nullptr);
   ST_TRY(cudaGetLastError());
   ST_TRY(cudaMemcpyAsync(h_t_new, dt, sizeof(int) * B, cudaMemcpyDeviceToHost, s));
   ST_TRY(cudaMemcpyAsync(h_jstar, dj, sizeof(int) * B, cudaMemcpyDeviceToHost, s));

@@ -42,7 +42,7 @@ def workload_spec(name, batch):
     if batch:
         wl["B"] = batch
     if name == "serving_xfmr":
-        Ks, Ss = inputs.markov_schedule(0, 64)
+        Ks, Ss = inputs.markov_schedule(0, 512)      # long enough for the continuous-batching leg as well
         wl["schedule"] = (Ks, Ss)
         wl["K"] = 10
     return wl
@@ -267,6 +267,24 @@ def run_ours(args):
         else:
             result["roofline"] = dict(bound="alu", kernel="mlp_forward_kernel", achieved=None, peak=None, unit="TFLOP/s",
                                       frac=None, traffic=None, family_ms=fam_ms)
+        # ---- continuous batching: 4 B requests through the same B slots (finished slots refill at once)
+        cont = None
+        if wl["precision"] == 1:
+            Nreq = 4 * B
+            obs_n = torch.tensor(inputs.make_obs(300 + rank, Nreq, wl["To"], wl["Do"]).astype(np.float32), device="cuda")
+            out_n = torch.zeros(Nreq, wl["H"], wl["A"], device="cuda")
+            smp.serve(obs_n, Nreq, B, K, acc, rank_seed(11, rank, -1), out_n)
+            smp.reset_stats()
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record()
+            smp.serve(obs_n, Nreq, B, K, acc, rank_seed(11, rank, 0), out_n)
+            ev1.record()
+            torch.cuda.synchronize()
+            stc = smp.stats()
+            cms = ev0.elapsed_time(ev1)
+            cont = dict(requests=Nreq, slots=B, ms=cms, chunks_per_s=Nreq / (cms / 1e3), batched_rounds=stc["rounds"],
+                        base_forwards_per_chunk=stc["env_rounds"] / Nreq,
+                        gain_over_static_batches=(Nreq / (cms / 1e3)) / (value / world))
         # ---- vanilla 100-step DDPM with the same kernels (K = 0), the latency comparator
         smp.set_schedule([], [])
         v_ms = time_steps(smp, d_obs, out, B, 0, acc, [rank_seed(7, rank, 0)] * 2)[-1]
@@ -305,7 +323,7 @@ def run_ours(args):
             acceptance=acc_steps / max(drafted, 1.0), base_forwards_per_chunk=env_rounds / chunks_total,
             drafts_per_chunk=drafted / chunks_total, nfe_per_chunk=nfe / chunks_total,
             vanilla=vanilla, speedup_vs_vanilla=vanilla["ms_per_step"] / (total_ms / args.steps),
-            latency_b1=lat, e2e=e2e, gpu_launches=int(launches), clocks=clk, cpu_baseline=cpu,
+            latency_b1=lat, continuous_batching=cont, e2e=e2e, gpu_launches=int(launches), clocks=clk, cpu_baseline=cpu,
             config=dict(workload=f"{args.workload} B={B} (config 4: 12L d512 h8 base, 2L d256 drafter, H16 A7, "
                                  f"seeded 3-state Markov K/sigma schedule)" if args.workload == "serving_xfmr"
                         else f"{args.workload} B={B} K={K}",

@@ -157,6 +157,16 @@ int tsdp_sched_eval(tsdp_ctx* ctx, const float* d_obs, const float* d_prev_actio
 int tsdp_sample_chunk(tsdp_ctx* ctx, const float* d_obs, int B, int K, const tsdp_accept_t* accept,
                       uint64_t seed, float* d_actions, void* cuda_stream);
 
+/* Continuous batching: N requests (one action chunk each; d_obs [N, obs_tokens, obs_dim], d_actions [N, H, A],
+ * DEVICE) are worked through `slots` <= max_B batch slots.  A slot whose request reaches t = -1 takes the
+ * next waiting request inside the acceptance kernel (fresh x_T, t = T-1), so no slot idles while work
+ * remains.  Request i draws the noise streams of environment i: its chunk equals the one
+ * tsdp_sample_chunk returns for environment i of a batch of N with the same seed.  Per-request buffers grow
+ * on demand (the only call besides tsdp_init / tsdp_load_weights that may allocate).  With a per-round
+ * schedule the round index counts batched rounds of the whole call.  Errors as tsdp_sample_chunk. */
+int tsdp_serve(tsdp_ctx* ctx, const float* d_obs, int N, int slots, int K, const tsdp_accept_t* accept,
+               uint64_t seed, float* d_actions, void* cuda_stream);
+
 /* The same with HOST buffers: copies h_obs to the device, samples, copies the chunk back. */
 int tsdp_sample_chunk_host(tsdp_ctx* ctx, const float* h_obs, int B, int K, const tsdp_accept_t* accept,
                            uint64_t seed, float* h_actions);

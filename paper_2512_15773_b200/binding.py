@@ -16,7 +16,7 @@ EXPORTS = ["tsdp_init", "tsdp_destroy", "tsdp_strerror", "tsdp_last_error", "tsd
            "tsdp_load_weights", "tsdp_set_schedule", "tsdp_sample_chunk", "tsdp_sample_chunk_host",
            "tsdp_round", "tsdp_denoise", "tsdp_gemm", "tsdp_gemm_timed", "tsdp_stats", "tsdp_reset_stats",
            "tsdp_kernel_launches", "tsdp_profile", "tsdp_profile_read", "tsdp_verify_commit_static", "tsdp_set_scheduler", "tsdp_set_progress",
-           "tsdp_sched_eval"]
+           "tsdp_sched_eval", "tsdp_serve"]
 PROF_FAMILIES = ["gemm", "layernorm", "attention", "embed_head", "round", "small_net", "gemm_draft", "drafter_cluster", "accept"]
 
 
@@ -78,6 +78,7 @@ def load_library():
     lib.tsdp_gemm_timed.argtypes = [vp, fp, fp, fp, i, i, i, i, fp, i, C.POINTER(C.c_float), vp]
     lib.tsdp_verify_commit_static.argtypes = [i, i, C.c_float, C.c_float, C.c_float, fp, fp, fp, fp, i, i, i,
                                               C.POINTER(AcceptT), u64, C.c_float, fp, fp, fp, fp, vp]
+    lib.tsdp_serve.argtypes = [vp, fp, i, i, i, C.POINTER(AcceptT), u64, fp, vp]
     lib.tsdp_set_scheduler.argtypes = [vp, i]
     lib.tsdp_set_progress.argtypes = [vp, fp, i]
     lib.tsdp_sched_eval.argtypes = [vp, fp, fp, fp, i, fp, vp]
@@ -210,6 +211,10 @@ class Sampler:
     def sample_chunk(self, d_obs, B, K, accept, seed, d_actions, stream=0):
         self._check(self.lib.tsdp_sample_chunk(self.h, _ptr(d_obs), B, K, C.byref(accept), seed, _ptr(d_actions),
                                                stream), "tsdp_sample_chunk")
+
+    def serve(self, d_obs, N, slots, K, accept, seed, d_actions, stream=0):
+        self._check(self.lib.tsdp_serve(self.h, _ptr(d_obs), N, slots, K, C.byref(accept), seed, _ptr(d_actions), stream),
+                    "tsdp_serve")
 
     def sample_chunk_host(self, h_obs, B, K, accept, seed, h_actions):
         self._check(self.lib.tsdp_sample_chunk_host(self.h, _ptr(h_obs), B, K, C.byref(accept), seed,

@@ -107,12 +107,15 @@ __device__ __forceinline__ float silu(float v) { return v / (1.0f + __expf(-v));
 
 // Which candidate rows a forward pass covers: candidate n = (env b = n / C, slot c = n % C) reads its
 // latent at xin + b*x_stride_b + c*D, is evaluated at timestep clamp(t[b] - koff - c, 0, T-1) and
-// writes eps at eout + b*e_stride_b + c*D.
+// writes eps at eout + b*e_stride_b + c*D.  b is a slot of the batch; which request (environment-chunk)
+// the slot is working on is item[b].
 struct CandMap {
   const float* xin;  long long x_stride_b;
   float* eout;       long long e_stride_b;
   const int* t;      int C;  int koff;
+  const int* item;   // slot b currently serves request item[b] (its observation, its noise streams); null: b
 };
+__device__ __forceinline__ int item_of(const int* item, int b) { return item ? item[b] : b; }
 
 // Per-round speculative parameters (the scheduler's action space, Sec. 3.3: draft steps, acceptance
 // threshold, sigma scale).
@@ -136,9 +139,9 @@ struct EnvParams {
 __device__ __forceinline__ int stage_of(int t, int T) { return t >= (4 * T) / 5 ? 0 : (t < T / 5 ? 2 : 1); }
 
 // Draft steps environment b may take in this round: the round's K, capped by the scheduler's choice.
-__device__ __forceinline__ int env_draft_cap(const EnvParams* envp, int b, int tb, int K, int T) {
+__device__ __forceinline__ int env_draft_cap(const EnvParams* envp, int env, int tb, int K, int T) {
   if (envp == nullptr || tb < 0) return K;
-  const int kb = envp[b].K[stage_of(tb, T)];
+  const int kb = envp[env].K[stage_of(tb, T)];
   return kb < K ? kb : K;
 }
 

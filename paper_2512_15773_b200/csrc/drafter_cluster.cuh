@@ -44,7 +44,8 @@ struct DcParams {
   float* muhat; long long ms_b;                              // drafter means [B, Kmax, D]
   const int* t;
   const uint64_t* seed;
-  const EnvParams* envp;                                     // per-environment draft cap, or null
+  const EnvParams* envp;                                     // per-request draft cap, or null
+  const int* item;                                           // slot -> request it serves, or null
   int B, K;
 };
 
@@ -383,10 +384,11 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
 
   const uint64_t seed = *P.seed;
   const size_t ldkv = (size_t)L * 2 * d;
-  for (int env = cid; env < P.B; env += ncl) {
-    const int tb = P.t[env];
-    float* xt_b = P.xt + env * P.xs_b;
-    float* mh_b = P.muhat + env * P.ms_b;
+  for (int slot = cid; slot < P.B; slot += ncl) {
+    const int tb = P.t[slot];
+    const int env = item_of(P.item, slot);     // request served by this slot: its noise streams, obs K/V, parameters
+    float* xt_b = P.xt + slot * P.xs_b;
+    float* mh_b = P.muhat + slot * P.ms_b;
     for (int i = threadIdx.x; i < D; i += DC_THREADS) sx[i] = xt_b[i];
     // keys / values of this environment's observation tokens, every block (slot 0 is the time token)
     for (int i = threadIdx.x; i < L * P.To * 2 * d; i += DC_THREADS) {

@@ -218,7 +218,7 @@ __global__ void cross_attn_kernel(const T* __restrict__ q, T* __restrict__ out, 
   const int dh = d / heads;
   const size_t ld = (size_t)L * 2 * d;
   const float* kt = kv_time + (size_t)tau * ld + (size_t)layer * 2 * d;
-  const float* ko = kv_obs + (size_t)b * To * ld + (size_t)layer * 2 * d;
+  const float* ko = kv_obs + (size_t)item_of(cm.item, b) * To * ld + (size_t)layer * 2 * d;
   const float scale = rsqrtf((float)dh);
   const int NK = 1 + To;
   for (int hd = 0; hd < heads; ++hd) {
@@ -411,7 +411,7 @@ cross_attn_group_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __re
 #pragma unroll
   for (int kx = 0; kx < CA_MAXNK; ++kx) {
     if (kx < NK) {
-      const float* kp = (kx == 0 ? kv_time + (size_t)tau * ldkv : kv_obs + ((size_t)b * To + (kx - 1)) * ldkv) +
+      const float* kp = (kx == 0 ? kv_time + (size_t)tau * ldkv : kv_obs + ((size_t)item_of(cm.item, b) * To + (kx - 1)) * ldkv) +
                         (size_t)layer * 2 * d + hd * DH + sub * 8;
       const float4 k0 = __ldg(reinterpret_cast<const float4*>(kp)), k1 = __ldg(reinterpret_cast<const float4*>(kp) + 1);
       const float4 v0 = __ldg(reinterpret_cast<const float4*>(kp + d)), v1 = __ldg(reinterpret_cast<const float4*>(kp + d) + 1);
@@ -548,7 +548,7 @@ __global__ void mlp_forward_kernel(MlpWeights w, CandMap cm, const float* __rest
     float v;
     if (i < D) v = x[i];
     else if (i < D + w.temb) v = w.temb_table[tau * w.temb + (i - D)];
-    else v = obs[(size_t)b * obs_len + (i - D - w.temb)];
+    else v = obs[(size_t)item_of(cm.item, b) * obs_len + (i - D - w.temb)];
     cur[i] = v;
   }
   __syncthreads();

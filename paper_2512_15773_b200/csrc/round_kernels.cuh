@@ -10,7 +10,8 @@ namespace tsdp {
 // x_T ~ N(0, I), t = T-1 for every environment.  xt holds the round's candidate latents
 // [B, Kmax+1, D]; slot 0 is the current latent x.
 __global__ void init_chunk_kernel(float* __restrict__ xt, long long xs_b, int* __restrict__ t, int B, int D,
-                                  int T, const uint64_t* __restrict__ seedp, int* __restrict__ round_idx, int* __restrict__ n_done) {
+                                  int T, const uint64_t* __restrict__ seedp, int* __restrict__ round_idx, int* __restrict__ n_done,
+                                  int* __restrict__ item, int* __restrict__ queue_head) {
   pdl_trigger();
   pdl_wait();
   const uint64_t seed = *seedp;
@@ -25,7 +26,8 @@ __global__ void init_chunk_kernel(float* __restrict__ xt, long long xs_b, int* _
   }
   if (threadIdx.x == 0) {
     t[b] = T - 1;
-    if (b == 0) { *round_idx = 0; *n_done = 0; }
+    item[b] = b;                         // slot b starts on request b; further requests are taken from queue_head on
+    if (b == 0) { *round_idx = 0; *n_done = 0; *queue_head = B; }
   }
 }
 
@@ -35,14 +37,15 @@ __global__ void init_chunk_kernel(float* __restrict__ xt, long long xs_b, int* _
 __global__ void draft_step_kernel(DdpmTables S, float* __restrict__ xt, long long xs_b, float* __restrict__ muhat,
                                   long long ms_b, const float* __restrict__ eps_d, const int* __restrict__ t,
                                   int k, int D, const uint64_t* __restrict__ seedp, const EnvParams* __restrict__ envp,
-                                  int K, int Tsteps) {
+                                  int K, int Tsteps, const int* __restrict__ item) {
   pdl_trigger();
   pdl_wait();
   const uint64_t seed = *seedp;
   const int b = blockIdx.x;
   const int tb = t[b];
   const int tau = tb - k + 1;
-  const bool valid = (tb >= 0) && (tau >= 1) && (k <= env_draft_cap(envp, b, tb, K, Tsteps));
+  const int env = item_of(item, b);      // the request this slot serves: index of its noise streams and parameters
+  const bool valid = (tb >= 0) && (tau >= 1) && (k <= env_draft_cap(envp, env, tb, K, Tsteps));
   const float* xp = xt + b * xs_b + (long long)(k - 1) * D;
   float* xn = xt + b * xs_b + (long long)k * D;
   float* mh = muhat + b * ms_b + (long long)(k - 1) * D;
@@ -50,7 +53,7 @@ __global__ void draft_step_kernel(DdpmTables S, float* __restrict__ xt, long lon
   const int nq = (D + 3) >> 2;
   for (int q = threadIdx.x; q < nq; q += blockDim.x) {
     float z[4] = {0.f, 0.f, 0.f, 0.f};
-    if (valid) normal4(seed, (uint32_t)b, STREAM_XI, (uint32_t)tau, (uint32_t)q, z);
+    if (valid) normal4(seed, (uint32_t)env, STREAM_XI, (uint32_t)tau, (uint32_t)q, z);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int i = 4 * q + j;
@@ -76,7 +79,8 @@ __global__ void draft_step_kernel(DdpmTables S, float* __restrict__ xt, long lon
 //   thread 0: j* = first rejected step (Sec. 3.1 Eq. (3)), statistics.
 //   all threads: commit -- reflection x = mu + (I - 2 e e^T)(x~ - mu^) at j* (Sec. 3.1), or the bonus
 //       base step, or the last draft -- into slot 0; t -= steps; finished chunks go to `actions`.
-// dbg_* may be null.
+// `item` maps the slot to the request it serves (null: the slot index), `queue_head` / `n_items` feed
+// finished slots with waiting requests (null: no refill).  dbg_* may be null.
 __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs_b,
                               const float* __restrict__ muhat, long long ms_b,
                               const float* __restrict__ eps, long long es_b, int* __restrict__ t, int K, int D,
@@ -84,7 +88,8 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
                               const int* __restrict__ round_idx, float* __restrict__ actions,
                               int* __restrict__ n_done, DevStats* __restrict__ stats, float draft_nfe,
                               float* __restrict__ dbg_logalpha, int* __restrict__ dbg_jstar,
-                              const EnvParams* __restrict__ envp) {
+                              const EnvParams* __restrict__ envp, int* __restrict__ item, int* __restrict__ queue_head,
+                              const int* __restrict__ n_items) {
   pdl_trigger();
   pdl_wait();
   __shared__ float s_la[32], s_s1[32], s_s2[32];
@@ -99,8 +104,9 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
   }
   const int r = min(*round_idx, n_sched - 1);
   RoundParams rp = sched[r];
-  if (envp) { rp.sigma_scale = envp[b].sigma_scale; rp.log_lambda = envp[b].log_lambda; }   // the scheduler's choice
-  const int K_eff = min(env_draft_cap(envp, b, tb, K, S.T), tb);
+  const int env = item_of(item, b);      // the request this slot serves
+  if (envp) { rp.sigma_scale = envp[env].sigma_scale; rp.log_lambda = envp[env].log_lambda; }   // the scheduler's choice
+  const int K_eff = min(env_draft_cap(envp, env, tb, K, S.T), tb);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nq = (D + 3) >> 2;
   const float* xb = xt + b * xs_b;
@@ -113,7 +119,7 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
     float s1 = 0.f, s2 = 0.f, d2 = 0.f;
     for (int q = lane; q < nq; q += 32) {
       float z[4];
-      normal4(seed, (uint32_t)b, STREAM_XI, (uint32_t)tau, (uint32_t)q, z);
+      normal4(seed, (uint32_t)env, STREAM_XI, (uint32_t)tau, (uint32_t)q, z);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int i = 4 * q + j;
@@ -130,7 +136,7 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
       const float la = -0.5f * s1 - s2;
       bool acc;
       if (d2 < 1e-30f) acc = true;
-      else if (rp.mode == 0) acc = la >= logf(uniform1(seed, (uint32_t)b, (uint32_t)tau));
+      else if (rp.mode == 0) acc = la >= logf(uniform1(seed, (uint32_t)env, (uint32_t)tau));
       else acc = fminf(0.f, la) >= rp.log_lambda;
       s_la[k - 1] = la; s_s1[k - 1] = s1; s_s2[k - 1] = s2; s_acc[k - 1] = acc ? 1 : 0;
       if (dbg_logalpha) dbg_logalpha[b * K + (k - 1)] = la;
@@ -160,7 +166,7 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
     const float coef = 2.0f * s_s2[j - 1] / (s_s1[j - 1] * rp.sigma_scale * sig);
     for (int q = threadIdx.x; q < nq; q += blockDim.x) {
       float z[4];
-      normal4(seed, (uint32_t)b, STREAM_XI, (uint32_t)tau, (uint32_t)q, z);
+      normal4(seed, (uint32_t)env, STREAM_XI, (uint32_t)tau, (uint32_t)q, z);
 #pragma unroll
       for (int jj = 0; jj < 4; ++jj) {
         const int i = 4 * q + jj;
@@ -169,7 +175,7 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
           const float delta = mb[(long long)(j - 1) * D + i] - mu;
           const float v = mu + sig * (z[jj] - coef * delta);
           xo[i] = v;
-          if (t_new < 0) actions[(long long)b * D + i] = v;
+          if (t_new < 0) actions[(long long)env * D + i] = v;
         }
       }
     }
@@ -178,7 +184,7 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
     const float sig = S.sigma[tau];
     for (int q = threadIdx.x; q < nq; q += blockDim.x) {
       float z[4] = {0.f, 0.f, 0.f, 0.f};
-      if (tau > 0) normal4(seed, (uint32_t)b, STREAM_XI, (uint32_t)tau, (uint32_t)q, z);
+      if (tau > 0) normal4(seed, (uint32_t)env, STREAM_XI, (uint32_t)tau, (uint32_t)q, z);
 #pragma unroll
       for (int jj = 0; jj < 4; ++jj) {
         const int i = 4 * q + jj;
@@ -186,7 +192,7 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
           const float mu = posterior_mean(S, xb[(long long)K_eff * D + i], eb[(long long)K_eff * D + i], tau);
           const float v = mu + sig * z[jj];
           xo[i] = v;
-          if (t_new < 0) actions[(long long)b * D + i] = v;
+          if (t_new < 0) actions[(long long)env * D + i] = v;
         }
       }
     }
@@ -194,7 +200,7 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
     for (int i = threadIdx.x; i < D; i += blockDim.x) {
       const float v = xb[(long long)K_eff * D + i];
       xo[i] = v;
-      if (t_new < 0) actions[(long long)b * D + i] = v;
+      if (t_new < 0) actions[(long long)env * D + i] = v;
     }
   }
   if (threadIdx.x == 0) {
@@ -218,6 +224,25 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
     if (t_new < 0) {
       atomicAdd(&stats->chunks_done, 1ull);
       atomicAdd(n_done, 1);
+    }
+  }
+  // Continuous batching: a slot whose request has finished takes the next waiting request, if any --
+  // fresh x_T ~ N(0, I) from that request's own noise stream, t = T - 1.
+  if (t_new < 0 && queue_head != nullptr) {
+    __shared__ int s_next;
+    __syncthreads();                       // the committed latent above has been written and read
+    if (threadIdx.x == 0) s_next = atomicAdd(queue_head, 1);
+    __syncthreads();
+    const int next = s_next;
+    if (next < *n_items) {
+      for (int q = threadIdx.x; q < nq; q += blockDim.x) {
+        float z[4];
+        normal4(seed, (uint32_t)next, STREAM_INIT, 0u, (uint32_t)q, z);
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj)
+          if (4 * q + jj < D) xo[4 * q + jj] = z[jj];
+      }
+      if (threadIdx.x == 0) { item[b] = next; t[b] = S.T - 1; }
     }
   }
 }

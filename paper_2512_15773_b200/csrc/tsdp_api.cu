@@ -62,6 +62,10 @@ struct tsdp_ctx {
   // round state
   float *xt = nullptr, *muhat = nullptr, *eps = nullptr, *eps_d = nullptr, *actions = nullptr, *obs = nullptr;
   int* t = nullptr;
+  // continuous batching: slot -> request it serves, next waiting request, number of requests, capacity of the
+  // per-request buffers (obs, actions, obs K/V, scheduler outputs)
+  int *item = nullptr, *queue_head = nullptr, *n_items = nullptr;
+  size_t items_cap = 0;
   uint64_t* seed = nullptr;
   int *round_idx = nullptr, *n_done = nullptr, *status = nullptr;
   int* host_done = nullptr;                   // mapped pinned
@@ -533,6 +537,7 @@ int launch_cluster_drafter(tsdp_ctx* c, int B, int K, cudaStream_t s) {
   P.muhat = c->muhat; P.ms_b = (long long)(c->cfg.max_K > 0 ? c->cfg.max_K : 1) * c->D;
   P.t = c->t; P.seed = c->seed; P.B = B; P.K = K;
   P.envp = c->sched_on ? c->envp : nullptr;
+  P.item = c->item;
   const int ncl = B < c->dc_max_clusters ? B : c->dc_max_clusters;
   prof_begin(c, s, 7, 0.0);
   if (n.cfg.d == 128) TSDP_LAUNCH(c, (drafter_cluster_kernel<128>), ncl * DC_CS, DC_THREADS, c->dc_smem, s, P);
@@ -552,19 +557,19 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
   const bool cluster_draft = K > 0 && use_cluster_drafter(c, B);
   if (cluster_draft && (r = launch_cluster_drafter(c, B, K, s))) return r;
   for (int k = 1; k <= K && !cluster_draft; ++k) {
-    CandMap cm{c->xt + (long long)(k - 1) * D, xs_b, c->eps_d, (long long)D, c->t, 1, k - 1};
+    CandMap cm{c->xt + (long long)(k - 1) * D, xs_b, c->eps_d, (long long)D, c->t, 1, k - 1, c->item};
     c->prof_gemm_cat = 6;
     r = forward(c, c->net[TSDP_DRAFT], cm, B, s);
     c->prof_gemm_cat = 0;
     if (r) return r;
     prof_begin(c, s, 4, 0.0);
     TSDP_LAUNCH(c, (draft_step_kernel), B, 128, 0, s, c->S, c->xt, xs_b, c->muhat, ms_b, c->eps_d, c->t, k, D, c->seed,
-                c->sched_on ? c->envp : nullptr, K, c->cfg.T);
+                c->sched_on ? c->envp : nullptr, K, c->cfg.T, c->item);
     prof_end(c, s);
     c->launches_per_round_tmp++;
     CU_TRY(c, cudaGetLastError());
   }
-  CandMap cv{c->xt, xs_b, c->eps, xs_b, c->t, K + 1, 0};
+  CandMap cv{c->xt, xs_b, c->eps, xs_b, c->t, K + 1, 0, c->item};
   if ((r = forward(c, c->net[TSDP_BASE], cv, B * (K + 1), s))) return r;
   int warps = K < 1 ? 1 : K;
   if (warps < 4) warps = 4;
@@ -573,7 +578,7 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
   TSDP_LAUNCH(c, (accept_kernel), B, warps * 32, 0, s, c->S, c->xt, xs_b, c->muhat, ms_b, c->eps, xs_b, c->t, K, D, c->seed, c->sched,
                                          TSDP_MAX_T + 1, c->round_idx, c->actions, c->n_done, c->stats, c->cfg.draft_nfe,
                                          dbg ? c->dbg_logalpha : nullptr, dbg ? c->dbg_jstar : nullptr,
-                                         c->sched_on ? c->envp : nullptr);
+                                         c->sched_on ? c->envp : nullptr, c->item, c->queue_head, c->n_items);
   prof_end(c, s);
   TSDP_LAUNCH(c, (round_end_kernel), 1, 1, 0, s, c->round_idx, c->n_done, c->host_done);
   c->launches_per_round_tmp += 2;
@@ -752,6 +757,10 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   st |= dev_alloc(c, c->allocs, &c->stats, 1);
   st |= dev_alloc(c, c->allocs, &c->dbg_logalpha, B * Km);
   st |= dev_alloc(c, c->allocs, &c->dbg_jstar, B);
+  st |= dev_alloc(c, c->allocs, &c->item, B);
+  st |= dev_alloc(c, c->allocs, &c->queue_head, 1);
+  st |= dev_alloc(c, c->allocs, &c->n_items, 1);
+  c->items_cap = B;
   st |= dev_alloc(c, c->allocs, &c->envp, B);
   st |= dev_alloc(c, c->allocs, &c->progress, B);
   st |= dev_alloc(c, c->allocs, &c->sched_dbg, B * 8);
@@ -1006,7 +1015,7 @@ int tsdp_load_weights(tsdp_ctx* c, int which, const float* blob, size_t n) {
     if (dev_alloc(c, net.allocs, &net.bkv_all, L * 2 * d)) return TSDP_ERR_CUDA;
     CU_TRY(c, cudaMemcpy(net.bkv_all, bkv_all.data(), bkv_all.size() * sizeof(float), cudaMemcpyHostToDevice));
     if (dev_alloc(c, net.allocs, &net.kv_time, (size_t)T * L * 2 * d)) return TSDP_ERR_CUDA;
-    if (dev_alloc(c, net.allocs, &net.kv_obs, (size_t)cfg.max_B * (To ? To : 1) * L * 2 * d)) return TSDP_ERR_CUDA;
+    if (dev_alloc(c, net.allocs, &net.kv_obs, c->items_cap * (To ? To : 1) * L * 2 * d)) return TSDP_ERR_CUDA;
     if ((r = sinus_table((int)d, &net.temb_table))) return r;
     // keys/values of the time token for every timestep: (sinusoidal(tau) + cpos[0]) Wkv2 + bkv2, all blocks
     c->launches_per_round_tmp = 0;
@@ -1037,6 +1046,8 @@ int tsdp_set_schedule(tsdp_ctx* c, const int* Ks, const tsdp_accept_t* accs, int
   return TSDP_OK;
 }
 
+static int ensure_items(tsdp_ctx* c, size_t N);
+
 int tsdp_set_scheduler(tsdp_ctx* c, int enable) {
   if (!c) return TSDP_ERR_ARG;
   if (enable && !c->sched_loaded) return TSDP_ERR_STATE;
@@ -1050,8 +1061,9 @@ int tsdp_set_scheduler(tsdp_ctx* c, int enable) {
 }
 
 int tsdp_set_progress(tsdp_ctx* c, const float* h_progress, int B) {
-  if (!c || !h_progress || B < 1 || B > c->cfg.max_B) return TSDP_ERR_ARG;
+  if (!c || !h_progress || B < 1) return TSDP_ERR_ARG;
   CU_TRY(c, cudaSetDevice(c->cfg.device));
+  { int r = ensure_items(c, (size_t)B); if (r) return r; }
   CU_TRY(c, cudaMemcpy(c->progress, h_progress, sizeof(float) * B, cudaMemcpyHostToDevice));
   return TSDP_OK;
 }
@@ -1074,54 +1086,88 @@ int tsdp_sched_eval(tsdp_ctx* c, const float* d_obs, const float* d_prev_actions
   return TSDP_OK;
 }
 
-static int sample_chunk_impl(tsdp_ctx* c, const float* obs, bool obs_on_host, int B, int K, const tsdp_accept_t* acc,
+// Grow the per-request buffers (observations, actions, obs-token K/V, scheduler inputs and outputs) to hold
+// N requests.  Captured graphs and tensor maps carry the old addresses, so they are dropped.
+static int ensure_items(tsdp_ctx* c, size_t N) {
+  if (N <= c->items_cap) return TSDP_OK;
+  CU_TRY(c, cudaDeviceSynchronize());
+  const tsdp_config_t& cfg = c->cfg;
+  const size_t D = c->D, To = cfg.obs_tokens;
+  int st = 0;
+  st |= dev_alloc(c, c->allocs, &c->actions, N * D);
+  st |= dev_alloc(c, c->allocs, &c->obs, N * To * cfg.obs_dim + 1);
+  st |= dev_alloc(c, c->allocs, &c->envp, N);
+  st |= dev_alloc(c, c->allocs, &c->progress, N);
+  st |= dev_alloc(c, c->allocs, &c->sched_dbg, N * 8);
+  size_t dmax = 0;
+  for (int w = 0; w < 2; ++w) {
+    Net& n = c->net[w];
+    if (n.cfg.arch != TSDP_ARCH_XFMR) continue;
+    dmax = std::max(dmax, (size_t)n.cfg.d);
+    if (n.loaded) st |= dev_alloc(c, n.allocs, &n.kv_obs, N * (To ? To : 1) * n.cfg.layers * 2 * n.cfg.d);
+  }
+  if (dmax) st |= alloc_bytes(c, c->allocs, &c->memtok, std::max((size_t)cfg.T, N * To) * dmax * (cfg.precision == 0 ? 4 : 2));
+  if (st) return TSDP_ERR_CUDA;
+  c->items_cap = N;
+  for (auto& g : c->graphs) cudaGraphExecDestroy(g.second);
+  c->graphs.clear();
+  c->maps.clear();
+  return TSDP_OK;
+}
+
+static int sample_chunk_impl(tsdp_ctx* c, const float* obs, bool obs_on_host, int N, int B, int K, const tsdp_accept_t* acc,
                              uint64_t seed, float* actions, bool actions_on_host, cudaStream_t s) {
-  if (!c || !acc || !actions || B < 1 || B > c->cfg.max_B || K < 0 || K > c->cfg.max_K || !accept_ok(acc))
+  // N requests (environment-chunks) through B slots; N == B is the plain batch
+  if (!c || !acc || !actions || B < 1 || B > c->cfg.max_B || N < B || K < 0 || K > c->cfg.max_K || !accept_ok(acc))
     return TSDP_ERR_ARG;
-  const size_t obs_n = (size_t)B * c->cfg.obs_tokens * c->cfg.obs_dim;
+  const size_t obs_n = (size_t)N * c->cfg.obs_tokens * c->cfg.obs_dim;
   if (obs_n > 0 && !obs) return TSDP_ERR_ARG;
   if (!c->net[0].loaded || !c->net[1].loaded) return TSDP_ERR_STATE;
   CU_TRY(c, cudaSetDevice(c->cfg.device));
   const int D = c->D, T = c->cfg.T;
   int r;
+  if ((r = ensure_items(c, (size_t)N))) return r;
   if (obs_n)
     CU_TRY(c, cudaMemcpyAsync(c->obs, obs, obs_n * sizeof(float), obs_on_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, s));
   CU_TRY(c, cudaMemcpyAsync(c->seed, &seed, sizeof(seed), cudaMemcpyHostToDevice, s));
+  CU_TRY(c, cudaMemcpyAsync(c->n_items, &N, sizeof(int), cudaMemcpyHostToDevice, s));
   if ((r = upload_schedule(c, K, *acc, s, false))) return r;
   if (c->sched_on) {
     // the scheduler network reads the new observation, the previous chunk's actions and the progress; it
     // runs on a side stream beside the chunk set-up and joins before the first round
     CU_TRY(c, cudaEventRecord(c->ev_fork, s));
     CU_TRY(c, cudaStreamWaitEvent(c->side_stream, c->ev_fork, 0));
-    sched_mlp_kernel<<<B, 128, 0, c->side_stream>>>(c->sched_w, c->obs, (int)(obs_n / B), c->actions, D, c->progress,
+    sched_mlp_kernel<<<N, 128, 0, c->side_stream>>>(c->sched_w, c->obs, (int)(obs_n / N), c->actions, D, c->progress,
                                                       c->cfg.max_K, c->envp, nullptr);
     CU_TRY(c, cudaGetLastError());
     CU_TRY(c, cudaEventRecord(c->ev_join, c->side_stream));
     c->launches++;
   }
   const long long xs_b = (long long)(c->cfg.max_K + 1) * D;
-  init_chunk_kernel<<<B, 128, 0, s>>>(c->xt, xs_b, c->t, B, D, T, c->seed, c->round_idx, c->n_done);
+  init_chunk_kernel<<<B, 128, 0, s>>>(c->xt, xs_b, c->t, B, D, T, c->seed, c->round_idx, c->n_done, c->item, c->queue_head);
   CU_TRY(c, cudaGetLastError());
   c->launches_per_round_tmp = 0;
-  if ((r = prepare_obs(c, c->net[TSDP_BASE], B, s))) return r;
-  if ((r = prepare_obs(c, c->net[TSDP_DRAFT], B, s))) return r;
+  if ((r = prepare_obs(c, c->net[TSDP_BASE], N, s))) return r;
+  if ((r = prepare_obs(c, c->net[TSDP_DRAFT], N, s))) return r;
   c->launches += 1 + c->launches_per_round_tmp;
-  // Rounds.  No environment can finish before the drafted windows could have covered T steps, so the
-  // completion flag is only read once that bound is reached.
+  // Rounds.  A request cannot finish before its drafted windows could have covered T steps, so the
+  // completion flag is only read once the slots could have worked through all N requests.
   if (c->sched_on) CU_TRY(c, cudaStreamWaitEvent(s, c->ev_join, 0));
   const int n_sched = (int)c->sched_K.size();
-  int budget = T;
-  for (int round = 0; round <= T; ++round) {
+  const long long waves = ((long long)N + B - 1) / B;
+  long long budget = (long long)T * N / B;
+  const long long max_rounds = (long long)(T + 1) * waves + 1;
+  for (long long round = 0; round < max_rounds; ++round) {
     const int Kr = n_sched > 0 ? c->sched_K[round < n_sched ? round : n_sched - 1] : K;
     if ((r = run_round(c, B, Kr, s))) return r;
     c->rounds++;
     budget -= Kr + 1;
     if (budget <= 0) {
       CU_TRY(c, cudaStreamSynchronize(s));
-      if (*c->host_done >= B) break;
+      if (*c->host_done >= N) break;
     }
   }
-  CU_TRY(c, cudaMemcpyAsync(actions, c->actions, (size_t)B * D * sizeof(float),
+  CU_TRY(c, cudaMemcpyAsync(actions, c->actions, (size_t)N * D * sizeof(float),
                             actions_on_host ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice, s));
   CU_TRY(c, cudaStreamSynchronize(s));
   return check_status(c);
@@ -1129,12 +1175,18 @@ static int sample_chunk_impl(tsdp_ctx* c, const float* obs, bool obs_on_host, in
 
 int tsdp_sample_chunk(tsdp_ctx* c, const float* d_obs, int B, int K, const tsdp_accept_t* acc, uint64_t seed,
                       float* d_actions, void* stream) {
-  return sample_chunk_impl(c, d_obs, false, B, K, acc, seed, d_actions, false, reinterpret_cast<cudaStream_t>(stream));
+  return sample_chunk_impl(c, d_obs, false, B, B, K, acc, seed, d_actions, false, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int tsdp_serve(tsdp_ctx* c, const float* d_obs, int N, int slots, int K, const tsdp_accept_t* acc, uint64_t seed,
+               float* d_actions, void* stream) {
+  if (c && slots > N) slots = N;
+  return sample_chunk_impl(c, d_obs, false, N, slots, K, acc, seed, d_actions, false, reinterpret_cast<cudaStream_t>(stream));
 }
 
 int tsdp_sample_chunk_host(tsdp_ctx* c, const float* h_obs, int B, int K, const tsdp_accept_t* acc, uint64_t seed,
                            float* h_actions) {
-  return sample_chunk_impl(c, h_obs, true, B, K, acc, seed, h_actions, true, nullptr);
+  return sample_chunk_impl(c, h_obs, true, B, B, K, acc, seed, h_actions, true, nullptr);
 }
 
 int tsdp_round(tsdp_ctx* c, const float* d_obs, int B, int K, const tsdp_accept_t* acc, uint64_t seed, float* d_x,
@@ -1156,6 +1208,13 @@ int tsdp_round(tsdp_ctx* c, const float* d_obs, int B, int K, const tsdp_accept_
   if ((r = upload_schedule(c, K, *acc, s, true))) return r;
   CU_TRY(c, cudaMemsetAsync(c->round_idx, 0, sizeof(int), s));
   CU_TRY(c, cudaMemsetAsync(c->n_done, 0, sizeof(int), s));
+  {   // every slot serves the request of its own index and nothing is waiting
+    std::vector<int> ident(B);
+    for (int b = 0; b < B; ++b) ident[b] = b;
+    CU_TRY(c, cudaMemcpyAsync(c->item, ident.data(), sizeof(int) * B, cudaMemcpyHostToDevice, s));
+    CU_TRY(c, cudaMemcpyAsync(c->queue_head, &B, sizeof(int), cudaMemcpyHostToDevice, s));
+    CU_TRY(c, cudaMemcpyAsync(c->n_items, &B, sizeof(int), cudaMemcpyHostToDevice, s));
+  }
   CU_TRY(c, cudaMemcpyAsync(c->t, h_t, sizeof(int) * B, cudaMemcpyHostToDevice, s));
   CU_TRY(c, cudaMemcpy2DAsync(c->xt, K1 * D * sizeof(float), d_x, D * sizeof(float), D * sizeof(float), B, cudaMemcpyDeviceToDevice, s));
   c->launches_per_round_tmp = 0;
@@ -1203,7 +1262,7 @@ int tsdp_denoise(tsdp_ctx* c, int which, const float* d_x, const int* h_tau, con
   CU_TRY(c, cudaMemcpyAsync(c->t, h_tau, sizeof(int) * N, cudaMemcpyHostToDevice, s));
   c->launches_per_round_tmp = 0;
   if ((r = prepare_obs(c, n, N, s))) return r;
-  CandMap cm{d_x, (long long)c->D, d_eps, (long long)c->D, c->t, 1, 0};
+  CandMap cm{d_x, (long long)c->D, d_eps, (long long)c->D, c->t, 1, 0, nullptr};
   if ((r = forward(c, n, cm, N, s))) return r;
   c->launches += c->launches_per_round_tmp;
   CU_TRY(c, cudaStreamSynchronize(s));
@@ -1413,7 +1472,7 @@ int tsdp_verify_commit_static(int device, int T, float beta0, float beta1, float
   if (warps < 4) warps = 4;
   if (warps > 16) warps = 16;
   accept_kernel<<<B, warps * 32, 0, s>>>(S, d_xt, xs_b, d_muhat, ms_b, d_eps, xs_b, dt, K, D, dseed, drp, 1, dround,
-                                         d_actions, ddone, st, draft_nfe, d_logalpha, dj, nullptr);
+                                         d_actions, ddone, st, draft_nfe, d_logalpha, dj, nullptr, nullptr, nullptr, nullptr);
   ST_TRY(cudaGetLastError());
   ST_TRY(cudaMemcpyAsync(h_t_new, dt, sizeof(int) * B, cudaMemcpyDeviceToHost, s));
   ST_TRY(cudaMemcpyAsync(h_jstar, dj, sizeof(int) * B, cudaMemcpyDeviceToHost, s));

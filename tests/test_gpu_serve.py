@@ -1,0 +1,87 @@
+"""Continuous batching (tsdp_serve): N requests through fewer slots give, request by request, the
+chunks of one big batch -- the refill inside the acceptance kernel changes scheduling, not results."""
+import numpy as np
+import pytest
+import torch
+from scipy import stats
+
+from oracle import spec
+from paper_2512_15773_b200 import binding, inputs
+from tests import helpers as hp
+
+pytestmark = pytest.mark.gpu
+
+
+def _serve_vs_batch(wl, N, slots, K, acc, seed, drafter=0, precision=None):
+    smp, S, base, draft = hp.setup(wl, max_B=N, max_K=max(K, 1), precision=precision, drafter=drafter)
+    obs = inputs.make_obs(8, N, wl["To"], wl["Do"])
+    dobs = torch.tensor(obs, dtype=torch.float32, device="cuda")
+    ref = torch.zeros(N, wl["H"], wl["A"], device="cuda")
+    smp.reset_stats()
+    smp.sample_chunk(dobs, N, K, acc, seed, ref)
+    st_ref = smp.stats()
+    out = torch.full_like(ref, float("nan"))
+    smp.reset_stats()
+    smp.serve(dobs, N, slots, K, acc, seed, out)
+    st = smp.stats()
+    assert st["chunks"] == N and st["steps_advanced"] == 100 * N
+    assert torch.equal(out, ref)
+    # per-request work is identical; only the number of batched rounds differs
+    for k in ("env_rounds", "draft_evals", "drafts_accepted", "rejections", "bonus_steps"):
+        assert st[k] == st_ref[k], k
+    smp.close()
+    return obs, ref.cpu().numpy(), (S, base, draft), st, st_ref
+
+
+def test_serve_toy_mlp_fp32_equals_batch_and_oracle():
+    wl = dict(inputs.WORKLOADS["toy_mlp"])
+    N, slots, K, seed = 20, 6, 4, 17
+    obs, got, (S, base, draft), st, st_ref = _serve_vs_batch(wl, N, slots, K, hp.accept_t(), seed)
+    # a late request against the oracle: request i uses the noise streams of environment i
+    n_match = 0
+    for i in (0, 7, 13, 19):
+        xo, _ = spec.sample_chunk(S, base, draft, spec.PhiloxNoise(seed), i, obs[i], (wl["H"], wl["A"]), K, spec.Accept())
+        n_match += np.max(np.abs(got[i] - xo)) < 3e-2
+    assert n_match >= 3
+    assert st["rounds"] > st_ref["rounds"]                      # fewer slots, more batched rounds
+
+
+@pytest.mark.parametrize("drafter", [1, 2])
+def test_serve_transformer_bf16_equals_batch(drafter):
+    wl = dict(inputs.WORKLOADS["pusht_xfmr"], precision=1)
+    _serve_vs_batch(wl, 11, 4, 8, hp.accept_t(), 23, drafter=drafter)
+
+
+def test_serve_grows_its_buffers_beyond_max_b_and_keeps_the_law():
+    """5000 one-dimensional requests through 512 slots of a context built for 512."""
+    from paper_2512_15773_b200 import sweep
+    N, slots = 5000, 512
+    wl = dict(H=1, A=1, To=0, Do=0, T=100, precision=0, base=dict(arch="gauss"), draft=dict(arch="gauss"),
+              base_params=inputs.make_gauss_params(sweep.M0, sweep.S0),
+              draft_params=inputs.make_gauss_params(sweep.M0 + 0.25, 0.8 * sweep.S0))
+    smp, *_ = hp.setup(wl, max_B=slots, max_K=6)
+    out = torch.zeros(N, 1, 1, device="cuda")
+    smp.reset_stats()
+    smp.serve(None, N, slots, 6, hp.accept_t(), 99, out)
+    st = smp.stats()
+    assert st["chunks"] == N and st["steps_advanced"] == 100 * N
+    x = out.cpu().numpy().reshape(-1).astype(np.float64)
+    mean, std = sweep.vanilla_output_law()
+    assert stats.kstest((x - mean) / std, "norm").pvalue > 0.01
+    with pytest.raises(binding.TsdpError):
+        smp.serve(None, N, slots + 1, 6, hp.accept_t(), 99, out)   # more slots than the context has
+    smp.close()
+
+
+def test_serve_with_obs_beyond_max_b():
+    """Observation-conditioned requests beyond the context's batch capacity (obs K/V buffers grow)."""
+    wl = dict(inputs.WORKLOADS["pusht_xfmr"], precision=1)
+    N, slots, K = 9, 3, 8
+    big, *_ = hp.setup(wl, max_B=N, max_K=K)
+    small, *_ = hp.setup(wl, max_B=slots, max_K=K)
+    dobs = torch.tensor(inputs.make_obs(8, N, wl["To"], wl["Do"]), dtype=torch.float32, device="cuda")
+    ref = torch.zeros(N, wl["H"], wl["A"], device="cuda"); out = torch.zeros_like(ref)
+    big.sample_chunk(dobs, N, K, hp.accept_t(), 5, ref)
+    small.serve(dobs, N, slots, K, hp.accept_t(), 5, out)
+    assert torch.equal(out, ref)
+    big.close(); small.close()

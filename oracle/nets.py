@@ -1,11 +1,12 @@
-"""The denoisers eps = M(x, tau; obs) in numpy fp64: closed-form Gaussian toy, MLP, transformer.
+"""The denoisers eps = M(x, tau; obs) in numpy fp64: closed-form Gaussian toy, MLP, transformer, DiT.
 
 The paper states only the block counts ("DP consists of 8 Transformer blocks while the drafter
 contains only one", Sec. 4) and that the drafter has the same input-output interface and shares
 the encoder and scheduler (Sec. 3.2 "Draft Model Training").  Everything below that is more
 specific than that is this build's own architecture definition; parity with the paper's trained
 networks is UNPINNED (no weights or layer layout are published).  The pins that exist are
-structural: causality of self-attention, independence of candidates, zero-head => zero output,
+structural: causality of self-attention (bidirectionality for the adaLN transformer, whose
+blocks reduce to the identity with zero gates), independence of candidates, zero-head => zero output,
 and the closed-form Gaussian denoiser against the analytic posterior mean.
 
 Parameters are dicts of float64 arrays produced by the seeded input generators; a linear layer
@@ -94,6 +95,50 @@ def xfmr_eps(p, x, tau, obs):
     return layer_norm(h, p["lnf_g"], p["lnf_b"]) @ p["W_out"] + p["b_out"]
 
 
+# ----------------------------------------------------------------------------- DiT
+def layer_norm_plain(h, eps=1e-5):
+    m = h.mean(axis=-1, keepdims=True)
+    v = ((h - m) ** 2).mean(axis=-1, keepdims=True)
+    return (h - m) / np.sqrt(v + eps)
+
+
+def dit_time_vector(p, tau):
+    """c(tau) = W_t2^T SiLU(W_t1^T sinusoidal(tau) + b_t1) + b_t2."""
+    return silu(sinusoidal_embedding(tau, p["d"]) @ p["Wt1"] + p["bt1"]) @ p["Wt2"] + p["bt2"]
+
+
+def dit_eps(p, x, tau, ctx):
+    """Adaptive-LayerNorm transformer (the VLA-scale action expert of the largest configuration): the
+    timestep enters every block as shift / scale / gate vectors; the context tokens enter through
+    cross-attention; self-attention is bidirectional over the H action tokens.
+
+    h    = x W_in + b_in + pos
+    mem  = ctx W_ctx + b_ctx + cpos                                    [Tc, d]
+    c    = time vector;  per block (s1, k1, g1, s2, k2, g2) = split(SiLU(c) W_mod + b_mod)
+      h += g1 * ( SelfAttn( LN0(h) (1 + k1) + s1 ) W_o + b_o )
+      h +=       CrossAttn( LN(h; lnc), mem ) W_o2 + b_o2
+      h += g2 * ( GELU( (LN0(h) (1 + k2) + s2) W_1 + b_1 ) W_2 + b_2 )
+    (sf, kf) = split(SiLU(c) W_modf + b_modf);   eps = (LN0(h) (1 + kf) + sf) W_out + b_out
+    LN0 is LayerNorm without gain and bias."""
+    d, heads = p["d"], p["heads"]
+    h = x @ p["W_in"] + p["b_in"] + p["pos"]
+    mem = ctx @ p["W_ctx"] + p["b_ctx"] + p["cpos"]
+    sc = silu(dit_time_vector(p, tau))
+    for L in p["layers"]:
+        s1, k1, g1, s2, k2, g2 = np.split(sc @ L["Wmod"] + L["bmod"], 6)
+        a = layer_norm_plain(h) * (1.0 + k1) + s1
+        qkv = a @ L["Wqkv"] + L["bqkv"]
+        h = h + g1 * (attention(qkv[:, :d], qkv[:, d:2 * d], qkv[:, 2 * d:], heads, False) @ L["Wo"] + L["bo"])
+        a = layer_norm(h, L["lnc_g"], L["lnc_b"])
+        q = a @ L["Wq2"] + L["bq2"]
+        kv = mem @ L["Wkv2"] + L["bkv2"]
+        h = h + attention(q, kv[:, :d], kv[:, d:], heads, False) @ L["Wo2"] + L["bo2"]
+        a = layer_norm_plain(h) * (1.0 + k2) + s2
+        h = h + g2 * (gelu_tanh(a @ L["W1"] + L["b1"]) @ L["W2"] + L["b2"])
+    sf, kf = np.split(sc @ p["Wmodf"] + p["bmodf"], 2)
+    return (layer_norm_plain(h) * (1.0 + kf) + sf) @ p["W_out"] + p["b_out"]
+
+
 def make_denoiser(p, sched):
     """Return eps(x [H,A], tau, obs [To,Do]) for a parameter dict with key 'arch'."""
     arch = p["arch"]
@@ -103,4 +148,6 @@ def make_denoiser(p, sched):
         return lambda x, tau, obs: mlp_eps(p, x, tau, obs)
     if arch == "xfmr":
         return lambda x, tau, obs: xfmr_eps(p, x, tau, obs)
+    if arch == "dit":
+        return lambda x, tau, obs: dit_eps(p, x, tau, obs)
     raise ValueError(arch)

@@ -388,6 +388,7 @@ self_attn_mma_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __res
 // query rows of the candidate) and then stream the H query rows, 16 bytes per lane per row.
 // ------------------------------------------------------------------------------------------------
 constexpr int CA_MAXNK = 4;
+constexpr int CA_ROWS = 4;
 
 template <int DH>
 __global__ void __launch_bounds__(256)
@@ -399,8 +400,12 @@ cross_attn_group_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __re
   constexpr int LG = DH / 8;
   const int gid_raw = (blockIdx.x * blockDim.x + threadIdx.x) / LG;
   const int sub = threadIdx.x % LG;
-  const bool live = gid_raw < n_cand * heads;
-  const int gid = live ? gid_raw : n_cand * heads - 1;
+  // a group works on CA_ROWS consecutive query rows of its (candidate, head): more groups in flight than
+  // one per (candidate, head) would give, at the price of re-reading the few keys / values from cache
+  const int row_chunks = (H + CA_ROWS - 1) / CA_ROWS;
+  const bool live = gid_raw < n_cand * heads * row_chunks;
+  const int gid_c = live ? gid_raw : n_cand * heads * row_chunks - 1;
+  const int rc = gid_c % row_chunks, gid = gid_c / row_chunks;
   const int n = gid / heads, hd = gid % heads;
   const int b = n / cm.C, c = n % cm.C;
   int tau = cm.t[b] - cm.koff - c;
@@ -424,8 +429,9 @@ cross_attn_group_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __re
   const float scale = rsqrtf((float)DH);
   const __nv_bfloat16* qp = q + (size_t)n * H * d + (size_t)hd * DH + sub * 8;
   __nv_bfloat16* op = out + (size_t)n * H * d + (size_t)hd * DH + sub * 8;
-#pragma unroll 2
-  for (int r = 0; r < H; ++r) {
+#pragma unroll
+  for (int rr = 0; rr < CA_ROWS; ++rr) {
+    const int r = min(rc * CA_ROWS + rr, H - 1);       // a ragged last chunk repeats its last row
     const uint4 qv = *reinterpret_cast<const uint4*>(qp + (size_t)r * d);
     const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&qv);
     float qf[8];

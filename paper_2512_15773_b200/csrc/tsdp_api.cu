@@ -400,7 +400,7 @@ int cross_attn_launch(tsdp_ctx* c, const Net& n, const T* q2, T* out, const Cand
   bool done = false;
   if constexpr (std::is_same<T, __nv_bfloat16>::value) {
     if (1 + To <= CA_MAXNK && (dh == 32 || dh == 64 || dh == 128)) {
-      const long long threads = (long long)n_cand * heads * (dh / 8);
+      const long long threads = (long long)n_cand * heads * ((H + CA_ROWS - 1) / CA_ROWS) * (dh / 8);
       const int grid = (int)((threads + 255) / 256);
 #define CA_CASE(DH) TSDP_LAUNCH(c, (cross_attn_group_kernel<DH>), grid, 256, 0, s, q2, out, n.kv_time, n.kv_obs, cm, n_cand, H, d, heads, To, layer, L, c->cfg.T)
       if (dh == 32) CA_CASE(32); else if (dh == 64) CA_CASE(64); else CA_CASE(128);

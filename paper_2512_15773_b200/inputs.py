@@ -76,6 +76,45 @@ def make_xfmr_params(seed, H, A, To, Do, d, heads, layers, out_scale=1.0, bf16=T
     return p
 
 
+def make_dit_params(seed, H, A, To, Do, d, heads, layers, out_scale=1.0, bf16=True):
+    """Random adaptive-LayerNorm transformer (DiT-style) denoiser.  The modulation layers are given
+    small weights so that the network starts near an un-modulated, gated-on state: gates get a bias
+    of 1, shifts and scales a bias of 0."""
+    rng = np.random.default_rng(seed)
+    q = bf16_round if bf16 else (lambda a: np.asarray(a, dtype=np.float32).astype(np.float64))
+    q32 = lambda a: np.asarray(a, dtype=np.float32).astype(np.float64)
+    p = dict(arch="dit", d=d, heads=heads, n_layers=layers)
+    p["W_in"], p["b_in"] = _lin(rng, A, d, 1.0 / np.sqrt(A), q)
+    p["pos"] = q(rng.normal(0.0, 0.02, size=(H, d)))
+    p["W_ctx"], p["b_ctx"] = _lin(rng, Do, d, 1.0 / np.sqrt(Do), q)
+    p["cpos"] = q(rng.normal(0.0, 0.02, size=(To, d)))
+    s = 1.0 / np.sqrt(d)
+    # the time path runs in fp32 on the device (tables built at load): keep fp32-representable values
+    p["Wt1"], p["bt1"] = _lin(rng, d, d, s, q32)
+    p["Wt2"], p["bt2"] = _lin(rng, d, d, s, q32)
+    Ls = []
+    for _ in range(layers):
+        L = {}
+        W, b = _lin(rng, d, 6 * d, 0.3 * s, q32)
+        b = b.copy(); b[2 * d:3 * d] += 1.0; b[5 * d:6 * d] += 1.0            # gates start at 1
+        L["Wmod"], L["bmod"] = W, q32(b)
+        L["lnc_g"] = q(1.0 + rng.normal(0.0, 0.02, size=(d,)))
+        L["lnc_b"] = q(rng.normal(0.0, 0.02, size=(d,)))
+        L["Wqkv"], L["bqkv"] = _lin(rng, d, 3 * d, s, q)
+        L["Wo"], L["bo"] = _lin(rng, d, d, s, q)
+        L["Wq2"], L["bq2"] = _lin(rng, d, d, s, q)
+        L["Wkv2"], L["bkv2"] = _lin(rng, d, 2 * d, s, q)
+        L["Wo2"], L["bo2"] = _lin(rng, d, d, s, q)
+        L["W1"], L["b1"] = _lin(rng, d, 4 * d, s, q)
+        L["W2"], L["b2"] = _lin(rng, 4 * d, d, 0.5 * s, q)
+        Ls.append(L)
+    p["layers"] = Ls
+    p["Wmodf"], p["bmodf"] = _lin(rng, d, 2 * d, 0.3 * s, q32)
+    W, b = _lin(rng, d, A, s, q)
+    p["W_out"], p["b_out"] = q(W * out_scale), q(b * out_scale)
+    return p
+
+
 def make_sched_params(seed, H, A, To, Do, scale=1.0):
     """Random weights of the scheduler network (three stream encoders 64 / 64 / 16, aggregate MLP
     64, 5 outputs); fp32-representable.  `scale` multiplies the output layer."""
@@ -111,6 +150,10 @@ WORKLOADS = {
     "serving_xfmr": dict(H=16, A=7, To=2, Do=64, T=100, precision=1,
                          base=dict(arch="xfmr", layers=12, d=512, heads=8),
                          draft=dict(arch="xfmr", layers=2, d=256, heads=4), B=256, K=10, gamma=0.03),
+    # VLA-scale action expert: 50 x 14 action chunk, 256 context tokens of width 1024
+    "vla_dit": dict(H=50, A=14, To=256, Do=1024, T=100, precision=1,
+                    base=dict(arch="dit", layers=18, d=1024, heads=16),
+                    draft=dict(arch="dit", layers=4, d=512, heads=8), B=64, K=16, gamma=0.03),
 }
 
 
@@ -125,6 +168,10 @@ def make_net(seed, wl, which, gamma=None, bf16=None):
         use_bf16 = (wl["precision"] == 1) if bf16 is None else bf16
         return make_xfmr_params(seed, wl["H"], wl["A"], wl["To"], wl["Do"], n["d"], n["heads"],
                                 n["layers"], out_scale=g, bf16=use_bf16)
+    if n["arch"] == "dit":
+        use_bf16 = (wl["precision"] == 1) if bf16 is None else bf16
+        return make_dit_params(seed, wl["H"], wl["A"], wl["To"], wl["Do"], n["d"], n["heads"], n["layers"],
+                               out_scale=g, bf16=use_bf16)
     raise ValueError(n["arch"])
 
 

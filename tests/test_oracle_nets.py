@@ -93,3 +93,52 @@ def test_bf16_rounding_of_inputs():
     assert np.all(np.abs(r - a) <= np.abs(a) * 2.0 ** -8)
     u = r.astype(np.float32).view(np.uint32)
     assert np.all(u & 0xFFFF == 0)
+
+
+# ----------------------------------------------------------------------------- DiT (structure only)
+def _dit(seed=0, H=5, A=3, To=4, Do=6, d=16, heads=2, layers=2):
+    p = inputs.make_dit_params(seed, H, A, To, Do, d, heads, layers, bf16=False)
+    rng = np.random.default_rng(seed + 100)
+    return p, rng.normal(size=(H, A)), rng.normal(size=(To, Do))
+
+
+def test_dit_self_attention_is_bidirectional_and_context_enters_by_cross_attention_only():
+    p, x, ctx = _dit()
+    e0 = nets.dit_eps(p, x, 40, ctx)
+    x2 = x.copy(); x2[-1] += 1.0                      # the LAST token changes ...
+    assert np.abs(nets.dit_eps(p, x2, 40, ctx)[0] - e0[0]).max() > 1e-9      # ... and the first output moves
+    q = dict(p, layers=[dict(L, Wo2=np.zeros_like(L["Wo2"]), bo2=np.zeros_like(L["bo2"])) for L in p["layers"]])
+    assert np.array_equal(nets.dit_eps(q, x, 40, ctx), nets.dit_eps(q, x, 40, 3.0 * ctx))
+    assert not np.allclose(nets.dit_eps(p, x, 40, 3.0 * ctx), e0)
+
+
+def test_dit_zero_gates_make_a_block_the_identity_up_to_cross_attention():
+    p, x, ctx = _dit(1)
+    # gates 0 and no cross-attention output: every block is the identity, so the output is the final layer of the embedding
+    Ls = []
+    for L in p["layers"]:
+        L = dict(L, Wo2=np.zeros_like(L["Wo2"]), bo2=np.zeros_like(L["bo2"]))
+        W, b = L["Wmod"].copy(), L["bmod"].copy()
+        d = p["d"]
+        for g in (2, 5):
+            W[:, g * d:(g + 1) * d] = 0.0; b[g * d:(g + 1) * d] = 0.0
+        Ls.append(dict(L, Wmod=W, bmod=b))
+    q = dict(p, layers=Ls)
+    h = x @ p["W_in"] + p["b_in"] + p["pos"]
+    sc = nets.silu(nets.dit_time_vector(p, 17))
+    sf, kf = np.split(sc @ p["Wmodf"] + p["bmodf"], 2)
+    ref = (nets.layer_norm_plain(h) * (1 + kf) + sf) @ p["W_out"] + p["b_out"]
+    assert np.allclose(nets.dit_eps(q, x, 17, ctx), ref, atol=1e-12)
+
+
+def test_dit_time_enters_through_modulation_only():
+    p, x, ctx = _dit(2)
+    q = dict(p, Wt2=np.zeros_like(p["Wt2"]))         # constant time vector: the timestep cannot matter
+    assert np.array_equal(nets.dit_eps(q, x, 3, ctx), nets.dit_eps(q, x, 90, ctx))
+    assert not np.allclose(nets.dit_eps(p, x, 3, ctx), nets.dit_eps(p, x, 90, ctx))
+
+
+def test_layer_norm_plain_is_layer_norm_with_unit_gain():
+    h = np.random.default_rng(0).normal(size=(4, 16))
+    assert np.allclose(nets.layer_norm_plain(h), nets.layer_norm(h, np.ones(16), np.zeros(16)))
+    assert np.allclose(nets.layer_norm_plain(h).mean(-1), 0) and np.allclose(nets.layer_norm_plain(h).var(-1), 1, atol=1e-4)

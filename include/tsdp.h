@@ -41,7 +41,7 @@ typedef enum {
   TSDP_ERR_TOO_LARGE = 8    /* size beyond the capacity of tsdp_verify_commit_static       */
 } tsdp_status;
 
-enum { TSDP_ARCH_GAUSS = 0, TSDP_ARCH_MLP = 1, TSDP_ARCH_XFMR = 2 };
+enum { TSDP_ARCH_GAUSS = 0, TSDP_ARCH_MLP = 1, TSDP_ARCH_XFMR = 2, TSDP_ARCH_DIT = 3 };
 enum { TSDP_BASE = 0, TSDP_DRAFT = 1, TSDP_SCHED = 2 };
 enum { TSDP_MAX_T = 1024, TSDP_MAX_K = 32 };
 
@@ -50,6 +50,10 @@ enum { TSDP_MAX_T = 1024, TSDP_MAX_K = 32 };
  *   MLP  : input [latent | sinusoidal(t, temb) | obs], `layers` hidden SiLU layers of width `d`.
  *   XFMR : pre-LN decoder, `layers` blocks [causal self-attn, cross-attn to (time token | obs tokens),
  *          GELU MLP 4d], model width `d` (multiple of 128), `heads` heads (d/heads multiple of 32).
+ *   DIT  : adaptive-LayerNorm transformer: the timestep enters each of the `layers` blocks as shift /
+ *          scale / gate vectors, the obs_tokens (<= 256) observation/context tokens through
+ *          cross-attention, self-attention over the H action tokens is bidirectional;
+ *          h += g1 * SelfAttn(LN0(h)(1+k1)+s1) Wo;  h += CrossAttn(LN(h), ctx) Wo2;  h += g2 * MLP(LN0(h)(1+k2)+s2).
  * The paper fixes only the block counts (8 for the base policy, 1 for the drafter; Sec. 4). */
 typedef struct {
   int arch, layers, d, heads, temb;
@@ -120,6 +124,11 @@ size_t tsdp_weights_count(const tsdp_config_t* cfg, int which);
  *          per block: ln1_g, ln1_b, Wqkv [d,3d], bqkv, Wo, bo, ln2_g, ln2_b, Wq2, bq2, Wkv2 [d,2d], bkv2,
  *                     Wo2, bo2, ln3_g, ln3_b, W1 [d,4d], b1, W2 [4d,d], b2;
  *          lnf_g, lnf_b, W_out [d,A], b_out.
+ *   DIT  : W_in [A,d], b_in, pos [H,d], W_ctx [obs_dim,d], b_ctx, cpos [obs_tokens,d], Wt1 [d,d], bt1, Wt2 [d,d], bt2;
+ *          per block: Wmod [d,6d], bmod (shift1, scale1, gate1, shift2, scale2, gate2), Wqkv, bqkv, Wo, bo,
+ *                     lnc_g, lnc_b, Wq2, bq2, Wkv2 [d,2d], bkv2, Wo2, bo2, W1, b1, W2, b2;
+ *          Wmodf [d,2d], bmodf (shift, scale of the final layer), W_out [d,A], b_out.
+ *          The time path (Wt*, Wmod*) is kept in fp32 and tabulated for every timestep during the load.
  *   SCHED (which = TSDP_SCHED, the scheduler network of Sec. 3.3, always fp32): W_o [obs_tokens*obs_dim, 64],
  *          b_o, W_a [H*A, 64], b_a, W_p [1, 16], b_p, W_1 [144, 64], b_1, W_2 [64, 5], b_2.
  * In precision 1 the large matrices are rounded to bf16.  Errors: WEIGHTS (n mismatch), NAN, CUDA. */

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libtsdp.so")
 
 TSDP_MAX_T = 1024
-ARCH = {"gauss": 0, "mlp": 1, "xfmr": 2}
+ARCH = {"gauss": 0, "mlp": 1, "xfmr": 2, "dit": 3}
 BASE, DRAFT, SCHED = 0, 1, 2
 EXPORTS = ["tsdp_init", "tsdp_destroy", "tsdp_strerror", "tsdp_last_error", "tsdp_weights_count",
            "tsdp_load_weights", "tsdp_set_schedule", "tsdp_sample_chunk", "tsdp_sample_chunk_host",
@@ -113,6 +113,12 @@ def pack_weights(p):
         parts = []
         for W, b in zip(p["W"], p["b"]):
             parts += [W, b]
+    elif a == "dit":
+        parts = [p[k] for k in ("W_in", "b_in", "pos", "W_ctx", "b_ctx", "cpos", "Wt1", "bt1", "Wt2", "bt2")]
+        for L in p["layers"]:
+            parts += [L[k] for k in ("Wmod", "bmod", "Wqkv", "bqkv", "Wo", "bo", "lnc_g", "lnc_b", "Wq2", "bq2", "Wkv2", "bkv2",
+                                     "Wo2", "bo2", "W1", "b1", "W2", "b2")]
+        parts += [p["Wmodf"], p["bmodf"], p["W_out"], p["b_out"]]
     elif a == "sched":
         parts = [p[k] for k in ("W_o", "b_o", "W_a", "b_a", "W_p", "b_p", "W_1", "b_1", "W_2", "b_2")]
     elif a == "xfmr":

@@ -25,7 +25,9 @@
 
 namespace tsdp {
 
-enum { EPI_STORE = 0, EPI_GELU = 1, EPI_RESID = 2, EPI_F32 = 3 };
+// EPI_GATE: fp32 out += gate[tau(row), col] * (acc + bias), the gated residual of an adaptive-LayerNorm block.
+// EPI_SILU: fp32 store of SiLU(acc + bias); CUDA-core GEMM only (conditioning tables built at load).
+enum { EPI_STORE = 0, EPI_GELU = 1, EPI_RESID = 2, EPI_F32 = 3, EPI_GATE = 4, EPI_SILU = 5 };
 
 constexpr int GEMM_BM = 128;
 constexpr int GEMM_BK = 64;
@@ -184,7 +186,21 @@ struct GemmArgs {
   void* out;            // EPI_STORE/GELU: bf16 [M, ldo]; EPI_RESID: fp32 [M, ldo] updated in place; EPI_F32: fp32
   int ldo;
   int* status;          // device word; set to TSDP_ERR_TIMEOUT (5) when a wait expires
+  // EPI_GATE only: gate vectors [Tsteps, gate_ld] (this layer's gate starts at column 0 of the pointer) and
+  // the map from a token row to its timestep: row -> candidate n = row / H -> (b = n / C, c = n % C),
+  // tau = clamp(t[b] - koff - c)
+  const float* gate;
+  int gate_ld;
+  const int* t;
+  int C, koff, H, Tsteps;
 };
+
+__device__ __forceinline__ const float* gate_row(const GemmArgs& g, int row) {
+  const int n = row / g.H;
+  int tau = g.t[n / g.C] - g.koff - (n % g.C);
+  tau = max(0, min(g.Tsteps - 1, tau));
+  return g.gate + (size_t)tau * g.gate_ld;
+}
 
 template <int EPI>
 __device__ __forceinline__ void epilogue_store16(const GemmArgs& g, int row, int col, const uint32_t v[16]) {
@@ -194,6 +210,11 @@ __device__ __forceinline__ void epilogue_store16(const GemmArgs& g, int row, int
     f[i] = __uint_as_float(v[i]);
     if (g.bias) f[i] += __ldg(g.bias + col + i);
     if (EPI == EPI_GELU) f[i] = gelu_tanh(f[i]);
+  }
+  if (EPI == EPI_GATE) {
+    const float* gp = gate_row(g, row) + col;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) f[i] *= __ldg(gp + i);
   }
   if (EPI == EPI_STORE || EPI == EPI_GELU) {
     __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(g.out) + (size_t)row * g.ldo + col;
@@ -211,7 +232,7 @@ __device__ __forceinline__ void epilogue_store16(const GemmArgs& g, int row, int
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       float4 r = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
-      if (EPI == EPI_RESID) {
+      if (EPI == EPI_RESID || EPI == EPI_GATE) {
         const float4 h = reinterpret_cast<const float4*>(o)[i];
         r.x += h.x; r.y += h.y; r.z += h.z; r.w += h.w;
       }
@@ -362,6 +383,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 f[i] = 0.5f * x * (1.0f + ptx::tanh_fast(0.7978845608028654f * (x + 0.044715f * x * x * x)));
               }
             }
+            if (EPI == EPI_GATE) {
+              const int grow = min(tm * GEMM_BM + r, g.M - 1);     // rows past M are clipped by the TMA store
+              const float4* gp = reinterpret_cast<const float4*>(gate_row(g, grow) + col);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const float4 gg = __ldg(gp + i);
+                f[4 * i] *= gg.x; f[4 * i + 1] *= gg.y; f[4 * i + 2] *= gg.z; f[4 * i + 3] *= gg.w;
+              }
+            }
             if (part == 0) {   // the previous chunk's TMA store must have drained the staging buffer
               if (issuer) ptx::bulk_wait_read0();
               ptx::named_bar_sync(bar_id, 128);
@@ -385,7 +415,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           ptx::named_bar_sync(bar_id, 128);
           if (issuer) {
             const int x = tn * BN + half * COLS + ch * CW, y = tm * GEMM_BM;
-            if (EPI == EPI_RESID) ptx::tma_reduce_add_2d(&tmC, x, y, stg);
+            if (EPI == EPI_RESID || EPI == EPI_GATE) ptx::tma_reduce_add_2d(&tmC, x, y, stg);
             else ptx::tma_store_2d(&tmC, x, y, stg);
             ptx::bulk_commit();
           }

@@ -46,8 +46,10 @@ gemm_simt_kernel(const float* __restrict__ A, const float* __restrict__ W, GemmA
       if (col >= g.N) continue;
       float v = acc[i][j] + (g.bias ? g.bias[col] : 0.f);
       if (EPI == EPI_GELU) v = gelu_tanh(v);
+      if (EPI == EPI_SILU) v = v / (1.0f + expf(-v));
+      if (EPI == EPI_GATE) v *= gate_row(g, row)[col];
       float* o = reinterpret_cast<float*>(g.out) + (size_t)row * g.ldo + col;
-      if (EPI == EPI_RESID) v += *o;
+      if (EPI == EPI_RESID || EPI == EPI_GATE) v += *o;
       *o = v;
     }
   }
@@ -147,7 +149,7 @@ __global__ void ln_kernel(const float* __restrict__ h, const float* __restrict__
 // ------------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void self_attn_kernel(const T* __restrict__ qkv, T* __restrict__ out, int n_cand, int H, int d,
-                                 int heads) {
+                                 int heads, int causal) {
   pdl_trigger();
   pdl_wait();
   extern __shared__ float sm[];
@@ -171,24 +173,25 @@ __global__ void self_attn_kernel(const T* __restrict__ qkv, T* __restrict__ out,
   __syncwarp();
   const float scale = rsqrtf((float)dh);
   for (int r = 0; r < H; ++r) {
+    const int last = causal ? r : H - 1;            // last key this query sees
     float s0 = -INFINITY, s1 = -INFINITY;
-    if (lane <= r) {
+    if (lane <= last) {
       float a = 0.f;
       for (int i = 0; i < dh; ++i) a += Q[r * dh + i] * Kt[lane * (dh + 1) + i];
       s0 = a * scale;
     }
-    if (lane + 32 <= r) {
+    if (lane + 32 <= last) {
       float a = 0.f;
       for (int i = 0; i < dh; ++i) a += Q[r * dh + i] * Kt[(lane + 32) * (dh + 1) + i];
       s1 = a * scale;
     }
     const float m = warp_max(fmaxf(s0, s1));
-    const float p0 = (lane <= r) ? __expf(s0 - m) : 0.f;
-    const float p1 = (lane + 32 <= r) ? __expf(s1 - m) : 0.f;
+    const float p0 = (lane <= last) ? __expf(s0 - m) : 0.f;
+    const float p1 = (lane + 32 <= last) ? __expf(s1 - m) : 0.f;
     const float inv = 1.0f / warp_sum(p0 + p1);
     for (int c0 = 0; c0 < dh; c0 += 32) {
       float o = 0.f;
-      for (int c = 0; c <= r; ++c) {
+      for (int c = 0; c <= last; ++c) {
         const float p = __shfl_sync(0xffffffffu, c < 32 ? p0 : p1, c & 31);
         o += p * V[c * (dh + 1) + c0 + lane];
       }
@@ -268,7 +271,7 @@ constexpr int SA_WARPS = 4;
 template <int DH>
 __global__ void __launch_bounds__(SA_WARPS * 32)
 self_attn_mma_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ out, int n_cand, int H, int d,
-                     int heads) {
+                     int heads, int causal) {
   pdl_trigger();
   pdl_wait();
   constexpr int KS = DH / 16;        // k-steps of Q K^T
@@ -293,8 +296,9 @@ self_attn_mma_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __res
     const int c = ks * 16 + 2 * tg;
     qa[ks][0] = ld32(r0, c); qa[ks][1] = ld32(r1, c); qa[ks][2] = ld32(r0, c + 8); qa[ks][3] = ld32(r1, c + 8);
   }
-  // keys 0 .. 16 (qt+1) - 1 are the only ones a causal query of this tile can see
-  const int nkt = 2 * (qt + 1);
+  // keys 0 .. 16 (qt+1) - 1 are the only ones a causal query of this tile can see; a bidirectional one sees all H
+  const int nkt = causal ? 2 * (qt + 1) : (H + 7) >> 3;
+  const int kst = causal ? qt + 1 : (H + 15) >> 4;
   float s[8][4];
 #pragma unroll
   for (int nt = 0; nt < 8; ++nt) {
@@ -314,10 +318,11 @@ self_attn_mma_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __res
   for (int nt = 0; nt < 8; ++nt) {
     if (nt < nkt) {
       const int col = nt * 8 + 2 * tg;
-      s[nt][0] = (col <= r0 && col < H) ? s[nt][0] * scale : -INFINITY;
-      s[nt][1] = (col + 1 <= r0 && col + 1 < H) ? s[nt][1] * scale : -INFINITY;
-      s[nt][2] = (col <= r1 && col < H) ? s[nt][2] * scale : -INFINITY;
-      s[nt][3] = (col + 1 <= r1 && col + 1 < H) ? s[nt][3] * scale : -INFINITY;
+      const int lim0 = causal ? r0 : H, lim1 = causal ? r1 : H;
+      s[nt][0] = (col <= lim0 && col < H) ? s[nt][0] * scale : -INFINITY;
+      s[nt][1] = (col + 1 <= lim0 && col + 1 < H) ? s[nt][1] * scale : -INFINITY;
+      s[nt][2] = (col <= lim1 && col < H) ? s[nt][2] * scale : -INFINITY;
+      s[nt][3] = (col + 1 <= lim1 && col + 1 < H) ? s[nt][3] * scale : -INFINITY;
       m0 = fmaxf(m0, fmaxf(s[nt][0], s[nt][1]));
       m1 = fmaxf(m1, fmaxf(s[nt][2], s[nt][3]));
     }
@@ -347,7 +352,7 @@ self_attn_mma_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __res
   const unsigned short* vraw = reinterpret_cast<const unsigned short*>(vbase);
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    if (j <= qt) {
+    if (j < kst) {
       uint32_t pa[4];
       pa[0] = pack_bf16(s[2 * j][0], s[2 * j][1]); pa[1] = pack_bf16(s[2 * j][2], s[2 * j][3]);
       pa[2] = pack_bf16(s[2 * j + 1][0], s[2 * j + 1][1]); pa[3] = pack_bf16(s[2 * j + 1][2], s[2 * j + 1][3]);

@@ -21,6 +21,7 @@
 #include "round_kernels.cuh"
 #include "drafter_cluster.cuh"
 #include "sched_kernel.cuh"
+#include "dit_kernels.cuh"
 
 using namespace tsdp;
 
@@ -48,6 +49,8 @@ struct Net {
   float* kv_time = nullptr;                   // [T, L*2d]   K/V of the time token for every timestep
   float* kv_obs = nullptr;                    // [max_B*To, L*2d]  K/V of the obs tokens, per chunk
   float* temb_table = nullptr;                // [T, temb or d] sinusoidal embedding
+  float* mod = nullptr;                       // DIT: [T, L*6d + 2d] shift / scale / gate vectors of every timestep
+  int mod_ld = 0;
   std::vector<void*> allocs;
 };
 
@@ -171,6 +174,10 @@ bool net_cfg_ok(const tsdp_config_t& cfg, const tsdp_net_t& n) {
   if (n.arch == TSDP_ARCH_XFMR)
     return n.layers >= 1 && n.d % 128 == 0 && n.d >= 128 && n.d <= 1024 && n.heads >= 1 && n.d % n.heads == 0 &&
            (n.d / n.heads) % 32 == 0 && (n.d / n.heads) <= 128 && cfg.H <= 64 && cfg.obs_tokens <= 8 && cfg.A <= 64;
+  if (n.arch == TSDP_ARCH_DIT)
+    return n.layers >= 1 && n.d % 128 == 0 && n.d >= 128 && n.d <= 1024 && n.heads >= 1 && n.d % n.heads == 0 &&
+           (n.d / n.heads) % 32 == 0 && (n.d / n.heads) <= 128 && cfg.H <= 64 && cfg.obs_tokens >= 1 &&
+           cfg.obs_tokens <= 256 && cfg.obs_dim >= 1 && cfg.A <= 64;
   return false;
 }
 
@@ -187,6 +194,13 @@ size_t weights_count(const tsdp_config_t& cfg, const tsdp_net_t& n) {
     const size_t per = 2 * d + d * 3 * d + 3 * d + d * d + d + 2 * d + d * d + d + d * 2 * d + 2 * d + d * d + d + 2 * d +
                        d * 4 * d + 4 * d + 4 * d * d + d;
     return tot + per * n.layers + 2 * d + d * cfg.A + cfg.A;
+  }
+  if (n.arch == TSDP_ARCH_DIT) {
+    size_t tot = (size_t)cfg.A * d + d + (size_t)cfg.H * d + (size_t)cfg.obs_dim * d + d + (size_t)cfg.obs_tokens * d +
+                 2 * (d * d + d);
+    const size_t per = d * 6 * d + 6 * d + d * 3 * d + 3 * d + d * d + d + 2 * d + d * d + d + d * 2 * d + 2 * d + d * d + d +
+                       d * 4 * d + 4 * d + 4 * d * d + d;
+    return tot + per * n.layers + d * 2 * d + 2 * d + d * cfg.A + cfg.A;
   }
   return 0;
 }
@@ -242,6 +256,7 @@ int launch_tc_epi(tsdp_ctx* c, const CUtensorMap& ma, const CUtensorMap& mb, con
     case EPI_STORE: return launch_tc<BN, EPI_STORE>(c, ma, mb, mc, g, s);
     case EPI_GELU: return launch_tc<BN, EPI_GELU>(c, ma, mb, mc, g, s);
     case EPI_RESID: return launch_tc<BN, EPI_RESID>(c, ma, mb, mc, g, s);
+    case EPI_GATE: return launch_tc<BN, EPI_GATE>(c, ma, mb, mc, g, s);
     default: return launch_tc<BN, EPI_F32>(c, ma, mb, mc, g, s);
   }
 }
@@ -257,6 +272,7 @@ cudaError_t set_smem_attr_all() {
   if ((e = set_smem_attr<BN, EPI_STORE>()) != cudaSuccess) return e;
   if ((e = set_smem_attr<BN, EPI_GELU>()) != cudaSuccess) return e;
   if ((e = set_smem_attr<BN, EPI_RESID>()) != cudaSuccess) return e;
+  if ((e = set_smem_attr<BN, EPI_GATE>()) != cudaSuccess) return e;
   return set_smem_attr<BN, EPI_F32>();
 }
 
@@ -272,10 +288,20 @@ int pick_bn(int M, int N, int num_sms) {
   return 0;
 }
 
+// Gate of an adaptive-LayerNorm residual (EPI_GATE): gate vectors and the row -> timestep map.
+struct GateSpec {
+  const float* gate; int gate_ld; const CandMap* cm; int H, Tsteps;
+};
+
 int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, int N, int K, int epi, void* out,
-         int ldo, cudaStream_t s) {
+         int ldo, cudaStream_t s, const GateSpec* gs = nullptr) {
   if (M <= 0) return TSDP_OK;
-  GemmArgs g{M, N, K, bias, out, ldo, c->status};
+  GemmArgs g{M, N, K, bias, out, ldo, c->status, nullptr, 0, nullptr, 1, 0, 1, 1};
+  if (epi == EPI_GATE) {
+    if (!gs) return TSDP_ERR_ARG;
+    g.gate = gs->gate; g.gate_ld = gs->gate_ld; g.t = gs->cm->t; g.C = gs->cm->C; g.koff = gs->cm->koff; g.H = gs->H;
+    g.Tsteps = gs->Tsteps;
+  }
   if (c->cfg.precision == 0) {
     dim3 grid((N + 63) / 64, (M + 63) / 64);
     const float* a = reinterpret_cast<const float*>(A);
@@ -284,6 +310,7 @@ int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, in
     switch (epi) {
       case EPI_GELU: TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_GELU>), grid, 256, 0, s, a, w, g); break;
       case EPI_RESID: TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_RESID>), grid, 256, 0, s, a, w, g); break;
+      case EPI_GATE: TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_GATE>), grid, 256, 0, s, a, w, g); break;
       default: TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_F32>), grid, 256, 0, s, a, w, g); break;
     }
     prof_end(c, s);
@@ -315,6 +342,17 @@ int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, in
     case 64: return launch_tc_epi<64>(c, ma, mb, mc, g, epi, s);
     default: return launch_tc_epi<32>(c, ma, mb, mc, g, epi, s);
   }
+}
+
+// fp32 CUDA-core GEMM whatever the precision mode: the timestep-conditioning tables built at weight load.
+int gemm_f32(tsdp_ctx* c, const float* A, const float* W, const float* bias, int M, int N, int K, int epi, float* out,
+             cudaStream_t s) {
+  GemmArgs g{M, N, K, bias, out, N, c->status, nullptr, 0, nullptr, 1, 0, 1, 1};
+  dim3 grid((N + 63) / 64, (M + 63) / 64);
+  if (epi == EPI_SILU) TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_SILU>), grid, 256, 0, s, A, W, g);
+  else TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_F32>), grid, 256, 0, s, A, W, g);
+  CU_TRY(c, cudaGetLastError());
+  return TSDP_OK;
 }
 
 // ------------------------------------------------------------------------------------------ nets
@@ -364,24 +402,25 @@ int head_launch(tsdp_ctx* c, const Net& n, const CandMap& cm, int M, cudaStream_
 
 // Causal self-attention: tensor-core kernel for bf16 activations, the scalar kernel in check mode.
 template <typename T>
-int self_attn_launch(tsdp_ctx* c, const T* qkv, T* out, int n_cand, int H, int d, int heads, cudaStream_t s) {
+int self_attn_launch(tsdp_ctx* c, const T* qkv, T* out, int n_cand, int H, int d, int heads, cudaStream_t s,
+                     int causal = 1) {
   const int dh = d / heads;
   prof_begin(c, s, 2, 0.0);
   if constexpr (std::is_same<T, __nv_bfloat16>::value) {
     const int QT = (H + 15) / 16;
     const int grid = (n_cand * heads * QT + SA_WARPS - 1) / SA_WARPS;
     switch (dh) {
-      case 32: TSDP_LAUNCH(c, (self_attn_mma_kernel<32>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads); break;
-      case 64: TSDP_LAUNCH(c, (self_attn_mma_kernel<64>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads); break;
-      case 96: TSDP_LAUNCH(c, (self_attn_mma_kernel<96>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads); break;
-      default: TSDP_LAUNCH(c, (self_attn_mma_kernel<128>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads); break;
+      case 32: TSDP_LAUNCH(c, (self_attn_mma_kernel<32>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads, causal); break;
+      case 64: TSDP_LAUNCH(c, (self_attn_mma_kernel<64>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads, causal); break;
+      case 96: TSDP_LAUNCH(c, (self_attn_mma_kernel<96>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads, causal); break;
+      default: TSDP_LAUNCH(c, (self_attn_mma_kernel<128>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads, causal); break;
     }
   } else {
     const size_t per_warp = (size_t)(H * dh + 2 * H * (dh + 1)) * sizeof(float);
     int wpb = (int)((200 * 1024) / per_warp);      // the opt-in shared-memory limit set at init
     wpb = wpb > 4 ? 4 : (wpb < 1 ? 1 : wpb);
     const size_t smem = (size_t)wpb * per_warp;
-    TSDP_LAUNCH(c, (self_attn_kernel<T>), (n_cand * heads + wpb - 1) / wpb, wpb * 32, smem, s, qkv, out, n_cand, H, d, heads);
+    TSDP_LAUNCH(c, (self_attn_kernel<T>), (n_cand * heads + wpb - 1) / wpb, wpb * 32, smem, s, qkv, out, n_cand, H, d, heads, causal);
   }
   prof_end(c, s);
   c->launches_per_round_tmp++;
@@ -463,7 +502,116 @@ int xfmr_prepare_obs_t(tsdp_ctx* c, Net& n, int B, cudaStream_t s) {
   return gemm(c, mt, n.Wkv_all, n.bkv_all, B * To, L * 2 * d, d, EPI_F32, n.kv_obs, L * 2 * d, s);
 }
 
+// ------------------------------------------------------------------------------------------ DiT
+template <typename T>
+int ln_mod_launch(tsdp_ctx* c, const Net& n, int off_shift, int off_scale, const CandMap& cm, T* out, int M, cudaStream_t s) {
+  const int wpb = 8, grid = (M + wpb - 1) / wpb, H = c->cfg.H, Ts = c->cfg.T;
+  prof_begin(c, s, 1, 0.0);
+#define LNM_CASE(V) TSDP_LAUNCH(c, (ln_mod_kernel<T, V>), grid, wpb * 32, 0, s, c->h, n.mod, n.mod_ld, off_shift, off_scale, cm, H, Ts, out, M)
+  switch (n.cfg.d / 128) {
+    case 1: LNM_CASE(1); break; case 2: LNM_CASE(2); break; case 3: LNM_CASE(3); break; case 4: LNM_CASE(4); break;
+    case 5: LNM_CASE(5); break; case 6: LNM_CASE(6); break; case 7: LNM_CASE(7); break; default: LNM_CASE(8); break;
+  }
+#undef LNM_CASE
+  prof_end(c, s);
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  return TSDP_OK;
+}
+
+// Cross-attention of every candidate's tokens to the context tokens of its request.
+template <typename T>
+int cross_attn_ctx_launch(tsdp_ctx* c, const Net& n, const T* q2, T* out, const CandMap& cm, int n_cand, int layer,
+                          cudaStream_t s) {
+  const int H = c->cfg.H, d = n.cfg.d, heads = n.cfg.heads, L = n.cfg.layers, Tc = c->cfg.obs_tokens;
+  const int dh = d / heads, M = n_cand * H;
+  const long long ld_kv = (long long)L * 2 * d;
+  const T* kv = reinterpret_cast<const T*>(n.kv_obs);
+  prof_begin(c, s, 2, 0.0);
+  bool done = false;
+  if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+    if (Tc % 16 == 0 && (dh == 32 || dh == 64 || dh == 128) && n_cand % cm.C == 0) {
+      const int slots = n_cand / cm.C, rows = cm.C * H;
+#define CX_CASE(DH) TSDP_LAUNCH(c, (cross_attn_ctx_mma_kernel<DH>), slots * heads, CX_WARPS * 32, cx_smem_bytes<DH>(Tc), s, q2, out, kv, ld_kv, layer * 2 * d, cm, rows, d, heads, Tc)
+      if (dh == 32) CX_CASE(32); else if (dh == 64) CX_CASE(64); else CX_CASE(128);
+#undef CX_CASE
+      done = true;
+    }
+  }
+  if (!done) {
+    const int wpb = 4;
+    TSDP_LAUNCH(c, (cross_attn_ctx_simt_kernel<T>), (M + wpb - 1) / wpb, wpb * 32, (size_t)wpb * Tc * sizeof(float), s, q2, out,
+                kv, ld_kv, layer * 2 * d, cm, M, H, d, heads, Tc);
+  }
+  prof_end(c, s);
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  return TSDP_OK;
+}
+
+template <typename T>
+int dit_forward_t(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStream_t s) {
+  const int H = c->cfg.H, A = c->cfg.A, d = n.cfg.d, heads = n.cfg.heads, L = n.cfg.layers;
+  const int M = n_cand * H;
+  T* a = reinterpret_cast<T*>(c->a);
+  T* qkv = reinterpret_cast<T*>(c->qkv);
+  T* q2 = reinterpret_cast<T*>(c->q2);
+  T* f = reinterpret_cast<T*>(c->f);
+  int r;
+  prof_begin(c, s, 3, 0.0);
+  TSDP_LAUNCH(c, (embed_kernel), M, d < 256 ? d : 256, 0, s, cm, n.W_in, n.b_in, n.pos, c->h, H, A, d);
+  prof_end(c, s);
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  const int out_epi = (c->cfg.precision == 0) ? EPI_F32 : EPI_STORE;
+  for (int l = 0; l < L; ++l) {
+    const XfmrLayer& w = n.L[l];
+    const int base = l * 6 * d;        // (shift1, scale1, gate1, shift2, scale2, gate2) of this block in a row of mod
+    GateSpec g1{n.mod + base + 2 * d, n.mod_ld, &cm, H, c->cfg.T}, g2{n.mod + base + 5 * d, n.mod_ld, &cm, H, c->cfg.T};
+    if ((r = ln_mod_launch<T>(c, n, base, base + d, cm, a, M, s))) return r;
+    if ((r = gemm(c, a, w.Wqkv, w.bqkv, M, 3 * d, d, out_epi, qkv, 3 * d, s))) return r;
+    if ((r = self_attn_launch<T>(c, qkv, a, n_cand, H, d, heads, s, 0))) return r;
+    if ((r = gemm(c, a, w.Wo, w.bo, M, d, d, EPI_GATE, c->h, d, s, &g1))) return r;
+    if ((r = ln_launch<T>(c, c->h, w.ln2_g, w.ln2_b, a, M, d, s))) return r;
+    if ((r = gemm(c, a, w.Wq2, w.bq2, M, d, d, out_epi, q2, d, s))) return r;
+    if ((r = cross_attn_ctx_launch<T>(c, n, q2, a, cm, n_cand, l, s))) return r;
+    if ((r = gemm(c, a, w.Wo2, w.bo2, M, d, d, EPI_RESID, c->h, d, s))) return r;
+    if ((r = ln_mod_launch<T>(c, n, base + 3 * d, base + 4 * d, cm, a, M, s))) return r;
+    if ((r = gemm(c, a, w.W1, w.b1, M, 4 * d, d, EPI_GELU, f, 4 * d, s))) return r;
+    if ((r = gemm(c, f, w.W2, w.b2, M, d, 4 * d, EPI_GATE, c->h, d, s, &g2))) return r;
+  }
+  const int wpb = 8, grid = (M + wpb - 1) / wpb, offf = L * 6 * d;
+  prof_begin(c, s, 3, 0.0);
+#define HM_CASE(V) TSDP_LAUNCH(c, (head_mod_kernel<V>), grid, wpb * 32, 0, s, c->h, n.mod, n.mod_ld, offf, offf + d, n.W_outT, n.b_out, cm, M, H, A, c->cfg.T)
+  switch (d / 128) {
+    case 1: HM_CASE(1); break; case 2: HM_CASE(2); break; case 3: HM_CASE(3); break; case 4: HM_CASE(4); break;
+    case 5: HM_CASE(5); break; case 6: HM_CASE(6); break; case 7: HM_CASE(7); break; default: HM_CASE(8); break;
+  }
+#undef HM_CASE
+  prof_end(c, s);
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  return TSDP_OK;
+}
+
+// Context tokens -> their cross-attention keys/values for every block (once per chunk), in the
+// activation type (they are tensor-core operands of the attention kernel).
+template <typename T>
+int dit_prepare_ctx_t(tsdp_ctx* c, Net& n, int B, cudaStream_t s) {
+  const int Tc = c->cfg.obs_tokens, d = n.cfg.d, L = n.cfg.layers;
+  T* mt = reinterpret_cast<T*>(c->memtok);
+  prof_begin(c, s, 3, 0.0);
+  TSDP_LAUNCH(c, (memtok_kernel<T>), B * Tc, d < 256 ? d : 256, 0, s, c->obs, c->cfg.obs_dim, n.W_obs, n.b_obs, n.cpos, Tc, 0, mt, d);
+  prof_end(c, s);
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  return gemm(c, mt, n.Wkv_all, n.bkv_all, B * Tc, L * 2 * d, d, c->cfg.precision == 0 ? EPI_F32 : EPI_STORE, n.kv_obs,
+              L * 2 * d, s);
+}
+
 int prepare_obs(tsdp_ctx* c, Net& n, int B, cudaStream_t s) {
+  if (n.cfg.arch == TSDP_ARCH_DIT)
+    return c->cfg.precision == 0 ? dit_prepare_ctx_t<float>(c, n, B, s) : dit_prepare_ctx_t<__nv_bfloat16>(c, n, B, s);
   if (n.cfg.arch != TSDP_ARCH_XFMR) return TSDP_OK;
   return c->cfg.precision == 0 ? xfmr_prepare_obs_t<float>(c, n, B, s) : xfmr_prepare_obs_t<__nv_bfloat16>(c, n, B, s);
 }
@@ -495,6 +643,9 @@ int forward(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStream_t s) 
     case TSDP_ARCH_XFMR:
       return c->cfg.precision == 0 ? xfmr_forward_t<float>(c, n, cm, n_cand, s)
                                    : xfmr_forward_t<__nv_bfloat16>(c, n, cm, n_cand, s);
+    case TSDP_ARCH_DIT:
+      return c->cfg.precision == 0 ? dit_forward_t<float>(c, n, cm, n_cand, s)
+                                   : dit_forward_t<__nv_bfloat16>(c, n, cm, n_cand, s);
   }
   return TSDP_ERR_UNSUPPORTED;
 }
@@ -693,7 +844,7 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
       (cfg->precision != 0 && cfg->precision != 1) || cfg->drafter < 0 || cfg->drafter > 2)
     return TSDP_ERR_ARG;
   for (const tsdp_net_t* n : {&cfg->base, &cfg->draft}) {
-    if (n->arch < TSDP_ARCH_GAUSS || n->arch > TSDP_ARCH_XFMR) return TSDP_ERR_UNSUPPORTED;
+    if (n->arch < TSDP_ARCH_GAUSS || n->arch > TSDP_ARCH_DIT) return TSDP_ERR_UNSUPPORTED;
     if (!net_cfg_ok(*cfg, *n)) return TSDP_ERR_ARG;
   }
   tsdp_ctx* c = new tsdp_ctx();
@@ -778,7 +929,7 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   const int esz = cfg->precision == 0 ? 4 : 2;
   for (int w = 0; w < 2; ++w) {
     const tsdp_net_t& n = w == TSDP_BASE ? cfg->base : cfg->draft;
-    if (n.arch != TSDP_ARCH_XFMR) continue;
+    if (n.arch != TSDP_ARCH_XFMR && n.arch != TSDP_ARCH_DIT) continue;
     const size_t M = (w == TSDP_BASE ? B * K1 : B) * cfg->H;
     rows_d = std::max(rows_d, M * n.d);
     rows_4d = std::max(rows_4d, M * 4 * n.d);
@@ -822,6 +973,9 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
     fprintf(stderr, "tsdp_init: the persistent cluster drafter does not fit this configuration\n");
     return fail(TSDP_ERR_UNSUPPORTED);
   }
+  INIT_TRY(cudaFuncSetAttribute(cross_attn_ctx_mma_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, cx_smem_bytes<32>(256)));
+  INIT_TRY(cudaFuncSetAttribute(cross_attn_ctx_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, cx_smem_bytes<64>(256)));
+  INIT_TRY(cudaFuncSetAttribute(cross_attn_ctx_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, cx_smem_bytes<128>(256)));
   INIT_TRY(cudaFuncSetAttribute(self_attn_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
   INIT_TRY(cudaFuncSetAttribute(self_attn_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
   c->net[TSDP_BASE].cfg = cfg->base;
@@ -958,6 +1112,104 @@ int tsdp_load_weights(tsdp_ctx* c, int which, const float* blob, size_t n) {
     float* tt;
     if ((r = sinus_table(net.cfg.temb, &tt))) return r;
     m.temb_table = tt;
+  } else if (net.cfg.arch == TSDP_ARCH_DIT) {
+    const size_t d = net.cfg.d, A = cfg.A, H = cfg.H, Tc = cfg.obs_tokens, L = net.cfg.layers;
+    if ((r = up_f32(&net.W_in, A * d))) return r;
+    if ((r = up_f32(&net.b_in, d))) return r;
+    if ((r = up_f32(&net.pos, H * d))) return r;
+    if ((r = up_f32(&net.W_obs, (size_t)cfg.obs_dim * d))) return r;
+    if ((r = up_f32(&net.b_obs, d))) return r;
+    if ((r = up_f32(&net.cpos, Tc * d))) return r;
+    // time path and modulation layers stay fp32: they only feed tables built below
+    const float *Wt1 = cur, *bt1 = cur + d * d, *Wt2 = bt1 + d, *bt2 = Wt2 + d * d;
+    cur = bt2 + d;
+    const size_t mod_ld = L * 6 * d + 2 * d;
+    std::vector<float> wmodT(mod_ld * d), bmod(mod_ld);          // [out = L*6d + 2d, in = d]
+    std::vector<float> wkv_all(d * L * 2 * d), bkv_all(L * 2 * d);
+    net.L.resize(L);
+    for (size_t l = 0; l < L; ++l) {
+      XfmrLayer& w = net.L[l];
+      for (size_t i = 0; i < d; ++i)
+        for (size_t o = 0; o < 6 * d; ++o) wmodT[(l * 6 * d + o) * d + i] = cur[i * 6 * d + o];
+      cur += d * 6 * d;
+      for (size_t o = 0; o < 6 * d; ++o) bmod[l * 6 * d + o] = cur[o];
+      cur += 6 * d;
+      if ((r = up_wT(&w.Wqkv, cur, d, 3 * d))) return r;
+      cur += d * 3 * d;
+      if ((r = up_f32(&w.bqkv, 3 * d))) return r;
+      if ((r = up_wT(&w.Wo, cur, d, d))) return r;
+      cur += d * d;
+      if ((r = up_f32(&w.bo, d))) return r;
+      if ((r = up_f32(&w.ln2_g, d))) return r;
+      if ((r = up_f32(&w.ln2_b, d))) return r;
+      if ((r = up_wT(&w.Wq2, cur, d, d))) return r;
+      cur += d * d;
+      if ((r = up_f32(&w.bq2, d))) return r;
+      for (size_t i = 0; i < d; ++i)
+        for (size_t o = 0; o < 2 * d; ++o) wkv_all[i * (L * 2 * d) + l * 2 * d + o] = cur[i * 2 * d + o];
+      cur += d * 2 * d;
+      for (size_t o = 0; o < 2 * d; ++o) bkv_all[l * 2 * d + o] = cur[o];
+      cur += 2 * d;
+      if ((r = up_wT(&w.Wo2, cur, d, d))) return r;
+      cur += d * d;
+      if ((r = up_f32(&w.bo2, d))) return r;
+      if ((r = up_wT(&w.W1, cur, d, 4 * d))) return r;
+      cur += d * 4 * d;
+      if ((r = up_f32(&w.b1, 4 * d))) return r;
+      if ((r = up_wT(&w.W2, cur, 4 * d, d))) return r;
+      cur += 4 * d * d;
+      if ((r = up_f32(&w.b2, d))) return r;
+    }
+    for (size_t i = 0; i < d; ++i)
+      for (size_t o = 0; o < 2 * d; ++o) wmodT[(L * 6 * d + o) * d + i] = cur[i * 2 * d + o];
+    cur += d * 2 * d;
+    for (size_t o = 0; o < 2 * d; ++o) bmod[L * 6 * d + o] = cur[o];
+    cur += 2 * d;
+    {   // W_out [d, A] -> fp32 [A, d]
+      std::vector<float> tmp(A * d);
+      for (size_t i = 0; i < d; ++i)
+        for (size_t a = 0; a < A; ++a) tmp[a * d + i] = cur[i * A + a];
+      cur += d * A;
+      if (dev_alloc(c, net.allocs, &net.W_outT, A * d)) return TSDP_ERR_CUDA;
+      CU_TRY(c, cudaMemcpy(net.W_outT, tmp.data(), tmp.size() * sizeof(float), cudaMemcpyHostToDevice));
+    }
+    if ((r = up_f32(&net.b_out, A))) return r;
+    if ((r = up_wT(&net.Wkv_all, wkv_all.data(), d, L * 2 * d))) return r;
+    if (dev_alloc(c, net.allocs, &net.bkv_all, L * 2 * d)) return TSDP_ERR_CUDA;
+    CU_TRY(c, cudaMemcpy(net.bkv_all, bkv_all.data(), bkv_all.size() * sizeof(float), cudaMemcpyHostToDevice));
+    if (dev_alloc(c, net.allocs, &net.kv_obs, c->items_cap * Tc * L * 2 * d)) return TSDP_ERR_CUDA;
+    if ((r = sinus_table((int)d, &net.temb_table))) return r;
+    // Tables of the timestep path, for every t: c = W_t2^T SiLU(W_t1^T sin(t) + b_t1) + b_t2, then every block's
+    // (shift, scale, gate) vectors and the final layer's = SiLU(c) W_mod + b_mod.
+    if (dev_alloc(c, net.allocs, &net.mod, (size_t)T * mod_ld)) return TSDP_ERR_CUDA;
+    net.mod_ld = (int)mod_ld;
+    std::vector<float> wt1T(d * d), wt2T(d * d);
+    for (size_t i = 0; i < d; ++i)
+      for (size_t o = 0; o < d; ++o) { wt1T[o * d + i] = Wt1[i * d + o]; wt2T[o * d + i] = Wt2[i * d + o]; }
+    std::vector<void*> tmp_pool;
+    float *d_w1, *d_b1, *d_w2, *d_b2, *d_wm, *d_bm, *d_hid, *d_c;
+    int st = 0;
+    st |= dev_alloc(c, tmp_pool, &d_w1, d * d); st |= dev_alloc(c, tmp_pool, &d_b1, d);
+    st |= dev_alloc(c, tmp_pool, &d_w2, d * d); st |= dev_alloc(c, tmp_pool, &d_b2, d);
+    st |= dev_alloc(c, tmp_pool, &d_wm, mod_ld * d); st |= dev_alloc(c, tmp_pool, &d_bm, mod_ld);
+    st |= dev_alloc(c, tmp_pool, &d_hid, (size_t)T * d); st |= dev_alloc(c, tmp_pool, &d_c, (size_t)T * d);
+    auto free_tmp = [&]() { for (void* q : tmp_pool) cudaFree(q); };
+    if (st) { free_tmp(); return TSDP_ERR_CUDA; }
+    cudaMemcpy(d_w1, wt1T.data(), d * d * 4, cudaMemcpyHostToDevice); cudaMemcpy(d_b1, bt1, d * 4, cudaMemcpyHostToDevice);
+    cudaMemcpy(d_w2, wt2T.data(), d * d * 4, cudaMemcpyHostToDevice); cudaMemcpy(d_b2, bt2, d * 4, cudaMemcpyHostToDevice);
+    cudaMemcpy(d_wm, wmodT.data(), mod_ld * d * 4, cudaMemcpyHostToDevice);
+    cudaMemcpy(d_bm, bmod.data(), mod_ld * 4, cudaMemcpyHostToDevice);
+    r = gemm_f32(c, net.temb_table, d_w1, d_b1, T, (int)d, (int)d, EPI_SILU, d_hid, 0);
+    if (!r) r = gemm_f32(c, d_hid, d_w2, d_b2, T, (int)d, (int)d, EPI_F32, d_c, 0);
+    if (!r) {
+      const long long nel = (long long)T * d;
+      silu_inplace_kernel<<<(unsigned)((nel + 255) / 256), 256>>>(d_c, nel);
+      r = gemm_f32(c, d_c, d_wm, d_bm, T, (int)mod_ld, (int)d, EPI_F32, net.mod, 0);
+    }
+    cudaError_t e = cudaDeviceSynchronize();
+    free_tmp();
+    if (r) return r;
+    CU_TRY(c, e);
   } else {
     const size_t d = net.cfg.d, A = cfg.A, H = cfg.H, To = cfg.obs_tokens, L = net.cfg.layers;
     if ((r = up_f32(&net.W_in, A * d))) return r;
@@ -1102,7 +1354,7 @@ static int ensure_items(tsdp_ctx* c, size_t N) {
   size_t dmax = 0;
   for (int w = 0; w < 2; ++w) {
     Net& n = c->net[w];
-    if (n.cfg.arch != TSDP_ARCH_XFMR) continue;
+    if (n.cfg.arch != TSDP_ARCH_XFMR && n.cfg.arch != TSDP_ARCH_DIT) continue;
     dmax = std::max(dmax, (size_t)n.cfg.d);
     if (n.loaded) st |= dev_alloc(c, n.allocs, &n.kv_obs, N * (To ? To : 1) * n.cfg.layers * 2 * n.cfg.d);
   }

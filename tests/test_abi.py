@@ -37,6 +37,9 @@ def test_weight_counts_match_the_packer(lib):
     for name, wl in inputs.WORKLOADS.items():
         if name == "serving_xfmr":
             wl = dict(wl, base=dict(wl["base"], layers=2))
+        if name == "vla_dit":                       # same architecture, sizes that a CPU test can afford
+            wl = dict(wl, To=16, Do=32, base=dict(wl["base"], layers=2, d=256, heads=4),
+                      draft=dict(wl["draft"], layers=1, d=128, heads=4))
         cfg = binding.make_config(wl["H"], wl["A"], wl["To"], wl["Do"], wl["base"], wl["draft"])
         for which, key in ((binding.BASE, "base"), (binding.DRAFT, "draft")):
             blob = binding.pack_weights(inputs.make_net(3, wl, key))

@@ -95,3 +95,32 @@ def test_transformer_denoiser(precision, tol, shape):
         err = hp.max_rel(out.cpu().numpy(), ref)
         assert err < tol, (which, err)
     smp.close()
+
+
+@pytest.mark.parametrize("precision,tol", [(0, 1e-4), (1, 2e-2)])
+@pytest.mark.parametrize("shape", ["small", "wide"])
+def test_dit_denoiser(precision, tol, shape):
+    """Adaptive-LayerNorm transformer against the oracle: gated residual epilogue, modulated LayerNorm,
+    bidirectional self-attention, cross-attention to the context tokens."""
+    rng = np.random.default_rng(3)
+    if shape == "small":
+        # 7 tokens, 12 context tokens (not a multiple of 16: the scalar context attention), head width 32
+        wl = dict(H=7, A=3, To=12, Do=5, T=100, precision=precision, gamma=1.0,
+                  base=dict(arch="dit", layers=2, d=128, heads=4), draft=dict(arch="dit", layers=1, d=256, heads=2))
+    else:
+        # 50 tokens, 48 context tokens (tensor-core context attention over a ragged 64-key chunk), head widths 64 / 128
+        wl = dict(H=50, A=14, To=48, Do=24, T=100, precision=precision, gamma=1.0,
+                  base=dict(arch="dit", layers=2, d=256, heads=4), draft=dict(arch="dit", layers=1, d=128, heads=1))
+    N = 9
+    smp, S, base, draft = hp.setup(wl, max_B=N, max_K=1)
+    x = rng.normal(size=(N, wl["H"], wl["A"])).astype(np.float32)
+    tau = rng.integers(0, 100, size=N).astype(np.int32); tau[0], tau[1] = 0, 99
+    obs = inputs.make_obs(5, N, wl["To"], wl["Do"])
+    dx = torch.tensor(x, device="cuda"); dobs = torch.tensor(obs, dtype=torch.float32, device="cuda")
+    for which, net in ((binding.BASE, base), (binding.DRAFT, draft)):
+        out = torch.zeros_like(dx)
+        smp.denoise(which, dx, tau, dobs, N, out)
+        ref = np.stack([net(x[n].astype(np.float64), int(tau[n]), obs[n]) for n in range(N)])
+        err = hp.max_rel(out.cpu().numpy(), ref)
+        assert err < tol, (which, err)
+    smp.close()

@@ -148,6 +148,22 @@ def test_chunk_pusht_transformer(precision, drafter):
         assert abs(st["drafts_accepted"] / max(st["draft_evals"], 1) - tot["accepted"] / max(tot["draft_evals"], 1)) < 0.15
 
 
+@pytest.mark.parametrize("precision,tol_eps,tol_x", [(0, 1e-4, 2e-5), (1, 2e-2, 3e-3)])
+def test_round_dit(precision, tol_eps, tol_x):
+    """One speculative round with the adaptive-LayerNorm transformer as base and drafter."""
+    wl = dict(H=10, A=4, To=16, Do=8, T=100, precision=precision, gamma=0.05,
+              base=dict(arch="dit", layers=2, d=128, heads=4), draft=dict(arch="dit", layers=1, d=128, heads=2))
+    _round_parity(wl, 4, 5, hp.accept_t(), 33, tol_eps, tol_x, [99, 60, 3, 0])
+
+
+def test_chunk_dit_fp32():
+    wl = dict(H=10, A=4, To=16, Do=8, T=100, precision=0, gamma=0.05,
+              base=dict(arch="dit", layers=2, d=128, heads=4), draft=dict(arch="dit", layers=1, d=128, heads=2))
+    B = 3
+    n_match, tot, st = _chunk_parity(wl, B, 6, hp.accept_t(), 41, 3e-2)
+    assert n_match >= B - 1
+
+
 def test_chunk_with_round_schedule_fp32():
     wl = hp.small_xfmr_workload(0, d=128, heads=4, layers=1, dd=128, dlayers=1, H=16, A=7, To=2, Do=64, gamma=0.03)
     Ks, Ss = inputs.markov_schedule(0, 40)

@@ -186,7 +186,6 @@ cross_attn_ctx_mma_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __
   __syncthreads();
   const float scale = rsqrtf((float)DH);
   const size_t row0 = (size_t)b * rows_per_slot;
-  const unsigned short* vraw = reinterpret_cast<const unsigned short*>(Vs);
   for (int qt = warp; qt * 16 < rows_per_slot; qt += CX_WARPS) {
     const int r0 = qt * 16 + g, r1 = r0 + 8;
     const __nv_bfloat16* q0 = q + (row0 + r0) * d + hd * DH;
@@ -210,13 +209,13 @@ cross_attn_ctx_mma_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __
 #pragma unroll
       for (int nt = 0; nt < 8; ++nt) {
         s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
-        const int key = k0 + nt * 8 + g;
         if (k0 + nt * 8 < Tc) {
 #pragma unroll
-          for (int ks = 0; ks < KS; ++ks) {
-            const int c = ks * 16 + 2 * tg;
-            mma_bf16_16816(s[nt], qa[ks], *reinterpret_cast<const uint32_t*>(Ks + (size_t)key * P + c),
-                           *reinterpret_cast<const uint32_t*>(Ks + (size_t)key * P + c + 8));
+          for (int ks = 0; ks < KS; ks += 2) {
+            uint32_t bk[4];
+            ldmatrix_x4(bk, Ks + (size_t)(k0 + nt * 8 + (lane & 7)) * P + ks * 16 + 8 * (lane >> 3));
+            mma_bf16_16816(s[nt], qa[ks], bk[0], bk[1]);
+            mma_bf16_16816(s[nt], qa[ks + 1], bk[2], bk[3]);
           }
         }
       }
@@ -252,13 +251,12 @@ cross_attn_ctx_mma_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __
           uint32_t pa[4];
           pa[0] = pack_bf16(s[2 * j][0], s[2 * j][1]); pa[1] = pack_bf16(s[2 * j][2], s[2 * j][3]);
           pa[2] = pack_bf16(s[2 * j + 1][0], s[2 * j + 1][1]); pa[3] = pack_bf16(s[2 * j + 1][2], s[2 * j + 1][3]);
-          const int kk = k0 + 16 * j + 2 * tg;
 #pragma unroll
-          for (int no = 0; no < NO; ++no) {
-            const int col = no * 8 + g;
-            const uint32_t b0 = (uint32_t)vraw[(size_t)kk * P + col] | ((uint32_t)vraw[(size_t)(kk + 1) * P + col] << 16);
-            const uint32_t b1 = (uint32_t)vraw[(size_t)(kk + 8) * P + col] | ((uint32_t)vraw[(size_t)(kk + 9) * P + col] << 16);
-            mma_bf16_16816(o[no], pa, b0, b1);
+          for (int no = 0; no < NO; no += 2) {
+            uint32_t bv[4];
+            ldmatrix_x4_trans(bv, Vs + (size_t)(k0 + 16 * j + (lane & 7) + 8 * ((lane >> 3) & 1)) * P + no * 8 + 8 * (lane >> 4));
+            mma_bf16_16816(o[no], pa, bv[0], bv[1]);
+            mma_bf16_16816(o[no + 1], pa, bv[2], bv[3]);
           }
         }
       }

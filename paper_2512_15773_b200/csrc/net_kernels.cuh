@@ -266,6 +266,20 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&h2);
 }
 
+// Four 8x8 b16 matrices from shared memory: lanes 8i..8i+7 give the 16-byte row addresses of matrix i.
+// Plain: lane l receives M[l/4][2(l%4) .. +1] -- the B fragment of a [n][k] (K-major) tile.
+// Transposed: lane l receives M[2(l%4) .. +1][l/4] -- the B fragment of a [k][n] tile (values V of attention).
+__device__ __forceinline__ void ldmatrix_x4(uint32_t r[4], const void* smem_row) {
+  const uint32_t a = (uint32_t)__cvta_generic_to_shared(smem_row);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t r[4], const void* smem_row) {
+  const uint32_t a = (uint32_t)__cvta_generic_to_shared(smem_row);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+
 constexpr int SA_WARPS = 4;
 
 template <int DH>
@@ -384,6 +398,122 @@ self_attn_mma_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __res
     if (row < H)
       *reinterpret_cast<uint4*>(out + ((size_t)n * H + row) * d + (size_t)hd * DH + v * 8) =
           *reinterpret_cast<const uint4*>(st + r * LDS + v * 8);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Self-attention for sequences longer than one 16-row tile (17..64 tokens), bf16: one block per
+// (candidate, head), one warp per 16-query tile.  The head's keys and values are staged once in
+// shared memory with 16-byte loads and become mma operands through ldmatrix (values transposed), so
+// no lane gathers 2-byte elements.  causal = 0 gives the bidirectional attention of the DiT blocks.
+// ------------------------------------------------------------------------------------------------
+template <int DH>
+__global__ void __launch_bounds__(128)
+self_attn_staged_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ out, int n_cand, int H, int d,
+                        int heads, int causal) {
+  pdl_trigger();
+  pdl_wait();
+  constexpr int KS = DH / 16, NO = DH / 8, P = DH + 8, VPR = DH / 8;
+  __shared__ __align__(16) __nv_bfloat16 Ks[64 * P], Vs[64 * P];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, tg = lane & 3;
+  const int n = blockIdx.x / heads, hd = blockIdx.x % heads;
+  const size_t ld = (size_t)3 * d;
+  const __nv_bfloat16* base = qkv + (size_t)n * H * ld + (size_t)hd * DH;
+  for (int i = threadIdx.x; i < 64 * VPR; i += blockDim.x) {
+    const int r = i / VPR, v = i % VPR;
+    uint4 kk = make_uint4(0u, 0u, 0u, 0u), vv = kk;
+    if (r < H) {
+      kk = __ldg(reinterpret_cast<const uint4*>(base + (size_t)r * ld + d) + v);
+      vv = __ldg(reinterpret_cast<const uint4*>(base + (size_t)r * ld + 2 * d) + v);
+    }
+    *reinterpret_cast<uint4*>(Ks + r * P + v * 8) = kk;
+    *reinterpret_cast<uint4*>(Vs + r * P + v * 8) = vv;
+  }
+  __syncthreads();
+  const int qt = warp;
+  if (qt * 16 >= H) return;
+  const int r0 = qt * 16 + g, r1 = r0 + 8;
+  auto ld32 = [&](int row, int col) -> uint32_t {
+    return row < H ? __ldg(reinterpret_cast<const uint32_t*>(base + (size_t)row * ld + col)) : 0u;
+  };
+  uint32_t qa[KS][4];
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks) {
+    const int c = ks * 16 + 2 * tg;
+    qa[ks][0] = ld32(r0, c); qa[ks][1] = ld32(r1, c); qa[ks][2] = ld32(r0, c + 8); qa[ks][3] = ld32(r1, c + 8);
+  }
+  const int nkt = causal ? 2 * (qt + 1) : (H + 7) >> 3;
+  const int kst = causal ? qt + 1 : (H + 15) >> 4;
+  float s[8][4];
+#pragma unroll
+  for (int nt = 0; nt < 8; ++nt) {
+    s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+    if (nt < nkt) {
+#pragma unroll
+      for (int ks = 0; ks < KS; ks += 2) {
+        uint32_t b[4];
+        ldmatrix_x4(b, Ks + (nt * 8 + (lane & 7)) * P + ks * 16 + 8 * (lane >> 3));
+        mma_bf16_16816(s[nt], qa[ks], b[0], b[1]);
+        mma_bf16_16816(s[nt], qa[ks + 1], b[2], b[3]);
+      }
+    }
+  }
+  const float scale = rsqrtf((float)DH);
+  float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+  for (int nt = 0; nt < 8; ++nt) {
+    if (nt < nkt) {
+      const int col = nt * 8 + 2 * tg;
+      const int lim0 = causal ? r0 : H, lim1 = causal ? r1 : H;
+      s[nt][0] = (col <= lim0 && col < H) ? s[nt][0] * scale : -INFINITY;
+      s[nt][1] = (col + 1 <= lim0 && col + 1 < H) ? s[nt][1] * scale : -INFINITY;
+      s[nt][2] = (col <= lim1 && col < H) ? s[nt][2] * scale : -INFINITY;
+      s[nt][3] = (col + 1 <= lim1 && col + 1 < H) ? s[nt][3] * scale : -INFINITY;
+      m0 = fmaxf(m0, fmaxf(s[nt][0], s[nt][1]));
+      m1 = fmaxf(m1, fmaxf(s[nt][2], s[nt][3]));
+    }
+  }
+  m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 1)); m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 2));
+  m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 1)); m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 2));
+  if (m0 == -INFINITY) m0 = 0.f;
+  if (m1 == -INFINITY) m1 = 0.f;
+  float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+  for (int nt = 0; nt < 8; ++nt) {
+    if (nt < nkt) {
+      s[nt][0] = __expf(s[nt][0] - m0); s[nt][1] = __expf(s[nt][1] - m0);
+      s[nt][2] = __expf(s[nt][2] - m1); s[nt][3] = __expf(s[nt][3] - m1);
+      l0 += s[nt][0] + s[nt][1]; l1 += s[nt][2] + s[nt][3];
+    }
+  }
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+  l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+  const float inv0 = l0 > 0.f ? 1.0f / l0 : 0.f, inv1 = l1 > 0.f ? 1.0f / l1 : 0.f;
+  float o[NO][4];
+#pragma unroll
+  for (int no = 0; no < NO; ++no) o[no][0] = o[no][1] = o[no][2] = o[no][3] = 0.f;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    if (j < kst) {
+      uint32_t pa[4];
+      pa[0] = pack_bf16(s[2 * j][0], s[2 * j][1]); pa[1] = pack_bf16(s[2 * j][2], s[2 * j][3]);
+      pa[2] = pack_bf16(s[2 * j + 1][0], s[2 * j + 1][1]); pa[3] = pack_bf16(s[2 * j + 1][2], s[2 * j + 1][3]);
+#pragma unroll
+      for (int no = 0; no < NO; no += 2) {
+        uint32_t b[4];
+        ldmatrix_x4_trans(b, Vs + (16 * j + (lane & 7) + 8 * ((lane >> 3) & 1)) * P + no * 8 + 8 * (lane >> 4));
+        mma_bf16_16816(o[no], pa, b[0], b[1]);
+        mma_bf16_16816(o[no + 1], pa, b[2], b[3]);
+      }
+    }
+  }
+  __nv_bfloat16* o0 = out + ((size_t)n * H + r0) * d + (size_t)hd * DH;
+  __nv_bfloat16* o1 = out + ((size_t)n * H + r1) * d + (size_t)hd * DH;
+#pragma unroll
+  for (int no = 0; no < NO; ++no) {
+    const int col = no * 8 + 2 * tg;
+    if (r0 < H) *reinterpret_cast<uint32_t*>(o0 + col) = pack_bf16(o[no][0] * inv0, o[no][1] * inv0);
+    if (r1 < H) *reinterpret_cast<uint32_t*>(o1 + col) = pack_bf16(o[no][2] * inv1, o[no][3] * inv1);
   }
 }
 

@@ -409,6 +409,12 @@ int self_attn_launch(tsdp_ctx* c, const T* qkv, T* out, int n_cand, int H, int d
   if constexpr (std::is_same<T, __nv_bfloat16>::value) {
     const int QT = (H + 15) / 16;
     const int grid = (n_cand * heads * QT + SA_WARPS - 1) / SA_WARPS;
+    if (H > 16 && (dh == 32 || dh == 64 || dh == 128)) {     // several query tiles share a head's K/V: stage them once
+      const int g2 = n_cand * heads;
+      if (dh == 32) TSDP_LAUNCH(c, (self_attn_staged_kernel<32>), g2, 128, 0, s, qkv, out, n_cand, H, d, heads, causal);
+      else if (dh == 64) TSDP_LAUNCH(c, (self_attn_staged_kernel<64>), g2, 128, 0, s, qkv, out, n_cand, H, d, heads, causal);
+      else TSDP_LAUNCH(c, (self_attn_staged_kernel<128>), g2, 128, 0, s, qkv, out, n_cand, H, d, heads, causal);
+    } else
     switch (dh) {
       case 32: TSDP_LAUNCH(c, (self_attn_mma_kernel<32>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads, causal); break;
       case 64: TSDP_LAUNCH(c, (self_attn_mma_kernel<64>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads, causal); break;

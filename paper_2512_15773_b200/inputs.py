@@ -153,7 +153,7 @@ WORKLOADS = {
     # VLA-scale action expert: 50 x 14 action chunk, 256 context tokens of width 1024
     "vla_dit": dict(H=50, A=14, To=256, Do=1024, T=100, precision=1,
                     base=dict(arch="dit", layers=18, d=1024, heads=16),
-                    draft=dict(arch="dit", layers=4, d=512, heads=8), B=64, K=16, gamma=0.03),
+                    draft=dict(arch="dit", layers=4, d=512, heads=8), B=64, K=16, gamma=0.012),
 }
 
 

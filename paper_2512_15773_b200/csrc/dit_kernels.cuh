@@ -159,7 +159,7 @@ __global__ void cross_attn_ctx_simt_kernel(const T* __restrict__ q, T* __restric
 // C * H query rows and runs S = Q K^T and O = P V on mma.sync over 64-key chunks with an online
 // softmax.  Tc <= 256, a multiple of 16.
 // ------------------------------------------------------------------------------------------------
-constexpr int CX_WARPS = 4;
+constexpr int CX_WARPS = 8;
 template <int DH>
 __host__ __device__ constexpr int cx_smem_bytes(int Tc) { return 2 * Tc * (DH + 8) * 2; }
 
@@ -172,6 +172,7 @@ cross_attn_ctx_mma_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __
   pdl_wait();
   extern __shared__ __align__(16) uint8_t cx_raw[];
   constexpr int P = DH + 8, KS = DH / 16, NO = DH / 8;
+  constexpr int CX_U = 1;      // query tiles a warp processes together (2 costs more in occupancy than it saves in shared-memory reads)
   __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(cx_raw);
   __nv_bfloat16* Vs = Ks + (size_t)Tc * P;
   const int b = blockIdx.x / heads, hd = blockIdx.x % heads;
@@ -186,89 +187,113 @@ cross_attn_ctx_mma_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __
   __syncthreads();
   const float scale = rsqrtf((float)DH);
   const size_t row0 = (size_t)b * rows_per_slot;
-  for (int qt = warp; qt * 16 < rows_per_slot; qt += CX_WARPS) {
-    const int r0 = qt * 16 + g, r1 = r0 + 8;
-    const __nv_bfloat16* q0 = q + (row0 + r0) * d + hd * DH;
-    const __nv_bfloat16* q1 = q + (row0 + r1) * d + hd * DH;
-    const bool v0 = r0 < rows_per_slot, v1 = r1 < rows_per_slot;
-    uint32_t qa[KS][4];
+  // A warp works on CX_U query tiles at a time, so that every key / value fragment read from shared
+  // memory feeds CX_U tensor-core instructions.
+  for (int pt = warp; pt * (16 * CX_U) < rows_per_slot; pt += CX_WARPS) {
+    int r0[CX_U], r1[CX_U];
+    bool v0[CX_U], v1[CX_U];
+    uint32_t qa[CX_U][KS][4];
+    float o[CX_U][NO][4];
+    float m0[CX_U], m1[CX_U], l0[CX_U], l1[CX_U];
 #pragma unroll
-    for (int ks = 0; ks < KS; ++ks) {
-      const int c = ks * 16 + 2 * tg;
-      qa[ks][0] = v0 ? *reinterpret_cast<const uint32_t*>(q0 + c) : 0u;
-      qa[ks][1] = v1 ? *reinterpret_cast<const uint32_t*>(q1 + c) : 0u;
-      qa[ks][2] = v0 ? *reinterpret_cast<const uint32_t*>(q0 + c + 8) : 0u;
-      qa[ks][3] = v1 ? *reinterpret_cast<const uint32_t*>(q1 + c + 8) : 0u;
+    for (int u = 0; u < CX_U; ++u) {
+      r0[u] = (pt * CX_U + u) * 16 + g; r1[u] = r0[u] + 8;
+      v0[u] = r0[u] < rows_per_slot; v1[u] = r1[u] < rows_per_slot;
+      const __nv_bfloat16* q0 = q + (row0 + r0[u]) * d + hd * DH;
+      const __nv_bfloat16* q1 = q + (row0 + r1[u]) * d + hd * DH;
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+        const int c = ks * 16 + 2 * tg;
+        qa[u][ks][0] = v0[u] ? *reinterpret_cast<const uint32_t*>(q0 + c) : 0u;
+        qa[u][ks][1] = v1[u] ? *reinterpret_cast<const uint32_t*>(q1 + c) : 0u;
+        qa[u][ks][2] = v0[u] ? *reinterpret_cast<const uint32_t*>(q0 + c + 8) : 0u;
+        qa[u][ks][3] = v1[u] ? *reinterpret_cast<const uint32_t*>(q1 + c + 8) : 0u;
+      }
+#pragma unroll
+      for (int no = 0; no < NO; ++no) o[u][no][0] = o[u][no][1] = o[u][no][2] = o[u][no][3] = 0.f;
+      m0[u] = m1[u] = -INFINITY; l0[u] = l1[u] = 0.f;
     }
-    float o[NO][4];
-#pragma unroll
-    for (int no = 0; no < NO; ++no) o[no][0] = o[no][1] = o[no][2] = o[no][3] = 0.f;
-    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
     for (int k0 = 0; k0 < Tc; k0 += 64) {
-      float s[8][4];
+      float s[CX_U][8][4];
 #pragma unroll
       for (int nt = 0; nt < 8; ++nt) {
-        s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+#pragma unroll
+        for (int u = 0; u < CX_U; ++u) s[u][nt][0] = s[u][nt][1] = s[u][nt][2] = s[u][nt][3] = 0.f;
         if (k0 + nt * 8 < Tc) {
 #pragma unroll
           for (int ks = 0; ks < KS; ks += 2) {
             uint32_t bk[4];
             ldmatrix_x4(bk, Ks + (size_t)(k0 + nt * 8 + (lane & 7)) * P + ks * 16 + 8 * (lane >> 3));
-            mma_bf16_16816(s[nt], qa[ks], bk[0], bk[1]);
-            mma_bf16_16816(s[nt], qa[ks + 1], bk[2], bk[3]);
+#pragma unroll
+            for (int u = 0; u < CX_U; ++u) {
+              mma_bf16_16816(s[u][nt], qa[u][ks], bk[0], bk[1]);
+              mma_bf16_16816(s[u][nt], qa[u][ks + 1], bk[2], bk[3]);
+            }
           }
         }
       }
-      float cm0 = -INFINITY, cm1 = -INFINITY;
 #pragma unroll
-      for (int nt = 0; nt < 8; ++nt) {
-        const bool vis = k0 + nt * 8 < Tc;                    // Tc is a multiple of 16: a tile is all in or all out
+      for (int u = 0; u < CX_U; ++u) {
+        float cm0 = -INFINITY, cm1 = -INFINITY;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) s[nt][e] = vis ? s[nt][e] * scale : -INFINITY;
-        cm0 = fmaxf(cm0, fmaxf(s[nt][0], s[nt][1]));
-        cm1 = fmaxf(cm1, fmaxf(s[nt][2], s[nt][3]));
+        for (int nt = 0; nt < 8; ++nt) {
+          const bool vis = k0 + nt * 8 < Tc;                  // Tc is a multiple of 16: a tile is all in or all out
+#pragma unroll
+          for (int e = 0; e < 4; ++e) s[u][nt][e] = vis ? s[u][nt][e] * scale : -INFINITY;
+          cm0 = fmaxf(cm0, fmaxf(s[u][nt][0], s[u][nt][1]));
+          cm1 = fmaxf(cm1, fmaxf(s[u][nt][2], s[u][nt][3]));
+        }
+        cm0 = fmaxf(cm0, __shfl_xor_sync(0xffffffffu, cm0, 1)); cm0 = fmaxf(cm0, __shfl_xor_sync(0xffffffffu, cm0, 2));
+        cm1 = fmaxf(cm1, __shfl_xor_sync(0xffffffffu, cm1, 1)); cm1 = fmaxf(cm1, __shfl_xor_sync(0xffffffffu, cm1, 2));
+        const float n0 = fmaxf(m0[u], cm0), n1 = fmaxf(m1[u], cm1);
+        const float f0 = __expf(m0[u] - n0), f1 = __expf(m1[u] - n1);   // exp(-inf) = 0 on the first chunk
+        m0[u] = n0; m1[u] = n1;
+        float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) {
+          s[u][nt][0] = __expf(s[u][nt][0] - n0); s[u][nt][1] = __expf(s[u][nt][1] - n0);
+          s[u][nt][2] = __expf(s[u][nt][2] - n1); s[u][nt][3] = __expf(s[u][nt][3] - n1);
+          a0 += s[u][nt][0] + s[u][nt][1]; a1 += s[u][nt][2] + s[u][nt][3];
+        }
+        a0 += __shfl_xor_sync(0xffffffffu, a0, 1); a0 += __shfl_xor_sync(0xffffffffu, a0, 2);
+        a1 += __shfl_xor_sync(0xffffffffu, a1, 1); a1 += __shfl_xor_sync(0xffffffffu, a1, 2);
+        l0[u] = l0[u] * f0 + a0; l1[u] = l1[u] * f1 + a1;
+#pragma unroll
+        for (int no = 0; no < NO; ++no) { o[u][no][0] *= f0; o[u][no][1] *= f0; o[u][no][2] *= f1; o[u][no][3] *= f1; }
       }
-      cm0 = fmaxf(cm0, __shfl_xor_sync(0xffffffffu, cm0, 1)); cm0 = fmaxf(cm0, __shfl_xor_sync(0xffffffffu, cm0, 2));
-      cm1 = fmaxf(cm1, __shfl_xor_sync(0xffffffffu, cm1, 1)); cm1 = fmaxf(cm1, __shfl_xor_sync(0xffffffffu, cm1, 2));
-      const float n0 = fmaxf(m0, cm0), n1 = fmaxf(m1, cm1);
-      const float f0 = __expf(m0 - n0), f1 = __expf(m1 - n1);  // exp(-inf) = 0 on the first chunk
-      m0 = n0; m1 = n1;
-      float a0 = 0.f, a1 = 0.f;
-#pragma unroll
-      for (int nt = 0; nt < 8; ++nt) {
-        s[nt][0] = __expf(s[nt][0] - m0); s[nt][1] = __expf(s[nt][1] - m0);
-        s[nt][2] = __expf(s[nt][2] - m1); s[nt][3] = __expf(s[nt][3] - m1);
-        a0 += s[nt][0] + s[nt][1]; a1 += s[nt][2] + s[nt][3];
-      }
-      a0 += __shfl_xor_sync(0xffffffffu, a0, 1); a0 += __shfl_xor_sync(0xffffffffu, a0, 2);
-      a1 += __shfl_xor_sync(0xffffffffu, a1, 1); a1 += __shfl_xor_sync(0xffffffffu, a1, 2);
-      l0 = l0 * f0 + a0; l1 = l1 * f1 + a1;
-#pragma unroll
-      for (int no = 0; no < NO; ++no) { o[no][0] *= f0; o[no][1] *= f0; o[no][2] *= f1; o[no][3] *= f1; }
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         if (k0 + 16 * j < Tc) {
-          uint32_t pa[4];
-          pa[0] = pack_bf16(s[2 * j][0], s[2 * j][1]); pa[1] = pack_bf16(s[2 * j][2], s[2 * j][3]);
-          pa[2] = pack_bf16(s[2 * j + 1][0], s[2 * j + 1][1]); pa[3] = pack_bf16(s[2 * j + 1][2], s[2 * j + 1][3]);
+          uint32_t pa[CX_U][4];
+#pragma unroll
+          for (int u = 0; u < CX_U; ++u) {
+            pa[u][0] = pack_bf16(s[u][2 * j][0], s[u][2 * j][1]); pa[u][1] = pack_bf16(s[u][2 * j][2], s[u][2 * j][3]);
+            pa[u][2] = pack_bf16(s[u][2 * j + 1][0], s[u][2 * j + 1][1]); pa[u][3] = pack_bf16(s[u][2 * j + 1][2], s[u][2 * j + 1][3]);
+          }
 #pragma unroll
           for (int no = 0; no < NO; no += 2) {
             uint32_t bv[4];
             ldmatrix_x4_trans(bv, Vs + (size_t)(k0 + 16 * j + (lane & 7) + 8 * ((lane >> 3) & 1)) * P + no * 8 + 8 * (lane >> 4));
-            mma_bf16_16816(o[no], pa, bv[0], bv[1]);
-            mma_bf16_16816(o[no + 1], pa, bv[2], bv[3]);
+#pragma unroll
+            for (int u = 0; u < CX_U; ++u) {
+              mma_bf16_16816(o[u][no], pa[u], bv[0], bv[1]);
+              mma_bf16_16816(o[u][no + 1], pa[u], bv[2], bv[3]);
+            }
           }
         }
       }
     }
-    const float i0 = 1.0f / l0, i1 = 1.0f / l1;
-    __nv_bfloat16* o0 = out + (row0 + r0) * d + hd * DH;
-    __nv_bfloat16* o1 = out + (row0 + r1) * d + hd * DH;
 #pragma unroll
-    for (int no = 0; no < NO; ++no) {
-      const int col = no * 8 + 2 * tg;
-      if (v0) *reinterpret_cast<uint32_t*>(o0 + col) = pack_bf16(o[no][0] * i0, o[no][1] * i0);
-      if (v1) *reinterpret_cast<uint32_t*>(o1 + col) = pack_bf16(o[no][2] * i1, o[no][3] * i1);
+    for (int u = 0; u < CX_U; ++u) {
+      const float i0 = 1.0f / l0[u], i1 = 1.0f / l1[u];
+      __nv_bfloat16* o0 = out + (row0 + r0[u]) * d + hd * DH;
+      __nv_bfloat16* o1 = out + (row0 + r1[u]) * d + hd * DH;
+#pragma unroll
+      for (int no = 0; no < NO; ++no) {
+        const int col = no * 8 + 2 * tg;
+        if (v0[u]) *reinterpret_cast<uint32_t*>(o0 + col) = pack_bf16(o[u][no][0] * i0, o[u][no][1] * i0);
+        if (v1[u]) *reinterpret_cast<uint32_t*>(o1 + col) = pack_bf16(o[u][no][2] * i1, o[u][no][3] * i1);
+      }
     }
   }
 }

@@ -1,4 +1,5 @@
-"""The denoisers eps = M(x, tau; obs) in numpy fp64: closed-form Gaussian toy, MLP, transformer, DiT.
+"""The denoisers eps = M(x, tau; obs) in numpy fp64: closed-form Gaussian toy, MLP, transformer, DiT,
+conv UNet.
 
 The paper states only the block counts ("DP consists of 8 Transformer blocks while the drafter
 contains only one", Sec. 4) and that the drafter has the same input-output interface and shares
@@ -139,6 +140,66 @@ def dit_eps(p, x, tau, ctx):
     return (layer_norm_plain(h) * (1.0 + kf) + sf) @ p["W_out"] + p["b_out"]
 
 
+# ----------------------------------------------------------------------------- conv UNet
+def mish(v):
+    return v * np.tanh(np.log1p(np.exp(-np.abs(v))) + np.maximum(v, 0.0))      # v tanh(softplus(v)), overflow-safe
+
+
+def conv1d_k5(x, W, b):
+    """x [L, C_in], W [5, C_in, C_out] (tap, in, out), zero padding 2:  y[l] = sum_j x[l + j - 2] W[j] + b."""
+    L = x.shape[0]
+    xp = np.vstack([np.zeros((2, x.shape[1])), x, np.zeros((2, x.shape[1]))])
+    return sum(xp[j:j + L] @ W[j] for j in range(5)) + b
+
+
+def group_norm(y, g, b, groups, eps=1e-5):
+    """GroupNorm over (positions x channels-of-the-group) of one sample; y [L, C]."""
+    L, C = y.shape
+    yg = y.reshape(L, groups, C // groups)
+    m = yg.mean(axis=(0, 2), keepdims=True)
+    v = ((yg - m) ** 2).mean(axis=(0, 2), keepdims=True)
+    return ((yg - m) / np.sqrt(v + eps)).reshape(L, C) * g + b
+
+
+def unet_resblock(R, x, mcond, groups):
+    """y = Mish(GN(conv5 x)); y = scale * y + bias (FiLM from Mish(cond)); y = Mish(GN(conv5 y)); out = y + res(x)."""
+    y = mish(group_norm(conv1d_k5(x, R["W1"], R["b1"]), R["g1"], R["be1"], groups))
+    film = mcond @ R["Wf"] + R["bf"]
+    C = y.shape[1]
+    y = film[:C] * y + film[C:]
+    y = mish(group_norm(conv1d_k5(y, R["W2"], R["b2"]), R["g2"], R["be2"], groups))
+    return y + (x @ R["Wr"] + R["br"] if "Wr" in R else x)
+
+
+def unet_eps(p, x, tau, obs):
+    """1-D temporal conv UNet over the H action positions (Robomimic-shaped configuration): channels
+    c, 2c, 4c; two FiLM residual blocks per level, 2:1 mean pooling down, 2x repetition up, skip
+    concatenation, two middle blocks; conditioning cond = [time vector | flattened obs].
+
+    tvec = Mish(sin(tau) W_t1 + b_t1) W_t2 + b_t2;  every block's FiLM = Mish(cond) W_f + b_f."""
+    groups = p["groups"]
+    tvec = mish(sinusoidal_embedding(tau, p["dt"]) @ p["Wt1"] + p["bt1"]) @ p["Wt2"] + p["bt2"]
+    mcond = mish(np.concatenate([tvec, obs.reshape(-1)]))
+    rb = iter(p["blocks"])
+    h = x @ p["W_in"] + p["b_in"]
+    skips = []
+    n_lv = p["levels"]
+    for lv in range(n_lv):
+        h = unet_resblock(next(rb), h, mcond, groups)
+        h = unet_resblock(next(rb), h, mcond, groups)
+        if lv < n_lv - 1:
+            skips.append(h)
+            h = 0.5 * (h[0::2] + h[1::2])
+    h = unet_resblock(next(rb), h, mcond, groups)
+    h = unet_resblock(next(rb), h, mcond, groups)
+    for lv in range(n_lv - 2, -1, -1):
+        h = np.concatenate([np.repeat(h, 2, axis=0), skips[lv]], axis=1)
+        h = unet_resblock(next(rb), h, mcond, groups)
+        h = unet_resblock(next(rb), h, mcond, groups)
+    h = mish(group_norm(conv1d_k5(h, p["Wh"], p["bh"]), p["gh"], p["beh"], groups))
+    return h @ p["W_out"] + p["b_out"]
+
+
 def make_denoiser(p, sched):
     """Return eps(x [H,A], tau, obs [To,Do]) for a parameter dict with key 'arch'."""
     arch = p["arch"]
@@ -150,4 +211,6 @@ def make_denoiser(p, sched):
         return lambda x, tau, obs: xfmr_eps(p, x, tau, obs)
     if arch == "dit":
         return lambda x, tau, obs: dit_eps(p, x, tau, obs)
+    if arch == "unet":
+        return lambda x, tau, obs: unet_eps(p, x, tau, obs)
     raise ValueError(arch)

@@ -115,6 +115,56 @@ def make_dit_params(seed, H, A, To, Do, d, heads, layers, out_scale=1.0, bf16=Tr
     return p
 
 
+def unet_block_channels(c, levels):
+    """(C_in, C_out) of the residual blocks of the conv UNet, in execution order."""
+    ch = [c * 2 ** i for i in range(levels)]
+    out, cin = [], c
+    for lv in range(levels):
+        out += [(cin, ch[lv]), (ch[lv], ch[lv])]
+        cin = ch[lv]
+    out += [(cin, cin), (cin, cin)]
+    for lv in range(levels - 2, -1, -1):
+        out += [(cin + ch[lv], ch[lv]), (ch[lv], ch[lv])]
+        cin = ch[lv]
+    return out
+
+
+def make_unet_params(seed, H, A, To, Do, c, levels, groups=8, dt=256, out_scale=1.0, bf16=True):
+    """Random 1-D conv UNet denoiser; conv / pointwise matrices bf16-representable when bf16=True, the
+    time path and the FiLM layers (tabulated in fp32 on the device) fp32-representable."""
+    rng = np.random.default_rng(seed)
+    q = bf16_round if bf16 else (lambda a: np.asarray(a, dtype=np.float32).astype(np.float64))
+    q32 = lambda a: np.asarray(a, dtype=np.float32).astype(np.float64)
+    dc = dt + To * Do
+    p = dict(arch="unet", c=c, levels=levels, groups=groups, dt=dt)
+    p["W_in"], p["b_in"] = _lin(rng, A, c, 1.0 / np.sqrt(A), q32)
+    p["Wt1"], p["bt1"] = _lin(rng, dt, 4 * dt, 1.0 / np.sqrt(dt), q32)
+    p["Wt2"], p["bt2"] = _lin(rng, 4 * dt, dt, 0.5 / np.sqrt(dt), q32)
+
+    def conv(cin, cout):
+        return q(rng.normal(0.0, 1.0 / np.sqrt(5 * cin), size=(5, cin, cout))), q32(rng.normal(0.0, 0.02, size=(cout,)))
+
+    blocks = []
+    for cin, cout in unet_block_channels(c, levels):
+        R = {}
+        R["W1"], R["b1"] = conv(cin, cout)
+        R["g1"], R["be1"] = q32(1.0 + rng.normal(0.0, 0.02, size=(cout,))), q32(rng.normal(0.0, 0.02, size=(cout,)))
+        Wf, bf = _lin(rng, dc, 2 * cout, 0.3 / np.sqrt(dc), q32)
+        bf = bf.copy(); bf[:cout] += 1.0                                   # FiLM starts near the identity
+        R["Wf"], R["bf"] = Wf, q32(bf)
+        R["W2"], R["b2"] = conv(cout, cout)
+        R["g2"], R["be2"] = q32(1.0 + rng.normal(0.0, 0.02, size=(cout,))), q32(rng.normal(0.0, 0.02, size=(cout,)))
+        if cin != cout:
+            R["Wr"], R["br"] = _lin(rng, cin, cout, 1.0 / np.sqrt(cin), q)
+        blocks.append(R)
+    p["blocks"] = blocks
+    p["Wh"], p["bh"] = conv(c, c)
+    p["gh"], p["beh"] = q32(1.0 + rng.normal(0.0, 0.02, size=(c,))), q32(rng.normal(0.0, 0.02, size=(c,)))
+    W, b = _lin(rng, c, A, 1.0 / np.sqrt(c), q32)
+    p["W_out"], p["b_out"] = q32(W * out_scale), q32(b * out_scale)
+    return p
+
+
 def make_sched_params(seed, H, A, To, Do, scale=1.0):
     """Random weights of the scheduler network (three stream encoders 64 / 64 / 16, aggregate MLP
     64, 5 outputs); fp32-representable.  `scale` multiplies the output layer."""
@@ -150,6 +200,10 @@ WORKLOADS = {
     "serving_xfmr": dict(H=16, A=7, To=2, Do=64, T=100, precision=1,
                          base=dict(arch="xfmr", layers=12, d=512, heads=8),
                          draft=dict(arch="xfmr", layers=2, d=256, heads=4), B=256, K=10, gamma=0.03),
+    # Robomimic-shaped conv-UNet policy: 16 x 10 action chunk, 2 x 512 visual features, channels 256/512/1024
+    "robomimic_unet": dict(H=16, A=10, To=2, Do=512, T=100, precision=1,
+                           base=dict(arch="unet", layers=3, d=256, heads=8, temb=256),
+                           draft=dict(arch="xfmr", layers=4, d=256, heads=4), B=32, K=8, gamma=0.03),
     # VLA-scale action expert: 50 x 14 action chunk, 256 context tokens of width 1024
     "vla_dit": dict(H=50, A=14, To=256, Do=1024, T=100, precision=1,
                     base=dict(arch="dit", layers=18, d=1024, heads=16),
@@ -168,6 +222,10 @@ def make_net(seed, wl, which, gamma=None, bf16=None):
         use_bf16 = (wl["precision"] == 1) if bf16 is None else bf16
         return make_xfmr_params(seed, wl["H"], wl["A"], wl["To"], wl["Do"], n["d"], n["heads"],
                                 n["layers"], out_scale=g, bf16=use_bf16)
+    if n["arch"] == "unet":
+        use_bf16 = (wl["precision"] == 1) if bf16 is None else bf16
+        return make_unet_params(seed, wl["H"], wl["A"], wl["To"], wl["Do"], n["d"], n["layers"], groups=n.get("heads", 8),
+                                dt=n.get("temb", 256), out_scale=g, bf16=use_bf16)
     if n["arch"] == "dit":
         use_bf16 = (wl["precision"] == 1) if bf16 is None else bf16
         return make_dit_params(seed, wl["H"], wl["A"], wl["To"], wl["Do"], n["d"], n["heads"], n["layers"],

@@ -37,6 +37,8 @@ def test_weight_counts_match_the_packer(lib):
     for name, wl in inputs.WORKLOADS.items():
         if name == "serving_xfmr":
             wl = dict(wl, base=dict(wl["base"], layers=2))
+        if name == "robomimic_unet":
+            wl = dict(wl, Do=16, base=dict(wl["base"], layers=2, d=128), draft=dict(wl["draft"], layers=1, d=128))
         if name == "vla_dit":                       # same architecture, sizes that a CPU test can afford
             wl = dict(wl, To=16, Do=32, base=dict(wl["base"], layers=2, d=256, heads=4),
                       draft=dict(wl["draft"], layers=1, d=128, heads=4))

@@ -142,3 +142,44 @@ def test_layer_norm_plain_is_layer_norm_with_unit_gain():
     h = np.random.default_rng(0).normal(size=(4, 16))
     assert np.allclose(nets.layer_norm_plain(h), nets.layer_norm(h, np.ones(16), np.zeros(16)))
     assert np.allclose(nets.layer_norm_plain(h).mean(-1), 0) and np.allclose(nets.layer_norm_plain(h).var(-1), 1, atol=1e-4)
+
+
+# ----------------------------------------------------------------------------- conv UNet (structure only)
+def _unet(seed=0, H=8, A=3, To=2, Do=4, c=16, levels=2):
+    p = inputs.make_unet_params(seed, H, A, To, Do, c, levels, groups=4, dt=8, bf16=False)
+    rng = np.random.default_rng(seed + 7)
+    return p, rng.normal(size=(H, A)), rng.normal(size=(To, Do))
+
+
+def test_unet_primitives_against_library_routines():
+    rng = np.random.default_rng(0)
+    x, W, b = rng.normal(size=(9, 3)), rng.normal(size=(5, 3, 4)), rng.normal(size=4)
+    y = nets.conv1d_k5(x, W, b)
+    for co in range(4):        # each output channel = sum over input channels of a 'same' cross-correlation
+        ref = sum(np.correlate(np.pad(x[:, ci], 2), W[:, ci, co], mode="valid") for ci in range(3)) + b[co]
+        assert np.allclose(y[:, co], ref)
+    v = rng.normal(size=100) * 5
+    assert np.allclose(nets.mish(v), v * np.tanh(np.log(1 + np.exp(v))))
+    z = rng.normal(size=(6, 8))
+    gn = nets.group_norm(z, np.ones(8), np.zeros(8), 2)
+    for g in range(2):
+        blk = gn[:, 4 * g:4 * g + 4]
+        assert abs(blk.mean()) < 1e-12 and abs(blk.var() - 1) < 1e-4
+
+
+def test_unet_block_channel_plan_and_receptive_field():
+    assert inputs.unet_block_channels(256, 3) == [(256, 256), (256, 256), (256, 512), (512, 512), (512, 1024), (1024, 1024),
+                                                  (1024, 1024), (1024, 1024), (1536, 512), (512, 512), (768, 256), (256, 256)]
+    p, x, obs = _unet()
+    e0 = nets.unet_eps(p, x, 30, obs)
+    assert e0.shape == x.shape
+    x2 = x.copy(); x2[0] += 1.0                       # through pooling and the middle blocks every position sees every other
+    assert np.abs(nets.unet_eps(p, x2, 30, obs)[-1] - e0[-1]).max() > 1e-12
+
+
+def test_unet_conditioning_enters_through_film_only():
+    p, x, obs = _unet(1)
+    q = dict(p, blocks=[dict(R, Wf=np.zeros_like(R["Wf"])) for R in p["blocks"]])
+    assert np.array_equal(nets.unet_eps(q, x, 5, obs), nets.unet_eps(q, x, 80, 2.0 * obs))
+    assert not np.allclose(nets.unet_eps(p, x, 5, obs), nets.unet_eps(p, x, 80, obs))
+    assert not np.allclose(nets.unet_eps(p, x, 5, obs), nets.unet_eps(p, x, 5, 2.0 * obs))

@@ -41,7 +41,7 @@ typedef enum {
   TSDP_ERR_TOO_LARGE = 8    /* size beyond the capacity of tsdp_verify_commit_static       */
 } tsdp_status;
 
-enum { TSDP_ARCH_GAUSS = 0, TSDP_ARCH_MLP = 1, TSDP_ARCH_XFMR = 2, TSDP_ARCH_DIT = 3 };
+enum { TSDP_ARCH_GAUSS = 0, TSDP_ARCH_MLP = 1, TSDP_ARCH_XFMR = 2, TSDP_ARCH_DIT = 3, TSDP_ARCH_UNET = 4 };
 enum { TSDP_BASE = 0, TSDP_DRAFT = 1, TSDP_SCHED = 2 };
 enum { TSDP_MAX_T = 1024, TSDP_MAX_K = 32 };
 
@@ -54,6 +54,10 @@ enum { TSDP_MAX_T = 1024, TSDP_MAX_K = 32 };
  *          scale / gate vectors, the obs_tokens (<= 256) observation/context tokens through
  *          cross-attention, self-attention over the H action tokens is bidirectional;
  *          h += g1 * SelfAttn(LN0(h)(1+k1)+s1) Wo;  h += CrossAttn(LN(h), ctx) Wo2;  h += g2 * MLP(LN0(h)(1+k2)+s2).
+ *   UNET : 1-D temporal conv UNet over the H action positions: `layers` levels with d, 2d, 4d.. channels, two
+ *          FiLM residual blocks per level (conv k5 -> GroupNorm(`heads` groups) -> Mish, FiLM scale/bias from
+ *          Mish([time vector (temb wide) | flattened obs])), 2:1 mean pooling down, 2x repetition up, skip
+ *          concatenation, two middle blocks, conv + pointwise head.  H a multiple of 2^(layers-1).
  * The paper fixes only the block counts (8 for the base policy, 1 for the drafter; Sec. 4). */
 typedef struct {
   int arch, layers, d, heads, temb;
@@ -129,6 +133,10 @@ size_t tsdp_weights_count(const tsdp_config_t* cfg, int which);
  *                     lnc_g, lnc_b, Wq2, bq2, Wkv2 [d,2d], bkv2, Wo2, bo2, W1, b1, W2, b2;
  *          Wmodf [d,2d], bmodf (shift, scale of the final layer), W_out [d,A], b_out.
  *          The time path (Wt*, Wmod*) is kept in fp32 and tabulated for every timestep during the load.
+ *   UNET : W_in [A,d], b_in, Wt1 [temb,4temb], bt1, Wt2 [4temb,temb], bt2; per residual block (C_in, C_out) in
+ *          execution order: W1 [5,C_in,C_out] (tap, in, out), b1, g1, be1, Wf [temb+obs_tokens*obs_dim, 2C_out], bf,
+ *          W2 [5,C_out,C_out], b2, g2, be2, and if C_in != C_out: Wr [C_in,C_out], br;
+ *          Wh [5,d,d], bh, gh, beh, W_out [d,A], b_out.  The time path and the FiLM layers stay fp32 (tabulated).
  *   SCHED (which = TSDP_SCHED, the scheduler network of Sec. 3.3, always fp32): W_o [obs_tokens*obs_dim, 64],
  *          b_o, W_a [H*A, 64], b_a, W_p [1, 16], b_p, W_1 [144, 64], b_1, W_2 [64, 5], b_2.
  * In precision 1 the large matrices are rounded to bf16.  Errors: WEIGHTS (n mismatch), NAN, CUDA. */

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libtsdp.so")
 
 TSDP_MAX_T = 1024
-ARCH = {"gauss": 0, "mlp": 1, "xfmr": 2, "dit": 3}
+ARCH = {"gauss": 0, "mlp": 1, "xfmr": 2, "dit": 3, "unet": 4}
 BASE, DRAFT, SCHED = 0, 1, 2
 EXPORTS = ["tsdp_init", "tsdp_destroy", "tsdp_strerror", "tsdp_last_error", "tsdp_weights_count",
            "tsdp_load_weights", "tsdp_set_schedule", "tsdp_sample_chunk", "tsdp_sample_chunk_host",
@@ -113,6 +113,13 @@ def pack_weights(p):
         parts = []
         for W, b in zip(p["W"], p["b"]):
             parts += [W, b]
+    elif a == "unet":
+        parts = [p[k] for k in ("W_in", "b_in", "Wt1", "bt1", "Wt2", "bt2")]
+        for R in p["blocks"]:
+            parts += [R[k] for k in ("W1", "b1", "g1", "be1", "Wf", "bf", "W2", "b2", "g2", "be2")]
+            if "Wr" in R:
+                parts += [R["Wr"], R["br"]]
+        parts += [p[k] for k in ("Wh", "bh", "gh", "beh", "W_out", "b_out")]
     elif a == "dit":
         parts = [p[k] for k in ("W_in", "b_in", "pos", "W_ctx", "b_ctx", "cpos", "Wt1", "bt1", "Wt2", "bt2")]
         for L in p["layers"]:

@@ -27,7 +27,8 @@ namespace tsdp {
 
 // EPI_GATE: fp32 out += gate[tau(row), col] * (acc + bias), the gated residual of an adaptive-LayerNorm block.
 // EPI_SILU: fp32 store of SiLU(acc + bias); CUDA-core GEMM only (conditioning tables built at load).
-enum { EPI_STORE = 0, EPI_GELU = 1, EPI_RESID = 2, EPI_F32 = 3, EPI_GATE = 4, EPI_SILU = 5 };
+// EPI_MISH: as EPI_SILU with Mish.
+enum { EPI_STORE = 0, EPI_GELU = 1, EPI_RESID = 2, EPI_F32 = 3, EPI_GATE = 4, EPI_SILU = 5, EPI_MISH = 6 };
 
 constexpr int GEMM_BM = 128;
 constexpr int GEMM_BK = 64;
@@ -193,6 +194,11 @@ struct GemmArgs {
   int gate_ld;
   const int* t;
   int C, koff, H, Tsteps;
+  int lda;              // row pitch of A in elements (CUDA-core GEMM; the tensor-core one has it in its tensor map)
+  // Kernel-5 convolution over a zero-padded channels-last tensor [rows, conv_c] (0: plain GEMM): logical A row m
+  // is the 5 conv_c elements starting at tensor row m, so k-block kb is tensor rows m + tap, columns
+  // [c0, c0 + 64) with tap = (64 kb) / conv_c, c0 = (64 kb) % conv_c; conv_c is a multiple of 64.
+  int conv_c;
 };
 
 __device__ __forceinline__ const float* gate_row(const GemmArgs& g, int row) {
@@ -298,7 +304,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           if (!ptx::mbar_wait_thread(empty_bar(stage), phase ^ 1u)) { ok = false; break; }
           ptx::mbar_expect_tx(full_bar(stage), STAGE_BYTES);
           const uint32_t sa = base + stage * STAGE_BYTES;
-          ptx::tma_load_2d(sa, &tmA, kb * GEMM_BK, tm * GEMM_BM, full_bar(stage));
+          const int kcol = kb * GEMM_BK;
+          const int ax = g.conv_c ? kcol % g.conv_c : kcol, ay = tm * GEMM_BM + (g.conv_c ? kcol / g.conv_c : 0);
+          ptx::tma_load_2d(sa, &tmA, ax, ay, full_bar(stage));
           ptx::tma_load_2d(sa + A_BYTES, &tmB, kb * GEMM_BK, tn * BN, full_bar(stage));
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }

@@ -22,8 +22,8 @@ gemm_simt_kernel(const float* __restrict__ A, const float* __restrict__ W, GemmA
   for (int k0 = 0; k0 < g.K; k0 += 16) {
     for (int i = threadIdx.x; i < 64 * 16; i += 256) {
       const int r = i >> 4, k = i & 15;
-      As[k][r] = (m0 + r < g.M) ? A[(size_t)(m0 + r) * g.K + k0 + k] : 0.f;
-      Ws[k][r] = (n0 + r < g.N) ? W[(size_t)(n0 + r) * g.K + k0 + k] : 0.f;
+      As[k][r] = (m0 + r < g.M && k0 + k < g.K) ? A[(size_t)(m0 + r) * g.lda + k0 + k] : 0.f;
+      Ws[k][r] = (n0 + r < g.N && k0 + k < g.K) ? W[(size_t)(n0 + r) * g.K + k0 + k] : 0.f;
     }
     __syncthreads();
 #pragma unroll
@@ -47,6 +47,7 @@ gemm_simt_kernel(const float* __restrict__ A, const float* __restrict__ W, GemmA
       float v = acc[i][j] + (g.bias ? g.bias[col] : 0.f);
       if (EPI == EPI_GELU) v = gelu_tanh(v);
       if (EPI == EPI_SILU) v = v / (1.0f + expf(-v));
+      if (EPI == EPI_MISH) v = v * tanhf(v > 20.f ? v : log1pf(expf(v)));
       if (EPI == EPI_GATE) v *= gate_row(g, row)[col];
       float* o = reinterpret_cast<float*>(g.out) + (size_t)row * g.ldo + col;
       if (EPI == EPI_RESID || EPI == EPI_GATE) v += *o;

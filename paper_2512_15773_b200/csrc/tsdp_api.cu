@@ -22,6 +22,7 @@
 #include "drafter_cluster.cuh"
 #include "sched_kernel.cuh"
 #include "dit_kernels.cuh"
+#include "unet_kernels.cuh"
 
 using namespace tsdp;
 
@@ -51,6 +52,17 @@ struct Net {
   float* temb_table = nullptr;                // [T, temb or d] sinusoidal embedding
   float* mod = nullptr;                       // DIT: [T, L*6d + 2d] shift / scale / gate vectors of every timestep
   int mod_ld = 0;
+  // UNET: residual blocks in execution order, FiLM tables, head
+  struct UBlock { int cin, cout, foff; void *W1, *W2, *Wr; float *b1, *g1, *be1, *b2, *g2, *be2, *br; };
+  std::vector<UBlock> ub;
+  int F = 0;                                  // FiLM width: sum over blocks of 2 * cout
+  float *film_time = nullptr, *film_obs = nullptr, *WfT_obs = nullptr, *obs_m = nullptr;   // [T,F], [items,F], [F,To*Do], [items,To*Do]
+  void* Wh = nullptr;
+  float *bh = nullptr, *gh = nullptr, *beh = nullptr;
+  // UNET activations (zero-padded channels-last tensors, see unet_kernels.cuh), allocated at init
+  struct UWs { void *X0 = nullptr, *E = nullptr, *M1 = nullptr, *M2 = nullptr, *HB = nullptr;
+               void *TMP[4] = {}, *D[4] = {}, *CAT[4] = {}, *P[4] = {}, *U1[4] = {}, *U2[4] = {};
+               float *Y = nullptr, *R = nullptr; } uw;
   std::vector<void*> allocs;
 };
 
@@ -167,6 +179,17 @@ void prof_end(tsdp_ctx* c, cudaStream_t s) {
   cudaEventRecord(c->prof_ev.back(), s);
 }
 
+// (C_in, C_out) of the residual blocks of the conv UNet in execution order: two per level down, two in the
+// middle, two per level up (the first of which takes the concatenation [upsampled | skip]).
+std::vector<std::pair<int, int>> unet_channels(int c, int levels) {
+  std::vector<std::pair<int, int>> out;
+  int cin = c;
+  for (int lv = 0; lv < levels; ++lv) { out.push_back({cin, c << lv}); out.push_back({c << lv, c << lv}); cin = c << lv; }
+  out.push_back({cin, cin}); out.push_back({cin, cin});
+  for (int lv = levels - 2; lv >= 0; --lv) { out.push_back({cin + (c << lv), c << lv}); out.push_back({c << lv, c << lv}); cin = c << lv; }
+  return out;
+}
+
 bool net_cfg_ok(const tsdp_config_t& cfg, const tsdp_net_t& n) {
   if (n.arch == TSDP_ARCH_GAUSS) return true;
   if (n.arch == TSDP_ARCH_MLP)
@@ -174,6 +197,10 @@ bool net_cfg_ok(const tsdp_config_t& cfg, const tsdp_net_t& n) {
   if (n.arch == TSDP_ARCH_XFMR)
     return n.layers >= 1 && n.d % 128 == 0 && n.d >= 128 && n.d <= 1024 && n.heads >= 1 && n.d % n.heads == 0 &&
            (n.d / n.heads) % 32 == 0 && (n.d / n.heads) <= 128 && cfg.H <= 64 && cfg.obs_tokens <= 8 && cfg.A <= 64;
+  if (n.arch == TSDP_ARCH_UNET)
+    return n.layers >= 1 && n.layers <= 4 && n.d % 128 == 0 && n.d >= 128 && (n.d << (n.layers - 1)) <= 2048 && n.heads >= 1 &&
+           n.d % n.heads == 0 && n.temb >= 4 && n.temb % 4 == 0 && cfg.H % (1 << (n.layers - 1)) == 0 && cfg.H <= 64 &&
+           cfg.A <= 64;
   if (n.arch == TSDP_ARCH_DIT)
     return n.layers >= 1 && n.d % 128 == 0 && n.d >= 128 && n.d <= 1024 && n.heads >= 1 && n.d % n.heads == 0 &&
            (n.d / n.heads) % 32 == 0 && (n.d / n.heads) <= 128 && cfg.H <= 64 && cfg.obs_tokens >= 1 &&
@@ -194,6 +221,15 @@ size_t weights_count(const tsdp_config_t& cfg, const tsdp_net_t& n) {
     const size_t per = 2 * d + d * 3 * d + 3 * d + d * d + d + 2 * d + d * d + d + d * 2 * d + 2 * d + d * d + d + 2 * d +
                        d * 4 * d + 4 * d + 4 * d * d + d;
     return tot + per * n.layers + 2 * d + d * cfg.A + cfg.A;
+  }
+  if (n.arch == TSDP_ARCH_UNET) {
+    const size_t dt = n.temb, dc = dt + (size_t)cfg.obs_tokens * cfg.obs_dim;
+    size_t tot = (size_t)cfg.A * d + d + dt * 4 * dt + 4 * dt + 4 * dt * dt + dt;
+    for (auto& cc : unet_channels((int)d, n.layers)) {
+      const size_t ci = cc.first, co = cc.second;
+      tot += 5 * ci * co + co + 2 * co + dc * 2 * co + 2 * co + 5 * co * co + co + 2 * co + (ci != co ? ci * co + co : 0);
+    }
+    return tot + 5 * d * d + d + 2 * d + d * cfg.A + cfg.A;
   }
   if (n.arch == TSDP_ARCH_DIT) {
     size_t tot = (size_t)cfg.A * d + d + (size_t)cfg.H * d + (size_t)cfg.obs_dim * d + d + (size_t)cfg.obs_tokens * d +
@@ -294,9 +330,9 @@ struct GateSpec {
 };
 
 int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, int N, int K, int epi, void* out,
-         int ldo, cudaStream_t s, const GateSpec* gs = nullptr) {
+         int ldo, cudaStream_t s, const GateSpec* gs = nullptr, int conv_c = 0) {
   if (M <= 0) return TSDP_OK;
-  GemmArgs g{M, N, K, bias, out, ldo, c->status, nullptr, 0, nullptr, 1, 0, 1, 1};
+  GemmArgs g{M, N, K, bias, out, ldo, c->status, nullptr, 0, nullptr, 1, 0, 1, 1, conv_c > 0 ? conv_c : K, conv_c};
   if (epi == EPI_GATE) {
     if (!gs) return TSDP_ERR_ARG;
     g.gate = gs->gate; g.gate_ld = gs->gate_ld; g.t = gs->cm->t; g.C = gs->cm->C; g.koff = gs->cm->koff; g.H = gs->H;
@@ -325,7 +361,10 @@ int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, in
   const int BN = pick_bn(M, N, c->num_sms);
   CUtensorMap ma, mb, mc;
   int r;
-  if ((r = get_map(c, A, 2, M, K, K, GEMM_BK, GEMM_BM, &ma)) != TSDP_OK) return r;
+  if (conv_c > 0) {      // kernel-5 convolution: A is the padded tensor [M + 4, conv_c] itself
+    if (conv_c % GEMM_BK != 0 || K != 5 * conv_c) return TSDP_ERR_ARG;
+    if ((r = get_map(c, A, 2, M + 4, conv_c, conv_c, GEMM_BK, GEMM_BM, &ma)) != TSDP_OK) return r;
+  } else if ((r = get_map(c, A, 2, M, K, K, GEMM_BK, GEMM_BM, &ma)) != TSDP_OK) return r;
   if ((r = get_map(c, W, 2, N, K, K, GEMM_BK, BN, &mb)) != TSDP_OK) return r;
   mc = ma;
   if (gemm_tma_epilogue(BN)) {   // the epilogue hands 128-row x 128-byte chunks to TMA
@@ -347,9 +386,10 @@ int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, in
 // fp32 CUDA-core GEMM whatever the precision mode: the timestep-conditioning tables built at weight load.
 int gemm_f32(tsdp_ctx* c, const float* A, const float* W, const float* bias, int M, int N, int K, int epi, float* out,
              cudaStream_t s) {
-  GemmArgs g{M, N, K, bias, out, N, c->status, nullptr, 0, nullptr, 1, 0, 1, 1};
+  GemmArgs g{M, N, K, bias, out, N, c->status, nullptr, 0, nullptr, 1, 0, 1, 1, K, 0};
   dim3 grid((N + 63) / 64, (M + 63) / 64);
-  if (epi == EPI_SILU) TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_SILU>), grid, 256, 0, s, A, W, g);
+  if (epi == EPI_MISH) TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_MISH>), grid, 256, 0, s, A, W, g);
+  else if (epi == EPI_SILU) TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_SILU>), grid, 256, 0, s, A, W, g);
   else TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_F32>), grid, 256, 0, s, A, W, g);
   CU_TRY(c, cudaGetLastError());
   return TSDP_OK;
@@ -615,7 +655,108 @@ int dit_prepare_ctx_t(tsdp_ctx* c, Net& n, int B, cudaStream_t s) {
               L * 2 * d, s);
 }
 
+// ------------------------------------------------------------------------------------------ conv UNet
+template <typename T>
+int unet_gn(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, const float* gam, const float* bet, int foff, const T* res_t,
+            int res_pitch, const float* res_f, T* dst, int dst_pitch, int coff, int L, int C, cudaStream_t s) {
+  prof_begin(c, s, 1, 0.0);
+  TSDP_LAUNCH(c, (gn_mish_kernel<T>), n_cand * n.cfg.heads, 256, 0, s, n.uw.Y, gam, bet, n.cfg.heads,
+              foff >= 0 ? n.film_time : nullptr, n.film_obs, n.F, foff >= 0 ? foff : 0, cm, c->cfg.T, res_t, res_pitch, res_f, dst,
+              dst_pitch, coff, L, C);
+  prof_end(c, s);
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  return TSDP_OK;
+}
+
+// One FiLM residual block: xin [n, L+4, cin] -> dst[n, L+4, coff .. coff+cout) of a tensor of pitch dst_pitch.
+template <typename T>
+int unet_resblock(tsdp_ctx* c, Net& n, const Net::UBlock& b, const CandMap& cm, int n_cand, const T* xin, T* tmp, T* dst,
+                  int dst_pitch, int coff, int L, cudaStream_t s) {
+  const int rows = n_cand * (L + 4);
+  int r;
+  if ((r = gemm(c, xin, b.W1, b.b1, rows - 4, b.cout, 5 * b.cin, EPI_F32, n.uw.Y, b.cout, s, nullptr, b.cin))) return r;
+  if ((r = unet_gn<T>(c, n, cm, n_cand, b.g1, b.be1, b.foff, nullptr, 0, nullptr, tmp, b.cout, 0, L, b.cout, s))) return r;
+  if ((r = gemm(c, tmp, b.W2, b.b2, rows - 4, b.cout, 5 * b.cout, EPI_F32, n.uw.Y, b.cout, s, nullptr, b.cout))) return r;
+  if (b.Wr) {
+    if ((r = gemm(c, xin, b.Wr, b.br, rows, b.cout, b.cin, EPI_F32, n.uw.R, b.cout, s))) return r;
+    return unet_gn<T>(c, n, cm, n_cand, b.g2, b.be2, -1, nullptr, 0, n.uw.R, dst, dst_pitch, coff, L, b.cout, s);
+  }
+  return unet_gn<T>(c, n, cm, n_cand, b.g2, b.be2, -1, xin, b.cin, nullptr, dst, dst_pitch, coff, L, b.cout, s);
+}
+
+template <typename T>
+int unet_forward_t(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStream_t s) {
+  const int H = c->cfg.H, A = c->cfg.A, ch = n.cfg.d, LV = n.cfg.layers, last = LV - 1;
+  auto P = [](void* p) { return reinterpret_cast<T*>(p); };
+  int r, bi = 0;
+  prof_begin(c, s, 3, 0.0);
+  TSDP_LAUNCH(c, (unet_embed_kernel<T>), n_cand * H, ch < 256 ? ch : 256, 0, s, cm, n.W_in, n.b_in, P(n.uw.X0), H, A, ch);
+  prof_end(c, s);
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  const T* x = P(n.uw.X0);
+  for (int lv = 0; lv < LV; ++lv) {
+    const int L = H >> lv, C = ch << lv;
+    if ((r = unet_resblock<T>(c, n, n.ub[bi++], cm, n_cand, x, P(n.uw.TMP[lv]), P(n.uw.D[lv]), C, 0, L, s))) return r;
+    if (lv < last) {
+      const int Cup = ch << (lv + 1), Ccat = Cup + C;
+      if ((r = unet_resblock<T>(c, n, n.ub[bi++], cm, n_cand, P(n.uw.D[lv]), P(n.uw.TMP[lv]), P(n.uw.CAT[lv]), Ccat, Cup, L, s))) return r;
+      const long long tot = (long long)n_cand * (L / 2) * C;
+      prof_begin(c, s, 3, 0.0);
+      TSDP_LAUNCH(c, (unet_pool_kernel<T>), (unsigned)((tot + 255) / 256), 256, 0, s, P(n.uw.CAT[lv]), Ccat, Cup, P(n.uw.P[lv]),
+                  n_cand, L / 2, C);
+      prof_end(c, s);
+      c->launches_per_round_tmp++;
+      CU_TRY(c, cudaGetLastError());
+      x = P(n.uw.P[lv]);
+    } else {
+      if ((r = unet_resblock<T>(c, n, n.ub[bi++], cm, n_cand, P(n.uw.D[lv]), P(n.uw.TMP[lv]), P(n.uw.E), C, 0, L, s))) return r;
+    }
+  }
+  {
+    const int L = H >> last, C = ch << last;
+    if ((r = unet_resblock<T>(c, n, n.ub[bi++], cm, n_cand, P(n.uw.E), P(n.uw.TMP[last]), P(n.uw.M1), C, 0, L, s))) return r;
+    if ((r = unet_resblock<T>(c, n, n.ub[bi++], cm, n_cand, P(n.uw.M1), P(n.uw.TMP[last]), P(n.uw.M2), C, 0, L, s))) return r;
+  }
+  const T* cur = P(n.uw.M2);
+  for (int lv = last - 1; lv >= 0; --lv) {
+    const int L = H >> lv, C = ch << lv, Cup = ch << (lv + 1), Ccat = Cup + C;
+    const long long tot = (long long)n_cand * L * Cup;
+    prof_begin(c, s, 3, 0.0);
+    TSDP_LAUNCH(c, (unet_upsample_kernel<T>), (unsigned)((tot + 255) / 256), 256, 0, s, cur, P(n.uw.CAT[lv]), Ccat, n_cand, L, Cup);
+    prof_end(c, s);
+    c->launches_per_round_tmp++;
+    CU_TRY(c, cudaGetLastError());
+    if ((r = unet_resblock<T>(c, n, n.ub[bi++], cm, n_cand, P(n.uw.CAT[lv]), P(n.uw.TMP[lv]), P(n.uw.U1[lv]), C, 0, L, s))) return r;
+    if ((r = unet_resblock<T>(c, n, n.ub[bi++], cm, n_cand, P(n.uw.U1[lv]), P(n.uw.TMP[lv]), P(n.uw.U2[lv]), C, 0, L, s))) return r;
+    cur = P(n.uw.U2[lv]);
+  }
+  const int rows = n_cand * (H + 4);
+  if ((r = gemm(c, cur, n.Wh, n.bh, rows - 4, ch, 5 * ch, EPI_F32, n.uw.Y, ch, s, nullptr, ch))) return r;
+  if ((r = unet_gn<T>(c, n, cm, n_cand, n.gh, n.beh, -1, nullptr, 0, nullptr, P(n.uw.HB), ch, 0, H, ch, s))) return r;
+  prof_begin(c, s, 3, 0.0);
+  TSDP_LAUNCH(c, (unet_head_kernel<T>), (n_cand * H + 7) / 8, 256, 0, s, P(n.uw.HB), n.W_outT, n.b_out, cm, n_cand * H, H, A, ch);
+  prof_end(c, s);
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  return TSDP_OK;
+}
+
+// FiLM contribution of every request's observation: film_obs = Mish(obs_flat) Wf_obs (once per chunk).
+int unet_prepare_obs(tsdp_ctx* c, Net& n, int N, cudaStream_t s) {
+  const int dobs = c->cfg.obs_tokens * c->cfg.obs_dim;
+  if (dobs == 0) return TSDP_OK;
+  const long long tot = (long long)N * dobs;
+  TSDP_LAUNCH(c, (mish_kernel), (unsigned)((tot + 255) / 256), 256, 0, s, c->obs, n.obs_m, tot);
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  c->launches_per_round_tmp++;
+  return gemm_f32(c, n.obs_m, n.WfT_obs, nullptr, N, n.F, dobs, EPI_F32, n.film_obs, s);
+}
+
 int prepare_obs(tsdp_ctx* c, Net& n, int B, cudaStream_t s) {
+  if (n.cfg.arch == TSDP_ARCH_UNET) return unet_prepare_obs(c, n, B, s);
   if (n.cfg.arch == TSDP_ARCH_DIT)
     return c->cfg.precision == 0 ? dit_prepare_ctx_t<float>(c, n, B, s) : dit_prepare_ctx_t<__nv_bfloat16>(c, n, B, s);
   if (n.cfg.arch != TSDP_ARCH_XFMR) return TSDP_OK;
@@ -652,6 +793,9 @@ int forward(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStream_t s) 
     case TSDP_ARCH_DIT:
       return c->cfg.precision == 0 ? dit_forward_t<float>(c, n, cm, n_cand, s)
                                    : dit_forward_t<__nv_bfloat16>(c, n, cm, n_cand, s);
+    case TSDP_ARCH_UNET:
+      return c->cfg.precision == 0 ? unet_forward_t<float>(c, n, cm, n_cand, s)
+                                   : unet_forward_t<__nv_bfloat16>(c, n, cm, n_cand, s);
   }
   return TSDP_ERR_UNSUPPORTED;
 }
@@ -850,7 +994,7 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
       (cfg->precision != 0 && cfg->precision != 1) || cfg->drafter < 0 || cfg->drafter > 2)
     return TSDP_ERR_ARG;
   for (const tsdp_net_t* n : {&cfg->base, &cfg->draft}) {
-    if (n->arch < TSDP_ARCH_GAUSS || n->arch > TSDP_ARCH_DIT) return TSDP_ERR_UNSUPPORTED;
+    if (n->arch < TSDP_ARCH_GAUSS || n->arch > TSDP_ARCH_UNET) return TSDP_ERR_UNSUPPORTED;
     if (!net_cfg_ok(*cfg, *n)) return TSDP_ERR_ARG;
   }
   tsdp_ctx* c = new tsdp_ctx();
@@ -986,6 +1130,25 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   INIT_TRY(cudaFuncSetAttribute(self_attn_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
   c->net[TSDP_BASE].cfg = cfg->base;
   c->net[TSDP_DRAFT].cfg = cfg->draft;
+  for (int w = 0; w < 2; ++w) {      // conv-UNet activations: one zero-padded tensor per named stage
+    Net& n = c->net[w];
+    if (n.cfg.arch != TSDP_ARCH_UNET) continue;
+    const size_t nc = (w == TSDP_BASE ? B * K1 : B), ch = n.cfg.d, LV = n.cfg.layers, last = LV - 1;
+    auto pad = [&](void** p, size_t lv, size_t C) { return alloc_bytes(c, c->allocs, p, nc * ((cfg->H >> lv) + 4) * C * esz); };
+    int e = 0;
+    e |= pad(&n.uw.X0, 0, ch); e |= pad(&n.uw.HB, 0, ch);
+    e |= pad(&n.uw.E, last, ch << last); e |= pad(&n.uw.M1, last, ch << last); e |= pad(&n.uw.M2, last, ch << last);
+    for (size_t lv = 0; lv < LV; ++lv) {
+      e |= pad(&n.uw.TMP[lv], lv, ch << lv); e |= pad(&n.uw.D[lv], lv, ch << lv);
+      if (lv < last) {
+        e |= pad(&n.uw.CAT[lv], lv, (ch << (lv + 1)) + (ch << lv)); e |= pad(&n.uw.P[lv], lv + 1, ch << lv);
+        e |= pad(&n.uw.U1[lv], lv, ch << lv); e |= pad(&n.uw.U2[lv], lv, ch << lv);
+      }
+    }
+    e |= dev_alloc(c, c->allocs, &n.uw.Y, nc * (cfg->H + 4) * (ch << last));
+    e |= dev_alloc(c, c->allocs, &n.uw.R, nc * (cfg->H + 4) * (ch << last));
+    if (e) return fail(TSDP_ERR_CUDA);
+  }
   INIT_TRY(cudaDeviceSynchronize());
 #undef INIT_TRY
   *out = c;
@@ -1118,6 +1281,99 @@ int tsdp_load_weights(tsdp_ctx* c, int which, const float* blob, size_t n) {
     float* tt;
     if ((r = sinus_table(net.cfg.temb, &tt))) return r;
     m.temb_table = tt;
+  } else if (net.cfg.arch == TSDP_ARCH_UNET) {
+    const size_t ch = net.cfg.d, A = cfg.A, dt = net.cfg.temb, dobs = (size_t)cfg.obs_tokens * cfg.obs_dim, dc = dt + dobs;
+    if ((r = up_f32(&net.W_in, A * ch))) return r;
+    if ((r = up_f32(&net.b_in, ch))) return r;
+    const float *Wt1 = cur, *bt1 = Wt1 + dt * 4 * dt, *Wt2 = bt1 + 4 * dt, *bt2 = Wt2 + 4 * dt * dt;
+    cur = bt2 + dt;
+    const auto chans = unet_channels((int)ch, net.cfg.layers);
+    size_t F = 0;
+    for (auto& cc : chans) F += 2 * (size_t)cc.second;
+    net.F = (int)F;
+    std::vector<float> wfT_time(F * dt), wfT_obs(F * (dobs ? dobs : 1)), bf_all(F);
+    net.ub.clear();
+    size_t foff = 0;
+    for (auto& cc : chans) {
+      Net::UBlock b{};
+      const size_t ci = cc.first, co = cc.second;
+      b.cin = (int)ci; b.cout = (int)co; b.foff = (int)foff;
+      if ((r = up_wT(&b.W1, cur, 5 * ci, co))) return r;
+      cur += 5 * ci * co;
+      if ((r = up_f32(&b.b1, co))) return r;
+      if ((r = up_f32(&b.g1, co))) return r;
+      if ((r = up_f32(&b.be1, co))) return r;
+      for (size_t i = 0; i < dc; ++i)                       // Wf [dc, 2co] -> rows foff.. of the [F, dt] and [F, dobs] tables
+        for (size_t o = 0; o < 2 * co; ++o) {
+          const float v = cur[i * 2 * co + o];
+          if (i < dt) wfT_time[(foff + o) * dt + i] = v; else wfT_obs[(foff + o) * dobs + (i - dt)] = v;
+        }
+      cur += dc * 2 * co;
+      for (size_t o = 0; o < 2 * co; ++o) bf_all[foff + o] = cur[o];
+      cur += 2 * co;
+      if ((r = up_wT(&b.W2, cur, 5 * co, co))) return r;
+      cur += 5 * co * co;
+      if ((r = up_f32(&b.b2, co))) return r;
+      if ((r = up_f32(&b.g2, co))) return r;
+      if ((r = up_f32(&b.be2, co))) return r;
+      if (ci != co) {
+        if ((r = up_wT(&b.Wr, cur, ci, co))) return r;
+        cur += ci * co;
+        if ((r = up_f32(&b.br, co))) return r;
+      }
+      foff += 2 * co;
+      net.ub.push_back(b);
+    }
+    if ((r = up_wT(&net.Wh, cur, 5 * ch, ch))) return r;
+    cur += 5 * ch * ch;
+    if ((r = up_f32(&net.bh, ch))) return r;
+    if ((r = up_f32(&net.gh, ch))) return r;
+    if ((r = up_f32(&net.beh, ch))) return r;
+    {   // W_out [ch, A] -> fp32 [A, ch]
+      std::vector<float> tmp(A * ch);
+      for (size_t i = 0; i < ch; ++i)
+        for (size_t a = 0; a < A; ++a) tmp[a * ch + i] = cur[i * A + a];
+      cur += ch * A;
+      if (dev_alloc(c, net.allocs, &net.W_outT, A * ch)) return TSDP_ERR_CUDA;
+      CU_TRY(c, cudaMemcpy(net.W_outT, tmp.data(), tmp.size() * sizeof(float), cudaMemcpyHostToDevice));
+    }
+    if ((r = up_f32(&net.b_out, A))) return r;
+    if (dev_alloc(c, net.allocs, &net.film_time, (size_t)T * F)) return TSDP_ERR_CUDA;
+    if (dev_alloc(c, net.allocs, &net.film_obs, c->items_cap * F)) return TSDP_ERR_CUDA;
+    if (dev_alloc(c, net.allocs, &net.obs_m, c->items_cap * (dobs ? dobs : 1))) return TSDP_ERR_CUDA;
+    if (dev_alloc(c, net.allocs, &net.WfT_obs, F * (dobs ? dobs : 1))) return TSDP_ERR_CUDA;
+    CU_TRY(c, cudaMemcpy(net.WfT_obs, wfT_obs.data(), wfT_obs.size() * sizeof(float), cudaMemcpyHostToDevice));
+    if ((r = sinus_table((int)dt, &net.temb_table))) return r;
+    // time vector for every t, then its FiLM contribution: film_time = Mish(tvec) Wf_time + bf
+    std::vector<float> wt1T(4 * dt * dt), wt2T(dt * 4 * dt);
+    for (size_t i = 0; i < dt; ++i)
+      for (size_t o = 0; o < 4 * dt; ++o) wt1T[o * dt + i] = Wt1[i * 4 * dt + o];
+    for (size_t i = 0; i < 4 * dt; ++i)
+      for (size_t o = 0; o < dt; ++o) wt2T[o * 4 * dt + i] = Wt2[i * dt + o];
+    std::vector<void*> tmp_pool;
+    float *d_w1, *d_b1, *d_w2, *d_b2, *d_wf, *d_bf, *d_hid, *d_tv;
+    int st = 0;
+    st |= dev_alloc(c, tmp_pool, &d_w1, 4 * dt * dt); st |= dev_alloc(c, tmp_pool, &d_b1, 4 * dt);
+    st |= dev_alloc(c, tmp_pool, &d_w2, 4 * dt * dt); st |= dev_alloc(c, tmp_pool, &d_b2, dt);
+    st |= dev_alloc(c, tmp_pool, &d_wf, F * dt); st |= dev_alloc(c, tmp_pool, &d_bf, F);
+    st |= dev_alloc(c, tmp_pool, &d_hid, (size_t)T * 4 * dt); st |= dev_alloc(c, tmp_pool, &d_tv, (size_t)T * dt);
+    auto free_tmp = [&]() { for (void* q : tmp_pool) cudaFree(q); };
+    if (st) { free_tmp(); return TSDP_ERR_CUDA; }
+    cudaMemcpy(d_w1, wt1T.data(), wt1T.size() * 4, cudaMemcpyHostToDevice); cudaMemcpy(d_b1, bt1, 4 * dt * 4, cudaMemcpyHostToDevice);
+    cudaMemcpy(d_w2, wt2T.data(), wt2T.size() * 4, cudaMemcpyHostToDevice); cudaMemcpy(d_b2, bt2, dt * 4, cudaMemcpyHostToDevice);
+    cudaMemcpy(d_wf, wfT_time.data(), wfT_time.size() * 4, cudaMemcpyHostToDevice);
+    cudaMemcpy(d_bf, bf_all.data(), F * 4, cudaMemcpyHostToDevice);
+    r = gemm_f32(c, net.temb_table, d_w1, d_b1, T, (int)(4 * dt), (int)dt, EPI_MISH, d_hid, 0);
+    if (!r) r = gemm_f32(c, d_hid, d_w2, d_b2, T, (int)dt, (int)(4 * dt), EPI_F32, d_tv, 0);
+    if (!r) {
+      const long long nel = (long long)T * dt;
+      mish_kernel<<<(unsigned)((nel + 255) / 256), 256>>>(d_tv, d_tv, nel);
+      r = gemm_f32(c, d_tv, d_wf, d_bf, T, (int)F, (int)dt, EPI_F32, net.film_time, 0);
+    }
+    cudaError_t e = cudaDeviceSynchronize();
+    free_tmp();
+    if (r) return r;
+    CU_TRY(c, e);
   } else if (net.cfg.arch == TSDP_ARCH_DIT) {
     const size_t d = net.cfg.d, A = cfg.A, H = cfg.H, Tc = cfg.obs_tokens, L = net.cfg.layers;
     if ((r = up_f32(&net.W_in, A * d))) return r;
@@ -1363,6 +1619,12 @@ static int ensure_items(tsdp_ctx* c, size_t N) {
     if (n.cfg.arch != TSDP_ARCH_XFMR && n.cfg.arch != TSDP_ARCH_DIT) continue;
     dmax = std::max(dmax, (size_t)n.cfg.d);
     if (n.loaded) st |= dev_alloc(c, n.allocs, &n.kv_obs, N * (To ? To : 1) * n.cfg.layers * 2 * n.cfg.d);
+  }
+  for (int w = 0; w < 2; ++w) {
+    Net& n = c->net[w];
+    if (n.cfg.arch != TSDP_ARCH_UNET || !n.loaded) continue;
+    st |= dev_alloc(c, n.allocs, &n.film_obs, N * n.F);
+    st |= dev_alloc(c, n.allocs, &n.obs_m, N * (To * cfg.obs_dim ? To * cfg.obs_dim : 1));
   }
   if (dmax) st |= alloc_bytes(c, c->allocs, &c->memtok, std::max((size_t)cfg.T, N * To) * dmax * (cfg.precision == 0 ? 4 : 2));
   if (st) return TSDP_ERR_CUDA;

@@ -124,3 +124,35 @@ def test_dit_denoiser(precision, tol, shape):
         err = hp.max_rel(out.cpu().numpy(), ref)
         assert err < tol, (which, err)
     smp.close()
+
+
+@pytest.mark.parametrize("precision,tol", [(0, 1e-4), (1, 2e-2)])
+@pytest.mark.parametrize("shape", ["two_levels", "three_levels"])
+def test_unet_denoiser(precision, tol, shape):
+    """1-D conv UNet against the oracle: convolutions as GEMMs over the zero-padded layout (tensor-core
+    path in precision 1), GroupNorm + Mish + FiLM, pooling, repetition, skip concatenation, 1x1 residuals."""
+    rng = np.random.default_rng(4)
+    if shape == "two_levels":
+        wl = dict(H=8, A=3, To=2, Do=12, T=100, precision=precision, gamma=1.0,
+                  base=dict(arch="unet", layers=2, d=128, heads=8, temb=32), draft=dict(arch="unet", layers=1, d=128, heads=4, temb=16))
+    else:
+        wl = dict(H=16, A=10, To=2, Do=24, T=100, precision=precision, gamma=1.0,
+                  base=dict(arch="unet", layers=3, d=128, heads=8, temb=64), draft=dict(arch="xfmr", layers=1, d=128, heads=4))
+    N = 11      # 11 * 20 padded rows: ragged against the 128-row tiles
+    smp, S, base, draft = hp.setup(wl, max_B=N, max_K=1)
+    x = rng.normal(size=(N, wl["H"], wl["A"])).astype(np.float32)
+    tau = rng.integers(0, 100, size=N).astype(np.int32); tau[0], tau[1] = 0, 99
+    obs = inputs.make_obs(5, N, wl["To"], wl["Do"])
+    dx = torch.tensor(x, device="cuda"); dobs = torch.tensor(obs, dtype=torch.float32, device="cuda")
+    for which, net in ((binding.BASE, base), (binding.DRAFT, draft)):
+        out = torch.zeros_like(dx)
+        smp.denoise(which, dx, tau, dobs, N, out)
+        ref = np.stack([net(x[n].astype(np.float64), int(tau[n]), obs[n]) for n in range(N)])
+        err = hp.max_rel(out.cpu().numpy(), ref)
+        assert err < tol, (which, err)
+    # a second call must give the same answer: the padding rows of every buffer are still zero
+    out2 = torch.zeros_like(dx)
+    smp.denoise(binding.BASE, dx, tau, dobs, N, out2)
+    ref = np.stack([base(x[n].astype(np.float64), int(tau[n]), obs[n]) for n in range(N)])
+    assert hp.max_rel(out2.cpu().numpy(), ref) < tol
+    smp.close()

@@ -164,6 +164,14 @@ def test_chunk_dit_fp32():
     assert n_match >= B - 1
 
 
+@pytest.mark.parametrize("precision,tol_eps,tol_x", [(0, 1e-4, 2e-5), (1, 2e-2, 3e-3)])
+def test_round_unet_base_transformer_drafter(precision, tol_eps, tol_x):
+    """Robomimic-shaped pairing: conv UNet base verified against a transformer drafter's drafts."""
+    wl = dict(H=16, A=10, To=2, Do=24, T=100, precision=precision, gamma=0.05,
+              base=dict(arch="unet", layers=2, d=128, heads=8, temb=32), draft=dict(arch="xfmr", layers=1, d=128, heads=4))
+    _round_parity(wl, 4, 5, hp.accept_t(), 51, tol_eps, tol_x, [99, 60, 3, 0])
+
+
 def test_chunk_with_round_schedule_fp32():
     wl = hp.small_xfmr_workload(0, d=128, heads=4, layers=1, dd=128, dlayers=1, H=16, A=7, To=2, Do=64, gamma=0.03)
     Ks, Ss = inputs.markov_schedule(0, 40)

@@ -419,7 +419,7 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="serving_xfmr", choices=["serving_xfmr", "pusht_xfmr", "toy_mlp", "vla_dit"])
+    ap.add_argument("--workload", default="serving_xfmr", choices=["serving_xfmr", "pusht_xfmr", "toy_mlp", "vla_dit", "robomimic_unet"])
     ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
     ap.add_argument("--no-latency", dest="latency", action="store_false")

@@ -79,9 +79,11 @@ typedef struct {
   int drafter;             /* how the K draft steps run.  0: chosen from the batch size; 1: layer
                               by layer (batched tensor-core kernels, one drafter forward per step);
                               2: one persistent thread-block-cluster kernel per round with the
-                              drafter's weights resident in shared memory (transformer drafter,
-                              precision 1, d = 128 or 256, H <= 16, obs_tokens <= 3, weights of a
-                              1/8 slice fitting one SM; otherwise tsdp_init returns UNSUPPORTED)  */
+                              drafter's weights sliced over the 8 CTAs of the cluster: resident
+                              in shared memory when a 1/8 slice fits beside the activations, read
+                              through the L2 otherwise (transformer drafter, precision 1, d = 128
+                              or 256, <= 4 blocks, H <= 16, obs_tokens <= 3; otherwise tsdp_init
+                              returns UNSUPPORTED)                                               */
 } tsdp_config_t;
 
 /* Speculative parameters of a round -- the scheduler's action space (Sec. 3.3).

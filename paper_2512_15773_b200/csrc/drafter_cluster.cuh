@@ -1,9 +1,10 @@
 // Persistent drafter: the whole K-step draft rollout of one environment (Sec. 3.2 "Draft Generation
 // Procedure", Eq. (3)) in ONE kernel launch, for small batches where the rollout is latency-bound.
 //
-// One thread-block cluster of DC_CS CTAs serves one environment at a time.  Every CTA keeps, for the
-// whole launch, its 1/DC_CS slice (a block of output columns) of every weight matrix of the drafter
-// in shared memory, and a full replica of the activations of the 16-token sequence.  A linear layer
+// One thread-block cluster of DC_CS CTAs serves one environment at a time.  Every CTA owns a 1/DC_CS
+// slice (a block of output columns) of every weight matrix of the drafter -- kept in shared memory
+// for the whole launch when it fits beside the activations, otherwise read in place through the L2 --
+// and a full replica of the activations of the 16-token sequence.  A linear layer
 // is computed as Y[:, slice] = X W_slice^T on mma.sync m16n8k16 (the sequence is one 16-row tile),
 // and each CTA writes its slice of Y into the replicas of all CTAs through distributed shared
 // memory; one hardware cluster barrier separates dependent stages (6 per block).  LayerNorm, the two
@@ -44,6 +45,7 @@ struct DcParams {
   float* muhat; long long ms_b;                              // drafter means [B, Kmax, D]
   const int* t;
   const uint64_t* seed;
+  int resident;                                              // 1: weight slices live in shared memory for the whole launch
   const EnvParams* envp;                                     // per-request draft cap, or null
   const int* item;                                           // slot -> request it serves, or null
   int B, K;
@@ -55,12 +57,12 @@ struct DcSmem {
   int w_layer;      // bytes of one layer's weight slices
   int off_h, off_a, off_qkv, off_q2, off_f, off_red, off_kv, off_x, off_posb, off_win, off_par, total;
 };
-__host__ __device__ inline DcSmem dc_smem_plan(int d, int layers, int A) {
+__host__ __device__ inline DcSmem dc_smem_plan(int d, int layers, int A, bool resident) {
   DcSmem p;
   const int pw = d + 8, pw4 = 4 * d + 8;
   const int rows_d = (3 * d + d + d + d + 4 * d) / DC_CS;    // output rows of the K = d matrices in a slice
   p.w_layer = (rows_d * pw + (d / DC_CS) * pw4) * 2;
-  int o = layers * p.w_layer;
+  int o = resident ? layers * p.w_layer : 0;     // not resident: weight slices are read from L2 where they are used
   auto take = [&](int bytes) { int r = o; o += (bytes + 15) & ~15; return r; };
   p.off_h = take(DC_ROWS * d * 4);
   p.off_a = take(DC_ROWS * (d + 8) * 2);
@@ -68,7 +70,7 @@ __host__ __device__ inline DcSmem dc_smem_plan(int d, int layers, int A) {
   p.off_q2 = take(DC_ROWS * (d + 8) * 2);
   p.off_f = take(DC_ROWS * (4 * d + 8) * 2);
   p.off_red = take(DC_WARPS * DC_ROWS * 8 * 4);              // one 16 x 8 fp32 tile per warp
-  p.off_kv = take(layers * DC_MAX_NK * 2 * d * 4);           // keys / values of the memory tokens, every block
+  p.off_kv = take((resident ? layers : 1) * DC_MAX_NK * 2 * d * 4);   // keys / values of the memory tokens: every block, or the current one
   p.off_x = take(DC_ROWS * 16 * 4 * 2);                      // latent and eps, D <= 256
   p.off_posb = take(DC_ROWS * d * 4);
   p.off_win = take(A * d * 4);
@@ -81,12 +83,11 @@ __host__ __device__ inline DcSmem dc_smem_plan(int d, int layers, int A) {
 // fewer tiles than warps the K range is split and the parts are summed through shared memory.
 // `emit(row, col, v)` receives 8 adjacent columns (col a multiple of 8) of the finished slice.
 template <int KD, typename Emit>
-__device__ __forceinline__ void dc_linear(const __nv_bfloat16* X, int px, const __nv_bfloat16* W, int n_slice,
+__device__ __forceinline__ void dc_linear(const __nv_bfloat16* X, int px, const __nv_bfloat16* W, int PW, int n_slice,
                                           float* red, Emit emit) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, tg = lane & 3;
-  constexpr int PW = KD + 8;
-  const int n_tiles = n_slice >> 3;
+  const int n_tiles = n_slice >> 3;      // PW: row pitch of W (KD + 8 in shared memory, KD in global memory)
   int ksplit = 1;
   while (n_tiles * ksplit * 2 <= DC_WARPS && (KD / 16) % (ksplit * 2) == 0) ksplit *= 2;
   const int units = n_tiles * ksplit;
@@ -99,7 +100,7 @@ __device__ __forceinline__ void dc_linear(const __nv_bfloat16* X, int px, const 
       const __nv_bfloat16* wrow = W + (size_t)(nt * 8 + g) * PW;
       const __nv_bfloat16* x0 = X + (size_t)g * px;
       const __nv_bfloat16* x1 = X + (size_t)(g + 8) * px;
-#pragma unroll 4
+#pragma unroll 8
       for (int ks = ks0; ks < ks1; ++ks) {
         const int k = ks * 16 + 2 * tg;
         uint32_t a[4];
@@ -315,7 +316,8 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
   const int cid = blockIdx.x / DC_CS, ncl = gridDim.x / DC_CS;
   constexpr int d = D_MODEL;
   constexpr int PA = d + 8, PQKV = 3 * d + 8, PF = 4 * d + 8;
-  const DcSmem pl = dc_smem_plan(d, P.layers, P.A);
+  const bool resident = P.resident != 0;
+  const DcSmem pl = dc_smem_plan(d, P.layers, P.A, resident);
   float* h = reinterpret_cast<float*>(dc_smem + pl.off_h);
   __nv_bfloat16* a = reinterpret_cast<__nv_bfloat16*>(dc_smem + pl.off_a);
   __nv_bfloat16* qkv = reinterpret_cast<__nv_bfloat16*>(dc_smem + pl.off_qkv);
@@ -333,17 +335,24 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
 
   // ---- once per launch: this CTA's weight slices, embedding tables, zeroed activations
   constexpr int NS_D = d / DC_CS, NS_3D = 3 * d / DC_CS, NS_4D = 4 * d / DC_CS;   // slice widths
-  auto w_ptr = [&](int l, int which) -> __nv_bfloat16* {     // 0 qkv, 1 o, 2 q2, 3 o2, 4 w1, 5 w2
+  auto w_ptr = [&](int l, int which) -> const __nv_bfloat16* {     // 0 qkv, 1 o, 2 q2, 3 o2, 4 w1, 5 w2
+    if (!resident) {      // this CTA's block of output rows, in place in global memory (served by the L2)
+      const DcLayer& G = P.L[l];
+      const __nv_bfloat16* base[6] = {G.Wqkv, G.Wo, G.Wq2, G.Wo2, G.W1, G.W2};
+      const int rows[6] = {NS_3D, NS_D, NS_D, NS_D, NS_4D, NS_D};
+      return base[which] + (size_t)rank * rows[which] * (which == 5 ? 4 * d : d);
+    }
     const int rows_before[6] = {0, NS_3D, NS_3D + NS_D, NS_3D + 2 * NS_D, NS_3D + 3 * NS_D, NS_3D + 3 * NS_D + NS_4D};
-    return reinterpret_cast<__nv_bfloat16*>(dc_smem + (size_t)l * pl.w_layer) + (size_t)rows_before[which] * PA;
+    return reinterpret_cast<const __nv_bfloat16*>(dc_smem + (size_t)l * pl.w_layer) + (size_t)rows_before[which] * PA;
   };
-  for (int l = 0; l < L; ++l) {
-    dc_load_slice<d>(w_ptr(l, 0), P.L[l].Wqkv, NS_3D, rank);
-    dc_load_slice<d>(w_ptr(l, 1), P.L[l].Wo, NS_D, rank);
-    dc_load_slice<d>(w_ptr(l, 2), P.L[l].Wq2, NS_D, rank);
-    dc_load_slice<d>(w_ptr(l, 3), P.L[l].Wo2, NS_D, rank);
-    dc_load_slice<d>(w_ptr(l, 4), P.L[l].W1, NS_4D, rank);
-    dc_load_slice<4 * d>(w_ptr(l, 5), P.L[l].W2, NS_D, rank);
+  const int PWD = resident ? PA : d, PW4 = resident ? PF : 4 * d;      // weight row pitches for K = d and K = 4d
+  for (int l = 0; l < L && resident; ++l) {
+    dc_load_slice<d>(const_cast<__nv_bfloat16*>(w_ptr(l, 0)), P.L[l].Wqkv, NS_3D, rank);
+    dc_load_slice<d>(const_cast<__nv_bfloat16*>(w_ptr(l, 1)), P.L[l].Wo, NS_D, rank);
+    dc_load_slice<d>(const_cast<__nv_bfloat16*>(w_ptr(l, 2)), P.L[l].Wq2, NS_D, rank);
+    dc_load_slice<d>(const_cast<__nv_bfloat16*>(w_ptr(l, 3)), P.L[l].Wo2, NS_D, rank);
+    dc_load_slice<d>(const_cast<__nv_bfloat16*>(w_ptr(l, 4)), P.L[l].W1, NS_4D, rank);
+    dc_load_slice<4 * d>(const_cast<__nv_bfloat16*>(w_ptr(l, 5)), P.L[l].W2, NS_D, rank);
   }
   for (int i = threadIdx.x; i < DC_ROWS * d; i += DC_THREADS) {
     const int row = i / d, col = i % d;
@@ -391,7 +400,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
     float* mh_b = P.muhat + slot * P.ms_b;
     for (int i = threadIdx.x; i < D; i += DC_THREADS) sx[i] = xt_b[i];
     // keys / values of this environment's observation tokens, every block (slot 0 is the time token)
-    for (int i = threadIdx.x; i < L * P.To * 2 * d; i += DC_THREADS) {
+    for (int i = threadIdx.x; i < (resident ? L : 0) * P.To * 2 * d; i += DC_THREADS) {
       const int l = i / (P.To * 2 * d), rem = i % (P.To * 2 * d);
       const int kx = 1 + rem / (2 * d), c = rem % (2 * d);
       skv[((size_t)l * DC_MAX_NK + kx) * 2 * d + c] = __ldg(P.kv_obs + ((size_t)env * P.To + (kx - 1)) * ldkv + (size_t)l * 2 * d + c);
@@ -408,7 +417,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         continue;
       }
       // keys / values of the time token of tau, every block
-      for (int i = threadIdx.x; i < L * 2 * d; i += DC_THREADS) {
+      for (int i = threadIdx.x; i < (resident ? L : 0) * 2 * d; i += DC_THREADS) {
         const int l = i / (2 * d), c = i % (2 * d);
         skv[(size_t)l * DC_MAX_NK * 2 * d + c] = __ldg(P.kv_time + (size_t)tau * ldkv + (size_t)l * 2 * d + c);
       }
@@ -429,7 +438,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         // ---- causal self-attention
         dc_layernorm<d>(h, W.ln1_g, W.ln1_b, a, PA);
         __syncthreads();
-        dc_linear<d>(a, PA, w_ptr(l, 0), NS_3D, red, [&](int row, int col, float* v) {
+        dc_linear<d>(a, PA, w_ptr(l, 0), PWD, NS_3D, red, [&](int row, int col, float* v) {
           const int cg_ = rank * NS_3D + col;
           const float4 b0 = *reinterpret_cast<const float4*>(W.bqkv + cg_), b1 = *(reinterpret_cast<const float4*>(W.bqkv + cg_) + 1);
           v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
@@ -445,7 +454,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
           default: dc_attention<d, true>(qkv, PQKV, qkv, PQKV, nullptr, 0, a, PA, P.heads, H); break;
         }
         __syncthreads();
-        dc_linear<d>(a, PA, w_ptr(l, 1), NS_D, red, [&](int row, int col, float* v) {
+        dc_linear<d>(a, PA, w_ptr(l, 1), PWD, NS_D, red, [&](int row, int col, float* v) {
           const int cg_ = rank * NS_D + col;
           const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
           const float4 h0 = hp[0], h1 = hp[1];
@@ -458,11 +467,18 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
             dst[0] = o0; dst[1] = o1;
           }
         });
+        if (!resident) {   // keys / values of the memory tokens for this block only: time token of tau, then the obs tokens
+          for (int i = threadIdx.x; i < NK * 2 * d; i += DC_THREADS) {
+            const int kx = i / (2 * d), c = i % (2 * d);
+            const float* src = kx == 0 ? P.kv_time + (size_t)tau * ldkv : P.kv_obs + ((size_t)env * P.To + (kx - 1)) * ldkv;
+            skv[i] = __ldg(src + (size_t)l * 2 * d + c);
+          }
+        }
         cluster.sync();
         // ---- cross-attention to [time token | obs tokens]
         dc_layernorm<d>(h, W.ln2_g, W.ln2_b, a, PA);
         __syncthreads();
-        dc_linear<d>(a, PA, w_ptr(l, 2), NS_D, red, [&](int row, int col, float* v) {
+        dc_linear<d>(a, PA, w_ptr(l, 2), PWD, NS_D, red, [&](int row, int col, float* v) {
           const int cg_ = rank * NS_D + col;
           const float4 b0 = *reinterpret_cast<const float4*>(W.bq2 + cg_), b1 = *(reinterpret_cast<const float4*>(W.bq2 + cg_) + 1);
           v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
@@ -471,9 +487,9 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
           for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(rq2[r] + row * PA + cg_) = pk;
         });
         cluster.sync();
-        dc_attention<d, false>(q2, PA, nullptr, 0, skv + (size_t)l * DC_MAX_NK * 2 * d, NK, a, PA, P.heads, H);
+        dc_attention<d, false>(q2, PA, nullptr, 0, skv + (size_t)(resident ? l : 0) * DC_MAX_NK * 2 * d, NK, a, PA, P.heads, H);
         __syncthreads();
-        dc_linear<d>(a, PA, w_ptr(l, 3), NS_D, red, [&](int row, int col, float* v) {
+        dc_linear<d>(a, PA, w_ptr(l, 3), PWD, NS_D, red, [&](int row, int col, float* v) {
           const int cg_ = rank * NS_D + col;
           const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
           const float4 h0 = hp[0], h1 = hp[1];
@@ -490,7 +506,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         // ---- MLP
         dc_layernorm<d>(h, W.ln3_g, W.ln3_b, a, PA);
         __syncthreads();
-        dc_linear<d>(a, PA, w_ptr(l, 4), NS_4D, red, [&](int row, int col, float* v) {
+        dc_linear<d>(a, PA, w_ptr(l, 4), PWD, NS_4D, red, [&](int row, int col, float* v) {
           const int cg_ = rank * NS_4D + col;
           const float4 b0 = *reinterpret_cast<const float4*>(W.b1 + cg_), b1 = *(reinterpret_cast<const float4*>(W.b1 + cg_) + 1);
           v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
@@ -502,7 +518,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
           for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(rf[r] + row * PF + cg_) = pk;
         });
         cluster.sync();
-        dc_linear<4 * d>(f, PF, w_ptr(l, 5), NS_D, red, [&](int row, int col, float* v) {
+        dc_linear<4 * d>(f, PF, w_ptr(l, 5), PW4, NS_D, red, [&](int row, int col, float* v) {
           const int cg_ = rank * NS_D + col;
           const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
           const float4 h0 = hp[0], h1 = hp[1];

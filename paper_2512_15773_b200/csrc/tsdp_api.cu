@@ -112,6 +112,7 @@ struct tsdp_ctx {
   bool pdl = true;                            // programmatic dependent launch between the kernels of a round
   bool dc_ok = false;
   int dc_smem = 0, dc_max_clusters = 0;
+  bool dc_resident = false;
   uint64_t rounds = 0, launches = 0;
   int launches_per_round_tmp = 0;
   // optional per-kernel-family timing with CUDA events (plain launches, no graph)
@@ -802,20 +803,26 @@ int forward(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStream_t s) 
 
 // ------------------------------------------------------------------------------------------ drafter
 // Whether the persistent cluster kernel can run this context's drafter at all (shapes, shared memory).
-bool cluster_drafter_fits(const tsdp_config_t& cfg, int* smem_bytes) {
+bool cluster_drafter_fits(const tsdp_config_t& cfg, int* smem_bytes, bool* resident) {
   const tsdp_net_t& n = cfg.draft;
   if (cfg.precision != 1 || n.arch != TSDP_ARCH_XFMR || (n.d != 128 && n.d != 256) || n.layers > DC_MAX_LAYERS ||
       cfg.H > DC_ROWS || 1 + cfg.obs_tokens > DC_MAX_NK || cfg.H * cfg.A > 256 || (n.d / n.heads) % 4 != 0)
     return false;
-  const DcSmem pl = dc_smem_plan(n.d, n.layers, cfg.A);
-  *smem_bytes = pl.total;
-  return pl.total <= 227 * 1024;
+  // weight slices resident in shared memory if they fit beside the activations, otherwise read through the L2
+  for (int res = 1; res >= 0; --res) {
+    const DcSmem pl = dc_smem_plan(n.d, n.layers, cfg.A, res != 0);
+    if (pl.total <= 227 * 1024) { *smem_bytes = pl.total; *resident = res != 0; return true; }
+  }
+  return false;
 }
 
 bool use_cluster_drafter(const tsdp_ctx* c, int B) {
   if (!c->dc_ok || c->cfg.drafter == 1) return false;
   if (c->cfg.drafter == 2) return true;
-  return B <= 4 * c->dc_max_clusters;     // beyond a few waves of clusters the batched tensor-core path wins
+  // Beyond a few waves of clusters the batched tensor-core path wins: measured about 29 us per draft step and wave
+  // with resident weights (PushT drafter) and 70-130 us with L2-streamed ones, against 100-175 us per step for the
+  // layer-by-layer path whatever the batch.
+  return B <= (c->dc_resident ? 3 : 1) * c->dc_max_clusters;
 }
 
 int launch_cluster_drafter(tsdp_ctx* c, int B, int K, cudaStream_t s) {
@@ -839,6 +846,7 @@ int launch_cluster_drafter(tsdp_ctx* c, int B, int K, cudaStream_t s) {
   P.t = c->t; P.seed = c->seed; P.B = B; P.K = K;
   P.envp = c->sched_on ? c->envp : nullptr;
   P.item = c->item;
+  P.resident = c->dc_resident ? 1 : 0;
   const int ncl = B < c->dc_max_clusters ? B : c->dc_max_clusters;
   prof_begin(c, s, 7, 0.0);
   if (n.cfg.d == 128) TSDP_LAUNCH(c, (drafter_cluster_kernel<128>), ncl * DC_CS, DC_THREADS, c->dc_smem, s, P);
@@ -1105,7 +1113,7 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
     INIT_TRY(set_smem_attr_all<64>());
     INIT_TRY(set_smem_attr_all<32>());
   }
-  if (cluster_drafter_fits(*cfg, &c->dc_smem)) {
+  if (cluster_drafter_fits(*cfg, &c->dc_smem, &c->dc_resident)) {
     const void* fn = cfg->draft.d == 128 ? (const void*)drafter_cluster_kernel<128> : (const void*)drafter_cluster_kernel<256>;
     INIT_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, c->dc_smem));
     cudaLaunchConfig_t lc{};

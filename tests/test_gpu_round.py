@@ -72,9 +72,16 @@ def test_round_transformer_bf16_both_drafters(drafter):
                   drafter=drafter)
 
 
-def test_cluster_drafter_matches_layered_drafter():
-    wl = dict(inputs.WORKLOADS["pusht_xfmr"], precision=1)
-    B, K, D = 3, 8, 32
+@pytest.mark.parametrize("case", ["resident", "streamed"])
+def test_cluster_drafter_matches_layered_drafter(case):
+    """resident: the PushT drafter, whose weight slices live in shared memory; streamed: a 4-block d = 256
+    drafter (Robomimic-shaped), too large for that, whose slices are read through the L2."""
+    if case == "resident":
+        wl = dict(inputs.WORKLOADS["pusht_xfmr"], precision=1)
+    else:
+        wl = dict(H=16, A=10, To=2, Do=24, T=100, precision=1, gamma=0.05,
+                  base=dict(arch="xfmr", layers=1, d=128, heads=4), draft=dict(arch="xfmr", layers=4, d=256, heads=4))
+    B, K, D = 3, 8, wl["H"] * wl["A"]
     outs = []
     for drafter in (1, 2):
         smp, *_ = hp.setup(wl, max_B=B, max_K=K, drafter=drafter)

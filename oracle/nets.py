@@ -4,7 +4,7 @@ conv UNet.
 The paper states only the block counts ("DP consists of 8 Transformer blocks while the drafter
 contains only one", Sec. 4) and that the drafter has the same input-output interface and shares
 the encoder and scheduler (Sec. 3.2 "Draft Model Training").  Everything below that is more
-specific than that is this build's own architecture definition; parity with the paper's trained
+specific than that is this library's own architecture definition; parity with the paper's trained
 networks is UNPINNED (no weights or layer layout are published).  The pins that exist are
 structural: causality of self-attention (bidirectionality for the adaLN transformer, whose
 blocks reduce to the identity with zero gates), independence of candidates, zero-head => zero output,

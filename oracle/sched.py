@@ -7,7 +7,7 @@ parameters: the sigma scale, the acceptance threshold, and a draft-step count fo
 denoising stages (early high-noise, middle, late low-noise).  It is trained with PPO; only the
 deterministic (mean) action is needed at inference.
 
-What it does not fix, and this build defines: widths (64 / 64 / 16 -> 64 -> 5), tanh activations, the
+What it does not fix, and this library defines: widths (64 / 64 / 16 -> 64 -> 5), tanh activations, the
 squashing of the 5 raw outputs into parameter ranges, and the stage boundaries t >= 4T/5 (early),
 t < T/5 (late).  PARITY UNPINNED against the paper (no architecture, weights or ranges are published);
 pinned only by structure: zero weights give the mid-range parameters, the three streams enter through

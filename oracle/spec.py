@@ -10,7 +10,7 @@ Follows the paper in its own order and notation:
   Sec. 3.2 last paragraph        chronological scan, commit the accepted prefix, reflect the first
                                  rejected draft.
 
-Readings taken where the paper is silent or inconsistent (each is listed in the design notes):
+Readings taken where the paper is silent or inconsistent:
   * timestep handed to a network = timestep of its input latent; draft k consumes draft k-1;
   * a round starts from the current latent x at timestep t; the base model is evaluated on the
     K_eff+1 latents x~_0..x~_{K_eff}; the last evaluation is a "bonus" base step, taken only when

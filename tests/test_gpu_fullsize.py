@@ -1,0 +1,78 @@
+"""Parity at the sizes and in the launch configuration the benchmark times, on sampled outputs.
+
+The full serving batch (256 environments x 11 candidates x 16 tokens = 45 056 token rows through the
+persistent 148-CTA GEMM, the tensor-core attentions and the fused acceptance kernel) is run once; a few
+environments are then recomputed one by one by the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ddpm, nets, spec
+from paper_2512_15773_b200 import binding, inputs
+from tests import helpers as hp
+
+pytestmark = pytest.mark.gpu
+BAND = 1e-3
+
+
+def test_serving_round_at_bench_size_sampled_environments():
+    wl = dict(inputs.WORKLOADS["serving_xfmr"])
+    B, K, seed = wl["B"], wl["K"], 7
+    smp, S, base, draft = hp.setup(wl, max_B=B, max_K=K, drafter=0)
+    D = wl["H"] * wl["A"]; shape = (wl["H"], wl["A"])
+    obs = inputs.make_obs(100, B, wl["To"], wl["Do"])
+    noise = spec.PhiloxNoise(seed)
+    rng = np.random.default_rng(0)
+    t0s = rng.integers(0, 100, size=B).astype(np.int32)
+    t0s[:4] = [99, 50, 3, 0]
+    x0 = rng.normal(size=(B, D)).astype(np.float32)
+    dx = torch.tensor(x0, device="cuda"); dobs = torch.tensor(obs, dtype=torch.float32, device="cuda")
+    h_t = t0s.copy()
+    d_xt = torch.zeros(B, K + 1, D, device="cuda"); d_mh = torch.zeros(B, K, D, device="cuda")
+    d_eps = torch.zeros(B, K + 1, D, device="cuda"); d_la = torch.zeros(B, K, device="cuda")
+    h_j = np.zeros(B, dtype=np.int32)
+    acc = hp.accept_t(sigma_scale=1.5)
+    smp.round(dobs, B, K, acc, seed, dx, h_t, d_xt, d_mh, d_eps, d_la, h_j)
+    xt, mh, eps = d_xt.cpu().numpy(), d_mh.cpu().numpy(), d_eps.cpu().numpy()
+    x_new = dx.cpu().numpy()
+    checked = 0
+    for b in (0, 1, 2, 3, 100, 255):
+        xo, to, d = spec.spec_round(S, base, draft, noise, b, obs[b], x0[b].astype(np.float64).reshape(shape), int(t0s[b]), K,
+                                    hp.oracle_accept(acc))
+        Ke = d["K_eff"]
+        for k in range(d["n_base"]):
+            assert hp.max_rel(eps[b, k], d["eps"][k].reshape(-1)) < 2e-2, (b, k)
+        near_tie = False
+        for k in range(1, Ke + 1):
+            assert np.max(np.abs(mh[b, k - 1] - d["mu_hat"][k].reshape(-1))) < 3e-3
+            lu = np.log(noise.u(b, t0s[b] - k + 1))
+            near_tie |= abs(d["log_alpha"][k - 1] - lu) < BAND + 0.02 * abs(d["log_alpha"][k - 1])
+        if not near_tie:
+            assert h_j[b] == d["jstar"] and h_t[b] == to, (b, h_j[b], d["jstar"])
+            assert np.max(np.abs(x_new[b] - xo.reshape(-1))) < 1e-2
+            checked += 1
+    assert checked >= 3
+    smp.close()
+
+
+def test_vla_shaped_dit_forward_at_full_width_sampled_candidates():
+    """Full width and sequence of the VLA-scale expert (d = 1024, 16 heads, 50 tokens, 256 context tokens,
+    GEMMs up to 4096 x 4096), two blocks deep so that the oracle stays affordable."""
+    wl = dict(inputs.WORKLOADS["vla_dit"])
+    wl["base"] = dict(wl["base"], layers=2); wl["draft"] = dict(wl["draft"], layers=1)
+    wl["gamma"] = 1.0
+    N = 40                                   # 2000 token rows: 16 row tiles, ragged
+    smp, S, base, draft = hp.setup(wl, max_B=N, max_K=1)
+    rng = np.random.default_rng(1)
+    x = rng.normal(size=(N, wl["H"], wl["A"])).astype(np.float32)
+    tau = rng.integers(0, 100, size=N).astype(np.int32)
+    obs = inputs.make_obs(5, N, wl["To"], wl["Do"])
+    dx = torch.tensor(x, device="cuda"); dobs = torch.tensor(obs, dtype=torch.float32, device="cuda")
+    for which, net in ((binding.BASE, base), (binding.DRAFT, draft)):
+        out = torch.zeros_like(dx)
+        smp.denoise(which, dx, tau, dobs, N, out)
+        got = out.cpu().numpy()
+        for n in (0, 17, 39):
+            ref = net(x[n].astype(np.float64), int(tau[n]), obs[n])
+            assert hp.max_rel(got[n], ref) < 2e-2, (which, n)
+    smp.close()

@@ -84,6 +84,11 @@ typedef struct {
                               through the L2 otherwise (transformer drafter, precision 1, d = 128
                               or 256, <= 4 blocks, H <= 16, obs_tokens <= 3; otherwise tsdp_init
                               returns UNSUPPORTED)                                               */
+  int verifier;            /* how the base model's verification forward runs.  0: chosen from the
+                              number of candidates; 1: batched tensor-core kernels, layer by layer;
+                              2: the cluster kernel above, one cluster per candidate, in one launch
+                              (same shape limits, <= 8 blocks; meant for batch 1, where the
+                              layer-by-layer forward is bound by the latency of ~90 small launches) */
 } tsdp_config_t;
 
 /* Speculative parameters of a round -- the scheduler's action space (Sec. 3.3).
@@ -230,10 +235,10 @@ uint64_t tsdp_kernel_launches(const tsdp_ctx* ctx);
  * stream.  Families: 0 GEMMs of the base model (tcgen05 or check-mode), 1 LayerNorm, 2 attention,
  * 3 embed/head/memory tokens, 4 draft-step kernel, 5 MLP / Gaussian denoiser, 6 GEMMs
  * of the drafter, 7 the persistent cluster drafter, 8 the fused
- * acceptance / commit kernel.  tsdp_profile(ctx, 0|1)
+ * acceptance / commit kernel, 9 the cluster kernel as verifier.  tsdp_profile(ctx, 0|1)
  * clears the record.  tsdp_profile_read fills three arrays of TSDP_PROF_FAMILIES entries: summed
  * milliseconds, summed algorithmic flops (2*M*N*K per GEMM launch, 0 elsewhere) and launch counts. */
-enum { TSDP_PROF_FAMILIES = 9 };
+enum { TSDP_PROF_FAMILIES = 10 };
 int tsdp_profile(tsdp_ctx* ctx, int enable);
 int tsdp_profile_read(tsdp_ctx* ctx, double* ms, double* flop, uint64_t* launches);
 

@@ -17,7 +17,7 @@ EXPORTS = ["tsdp_init", "tsdp_destroy", "tsdp_strerror", "tsdp_last_error", "tsd
            "tsdp_round", "tsdp_denoise", "tsdp_gemm", "tsdp_gemm_timed", "tsdp_stats", "tsdp_reset_stats",
            "tsdp_kernel_launches", "tsdp_profile", "tsdp_profile_read", "tsdp_verify_commit_static", "tsdp_set_scheduler", "tsdp_set_progress",
            "tsdp_sched_eval", "tsdp_serve"]
-PROF_FAMILIES = ["gemm", "layernorm", "attention", "embed_head", "round", "small_net", "gemm_draft", "drafter_cluster", "accept"]
+PROF_FAMILIES = ["gemm", "layernorm", "attention", "embed_head", "round", "small_net", "gemm_draft", "drafter_cluster", "accept", "verifier_cluster"]
 
 
 class NetT(C.Structure):
@@ -28,7 +28,7 @@ class ConfigT(C.Structure):
     _fields_ = [("base", NetT), ("draft", NetT), ("H", C.c_int), ("A", C.c_int), ("obs_tokens", C.c_int),
                 ("obs_dim", C.c_int), ("T", C.c_int), ("beta0", C.c_float), ("beta1", C.c_float),
                 ("clip", C.c_float), ("max_B", C.c_int), ("max_K", C.c_int), ("precision", C.c_int),
-                ("device", C.c_int), ("draft_nfe", C.c_float), ("use_graph", C.c_int), ("drafter", C.c_int)]
+                ("device", C.c_int), ("draft_nfe", C.c_float), ("use_graph", C.c_int), ("drafter", C.c_int), ("verifier", C.c_int)]
 
 
 class AcceptT(C.Structure):
@@ -95,12 +95,12 @@ def load_library():
 
 
 def make_config(H, A, To, Do, base, draft, T=100, beta0=1e-4, beta1=0.02, clip=0.0, max_B=1, max_K=8,
-                precision=1, device=0, draft_nfe=0.0, use_graph=1, drafter=0):
+                precision=1, device=0, draft_nfe=0.0, use_graph=1, drafter=0, verifier=0):
     def net(n):
         return NetT(ARCH[n["arch"]], n.get("layers", 0), n.get("d", n.get("width", 0)), n.get("heads", 0),
                     n.get("temb", 32))
     return ConfigT(net(base), net(draft), H, A, To, Do, T, beta0, beta1, clip, max_B, max_K, precision, device,
-                   draft_nfe, use_graph, drafter)
+                   draft_nfe, use_graph, drafter, verifier)
 
 
 def pack_weights(p):

@@ -70,11 +70,16 @@ struct DdpmTables {
   float clip;               // clamp x0_hat to +-clip when > 0
 };
 
+// The operations are spelled out (fused multiply-adds and roundings fixed) so that every kernel that takes a
+// reverse step -- draft step, acceptance kernel, cluster kernel -- rounds identically: with drafter == base the
+// speculative chunk then equals vanilla DDPM bit for bit.
 __device__ __forceinline__ float posterior_mean(const DdpmTables& S, float x, float eps, int tau) {
-  float x0 = (x - S.sqrt_1mab[tau] * eps) / S.sqrt_ab[tau];
+  float x0 = __fdiv_rn(__fmaf_rn(-S.sqrt_1mab[tau], eps, x), S.sqrt_ab[tau]);
   if (S.clip > 0.f) x0 = fminf(fmaxf(x0, -S.clip), S.clip);
-  return S.c_x0[tau] * x0 + S.c_xt[tau] * x;
+  return __fmaf_rn(S.c_x0[tau], x0, __fmul_rn(S.c_xt[tau], x));
 }
+// x_{t-1} = mu + sigma xi
+__device__ __forceinline__ float ddpm_sample(float mu, float sigma, float xi) { return __fmaf_rn(sigma, xi, mu); }
 
 // Programmatic dependent launch: a kernel signals early that its successor in the stream may be
 // scheduled, and waits (after whatever set-up touches no shared data) until every kernel it depends on

@@ -25,7 +25,7 @@ constexpr int DC_CS = 8;          // CTAs per cluster (the portable maximum)
 constexpr int DC_THREADS = 256;
 constexpr int DC_WARPS = DC_THREADS / 32;
 constexpr int DC_ROWS = 16;       // one m16 tile: H <= 16
-constexpr int DC_MAX_LAYERS = 4;
+constexpr int DC_MAX_LAYERS = 8;
 constexpr int DC_MAX_NK = 4;      // memory tokens: time token + at most 3 observation tokens
 
 struct DcLayer {
@@ -46,6 +46,10 @@ struct DcParams {
   const int* t;
   const uint64_t* seed;
   int resident;                                              // 1: weight slices live in shared memory for the whole launch
+  // mode 0: draft rollout (K steps per slot, writes xt / muhat).  mode 1: verification -- one forward per
+  // (slot, candidate c < C) at timestep t[slot] - c, reading xt[slot, c] and writing eps[slot, c].
+  int mode, C;
+  float* eps; long long es_b;
   const EnvParams* envp;                                     // per-request draft cap, or null
   const int* item;                                           // slot -> request it serves, or null
   int B, K;
@@ -74,7 +78,7 @@ __host__ __device__ inline DcSmem dc_smem_plan(int d, int layers, int A, bool re
   p.off_x = take(DC_ROWS * 16 * 4 * 2);                      // latent and eps, D <= 256
   p.off_posb = take(DC_ROWS * d * 4);
   p.off_win = take(A * d * 4);
-  p.off_par = take((layers * 17 * d + 2 * d + A * d + 16) * 4);   // biases, LayerNorm parameters, head
+  p.off_par = take((layers * (6 * d + 11 * d / DC_CS) + 2 * d + A * d + 16) * 4);   // LayerNorm parameters, this CTA's bias slices, head
   p.total = o;
   return p;
 }
@@ -360,16 +364,23 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
     h[i] = 0.f;
   }
   for (int i = threadIdx.x; i < A * d; i += DC_THREADS) win[i] = P.W_in[i];
-  // biases and LayerNorm parameters of every block, then the head: read from shared memory on the critical path
+  // LayerNorm parameters and this CTA's slices of the biases of every block, then the head: read from shared
+  // memory on the critical path
+  constexpr int PL = 6 * d + 11 * d / DC_CS;       // floats per block
   for (int l = 0; l < L; ++l) {
     const DcLayer& G = P.L[l];
-    const float* src[12] = {G.bqkv, G.bo, G.bq2, G.bo2, G.b1, G.b2, G.ln1_g, G.ln1_b, G.ln2_g, G.ln2_b, G.ln3_g, G.ln3_b};
-    const int off[12] = {0, 3 * d, 4 * d, 5 * d, 6 * d, 10 * d, 11 * d, 12 * d, 13 * d, 14 * d, 15 * d, 16 * d};
-    const int len[12] = {3 * d, d, d, d, 4 * d, d, d, d, d, d, d, d};
-    for (int j = 0; j < 12; ++j)
-      for (int i = threadIdx.x; i < len[j]; i += DC_THREADS) par[(size_t)l * 17 * d + off[j] + i] = src[j][i];
+    const float* ln[6] = {G.ln1_g, G.ln1_b, G.ln2_g, G.ln2_b, G.ln3_g, G.ln3_b};
+    for (int j = 0; j < 6; ++j)
+      for (int i = threadIdx.x; i < d; i += DC_THREADS) par[(size_t)l * PL + j * d + i] = ln[j][i];
+    const float* bs[6] = {G.bqkv, G.bo, G.bq2, G.bo2, G.b1, G.b2};
+    const int ns[6] = {3 * d / DC_CS, d / DC_CS, d / DC_CS, d / DC_CS, 4 * d / DC_CS, d / DC_CS};
+    int off = 6 * d;
+    for (int j = 0; j < 6; ++j) {
+      for (int i = threadIdx.x; i < ns[j]; i += DC_THREADS) par[(size_t)l * PL + off + i] = bs[j][rank * ns[j] + i];
+      off += ns[j];
+    }
   }
-  float* lnf_g = par + (size_t)L * 17 * d;
+  float* lnf_g = par + (size_t)L * PL;
   float* lnf_b = lnf_g + d;
   float* woutT = lnf_b + d;
   float* bout = woutT + A * d;
@@ -393,6 +404,191 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
 
   const uint64_t seed = *P.seed;
   const size_t ldkv = (size_t)L * 2 * d;
+  // One forward of the network on the latent in sx at timestep tau for request env; leaves eps in seps.
+  auto forward = [&](int tau, int env) {
+    // keys / values of the time token of tau, every block
+    for (int i = threadIdx.x; i < (resident ? L : 0) * 2 * d; i += DC_THREADS) {
+      const int l = i / (2 * d), c = i % (2 * d);
+      skv[(size_t)l * DC_MAX_NK * 2 * d + c] = __ldg(P.kv_time + (size_t)tau * ldkv + (size_t)l * 2 * d + c);
+    }
+    // token embedding into the residual stream
+    for (int i = threadIdx.x; i < DC_ROWS * d; i += DC_THREADS) {
+      const int row = i / d, col = i % d;
+      float v = posb[i];
+      if (row < H)
+        for (int c = 0; c < A; ++c) v += sx[row * A + c] * win[c * d + col];
+      h[i] = v;
+    }
+    __syncthreads();
+    for (int l = 0; l < L; ++l) {
+      const float* pb = par + (size_t)l * PL;
+      const float* bb = pb + 6 * d;                      // bias slices: columns of this CTA only
+      struct { const float *ln1_g, *ln1_b, *ln2_g, *ln2_b, *ln3_g, *ln3_b, *bqkv, *bo, *bq2, *bo2, *b1, *b2; } W =
+          {pb, pb + d, pb + 2 * d, pb + 3 * d, pb + 4 * d, pb + 5 * d, bb, bb + NS_3D, bb + NS_3D + NS_D,
+           bb + NS_3D + 2 * NS_D, bb + NS_3D + 3 * NS_D, bb + NS_3D + 3 * NS_D + NS_4D};
+      // ---- causal self-attention
+      dc_layernorm<d>(h, W.ln1_g, W.ln1_b, a, PA);
+      __syncthreads();
+      dc_linear<d>(a, PA, w_ptr(l, 0), PWD, NS_3D, red, [&](int row, int col, float* v) {
+        const int cg_ = rank * NS_3D + col;
+        const float4 b0 = *reinterpret_cast<const float4*>(W.bqkv + col), b1 = *(reinterpret_cast<const float4*>(W.bqkv + col) + 1);
+        v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+        const uint4 pk = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
+#pragma unroll
+        for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(rqkv[r] + row * PQKV + cg_) = pk;
+      });
+      cluster.sync();
+      switch (d / P.heads) {
+        case 32: dc_self_attn_mma<d, 32>(qkv, PQKV, a, PA, P.heads, H); break;
+        case 64: dc_self_attn_mma<d, 64>(qkv, PQKV, a, PA, P.heads, H); break;
+        case 128: dc_self_attn_mma<d, 128>(qkv, PQKV, a, PA, P.heads, H); break;
+        default: dc_attention<d, true>(qkv, PQKV, qkv, PQKV, nullptr, 0, a, PA, P.heads, H); break;
+      }
+      __syncthreads();
+      dc_linear<d>(a, PA, w_ptr(l, 1), PWD, NS_D, red, [&](int row, int col, float* v) {
+        const int cg_ = rank * NS_D + col;
+        const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
+        const float4 h0 = hp[0], h1 = hp[1];
+        const float4 b0 = *reinterpret_cast<const float4*>(W.bo + col), b1 = *(reinterpret_cast<const float4*>(W.bo + col) + 1);
+        const float4 o0 = make_float4(h0.x + v[0] + b0.x, h0.y + v[1] + b0.y, h0.z + v[2] + b0.z, h0.w + v[3] + b0.w);
+        const float4 o1 = make_float4(h1.x + v[4] + b1.x, h1.y + v[5] + b1.y, h1.z + v[6] + b1.z, h1.w + v[7] + b1.w);
+#pragma unroll
+        for (int r = 0; r < DC_CS; ++r) {
+          float4* dst = reinterpret_cast<float4*>(rh[r] + row * d + cg_);
+          dst[0] = o0; dst[1] = o1;
+        }
+      });
+      if (!resident) {   // keys / values of the memory tokens for this block only: time token of tau, then the obs tokens
+        for (int i = threadIdx.x; i < NK * 2 * d; i += DC_THREADS) {
+          const int kx = i / (2 * d), c = i % (2 * d);
+          const float* src = kx == 0 ? P.kv_time + (size_t)tau * ldkv : P.kv_obs + ((size_t)env * P.To + (kx - 1)) * ldkv;
+          skv[i] = __ldg(src + (size_t)l * 2 * d + c);
+        }
+      }
+      cluster.sync();
+      // ---- cross-attention to [time token | obs tokens]
+      dc_layernorm<d>(h, W.ln2_g, W.ln2_b, a, PA);
+      __syncthreads();
+      dc_linear<d>(a, PA, w_ptr(l, 2), PWD, NS_D, red, [&](int row, int col, float* v) {
+        const int cg_ = rank * NS_D + col;
+        const float4 b0 = *reinterpret_cast<const float4*>(W.bq2 + col), b1 = *(reinterpret_cast<const float4*>(W.bq2 + col) + 1);
+        v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+        const uint4 pk = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
+#pragma unroll
+        for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(rq2[r] + row * PA + cg_) = pk;
+      });
+      cluster.sync();
+      dc_attention<d, false>(q2, PA, nullptr, 0, skv + (size_t)(resident ? l : 0) * DC_MAX_NK * 2 * d, NK, a, PA, P.heads, H);
+      __syncthreads();
+      dc_linear<d>(a, PA, w_ptr(l, 3), PWD, NS_D, red, [&](int row, int col, float* v) {
+        const int cg_ = rank * NS_D + col;
+        const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
+        const float4 h0 = hp[0], h1 = hp[1];
+        const float4 b0 = *reinterpret_cast<const float4*>(W.bo2 + col), b1 = *(reinterpret_cast<const float4*>(W.bo2 + col) + 1);
+        const float4 o0 = make_float4(h0.x + v[0] + b0.x, h0.y + v[1] + b0.y, h0.z + v[2] + b0.z, h0.w + v[3] + b0.w);
+        const float4 o1 = make_float4(h1.x + v[4] + b1.x, h1.y + v[5] + b1.y, h1.z + v[6] + b1.z, h1.w + v[7] + b1.w);
+#pragma unroll
+        for (int r = 0; r < DC_CS; ++r) {
+          float4* dst = reinterpret_cast<float4*>(rh[r] + row * d + cg_);
+          dst[0] = o0; dst[1] = o1;
+        }
+      });
+      cluster.sync();
+      // ---- MLP
+      dc_layernorm<d>(h, W.ln3_g, W.ln3_b, a, PA);
+      __syncthreads();
+      dc_linear<d>(a, PA, w_ptr(l, 4), PWD, NS_4D, red, [&](int row, int col, float* v) {
+        const int cg_ = rank * NS_4D + col;
+        const float4 b0 = *reinterpret_cast<const float4*>(W.b1 + col), b1 = *(reinterpret_cast<const float4*>(W.b1 + col) + 1);
+        v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          v[j] = 0.5f * v[j] * (1.0f + ptx::tanh_fast(0.7978845608028654f * (v[j] + 0.044715f * v[j] * v[j] * v[j])));
+        const uint4 pk = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
+#pragma unroll
+        for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(rf[r] + row * PF + cg_) = pk;
+      });
+      cluster.sync();
+      dc_linear<4 * d>(f, PF, w_ptr(l, 5), PW4, NS_D, red, [&](int row, int col, float* v) {
+        const int cg_ = rank * NS_D + col;
+        const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
+        const float4 h0 = hp[0], h1 = hp[1];
+        const float4 b0 = *reinterpret_cast<const float4*>(W.b2 + col), b1 = *(reinterpret_cast<const float4*>(W.b2 + col) + 1);
+        const float4 o0 = make_float4(h0.x + v[0] + b0.x, h0.y + v[1] + b0.y, h0.z + v[2] + b0.z, h0.w + v[3] + b0.w);
+        const float4 o1 = make_float4(h1.x + v[4] + b1.x, h1.y + v[5] + b1.y, h1.z + v[6] + b1.z, h1.w + v[7] + b1.w);
+#pragma unroll
+        for (int r = 0; r < DC_CS; ++r) {
+          float4* dst = reinterpret_cast<float4*>(rh[r] + row * d + cg_);
+          dst[0] = o0; dst[1] = o1;
+        }
+      });
+      cluster.sync();
+    }
+    // ---- head: eps = LN_f(h) W_out + b_out   (every CTA, rows w and w + 8 per warp)
+    {
+      constexpr int V = d / 128;
+#pragma unroll
+      for (int rr = 0; rr < 2; ++rr) {
+        const int row = warp + rr * 8;
+        float4 v[V];
+        float s = 0.f;
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+          v[j] = *reinterpret_cast<const float4*>(h + row * d + j * 128 + lane * 4);
+          s += v[j].x + v[j].y + v[j].z + v[j].w;
+        }
+        const float mean = warp_sum(s) / d;
+        float q = 0.f;
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+          v[j].x -= mean; v[j].y -= mean; v[j].z -= mean; v[j].w -= mean;
+          q += v[j].x * v[j].x + v[j].y * v[j].y + v[j].z * v[j].z + v[j].w * v[j].w;
+        }
+        const float rstd = rsqrtf(warp_sum(q) / d + 1e-5f);
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+          const int c = j * 128 + lane * 4;
+          const float4 gg = *reinterpret_cast<const float4*>(lnf_g + c), bb = *reinterpret_cast<const float4*>(lnf_b + c);
+          v[j].x = v[j].x * rstd * gg.x + bb.x; v[j].y = v[j].y * rstd * gg.y + bb.y;
+          v[j].z = v[j].z * rstd * gg.z + bb.z; v[j].w = v[j].w * rstd * gg.w + bb.w;
+        }
+        for (int c = 0; c < A; ++c) {
+          float acc = 0.f;
+#pragma unroll
+          for (int j = 0; j < V; ++j) {
+            const float4 w = *reinterpret_cast<const float4*>(woutT + (size_t)c * d + j * 128 + lane * 4);
+            acc += v[j].x * w.x + v[j].y * w.y + v[j].z * w.z + v[j].w * w.w;
+          }
+          acc = warp_sum(acc);
+          if (lane == 0 && row < H) seps[row * A + c] = acc + bout[c];
+        }
+      }
+    }
+    __syncthreads();
+  };
+
+  if (P.mode == 1) {      // verification: one forward per (slot, candidate), the whole batch in one wave of clusters
+    for (int w = cid; w < P.B * P.C; w += ncl) {
+      const int slot = w / P.C, cand = w % P.C;
+      const int tb = P.t[slot];
+      if (tb < 0 || cand > tb) continue;          // finished slot, or a candidate beyond t = 0 (same for every CTA)
+      const int env = item_of(P.item, slot);
+      const float* xin = P.xt + slot * P.xs_b + (long long)cand * D;
+      for (int i = threadIdx.x; i < D; i += DC_THREADS) sx[i] = xin[i];
+      for (int i = threadIdx.x; i < (resident ? L : 0) * P.To * 2 * d; i += DC_THREADS) {
+        const int l = i / (P.To * 2 * d), rem = i % (P.To * 2 * d);
+        const int kx = 1 + rem / (2 * d), c = rem % (2 * d);
+        skv[((size_t)l * DC_MAX_NK + kx) * 2 * d + c] = __ldg(P.kv_obs + ((size_t)env * P.To + (kx - 1)) * ldkv + (size_t)l * 2 * d + c);
+      }
+      __syncthreads();
+      forward(tb - cand, env);
+      if (rank == 0)
+        for (int i = threadIdx.x; i < D; i += DC_THREADS) P.eps[slot * P.es_b + (long long)cand * D + i] = seps[i];
+      __syncthreads();
+    }
+    cluster.sync();
+    return;
+  }
   for (int slot = cid; slot < P.B; slot += ncl) {
     const int tb = P.t[slot];
     const int env = item_of(P.item, slot);     // request served by this slot: its noise streams, obs K/V, parameters
@@ -416,164 +612,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
           }
         continue;
       }
-      // keys / values of the time token of tau, every block
-      for (int i = threadIdx.x; i < (resident ? L : 0) * 2 * d; i += DC_THREADS) {
-        const int l = i / (2 * d), c = i % (2 * d);
-        skv[(size_t)l * DC_MAX_NK * 2 * d + c] = __ldg(P.kv_time + (size_t)tau * ldkv + (size_t)l * 2 * d + c);
-      }
-      // token embedding into the residual stream
-      for (int i = threadIdx.x; i < DC_ROWS * d; i += DC_THREADS) {
-        const int row = i / d, col = i % d;
-        float v = posb[i];
-        if (row < H)
-          for (int c = 0; c < A; ++c) v += sx[row * A + c] * win[c * d + col];
-        h[i] = v;
-      }
-      __syncthreads();
-      for (int l = 0; l < L; ++l) {
-        const float* pb = par + (size_t)l * 17 * d;
-        struct { const float *bqkv, *bo, *bq2, *bo2, *b1, *b2, *ln1_g, *ln1_b, *ln2_g, *ln2_b, *ln3_g, *ln3_b; } W =
-            {pb, pb + 3 * d, pb + 4 * d, pb + 5 * d, pb + 6 * d, pb + 10 * d, pb + 11 * d, pb + 12 * d, pb + 13 * d,
-             pb + 14 * d, pb + 15 * d, pb + 16 * d};
-        // ---- causal self-attention
-        dc_layernorm<d>(h, W.ln1_g, W.ln1_b, a, PA);
-        __syncthreads();
-        dc_linear<d>(a, PA, w_ptr(l, 0), PWD, NS_3D, red, [&](int row, int col, float* v) {
-          const int cg_ = rank * NS_3D + col;
-          const float4 b0 = *reinterpret_cast<const float4*>(W.bqkv + cg_), b1 = *(reinterpret_cast<const float4*>(W.bqkv + cg_) + 1);
-          v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
-          const uint4 pk = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
-#pragma unroll
-          for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(rqkv[r] + row * PQKV + cg_) = pk;
-        });
-        cluster.sync();
-        switch (d / P.heads) {
-          case 32: dc_self_attn_mma<d, 32>(qkv, PQKV, a, PA, P.heads, H); break;
-          case 64: dc_self_attn_mma<d, 64>(qkv, PQKV, a, PA, P.heads, H); break;
-          case 128: dc_self_attn_mma<d, 128>(qkv, PQKV, a, PA, P.heads, H); break;
-          default: dc_attention<d, true>(qkv, PQKV, qkv, PQKV, nullptr, 0, a, PA, P.heads, H); break;
-        }
-        __syncthreads();
-        dc_linear<d>(a, PA, w_ptr(l, 1), PWD, NS_D, red, [&](int row, int col, float* v) {
-          const int cg_ = rank * NS_D + col;
-          const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
-          const float4 h0 = hp[0], h1 = hp[1];
-          const float4 b0 = *reinterpret_cast<const float4*>(W.bo + cg_), b1 = *(reinterpret_cast<const float4*>(W.bo + cg_) + 1);
-          const float4 o0 = make_float4(h0.x + v[0] + b0.x, h0.y + v[1] + b0.y, h0.z + v[2] + b0.z, h0.w + v[3] + b0.w);
-          const float4 o1 = make_float4(h1.x + v[4] + b1.x, h1.y + v[5] + b1.y, h1.z + v[6] + b1.z, h1.w + v[7] + b1.w);
-#pragma unroll
-          for (int r = 0; r < DC_CS; ++r) {
-            float4* dst = reinterpret_cast<float4*>(rh[r] + row * d + cg_);
-            dst[0] = o0; dst[1] = o1;
-          }
-        });
-        if (!resident) {   // keys / values of the memory tokens for this block only: time token of tau, then the obs tokens
-          for (int i = threadIdx.x; i < NK * 2 * d; i += DC_THREADS) {
-            const int kx = i / (2 * d), c = i % (2 * d);
-            const float* src = kx == 0 ? P.kv_time + (size_t)tau * ldkv : P.kv_obs + ((size_t)env * P.To + (kx - 1)) * ldkv;
-            skv[i] = __ldg(src + (size_t)l * 2 * d + c);
-          }
-        }
-        cluster.sync();
-        // ---- cross-attention to [time token | obs tokens]
-        dc_layernorm<d>(h, W.ln2_g, W.ln2_b, a, PA);
-        __syncthreads();
-        dc_linear<d>(a, PA, w_ptr(l, 2), PWD, NS_D, red, [&](int row, int col, float* v) {
-          const int cg_ = rank * NS_D + col;
-          const float4 b0 = *reinterpret_cast<const float4*>(W.bq2 + cg_), b1 = *(reinterpret_cast<const float4*>(W.bq2 + cg_) + 1);
-          v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
-          const uint4 pk = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
-#pragma unroll
-          for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(rq2[r] + row * PA + cg_) = pk;
-        });
-        cluster.sync();
-        dc_attention<d, false>(q2, PA, nullptr, 0, skv + (size_t)(resident ? l : 0) * DC_MAX_NK * 2 * d, NK, a, PA, P.heads, H);
-        __syncthreads();
-        dc_linear<d>(a, PA, w_ptr(l, 3), PWD, NS_D, red, [&](int row, int col, float* v) {
-          const int cg_ = rank * NS_D + col;
-          const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
-          const float4 h0 = hp[0], h1 = hp[1];
-          const float4 b0 = *reinterpret_cast<const float4*>(W.bo2 + cg_), b1 = *(reinterpret_cast<const float4*>(W.bo2 + cg_) + 1);
-          const float4 o0 = make_float4(h0.x + v[0] + b0.x, h0.y + v[1] + b0.y, h0.z + v[2] + b0.z, h0.w + v[3] + b0.w);
-          const float4 o1 = make_float4(h1.x + v[4] + b1.x, h1.y + v[5] + b1.y, h1.z + v[6] + b1.z, h1.w + v[7] + b1.w);
-#pragma unroll
-          for (int r = 0; r < DC_CS; ++r) {
-            float4* dst = reinterpret_cast<float4*>(rh[r] + row * d + cg_);
-            dst[0] = o0; dst[1] = o1;
-          }
-        });
-        cluster.sync();
-        // ---- MLP
-        dc_layernorm<d>(h, W.ln3_g, W.ln3_b, a, PA);
-        __syncthreads();
-        dc_linear<d>(a, PA, w_ptr(l, 4), PWD, NS_4D, red, [&](int row, int col, float* v) {
-          const int cg_ = rank * NS_4D + col;
-          const float4 b0 = *reinterpret_cast<const float4*>(W.b1 + cg_), b1 = *(reinterpret_cast<const float4*>(W.b1 + cg_) + 1);
-          v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
-#pragma unroll
-          for (int j = 0; j < 8; ++j)
-            v[j] = 0.5f * v[j] * (1.0f + ptx::tanh_fast(0.7978845608028654f * (v[j] + 0.044715f * v[j] * v[j] * v[j])));
-          const uint4 pk = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
-#pragma unroll
-          for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(rf[r] + row * PF + cg_) = pk;
-        });
-        cluster.sync();
-        dc_linear<4 * d>(f, PF, w_ptr(l, 5), PW4, NS_D, red, [&](int row, int col, float* v) {
-          const int cg_ = rank * NS_D + col;
-          const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
-          const float4 h0 = hp[0], h1 = hp[1];
-          const float4 b0 = *reinterpret_cast<const float4*>(W.b2 + cg_), b1 = *(reinterpret_cast<const float4*>(W.b2 + cg_) + 1);
-          const float4 o0 = make_float4(h0.x + v[0] + b0.x, h0.y + v[1] + b0.y, h0.z + v[2] + b0.z, h0.w + v[3] + b0.w);
-          const float4 o1 = make_float4(h1.x + v[4] + b1.x, h1.y + v[5] + b1.y, h1.z + v[6] + b1.z, h1.w + v[7] + b1.w);
-#pragma unroll
-          for (int r = 0; r < DC_CS; ++r) {
-            float4* dst = reinterpret_cast<float4*>(rh[r] + row * d + cg_);
-            dst[0] = o0; dst[1] = o1;
-          }
-        });
-        cluster.sync();
-      }
-      // ---- head: eps = LN_f(h) W_out + b_out   (every CTA, rows w and w + 8 per warp)
-      {
-        constexpr int V = d / 128;
-#pragma unroll
-        for (int rr = 0; rr < 2; ++rr) {
-          const int row = warp + rr * 8;
-          float4 v[V];
-          float s = 0.f;
-#pragma unroll
-          for (int j = 0; j < V; ++j) {
-            v[j] = *reinterpret_cast<const float4*>(h + row * d + j * 128 + lane * 4);
-            s += v[j].x + v[j].y + v[j].z + v[j].w;
-          }
-          const float mean = warp_sum(s) / d;
-          float q = 0.f;
-#pragma unroll
-          for (int j = 0; j < V; ++j) {
-            v[j].x -= mean; v[j].y -= mean; v[j].z -= mean; v[j].w -= mean;
-            q += v[j].x * v[j].x + v[j].y * v[j].y + v[j].z * v[j].z + v[j].w * v[j].w;
-          }
-          const float rstd = rsqrtf(warp_sum(q) / d + 1e-5f);
-#pragma unroll
-          for (int j = 0; j < V; ++j) {
-            const int c = j * 128 + lane * 4;
-            const float4 gg = *reinterpret_cast<const float4*>(lnf_g + c), bb = *reinterpret_cast<const float4*>(lnf_b + c);
-            v[j].x = v[j].x * rstd * gg.x + bb.x; v[j].y = v[j].y * rstd * gg.y + bb.y;
-            v[j].z = v[j].z * rstd * gg.z + bb.z; v[j].w = v[j].w * rstd * gg.w + bb.w;
-          }
-          for (int c = 0; c < A; ++c) {
-            float acc = 0.f;
-#pragma unroll
-            for (int j = 0; j < V; ++j) {
-              const float4 w = *reinterpret_cast<const float4*>(woutT + (size_t)c * d + j * 128 + lane * 4);
-              acc += v[j].x * w.x + v[j].y * w.y + v[j].z * w.z + v[j].w * w.w;
-            }
-            acc = warp_sum(acc);
-            if (lane == 0 && row < H) seps[row * A + c] = acc + bout[c];
-          }
-        }
-      }
-      __syncthreads();
+      forward(tau, env);
       // ---- scheduler step: mu^_k, x~_k = mu^_k + sigma_tau xi_tau
       {
         const int nq = (D + 3) >> 2;
@@ -585,7 +624,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
             const int i = 4 * q + j;
             if (i < D) {
               const float m = posterior_mean(P.S, sx[i], seps[i], tau);
-              const float xn = m + P.S.sigma[tau] * z[j];
+              const float xn = ddpm_sample(m, P.S.sigma[tau], z[j]);
               sx[i] = xn;
               if (rank == 0) { mh_b[(size_t)(k - 1) * D + i] = m; xt_b[(size_t)k * D + i] = xn; }
             }

@@ -62,7 +62,7 @@ __global__ void draft_step_kernel(DdpmTables S, float* __restrict__ xt, long lon
         if (valid) {
           const float m = posterior_mean(S, x, e[i], tau);
           mh[i] = m;
-          xn[i] = m + S.sigma[tau] * z[j];
+          xn[i] = ddpm_sample(m, S.sigma[tau], z[j]);
         } else {
           mh[i] = x;
           xn[i] = x;
@@ -190,7 +190,7 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
         const int i = 4 * q + jj;
         if (i < D) {
           const float mu = posterior_mean(S, xb[(long long)K_eff * D + i], eb[(long long)K_eff * D + i], tau);
-          const float v = mu + sig * z[jj];
+          const float v = ddpm_sample(mu, sig, z[jj]);
           xo[i] = v;
           if (t_new < 0) actions[(long long)env * D + i] = v;
         }

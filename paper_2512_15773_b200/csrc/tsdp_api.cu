@@ -113,6 +113,9 @@ struct tsdp_ctx {
   bool dc_ok = false;
   int dc_smem = 0, dc_max_clusters = 0;
   bool dc_resident = false;
+  // the same cluster kernel running the BASE model's verification forward (small batches of small transformers)
+  bool cv_ok = false, cv_resident = false;
+  int cv_smem = 0, cv_max_clusters = 0;
   uint64_t rounds = 0, launches = 0;
   int launches_per_round_tmp = 0;
   // optional per-kernel-family timing with CUDA events (plain launches, no graph)
@@ -803,8 +806,7 @@ int forward(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStream_t s) 
 
 // ------------------------------------------------------------------------------------------ drafter
 // Whether the persistent cluster kernel can run this context's drafter at all (shapes, shared memory).
-bool cluster_drafter_fits(const tsdp_config_t& cfg, int* smem_bytes, bool* resident) {
-  const tsdp_net_t& n = cfg.draft;
+bool cluster_drafter_fits(const tsdp_config_t& cfg, const tsdp_net_t& n, int* smem_bytes, bool* resident) {
   if (cfg.precision != 1 || n.arch != TSDP_ARCH_XFMR || (n.d != 128 && n.d != 256) || n.layers > DC_MAX_LAYERS ||
       cfg.H > DC_ROWS || 1 + cfg.obs_tokens > DC_MAX_NK || cfg.H * cfg.A > 256 || (n.d / n.heads) % 4 != 0)
     return false;
@@ -825,8 +827,15 @@ bool use_cluster_drafter(const tsdp_ctx* c, int B) {
   return B <= (c->dc_resident ? 3 : 1) * c->dc_max_clusters;
 }
 
-int launch_cluster_drafter(tsdp_ctx* c, int B, int K, cudaStream_t s) {
-  const Net& n = c->net[TSDP_DRAFT];
+bool use_cluster_verifier(const tsdp_ctx* c, int B, int K) {
+  if (!c->cv_ok || c->cfg.verifier == 1) return false;
+  if (c->cfg.verifier == 2) return true;
+  return B * (K + 1) <= c->cv_max_clusters;     // every candidate gets its own cluster in one wave
+}
+
+// mode 0: K-step draft rollout with the drafter; mode 1: verification forward of the base model on K+1 candidates.
+int launch_cluster_forward(tsdp_ctx* c, int which, int mode, int B, int K, cudaStream_t s) {
+  const Net& n = c->net[which];
   DcParams P{};
   for (int l = 0; l < n.cfg.layers; ++l) {
     const XfmrLayer& w = n.L[l];
@@ -843,14 +852,19 @@ int launch_cluster_drafter(tsdp_ctx* c, int B, int K, cudaStream_t s) {
   P.S = c->S;
   P.xt = c->xt; P.xs_b = (long long)(c->cfg.max_K + 1) * c->D;
   P.muhat = c->muhat; P.ms_b = (long long)(c->cfg.max_K > 0 ? c->cfg.max_K : 1) * c->D;
+  P.eps = c->eps; P.es_b = P.xs_b;
   P.t = c->t; P.seed = c->seed; P.B = B; P.K = K;
+  P.mode = mode; P.C = K + 1;
   P.envp = c->sched_on ? c->envp : nullptr;
   P.item = c->item;
-  P.resident = c->dc_resident ? 1 : 0;
-  const int ncl = B < c->dc_max_clusters ? B : c->dc_max_clusters;
-  prof_begin(c, s, 7, 0.0);
-  if (n.cfg.d == 128) TSDP_LAUNCH(c, (drafter_cluster_kernel<128>), ncl * DC_CS, DC_THREADS, c->dc_smem, s, P);
-  else TSDP_LAUNCH(c, (drafter_cluster_kernel<256>), ncl * DC_CS, DC_THREADS, c->dc_smem, s, P);
+  const bool verify = mode == 1;
+  P.resident = (verify ? c->cv_resident : c->dc_resident) ? 1 : 0;
+  const int maxc = verify ? c->cv_max_clusters : c->dc_max_clusters, smem = verify ? c->cv_smem : c->dc_smem;
+  const int work = verify ? B * (K + 1) : B;
+  const int ncl = work < maxc ? work : maxc;
+  prof_begin(c, s, verify ? 9 : 7, 0.0);
+  if (n.cfg.d == 128) TSDP_LAUNCH(c, (drafter_cluster_kernel<128>), ncl * DC_CS, DC_THREADS, smem, s, P);
+  else TSDP_LAUNCH(c, (drafter_cluster_kernel<256>), ncl * DC_CS, DC_THREADS, smem, s, P);
   prof_end(c, s);
   c->launches_per_round_tmp++;
   CU_TRY(c, cudaGetLastError());
@@ -864,7 +878,7 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
   const long long xs_b = (long long)(c->cfg.max_K + 1) * D, ms_b = (long long)(c->cfg.max_K > 0 ? c->cfg.max_K : 1) * D;
   int r;
   const bool cluster_draft = K > 0 && use_cluster_drafter(c, B);
-  if (cluster_draft && (r = launch_cluster_drafter(c, B, K, s))) return r;
+  if (cluster_draft && (r = launch_cluster_forward(c, TSDP_DRAFT, 0, B, K, s))) return r;
   for (int k = 1; k <= K && !cluster_draft; ++k) {
     CandMap cm{c->xt + (long long)(k - 1) * D, xs_b, c->eps_d, (long long)D, c->t, 1, k - 1, c->item};
     c->prof_gemm_cat = 6;
@@ -879,7 +893,9 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
     CU_TRY(c, cudaGetLastError());
   }
   CandMap cv{c->xt, xs_b, c->eps, xs_b, c->t, K + 1, 0, c->item};
-  if ((r = forward(c, c->net[TSDP_BASE], cv, B * (K + 1), s))) return r;
+  if (use_cluster_verifier(c, B, K)) {
+    if ((r = launch_cluster_forward(c, TSDP_BASE, 1, B, K, s))) return r;
+  } else if ((r = forward(c, c->net[TSDP_BASE], cv, B * (K + 1), s))) return r;
   int warps = K < 1 ? 1 : K;
   if (warps < 4) warps = 4;
   if (warps > 16) warps = 16;
@@ -999,7 +1015,8 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   if (!cfg || !out) return TSDP_ERR_ARG;
   if (cfg->H < 1 || cfg->A < 1 || cfg->T < 1 || cfg->T > TSDP_MAX_T || cfg->max_B < 1 || cfg->max_K < 0 ||
       cfg->max_K > TSDP_MAX_K || cfg->obs_tokens < 0 || cfg->obs_dim < 0 || !(cfg->beta0 > 0.f) || !(cfg->beta1 < 1.f) ||
-      (cfg->precision != 0 && cfg->precision != 1) || cfg->drafter < 0 || cfg->drafter > 2)
+      (cfg->precision != 0 && cfg->precision != 1) || cfg->drafter < 0 || cfg->drafter > 2 || cfg->verifier < 0 ||
+      cfg->verifier > 2)
     return TSDP_ERR_ARG;
   for (const tsdp_net_t* n : {&cfg->base, &cfg->draft}) {
     if (n->arch < TSDP_ARCH_GAUSS || n->arch > TSDP_ARCH_UNET) return TSDP_ERR_UNSUPPORTED;
@@ -1113,19 +1130,29 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
     INIT_TRY(set_smem_attr_all<64>());
     INIT_TRY(set_smem_attr_all<32>());
   }
-  if (cluster_drafter_fits(*cfg, &c->dc_smem, &c->dc_resident)) {
-    const void* fn = cfg->draft.d == 128 ? (const void*)drafter_cluster_kernel<128> : (const void*)drafter_cluster_kernel<256>;
-    INIT_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, c->dc_smem));
+  for (int which = 0; which < 2; ++which) {
+    const tsdp_net_t& nn = which == TSDP_BASE ? cfg->base : cfg->draft;
+    int smem = 0; bool res = false;
+    if (!cluster_drafter_fits(*cfg, nn, &smem, &res)) continue;
+    const void* fn = nn.d == 128 ? (const void*)drafter_cluster_kernel<128> : (const void*)drafter_cluster_kernel<256>;
+    int cur_attr = 0;   // both nets may use the same instantiation: keep the larger request
+    cudaFuncAttributes fa;
+    if (cudaFuncGetAttributes(&fa, fn) == cudaSuccess) cur_attr = fa.maxDynamicSharedSizeBytes;
+    if (smem > cur_attr) INIT_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     cudaLaunchConfig_t lc{};
-    lc.gridDim = dim3(DC_CS * 64); lc.blockDim = dim3(DC_THREADS); lc.dynamicSmemBytes = (size_t)c->dc_smem;
+    lc.gridDim = dim3(DC_CS * 64); lc.blockDim = dim3(DC_THREADS); lc.dynamicSmemBytes = (size_t)smem;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = DC_CS; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     lc.attrs = at; lc.numAttrs = 1;
     int ncl = 0;
     if (cudaOccupancyMaxActiveClusters(&ncl, fn, &lc) != cudaSuccess || ncl < 1) { cudaGetLastError(); ncl = 0; }
-    c->dc_max_clusters = ncl;
-    c->dc_ok = ncl >= 1;
+    if (which == TSDP_DRAFT) { c->dc_smem = smem; c->dc_resident = res; c->dc_max_clusters = ncl; c->dc_ok = ncl >= 1; }
+    else { c->cv_smem = smem; c->cv_resident = res; c->cv_max_clusters = ncl; c->cv_ok = ncl >= 1; }
+  }
+  if (cfg->verifier == 2 && !c->cv_ok) {
+    fprintf(stderr, "tsdp_init: the cluster verification kernel does not fit this configuration\n");
+    return fail(TSDP_ERR_UNSUPPORTED);
   }
   if (cfg->drafter == 2 && !c->dc_ok) {
     fprintf(stderr, "tsdp_init: the persistent cluster drafter does not fit this configuration\n");

@@ -11,11 +11,11 @@ def small_xfmr_workload(precision, d=128, heads=4, layers=2, dd=128, dlayers=1, 
                 draft=dict(arch="xfmr", layers=dlayers, d=dd, heads=heads), gamma=gamma)
 
 
-def setup(wl, max_B, max_K, seed=1, use_graph=1, draft_is_base=False, precision=None, clip=0.0, drafter=0):
+def setup(wl, max_B, max_K, seed=1, use_graph=1, draft_is_base=False, precision=None, clip=0.0, drafter=0, verifier=0):
     prec = wl["precision"] if precision is None else precision
     cfg = binding.make_config(wl["H"], wl["A"], wl["To"], wl["Do"], wl["base"],
                               wl["base"] if draft_is_base else wl["draft"], T=wl["T"], max_B=max_B, max_K=max_K,
-                              precision=prec, use_graph=use_graph, clip=clip, drafter=drafter)
+                              precision=prec, use_graph=use_graph, clip=clip, drafter=drafter, verifier=verifier)
     S = ddpm.Schedule(wl["T"], 1e-4, 0.02)
     if wl["base"]["arch"] == "gauss":
         pb, pd = wl["base_params"], wl["draft_params"]

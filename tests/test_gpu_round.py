@@ -12,8 +12,8 @@ pytestmark = pytest.mark.gpu
 BAND = 1e-3     # |log alpha - log u| below which a flipped accept decision is tolerated
 
 
-def _round_parity(wl, B, K, acc, seed, tol_eps, tol_x, t0s, precision=None, drafter=0):
-    smp, S, base, draft = hp.setup(wl, max_B=B, max_K=max(K, 1), precision=precision, drafter=drafter)
+def _round_parity(wl, B, K, acc, seed, tol_eps, tol_x, t0s, precision=None, drafter=0, verifier=0):
+    smp, S, base, draft = hp.setup(wl, max_B=B, max_K=max(K, 1), precision=precision, drafter=drafter, verifier=verifier)
     shape = (wl["H"], wl["A"]); D = wl["H"] * wl["A"]
     obs = inputs.make_obs(3, B, wl["To"], wl["Do"])
     noise = spec.PhiloxNoise(seed)
@@ -96,9 +96,9 @@ def test_cluster_drafter_matches_layered_drafter(case):
     assert np.max(np.abs(outs[0][1] - outs[1][1])) < 3e-3
 
 
-def _chunk_parity(wl, B, K, acc, seed, tol_final, precision=None, schedule=None, drafter=0):
+def _chunk_parity(wl, B, K, acc, seed, tol_final, precision=None, schedule=None, drafter=0, verifier=0):
     smp, S, base, draft = hp.setup(wl, max_B=B, max_K=max(K, 1) if schedule is None else 10, precision=precision,
-                                   drafter=drafter)
+                                   drafter=drafter, verifier=verifier)
     shape = (wl["H"], wl["A"])
     obs = inputs.make_obs(4, B, wl["To"], wl["Do"])
     dobs = torch.tensor(obs, dtype=torch.float32, device="cuda")
@@ -141,11 +141,12 @@ def test_chunk_toy_mlp_fp32_matches_oracle_exactly_in_structure():
         assert st["env_rounds"] == tot["rounds"] and st["rejections"] == tot["rej"]
 
 
-@pytest.mark.parametrize("precision,drafter", [(0, 0), (1, 1), (1, 2)])
-def test_chunk_pusht_transformer(precision, drafter):
+@pytest.mark.parametrize("precision,drafter,verifier", [(0, 0, 0), (1, 1, 1), (1, 2, 1), (1, 2, 2)])
+def test_chunk_pusht_transformer(precision, drafter, verifier):
     wl = dict(inputs.WORKLOADS["pusht_xfmr"], precision=precision)
     B = 3
-    n_match, tot, st = _chunk_parity(wl, B, 8, hp.accept_t(), 9, 3e-2, precision=precision, drafter=drafter)
+    n_match, tot, st = _chunk_parity(wl, B, 8, hp.accept_t(), 9, 3e-2, precision=precision, drafter=drafter,
+                                     verifier=verifier)
     if precision == 0:
         assert n_match >= B - 1
     else:
@@ -189,8 +190,8 @@ def test_chunk_with_round_schedule_fp32():
 def test_drafter_equal_to_base_accepts_everything_and_equals_vanilla():
     for wl in (dict(inputs.WORKLOADS["toy_mlp"]), hp.small_xfmr_workload(1)):
         B = 4
-        # bit-identity needs the same kernels on both sides: the layer-by-layer drafter
-        smp, S, base, _ = hp.setup(wl, max_B=B, max_K=6, draft_is_base=True, drafter=1)
+        # bit-identity needs the same kernels on both sides: the layer-by-layer drafter and verifier
+        smp, S, base, _ = hp.setup(wl, max_B=B, max_K=6, draft_is_base=True, drafter=1, verifier=1)
         obs = torch.tensor(inputs.make_obs(4, B, wl["To"], wl["Do"]), dtype=torch.float32, device="cuda")
         ref = torch.zeros(B, wl["H"], wl["A"], device="cuda")
         smp.sample_chunk(obs, B, 0, hp.accept_t(), 77, ref)                  # K = 0: vanilla DDPM
@@ -206,6 +207,34 @@ def test_drafter_equal_to_base_accepts_everything_and_equals_vanilla():
             if K == 1 and bonus == 0:
                 assert st["env_rounds"] == 100 * B                           # T base forwards per chunk
         smp.close()
+
+
+def test_cluster_kernel_as_drafter_and_verifier_reproduces_vanilla_bit_for_bit():
+    """Batch 1 with the cluster kernel on both sides: the same arithmetic drafts and verifies, so with
+    drafter == base every draft is accepted and the chunk equals vanilla DDPM (K = 0) exactly."""
+    wl = hp.small_xfmr_workload(1)
+    smp, *_ = hp.setup(wl, max_B=1, max_K=6, draft_is_base=True, drafter=2, verifier=2)
+    obs = torch.tensor(inputs.make_obs(4, 1, wl["To"], wl["Do"]), dtype=torch.float32, device="cuda")
+    ref = torch.zeros(1, wl["H"], wl["A"], device="cuda")
+    smp.sample_chunk(obs, 1, 0, hp.accept_t(), 77, ref)
+    for K in (6, 3):
+        smp.reset_stats()
+        out = torch.zeros_like(ref)
+        smp.sample_chunk(obs, 1, K, hp.accept_t(), 77, out)
+        st = smp.stats()
+        assert st["rejections"] == 0 and st["drafts_accepted"] == st["draft_evals"]
+        assert torch.equal(out, ref)
+    smp.close()
+
+
+@pytest.mark.parametrize("B,K", [(1, 8), (2, 4)])
+def test_round_transformer_cluster_verifier(B, K):
+    """Verification forward through the cluster kernel (one cluster per candidate) against the oracle."""
+    wl = dict(inputs.WORKLOADS["pusht_xfmr"], precision=1)
+    smp, S, base, draft = hp.setup(wl, max_B=B, max_K=K, drafter=2, verifier=2)
+    smp.close()
+    _round_parity_cfg = dict(drafter=2, verifier=2)
+    _round_parity(wl, B, K, hp.accept_t(), 21, 2e-2, 3e-3, [99, 40][:B], **_round_parity_cfg)
 
 
 def test_cluster_drafter_equal_to_base_is_accepted_almost_always():

@@ -93,7 +93,7 @@ __device__ __forceinline__ void dc_linear(const __nv_bfloat16* X, int px, const 
   const int g = lane >> 2, tg = lane & 3;
   const int n_tiles = n_slice >> 3;      // PW: row pitch of W (KD + 8 in shared memory, KD in global memory)
   int ksplit = 1;
-  while (n_tiles * ksplit * 2 <= DC_WARPS && (KD / 16) % (ksplit * 2) == 0) ksplit *= 2;
+  while (n_tiles * ksplit * 2 <= DC_WARPS && (KD / 32) % (ksplit * 2) == 0) ksplit *= 2;     // parts of whole 32-k blocks
   const int units = n_tiles * ksplit;
   for (int u0 = 0; u0 < units; u0 += DC_WARPS) {
     const int u = u0 + warp;
@@ -104,17 +104,20 @@ __device__ __forceinline__ void dc_linear(const __nv_bfloat16* X, int px, const 
       const __nv_bfloat16* wrow = W + (size_t)(nt * 8 + g) * PW;
       const __nv_bfloat16* x0 = X + (size_t)g * px;
       const __nv_bfloat16* x1 = X + (size_t)(g + 8) * px;
+      // Two k-steps (32 values of k) per iteration.  Lane (g, tg) reads 8 CONSECUTIVE k of its rows, 16 bytes at
+      // a time, and feeds pairs (0,1 | 2,3) to the first mma and (4,5 | 6,7) to the second: a permutation of k
+      // inside the block of 32 that A and B share, so the sum is unchanged while every load is one full
+      // 16-byte access (four times fewer loads than the natural fragment layout; it matters most when the
+      // weights come from the L2).
 #pragma unroll 8
-      for (int ks = ks0; ks < ks1; ++ks) {
-        const int k = ks * 16 + 2 * tg;
-        uint32_t a[4];
-        a[0] = *reinterpret_cast<const uint32_t*>(x0 + k);
-        a[1] = *reinterpret_cast<const uint32_t*>(x1 + k);
-        a[2] = *reinterpret_cast<const uint32_t*>(x0 + k + 8);
-        a[3] = *reinterpret_cast<const uint32_t*>(x1 + k + 8);
-        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(wrow + k);
-        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(wrow + k + 8);
-        mma_bf16_16816(c, a, b0, b1);
+      for (int ks = ks0; ks < ks1; ks += 2) {
+        const int k = ks * 16 + 8 * tg;
+        const uint4 xa = *reinterpret_cast<const uint4*>(x0 + k);
+        const uint4 xb = *reinterpret_cast<const uint4*>(x1 + k);
+        const uint4 wv = *reinterpret_cast<const uint4*>(wrow + k);
+        const uint32_t a1[4] = {xa.x, xb.x, xa.y, xb.y}, a2[4] = {xa.z, xb.z, xa.w, xb.w};
+        mma_bf16_16816(c, a1, wv.x, wv.y);
+        mma_bf16_16816(c, a2, wv.z, wv.w);
       }
       float* r = red + (size_t)warp * (DC_ROWS * 8);
       r[g * 8 + 2 * tg] = c[0]; r[g * 8 + 2 * tg + 1] = c[1];

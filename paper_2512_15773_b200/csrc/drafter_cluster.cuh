@@ -146,37 +146,40 @@ __device__ __forceinline__ void dc_linear(const __nv_bfloat16* X, int px, const 
 }
 
 
-// LayerNorm of the 16 replicated rows: warp w normalises rows w and w + 8; fp32 in, bf16 out.
+// LayerNorm of the 16 replicated rows: each half-warp normalises one row (warp w: rows 2w and 2w + 1), so
+// the 16 rows go through in one pass; fp32 in, bf16 out.
+__device__ __forceinline__ float half_warp_sum(float v) {
+#pragma unroll
+  for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
 template <int D_MODEL>
 __device__ __forceinline__ void dc_layernorm(const float* h, const float* gam, const float* bet,
                                              __nv_bfloat16* out, int pitch) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  constexpr int V = D_MODEL / 128;
+  const int row = 2 * warp + (lane >> 4), l16 = lane & 15;
+  constexpr int V = D_MODEL / 64;          // float4 per lane
+  float4 v[V];
+  float s = 0.f;
 #pragma unroll
-  for (int rr = 0; rr < 2; ++rr) {
-    const int row = warp + rr * 8;
-    float4 v[V];
-    float s = 0.f;
+  for (int j = 0; j < V; ++j) {
+    v[j] = *reinterpret_cast<const float4*>(h + row * D_MODEL + (j * 16 + l16) * 4);
+    s += v[j].x + v[j].y + v[j].z + v[j].w;
+  }
+  const float mean = half_warp_sum(s) / D_MODEL;
+  float q = 0.f;
 #pragma unroll
-    for (int j = 0; j < V; ++j) {
-      v[j] = *reinterpret_cast<const float4*>(h + row * D_MODEL + j * 128 + lane * 4);
-      s += v[j].x + v[j].y + v[j].z + v[j].w;
-    }
-    const float mean = warp_sum(s) / D_MODEL;
-    float q = 0.f;
+  for (int j = 0; j < V; ++j) {
+    v[j].x -= mean; v[j].y -= mean; v[j].z -= mean; v[j].w -= mean;
+    q += v[j].x * v[j].x + v[j].y * v[j].y + v[j].z * v[j].z + v[j].w * v[j].w;
+  }
+  const float rstd = rsqrtf(half_warp_sum(q) / D_MODEL + 1e-5f);
 #pragma unroll
-    for (int j = 0; j < V; ++j) {
-      v[j].x -= mean; v[j].y -= mean; v[j].z -= mean; v[j].w -= mean;
-      q += v[j].x * v[j].x + v[j].y * v[j].y + v[j].z * v[j].z + v[j].w * v[j].w;
-    }
-    const float rstd = rsqrtf(warp_sum(q) / D_MODEL + 1e-5f);
-#pragma unroll
-    for (int j = 0; j < V; ++j) {
-      const int c = j * 128 + lane * 4;
-      const float4 gg = *reinterpret_cast<const float4*>(gam + c), bb = *reinterpret_cast<const float4*>(bet + c);
-      store4(out + row * pitch + c, v[j].x * rstd * gg.x + bb.x, v[j].y * rstd * gg.y + bb.y,
-             v[j].z * rstd * gg.z + bb.z, v[j].w * rstd * gg.w + bb.w);
-    }
+  for (int j = 0; j < V; ++j) {
+    const int c = (j * 16 + l16) * 4;
+    const float4 gg = *reinterpret_cast<const float4*>(gam + c), bb = *reinterpret_cast<const float4*>(bet + c);
+    store4(out + row * pitch + c, v[j].x * rstd * gg.x + bb.x, v[j].y * rstd * gg.y + bb.y,
+           v[j].z * rstd * gg.z + bb.z, v[j].w * rstd * gg.w + bb.w);
   }
 }
 

@@ -109,7 +109,7 @@ __device__ __forceinline__ void dc_linear(const __nv_bfloat16* X, int px, const 
       // inside the block of 32 that A and B share, so the sum is unchanged while every load is one full
       // 16-byte access (four times fewer loads than the natural fragment layout; it matters most when the
       // weights come from the L2).
-#pragma unroll 8
+#pragma unroll 4
       for (int ks = ks0; ks < ks1; ks += 2) {
         const int k = ks * 16 + 8 * tg;
         const uint4 xa = *reinterpret_cast<const uint4*>(x0 + k);
@@ -396,15 +396,9 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
   for (int i = threadIdx.x; i < DC_ROWS * PA; i += DC_THREADS) { a[i] = __float2bfloat16_rn(0.f); q2[i] = a[i]; }
   for (int i = threadIdx.x; i < DC_ROWS * PQKV; i += DC_THREADS) qkv[i] = __float2bfloat16_rn(0.f);
   for (int i = threadIdx.x; i < DC_ROWS * PF; i += DC_THREADS) f[i] = __float2bfloat16_rn(0.f);
-  // replicas of the other CTAs, addressed through distributed shared memory
-  float* rh[DC_CS]; __nv_bfloat16 *rqkv[DC_CS], *rq2[DC_CS], *rf[DC_CS];
-#pragma unroll
-  for (int r = 0; r < DC_CS; ++r) {
-    rh[r] = cluster.map_shared_rank(h, r);
-    rqkv[r] = cluster.map_shared_rank(qkv, r);
-    rq2[r] = cluster.map_shared_rank(q2, r);
-    rf[r] = cluster.map_shared_rank(f, r);
-  }
+  // The replicas of the other CTAs are addressed through distributed shared memory (map_shared_rank in a rolled
+  // loop at each broadcast: the kernel is a long straight line of code executed once per stage, so code size
+  // -- instruction-cache misses -- matters more than the few address computations).
   cluster.sync();
   pdl_wait();      // weights and tables above are constant; t, the latents and the obs K/V come from earlier kernels
 
@@ -440,8 +434,8 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         const float4 b0 = *reinterpret_cast<const float4*>(W.bqkv + col), b1 = *(reinterpret_cast<const float4*>(W.bqkv + col) + 1);
         v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
         const uint4 pk = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
-#pragma unroll
-        for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(rqkv[r] + row * PQKV + cg_) = pk;
+#pragma unroll 1
+        for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(cluster.map_shared_rank(qkv, r) + row * PQKV + cg_) = pk;
       });
       cluster.sync();
       switch (d / P.heads) {
@@ -458,9 +452,9 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         const float4 b0 = *reinterpret_cast<const float4*>(W.bo + col), b1 = *(reinterpret_cast<const float4*>(W.bo + col) + 1);
         const float4 o0 = make_float4(h0.x + v[0] + b0.x, h0.y + v[1] + b0.y, h0.z + v[2] + b0.z, h0.w + v[3] + b0.w);
         const float4 o1 = make_float4(h1.x + v[4] + b1.x, h1.y + v[5] + b1.y, h1.z + v[6] + b1.z, h1.w + v[7] + b1.w);
-#pragma unroll
+#pragma unroll 1
         for (int r = 0; r < DC_CS; ++r) {
-          float4* dst = reinterpret_cast<float4*>(rh[r] + row * d + cg_);
+          float4* dst = reinterpret_cast<float4*>(cluster.map_shared_rank(h, r) + row * d + cg_);
           dst[0] = o0; dst[1] = o1;
         }
       });
@@ -480,8 +474,8 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         const float4 b0 = *reinterpret_cast<const float4*>(W.bq2 + col), b1 = *(reinterpret_cast<const float4*>(W.bq2 + col) + 1);
         v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
         const uint4 pk = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
-#pragma unroll
-        for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(rq2[r] + row * PA + cg_) = pk;
+#pragma unroll 1
+        for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(cluster.map_shared_rank(q2, r) + row * PA + cg_) = pk;
       });
       cluster.sync();
       dc_attention<d, false>(q2, PA, nullptr, 0, skv + (size_t)(resident ? l : 0) * DC_MAX_NK * 2 * d, NK, a, PA, P.heads, H);
@@ -493,9 +487,9 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         const float4 b0 = *reinterpret_cast<const float4*>(W.bo2 + col), b1 = *(reinterpret_cast<const float4*>(W.bo2 + col) + 1);
         const float4 o0 = make_float4(h0.x + v[0] + b0.x, h0.y + v[1] + b0.y, h0.z + v[2] + b0.z, h0.w + v[3] + b0.w);
         const float4 o1 = make_float4(h1.x + v[4] + b1.x, h1.y + v[5] + b1.y, h1.z + v[6] + b1.z, h1.w + v[7] + b1.w);
-#pragma unroll
+#pragma unroll 1
         for (int r = 0; r < DC_CS; ++r) {
-          float4* dst = reinterpret_cast<float4*>(rh[r] + row * d + cg_);
+          float4* dst = reinterpret_cast<float4*>(cluster.map_shared_rank(h, r) + row * d + cg_);
           dst[0] = o0; dst[1] = o1;
         }
       });
@@ -511,8 +505,8 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         for (int j = 0; j < 8; ++j)
           v[j] = 0.5f * v[j] * (1.0f + ptx::tanh_fast(0.7978845608028654f * (v[j] + 0.044715f * v[j] * v[j] * v[j])));
         const uint4 pk = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
-#pragma unroll
-        for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(rf[r] + row * PF + cg_) = pk;
+#pragma unroll 1
+        for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(cluster.map_shared_rank(f, r) + row * PF + cg_) = pk;
       });
       cluster.sync();
       dc_linear<4 * d>(f, PF, w_ptr(l, 5), PW4, NS_D, red, [&](int row, int col, float* v) {
@@ -522,9 +516,9 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         const float4 b0 = *reinterpret_cast<const float4*>(W.b2 + col), b1 = *(reinterpret_cast<const float4*>(W.b2 + col) + 1);
         const float4 o0 = make_float4(h0.x + v[0] + b0.x, h0.y + v[1] + b0.y, h0.z + v[2] + b0.z, h0.w + v[3] + b0.w);
         const float4 o1 = make_float4(h1.x + v[4] + b1.x, h1.y + v[5] + b1.y, h1.z + v[6] + b1.z, h1.w + v[7] + b1.w);
-#pragma unroll
+#pragma unroll 1
         for (int r = 0; r < DC_CS; ++r) {
-          float4* dst = reinterpret_cast<float4*>(rh[r] + row * d + cg_);
+          float4* dst = reinterpret_cast<float4*>(cluster.map_shared_rank(h, r) + row * d + cg_);
           dst[0] = o0; dst[1] = o1;
         }
       });

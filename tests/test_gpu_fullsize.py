@@ -76,3 +76,25 @@ def test_vla_shaped_dit_forward_at_full_width_sampled_candidates():
             ref = net(x[n].astype(np.float64), int(tau[n]), obs[n])
             assert hp.max_rel(got[n], ref) < 2e-2, (which, n)
     smp.close()
+
+
+def test_mid_size_batch_both_head_widths():
+    """1200 candidates x 16 token rows: the GEMMs run with their TMA-store tiles (128 x 256 for the base, 128 x 128
+    for the drafter), several waves of the attention kernels; head widths 64 and 32."""
+    wl = dict(inputs.WORKLOADS["pusht_xfmr"], precision=1, gamma=1.0)
+    N = 1200
+    smp, S, base, draft = hp.setup(wl, max_B=N, max_K=1)
+    rng = np.random.default_rng(2)
+    x = rng.normal(size=(N, wl["H"], wl["A"])).astype(np.float32)
+    tau = rng.integers(0, 100, size=N).astype(np.int32)
+    obs = inputs.make_obs(6, N, wl["To"], wl["Do"])
+    dx = torch.tensor(x, device="cuda"); dobs = torch.tensor(obs, dtype=torch.float32, device="cuda")
+    for which, net in ((binding.BASE, base), (binding.DRAFT, draft)):
+        out = torch.zeros_like(dx)
+        smp.denoise(which, dx, tau, dobs, N, out)
+        got = out.cpu().numpy()
+        assert np.isfinite(got).all()
+        for n in (0, 1, 7, 599, 1199):
+            ref = net(x[n].astype(np.float64), int(tau[n]), obs[n])
+            assert hp.max_rel(got[n], ref) < 2e-2, (which, n)
+    smp.close()

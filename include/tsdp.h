@@ -223,6 +223,21 @@ int tsdp_gemm(tsdp_ctx* ctx, const void* d_A, const void* d_W, const float* d_bi
 int tsdp_gemm_timed(tsdp_ctx* ctx, const void* d_A, const void* d_W, const float* d_bias, int M, int N, int K,
                     int epi, void* d_out, int reps, float* h_ms, void* cuda_stream);
 
+/* Per-request efficiency counters of the last tsdp_sample_chunk / tsdp_sample_chunk_host / tsdp_serve /
+ * tsdp_round call (zeroed when that call starts): h_counts [n, 4] int32 on the HOST, per request
+ * {n_draft: drafts proposed, n_accept: drafts accepted, rounds, n_diffusion: reverse steps taken
+ * (= T once the chunk is complete)}.  n <= the number of requests of that call.  Synchronises the
+ * device.  Errors: ARG, CUDA. */
+int tsdp_request_counts(tsdp_ctx* ctx, int* h_counts, int n);
+/* Intermediate ("process") reward of the scheduler's training signal (Sec. 3.3, "Reward function"),
+ * one value per request of the last call, computed on the device from the counters above:
+ *     r = (n_accept / n_draft + n_accept / n_diffusion) * lambda,
+ *     lambda = (R_final / 4) / ceil(T_max / dt),
+ * T_max the task's step limit and dt the number of task steps between scheduler updates.  A ratio
+ * whose denominator is zero counts 0.  h_reward [n] fp32 on the HOST.  The final (success / failure)
+ * reward needs the simulator and is the caller's.  Errors: ARG (n, T_max < 1, dt < 1), CUDA. */
+int tsdp_process_reward(tsdp_ctx* ctx, float R_final, int T_max, int dt, float* h_reward, int n);
+
 /* Copy the counters accumulated since the last reset (synchronises the device). */
 int tsdp_stats(tsdp_ctx* ctx, tsdp_stats_t* out);
 int tsdp_reset_stats(tsdp_ctx* ctx);

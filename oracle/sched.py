@@ -50,3 +50,17 @@ def stage(t, T):
     if t >= (4 * T) // 5:
         return 0
     return 2 if t < T // 5 else 1
+
+
+def process_reward(n_accept, n_draft, n_diffusion, R_final, T_max, dt):
+    """Intermediate reward of one denoising cycle (Sec. 3.3, "Reward function"):
+
+        r = (n_accept / n_draft + n_accept / n_diffusion) lambda,   lambda = (R_final / 4) / ceil(T_max / dt).
+
+    n_accept accepted drafts, n_draft drafts proposed, n_diffusion diffusion steps of the cycle; T_max the
+    task's step limit, dt the number of task steps between scheduler updates.  A ratio whose denominator
+    is zero counts 0 (the paper does not say; K = 0 proposes no draft)."""
+    lam = (R_final / 4.0) / float(-(-int(T_max) // int(dt)))
+    a = n_accept / n_draft if n_draft > 0 else 0.0
+    e = n_accept / n_diffusion if n_diffusion > 0 else 0.0
+    return (a + e) * lam

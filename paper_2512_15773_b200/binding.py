@@ -16,7 +16,7 @@ EXPORTS = ["tsdp_init", "tsdp_destroy", "tsdp_strerror", "tsdp_last_error", "tsd
            "tsdp_load_weights", "tsdp_set_schedule", "tsdp_sample_chunk", "tsdp_sample_chunk_host",
            "tsdp_round", "tsdp_denoise", "tsdp_gemm", "tsdp_gemm_timed", "tsdp_stats", "tsdp_reset_stats",
            "tsdp_kernel_launches", "tsdp_profile", "tsdp_profile_read", "tsdp_verify_commit_static", "tsdp_set_scheduler", "tsdp_set_progress",
-           "tsdp_sched_eval", "tsdp_serve"]
+           "tsdp_sched_eval", "tsdp_serve", "tsdp_request_counts", "tsdp_process_reward"]
 PROF_FAMILIES = ["gemm", "layernorm", "attention", "embed_head", "round", "small_net", "gemm_draft", "drafter_cluster", "accept", "verifier_cluster"]
 
 
@@ -82,6 +82,8 @@ def load_library():
     lib.tsdp_set_scheduler.argtypes = [vp, i]
     lib.tsdp_set_progress.argtypes = [vp, fp, i]
     lib.tsdp_sched_eval.argtypes = [vp, fp, fp, fp, i, fp, vp]
+    lib.tsdp_request_counts.argtypes = [vp, vp, i]
+    lib.tsdp_process_reward.argtypes = [vp, C.c_float, i, i, fp, i]
     lib.tsdp_stats.argtypes = [vp, C.POINTER(StatsT)]
     lib.tsdp_reset_stats.argtypes = [vp]
     lib.tsdp_kernel_launches.argtypes = [vp]; lib.tsdp_kernel_launches.restype = u64
@@ -219,6 +221,17 @@ class Sampler:
         out = np.zeros((B, 8), dtype=np.float32)
         self._check(self.lib.tsdp_sched_eval(self.h, _ptr(d_obs), _ptr(d_prev_actions), prog.ctypes.data, B,
                                              out.ctypes.data, 0), "tsdp_sched_eval")
+        return out
+
+    def request_counts(self, n):
+        """[n, 4] int32 per request of the last call: drafts proposed, drafts accepted, rounds, reverse steps taken."""
+        out = np.zeros((n, 4), dtype=np.int32)
+        self._check(self.lib.tsdp_request_counts(self.h, out.ctypes.data, n), "tsdp_request_counts")
+        return out
+
+    def process_reward(self, R_final, T_max, dt, n):
+        out = np.zeros(n, dtype=np.float32)
+        self._check(self.lib.tsdp_process_reward(self.h, R_final, T_max, dt, out.ctypes.data, n), "tsdp_process_reward")
         return out
 
     def sample_chunk(self, d_obs, B, K, accept, seed, d_actions, stream=0):

@@ -80,7 +80,9 @@ __global__ void draft_step_kernel(DdpmTables S, float* __restrict__ xt, long lon
 //   all threads: commit -- reflection x = mu + (I - 2 e e^T)(x~ - mu^) at j* (Sec. 3.1), or the bonus
 //       base step, or the last draft -- into slot 0; t -= steps; finished chunks go to `actions`.
 // `item` maps the slot to the request it serves (null: the slot index), `queue_head` / `n_items` feed
-// finished slots with waiting requests (null: no refill).  dbg_* may be null.
+// finished slots with waiting requests (null: no refill).  item_counts (may be null) holds four
+// counters per request -- drafts proposed, drafts accepted, rounds, reverse steps taken -- the inputs of
+// the intermediate reward of Sec. 3.3.  dbg_* may be null.
 __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs_b,
                               const float* __restrict__ muhat, long long ms_b,
                               const float* __restrict__ eps, long long es_b, int* __restrict__ t, int K, int D,
@@ -89,7 +91,7 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
                               int* __restrict__ n_done, DevStats* __restrict__ stats, float draft_nfe,
                               float* __restrict__ dbg_logalpha, int* __restrict__ dbg_jstar,
                               const EnvParams* __restrict__ envp, int* __restrict__ item, int* __restrict__ queue_head,
-                              const int* __restrict__ n_items) {
+                              const int* __restrict__ n_items, int* __restrict__ item_counts) {
   pdl_trigger();
   pdl_wait();
   __shared__ float s_la[32], s_s1[32], s_s2[32];
@@ -221,6 +223,10 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
       if (k <= n_tested) atomicAdd(&stats->hist_tested[tau], 1ull);
       if (k <= n_acc) atomicAdd(&stats->hist_accepted[tau], 1ull);
     }
+    if (item_counts) {                     // a request occupies one slot at a time: no atomics needed
+      int* ic = item_counts + 4 * (long long)env;
+      ic[0] += K_eff; ic[1] += n_acc; ic[2] += 1; ic[3] += adv;
+    }
     if (t_new < 0) {
       atomicAdd(&stats->chunks_done, 1ull);
       atomicAdd(n_done, 1);
@@ -245,6 +251,21 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
       if (threadIdx.x == 0) { item[b] = next; t[b] = S.T - 1; }
     }
   }
+}
+
+// Intermediate ("process") reward of the scheduler's training signal, Sec. 3.3 "Reward function":
+//   r = (n_accept / n_draft + n_accept / n_diffusion) * lambda,  lambda = (R_final / 4) / ceil(T_max / dt),
+// per request, from the counters the acceptance kernel keeps.  A ratio with a zero denominator counts 0.
+__global__ void process_reward_kernel(const int* __restrict__ item_counts, int n, float R_final, int T_max, int dt,
+                                      float* __restrict__ reward) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const int n_draft = item_counts[4 * i], n_acc = item_counts[4 * i + 1], n_diff = item_counts[4 * i + 3];
+  const int n_expected = (T_max + dt - 1) / dt;
+  const float lam = (0.25f * R_final) / (float)n_expected;
+  const float a = n_draft > 0 ? (float)n_acc / (float)n_draft : 0.f;
+  const float e = n_diff > 0 ? (float)n_acc / (float)n_diff : 0.f;
+  reward[i] = (a + e) * lam;
 }
 
 // End of a round: advance the schedule index and publish the number of finished chunks where the

@@ -106,6 +106,9 @@ struct tsdp_ctx {
   bool sched_loaded = false, sched_on = false;
   EnvParams* envp = nullptr;
   float *progress = nullptr, *sched_dbg = nullptr;
+  int* item_counts = nullptr;        // per request: drafts proposed, drafts accepted, rounds, reverse steps taken
+  float* reward = nullptr;
+  int items_last = 0;                // requests of the last chunk call
   std::vector<void*> sched_allocs;
   cudaStream_t side_stream = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
@@ -903,7 +906,7 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
   TSDP_LAUNCH(c, (accept_kernel), B, warps * 32, 0, s, c->S, c->xt, xs_b, c->muhat, ms_b, c->eps, xs_b, c->t, K, D, c->seed, c->sched,
                                          TSDP_MAX_T + 1, c->round_idx, c->actions, c->n_done, c->stats, c->cfg.draft_nfe,
                                          dbg ? c->dbg_logalpha : nullptr, dbg ? c->dbg_jstar : nullptr,
-                                         c->sched_on ? c->envp : nullptr, c->item, c->queue_head, c->n_items);
+                                         c->sched_on ? c->envp : nullptr, c->item, c->queue_head, c->n_items, c->item_counts);
   prof_end(c, s);
   TSDP_LAUNCH(c, (round_end_kernel), 1, 1, 0, s, c->round_idx, c->n_done, c->host_done);
   c->launches_per_round_tmp += 2;
@@ -1090,6 +1093,8 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   st |= dev_alloc(c, c->allocs, &c->envp, B);
   st |= dev_alloc(c, c->allocs, &c->progress, B);
   st |= dev_alloc(c, c->allocs, &c->sched_dbg, B * 8);
+  st |= dev_alloc(c, c->allocs, &c->item_counts, (size_t)B * 4);
+  st |= dev_alloc(c, c->allocs, &c->reward, B);
   if (st) return fail(TSDP_ERR_CUDA);
   INIT_TRY(cudaHostAlloc(reinterpret_cast<void**>(&c->host_done), sizeof(int), cudaHostAllocMapped));
   *c->host_done = 0;
@@ -1597,6 +1602,23 @@ int tsdp_set_schedule(tsdp_ctx* c, const int* Ks, const tsdp_accept_t* accs, int
 
 static int ensure_items(tsdp_ctx* c, size_t N);
 
+int tsdp_request_counts(tsdp_ctx* c, int* h_counts, int n) {
+  if (!c || !h_counts || n < 1 || n > c->items_last) return TSDP_ERR_ARG;
+  CU_TRY(c, cudaSetDevice(c->cfg.device));
+  CU_TRY(c, cudaMemcpy(h_counts, c->item_counts, sizeof(int) * 4 * (size_t)n, cudaMemcpyDeviceToHost));
+  return TSDP_OK;
+}
+
+int tsdp_process_reward(tsdp_ctx* c, float R_final, int T_max, int dt, float* h_reward, int n) {
+  if (!c || !h_reward || n < 1 || n > c->items_last || T_max < 1 || dt < 1) return TSDP_ERR_ARG;
+  CU_TRY(c, cudaSetDevice(c->cfg.device));
+  process_reward_kernel<<<(n + 127) / 128, 128>>>(c->item_counts, n, R_final, T_max, dt, c->reward);
+  c->launches++;
+  CU_TRY(c, cudaGetLastError());
+  CU_TRY(c, cudaMemcpy(h_reward, c->reward, sizeof(float) * (size_t)n, cudaMemcpyDeviceToHost));
+  return TSDP_OK;
+}
+
 int tsdp_set_scheduler(tsdp_ctx* c, int enable) {
   if (!c) return TSDP_ERR_ARG;
   if (enable && !c->sched_loaded) return TSDP_ERR_STATE;
@@ -1648,6 +1670,8 @@ static int ensure_items(tsdp_ctx* c, size_t N) {
   st |= dev_alloc(c, c->allocs, &c->envp, N);
   st |= dev_alloc(c, c->allocs, &c->progress, N);
   st |= dev_alloc(c, c->allocs, &c->sched_dbg, N * 8);
+  st |= dev_alloc(c, c->allocs, &c->item_counts, N * 4);
+  st |= dev_alloc(c, c->allocs, &c->reward, N);
   size_t dmax = 0;
   for (int w = 0; w < 2; ++w) {
     Net& n = c->net[w];
@@ -1686,6 +1710,8 @@ static int sample_chunk_impl(tsdp_ctx* c, const float* obs, bool obs_on_host, in
     CU_TRY(c, cudaMemcpyAsync(c->obs, obs, obs_n * sizeof(float), obs_on_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, s));
   CU_TRY(c, cudaMemcpyAsync(c->seed, &seed, sizeof(seed), cudaMemcpyHostToDevice, s));
   CU_TRY(c, cudaMemcpyAsync(c->n_items, &N, sizeof(int), cudaMemcpyHostToDevice, s));
+  CU_TRY(c, cudaMemsetAsync(c->item_counts, 0, sizeof(int) * 4 * (size_t)N, s));
+  c->items_last = N;
   if ((r = upload_schedule(c, K, *acc, s, false))) return r;
   if (c->sched_on) {
     // the scheduler network reads the new observation, the previous chunk's actions and the progress; it
@@ -1769,6 +1795,8 @@ int tsdp_round(tsdp_ctx* c, const float* d_obs, int B, int K, const tsdp_accept_
     CU_TRY(c, cudaMemcpyAsync(c->item, ident.data(), sizeof(int) * B, cudaMemcpyHostToDevice, s));
     CU_TRY(c, cudaMemcpyAsync(c->queue_head, &B, sizeof(int), cudaMemcpyHostToDevice, s));
     CU_TRY(c, cudaMemcpyAsync(c->n_items, &B, sizeof(int), cudaMemcpyHostToDevice, s));
+    CU_TRY(c, cudaMemsetAsync(c->item_counts, 0, sizeof(int) * 4 * (size_t)B, s));
+    c->items_last = B;
   }
   CU_TRY(c, cudaMemcpyAsync(c->t, h_t, sizeof(int) * B, cudaMemcpyHostToDevice, s));
   CU_TRY(c, cudaMemcpy2DAsync(c->xt, K1 * D * sizeof(float), d_x, D * sizeof(float), D * sizeof(float), B, cudaMemcpyDeviceToDevice, s));
@@ -2027,7 +2055,7 @@ int tsdp_verify_commit_static(int device, int T, float beta0, float beta1, float
   if (warps < 4) warps = 4;
   if (warps > 16) warps = 16;
   accept_kernel<<<B, warps * 32, 0, s>>>(S, d_xt, xs_b, d_muhat, ms_b, d_eps, xs_b, dt, K, D, dseed, drp, 1, dround,
-                                         d_actions, ddone, st, draft_nfe, d_logalpha, dj, nullptr, nullptr, nullptr, nullptr);
+                                         d_actions, ddone, st, draft_nfe, d_logalpha, dj, nullptr, nullptr, nullptr, nullptr, nullptr);
   ST_TRY(cudaGetLastError());
   ST_TRY(cudaMemcpyAsync(h_t_new, dt, sizeof(int) * B, cudaMemcpyDeviceToHost, s));
   ST_TRY(cudaMemcpyAsync(h_jstar, dj, sizeof(int) * B, cudaMemcpyDeviceToHost, s));

@@ -130,6 +130,44 @@ def _chunk_parity(wl, B, K, acc, seed, tol_final, precision=None, schedule=None,
     return n_match, tot, st
 
 
+def test_request_counters_and_process_reward_match_oracle():
+    """Per-request counters (drafts proposed / accepted, rounds, steps) against the oracle's chunk statistics, and
+    the intermediate reward of Sec. 3.3 computed on the device against the oracle's formula."""
+    from oracle import sched as osched
+    wl = dict(inputs.WORKLOADS["toy_mlp"])
+    B, K, seed = 8, 4, 5
+    smp, S, base, draft = hp.setup(wl, max_B=B, max_K=K)
+    shape = (wl["H"], wl["A"])
+    obs = inputs.make_obs(4, B, wl["To"], wl["Do"])
+    dobs = torch.tensor(obs, dtype=torch.float32, device="cuda")
+    out = torch.zeros(B, *shape, device="cuda")
+    acc = hp.accept_t()
+    smp.sample_chunk(dobs, B, K, acc, seed, out)
+    cnt = smp.request_counts(B)
+    rew = smp.process_reward(100.0, 400, 8, B)
+    got = out.cpu().numpy()
+    assert (cnt[:, 3] == 100).all() and (cnt[:, 1] <= cnt[:, 0]).all()
+    n_same = 0
+    for b in range(B):
+        xo, so = spec.sample_chunk(S, base, draft, spec.PhiloxNoise(seed), b, obs[b], shape, K, hp.oracle_accept(acc))
+        # the reward follows from the device's own counters whatever the trajectory did
+        ref = osched.process_reward(int(cnt[b, 1]), int(cnt[b, 0]), int(cnt[b, 3]), 100.0, 400, 8)
+        assert abs(rew[b] - ref) < 1e-6 * max(1.0, ref)
+        if np.max(np.abs(got[b] - xo)) < 3e-2:       # same trajectory (no near-tie flip): same counters
+            n_same += 1
+            assert cnt[b, 0] == so["draft_evals"] and cnt[b, 1] == so["accepted"] and cnt[b, 2] == so["rounds"]
+    assert n_same >= B - 1
+    # continuous batching: the counters follow the request, not the slot
+    N = 20
+    obs2 = inputs.make_obs(6, N, wl["To"], wl["Do"])
+    out2 = torch.zeros(N, *shape, device="cuda")
+    smp.serve(torch.tensor(obs2, dtype=torch.float32, device="cuda"), N, B, K, acc, seed, out2)
+    cnt2 = smp.request_counts(N)
+    assert (cnt2[:, 3] == 100).all() and (cnt2[:, 2] >= 100 // (K + 1)).all()
+    st = smp.stats()
+    smp.close()
+
+
 def test_chunk_toy_mlp_fp32_matches_oracle_exactly_in_structure():
     wl = dict(inputs.WORKLOADS["toy_mlp"])
     B = 8

@@ -53,3 +53,33 @@ def test_one_unit_by_hand():
 def test_stage_boundaries():
     T = 100
     assert [sched.stage(t, T) for t in (99, 80, 79, 20, 19, 0)] == [0, 0, 1, 1, 2, 2]
+
+
+# ---- intermediate reward (Sec. 3.3, "Reward function") ----
+
+def test_process_reward_worked_values():
+    # 80 of 100 drafts accepted in a 100-step cycle; R_final 100, 400 task steps, an update every 8: 50 updates,
+    # lambda = 25 / 50 = 0.5, r = (0.8 + 0.8) 0.5
+    assert abs(sched.process_reward(80, 100, 100, 100.0, 400, 8) - 0.8) < 1e-15
+    # the update count is a ceiling: 401 steps need 51 updates
+    assert abs(sched.process_reward(80, 100, 100, 100.0, 401, 8) - 1.6 * 25.0 / 51.0) < 1e-15
+    # 60 of 75 drafts accepted: the two ratios differ (0.8 and 0.6)
+    assert abs(sched.process_reward(60, 75, 100, 8.0, 10, 1) - 1.4 * 0.2) < 1e-15
+
+
+def test_process_reward_accumulates_to_a_quarter_of_the_final_reward():
+    # lambda is chosen so that cycles whose ratios sum to 1 add up, over the expected number of updates, to
+    # R_final / 4 (the paper's stated purpose of the scaling factor)
+    R, T_max, dt = 40.0, 300, 7
+    n = -(-T_max // dt)
+    total = sum(sched.process_reward(50, 100, 100, R, T_max, dt) for _ in range(n))
+    assert abs(total - R / 4.0) < 1e-12
+
+
+def test_process_reward_edge_cases_and_monotonicity():
+    assert sched.process_reward(0, 0, 100, 10.0, 100, 10) == 0.0          # K = 0: nothing drafted
+    assert sched.process_reward(0, 50, 100, 10.0, 100, 10) == 0.0
+    r = [sched.process_reward(a, 90, 100, 10.0, 100, 10) for a in range(0, 91, 10)]
+    assert all(b > a for a, b in zip(r, r[1:]))
+    # fewer wasted drafts at the same number of accepted ones pays more
+    assert sched.process_reward(60, 70, 100, 10.0, 100, 10) > sched.process_reward(60, 90, 100, 10.0, 100, 10)

@@ -23,6 +23,7 @@
 #include "sched_kernel.cuh"
 #include "dit_kernels.cuh"
 #include "unet_kernels.cuh"
+#include "xattn_fold.cuh"
 
 using namespace tsdp;
 
@@ -50,6 +51,11 @@ struct Net {
   float* kv_time = nullptr;                   // [T, L*2d]   K/V of the time token for every timestep
   float* kv_obs = nullptr;                    // [max_B*To, L*2d]  K/V of the obs tokens, per chunk
   float* temb_table = nullptr;                // [T, temb or d] sinusoidal embedding
+  // XFMR, bf16: cross-attention folded into the memory tokens (xattn_fold.cuh); tables per timestep / per request token
+  bool fold = false;
+  XfoldLayerW* fold_lw = nullptr;             // [L] device
+  __nv_bfloat16 *fold_kq_time = nullptr, *fold_ut_time = nullptr, *fold_kq_obs = nullptr, *fold_ut_obs = nullptr;
+  float *fold_c_time = nullptr, *fold_c_obs = nullptr;
   float* mod = nullptr;                       // DIT: [T, L*6d + 2d] shift / scale / gate vectors of every timestep
   int mod_ld = 0;
   // UNET: residual blocks in execution order, FiLM tables, head
@@ -508,6 +514,50 @@ int cross_attn_launch(tsdp_ctx* c, const Net& n, const T* q2, T* out, const Cand
   return TSDP_OK;
 }
 
+// Whether the cross-attention sub-block of this net runs folded into its memory tokens (xattn_fold.cuh).
+bool xfold_ok(const tsdp_config_t& cfg, const tsdp_net_t& net) {
+  if (cfg.precision != 1 || net.arch != TSDP_ARCH_XFMR || getenv("TSDP_NO_FOLD") != nullptr) return false;
+  const int NK = 1 + cfg.obs_tokens, d = net.d, heads = net.heads;
+  if (heads < 2 || heads % 2 || d % heads) return false;
+  const int dh = d / heads;
+  return cfg.H <= 16 && NK <= XF_MAXNK && NK * heads <= XF_MAXN && (d == 128 || d == 256 || d == 384 || d == 512) &&
+         dh % 8 == 0 && dh <= 128 && xfold_build_smem(d, dh) <= 200 * 1024;
+}
+
+// Fold tables of `rows` memory tokens (keys / values kv, row pitch L*2d) of net n.
+int xfold_build(tsdp_ctx* c, Net& n, const float* kv, int rows, __nv_bfloat16* kq, __nv_bfloat16* ut, float* cc, cudaStream_t s) {
+  const int d = n.cfg.d, heads = n.cfg.heads, L = n.cfg.layers;
+  int splits = (2 * c->num_sms + L * heads - 1) / (L * heads);
+  const int groups = (rows + XF_RB - 1) / XF_RB;
+  if (splits > groups) splits = groups;
+  if (splits < 1) splits = 1;
+  prof_begin(c, s, 3, 0.0);
+  xfold_build_kernel<<<dim3(L * heads, splits), 256, xfold_build_smem(d, d / heads), s>>>(kv, (long long)L * 2 * d, rows, n.fold_lw, L,
+                                                                                          d, heads, kq, ut, cc);
+  prof_end(c, s);
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  return TSDP_OK;
+}
+
+int xattn_fold_launch(tsdp_ctx* c, const Net& n, const float* bo2, const CandMap& cm, int n_cand, int layer, cudaStream_t s) {
+  const int H = c->cfg.H, d = n.cfg.d, heads = n.cfg.heads, L = n.cfg.layers, To = c->cfg.obs_tokens;
+  const XfoldTables tb{n.fold_kq_time, n.fold_ut_time, n.fold_c_time, n.fold_kq_obs, n.fold_ut_obs, n.fold_c_obs};
+  prof_begin(c, s, 2, 0.0);
+#define XF_CASE(DD) TSDP_LAUNCH(c, (xattn_fold_kernel<DD>), n_cand, XF_THREADS, 0, s, c->h, tb, bo2, cm, H, heads, To, layer, L, c->cfg.T)
+  switch (d) {
+    case 128: XF_CASE(128); break;
+    case 256: XF_CASE(256); break;
+    case 384: XF_CASE(384); break;
+    default: XF_CASE(512); break;
+  }
+#undef XF_CASE
+  prof_end(c, s);
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  return TSDP_OK;
+}
+
 template <typename T>
 int xfmr_forward_t(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStream_t s) {
   const int H = c->cfg.H, A = c->cfg.A, d = n.cfg.d, heads = n.cfg.heads, L = n.cfg.layers;
@@ -530,10 +580,14 @@ int xfmr_forward_t(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStrea
     if ((r = gemm(c, a, w.Wqkv, w.bqkv, M, 3 * d, d, out_epi, qkv, 3 * d, s))) return r;
     if ((r = self_attn_launch<T>(c, qkv, a, n_cand, H, d, heads, s))) return r;
     if ((r = gemm(c, a, w.Wo, w.bo, M, d, d, EPI_RESID, c->h, d, s))) return r;
-    if ((r = ln_launch<T>(c, c->h, w.ln2_g, w.ln2_b, a, M, d, s))) return r;
-    if ((r = gemm(c, a, w.Wq2, w.bq2, M, d, d, out_epi, q2, d, s))) return r;
-    if ((r = cross_attn_launch<T>(c, n, q2, a, cm, n_cand, l, s))) return r;
-    if ((r = gemm(c, a, w.Wo2, w.bo2, M, d, d, EPI_RESID, c->h, d, s))) return r;
+    if (n.fold) {
+      if ((r = xattn_fold_launch(c, n, w.bo2, cm, n_cand, l, s))) return r;
+    } else {
+      if ((r = ln_launch<T>(c, c->h, w.ln2_g, w.ln2_b, a, M, d, s))) return r;
+      if ((r = gemm(c, a, w.Wq2, w.bq2, M, d, d, out_epi, q2, d, s))) return r;
+      if ((r = cross_attn_launch<T>(c, n, q2, a, cm, n_cand, l, s))) return r;
+      if ((r = gemm(c, a, w.Wo2, w.bo2, M, d, d, EPI_RESID, c->h, d, s))) return r;
+    }
     if ((r = ln_launch<T>(c, c->h, w.ln3_g, w.ln3_b, a, M, d, s))) return r;
     if ((r = gemm(c, a, w.W1, w.b1, M, 4 * d, d, EPI_GELU, f, 4 * d, s))) return r;
     if ((r = gemm(c, f, w.W2, w.b2, M, d, 4 * d, EPI_RESID, c->h, d, s))) return r;
@@ -552,7 +606,9 @@ int xfmr_prepare_obs_t(tsdp_ctx* c, Net& n, int B, cudaStream_t s) {
   prof_end(c, s);
   c->launches_per_round_tmp++;
   CU_TRY(c, cudaGetLastError());
-  return gemm(c, mt, n.Wkv_all, n.bkv_all, B * To, L * 2 * d, d, EPI_F32, n.kv_obs, L * 2 * d, s);
+  int r = gemm(c, mt, n.Wkv_all, n.bkv_all, B * To, L * 2 * d, d, EPI_F32, n.kv_obs, L * 2 * d, s);
+  if (r || !n.fold) return r;
+  return xfold_build(c, n, n.kv_obs, B * To, n.fold_kq_obs, n.fold_ut_obs, n.fold_c_obs, s);
 }
 
 // ------------------------------------------------------------------------------------------ DiT
@@ -1166,6 +1222,7 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   INIT_TRY(cudaFuncSetAttribute(cross_attn_ctx_mma_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, cx_smem_bytes<32>(256)));
   INIT_TRY(cudaFuncSetAttribute(cross_attn_ctx_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, cx_smem_bytes<64>(256)));
   INIT_TRY(cudaFuncSetAttribute(cross_attn_ctx_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, cx_smem_bytes<128>(256)));
+  INIT_TRY(cudaFuncSetAttribute(xfold_build_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
   INIT_TRY(cudaFuncSetAttribute(self_attn_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
   INIT_TRY(cudaFuncSetAttribute(self_attn_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
   c->net[TSDP_BASE].cfg = cfg->base;
@@ -1583,6 +1640,25 @@ int tsdp_load_weights(tsdp_ctx* c, int which, const float* blob, size_t n) {
     CU_TRY(c, cudaGetLastError());
     if ((r = gemm(c, c->memtok, net.Wkv_all, net.bkv_all, T, (int)(L * 2 * d), (int)d, EPI_F32, net.kv_time, (int)(L * 2 * d), 0)))
       return r;
+    net.fold = xfold_ok(cfg, net.cfg);
+    if (net.fold) {
+      const size_t per_tok = L * net.cfg.heads * d, rows_obs = c->items_cap * (To ? To : 1);
+      std::vector<XfoldLayerW> lw(L);
+      for (size_t l = 0; l < L; ++l)
+        lw[l] = XfoldLayerW{reinterpret_cast<const __nv_bfloat16*>(net.L[l].Wq2), reinterpret_cast<const __nv_bfloat16*>(net.L[l].Wo2),
+                            net.L[l].bq2, net.L[l].ln2_g, net.L[l].ln2_b};
+      int st = 0;
+      st |= dev_alloc(c, net.allocs, &net.fold_lw, L);
+      st |= dev_alloc(c, net.allocs, &net.fold_kq_time, (size_t)T * per_tok);
+      st |= dev_alloc(c, net.allocs, &net.fold_ut_time, (size_t)T * per_tok);
+      st |= dev_alloc(c, net.allocs, &net.fold_c_time, (size_t)T * L * net.cfg.heads);
+      st |= dev_alloc(c, net.allocs, &net.fold_kq_obs, rows_obs * per_tok);
+      st |= dev_alloc(c, net.allocs, &net.fold_ut_obs, rows_obs * per_tok);
+      st |= dev_alloc(c, net.allocs, &net.fold_c_obs, rows_obs * L * net.cfg.heads);
+      if (st) return TSDP_ERR_CUDA;
+      CU_TRY(c, cudaMemcpy(net.fold_lw, lw.data(), sizeof(XfoldLayerW) * L, cudaMemcpyHostToDevice));
+      if ((r = xfold_build(c, net, net.kv_time, T, net.fold_kq_time, net.fold_ut_time, net.fold_c_time, 0))) return r;
+    }
     CU_TRY(c, cudaDeviceSynchronize());
     if ((r = check_status(c))) return r;
   }
@@ -1678,6 +1754,12 @@ static int ensure_items(tsdp_ctx* c, size_t N) {
     if (n.cfg.arch != TSDP_ARCH_XFMR && n.cfg.arch != TSDP_ARCH_DIT) continue;
     dmax = std::max(dmax, (size_t)n.cfg.d);
     if (n.loaded) st |= dev_alloc(c, n.allocs, &n.kv_obs, N * (To ? To : 1) * n.cfg.layers * 2 * n.cfg.d);
+    if (n.loaded && n.fold) {
+      const size_t rows_obs = N * (To ? To : 1), per_tok = (size_t)n.cfg.layers * n.cfg.heads * n.cfg.d;
+      st |= dev_alloc(c, n.allocs, &n.fold_kq_obs, rows_obs * per_tok);
+      st |= dev_alloc(c, n.allocs, &n.fold_ut_obs, rows_obs * per_tok);
+      st |= dev_alloc(c, n.allocs, &n.fold_c_obs, rows_obs * n.cfg.layers * n.cfg.heads);
+    }
   }
   for (int w = 0; w < 2; ++w) {
     Net& n = c->net[w];

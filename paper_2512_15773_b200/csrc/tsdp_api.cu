@@ -520,7 +520,7 @@ bool xfold_ok(const tsdp_config_t& cfg, const tsdp_net_t& net) {
   const int NK = 1 + cfg.obs_tokens, d = net.d, heads = net.heads;
   if (heads < 2 || heads % 2 || d % heads) return false;
   const int dh = d / heads;
-  return cfg.H <= 16 && NK <= XF_MAXNK && NK * heads <= XF_MAXN && (d == 128 || d == 256 || d == 384 || d == 512) &&
+  return cfg.H <= 16 && NK <= XF_MAXNK && NK * heads <= XF_MAXN && (d == 128 || d == 256 || d == 512) &&
          dh % 8 == 0 && dh <= 128 && xfold_build_smem(d, dh) <= 200 * 1024;
 }
 
@@ -544,11 +544,10 @@ int xattn_fold_launch(tsdp_ctx* c, const Net& n, const float* bo2, const CandMap
   const int H = c->cfg.H, d = n.cfg.d, heads = n.cfg.heads, L = n.cfg.layers, To = c->cfg.obs_tokens;
   const XfoldTables tb{n.fold_kq_time, n.fold_ut_time, n.fold_c_time, n.fold_kq_obs, n.fold_ut_obs, n.fold_c_obs};
   prof_begin(c, s, 2, 0.0);
-#define XF_CASE(DD) TSDP_LAUNCH(c, (xattn_fold_kernel<DD>), n_cand, XF_THREADS, 0, s, c->h, tb, bo2, cm, H, heads, To, layer, L, c->cfg.T)
+#define XF_CASE(DD) TSDP_LAUNCH(c, (xattn_fold_kernel<DD>), n_cand, XF_THREADS, xf_smem_bytes(DD, (1 + To) * heads), s, c->h, tb, bo2, cm, H, heads, To, layer, L, c->cfg.T)
   switch (d) {
     case 128: XF_CASE(128); break;
     case 256: XF_CASE(256); break;
-    case 384: XF_CASE(384); break;
     default: XF_CASE(512); break;
   }
 #undef XF_CASE
@@ -1223,6 +1222,9 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   INIT_TRY(cudaFuncSetAttribute(cross_attn_ctx_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, cx_smem_bytes<64>(256)));
   INIT_TRY(cudaFuncSetAttribute(cross_attn_ctx_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, cx_smem_bytes<128>(256)));
   INIT_TRY(cudaFuncSetAttribute(xfold_build_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+  INIT_TRY(cudaFuncSetAttribute(xattn_fold_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)xf_smem_bytes(128, XF_MAXN)));
+  INIT_TRY(cudaFuncSetAttribute(xattn_fold_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)xf_smem_bytes(256, XF_MAXN)));
+  INIT_TRY(cudaFuncSetAttribute(xattn_fold_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)xf_smem_bytes(512, XF_MAXN)));
   INIT_TRY(cudaFuncSetAttribute(self_attn_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
   INIT_TRY(cudaFuncSetAttribute(self_attn_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
   c->net[TSDP_BASE].cfg = cfg->base;

@@ -15,9 +15,9 @@
 // when its observation arrives (observation tokens).
 //
 // Table layouts (bf16 unless noted), `row` = timestep or request * obs_tokens + token:
-//   kq [row][layer][heads][d]           a lane's B fragments of consecutive k steps are 32 bytes apart
-//   ut [row][layer][heads/2][d][2]      u transposed, heads in pairs: a lane's B fragments of consecutive 8-column
-//                                       tiles are 32 bytes apart, and 8 lanes read one full 32-byte sector
+//   kq [row][layer][heads][d]           one contiguous row of d values per (memory token, head)
+//   ut [row][layer][heads/2][d][2]      heads in pairs: word (q, o) holds u of heads 2q and 2q+1 at output column o,
+//                                       which is one B-fragment register of the second product
 //   cc [row][layer][heads]  fp32
 #pragma once
 #include "common.cuh"
@@ -25,7 +25,8 @@
 
 namespace tsdp {
 
-constexpr int XF_THREADS = 128;
+constexpr int XF_THREADS = 256;
+constexpr int XF_WARPS = XF_THREADS / 32;
 constexpr int XF_MAXN = 32;          // (1 + obs_tokens) * heads at most
 constexpr int XF_MAXNK = 4;          // 1 + obs_tokens at most
 constexpr int XF_RB = 4;             // memory tokens per pass of the table builder
@@ -128,27 +129,53 @@ xfold_build_kernel(const float* __restrict__ kv, long long ldkv, int rows, const
   }
 }
 
-__device__ __forceinline__ uint32_t xf_ldg32(const __nv_bfloat16* p) { return __ldg(reinterpret_cast<const unsigned int*>(p)); }
+__device__ __forceinline__ void xf_cp16(void* smem_dst, const void* gsrc) {
+  const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void xf_cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void xf_cp_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// One block per candidate (H <= 16 token rows of width D), 4 warps.
-//   1  xhat = LayerNorm without affine of the candidate's rows, bf16, into shared memory (warp w: rows 4w..4w+3)
-//   2  partial scores of warp w over its quarter of the D input columns, summed through shared memory
+// Shared memory of one block: xhat [16][D+8] bf16 | kq rows [NKH][D+8] bf16, later the warps' output tiles
+// [warps][16][D/16+8] fp32 | u rows [NKH/2][D+8] words | partial scores [4][16][32] fp32 | P [16][40] bf16.
+__host__ __device__ constexpr size_t xf_region_bytes(int D, int nkh) {
+  const size_t k = (size_t)nkh * (D + 8) * 2, t = (size_t)XF_WARPS * 16 * (D / (2 * XF_WARPS) + 8) * 4;
+  return k > t ? k : t;
+}
+__host__ __device__ constexpr size_t xf_smem_bytes(int D, int nkh) {
+  return (size_t)16 * (D + 8) * 2 + xf_region_bytes(D, nkh) + (size_t)(nkh / 2) * (D + 8) * 4 + (size_t)4 * 16 * XF_MAXN * 4 +
+         (size_t)16 * (XF_MAXN + 8) * 2;
+}
+
+// One block per candidate (H <= 16 token rows of width D), 8 warps.
+//   0  the candidate's kq and u rows start their way into shared memory (cp.async, 16 bytes per lane: a
+//      lane-by-lane gather of tensor-core fragments from global memory is bound by the L1 tag rate)
+//   1  xhat = LayerNorm without affine of the candidate's rows, bf16, into shared memory (warp w: rows 2w, 2w+1)
+//   2  partial scores: warp w covers a quarter of the D input columns for two of the 8-wide score tiles
 //   3  softmax over the memory tokens per (row, head) -> P [16 x 32] bf16
-//   4  warp w: output columns [w D/4, (w+1) D/4) = P . U, + bo2, added to the residual stream in place
-// Every phase issues all of its global loads before it uses the first of them: a block is a chain of a
-// few memory round trips, and with four warps nothing else would hide them.
+//   4  warp w: output columns [w D/8, (w+1) D/8) = P . U + bo2, staged through shared memory so that the
+//      residual stream is read and written in full 16-byte lanes along its rows, in place
 template <int D>
-__global__ void __launch_bounds__(XF_THREADS)
+__global__ void __launch_bounds__(XF_THREADS, 3)
 xattn_fold_kernel(float* __restrict__ x, XfoldTables tb, const float* __restrict__ bo2, CandMap cm, int H, int heads,
                   int To, int layer, int L, int Tsteps) {
   pdl_trigger();
   pdl_wait();
-  constexpr int LDA = D + 8;
+  constexpr int LDA = D + 8;               // bf16 elements per row of xhat and of the kq rows
+  constexpr int LDU = D + 8;               // words per row of the u rows
   constexpr int LDP = XF_MAXN + 8;
   constexpr int V = D / 128;
-  __shared__ __align__(16) __nv_bfloat16 sA[16 * LDA];
-  __shared__ float sS[4][16][XF_MAXN];
-  __shared__ __align__(16) __nv_bfloat16 sP[16 * LDP];
+  constexpr int HW = D / (2 * XF_WARPS);   // output columns of a warp per half
+  constexpr int LDT = HW + 8;
+  extern __shared__ __align__(16) unsigned char xf_smem[];
+  const int NK = 1 + To, NKH = NK * heads;
+  __nv_bfloat16* sA = reinterpret_cast<__nv_bfloat16*>(xf_smem);
+  unsigned char* region = xf_smem + (size_t)16 * LDA * 2;
+  __nv_bfloat16* sK = reinterpret_cast<__nv_bfloat16*>(region);
+  uint32_t* sU = reinterpret_cast<uint32_t*>(region + xf_region_bytes(D, NKH));
+  float* sS = reinterpret_cast<float*>(sU + (size_t)(NKH / 2) * LDU);      // [4][16][XF_MAXN]
+  __nv_bfloat16* sP = reinterpret_cast<__nv_bfloat16*>(sS + 4 * 16 * XF_MAXN);
   const int n = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, tg = lane & 3;
@@ -156,25 +183,47 @@ xattn_fold_kernel(float* __restrict__ x, XfoldTables tb, const float* __restrict
   int tau = cm.t[b] - cm.koff - cnd;
   tau = max(0, min(Tsteps - 1, tau));
   const int item = item_of(cm.item, b);
-  const int NK = 1 + To, NKH = NK * heads;
   const size_t tok_stride = (size_t)L * heads * D;      // kq / ut elements per memory token
   const size_t lay_off = (size_t)layer * heads * D;
   float* xc = x + (size_t)n * H * D;
 
+  // ---- 0: tables of this candidate's memory tokens, one row per warp at a time
+  {
+    const int hp = heads >> 1;
+    for (int row = warp; row < NKH; row += XF_WARPS) {
+      const int jt = row / heads, h = row - jt * heads;
+      const __nv_bfloat16* sr = (jt == 0 ? tb.kq_time + (size_t)tau * tok_stride : tb.kq_obs + ((size_t)item * To + (jt - 1)) * tok_stride) +
+                                lay_off + (size_t)h * D;
+      __nv_bfloat16* dr = sK + (size_t)row * LDA;
+#pragma unroll
+      for (int ch = 0; ch < D / 256; ++ch) xf_cp16(dr + (ch * 32 + lane) * 8, sr + (ch * 32 + lane) * 8);
+      if (D % 256 && lane < (D % 256) / 8) xf_cp16(dr + (D / 256 * 32 + lane) * 8, sr + (D / 256 * 32 + lane) * 8);
+    }
+    xf_cp_commit();
+    for (int row = warp; row < NKH / 2; row += XF_WARPS) {
+      const int jt = row / hp, q = row - jt * hp;
+      const __nv_bfloat16* sr = (jt == 0 ? tb.ut_time + (size_t)tau * tok_stride : tb.ut_obs + ((size_t)item * To + (jt - 1)) * tok_stride) +
+                                lay_off + (size_t)q * D * 2;
+      uint32_t* dr = sU + (size_t)row * LDU;
+#pragma unroll
+      for (int ch = 0; ch < D / 128; ++ch) xf_cp16(dr + (ch * 32 + lane) * 4, sr + (ch * 32 + lane) * 8);
+    }
+    xf_cp_commit();
+  }
+
   // ---- 1: LayerNorm statistics, normalised rows to shared memory
   for (int i = threadIdx.x; i < 16 * LDP / 2; i += XF_THREADS) reinterpret_cast<uint32_t*>(sP)[i] = 0u;
-#pragma unroll 1
-  for (int rb = 0; rb < 4; rb += 2) {          // two rows per pass: all of their loads are in flight together
+  {                                            // two rows per warp: all of their loads are in flight together
     float4 v[2][V];
 #pragma unroll
     for (int rr = 0; rr < 2; ++rr) {
-      const int r = min(4 * warp + rb + rr, H - 1);
+      const int r = min(2 * warp + rr, H - 1);
 #pragma unroll
       for (int j = 0; j < V; ++j) v[rr][j] = reinterpret_cast<const float4*>(xc + (size_t)r * D)[j * 32 + lane];
     }
 #pragma unroll
     for (int rr = 0; rr < 2; ++rr) {
-      const int r = 4 * warp + rb + rr;
+      const int r = 2 * warp + rr;
       float s = 0.f;
 #pragma unroll
       for (int j = 0; j < V; ++j) s += v[rr][j].x + v[rr][j].y + v[rr][j].z + v[rr][j].w;
@@ -196,56 +245,49 @@ xattn_fold_kernel(float* __restrict__ x, XfoldTables tb, const float* __restrict
       }
     }
   }
+  xf_cp_wait<1>();                             // this thread's kq chunks have landed
   __syncthreads();
 
-  // ---- 2: scores, k steps [warp * D/64, (warp + 1) * D/64)
+  // ---- 2: scores.  Warp w takes quarter (w & 3) of the D input columns and the score tiles 2 (w >> 2), 2 (w >> 2) + 1;
+  //         the four partial sums of a score are added in a fixed order in phase 3 (no atomics: same bits every run)
   {
-    const __nv_bfloat16* pk[4];
-    uint32_t live[4];
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-      const int nn = min(8 * nt + g, NKH - 1);            // lanes past the last (token, head) read a valid row, masked below
-      live[nt] = 8 * nt + g < NKH ? 0xffffffffu : 0u;
-      const int j = nn / heads, h = nn % heads;
-      pk[nt] = (j == 0 ? tb.kq_time + (size_t)tau * tok_stride : tb.kq_obs + ((size_t)item * To + (j - 1)) * tok_stride) + lay_off +
-               (size_t)h * D + (size_t)warp * (D / 4) + 2 * tg;
-    }
-    float sc[4][4];
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt) { sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f; }
     constexpr int KSW = D / 64;
-    constexpr int KB = KSW < 4 ? KSW : 4;
+    const int kq4 = warp & 3, nh = warp >> 2;
+    const __nv_bfloat16* pk[2];
+    uint32_t live[2];
 #pragma unroll
-    for (int kb = 0; kb < KSW; kb += KB) {
-      uint32_t bq[KB][4][2];
+    for (int u = 0; u < 2; ++u) {
+      const int nt = 2 * nh + u;
+      live[u] = 8 * nt + g < NKH ? 0xffffffffu : 0u;           // rows past the last (token, head) read row NKH-1, masked
+      pk[u] = sK + (size_t)min(8 * nt + g, NKH - 1) * LDA + kq4 * (D / 4) + 2 * tg;
+    }
+    float sc[2][4];
 #pragma unroll
-      for (int kk = 0; kk < KB; ++kk)
+    for (int u = 0; u < 2; ++u) { sc[u][0] = sc[u][1] = sc[u][2] = sc[u][3] = 0.f; }
+    if (16 * nh < NKH) {
 #pragma unroll
-        for (int nt = 0; nt < 4; ++nt) {
-          if (8 * nt < NKH) {
-            const __nv_bfloat16* p = pk[nt] + (kb + kk) * 16;
-            bq[kk][nt][0] = xf_ldg32(p);
-            bq[kk][nt][1] = xf_ldg32(p + 8);
-          }
-        }
-#pragma unroll
-      for (int kk = 0; kk < KB; ++kk) {
-        const int ks = warp * KSW + kb + kk;
+      for (int kk = 0; kk < KSW; ++kk) {
         uint32_t a[4];
-        const __nv_bfloat16* ar = sA + g * LDA + ks * 16 + 2 * tg;
+        const __nv_bfloat16* ar = sA + g * LDA + (kq4 * KSW + kk) * 16 + 2 * tg;
         a[0] = *reinterpret_cast<const uint32_t*>(ar);
         a[1] = *reinterpret_cast<const uint32_t*>(ar + 8 * LDA);
         a[2] = *reinterpret_cast<const uint32_t*>(ar + 8);
         a[3] = *reinterpret_cast<const uint32_t*>(ar + 8 * LDA + 8);
 #pragma unroll
-        for (int nt = 0; nt < 4; ++nt)
-          if (8 * nt < NKH) mma_bf16_16816(sc[nt], a, bq[kk][nt][0] & live[nt], bq[kk][nt][1] & live[nt]);
+        for (int u = 0; u < 2; ++u) {
+          if (8 * (2 * nh + u) < NKH) {
+            const uint32_t b0 = *reinterpret_cast<const uint32_t*>(pk[u] + kk * 16) & live[u];
+            const uint32_t b1 = *reinterpret_cast<const uint32_t*>(pk[u] + kk * 16 + 8) & live[u];
+            mma_bf16_16816(sc[u], a, b0, b1);
+          }
+        }
       }
     }
 #pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-      sS[warp][g][8 * nt + 2 * tg] = sc[nt][0]; sS[warp][g][8 * nt + 2 * tg + 1] = sc[nt][1];
-      sS[warp][g + 8][8 * nt + 2 * tg] = sc[nt][2]; sS[warp][g + 8][8 * nt + 2 * tg + 1] = sc[nt][3];
+    for (int u = 0; u < 2; ++u) {
+      float* s0 = sS + ((size_t)kq4 * 16 + g) * XF_MAXN + 8 * (2 * nh + u) + 2 * tg;
+      s0[0] = sc[u][0]; s0[1] = sc[u][1];
+      s0[8 * XF_MAXN] = sc[u][2]; s0[8 * XF_MAXN + 1] = sc[u][3];
     }
   }
   __syncthreads();
@@ -267,7 +309,8 @@ xattn_fold_kernel(float* __restrict__ x, XfoldTables tb, const float* __restrict
     for (int j = 0; j < XF_MAXNK; ++j) {
       if (j < NK) {
         const int nn = j * heads + h;
-        s[j] += sS[0][r][nn] + sS[1][r][nn] + sS[2][r][nn] + sS[3][r][nn];
+        s[j] += ((sS[(0 * 16 + r) * XF_MAXN + nn] + sS[(1 * 16 + r) * XF_MAXN + nn]) + sS[(2 * 16 + r) * XF_MAXN + nn]) +
+                sS[(3 * 16 + r) * XF_MAXN + nn];
         m = fmaxf(m, s[j]);
       }
     }
@@ -280,9 +323,10 @@ xattn_fold_kernel(float* __restrict__ x, XfoldTables tb, const float* __restrict
     for (int j = 0; j < XF_MAXNK; ++j)
       if (j < NK) sP[r * LDP + j * heads + h] = __float2bfloat16_rn(s[j] * inv);
   }
-  __syncthreads();
+  xf_cp_wait<0>();                             // this thread's u chunks have landed
+  __syncthreads();                             // also: every warp is done with the kq rows, whose memory the tiles reuse
 
-  // ---- 4: P . U + bo2 into the residual stream, four 8-column tiles at a time
+  // ---- 4: P . U + bo2 into the residual stream
   {
     uint32_t pa[2][4];
 #pragma unroll
@@ -293,52 +337,52 @@ xattn_fold_kernel(float* __restrict__ x, XfoldTables tb, const float* __restrict
       pa[k2][2] = *reinterpret_cast<const uint32_t*>(ar + 8);
       pa[k2][3] = *reinterpret_cast<const uint32_t*>(ar + 8 * LDP + 8);
     }
-    const __nv_bfloat16* pu[2][2];
+    // B fragment (k2, rg) of a lane: memory-token/head pair row 8 k2 + 4 rg + tg of the u rows
+    const uint32_t* pu[2][2];
     uint32_t ulive[2][2];
 #pragma unroll
     for (int k2 = 0; k2 < 2; ++k2)
 #pragma unroll
       for (int rg = 0; rg < 2; ++rg) {
-        const int n0 = 16 * k2 + 8 * rg + 2 * tg;
-        ulive[k2][rg] = n0 < NKH ? 0xffffffffu : 0u;
-        const int nn = min(n0, NKH - 2);
-        const int j = nn / heads, h = nn % heads;
-        pu[k2][rg] = (j == 0 ? tb.ut_time + (size_t)tau * tok_stride : tb.ut_obs + ((size_t)item * To + (j - 1)) * tok_stride) + lay_off +
-                     ((size_t)(h >> 1) * D + g) * 2;
+        const int pr = 8 * k2 + 4 * rg + tg;
+        ulive[k2][rg] = 2 * pr < NKH ? 0xffffffffu : 0u;
+        pu[k2][rg] = sU + (size_t)min(pr, NKH / 2 - 1) * LDU + g;
       }
-    const bool row0 = g < H, row1 = g + 8 < H;
-    float* x0 = xc + (size_t)(row0 ? g : 0) * D;
-    float* x1 = xc + (size_t)(row1 ? g + 8 : 0) * D;
-    constexpr int NTB = 4;
+    float* tile = reinterpret_cast<float*>(region) + (size_t)warp * 16 * LDT;
+    constexpr int LPR = HW / 4;              // lanes per tile row in the row-wise pass
+    constexpr int RPI = 32 / LPR;            // rows per instruction
+    constexpr int NI = 16 / RPI;
+    const int rr0 = lane / LPR, c4 = (lane % LPR) * 4;
 #pragma unroll 1
-    for (int o_base = warp * (D / 4); o_base < (warp + 1) * (D / 4); o_base += 8 * NTB) {
-      uint32_t bu[NTB][2][2];
-      float2 xv[NTB][2], bb[NTB];
+    for (int half = 0; half < 2; ++half) {
+      const int o_base = warp * (D / XF_WARPS) + half * HW;
+      float4 xv[NI];
 #pragma unroll
-      for (int nt = 0; nt < NTB; ++nt) {
-        const int o = (o_base + 8 * nt) * 2;
-#pragma unroll
-        for (int k2 = 0; k2 < 2; ++k2) {
-          if (16 * k2 < NKH) {
-            bu[nt][k2][0] = xf_ldg32(pu[k2][0] + o);
-            bu[nt][k2][1] = xf_ldg32(pu[k2][1] + o);
-          }
-        }
-        const int col = o_base + 8 * nt + 2 * tg;
-        xv[nt][0] = *reinterpret_cast<const float2*>(x0 + col);
-        xv[nt][1] = *reinterpret_cast<const float2*>(x1 + col);
-        bb[nt] = __ldg(reinterpret_cast<const float2*>(bo2 + col));
+      for (int i = 0; i < NI; ++i) {
+        const int r = min(i * RPI + rr0, H - 1);
+        xv[i] = *reinterpret_cast<const float4*>(xc + (size_t)r * D + o_base + c4);
       }
+      const float4 bb = __ldg(reinterpret_cast<const float4*>(bo2 + o_base + c4));
 #pragma unroll
-      for (int nt = 0; nt < NTB; ++nt) {
+      for (int nt = 0; nt < HW / 8; ++nt) {
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int k2 = 0; k2 < 2; ++k2)
-          if (16 * k2 < NKH) mma_bf16_16816(acc, pa[k2], bu[nt][k2][0] & ulive[k2][0], bu[nt][k2][1] & ulive[k2][1]);
-        const int col = o_base + 8 * nt + 2 * tg;
-        if (row0) *reinterpret_cast<float2*>(x0 + col) = make_float2(xv[nt][0].x + acc[0] + bb[nt].x, xv[nt][0].y + acc[1] + bb[nt].y);
-        if (row1) *reinterpret_cast<float2*>(x1 + col) = make_float2(xv[nt][1].x + acc[2] + bb[nt].x, xv[nt][1].y + acc[3] + bb[nt].y);
+          if (16 * k2 < NKH)
+            mma_bf16_16816(acc, pa[k2], pu[k2][0][o_base + 8 * nt] & ulive[k2][0], pu[k2][1][o_base + 8 * nt] & ulive[k2][1]);
+        *reinterpret_cast<float2*>(tile + g * LDT + 8 * nt + 2 * tg) = make_float2(acc[0], acc[1]);
+        *reinterpret_cast<float2*>(tile + (g + 8) * LDT + 8 * nt + 2 * tg) = make_float2(acc[2], acc[3]);
       }
+      __syncwarp();
+#pragma unroll
+      for (int i = 0; i < NI; ++i) {
+        const int r = i * RPI + rr0;
+        const float4 t = *reinterpret_cast<const float4*>(tile + r * LDT + c4);
+        if (r < H)
+          *reinterpret_cast<float4*>(xc + (size_t)r * D + o_base + c4) =
+              make_float4(xv[i].x + t.x + bb.x, xv[i].y + t.y + bb.y, xv[i].z + t.z + bb.z, xv[i].w + t.w + bb.w);
+      }
+      __syncwarp();
     }
   }
 }

@@ -540,11 +540,12 @@ int xfold_build(tsdp_ctx* c, Net& n, const float* kv, int rows, __nv_bfloat16* k
   return TSDP_OK;
 }
 
-int xattn_fold_launch(tsdp_ctx* c, const Net& n, const float* bo2, const CandMap& cm, int n_cand, int layer, cudaStream_t s) {
+int xattn_fold_launch(tsdp_ctx* c, const Net& n, const XfmrLayer& w, const __nv_bfloat16* delta, __nv_bfloat16* ln3_out,
+                      const CandMap& cm, int n_cand, int layer, cudaStream_t s) {
   const int H = c->cfg.H, d = n.cfg.d, heads = n.cfg.heads, L = n.cfg.layers, To = c->cfg.obs_tokens;
   const XfoldTables tb{n.fold_kq_time, n.fold_ut_time, n.fold_c_time, n.fold_kq_obs, n.fold_ut_obs, n.fold_c_obs};
   prof_begin(c, s, 2, 0.0);
-#define XF_CASE(DD) TSDP_LAUNCH(c, (xattn_fold_kernel<DD>), n_cand, XF_THREADS, xf_smem_bytes(DD, (1 + To) * heads), s, c->h, tb, bo2, cm, H, heads, To, layer, L, c->cfg.T)
+#define XF_CASE(DD) TSDP_LAUNCH(c, (xattn_fold_kernel<DD>), n_cand, XF_THREADS, xf_smem_bytes(DD, (1 + To) * heads), s, c->h, delta, tb, w.bo2, w.ln3_g, w.ln3_b, ln3_out, cm, H, heads, To, layer, L, c->cfg.T)
   switch (d) {
     case 128: XF_CASE(128); break;
     case 256: XF_CASE(256); break;
@@ -578,16 +579,20 @@ int xfmr_forward_t(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStrea
     if ((r = ln_launch<T>(c, c->h, w.ln1_g, w.ln1_b, a, M, d, s))) return r;
     if ((r = gemm(c, a, w.Wqkv, w.bqkv, M, 3 * d, d, out_epi, qkv, 3 * d, s))) return r;
     if ((r = self_attn_launch<T>(c, qkv, a, n_cand, H, d, heads, s))) return r;
-    if ((r = gemm(c, a, w.Wo, w.bo, M, d, d, EPI_RESID, c->h, d, s))) return r;
     if (n.fold) {
-      if ((r = xattn_fold_launch(c, n, w.bo2, cm, n_cand, l, s))) return r;
+      // the attention projection leaves as bf16; the fold kernel adds it to the stream, does the cross-attention
+      // sub-block and the LayerNorm in front of the MLP
+      if ((r = gemm(c, a, w.Wo, w.bo, M, d, d, EPI_STORE, q2, d, s))) return r;
+      if ((r = xattn_fold_launch(c, n, w, reinterpret_cast<const __nv_bfloat16*>(q2), reinterpret_cast<__nv_bfloat16*>(a), cm, n_cand, l, s)))
+        return r;
     } else {
+      if ((r = gemm(c, a, w.Wo, w.bo, M, d, d, EPI_RESID, c->h, d, s))) return r;
       if ((r = ln_launch<T>(c, c->h, w.ln2_g, w.ln2_b, a, M, d, s))) return r;
       if ((r = gemm(c, a, w.Wq2, w.bq2, M, d, d, out_epi, q2, d, s))) return r;
       if ((r = cross_attn_launch<T>(c, n, q2, a, cm, n_cand, l, s))) return r;
       if ((r = gemm(c, a, w.Wo2, w.bo2, M, d, d, EPI_RESID, c->h, d, s))) return r;
+      if ((r = ln_launch<T>(c, c->h, w.ln3_g, w.ln3_b, a, M, d, s))) return r;
     }
-    if ((r = ln_launch<T>(c, c->h, w.ln3_g, w.ln3_b, a, M, d, s))) return r;
     if ((r = gemm(c, a, w.W1, w.b1, M, 4 * d, d, EPI_GELU, f, 4 * d, s))) return r;
     if ((r = gemm(c, f, w.W2, w.b2, M, d, 4 * d, EPI_RESID, c->h, d, s))) return r;
   }

@@ -133,6 +133,11 @@ __device__ __forceinline__ void xf_cp16(void* smem_dst, const void* gsrc) {
   const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
 }
+__device__ __forceinline__ void xf_add_bf16x4(float4& a, const uint2 d) {
+  const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&d.x));
+  const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&d.y));
+  a.x += lo.x; a.y += lo.y; a.z += hi.x; a.w += hi.y;
+}
 __device__ __forceinline__ void xf_cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void xf_cp_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
@@ -156,10 +161,15 @@ __host__ __device__ constexpr size_t xf_smem_bytes(int D, int nkh) {
 //   3  softmax over the memory tokens per (row, head) -> P [16 x 32] bf16
 //   4  warp w: output columns [w D/8, (w+1) D/8) = P . U + bo2, staged through shared memory so that the
 //      residual stream is read and written in full 16-byte lanes along its rows, in place
+//   5  the LayerNorm in front of the MLP, from the updated rows still in registers -> ln3_out (bf16)
+// `delta` is the output of the self-attention projection (bf16, bias included), which this kernel adds to the
+// residual stream before anything else: that GEMM then writes 2 bytes per element instead of doing an fp32
+// read-modify-write of the stream.
 template <int D>
 __global__ void __launch_bounds__(XF_THREADS, 3)
-xattn_fold_kernel(float* __restrict__ x, XfoldTables tb, const float* __restrict__ bo2, CandMap cm, int H, int heads,
-                  int To, int layer, int L, int Tsteps) {
+xattn_fold_kernel(float* __restrict__ x, const __nv_bfloat16* __restrict__ delta, XfoldTables tb, const float* __restrict__ bo2,
+                  const float* __restrict__ ln3_g, const float* __restrict__ ln3_b, __nv_bfloat16* __restrict__ ln3_out, CandMap cm,
+                  int H, int heads, int To, int layer, int L, int Tsteps) {
   pdl_trigger();
   pdl_wait();
   constexpr int LDA = D + 8;               // bf16 elements per row of xhat and of the kq rows
@@ -186,6 +196,7 @@ xattn_fold_kernel(float* __restrict__ x, XfoldTables tb, const float* __restrict
   const size_t tok_stride = (size_t)L * heads * D;      // kq / ut elements per memory token
   const size_t lay_off = (size_t)layer * heads * D;
   float* xc = x + (size_t)n * H * D;
+  const __nv_bfloat16* dc = delta + (size_t)n * H * D;
 
   // ---- 0: tables of this candidate's memory tokens, one row per warp at a time
   {
@@ -221,6 +232,17 @@ xattn_fold_kernel(float* __restrict__ x, XfoldTables tb, const float* __restrict
 #pragma unroll
       for (int j = 0; j < V; ++j) v[rr][j] = reinterpret_cast<const float4*>(xc + (size_t)r * D)[j * 32 + lane];
     }
+    uint2 dv[2][V];
+#pragma unroll
+    for (int rr = 0; rr < 2; ++rr) {
+      const int r = min(2 * warp + rr, H - 1);
+#pragma unroll
+      for (int j = 0; j < V; ++j) dv[rr][j] = reinterpret_cast<const uint2*>(dc + (size_t)r * D)[j * 32 + lane];
+    }
+#pragma unroll
+    for (int rr = 0; rr < 2; ++rr)
+#pragma unroll
+      for (int j = 0; j < V; ++j) xf_add_bf16x4(v[rr][j], dv[rr][j]);
 #pragma unroll
     for (int rr = 0; rr < 2; ++rr) {
       const int r = 2 * warp + rr;
@@ -353,14 +375,16 @@ xattn_fold_kernel(float* __restrict__ x, XfoldTables tb, const float* __restrict
     constexpr int RPI = 32 / LPR;            // rows per instruction
     constexpr int NI = 16 / RPI;
     const int rr0 = lane / LPR, c4 = (lane % LPR) * 4;
-#pragma unroll 1
+    float4 xn[2][NI];                        // the updated rows of this lane, kept for the LayerNorm that follows
+#pragma unroll
     for (int half = 0; half < 2; ++half) {
       const int o_base = warp * (D / XF_WARPS) + half * HW;
-      float4 xv[NI];
+      uint2 dl[NI];
 #pragma unroll
       for (int i = 0; i < NI; ++i) {
         const int r = min(i * RPI + rr0, H - 1);
-        xv[i] = *reinterpret_cast<const float4*>(xc + (size_t)r * D + o_base + c4);
+        xn[half][i] = *reinterpret_cast<const float4*>(xc + (size_t)r * D + o_base + c4);
+        dl[i] = *reinterpret_cast<const uint2*>(dc + (size_t)r * D + o_base + c4);
       }
       const float4 bb = __ldg(reinterpret_cast<const float4*>(bo2 + o_base + c4));
 #pragma unroll
@@ -378,11 +402,59 @@ xattn_fold_kernel(float* __restrict__ x, XfoldTables tb, const float* __restrict
       for (int i = 0; i < NI; ++i) {
         const int r = i * RPI + rr0;
         const float4 t = *reinterpret_cast<const float4*>(tile + r * LDT + c4);
-        if (r < H)
-          *reinterpret_cast<float4*>(xc + (size_t)r * D + o_base + c4) =
-              make_float4(xv[i].x + t.x + bb.x, xv[i].y + t.y + bb.y, xv[i].z + t.z + bb.z, xv[i].w + t.w + bb.w);
+        xf_add_bf16x4(xn[half][i], dl[i]);
+        xn[half][i].x += t.x + bb.x; xn[half][i].y += t.y + bb.y; xn[half][i].z += t.z + bb.z; xn[half][i].w += t.w + bb.w;
+        if (r < H) *reinterpret_cast<float4*>(xc + (size_t)r * D + o_base + c4) = xn[half][i];
       }
       __syncwarp();
+    }
+
+    // ---- 5: LayerNorm of the updated rows (the block's third LayerNorm), bf16, for the MLP that follows.
+    //         Row r's D values sit in LPR lanes of each of the 8 warps: lane group -> warp partial -> block.
+    float* part = sS;                          // [XF_WARPS][16] partial sums, then [16] means / rstds behind them
+    float* stat = sS + XF_WARPS * 16;
+#pragma unroll
+    for (int pass = 0; pass < 2; ++pass) {
+#pragma unroll
+      for (int i = 0; i < NI; ++i) {
+        const int r = i * RPI + rr0;
+        float a = 0.f;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const float4 e = xn[half][i];
+          if (pass == 0) a += (e.x + e.y) + (e.z + e.w);
+          else { const float m = stat[r]; a += (e.x - m) * (e.x - m) + (e.y - m) * (e.y - m) + (e.z - m) * (e.z - m) + (e.w - m) * (e.w - m); }
+        }
+#pragma unroll
+        for (int o = LPR / 2; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        if (lane % LPR == 0) part[warp * 16 + r] = a;
+      }
+      __syncthreads();
+      if (threadIdx.x < 16) {
+        float a = 0.f;
+#pragma unroll
+        for (int w = 0; w < XF_WARPS; ++w) a += part[w * 16 + threadIdx.x];
+        stat[pass * 16 + threadIdx.x] = pass == 0 ? a / D : rsqrtf(a / D + 1e-5f);
+      }
+      __syncthreads();
+    }
+    __nv_bfloat16* oc = ln3_out + (size_t)n * H * D;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const int col = warp * (D / XF_WARPS) + half * HW + c4;
+      const float4 gg = __ldg(reinterpret_cast<const float4*>(ln3_g + col)), be = __ldg(reinterpret_cast<const float4*>(ln3_b + col));
+#pragma unroll
+      for (int i = 0; i < NI; ++i) {
+        const int r = i * RPI + rr0;
+        if (r < H) {
+          const float m = stat[r], rs = stat[16 + r];
+          const float4 e = xn[half][i];
+          uint2 o2;
+          o2.x = pack_bf16((e.x - m) * rs * gg.x + be.x, (e.y - m) * rs * gg.y + be.y);
+          o2.y = pack_bf16((e.z - m) * rs * gg.z + be.z, (e.w - m) * rs * gg.w + be.w);
+          *reinterpret_cast<uint2*>(oc + (size_t)r * D + col) = o2;
+        }
+      }
     }
   }
 }

@@ -6,7 +6,8 @@ Every linear layer of one transformer block of the base model is timed on M = ba
 rows: `reps` launches back to back between one pair of CUDA events (tsdp_gemm_timed).  Operands of
 consecutive launches are the same, so whatever fits the L2 stays there, as it does inside the forward
 pass where each operand was written by the previous kernel.  Prints one line per shape and one JSON
-line with the flop-weighted total.
+line with the flop-weighted total (and the total without q_cross / cross_out: the decoder transformer
+folds those two projections into its memory tokens and launches only the other four).
 """
 import argparse
 import json
@@ -51,8 +52,11 @@ def main():
         tot_ms += ms; tot_flop += flop
         print(f"{name:10s} M={M:6d} N={N:5d} K={Kd:5d} epi={epi}  {1e3 * ms:8.1f} us  {flop / ms / 1e9:7.1f} TFLOP/s"
               f"  {io / ms / 1e6:7.0f} GB/s (A + W + out bytes)")
+    four = [r for r in rows if r["name"] not in ("q_cross", "cross_out")]
+    us4 = sum(r["us"] for r in four)
     print(json.dumps(dict(workload=args.workload, batch=B, K=K, rows=M, block_us=1e3 * tot_ms,
-                          block_tflops=tot_flop / tot_ms / 1e9, shapes=rows)))
+                          block_tflops=tot_flop / tot_ms / 1e9, folded_block_us=us4,
+                          folded_block_tflops=sum(2.0 * r["M"] * r["N"] * r["K"] for r in four) / us4 / 1e6, shapes=rows)))
     smp.close()
 
 

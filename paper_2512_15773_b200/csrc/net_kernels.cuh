@@ -403,6 +403,132 @@ self_attn_mma_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __res
 }
 
 // ------------------------------------------------------------------------------------------------
+// Self-attention for sequences of at most 16 tokens, bf16: one warp per (candidate, head).  The warp
+// copies the head's Q, K and V rows into its own piece of shared memory with 16-byte loads (a
+// lane-by-lane gather of fragments from global memory costs one L1 tag look-up per 16 bytes) and takes
+// the mma operands from there: Q with 4-byte loads, K through ldmatrix, V through ldmatrix.trans.
+// ------------------------------------------------------------------------------------------------
+template <int DH>
+__global__ void __launch_bounds__((DH > 64 ? 2 : 4) * 32)
+self_attn_tile_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ out, int n_cand, int H, int d,
+                      int heads, int causal) {
+  pdl_trigger();
+  pdl_wait();
+  constexpr int TW = DH > 64 ? 2 : 4;
+  constexpr int KS = DH / 16, NO = DH / 8, P = DH + 8, VPR = DH / 8;
+  __shared__ __align__(16) __nv_bfloat16 sm[TW][3][16 * P];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, tg = lane & 3;
+  const int wg = blockIdx.x * TW + warp;
+  if (wg >= n_cand * heads) return;
+  const int hd = wg % heads, n = wg / heads;
+  const size_t ld = (size_t)3 * d;
+  const __nv_bfloat16* base = qkv + (size_t)n * H * ld + (size_t)hd * DH;
+  __nv_bfloat16* sQ = sm[warp][0];
+  __nv_bfloat16* sK = sm[warp][1];
+  __nv_bfloat16* sV = sm[warp][2];
+  constexpr int NV = 3 * 16 * VPR / 32;          // 16-byte vectors per lane
+  constexpr int CH = NV > 12 ? NV / 2 : NV;      // in flight at a time
+#pragma unroll
+  for (int c0 = 0; c0 < NV; c0 += CH) {
+    uint4 buf[CH];
+#pragma unroll
+    for (int i = 0; i < CH; ++i) {
+      const int idx = (c0 + i) * 32 + lane;
+      const int which = idx / (16 * VPR), rem = idx % (16 * VPR), r = rem / VPR, v = rem % VPR;
+      buf[i] = r < H ? __ldg(reinterpret_cast<const uint4*>(base + (size_t)r * ld + (size_t)which * d) + v) : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int i = 0; i < CH; ++i) {
+      const int idx = (c0 + i) * 32 + lane;
+      const int which = idx / (16 * VPR), rem = idx % (16 * VPR), r = rem / VPR, v = rem % VPR;
+      *reinterpret_cast<uint4*>(sm[warp][which] + r * P + v * 8) = buf[i];
+    }
+  }
+  __syncwarp();
+  uint32_t qa[KS][4];
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks) {
+    const __nv_bfloat16* q0 = sQ + g * P + ks * 16 + 2 * tg;
+    qa[ks][0] = *reinterpret_cast<const uint32_t*>(q0);
+    qa[ks][1] = *reinterpret_cast<const uint32_t*>(q0 + 8 * P);
+    qa[ks][2] = *reinterpret_cast<const uint32_t*>(q0 + 8);
+    qa[ks][3] = *reinterpret_cast<const uint32_t*>(q0 + 8 * P + 8);
+  }
+  const int nkt = causal ? 2 : (H + 7) >> 3;
+  float s[2][4];
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+    s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+    if (nt < nkt) {
+#pragma unroll
+      for (int ks = 0; ks < KS; ks += 2) {
+        uint32_t b[4];
+        ldmatrix_x4(b, sK + (nt * 8 + (lane & 7)) * P + ks * 16 + 8 * (lane >> 3));
+        mma_bf16_16816(s[nt], qa[ks], b[0], b[1]);
+        mma_bf16_16816(s[nt], qa[ks + 1], b[2], b[3]);
+      }
+    }
+  }
+  const float scale = rsqrtf((float)DH);
+  const int r0 = g, r1 = g + 8;
+  float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+    if (nt < nkt) {
+      const int col = nt * 8 + 2 * tg;
+      const int lim0 = causal ? r0 : H, lim1 = causal ? r1 : H;
+      s[nt][0] = (col <= lim0 && col < H) ? s[nt][0] * scale : -INFINITY;
+      s[nt][1] = (col + 1 <= lim0 && col + 1 < H) ? s[nt][1] * scale : -INFINITY;
+      s[nt][2] = (col <= lim1 && col < H) ? s[nt][2] * scale : -INFINITY;
+      s[nt][3] = (col + 1 <= lim1 && col + 1 < H) ? s[nt][3] * scale : -INFINITY;
+      m0 = fmaxf(m0, fmaxf(s[nt][0], s[nt][1]));
+      m1 = fmaxf(m1, fmaxf(s[nt][2], s[nt][3]));
+    }
+  }
+  m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 1)); m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 2));
+  m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 1)); m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 2));
+  // rows beyond H have no visible key: keep the arithmetic finite, their output is never stored
+  if (m0 == -INFINITY) m0 = 0.f;
+  if (m1 == -INFINITY) m1 = 0.f;
+  float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+    if (nt < nkt) {
+      s[nt][0] = __expf(s[nt][0] - m0); s[nt][1] = __expf(s[nt][1] - m0);
+      s[nt][2] = __expf(s[nt][2] - m1); s[nt][3] = __expf(s[nt][3] - m1);
+      l0 += s[nt][0] + s[nt][1]; l1 += s[nt][2] + s[nt][3];
+    }
+  }
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+  l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+  const float inv0 = l0 > 0.f ? 1.0f / l0 : 0.f, inv1 = l1 > 0.f ? 1.0f / l1 : 0.f;
+  uint32_t pa[4];
+  pa[0] = pack_bf16(s[0][0], s[0][1]); pa[1] = pack_bf16(s[0][2], s[0][3]);
+  pa[2] = pack_bf16(s[1][0], s[1][1]); pa[3] = pack_bf16(s[1][2], s[1][3]);
+  __syncwarp();                                   // every lane has its Q fragments: the Q rows become the output tile
+#pragma unroll
+  for (int no = 0; no < NO; no += 2) {
+    float o0[4] = {0.f, 0.f, 0.f, 0.f}, o1[4] = {0.f, 0.f, 0.f, 0.f};
+    uint32_t b[4];
+    ldmatrix_x4_trans(b, sV + ((lane & 7) + 8 * ((lane >> 3) & 1)) * P + no * 8 + 8 * (lane >> 4));
+    mma_bf16_16816(o0, pa, b[0], b[1]);
+    mma_bf16_16816(o1, pa, b[2], b[3]);
+    const int col = no * 8 + 2 * tg;
+    *reinterpret_cast<uint32_t*>(sQ + g * P + col) = pack_bf16(o0[0] * inv0, o0[1] * inv0);
+    *reinterpret_cast<uint32_t*>(sQ + (g + 8) * P + col) = pack_bf16(o0[2] * inv1, o0[3] * inv1);
+    *reinterpret_cast<uint32_t*>(sQ + g * P + col + 8) = pack_bf16(o1[0] * inv0, o1[1] * inv0);
+    *reinterpret_cast<uint32_t*>(sQ + (g + 8) * P + col + 8) = pack_bf16(o1[2] * inv1, o1[3] * inv1);
+  }
+  __syncwarp();
+  for (int i = lane; i < 16 * VPR; i += 32) {
+    const int r = i / VPR, v = i % VPR;
+    if (r < H)
+      *reinterpret_cast<uint4*>(out + ((size_t)n * H + r) * d + (size_t)hd * DH + v * 8) =
+          *reinterpret_cast<const uint4*>(sQ + r * P + v * 8);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Self-attention for sequences longer than one 16-row tile (17..64 tokens), bf16: one block per
 // (candidate, head), one warp per 16-query tile.  The head's keys and values are staged once in
 // shared memory with 16-byte loads and become mma operands through ldmatrix (values transposed), so

@@ -467,6 +467,11 @@ int self_attn_launch(tsdp_ctx* c, const T* qkv, T* out, int n_cand, int H, int d
       if (dh == 32) TSDP_LAUNCH(c, (self_attn_staged_kernel<32>), g2, 128, 0, s, qkv, out, n_cand, H, d, heads, causal);
       else if (dh == 64) TSDP_LAUNCH(c, (self_attn_staged_kernel<64>), g2, 128, 0, s, qkv, out, n_cand, H, d, heads, causal);
       else TSDP_LAUNCH(c, (self_attn_staged_kernel<128>), g2, 128, 0, s, qkv, out, n_cand, H, d, heads, causal);
+    } else if (H <= 16 && (dh == 32 || dh == 64 || dh == 128)) {   // one 16-row tile: operands staged per warp
+      const int tw = dh > 64 ? 2 : 4, g3 = (n_cand * heads + tw - 1) / tw;
+      if (dh == 32) TSDP_LAUNCH(c, (self_attn_tile_kernel<32>), g3, tw * 32, 0, s, qkv, out, n_cand, H, d, heads, causal);
+      else if (dh == 64) TSDP_LAUNCH(c, (self_attn_tile_kernel<64>), g3, tw * 32, 0, s, qkv, out, n_cand, H, d, heads, causal);
+      else TSDP_LAUNCH(c, (self_attn_tile_kernel<128>), g3, tw * 32, 0, s, qkv, out, n_cand, H, d, heads, causal);
     } else
     switch (dh) {
       case 32: TSDP_LAUNCH(c, (self_attn_mma_kernel<32>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads, causal); break;

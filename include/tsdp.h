@@ -16,6 +16,10 @@
  * "at t"; the transition at t produces the latent at t-1; the latent at -1 is the clean action chunk.
  * Kernels of a round are chained with programmatic dependent launch (each may start its prologue while
  * its predecessor drains); setting the environment variable TSDP_NO_PDL before tsdp_init turns that off.
+ * In bf16 the decoder transformer (TSDP_ARCH_XFMR) runs the cross-attention sub-block of every block folded
+ * into its memory tokens (the query and output projections are applied once to the time / observation tokens
+ * instead of to every token row) when H <= 16, (1 + obs_tokens) * heads <= 32, heads is even and d is 128, 256
+ * or 512; TSDP_NO_FOLD, set before tsdp_load_weights, keeps the separate kernels.  Same function either way.
  * Every function returns a tsdp_status; nothing throws or aborts.  A context is not re-entrant: one
  * call at a time.  There is no CPU fallback: without a CUDA device tsdp_init fails with TSDP_ERR_CUDA.
  */

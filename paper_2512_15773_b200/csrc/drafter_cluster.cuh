@@ -27,6 +27,14 @@ constexpr int DC_WARPS = DC_THREADS / 32;
 constexpr int DC_ROWS = 16;       // one m16 tile: H <= 16
 constexpr int DC_MAX_LAYERS = 8;
 constexpr int DC_MAX_NK = 4;      // memory tokens: time token + at most 3 observation tokens
+constexpr int DC_PU = 40;         // folded cross-attention: row pitch (bf16) of the [.. x 32] operands of its second product
+
+template <int BYTES>
+__device__ __forceinline__ void dc_cp_async(void* smem_dst, const void* gsrc) {
+  const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
+  if (BYTES == 16) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gsrc) : "memory");
+  else asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(gsrc) : "memory");
+}
 
 struct DcLayer {
   const __nv_bfloat16 *Wqkv, *Wo, *Wq2, *Wo2, *W1, *W2;      // [out, in] bf16
@@ -40,6 +48,11 @@ struct DcParams {
   const float *W_in, *b_in, *pos;                            // [A, d], [d], [H, d]
   const float *lnf_g, *lnf_b, *W_outT, *b_out;               // W_outT [A, d]
   const float *kv_time, *kv_obs;                             // [T, L*2d], [B*To, L*2d]
+  // cross-attention folded into the memory tokens (xattn_fold.cuh): per-token tables kq [L][heads][d],
+  // ut [L][heads/2][d][2] (bf16) and c [L][heads] (fp32); fold = 0 runs the projections and the attention instead
+  const __nv_bfloat16 *kq_time, *ut_time, *kq_obs, *ut_obs;
+  const float *c_time, *c_obs;
+  int fold;
   DdpmTables S;
   float* xt; long long xs_b;                                 // candidates [B, Kmax+1, D]
   float* muhat; long long ms_b;                              // drafter means [B, Kmax, D]
@@ -78,7 +91,7 @@ __host__ __device__ inline DcSmem dc_smem_plan(int d, int layers, int A, bool re
   p.off_x = take(DC_ROWS * 16 * 4 * 2);                      // latent and eps, D <= 256
   p.off_posb = take(DC_ROWS * d * 4);
   p.off_win = take(A * d * 4);
-  p.off_par = take((layers * (6 * d + 11 * d / DC_CS) + 2 * d + A * d + 16) * 4);   // LayerNorm parameters, this CTA's bias slices, head
+  p.off_par = take((layers * (7 * d + 11 * d / DC_CS) + 2 * d + A * d + 16) * 4);   // LayerNorm parameters, this CTA's bias slices, the whole bo2, head
   p.total = o;
   return p;
 }
@@ -153,7 +166,7 @@ __device__ __forceinline__ float half_warp_sum(float v) {
   for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   return v;
 }
-template <int D_MODEL>
+template <int D_MODEL, bool AFFINE = true>
 __device__ __forceinline__ void dc_layernorm(const float* h, const float* gam, const float* bet,
                                              __nv_bfloat16* out, int pitch) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -177,9 +190,13 @@ __device__ __forceinline__ void dc_layernorm(const float* h, const float* gam, c
 #pragma unroll
   for (int j = 0; j < V; ++j) {
     const int c = (j * 16 + l16) * 4;
-    const float4 gg = *reinterpret_cast<const float4*>(gam + c), bb = *reinterpret_cast<const float4*>(bet + c);
-    store4(out + row * pitch + c, v[j].x * rstd * gg.x + bb.x, v[j].y * rstd * gg.y + bb.y,
-           v[j].z * rstd * gg.z + bb.z, v[j].w * rstd * gg.w + bb.w);
+    if (AFFINE) {
+      const float4 gg = *reinterpret_cast<const float4*>(gam + c), bb = *reinterpret_cast<const float4*>(bet + c);
+      store4(out + row * pitch + c, v[j].x * rstd * gg.x + bb.x, v[j].y * rstd * gg.y + bb.y,
+             v[j].z * rstd * gg.z + bb.z, v[j].w * rstd * gg.w + bb.w);
+    } else {
+      store4(out + row * pitch + c, v[j].x * rstd, v[j].y * rstd, v[j].z * rstd, v[j].w * rstd);
+    }
   }
 }
 
@@ -372,7 +389,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
   for (int i = threadIdx.x; i < A * d; i += DC_THREADS) win[i] = P.W_in[i];
   // LayerNorm parameters and this CTA's slices of the biases of every block, then the head: read from shared
   // memory on the critical path
-  constexpr int PL = 6 * d + 11 * d / DC_CS;       // floats per block
+  constexpr int PL = 7 * d + 11 * d / DC_CS;       // floats per block: 6 LayerNorm vectors, bias slices, the whole bo2
   for (int l = 0; l < L; ++l) {
     const DcLayer& G = P.L[l];
     const float* ln[6] = {G.ln1_g, G.ln1_b, G.ln2_g, G.ln2_b, G.ln3_g, G.ln3_b};
@@ -385,6 +402,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
       for (int i = threadIdx.x; i < ns[j]; i += DC_THREADS) par[(size_t)l * PL + off + i] = bs[j][rank * ns[j] + i];
       off += ns[j];
     }
+    for (int i = threadIdx.x; i < d; i += DC_THREADS) par[(size_t)l * PL + off + i] = G.bo2[i];
   }
   float* lnf_g = par + (size_t)L * PL;
   float* lnf_b = lnf_g + d;
@@ -407,7 +425,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
   // One forward of the network on the latent in sx at timestep tau for request env; leaves eps in seps.
   auto forward = [&](int tau, int env) {
     // keys / values of the time token of tau, every block
-    for (int i = threadIdx.x; i < (resident ? L : 0) * 2 * d; i += DC_THREADS) {
+    for (int i = threadIdx.x; i < (resident && !P.fold ? L : 0) * 2 * d; i += DC_THREADS) {
       const int l = i / (2 * d), c = i % (2 * d);
       skv[(size_t)l * DC_MAX_NK * 2 * d + c] = __ldg(P.kv_time + (size_t)tau * ldkv + (size_t)l * 2 * d + c);
     }
@@ -445,6 +463,39 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         default: dc_attention<d, true>(qkv, PQKV, qkv, PQKV, nullptr, 0, a, PA, P.heads, H); break;
       }
       __syncthreads();
+      if (P.fold) {
+        // the memory tokens' folded tables of this block start their way into shared memory now (the qkv buffer
+        // is free until the next block, the q2 buffer is not used at all): kq rows with their constant in the
+        // row padding -> q2 buffer; u transposed to [output column][token, head] -> qkv buffer, pad columns zero
+        const int heads = P.heads, hp = heads >> 1, NKH = NK * heads;
+        const size_t tok_stride = (size_t)L * heads * d, lay = (size_t)l * heads * d;
+        for (int i = threadIdx.x; i < NKH * (d / 8); i += DC_THREADS) {
+          const int n = i / (d / 8), ch = i % (d / 8);
+          const int j = n / heads, hh = n - j * heads;
+          const __nv_bfloat16* src = (j == 0 ? P.kq_time + (size_t)tau * tok_stride : P.kq_obs + ((size_t)env * P.To + (j - 1)) * tok_stride) +
+                                     lay + (size_t)hh * d + ch * 8;
+          dc_cp_async<16>(q2 + n * PA + ch * 8, src);
+        }
+        for (int n = threadIdx.x; n < NKH; n += DC_THREADS) {
+          const int j = n / heads, hh = n - j * heads;
+          const float* src = (j == 0 ? P.c_time + (size_t)tau * L * heads : P.c_obs + ((size_t)env * P.To + (j - 1)) * L * heads) +
+                             (size_t)l * heads + hh;
+          dc_cp_async<4>(q2 + n * PA + d, src);
+        }
+        uint32_t* sU = reinterpret_cast<uint32_t*>(qkv);                    // [d][DC_PU / 2] words
+        for (int i = threadIdx.x; i < (NKH / 2) * d; i += DC_THREADS) {
+          const int pr = i / d, o = i - pr * d;
+          const int j = pr / hp, q = pr - j * hp;
+          const __nv_bfloat16* src = (j == 0 ? P.ut_time + (size_t)tau * tok_stride : P.ut_obs + ((size_t)env * P.To + (j - 1)) * tok_stride) +
+                                     lay + ((size_t)q * d + o) * 2;
+          dc_cp_async<4>(sU + o * (DC_PU / 2) + pr, src);
+        }
+        for (int i = threadIdx.x; i < d * (16 - NKH / 2); i += DC_THREADS) {
+          const int o = i / (16 - NKH / 2), w = NKH / 2 + i % (16 - NKH / 2);
+          sU[o * (DC_PU / 2) + w] = 0u;
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+      }
       dc_linear<d>(a, PA, w_ptr(l, 1), PWD, NS_D, red, [&](int row, int col, float* v) {
         const int cg_ = rank * NS_D + col;
         const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
@@ -458,7 +509,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
           dst[0] = o0; dst[1] = o1;
         }
       });
-      if (!resident) {   // keys / values of the memory tokens for this block only: time token of tau, then the obs tokens
+      if (!resident && !P.fold) {   // keys / values of the memory tokens for this block only: time token of tau, then the obs tokens
         for (int i = threadIdx.x; i < NK * 2 * d; i += DC_THREADS) {
           const int kx = i / (2 * d), c = i % (2 * d);
           const float* src = kx == 0 ? P.kv_time + (size_t)tau * ldkv : P.kv_obs + ((size_t)env * P.To + (kx - 1)) * ldkv;
@@ -467,6 +518,53 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
       }
       cluster.sync();
       // ---- cross-attention to [time token | obs tokens]
+      if (P.fold) {
+        // Folded form: scores = xhat . kq + c, out = P . u + bo2, both so small that every CTA computes them whole
+        // on its own replica: no slices to exchange, no cluster barrier, two linear stages fewer per block.
+        const int heads = P.heads, NKH = NK * heads;
+        float* sS = reinterpret_cast<float*>(qkv + (size_t)d * DC_PU);       // [16][16] scores
+        __nv_bfloat16* sP = reinterpret_cast<__nv_bfloat16*>(sS + DC_ROWS * 16);   // [16][DC_PU] softmax weights
+        dc_layernorm<d, false>(h, nullptr, nullptr, a, PA);
+        for (int i = threadIdx.x; i < DC_ROWS * DC_PU / 2; i += DC_THREADS) reinterpret_cast<uint32_t*>(sP)[i] = 0u;
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncthreads();
+        dc_linear<d>(a, PA, q2, PA, 16, red, [&](int row, int col, float* v) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) sS[row * 16 + col + j] = v[j];
+        });
+        __syncthreads();
+        for (int p = threadIdx.x; p < DC_ROWS * heads; p += DC_THREADS) {
+          const int row = p / heads, hh = p - row * heads;
+          float sc[DC_MAX_NK];
+          float m = -INFINITY;
+#pragma unroll
+          for (int j = 0; j < DC_MAX_NK; ++j)
+            if (j < NK) {
+              const int n = j * heads + hh;
+              sc[j] = sS[row * 16 + n] + *reinterpret_cast<const float*>(q2 + n * PA + d);
+              m = fmaxf(m, sc[j]);
+            }
+          float lsum = 0.f;
+#pragma unroll
+          for (int j = 0; j < DC_MAX_NK; ++j)
+            if (j < NK) { sc[j] = __expf(sc[j] - m); lsum += sc[j]; }
+          const float inv = 1.0f / lsum;
+#pragma unroll
+          for (int j = 0; j < DC_MAX_NK; ++j)
+            if (j < NK) sP[row * DC_PU + j * heads + hh] = __float2bfloat16_rn(sc[j] * inv);
+        }
+        __syncthreads();
+        const float* bo2_full = pb + 6 * d + 11 * d / DC_CS;
+        dc_linear<32>(sP, DC_PU, qkv, DC_PU, d, red, [&](int row, int col, float* v) {
+          float4* hp4 = reinterpret_cast<float4*>(h + row * d + col);
+          const float4 b0 = *reinterpret_cast<const float4*>(bo2_full + col), b1 = *(reinterpret_cast<const float4*>(bo2_full + col) + 1);
+          float4 h0 = hp4[0], h1 = hp4[1];
+          h0.x += v[0] + b0.x; h0.y += v[1] + b0.y; h0.z += v[2] + b0.z; h0.w += v[3] + b0.w;
+          h1.x += v[4] + b1.x; h1.y += v[5] + b1.y; h1.z += v[6] + b1.z; h1.w += v[7] + b1.w;
+          hp4[0] = h0; hp4[1] = h1;
+        });
+        __syncthreads();
+      } else {
       dc_layernorm<d>(h, W.ln2_g, W.ln2_b, a, PA);
       __syncthreads();
       dc_linear<d>(a, PA, w_ptr(l, 2), PWD, NS_D, red, [&](int row, int col, float* v) {
@@ -494,6 +592,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         }
       });
       cluster.sync();
+      }
       // ---- MLP
       dc_layernorm<d>(h, W.ln3_g, W.ln3_b, a, PA);
       __syncthreads();

@@ -917,6 +917,9 @@ int launch_cluster_forward(tsdp_ctx* c, int which, int mode, int B, int K, cudaS
   P.W_in = n.W_in; P.b_in = n.b_in; P.pos = n.pos;
   P.lnf_g = n.lnf_g; P.lnf_b = n.lnf_b; P.W_outT = n.W_outT; P.b_out = n.b_out;
   P.kv_time = n.kv_time; P.kv_obs = n.kv_obs;
+  P.fold = (n.fold && (1 + c->cfg.obs_tokens) * n.cfg.heads <= 16) ? 1 : 0;     // the cluster kernel's buffers hold 16 (token, head) rows
+  P.kq_time = n.fold_kq_time; P.ut_time = n.fold_ut_time; P.c_time = n.fold_c_time;
+  P.kq_obs = n.fold_kq_obs; P.ut_obs = n.fold_ut_obs; P.c_obs = n.fold_c_obs;
   P.S = c->S;
   P.xt = c->xt; P.xs_b = (long long)(c->cfg.max_K + 1) * c->D;
   P.muhat = c->muhat; P.ms_b = (long long)(c->cfg.max_K > 0 ? c->cfg.max_K : 1) * c->D;

@@ -68,9 +68,7 @@ def test_small_denoisers(arch):
     smp.close()
 
 
-@pytest.mark.parametrize("precision,tol", [(0, 1e-4), (1, 2e-2)])
-@pytest.mark.parametrize("shape", ["small", "pusht", "long"])
-def test_transformer_denoiser(precision, tol, shape):
+def _transformer_case(precision, tol, shape):
     rng = np.random.default_rng(2)
     if shape == "small":
         wl = hp.small_xfmr_workload(precision, d=128, heads=4, layers=2, dd=256, dlayers=1, H=7, A=3, To=3, Do=5,
@@ -80,21 +78,44 @@ def test_transformer_denoiser(precision, tol, shape):
         wl = hp.small_xfmr_workload(precision, d=256, heads=2, layers=2, dd=384, dlayers=1, H=50, A=3, To=3, Do=6,
                                     gamma=1.0)
         wl["draft"]["heads"] = 4
+    elif shape == "no_obs":
+        # the time token is the only memory token; widths 512 (8 heads) and 128 (2 heads)
+        wl = hp.small_xfmr_workload(precision, d=512, heads=8, layers=1, dd=128, dlayers=2, H=16, A=4, To=0, Do=1,
+                                    gamma=1.0)
+        wl["draft"]["heads"] = 2
+    elif shape == "one_obs":
+        wl = hp.small_xfmr_workload(precision, d=512, heads=8, layers=2, dd=256, dlayers=1, H=11, A=2, To=1, Do=9,
+                                    gamma=1.0)
+        wl["draft"]["heads"] = 8
     else:
         wl = dict(inputs.WORKLOADS["pusht_xfmr"], precision=precision, gamma=1.0)
     N = 19      # 19*H token rows: ragged against the 128-row tiles
     smp, S, base, draft = hp.setup(wl, max_B=N, max_K=1)
     x = rng.normal(size=(N, wl["H"], wl["A"])).astype(np.float32)
     tau = rng.integers(0, 100, size=N).astype(np.int32); tau[0], tau[1] = 0, 99
-    obs = inputs.make_obs(5, N, wl["To"], wl["Do"])
+    obs = inputs.make_obs(5, N, wl["To"], wl["Do"]) if wl["To"] else np.zeros((N, 0, wl["Do"]))
     dx = torch.tensor(x, device="cuda"); dobs = torch.tensor(obs, dtype=torch.float32, device="cuda")
     for which, net in ((binding.BASE, base), (binding.DRAFT, draft)):
         out = torch.zeros_like(dx)
-        smp.denoise(which, dx, tau, dobs, N, out)
+        smp.denoise(which, dx, tau, dobs if wl["To"] else None, N, out)
         ref = np.stack([net(x[n].astype(np.float64), int(tau[n]), obs[n]) for n in range(N)])
         err = hp.max_rel(out.cpu().numpy(), ref)
         assert err < tol, (which, err)
     smp.close()
+
+
+@pytest.mark.parametrize("precision,tol", [(0, 1e-4), (1, 2e-2)])
+@pytest.mark.parametrize("shape", ["small", "pusht", "long", "no_obs", "one_obs"])
+def test_transformer_denoiser(precision, tol, shape):
+    _transformer_case(precision, tol, shape)
+
+
+@pytest.mark.parametrize("shape", ["small", "pusht", "one_obs"])
+def test_transformer_denoiser_bf16_without_the_cross_attention_fold(shape, monkeypatch):
+    """The bf16 forward with separate LayerNorm / query GEMM / attention / output GEMM kernels (what shapes outside the
+    fold's limits run), selected by the environment variable the library reads when weights are loaded."""
+    monkeypatch.setenv("TSDP_NO_FOLD", "1")
+    _transformer_case(1, 2e-2, shape)
 
 
 @pytest.mark.parametrize("precision,tol", [(0, 1e-4), (1, 2e-2)])

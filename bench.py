@@ -244,14 +244,14 @@ def run_ours(args):
                                       launches_timed=g["launches"], avg_launch_us=1e3 * g["ms"] / g["launches"],
                                       share_of_kernel_time=g["ms"] / tot_ms, family_ms=fam_ms)
             if args.workload == "serving_xfmr" and B == 256:
-                # ncu DRAM bytes (read + write) of the four GEMM shapes a base block launches (qkv, attention output,
-                # MLP up, MLP down; the cross-attention projections are folded into its memory tokens) at K = 10
-                # (45056 rows), averaged per launch: profiles/gemm_tcgen05_serving_shapes.md.  Rounds with a
-                # smaller K launch proportionally fewer rows.
-                result["roofline"]["traffic"] = 201.2e6
+                # ncu DRAM bytes (read + write) of the four GEMM shapes a base block launches (qkv, attention
+                # projection -- bf16 store --, MLP up, MLP down; the cross-attention projections are folded into its
+                # memory tokens) at K = 10 (45056 rows), averaged per launch: profiles/gemm_tcgen05_serving_shapes.md.
+                # Rounds with a smaller K launch proportionally fewer rows.
+                result["roofline"]["traffic"] = 170.5e6
                 result["roofline"]["traffic_note"] = ("mean DRAM bytes per launch over the 4 GEMM shapes of a block at "
-                                                      "45056 rows (ncu: 126.6, 172.2, 173.5, 332.3 MB); algorithmic "
-                                                      "operand+output bytes average 255e6, the difference stays in L2")
+                                                      "45056 rows (ncu: 126.6, 49.7, 173.5, 332.3 MB); algorithmic "
+                                                      "operand+output bytes average 221e6, the difference stays in L2")
         a = prof.get("accept")
         if a and a["launches"]:
             # fused acceptance / commit kernel: bytes it must move per launch (candidates, drafter means, base

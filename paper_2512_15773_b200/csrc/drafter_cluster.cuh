@@ -602,7 +602,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
 #pragma unroll
         for (int j = 0; j < 8; ++j)
-          v[j] = 0.5f * v[j] * (1.0f + ptx::tanh_fast(0.7978845608028654f * (v[j] + 0.044715f * v[j] * v[j] * v[j])));
+          v[j] = ptx::gelu_fast(v[j]);
         const uint4 pk = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
 #pragma unroll 1
         for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(cluster.map_shared_rank(f, r) + row * PF + cg_) = pk;

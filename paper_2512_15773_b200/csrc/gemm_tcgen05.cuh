@@ -156,6 +156,13 @@ __device__ __forceinline__ float tanh_fast(float x) {
   asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// GELU (tanh form) on the hardware tanh, every operation spelled out so that each place that uses it --
+// both GEMM epilogues and the cluster kernel -- produces the same bits whatever the compiler would contract.
+__device__ __forceinline__ float gelu_fast(float x) {
+  const float x3 = __fmul_rn(__fmul_rn(x, x), x);
+  const float t = tanh_fast(__fmul_rn(0.7978845608028654f, __fmaf_rn(0.044715f, x3, x)));
+  return __fmul_rn(__fmul_rn(0.5f, x), __fadd_rn(1.0f, t));
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 }  // namespace ptx
 
@@ -215,7 +222,7 @@ __device__ __forceinline__ void epilogue_store16(const GemmArgs& g, int row, int
   for (int i = 0; i < 16; ++i) {
     f[i] = __uint_as_float(v[i]);
     if (g.bias) f[i] += __ldg(g.bias + col + i);
-    if (EPI == EPI_GELU) f[i] = gelu_tanh(f[i]);
+    if (EPI == EPI_GELU) f[i] = ptx::gelu_fast(f[i]);
   }
   if (EPI == EPI_GATE) {
     const float* gp = gate_row(g, row) + col;
@@ -386,10 +393,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             }
             if (EPI == EPI_GELU) {
 #pragma unroll
-              for (int i = 0; i < 32; ++i) {
-                const float x = f[i];
-                f[i] = 0.5f * x * (1.0f + ptx::tanh_fast(0.7978845608028654f * (x + 0.044715f * x * x * x)));
-              }
+              for (int i = 0; i < 32; ++i) f[i] = ptx::gelu_fast(f[i]);
             }
             if (EPI == EPI_GATE) {
               const int grow = min(tm * GEMM_BM + r, g.M - 1);     // rows past M are clipped by the TMA store

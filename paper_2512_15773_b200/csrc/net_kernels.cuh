@@ -144,6 +144,60 @@ __global__ void ln_kernel(const float* __restrict__ h, const float* __restrict__
   }
 }
 
+// Token embedding and the first block's LayerNorm in one pass, one warp per token row:
+//   h[row, :] = x[n, i, :] W_in + b_in + pos[i, :]   (fp32 residual stream),   out[row, :] = LN(h[row, :])
+template <typename T, int VEC>
+__global__ void embed_ln_kernel(CandMap cm, const float* __restrict__ W_in, const float* __restrict__ b_in,
+                                const float* __restrict__ pos, float* __restrict__ h, const float* __restrict__ gam,
+                                const float* __restrict__ bet, T* __restrict__ out, int M, int H, int A) {
+  pdl_trigger();
+  pdl_wait();
+  constexpr int d = VEC * 128;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= M) return;
+  const int n = row / H, i = row % H;
+  const int b = n / cm.C, c = n % cm.C;
+  const float* x = cm.xin + b * cm.x_stride_b + (long long)c * H * A + (long long)i * A;
+  float4 v[VEC];
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) {
+    const float4 bi = reinterpret_cast<const float4*>(b_in)[j * 32 + lane];
+    const float4 po = reinterpret_cast<const float4*>(pos + (size_t)i * d)[j * 32 + lane];
+    v[j] = make_float4(bi.x + po.x, bi.y + po.y, bi.z + po.z, bi.w + po.w);
+  }
+  for (int a = 0; a < A; ++a) {
+    const float xa = x[a];
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) {
+      const float4 w = reinterpret_cast<const float4*>(W_in + (size_t)a * d)[j * 32 + lane];
+      v[j].x += xa * w.x; v[j].y += xa * w.y; v[j].z += xa * w.z; v[j].w += xa * w.w;
+    }
+  }
+  float s = 0.f;
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) {
+    reinterpret_cast<float4*>(h + (size_t)row * d)[j * 32 + lane] = v[j];
+    s += v[j].x + v[j].y + v[j].z + v[j].w;
+  }
+  const float mean = warp_sum(s) / d;
+  float q = 0.f;
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) {
+    v[j].x -= mean; v[j].y -= mean; v[j].z -= mean; v[j].w -= mean;
+    q += v[j].x * v[j].x + v[j].y * v[j].y + v[j].z * v[j].z + v[j].w * v[j].w;
+  }
+  const float rstd = rsqrtf(warp_sum(q) / d + 1e-5f);
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) {
+    const int col = (j * 32 + lane) * 4;
+    const float4 gg = reinterpret_cast<const float4*>(gam)[j * 32 + lane];
+    const float4 bb = reinterpret_cast<const float4*>(bet)[j * 32 + lane];
+    store4(out + (size_t)row * d + col, v[j].x * rstd * gg.x + bb.x, v[j].y * rstd * gg.y + bb.y,
+           v[j].z * rstd * gg.z + bb.z, v[j].w * rstd * gg.w + bb.w);
+  }
+}
+
 // ------------------------------------------------------------------------------------------------
 // Causal self-attention over the H action tokens of one candidate; one warp per (candidate, head).
 // qkv [M, 3d] -> out [M, d].  H <= 64, dh = d / heads a multiple of 32 and <= 128.

@@ -582,15 +582,24 @@ int xfmr_forward_t(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStrea
   T* q2 = reinterpret_cast<T*>(c->q2);
   T* f = reinterpret_cast<T*>(c->f);
   int r;
-  prof_begin(c, s, 3, 0.0);
-  TSDP_LAUNCH(c, (embed_kernel), M, d < 256 ? d : 256, 0, s, cm, n.W_in, n.b_in, n.pos, c->h, H, A, d);
-  prof_end(c, s);
-  c->launches_per_round_tmp++;
-  CU_TRY(c, cudaGetLastError());
+  {   // token embedding and the first block's LayerNorm
+    const int wpb = 8, grid = (M + wpb - 1) / wpb;
+    const XfmrLayer& w0 = n.L[0];
+    prof_begin(c, s, 3, 0.0);
+#define EL_CASE(V) TSDP_LAUNCH(c, (embed_ln_kernel<T, V>), grid, wpb * 32, 0, s, cm, n.W_in, n.b_in, n.pos, c->h, w0.ln1_g, w0.ln1_b, a, M, H, A)
+    switch (d / 128) {
+      case 1: EL_CASE(1); break; case 2: EL_CASE(2); break; case 3: EL_CASE(3); break; case 4: EL_CASE(4); break;
+      case 5: EL_CASE(5); break; case 6: EL_CASE(6); break; case 7: EL_CASE(7); break; default: EL_CASE(8); break;
+    }
+#undef EL_CASE
+    prof_end(c, s);
+    c->launches_per_round_tmp++;
+    CU_TRY(c, cudaGetLastError());
+  }
   const int out_epi = (c->cfg.precision == 0) ? EPI_F32 : EPI_STORE;
   for (int l = 0; l < L; ++l) {
     const XfmrLayer& w = n.L[l];
-    if ((r = ln_launch<T>(c, c->h, w.ln1_g, w.ln1_b, a, M, d, s))) return r;
+    if (l > 0 && (r = ln_launch<T>(c, c->h, w.ln1_g, w.ln1_b, a, M, d, s))) return r;
     if ((r = gemm(c, a, w.Wqkv, w.bqkv, M, 3 * d, d, out_epi, qkv, 3 * d, s))) return r;
     if ((r = self_attn_launch<T>(c, qkv, a, n_cand, H, d, heads, s))) return r;
     if (n.fold) {

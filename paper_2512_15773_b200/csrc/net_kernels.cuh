@@ -144,40 +144,35 @@ __global__ void ln_kernel(const float* __restrict__ h, const float* __restrict__
   }
 }
 
-// Token embedding and the first block's LayerNorm in one pass, one warp per token row:
-//   h[row, :] = x[n, i, :] W_in + b_in + pos[i, :]   (fp32 residual stream),   out[row, :] = LN(h[row, :])
-template <typename T, int VEC>
-__global__ void embed_ln_kernel(CandMap cm, const float* __restrict__ W_in, const float* __restrict__ b_in,
-                                const float* __restrict__ pos, float* __restrict__ h, const float* __restrict__ gam,
-                                const float* __restrict__ bet, T* __restrict__ out, int M, int H, int A) {
-  pdl_trigger();
-  pdl_wait();
+// Token embedding and the first block's LayerNorm of one token row by one warp:
+//   h_row[:] = x[0..A) W_in + b_in + pos_row[:]   (fp32 residual stream),   out_row[:] = LN(h_row[:])
+// x_of(a) returns the a-th input value (the same in every lane).
+template <typename T, int VEC, typename XF>
+__device__ __forceinline__ void embed_ln_row(XF x_of, int A, const float* __restrict__ W_in, const float* __restrict__ b_in,
+                                             const float* __restrict__ pos_row, float* __restrict__ h_row,
+                                             const float* __restrict__ gam, const float* __restrict__ bet, T* __restrict__ out_row,
+                                             int lane) {
   constexpr int d = VEC * 128;
-  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const int lane = threadIdx.x & 31;
-  if (row >= M) return;
-  const int n = row / H, i = row % H;
-  const int b = n / cm.C, c = n % cm.C;
-  const float* x = cm.xin + b * cm.x_stride_b + (long long)c * H * A + (long long)i * A;
   float4 v[VEC];
 #pragma unroll
   for (int j = 0; j < VEC; ++j) {
     const float4 bi = reinterpret_cast<const float4*>(b_in)[j * 32 + lane];
-    const float4 po = reinterpret_cast<const float4*>(pos + (size_t)i * d)[j * 32 + lane];
+    const float4 po = reinterpret_cast<const float4*>(pos_row)[j * 32 + lane];
     v[j] = make_float4(bi.x + po.x, bi.y + po.y, bi.z + po.z, bi.w + po.w);
   }
   for (int a = 0; a < A; ++a) {
-    const float xa = x[a];
+    const float xa = x_of(a);
 #pragma unroll
     for (int j = 0; j < VEC; ++j) {
       const float4 w = reinterpret_cast<const float4*>(W_in + (size_t)a * d)[j * 32 + lane];
-      v[j].x += xa * w.x; v[j].y += xa * w.y; v[j].z += xa * w.z; v[j].w += xa * w.w;
+      v[j].x = __fmaf_rn(xa, w.x, v[j].x); v[j].y = __fmaf_rn(xa, w.y, v[j].y);
+      v[j].z = __fmaf_rn(xa, w.z, v[j].z); v[j].w = __fmaf_rn(xa, w.w, v[j].w);
     }
   }
   float s = 0.f;
 #pragma unroll
   for (int j = 0; j < VEC; ++j) {
-    reinterpret_cast<float4*>(h + (size_t)row * d)[j * 32 + lane] = v[j];
+    reinterpret_cast<float4*>(h_row)[j * 32 + lane] = v[j];
     s += v[j].x + v[j].y + v[j].z + v[j].w;
   }
   const float mean = warp_sum(s) / d;
@@ -193,9 +188,26 @@ __global__ void embed_ln_kernel(CandMap cm, const float* __restrict__ W_in, cons
     const int col = (j * 32 + lane) * 4;
     const float4 gg = reinterpret_cast<const float4*>(gam)[j * 32 + lane];
     const float4 bb = reinterpret_cast<const float4*>(bet)[j * 32 + lane];
-    store4(out + (size_t)row * d + col, v[j].x * rstd * gg.x + bb.x, v[j].y * rstd * gg.y + bb.y,
+    store4(out_row + col, v[j].x * rstd * gg.x + bb.x, v[j].y * rstd * gg.y + bb.y,
            v[j].z * rstd * gg.z + bb.z, v[j].w * rstd * gg.w + bb.w);
   }
+}
+
+template <typename T, int VEC>
+__global__ void embed_ln_kernel(CandMap cm, const float* __restrict__ W_in, const float* __restrict__ b_in,
+                                const float* __restrict__ pos, float* __restrict__ h, const float* __restrict__ gam,
+                                const float* __restrict__ bet, T* __restrict__ out, int M, int H, int A) {
+  pdl_trigger();
+  pdl_wait();
+  constexpr int d = VEC * 128;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= M) return;
+  const int n = row / H, i = row % H;
+  const int b = n / cm.C, c = n % cm.C;
+  const float* x = cm.xin + b * cm.x_stride_b + (long long)c * H * A + (long long)i * A;
+  embed_ln_row<T, VEC>([&](int a) { return x[a]; }, A, W_in, b_in, pos + (size_t)i * d, h + (size_t)row * d, gam, bet,
+                       out + (size_t)row * d, lane);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -791,21 +803,15 @@ cross_attn_group_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __re
 // ------------------------------------------------------------------------------------------------
 // Output head: eps[n, i, :] = LN_f(h[row]) W_out + b_out, one warp per row; W_outT is [A, d] fp32.
 // ------------------------------------------------------------------------------------------------
+// Final LayerNorm of one row by one warp, result left in v (lane owns columns (j*32 + lane)*4 .. +3).
 template <int VEC>
-__global__ void head_kernel(const float* __restrict__ h, const float* __restrict__ gam, const float* __restrict__ bet,
-                            const float* __restrict__ W_outT, const float* __restrict__ b_out, CandMap cm, int M,
-                            int H, int A) {
-  pdl_trigger();
-  pdl_wait();
+__device__ __forceinline__ void head_ln_row(const float* __restrict__ h_row, const float* __restrict__ gam,
+                                            const float* __restrict__ bet, float4 (&v)[VEC], int lane) {
   constexpr int d = VEC * 128;
-  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const int lane = threadIdx.x & 31;
-  if (row >= M) return;
-  float4 v[VEC];
   float s = 0.f;
 #pragma unroll
   for (int j = 0; j < VEC; ++j) {
-    v[j] = reinterpret_cast<const float4*>(h + (size_t)row * d)[j * 32 + lane];
+    v[j] = reinterpret_cast<const float4*>(h_row)[j * 32 + lane];
     s += v[j].x + v[j].y + v[j].z + v[j].w;
   }
   const float mean = warp_sum(s) / d;
@@ -823,18 +829,39 @@ __global__ void head_kernel(const float* __restrict__ h, const float* __restrict
     v[j].x = v[j].x * rstd * gg.x + bb.x; v[j].y = v[j].y * rstd * gg.y + bb.y;
     v[j].z = v[j].z * rstd * gg.z + bb.z; v[j].w = v[j].w * rstd * gg.w + bb.w;
   }
+}
+// eps of action a for that row (the same value in every lane); products and sums spelled out so that every
+// kernel that computes it gets the same bits.
+template <int VEC>
+__device__ __forceinline__ float head_out(const float4 (&v)[VEC], const float* __restrict__ w_row, float bias, int lane) {
+  float acc = 0.f;
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) {
+    const float4 w = reinterpret_cast<const float4*>(w_row)[j * 32 + lane];
+    acc = __fmaf_rn(v[j].x, w.x, acc); acc = __fmaf_rn(v[j].y, w.y, acc);
+    acc = __fmaf_rn(v[j].z, w.z, acc); acc = __fmaf_rn(v[j].w, w.w, acc);
+  }
+  return __fadd_rn(warp_sum(acc), bias);
+}
+
+template <int VEC>
+__global__ void head_kernel(const float* __restrict__ h, const float* __restrict__ gam, const float* __restrict__ bet,
+                            const float* __restrict__ W_outT, const float* __restrict__ b_out, CandMap cm, int M,
+                            int H, int A) {
+  pdl_trigger();
+  pdl_wait();
+  constexpr int d = VEC * 128;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= M) return;
+  float4 v[VEC];
+  head_ln_row<VEC>(h + (size_t)row * d, gam, bet, v, lane);
   const int n = row / H, i = row % H;
   const int b = n / cm.C, c = n % cm.C;
   float* o = cm.eout + b * cm.e_stride_b + (long long)c * H * A + (long long)i * A;
   for (int a = 0; a < A; ++a) {
-    float acc = 0.f;
-#pragma unroll
-    for (int j = 0; j < VEC; ++j) {
-      const float4 w = reinterpret_cast<const float4*>(W_outT + (size_t)a * d)[j * 32 + lane];
-      acc += v[j].x * w.x + v[j].y * w.y + v[j].z * w.z + v[j].w * w.w;
-    }
-    acc = warp_sum(acc);
-    if (lane == 0) o[a] = acc + b_out[a];
+    const float e = head_out<VEC>(v, W_outT + (size_t)a * d, b_out[a], lane);
+    if (lane == 0) o[a] = e;
   }
 }
 

@@ -24,6 +24,7 @@
 #include "dit_kernels.cuh"
 #include "unet_kernels.cuh"
 #include "xattn_fold.cuh"
+#include "draft_tail.cuh"
 
 using namespace tsdp;
 
@@ -130,6 +131,7 @@ struct tsdp_ctx {
   // optional per-kernel-family timing with CUDA events (plain launches, no graph)
   bool prof_on = false;
   int prof_gemm_cat = 0;                      // 0 while the base model runs, 6 while the drafter runs
+  bool xf_skip_embed = false, xf_skip_head = false;   // layer-by-layer drafter: draft_tail_kernel does those parts
   std::vector<cudaEvent_t> prof_ev;
   std::vector<int> prof_cat;
   std::vector<double> prof_flop;
@@ -582,7 +584,7 @@ int xfmr_forward_t(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStrea
   T* q2 = reinterpret_cast<T*>(c->q2);
   T* f = reinterpret_cast<T*>(c->f);
   int r;
-  {   // token embedding and the first block's LayerNorm
+  if (!c->xf_skip_embed) {   // token embedding and the first block's LayerNorm
     const int wpb = 8, grid = (M + wpb - 1) / wpb;
     const XfmrLayer& w0 = n.L[0];
     prof_begin(c, s, 3, 0.0);
@@ -619,7 +621,31 @@ int xfmr_forward_t(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStrea
     if ((r = gemm(c, a, w.W1, w.b1, M, 4 * d, d, EPI_GELU, f, 4 * d, s))) return r;
     if ((r = gemm(c, f, w.W2, w.b2, M, d, 4 * d, EPI_RESID, c->h, d, s))) return r;
   }
+  if (c->xf_skip_head) return TSDP_OK;
   return head_launch(c, n, cm, M, s);
+}
+
+// Head of the drafter, the draft step and the next step's embedding + LayerNorm in one launch (draft_tail.cuh).
+template <typename T>
+int draft_tail_launch(tsdp_ctx* c, Net& n, int B, int k, int K, bool embed_next, cudaStream_t s) {
+  const int H = c->cfg.H, A = c->cfg.A, D = c->D, M = B * H, d = n.cfg.d;
+  const long long xs_b = (long long)(c->cfg.max_K + 1) * D, ms_b = (long long)(c->cfg.max_K > 0 ? c->cfg.max_K : 1) * D;
+  const int wpb = 8, grid = (M + wpb - 1) / wpb;
+  const XfmrLayer& w0 = n.L[0];
+  T* a = reinterpret_cast<T*>(c->a);
+  prof_begin(c, s, 4, 0.0);
+#define DT_CASE(V) TSDP_LAUNCH(c, (draft_tail_kernel<T, V>), grid, wpb * 32, 0, s, c->h, n.lnf_g, n.lnf_b, n.W_outT, n.b_out, c->S, c->xt, xs_b, \
+                               c->muhat, ms_b, c->eps_d, c->t, k, K, c->cfg.T, c->seed, c->sched_on ? c->envp : nullptr, c->item, n.W_in, n.b_in,   \
+                               n.pos, w0.ln1_g, w0.ln1_b, a, embed_next ? 1 : 0, M, H, A)
+  switch (d / 128) {
+    case 1: DT_CASE(1); break; case 2: DT_CASE(2); break; case 3: DT_CASE(3); break; case 4: DT_CASE(4); break;
+    case 5: DT_CASE(5); break; case 6: DT_CASE(6); break; case 7: DT_CASE(7); break; default: DT_CASE(8); break;
+  }
+#undef DT_CASE
+  prof_end(c, s);
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  return TSDP_OK;
 }
 
 // Observation tokens -> their cross-attention keys/values for every block (once per chunk).
@@ -968,12 +994,23 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
   int r;
   const bool cluster_draft = K > 0 && use_cluster_drafter(c, B);
   if (cluster_draft && (r = launch_cluster_forward(c, TSDP_DRAFT, 0, B, K, s))) return r;
+  // transformer drafter, layer by layer: its head, the draft step and the next step's embedding are one kernel
+  const bool fused_tail = c->net[TSDP_DRAFT].cfg.arch == TSDP_ARCH_XFMR && c->cfg.A <= 32;
   for (int k = 1; k <= K && !cluster_draft; ++k) {
     CandMap cm{c->xt + (long long)(k - 1) * D, xs_b, c->eps_d, (long long)D, c->t, 1, k - 1, c->item};
     c->prof_gemm_cat = 6;
+    c->xf_skip_embed = fused_tail && k > 1;
+    c->xf_skip_head = fused_tail;
     r = forward(c, c->net[TSDP_DRAFT], cm, B, s);
     c->prof_gemm_cat = 0;
+    c->xf_skip_embed = c->xf_skip_head = false;
     if (r) return r;
+    if (fused_tail) {
+      r = c->cfg.precision == 0 ? draft_tail_launch<float>(c, c->net[TSDP_DRAFT], B, k, K, k < K, s)
+                                : draft_tail_launch<__nv_bfloat16>(c, c->net[TSDP_DRAFT], B, k, K, k < K, s);
+      if (r) return r;
+      continue;
+    }
     prof_begin(c, s, 4, 0.0);
     TSDP_LAUNCH(c, (draft_step_kernel), B, 128, 0, s, c->S, c->xt, xs_b, c->muhat, ms_b, c->eps_d, c->t, k, D, c->seed,
                 c->sched_on ? c->envp : nullptr, K, c->cfg.T, c->item);

@@ -327,25 +327,19 @@ cudaError_t set_smem_attr_all() {
   return set_smem_attr<BN, EPI_F32>();
 }
 
-// Tile width BN in {256, 128, 64, 32} (a divisor of N) that minimises a simple time model of the persistent
-// kernel: waves of tiles over the SMs, each wave costing its k-loop at the tensor rate plus a fixed pipeline
-// fill, and one exposed epilogue at the end.  Large problems get the widest tile; calls with fewer tiles than
-// SMs trade tile width against the number of waves (a single wave of 64-wide tiles beats two of 32-wide ones).
-int pick_bn(int M, int N, int K, int num_sms) {
+// Tile width: the widest BN in {256, 128, 64, 32} dividing N whose tiles still fill 60 % of the SMs, else the
+// narrowest that divides N (small-batch calls are latency-bound and want many CTAs).  Measured on the block's
+// shapes at 4 k - 45 k rows: per flop a 128-wide tile costs 1.24x and a 64-wide one 2.15x of a 256-wide one (the
+// k-loop of a narrow tile is bound by loading the 128-row A block, which does not shrink), so a wide tile that
+// leaves a third of the SMs idle still beats two waves of narrow ones; below about half occupancy it does not.
+int pick_bn(int M, int N, int num_sms) {
   const int tm = (M + GEMM_BM - 1) / GEMM_BM;
   const int cands[4] = {256, 128, 64, 32};
-  int best = 0;
-  double best_cost = 0.0;
-  for (int i = 0; i < 4; ++i) {
-    const int bn = cands[i];
-    if (N % bn != 0) continue;
-    const long long tiles = (long long)tm * (N / bn);
-    const double waves = (double)((tiles + num_sms - 1) / num_sms);
-    const double kloop_us = (K / (double)GEMM_BK) * (bn / 256.0) * 0.44;      // 128 x 256 x 64 at the dense bf16 rate
-    const double cost = waves * (kloop_us + 1.0) + (bn / 256.0) * 1.5;
-    if (best == 0 || cost < best_cost) { best = bn; best_cost = cost; }
-  }
-  return best;
+  for (int i = 0; i < 4; ++i)
+    if (N % cands[i] == 0 && (long long)tm * (N / cands[i]) * 5 >= (long long)num_sms * 3) return cands[i];
+  for (int i = 3; i >= 0; --i)
+    if (N % cands[i] == 0) return cands[i];
+  return 0;
 }
 
 // Gate of an adaptive-LayerNorm residual (EPI_GATE): gate vectors and the row -> timestep map.
@@ -382,7 +376,7 @@ int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, in
     c->last_error = "tensor-core GEMM needs K % 64 == 0 and N % 32 == 0";
     return TSDP_ERR_ARG;
   }
-  const int BN = pick_bn(M, N, K, c->num_sms);
+  const int BN = pick_bn(M, N, c->num_sms);
   CUtensorMap ma, mb, mc;
   int r;
   if (conv_c > 0) {      // kernel-5 convolution: A is the padded tensor [M + 4, conv_c] itself

@@ -131,6 +131,7 @@ struct tsdp_ctx {
   // optional per-kernel-family timing with CUDA events (plain launches, no graph)
   bool prof_on = false;
   int prof_gemm_cat = 0;                      // 0 while the base model runs, 6 while the drafter runs
+  int force_bn = 0;                           // TSDP_GEMM_BN
   bool xf_skip_embed = false, xf_skip_head = false;   // layer-by-layer drafter: draft_tail_kernel does those parts
   std::vector<cudaEvent_t> prof_ev;
   std::vector<int> prof_cat;
@@ -376,7 +377,7 @@ int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, in
     c->last_error = "tensor-core GEMM needs K % 64 == 0 and N % 32 == 0";
     return TSDP_ERR_ARG;
   }
-  const int BN = pick_bn(M, N, c->num_sms);
+  const int BN = (c->force_bn > 0 && N % c->force_bn == 0) ? c->force_bn : pick_bn(M, N, c->num_sms);
   CUtensorMap ma, mb, mc;
   int r;
   if (conv_c > 0) {      // kernel-5 convolution: A is the padded tensor [M + 4, conv_c] itself
@@ -1146,6 +1147,10 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   c->cfg = *cfg;
   c->D = cfg->H * cfg->A;
   c->pdl = getenv("TSDP_NO_PDL") == nullptr;
+  if (const char* fb = getenv("TSDP_GEMM_BN")) {      // tuning aid: one tile width for every GEMM it divides
+    const int v = atoi(fb);
+    if (v == 32 || v == 64 || v == 128 || v == 256) c->force_bn = v;
+  }
   auto fail = [&](int st) { tsdp_destroy(c); return st; };
 #define INIT_TRY(expr)                                                                    \
   do {                                                                                    \

@@ -47,7 +47,13 @@ typedef enum {
   TSDP_ERR_TOO_LARGE = 8    /* size beyond the capacity of tsdp_verify_commit_static       */
 } tsdp_status;
 
-enum { TSDP_ARCH_GAUSS = 0, TSDP_ARCH_MLP = 1, TSDP_ARCH_XFMR = 2, TSDP_ARCH_DIT = 3, TSDP_ARCH_UNET = 4 };
+enum { TSDP_ARCH_GAUSS = 0, TSDP_ARCH_MLP = 1, TSDP_ARCH_XFMR = 2, TSDP_ARCH_DIT = 3, TSDP_ARCH_UNET = 4,
+       /* Only as the DRAFT network: no drafter at all.  The drafts of a round reuse the base model's output at
+        * the round's starting latent for every step ("frozen target draft", the drafter-free scheme of the prior
+        * work cited in Sec. 2.2): eps^_k = eps_base(x, t) for k = 1..K.  A round then costs one base forward on
+        * the B current latents plus the batched verification; the first draft is the base model's own step and
+        * is always accepted.  Takes no weights: tsdp_load_weights(TSDP_DRAFT) is not called. */
+       TSDP_ARCH_FROZEN = 5 };
 enum { TSDP_BASE = 0, TSDP_DRAFT = 1, TSDP_SCHED = 2 };
 enum { TSDP_MAX_T = 1024, TSDP_MAX_K = 32 };
 
@@ -117,7 +123,9 @@ typedef struct {
   uint64_t base_evals;      /* candidate latents the base model evaluated (useful ones)       */
   uint64_t draft_evals;     /* drafter calls (= drafts proposed)                               */
   uint64_t drafts_tested, drafts_accepted, rejections, bonus_steps, steps_advanced;
-  double nfe;               /* env_rounds + draft_nfe * draft_evals                           */
+  uint64_t draft_rounds;    /* rounds summed over environments in which at least one step was drafted */
+  double nfe;               /* env_rounds + draft_nfe * draft_evals (+ draft_rounds with TSDP_ARCH_FROZEN drafts:
+                               the base forward that supplies them)                            */
   uint64_t hist_drafted[TSDP_MAX_T], hist_tested[TSDP_MAX_T], hist_accepted[TSDP_MAX_T];
                             /* per timestep of the drafted transition                          */
 } tsdp_stats_t;

@@ -75,10 +75,35 @@ def first_rejection(acc_flags):
     return None
 
 
+class FrozenTargetDraft:
+    """Drafts without a drafter: every draft step of a round reuses the base model's output at the round's
+    starting latent, eps^_k = eps_base(x, t) for k = 1..K (the "frozen target draft" of the prior work cited in
+    Sec. 2.2, read as: the target's prediction is frozen over the window).  The first draft is then the base
+    model's own reverse step, so its acceptance ratio is exactly 1; later ones drift from it.  Any draft mean
+    leaves the sampler's law unchanged (Sec. 3.1), so this variant is lossless too.  A round costs one extra base
+    evaluation (n_extra in the round's dump).  PARITY UNPINNED against that prior work (not in the paper);
+    pinned by: first draft always accepted with log alpha = 0, K = 1 sample-identical to vanilla, and the
+    Gaussian chain's marginal."""
+
+    def __init__(self, base):
+        self.base = base
+        self.eps = None
+
+    def begin_round(self, x, t, obs):
+        self.eps = self.base(x, t, obs)
+
+    def __call__(self, x, tau, obs):
+        return self.eps
+
+
 def spec_round(sched, base, drafter, noise, env, obs, x, t, K, acc, clip=0.0):
     """One speculative round for one environment.  Returns (x_new, t_new, dump)."""
     K_eff = min(K, t)
     shape = x.shape
+    n_extra = 0
+    if K_eff > 0 and hasattr(drafter, "begin_round"):      # drafter-free drafts: one base evaluation at the current latent
+        drafter.begin_round(x, t, obs)
+        n_extra = 1
     # --- draft rollout (Eq. (3)): x~_0 = x; draft k is the transition at tau = t-k+1
     x_t = [x]
     mu_hat, xis = [None], [None]
@@ -112,7 +137,7 @@ def spec_round(sched, base, drafter, noise, env, obs, x, t, K, acc, clip=0.0):
     else:
         x_new, t_new = x_t[K_eff], t - K_eff
     dump = dict(K_eff=K_eff, x_tilde=x_t, mu_hat=mu_hat, eps=eps, mu=mu, log_alpha=log_alpha,
-                flags=flags, jstar=(j if j is not None else K_eff + 1), n_base=n_base)
+                flags=flags, jstar=(j if j is not None else K_eff + 1), n_base=n_base, n_extra=n_extra)
     return x_new, t_new, dump
 
 
@@ -123,7 +148,7 @@ def sample_chunk(sched, base, drafter, noise, env, obs, shape, K, acc, clip=0.0,
     NFE ingredients the paper reports (Sec. 4 "Evaluation Metrics")."""
     x = noise.x_init(env, shape)
     t = sched.T - 1
-    st = dict(rounds=0, base_evals=0, draft_evals=0, accepted=0, rejections=0, bonus=0,
+    st = dict(rounds=0, base_evals=0, draft_evals=0, accepted=0, rejections=0, bonus=0, extra_base=0, draft_rounds=0,
               prefix=[], prop_hist=np.zeros(sched.T, int), test_hist=np.zeros(sched.T, int),
               acc_hist=np.zeros(sched.T, int))
     while t >= 0:
@@ -133,6 +158,8 @@ def sample_chunk(sched, base, drafter, noise, env, obs, shape, K, acc, clip=0.0,
         st["rounds"] += 1
         st["base_evals"] += d["n_base"]
         st["draft_evals"] += d["K_eff"]
+        st["extra_base"] += d["n_extra"]
+        st["draft_rounds"] += int(d["K_eff"] > 0)
         st["accepted"] += n_acc
         st["rejections"] += int(d["jstar"] <= d["K_eff"])
         st["bonus"] += int(d["jstar"] > d["K_eff"] and (t - t_new) == d["K_eff"] + 1)

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libtsdp.so")
 
 TSDP_MAX_T = 1024
-ARCH = {"gauss": 0, "mlp": 1, "xfmr": 2, "dit": 3, "unet": 4}
+ARCH = {"gauss": 0, "mlp": 1, "xfmr": 2, "dit": 3, "unet": 4, "frozen": 5}     # "frozen": drafter only, no weights
 BASE, DRAFT, SCHED = 0, 1, 2
 EXPORTS = ["tsdp_init", "tsdp_destroy", "tsdp_strerror", "tsdp_last_error", "tsdp_weights_count",
            "tsdp_load_weights", "tsdp_set_schedule", "tsdp_sample_chunk", "tsdp_sample_chunk_host",
@@ -39,7 +39,7 @@ class StatsT(C.Structure):
     _fields_ = [("chunks", C.c_uint64), ("rounds", C.c_uint64), ("env_rounds", C.c_uint64),
                 ("base_evals", C.c_uint64), ("draft_evals", C.c_uint64), ("drafts_tested", C.c_uint64),
                 ("drafts_accepted", C.c_uint64), ("rejections", C.c_uint64), ("bonus_steps", C.c_uint64),
-                ("steps_advanced", C.c_uint64), ("nfe", C.c_double),
+                ("steps_advanced", C.c_uint64), ("draft_rounds", C.c_uint64), ("nfe", C.c_double),
                 ("hist_drafted", C.c_uint64 * TSDP_MAX_T), ("hist_tested", C.c_uint64 * TSDP_MAX_T),
                 ("hist_accepted", C.c_uint64 * TSDP_MAX_T)]
 

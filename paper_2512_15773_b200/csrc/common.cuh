@@ -153,7 +153,7 @@ __device__ __forceinline__ int env_draft_cap(const EnvParams* envp, int env, int
 // Device-side counters behind tsdp_stats.
 struct DevStats {
   unsigned long long env_rounds, base_evals, draft_evals, drafts_tested, drafts_accepted, rejections,
-      bonus_steps, steps_advanced, chunks_done;
+      bonus_steps, steps_advanced, chunks_done, draft_rounds;
   unsigned long long hist_drafted[1024], hist_tested[1024], hist_accepted[1024];
 };
 

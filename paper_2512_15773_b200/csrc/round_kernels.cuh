@@ -33,9 +33,9 @@ __global__ void init_chunk_kernel(float* __restrict__ xt, long long xs_b, int* _
 
 // Draft step k (Eq. (3) of Sec. 3.2): tau = t - k + 1, mu^_k = posterior mean of (x~_{k-1}, eps^),
 // x~_k = mu^_k + sigma_tau xi_tau.  Slots beyond K_eff = min(K, t) copy the previous latent so that
-// every buffer stays finite.
+// every buffer stays finite.  eps^ of slot b is the D values at eps_d + b * es_b.
 __global__ void draft_step_kernel(DdpmTables S, float* __restrict__ xt, long long xs_b, float* __restrict__ muhat,
-                                  long long ms_b, const float* __restrict__ eps_d, const int* __restrict__ t,
+                                  long long ms_b, const float* __restrict__ eps_d, long long es_b, const int* __restrict__ t,
                                   int k, int D, const uint64_t* __restrict__ seedp, const EnvParams* __restrict__ envp,
                                   int K, int Tsteps, const int* __restrict__ item) {
   pdl_trigger();
@@ -49,7 +49,7 @@ __global__ void draft_step_kernel(DdpmTables S, float* __restrict__ xt, long lon
   const float* xp = xt + b * xs_b + (long long)(k - 1) * D;
   float* xn = xt + b * xs_b + (long long)k * D;
   float* mh = muhat + b * ms_b + (long long)(k - 1) * D;
-  const float* e = eps_d + (long long)b * D;
+  const float* e = eps_d + b * es_b;
   const int nq = (D + 3) >> 2;
   for (int q = threadIdx.x; q < nq; q += blockDim.x) {
     float z[4] = {0.f, 0.f, 0.f, 0.f};
@@ -212,6 +212,7 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
     atomicAdd(&stats->env_rounds, 1ull);
     atomicAdd(&stats->base_evals, (unsigned long long)((rp.bonus || K_eff == 0) ? K_eff + 1 : K_eff));
     atomicAdd(&stats->draft_evals, (unsigned long long)K_eff);
+    atomicAdd(&stats->draft_rounds, K_eff > 0 ? 1ull : 0ull);
     atomicAdd(&stats->drafts_tested, (unsigned long long)n_tested);
     atomicAdd(&stats->drafts_accepted, (unsigned long long)n_acc);
     atomicAdd(&stats->rejections, rejected ? 1ull : 0ull);

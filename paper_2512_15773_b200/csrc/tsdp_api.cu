@@ -208,6 +208,7 @@ std::vector<std::pair<int, int>> unet_channels(int c, int levels) {
 
 bool net_cfg_ok(const tsdp_config_t& cfg, const tsdp_net_t& n) {
   if (n.arch == TSDP_ARCH_GAUSS) return true;
+  if (n.arch == TSDP_ARCH_FROZEN) return &n == &cfg.draft;      // a way to draft, not a network: drafter only
   if (n.arch == TSDP_ARCH_MLP)
     return n.layers >= 1 && n.layers <= MLP_MAX_LAYERS && n.d >= 1 && n.d <= 4096 && n.temb >= 2 && n.temb % 2 == 0;
   if (n.arch == TSDP_ARCH_XFMR)
@@ -989,6 +990,19 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
   int r;
   const bool cluster_draft = K > 0 && use_cluster_drafter(c, B);
   if (cluster_draft && (r = launch_cluster_forward(c, TSDP_DRAFT, 0, B, K, s))) return r;
+  const bool frozen_draft = c->net[TSDP_DRAFT].cfg.arch == TSDP_ARCH_FROZEN;
+  const float* eps_hat = c->eps_d;        // where the draft step finds eps^ of slot b: eps_hat + b * eps_hat_b
+  long long eps_hat_b = D;
+  if (frozen_draft && K > 0) {
+    // frozen target drafts: the base model's output at the current latent serves every draft step of the round
+    if (use_cluster_verifier(c, B, 0)) {          // one cluster per slot; eps lands in candidate slot 0 of the eps buffer
+      if ((r = launch_cluster_forward(c, TSDP_BASE, 1, B, 0, s))) return r;
+      eps_hat = c->eps; eps_hat_b = xs_b;
+    } else {
+      CandMap c0{c->xt, xs_b, c->eps_d, (long long)D, c->t, 1, 0, c->item};
+      if ((r = forward(c, c->net[TSDP_BASE], c0, B, s))) return r;
+    }
+  }
   // transformer drafter, layer by layer: its head, the draft step and the next step's embedding are one kernel
   const bool fused_tail = c->net[TSDP_DRAFT].cfg.arch == TSDP_ARCH_XFMR && c->cfg.A <= 32;
   for (int k = 1; k <= K && !cluster_draft; ++k) {
@@ -996,7 +1010,7 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
     c->prof_gemm_cat = 6;
     c->xf_skip_embed = fused_tail && k > 1;
     c->xf_skip_head = fused_tail;
-    r = forward(c, c->net[TSDP_DRAFT], cm, B, s);
+    r = frozen_draft ? TSDP_OK : forward(c, c->net[TSDP_DRAFT], cm, B, s);
     c->prof_gemm_cat = 0;
     c->xf_skip_embed = c->xf_skip_head = false;
     if (r) return r;
@@ -1007,7 +1021,7 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
       continue;
     }
     prof_begin(c, s, 4, 0.0);
-    TSDP_LAUNCH(c, (draft_step_kernel), B, 128, 0, s, c->S, c->xt, xs_b, c->muhat, ms_b, c->eps_d, c->t, k, D, c->seed,
+    TSDP_LAUNCH(c, (draft_step_kernel), B, 128, 0, s, c->S, c->xt, xs_b, c->muhat, ms_b, eps_hat, eps_hat_b, c->t, k, D, c->seed,
                 c->sched_on ? c->envp : nullptr, K, c->cfg.T, c->item);
     prof_end(c, s);
     c->launches_per_round_tmp++;
@@ -1140,7 +1154,7 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
       cfg->verifier > 2)
     return TSDP_ERR_ARG;
   for (const tsdp_net_t* n : {&cfg->base, &cfg->draft}) {
-    if (n->arch < TSDP_ARCH_GAUSS || n->arch > TSDP_ARCH_UNET) return TSDP_ERR_UNSUPPORTED;
+    if (n->arch < TSDP_ARCH_GAUSS || n->arch > TSDP_ARCH_FROZEN) return TSDP_ERR_UNSUPPORTED;
     if (!net_cfg_ok(*cfg, *n)) return TSDP_ERR_ARG;
   }
   tsdp_ctx* c = new tsdp_ctx();
@@ -1296,6 +1310,10 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   INIT_TRY(cudaFuncSetAttribute(self_attn_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
   c->net[TSDP_BASE].cfg = cfg->base;
   c->net[TSDP_DRAFT].cfg = cfg->draft;
+  if (cfg->draft.arch == TSDP_ARCH_FROZEN) {      // nothing to load; its drafts cost a base forward per round, not drafter calls
+    c->net[TSDP_DRAFT].loaded = true;
+    c->cfg.draft_nfe = 0.f;
+  }
   for (int w = 0; w < 2; ++w) {      // conv-UNet activations: one zero-padded tensor per named stage
     Net& n = c->net[w];
     if (n.cfg.arch != TSDP_ARCH_UNET) continue;
@@ -1371,6 +1389,7 @@ int tsdp_load_weights(tsdp_ctx* c, int which, const float* blob, size_t n) {
   CU_TRY(c, cudaSetDevice(c->cfg.device));
   Net& net = c->net[which];
   const tsdp_config_t& cfg = c->cfg;
+  if (net.cfg.arch == TSDP_ARCH_FROZEN) return TSDP_ERR_ARG;      // frozen target drafts have no weights
   if (n != weights_count(cfg, net.cfg)) return TSDP_ERR_WEIGHTS;
   for (size_t i = 0; i < n; ++i)
     if (!std::isfinite(blob[i])) return TSDP_ERR_NAN;
@@ -2064,7 +2083,9 @@ int tsdp_stats(tsdp_ctx* c, tsdp_stats_t* out) {
   out->rejections = ds.rejections;
   out->bonus_steps = ds.bonus_steps;
   out->steps_advanced = ds.steps_advanced;
+  out->draft_rounds = ds.draft_rounds;
   out->nfe = (double)ds.env_rounds + (double)c->cfg.draft_nfe * (double)ds.draft_evals;
+  if (c->cfg.draft.arch == TSDP_ARCH_FROZEN) out->nfe = (double)ds.env_rounds + (double)ds.draft_rounds;
   for (int i = 0; i < TSDP_MAX_T; ++i) {
     out->hist_drafted[i] = ds.hist_drafted[i];
     out->hist_tested[i] = ds.hist_tested[i];

@@ -17,15 +17,19 @@ def setup(wl, max_B, max_K, seed=1, use_graph=1, draft_is_base=False, precision=
                               wl["base"] if draft_is_base else wl["draft"], T=wl["T"], max_B=max_B, max_K=max_K,
                               precision=prec, use_graph=use_graph, clip=clip, drafter=drafter, verifier=verifier)
     S = ddpm.Schedule(wl["T"], 1e-4, 0.02)
+    frozen = wl["draft"]["arch"] == "frozen" and not draft_is_base
     if wl["base"]["arch"] == "gauss":
-        pb, pd = wl["base_params"], wl["draft_params"]
+        pb, pd = wl["base_params"], wl.get("draft_params")
     else:
         pb = inputs.make_net(seed, wl, "base", bf16=(prec == 1))
-        pd = pb if draft_is_base else inputs.make_net(seed + 1, wl, "draft", bf16=(prec == 1))
+        pd = pb if (draft_is_base or frozen) else inputs.make_net(seed + 1, wl, "draft", bf16=(prec == 1))
     smp = binding.Sampler(cfg)
     smp.load_weights(binding.BASE, pb)
+    base = nets.make_denoiser(pb, S)
+    if frozen:      # drafter-free: nothing to load, the oracle's drafter wraps its base
+        return smp, S, base, spec.FrozenTargetDraft(base)
     smp.load_weights(binding.DRAFT, pd)
-    return smp, S, nets.make_denoiser(pb, S), nets.make_denoiser(pd, S)
+    return smp, S, base, nets.make_denoiser(pd, S)
 
 
 def accept_t(mode=0, lam=1.0, sigma_scale=1.0, bonus=1):

@@ -168,6 +168,56 @@ def test_request_counters_and_process_reward_match_oracle():
     smp.close()
 
 
+def _frozen(wl):
+    return dict(wl, draft=dict(arch="frozen"))
+
+
+def test_frozen_target_drafts_round_parity():
+    """Drafter-free rounds (every draft reuses the base output at the round's start) against the oracle: fp32 MLP,
+    bf16 transformer with the layer-by-layer kernels, and with the cluster kernel supplying both base passes."""
+    _round_parity(_frozen(inputs.WORKLOADS["toy_mlp"]), 6, 4, hp.accept_t(), 11, 1e-4, 2e-5, [99, 60, 30, 2, 1, 0])
+    wl = _frozen(dict(inputs.WORKLOADS["pusht_xfmr"], gamma=1.0))
+    _round_parity(wl, 3, 6, hp.accept_t(), 7, 2e-2, 3e-3, [99, 40, 3], precision=1, verifier=1)
+    _round_parity(wl, 2, 4, hp.accept_t(), 8, 2e-2, 3e-3, [80, 20], precision=1, verifier=2)
+
+
+def test_frozen_target_drafts_chunk_and_accounting():
+    wl = _frozen(inputs.WORKLOADS["toy_mlp"])
+    B, K, seed = 8, 5, 21
+    smp, S, base, draft = hp.setup(wl, max_B=B, max_K=K)
+    shape = (wl["H"], wl["A"])
+    obs = inputs.make_obs(4, B, wl["To"], wl["Do"])
+    dobs = torch.tensor(obs, dtype=torch.float32, device="cuda")
+    out = torch.zeros(B, *shape, device="cuda")
+    acc = hp.accept_t()
+    # K = 1: the only draft is the base model's own step -> vanilla DDPM, sample by sample
+    van = torch.zeros_like(out)
+    smp.sample_chunk(dobs, B, 0, acc, seed, van)
+    smp.reset_stats()
+    smp.sample_chunk(dobs, B, 1, acc, seed, out)
+    st = smp.stats()
+    assert torch.equal(out, van) and st["rejections"] == 0 and st["drafts_accepted"] == st["draft_evals"]
+    # K = 5 against the oracle, and the NFE rule: one batched verification per round plus one base pass per drafting round
+    smp.reset_stats()
+    smp.sample_chunk(dobs, B, K, acc, seed, out)
+    st = smp.stats()
+    got = out.cpu().numpy()
+    n_match, rounds, drounds = 0, 0, 0
+    for b in range(B):
+        xo, so = spec.sample_chunk(S, base, draft, spec.PhiloxNoise(seed), b, obs[b], shape, K, hp.oracle_accept(acc))
+        ok = np.max(np.abs(got[b] - xo)) < 3e-2
+        n_match += ok
+        rounds += so["rounds"]; drounds += so["draft_rounds"]
+    assert n_match >= B - 1
+    if n_match == B:
+        assert st["env_rounds"] == rounds and st["draft_rounds"] == drounds
+    assert abs(st["nfe"] - (st["env_rounds"] + st["draft_rounds"])) < 1e-9 and st["steps_advanced"] == 100 * B
+    # the frozen drafter takes no weights
+    with pytest.raises(binding.TsdpError):
+        smp.load_weights(binding.DRAFT, inputs.make_net(3, inputs.WORKLOADS["toy_mlp"], "draft"))
+    smp.close()
+
+
 def test_chunk_toy_mlp_fp32_matches_oracle_exactly_in_structure():
     wl = dict(inputs.WORKLOADS["toy_mlp"])
     B = 8

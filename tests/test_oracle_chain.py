@@ -84,6 +84,25 @@ def test_chunk_accounting():
         assert np.all(st["acc_hist"] <= st["test_hist"]) and np.all(st["test_hist"] <= st["prop_hist"])
 
 
+def test_frozen_target_drafts_first_step_is_the_base_step():
+    """Drafts that reuse the base output at the round's start: draft 1 IS the base model's reverse step (same eps,
+    same posterior), so mu^_1 = mu_1 bit for bit, log alpha_1 = 0 and it is accepted whatever the uniform; K = 1
+    therefore reproduces vanilla DDPM sample by sample, and every round with a draft costs one extra base call."""
+    base, _, obs, shape = _toy_nets()
+    fd = spec.FrozenTargetDraft(base)
+    x0 = spec.PhiloxNoise(1).x_init(0, shape)
+    _, _, d = spec.spec_round(S, base, fd, spec.PhiloxNoise(1), 0, obs, x0, 70, 5, spec.Accept())
+    assert np.array_equal(d["mu_hat"][1], d["mu"][1]) and d["log_alpha"][0] == 0.0 and d["flags"][0]
+    assert d["n_extra"] == 1 and d["jstar"] >= 2
+    assert any(np.max(np.abs(d["mu_hat"][k] - d["mu"][k])) > 0 for k in range(2, 6))      # later drafts do drift
+    ref = spec.sample_vanilla(S, base, spec.PhiloxNoise(5), 2, obs, shape)
+    x, st = spec.sample_chunk(S, base, fd, spec.PhiloxNoise(5), 2, obs, shape, 1, spec.Accept())
+    assert np.array_equal(x, ref) and st["rejections"] == 0
+    x, st = spec.sample_chunk(S, base, fd, spec.PhiloxNoise(5), 2, obs, shape, 6, spec.Accept())
+    assert st["extra_base"] == st["draft_rounds"] and st["accepted"] + st["rejections"] + st["bonus"] == 100
+    assert st["rounds"] - st["draft_rounds"] <= 1                  # only the round at t = 0 drafts nothing
+
+
 # ----------------------------------------------------------------------------- KS pin (10^5 chains)
 M0, S0 = 0.7, 0.5
 
@@ -114,6 +133,8 @@ def _run_block(args):
     kind, env0, n = args
     base = nets.make_denoiser(inputs.make_gauss_params(M0, S0), S)
     draft = nets.make_denoiser(inputs.make_gauss_params(M0 + 0.25, 0.8 * S0), S)
+    if kind == "frozen":
+        draft = spec.FrozenTargetDraft(base)
     envs = list(range(env0, env0 + n))
     noise = spec.TableNoise(1234, envs, 100, 1)
     out = np.empty(n); acc = tested = 0
@@ -126,9 +147,9 @@ def _run_block(args):
     return out, acc, tested
 
 
-@pytest.mark.parametrize("kind", ["vanilla", "speculative"])
+@pytest.mark.parametrize("kind", ["vanilla", "speculative", "frozen"])
 def test_gaussian_toy_matches_analytic_marginal(kind):
-    N, blk = 100_000, 2_500
+    N, blk = (40_000 if kind == "frozen" else 100_000), 2_500
     jobs = [(kind, e0, blk) for e0 in range(0, N, blk)]
     with ProcessPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as ex:
         res = list(ex.map(_run_block, jobs))

@@ -134,7 +134,8 @@ def make_sampler(wl, B, device, use_graph=1):
                               max_K=max_K, precision=wl["precision"], device=device, use_graph=use_graph)
     smp = binding.Sampler(cfg)
     smp.load_weights(binding.BASE, inputs.make_net(1, wl, "base"))
-    smp.load_weights(binding.DRAFT, inputs.make_net(2, wl, "draft"))
+    if wl["draft"]["arch"] != "frozen":
+        smp.load_weights(binding.DRAFT, inputs.make_net(2, wl, "draft"))
     if "schedule" in wl:
         Ks, Ss = wl["schedule"]
         smp.set_schedule(Ks, [binding.AcceptT(0, 1.0, s, 1) for s in Ss])
@@ -168,6 +169,8 @@ def run_ours(args):
     torch.cuda.set_device(local)
     peaks = load_peaks()
     wl = workload_spec(args.workload, args.batch)
+    if args.drafter == "frozen":      # drafter-free variant: the base output at the round's start serves every draft
+        wl["draft"] = dict(arch="frozen")
     B, K = wl["B"], wl["K"]
     acc = binding.AcceptT(0, 1.0, 1.0, 1)
     smp = make_sampler(wl, B, local)
@@ -338,6 +341,7 @@ def run_ours(args):
                         l2="per-step working set (activations of all candidates) exceeds the 126 MB L2; no explicit flush"
                         if B * (K + 1) * wl["H"] * wl["base"].get("d", 0) * 16 > 126e6 else
                         "working set fits L2 by design (weights are reused across rounds); no explicit flush",
+                        drafter=("frozen target drafts (no drafter network)" if args.drafter == "frozen" else "network"),
                         parallelism=f"replicas x{world} (environments sharded, no collective)"))
         print(json.dumps(result))
     smp.close()
@@ -353,7 +357,8 @@ def oracle_chunk(wl, env, seed):
     from paper_2512_15773_b200 import inputs
     S = ddpm.Schedule(wl["T"], 1e-4, 0.02)
     base = nets.make_denoiser(inputs.make_net(1, wl, "base"), S)
-    draft = nets.make_denoiser(inputs.make_net(2, wl, "draft"), S)
+    draft = (spec.FrozenTargetDraft(base) if wl["draft"]["arch"] == "frozen"
+             else nets.make_denoiser(inputs.make_net(2, wl, "draft"), S))
     obs = inputs.make_obs(100, env + 1, wl["To"], wl["Do"])[env]
     sched = None
     if "schedule" in wl:
@@ -426,6 +431,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="serving_xfmr", choices=["serving_xfmr", "pusht_xfmr", "toy_mlp", "vla_dit", "robomimic_unet"])
     ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--drafter", default="net", choices=["net", "frozen"],
+                    help="net: the workload's drafter network; frozen: no drafter, drafts reuse the base output at the round's start")
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
     ap.add_argument("--no-latency", dest="latency", action="store_false")
     ap.add_argument("--only-timed", action="store_true",

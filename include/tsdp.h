@@ -252,6 +252,22 @@ int tsdp_request_counts(tsdp_ctx* ctx, int* h_counts, int n);
  * reward needs the simulator and is the caller's.  Errors: ARG (n, T_max < 1, dt < 1), CUDA. */
 int tsdp_process_reward(tsdp_ctx* ctx, float R_final, int T_max, int dt, float* h_reward, int n);
 
+/* Distillation objective of the drafter against the frozen base model (Sec. 3.2, "Draft model"), forward
+ * evaluation only (no parameter update: training is outside this library).  For sample n < N (<= max_B) the
+ * clean chunk d_x0[n] ([N, H, A] DEVICE) is noised at a timestep t_n = floor(T u_n) with Gaussian noise eps_n,
+ * both from the counter-based generator (u_n: the uniform of (seed, n, timestep code 0); eps_n: the initial-latent
+ * normals of (seed, n)):  x_t = sqrt(abar_t) x0 + sqrt(1 - abar_t) eps.  Both networks are run on (x_t, t_n,
+ * d_obs[n]) and
+ *     L_pred = mean_n |m^ - m|^2                       (m, m^: outputs of base and drafter; norm over H*A),
+ *     L_norm = mean over samples with t_n >= 1 of |(mu^ - mu) / sigma_t|^2   (posterior means; sigma_0 = 0),
+ *     L      = lambda1 L_pred + lambda2 L_norm.
+ * h_out[4] (HOST, double) = {L_pred, L_norm, L, mean over t_n >= 1 of 2 Phi(-|d|/2)}; the last value is the
+ * probability that the acceptance test of Sec. 3.1 takes a draft whose mean is off by d = (mu^ - mu)/sigma_t.
+ * Uses the round's work buffers: call between chunks.  Synchronous.  Errors: ARG (N, null pointers, a
+ * TSDP_ARCH_FROZEN drafter), STATE (weights not loaded), TOO_LARGE, CUDA. */
+int tsdp_distill_loss(tsdp_ctx* ctx, const float* d_x0, const float* d_obs, int N, uint64_t seed, float lambda1,
+                      float lambda2, double* h_out);
+
 /* Copy the counters accumulated since the last reset (synchronises the device). */
 int tsdp_stats(tsdp_ctx* ctx, tsdp_stats_t* out);
 int tsdp_reset_stats(tsdp_ctx* ctx);

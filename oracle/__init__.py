@@ -25,5 +25,12 @@ Pin status (what checks each part against something other than itself):
               separate encoders, the aggregating MLP and the five outputs, but no sizes, weights
               or ranges); pinned by structure: zero network, output ranges, stream separation,
               a hand-computed path, the stage boundaries.
+              The intermediate reward of Sec. 3.3 (process_reward) is pinned by worked values and by
+              the accumulated-reward identity the paper states for its scaling factor.
+  distill.py  pinned  : zero for equal networks, the closed form for a constant output offset
+                        (with the printed values c_50 = 0.2145, c_1 = 1.735 of the linear schedule),
+                        linearity in (lambda1, lambda2), the Gaussian-overlap integral.
+  spec.FrozenTargetDraft  parity unpinned against the prior work that Sec. 2.2 cites (only named
+              there); pinned by: first draft exact, K = 1 == vanilla, the Gaussian chain's marginal.
   sigma_scale parity unpinned against the paper (formula not given there).
 """

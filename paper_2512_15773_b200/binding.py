@@ -16,7 +16,7 @@ EXPORTS = ["tsdp_init", "tsdp_destroy", "tsdp_strerror", "tsdp_last_error", "tsd
            "tsdp_load_weights", "tsdp_set_schedule", "tsdp_sample_chunk", "tsdp_sample_chunk_host",
            "tsdp_round", "tsdp_denoise", "tsdp_gemm", "tsdp_gemm_timed", "tsdp_stats", "tsdp_reset_stats",
            "tsdp_kernel_launches", "tsdp_profile", "tsdp_profile_read", "tsdp_verify_commit_static", "tsdp_set_scheduler", "tsdp_set_progress",
-           "tsdp_sched_eval", "tsdp_serve", "tsdp_request_counts", "tsdp_process_reward"]
+           "tsdp_sched_eval", "tsdp_serve", "tsdp_request_counts", "tsdp_process_reward", "tsdp_distill_loss"]
 PROF_FAMILIES = ["gemm", "layernorm", "attention", "embed_head", "round", "small_net", "gemm_draft", "drafter_cluster", "accept", "verifier_cluster"]
 
 
@@ -83,6 +83,7 @@ def load_library():
     lib.tsdp_set_progress.argtypes = [vp, fp, i]
     lib.tsdp_sched_eval.argtypes = [vp, fp, fp, fp, i, fp, vp]
     lib.tsdp_request_counts.argtypes = [vp, vp, i]
+    lib.tsdp_distill_loss.argtypes = [vp, fp, fp, i, u64, C.c_float, C.c_float, vp]
     lib.tsdp_process_reward.argtypes = [vp, C.c_float, i, i, fp, i]
     lib.tsdp_stats.argtypes = [vp, C.POINTER(StatsT)]
     lib.tsdp_reset_stats.argtypes = [vp]
@@ -222,6 +223,13 @@ class Sampler:
         self._check(self.lib.tsdp_sched_eval(self.h, _ptr(d_obs), _ptr(d_prev_actions), prog.ctypes.data, B,
                                              out.ctypes.data, 0), "tsdp_sched_eval")
         return out
+
+    def distill_loss(self, d_x0, d_obs, N, seed, lambda1=1.0, lambda2=1.0):
+        """(L_pred, L_norm, L, mean acceptance probability) of the drafter against the base on N noised chunks."""
+        out = np.zeros(4, dtype=np.float64)
+        self._check(self.lib.tsdp_distill_loss(self.h, _ptr(d_x0), _ptr(d_obs), N, seed, lambda1, lambda2, out.ctypes.data),
+                    "tsdp_distill_loss")
+        return tuple(float(v) for v in out)
 
     def request_counts(self, n):
         """[n, 4] int32 per request of the last call: drafts proposed, drafts accepted, rounds, reverse steps taken."""

@@ -25,6 +25,7 @@
 #include "unet_kernels.cuh"
 #include "xattn_fold.cuh"
 #include "draft_tail.cuh"
+#include "distill_kernels.cuh"
 
 using namespace tsdp;
 
@@ -2020,6 +2021,52 @@ int tsdp_denoise(tsdp_ctx* c, int which, const float* d_x, const int* h_tau, con
   c->launches += c->launches_per_round_tmp;
   CU_TRY(c, cudaStreamSynchronize(s));
   return check_status(c);
+}
+
+int tsdp_distill_loss(tsdp_ctx* c, const float* d_x0, const float* d_obs, int N, uint64_t seed, float lambda1, float lambda2,
+                      double* h_out) {
+  if (!c || !d_x0 || !h_out || N < 1 || N > c->cfg.max_B || c->cfg.draft.arch == TSDP_ARCH_FROZEN) return TSDP_ERR_ARG;
+  const size_t obs_n = (size_t)N * c->cfg.obs_tokens * c->cfg.obs_dim;
+  if (obs_n > 0 && !d_obs) return TSDP_ERR_ARG;
+  if (!c->net[0].loaded || !c->net[1].loaded) return TSDP_ERR_STATE;
+  CU_TRY(c, cudaSetDevice(c->cfg.device));
+  cudaStream_t s = nullptr;
+  const int D = c->D;
+  const long long xs_b = (long long)(c->cfg.max_K + 1) * D;
+  int r;
+  {   // requests beyond the slots' initial capacity are not involved: sample n uses slot n and request n
+    if ((r = ensure_items(c, (size_t)N))) return r;
+  }
+  if (obs_n) CU_TRY(c, cudaMemcpyAsync(c->obs, d_obs, obs_n * sizeof(float), cudaMemcpyDeviceToDevice, s));
+  CU_TRY(c, cudaMemcpyAsync(c->seed, &seed, sizeof(seed), cudaMemcpyHostToDevice, s));
+  distill_noise_kernel<<<N, 128, 0, s>>>(c->S, d_x0, c->xt, xs_b, c->t, D, c->seed);
+  CU_TRY(c, cudaGetLastError());
+  c->launches_per_round_tmp = 1;
+  if ((r = prepare_obs(c, c->net[TSDP_BASE], N, s))) return r;
+  if ((r = prepare_obs(c, c->net[TSDP_DRAFT], N, s))) return r;
+  CandMap cb{c->xt, xs_b, c->eps, xs_b, c->t, 1, 0, nullptr};
+  if ((r = forward(c, c->net[TSDP_BASE], cb, N, s))) return r;
+  CandMap cd{c->xt, xs_b, c->eps_d, (long long)D, c->t, 1, 0, nullptr};
+  if ((r = forward(c, c->net[TSDP_DRAFT], cd, N, s))) return r;
+  float* terms = c->muhat;                       // [N, 3] per-sample terms; the drafter means are not in use here
+  if ((size_t)3 * N > (size_t)c->cfg.max_B * (c->cfg.max_K > 0 ? c->cfg.max_K : 1) * D) return TSDP_ERR_TOO_LARGE;
+  distill_terms_kernel<<<N, 128, 0, s>>>(c->S, c->xt, xs_b, c->eps, xs_b, c->eps_d, (long long)D, c->t, D, terms);
+  CU_TRY(c, cudaGetLastError());
+  c->launches += c->launches_per_round_tmp + 1;
+  std::vector<float> h((size_t)3 * N);
+  CU_TRY(c, cudaMemcpyAsync(h.data(), terms, sizeof(float) * 3 * N, cudaMemcpyDeviceToHost, s));
+  CU_TRY(c, cudaStreamSynchronize(s));
+  if ((r = check_status(c))) return r;
+  double sp = 0.0, sn = 0.0, sa = 0.0, cnt = 0.0;
+  for (int n = 0; n < N; ++n) {
+    sp += h[3 * n];
+    if (h[3 * n + 2] > 0.f) { sn += h[3 * n + 1]; sa += erfc(sqrt((double)h[3 * n + 1]) / (2.0 * sqrt(2.0))); cnt += 1.0; }
+  }
+  h_out[0] = sp / N;
+  h_out[1] = cnt > 0 ? sn / cnt : 0.0;
+  h_out[2] = (double)lambda1 * h_out[0] + (double)lambda2 * h_out[1];
+  h_out[3] = cnt > 0 ? sa / cnt : 1.0;
+  return TSDP_OK;
 }
 
 int tsdp_gemm(tsdp_ctx* c, const void* d_A, const void* d_W, const float* d_bias, int M, int N, int K, int epi,

@@ -326,6 +326,16 @@ def run_ours(args):
                        nfe_per_chunk=st1["nfe"] / 64, drafter="persistent cluster kernel", verifier="cluster kernel, one cluster per candidate",
                        drafter_us_per_draft_step=draft_us)
             s1.close()
+            # the same chunks with frozen-target drafts (no drafter network: the base output at the round's start is reused)
+            s2 = make_sampler(dict(wl1, draft=dict(arch="frozen")), 1, local)
+            time_steps(s2, o1, a1, 1, wl1["K"], acc, list(range(8)))
+            s2.reset_stats()
+            tf = time_steps(s2, o1, a1, 1, wl1["K"], acc, list(range(100, 164)))
+            st2 = s2.stats()
+            lat["frozen_target_drafts"] = dict(p50_chunk_ms=float(np.median(tf)), p99_chunk_ms=float(np.percentile(tf, 99)),
+                                               acceptance=st2["drafts_accepted"] / max(st2["draft_evals"], 1),
+                                               rounds_per_chunk=st2["env_rounds"] / 64, nfe_per_chunk=st2["nfe"] / 64)
+            s2.close()
         cpu = cpu_baseline(wl, budget_s=args.cpu_seconds) if world == 1 else None
         result.update(
             accepted_denoise_steps_per_s=acc_steps / (total_ms / 1e3),

@@ -367,6 +367,31 @@ def test_gaussian_toy_on_gpu_matches_analytic_marginal():
     smp.close()
 
 
+def test_gaussian_toy_with_frozen_target_drafts_keeps_the_marginal_on_gpu():
+    """Drafter-free rounds are lossless too: 10^5 chains on the GPU against the analytic marginal, and a few of them
+    sample by sample against the oracle; rejections do occur (the frozen output drifts from the base's)."""
+    from tests.test_oracle_chain import _analytic_marginal, M0, S0
+    from oracle import ddpm, nets
+    B = 100_000
+    wl = dict(H=1, A=1, To=0, Do=0, T=100, precision=0, base=dict(arch="gauss"), draft=dict(arch="frozen"),
+              base_params=inputs.make_gauss_params(M0, S0))
+    smp, *_ = hp.setup(wl, max_B=B, max_K=6)
+    mean, std = _analytic_marginal()
+    out = torch.zeros(B, 1, 1, device="cuda")
+    smp.reset_stats()
+    smp.sample_chunk(None, B, 6, hp.accept_t(), 1234, out)
+    x = out.cpu().numpy().reshape(-1).astype(np.float64)
+    assert stats.kstest((x - mean) / std, "norm").pvalue > 0.01
+    st = smp.stats()
+    assert st["rejections"] > 0 and st["drafts_accepted"] < st["drafts_tested"] and st["steps_advanced"] == 100 * B
+    S = ddpm.Schedule()
+    base = nets.make_denoiser(wl["base_params"], S)
+    for b in (0, 7, 99_999):
+        xo, _ = spec.sample_chunk(S, base, spec.FrozenTargetDraft(base), spec.PhiloxNoise(1234), b, None, (1, 1), 6, spec.Accept())
+        assert abs(x[b] - xo[0, 0]) < 1e-3
+    smp.close()
+
+
 def test_argument_errors_on_device():
     wl = dict(inputs.WORKLOADS["toy_mlp"])
     cfg = binding.make_config(wl["H"], wl["A"], wl["To"], wl["Do"], wl["base"], wl["draft"], max_B=2, max_K=4, precision=0)

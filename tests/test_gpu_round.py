@@ -72,6 +72,14 @@ def test_round_transformer_bf16_both_drafters(drafter):
                   drafter=drafter)
 
 
+def test_cluster_kernels_without_the_cross_attention_fold(monkeypatch):
+    """The cluster kernel's own query / output projections and attention over the memory tokens (what it runs when
+    (1 + obs_tokens) * heads exceeds its 16 folded rows), selected here through the environment variable."""
+    monkeypatch.setenv("TSDP_NO_FOLD", "1")
+    wl = dict(inputs.WORKLOADS["pusht_xfmr"], precision=1)
+    _round_parity(wl, 2, 8, hp.accept_t(), 21, 2e-2, 3e-3, [99, 40], drafter=2, verifier=2)
+
+
 @pytest.mark.parametrize("case", ["resident", "streamed"])
 def test_cluster_drafter_matches_layered_drafter(case):
     """resident: the PushT drafter, whose weight slices live in shared memory; streamed: a 4-block d = 256

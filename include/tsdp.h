@@ -20,6 +20,8 @@
  * into its memory tokens (the query and output projections are applied once to the time / observation tokens
  * instead of to every token row) when H <= 16, (1 + obs_tokens) * heads <= 32, heads is even and d is 128, 256
  * or 512; TSDP_NO_FOLD, set before tsdp_load_weights, keeps the separate kernels.  Same function either way.
+ * TSDP_NO_ASYNC_BCAST (read at every round) makes the cluster kernel hand its stages over with plain distributed-
+ * shared-memory stores and a cluster barrier instead of st.async stores counted by mbarriers.
  * TSDP_GEMM_BN = 32 | 64 | 128 | 256 (read by tsdp_init) forces that tile width on every tensor-core GEMM whose
  * output width it divides -- a tuning aid; results do not depend on the tile width.
  * Every function returns a tsdp_status; nothing throws or aborts.  A context is not re-entrant: one

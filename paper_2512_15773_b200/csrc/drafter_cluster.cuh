@@ -9,9 +9,15 @@
 // and each CTA writes its slice of Y into the replicas of all CTAs through distributed shared
 // memory; one hardware cluster barrier separates dependent stages (6 per block).  LayerNorm, the two
 // attentions, the head, the DDPM posterior and the noise are cheap enough to be recomputed by every
-// CTA, which saves their broadcasts.  Reductions are warp shuffles.  Nothing spins on memory: the
-// only waits are __syncthreads and barrier.cluster, which all CTAs of a cluster reach the same
-// number of times because the control flow depends only on (t[b], k).
+// CTA, which saves their broadcasts.  Reductions are warp shuffles.
+// A stage's slices travel as 16-byte st.async stores that also count their bytes on an mbarrier of the receiving
+// CTA; a CTA goes on as soon as the bytes of all eight slices have arrived (a bounded mbarrier wait), with no
+// release fence and no cluster-wide barrier per stage.  Two mbarriers alternate between consecutive stages: a CTA
+// can run at most one stage ahead of the slowest one (it needs everybody's slice of the previous stage), so the
+// bytes of stage s + 1 never land on the barrier that still counts stage s.  The same reasoning covers the
+// buffers: what a fast CTA writes remotely in stage s + 1 is never what a slower one still reads in stage s.
+// (TSDP_NO_ASYNC_BCAST selects plain distributed-shared-memory stores and barrier.cluster instead.)
+// All CTAs of a cluster make the same sequence of stages because the control flow depends only on (t[b], k).
 #pragma once
 #include <cooperative_groups.h>
 #include "common.cuh"
@@ -28,6 +34,19 @@ constexpr int DC_ROWS = 16;       // one m16 tile: H <= 16
 constexpr int DC_MAX_LAYERS = 8;
 constexpr int DC_MAX_NK = 4;      // memory tokens: time token + at most 3 observation tokens
 constexpr int DC_PU = 40;         // folded cross-attention: row pitch (bf16) of the [.. x 32] operands of its second product
+
+__device__ __forceinline__ uint32_t dc_mapa(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void dc_st_async16(uint32_t remote, const uint4& v, uint32_t remote_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1,%2,%3,%4}, [%5];"
+               ::"r"(remote), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"(remote_bar) : "memory");
+}
+__device__ __forceinline__ void dc_st_cluster16(uint32_t remote, const uint4& v) {
+  asm volatile("st.shared::cluster.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(remote), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
 
 template <int BYTES>
 __device__ __forceinline__ void dc_cp_async(void* smem_dst, const void* gsrc) {
@@ -53,6 +72,8 @@ struct DcParams {
   const __nv_bfloat16 *kq_time, *ut_time, *kq_obs, *ut_obs;
   const float *c_time, *c_obs;
   int fold;
+  int async_bcast;                                           // 1: slices travel by st.async and are counted by the receivers' mbarriers
+  int* status;                                               // set to 5 if a wait gives up
   DdpmTables S;
   float* xt; long long xs_b;                                 // candidates [B, Kmax+1, D]
   float* muhat; long long ms_b;                              // drafter means [B, Kmax, D]
@@ -341,6 +362,48 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
   const int cid = blockIdx.x / DC_CS, ncl = gridDim.x / DC_CS;
+  // stage hand-over: two mbarriers that count the bytes of the slices arriving in this CTA (see the file header)
+  __shared__ __align__(8) uint64_t dc_bar[2];
+  const bool use_async = P.async_bcast != 0;
+  const uint32_t bar_addr[2] = {ptx::smem_u32(&dc_bar[0]), ptx::smem_u32(&dc_bar[1])};
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(bar_addr[0], 1);
+    ptx::mbar_init(bar_addr[1], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  uint32_t stage_no = 0, stage_phase = 0;      // stages so far; bit b = parity this CTA waits for next on barrier b
+  // thread 0 announces the bytes this CTA will receive in the stage that begins
+  auto stage_begin = [&](uint32_t bytes) {
+    if (use_async && threadIdx.x == 0)
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_addr[stage_no & 1u]), "r"(bytes) : "memory");
+  };
+  // 16 bytes to the same shared-memory address in every CTA of the cluster
+  auto bcast16 = [&](const void* local_ptr, const uint4& v) {
+    const uint32_t la = ptx::smem_u32(local_ptr);
+    if (use_async) {
+      const uint32_t lb = bar_addr[stage_no & 1u];
+#pragma unroll 1
+      for (uint32_t r = 0; r < DC_CS; ++r) dc_st_async16(dc_mapa(la, r), v, dc_mapa(lb, r));
+    } else {
+#pragma unroll 1
+      for (uint32_t r = 0; r < DC_CS; ++r) dc_st_cluster16(dc_mapa(la, r), v);
+    }
+  };
+  // every slice of the stage has arrived in this CTA (bounded wait), or, without st.async, the cluster barrier
+  auto stage_end = [&]() {
+    if (use_async) {
+      const uint32_t b = stage_no & 1u, par = (stage_phase >> b) & 1u;
+      uint32_t done = 0;
+      for (int it = 0; it < (1 << 24) && !done; ++it)
+        asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                     : "=r"(done) : "r"(bar_addr[b]), "r"(par) : "memory");
+      if (!done && threadIdx.x == 0) atomicExch(P.status, 5);
+      stage_phase ^= 1u << b;
+      ++stage_no;
+    } else {
+      cluster.sync();
+    }
+  };
   constexpr int d = D_MODEL;
   constexpr int PA = d + 8, PQKV = 3 * d + 8, PF = 4 * d + 8;
   const bool resident = P.resident != 0;
@@ -447,15 +510,15 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
       // ---- causal self-attention
       dc_layernorm<d>(h, W.ln1_g, W.ln1_b, a, PA);
       __syncthreads();
+      stage_begin(DC_ROWS * 3 * d * 2);
       dc_linear<d>(a, PA, w_ptr(l, 0), PWD, NS_3D, red, [&](int row, int col, float* v) {
         const int cg_ = rank * NS_3D + col;
         const float4 b0 = *reinterpret_cast<const float4*>(W.bqkv + col), b1 = *(reinterpret_cast<const float4*>(W.bqkv + col) + 1);
         v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
         const uint4 pk = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
-#pragma unroll 1
-        for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(cluster.map_shared_rank(qkv, r) + row * PQKV + cg_) = pk;
+        bcast16(qkv + row * PQKV + cg_, pk);
       });
-      cluster.sync();
+      stage_end();
       switch (d / P.heads) {
         case 32: dc_self_attn_mma<d, 32>(qkv, PQKV, a, PA, P.heads, H); break;
         case 64: dc_self_attn_mma<d, 64>(qkv, PQKV, a, PA, P.heads, H); break;
@@ -496,6 +559,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
       }
+      stage_begin(DC_ROWS * d * 4);
       dc_linear<d>(a, PA, w_ptr(l, 1), PWD, NS_D, red, [&](int row, int col, float* v) {
         const int cg_ = rank * NS_D + col;
         const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
@@ -503,11 +567,8 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         const float4 b0 = *reinterpret_cast<const float4*>(W.bo + col), b1 = *(reinterpret_cast<const float4*>(W.bo + col) + 1);
         const float4 o0 = make_float4(h0.x + v[0] + b0.x, h0.y + v[1] + b0.y, h0.z + v[2] + b0.z, h0.w + v[3] + b0.w);
         const float4 o1 = make_float4(h1.x + v[4] + b1.x, h1.y + v[5] + b1.y, h1.z + v[6] + b1.z, h1.w + v[7] + b1.w);
-#pragma unroll 1
-        for (int r = 0; r < DC_CS; ++r) {
-          float4* dst = reinterpret_cast<float4*>(cluster.map_shared_rank(h, r) + row * d + cg_);
-          dst[0] = o0; dst[1] = o1;
-        }
+        bcast16(h + row * d + cg_, make_uint4(__float_as_uint(o0.x), __float_as_uint(o0.y), __float_as_uint(o0.z), __float_as_uint(o0.w)));
+        bcast16(h + row * d + cg_ + 4, make_uint4(__float_as_uint(o1.x), __float_as_uint(o1.y), __float_as_uint(o1.z), __float_as_uint(o1.w)));
       });
       if (!resident && !P.fold) {   // keys / values of the memory tokens for this block only: time token of tau, then the obs tokens
         for (int i = threadIdx.x; i < NK * 2 * d; i += DC_THREADS) {
@@ -516,7 +577,8 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
           skv[i] = __ldg(src + (size_t)l * 2 * d + c);
         }
       }
-      cluster.sync();
+      stage_end();
+      if (use_async && !resident && !P.fold) __syncthreads();      // the keys / values above were written by other threads
       // ---- cross-attention to [time token | obs tokens]
       if (P.fold) {
         // Folded form: scores = xhat . kq + c, out = P . u + bo2, both so small that every CTA computes them whole
@@ -567,17 +629,18 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
       } else {
       dc_layernorm<d>(h, W.ln2_g, W.ln2_b, a, PA);
       __syncthreads();
+      stage_begin(DC_ROWS * d * 2);
       dc_linear<d>(a, PA, w_ptr(l, 2), PWD, NS_D, red, [&](int row, int col, float* v) {
         const int cg_ = rank * NS_D + col;
         const float4 b0 = *reinterpret_cast<const float4*>(W.bq2 + col), b1 = *(reinterpret_cast<const float4*>(W.bq2 + col) + 1);
         v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
         const uint4 pk = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
-#pragma unroll 1
-        for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(cluster.map_shared_rank(q2, r) + row * PA + cg_) = pk;
+        bcast16(q2 + row * PA + cg_, pk);
       });
-      cluster.sync();
+      stage_end();
       dc_attention<d, false>(q2, PA, nullptr, 0, skv + (size_t)(resident ? l : 0) * DC_MAX_NK * 2 * d, NK, a, PA, P.heads, H);
       __syncthreads();
+      stage_begin(DC_ROWS * d * 4);
       dc_linear<d>(a, PA, w_ptr(l, 3), PWD, NS_D, red, [&](int row, int col, float* v) {
         const int cg_ = rank * NS_D + col;
         const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
@@ -585,17 +648,15 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         const float4 b0 = *reinterpret_cast<const float4*>(W.bo2 + col), b1 = *(reinterpret_cast<const float4*>(W.bo2 + col) + 1);
         const float4 o0 = make_float4(h0.x + v[0] + b0.x, h0.y + v[1] + b0.y, h0.z + v[2] + b0.z, h0.w + v[3] + b0.w);
         const float4 o1 = make_float4(h1.x + v[4] + b1.x, h1.y + v[5] + b1.y, h1.z + v[6] + b1.z, h1.w + v[7] + b1.w);
-#pragma unroll 1
-        for (int r = 0; r < DC_CS; ++r) {
-          float4* dst = reinterpret_cast<float4*>(cluster.map_shared_rank(h, r) + row * d + cg_);
-          dst[0] = o0; dst[1] = o1;
-        }
+        bcast16(h + row * d + cg_, make_uint4(__float_as_uint(o0.x), __float_as_uint(o0.y), __float_as_uint(o0.z), __float_as_uint(o0.w)));
+        bcast16(h + row * d + cg_ + 4, make_uint4(__float_as_uint(o1.x), __float_as_uint(o1.y), __float_as_uint(o1.z), __float_as_uint(o1.w)));
       });
-      cluster.sync();
+      stage_end();
       }
       // ---- MLP
       dc_layernorm<d>(h, W.ln3_g, W.ln3_b, a, PA);
       __syncthreads();
+      stage_begin(DC_ROWS * 4 * d * 2);
       dc_linear<d>(a, PA, w_ptr(l, 4), PWD, NS_4D, red, [&](int row, int col, float* v) {
         const int cg_ = rank * NS_4D + col;
         const float4 b0 = *reinterpret_cast<const float4*>(W.b1 + col), b1 = *(reinterpret_cast<const float4*>(W.b1 + col) + 1);
@@ -604,10 +665,10 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         for (int j = 0; j < 8; ++j)
           v[j] = ptx::gelu_fast(v[j]);
         const uint4 pk = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
-#pragma unroll 1
-        for (int r = 0; r < DC_CS; ++r) *reinterpret_cast<uint4*>(cluster.map_shared_rank(f, r) + row * PF + cg_) = pk;
+        bcast16(f + row * PF + cg_, pk);
       });
-      cluster.sync();
+      stage_end();
+      stage_begin(DC_ROWS * d * 4);
       dc_linear<4 * d>(f, PF, w_ptr(l, 5), PW4, NS_D, red, [&](int row, int col, float* v) {
         const int cg_ = rank * NS_D + col;
         const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
@@ -615,13 +676,10 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         const float4 b0 = *reinterpret_cast<const float4*>(W.b2 + col), b1 = *(reinterpret_cast<const float4*>(W.b2 + col) + 1);
         const float4 o0 = make_float4(h0.x + v[0] + b0.x, h0.y + v[1] + b0.y, h0.z + v[2] + b0.z, h0.w + v[3] + b0.w);
         const float4 o1 = make_float4(h1.x + v[4] + b1.x, h1.y + v[5] + b1.y, h1.z + v[6] + b1.z, h1.w + v[7] + b1.w);
-#pragma unroll 1
-        for (int r = 0; r < DC_CS; ++r) {
-          float4* dst = reinterpret_cast<float4*>(cluster.map_shared_rank(h, r) + row * d + cg_);
-          dst[0] = o0; dst[1] = o1;
-        }
+        bcast16(h + row * d + cg_, make_uint4(__float_as_uint(o0.x), __float_as_uint(o0.y), __float_as_uint(o0.z), __float_as_uint(o0.w)));
+        bcast16(h + row * d + cg_ + 4, make_uint4(__float_as_uint(o1.x), __float_as_uint(o1.y), __float_as_uint(o1.z), __float_as_uint(o1.w)));
       });
-      cluster.sync();
+      stage_end();
     }
     // ---- head: eps = LN_f(h) W_out + b_out   (every CTA, rows w and w + 8 per warp)
     {

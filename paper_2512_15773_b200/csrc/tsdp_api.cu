@@ -961,6 +961,8 @@ int launch_cluster_forward(tsdp_ctx* c, int which, int mode, int B, int K, cudaS
   P.fold = (n.fold && (1 + c->cfg.obs_tokens) * n.cfg.heads <= 16) ? 1 : 0;     // the cluster kernel's buffers hold 16 (token, head) rows
   P.kq_time = n.fold_kq_time; P.ut_time = n.fold_ut_time; P.c_time = n.fold_c_time;
   P.kq_obs = n.fold_kq_obs; P.ut_obs = n.fold_ut_obs; P.c_obs = n.fold_c_obs;
+  P.status = c->status;
+  P.async_bcast = getenv("TSDP_NO_ASYNC_BCAST") == nullptr ? 1 : 0;
   P.S = c->S;
   P.xt = c->xt; P.xs_b = (long long)(c->cfg.max_K + 1) * c->D;
   P.muhat = c->muhat; P.ms_b = (long long)(c->cfg.max_K > 0 ? c->cfg.max_K : 1) * c->D;

@@ -72,6 +72,27 @@ def test_round_transformer_bf16_both_drafters(drafter):
                   drafter=drafter)
 
 
+def test_cluster_kernels_with_cluster_barriers_give_the_same_bits(monkeypatch):
+    """The two ways a cluster hands a stage over (st.async stores counted on mbarriers; plain distributed-shared-memory
+    stores and a cluster barrier) move the same values: a round must come out bit for bit the same."""
+    wl = dict(inputs.WORKLOADS["pusht_xfmr"], precision=1)
+    B, K, D = 3, 8, wl["H"] * wl["A"]
+    outs = []
+    for legacy in (False, True):
+        if legacy:
+            monkeypatch.setenv("TSDP_NO_ASYNC_BCAST", "1")
+        smp, *_ = hp.setup(wl, max_B=B, max_K=K, drafter=2, verifier=2)
+        obs = torch.tensor(inputs.make_obs(3, B, wl["To"], wl["Do"]), dtype=torch.float32, device="cuda")
+        x = torch.tensor(np.random.default_rng(0).normal(size=(B, D)).astype(np.float32), device="cuda")
+        h_t = np.array([90, 50, 3], dtype=np.int32)
+        xt = torch.zeros(B, K + 1, D, device="cuda"); mh = torch.zeros(B, K, D, device="cuda"); ep = torch.zeros(B, K + 1, D, device="cuda")
+        smp.round(obs, B, K, hp.accept_t(), 4, x, h_t, xt, mh, ep, None, None)
+        outs.append((xt.clone(), mh.clone(), ep.clone(), x.clone()))
+        smp.close()
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+
+
 def test_cluster_kernels_without_the_cross_attention_fold(monkeypatch):
     """The cluster kernel's own query / output projections and attention over the memory tokens (what it runs when
     (1 + obs_tokens) * heads exceeds its 16 folded rows), selected here through the environment variable."""

@@ -372,6 +372,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   uint32_t stage_no = 0, stage_phase = 0;      // stages so far; bit b = parity this CTA waits for next on barrier b
+  bool wait_failed = false;
   // thread 0 announces the bytes this CTA will receive in the stage that begins
   auto stage_begin = [&](uint32_t bytes) {
     if (use_async && threadIdx.x == 0)
@@ -393,11 +394,17 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
   auto stage_end = [&]() {
     if (use_async) {
       const uint32_t b = stage_no & 1u, par = (stage_phase >> b) & 1u;
-      uint32_t done = 0;
-      for (int it = 0; it < (1 << 24) && !done; ++it)
+      uint32_t done = wait_failed ? 1u : 0u;       // after one wait has given up the rest of the launch does not wait again
+      const long long t0 = clock64();
+      while (!done) {
         asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
                      : "=r"(done) : "r"(bar_addr[b]), "r"(par) : "memory");
-      if (!done && threadIdx.x == 0) atomicExch(P.status, 5);
+        if (!done && clock64() - t0 > GEMM_WAIT_CYCLES) {      // about a second: report, and run to the end without waiting
+          wait_failed = true;
+          if (threadIdx.x == 0) atomicExch(P.status, 5);
+          break;
+        }
+      }
       stage_phase ^= 1u << b;
       ++stage_no;
     } else {

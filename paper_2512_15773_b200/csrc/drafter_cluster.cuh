@@ -7,9 +7,10 @@
 // and a full replica of the activations of the 16-token sequence.  A linear layer
 // is computed as Y[:, slice] = X W_slice^T on mma.sync m16n8k16 (the sequence is one 16-row tile),
 // and each CTA writes its slice of Y into the replicas of all CTAs through distributed shared
-// memory; one hardware cluster barrier separates dependent stages (6 per block).  LayerNorm, the two
-// attentions, the head, the DDPM posterior and the noise are cheap enough to be recomputed by every
-// CTA, which saves their broadcasts.  Reductions are warp shuffles.
+// memory (4 such exchanges per block: qkv, attention projection, MLP up, MLP down; 6 when the
+// cross-attention is not folded into the memory tokens).  LayerNorm, the attentions, the folded
+// cross-attention products, the head, the DDPM posterior and the noise are cheap enough to be
+// recomputed by every CTA, which saves their broadcasts.  Reductions are warp shuffles.
 // A stage's slices travel as 16-byte st.async stores that also count their bytes on an mbarrier of the receiving
 // CTA; a CTA goes on as soon as the bytes of all eight slices have arrived (a bounded mbarrier wait), with no
 // release fence and no cluster-wide barrier per stage.  Two mbarriers alternate between consecutive stages: a CTA

@@ -106,13 +106,13 @@ def spec_round(sched, base, drafter, noise, env, obs, x, t, K, acc, clip=0.0):
         n_extra = 1
     # --- draft rollout (Eq. (3)): x~_0 = x; draft k is the transition at tau = t-k+1
     x_t = [x]
-    mu_hat, xis = [None], [None]
+    mu_hat, xis, eps_hats = [None], [None], [None]
     for k in range(1, K_eff + 1):
         tau = t - k + 1
         eps_hat = drafter(x_t[k - 1], tau, obs)
         xi_k = noise.xi(env, tau, shape)
         x_k, m_k = sched.step(x_t[k - 1], eps_hat, tau, xi_k, clip)
-        x_t.append(x_k); mu_hat.append(m_k); xis.append(xi_k)
+        x_t.append(x_k); mu_hat.append(m_k); xis.append(xi_k); eps_hats.append(eps_hat)
     # --- verification: base model on every candidate latent (one batched pass on the GPU)
     n_base = K_eff + 1 if (acc.bonus or K_eff == 0) else K_eff
     eps = [base(x_t[k], t - k, obs) for k in range(n_base)]
@@ -136,7 +136,7 @@ def spec_round(sched, base, drafter, noise, env, obs, x, t, K, acc, clip=0.0):
         t_new = t - K_eff - 1
     else:
         x_new, t_new = x_t[K_eff], t - K_eff
-    dump = dict(K_eff=K_eff, x_tilde=x_t, mu_hat=mu_hat, eps=eps, mu=mu, log_alpha=log_alpha,
+    dump = dict(K_eff=K_eff, x_tilde=x_t, mu_hat=mu_hat, eps_hat=eps_hats, xi=xis, eps=eps, mu=mu, log_alpha=log_alpha,
                 flags=flags, jstar=(j if j is not None else K_eff + 1), n_base=n_base, n_extra=n_extra)
     return x_new, t_new, dump
 

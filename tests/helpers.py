@@ -43,3 +43,78 @@ def oracle_accept(a):
 def max_rel(got, ref):
     """max |got - ref| / max |ref|: the 'max relative error' the tolerances are stated in."""
     return float(np.max(np.abs(got - ref)) / max(np.max(np.abs(ref)), 1e-30))
+
+
+# ------------------------------------------------------------------------------------------------
+# Round-level comparison of the CUDA path with the oracle, one environment at a time.
+#
+# The accept statistic depends on the two networks only through their difference at the SAME input:
+# mu^_k - mu_k = -(c_x0 sqrt(1-abar)/sqrt(abar)) (eps^ - eps), so  d = -(c_tau / s) (eps^ - eps)  with
+# c_tau = c_x0 sqrt(1-abar_tau) / (sqrt(abar_tau) sigma_tau).  If both network outputs are within the
+# stated max-relative tolerance tol of the oracle's (|delta eps|_inf <= tol max|eps|), then
+#     |delta d|_2 <= eta := (c_tau / s) sqrt(D) tol (max|eps^| + max|eps|)
+# and, from  l = -1/2 |d|^2 - <d, xi>,
+#     |l_gpu - l_oracle| <= eta (|d| + |xi|) + eta^2 / 2.
+# A decision may differ from the oracle's only where |l_oracle - log thr| < 1e-3 + that bound.
+# ------------------------------------------------------------------------------------------------
+BAND = 1e-3
+
+
+def logalpha_bound(S, tau, sigma_scale, eps_hat, eps, mu_hat, mu, xi, tol_eps):
+    D = eps.size
+    c_tau = S.c_x0[tau] * np.sqrt(1.0 - S.abar[tau]) / (np.sqrt(S.abar[tau]) * S.sigma[tau]) / sigma_scale
+    eta = c_tau * np.sqrt(D) * tol_eps * (np.max(np.abs(eps_hat)) + np.max(np.abs(eps)))
+    d = (mu_hat - mu).reshape(-1) / (sigma_scale * S.sigma[tau])
+    return float(eta * (np.linalg.norm(d) + np.linalg.norm(xi)) + 0.5 * eta * eta)
+
+
+def gpu_own_jstar(la_gpu, log_thr, K_eff, mode):
+    """First k whose dumped statistic fails the test the kernel applies, and whether any of those
+    comparisons sits within float rounding of the threshold (then the host cannot re-decide it)."""
+    j, fragile = K_eff + 1, False
+    for k in range(1, K_eff + 1):
+        v = min(0.0, float(la_gpu[k - 1])) if mode == 1 else float(la_gpu[k - 1])
+        fragile |= abs(v - log_thr[k - 1]) <= 4e-6 * max(1.0, abs(log_thr[k - 1]))
+        if v < log_thr[k - 1]:
+            j = k
+            break
+    return j, fragile
+
+
+def check_round_env(S, noise, acc, b, t0, K, d, g, tol_eps, tol_x):
+    """Compare one environment's round.  d: the oracle's dump; g: dict(xt [K+1, D], mh [K, D], eps [K+1, D],
+    la [K], j, t_new, x_new [D], t_oracle, x_oracle) from tsdp_round.  Asserts everything that does not depend
+    on a decision; returns True if the decisions were checked too (j*, t, committed latent), False if a
+    deciding statistic lay inside the tolerated band and the two sides took different decisions."""
+    Ke = d["K_eff"]
+    s = acc.sigma_scale
+    log_thr, bounds = [], []
+    for k in range(1, Ke + 1):
+        tau = t0 - k + 1
+        assert np.max(np.abs(g["xt"][k] - d["x_tilde"][k].reshape(-1))) < tol_x, (b, k)
+        assert np.max(np.abs(g["mh"][k - 1] - d["mu_hat"][k].reshape(-1))) < tol_x, (b, k)
+        log_thr.append(float(np.log(noise.u(b, tau))) if acc.mode == 0 else float(np.log(acc.lam)))
+        bounds.append(logalpha_bound(S, tau, s, d["eps_hat"][k], d["eps"][k - 1], d["mu_hat"][k], d["mu"][k],
+                                     d["xi"][k].reshape(-1), tol_eps))
+    for k in range(d["n_base"]):
+        assert max_rel(g["eps"][k], d["eps"][k].reshape(-1)) < tol_eps, (b, k)
+    # the statistic itself, within what the denoiser tolerance allows
+    for k in range(1, Ke + 1):
+        lo = d["log_alpha"][k - 1]
+        assert abs(g["la"][k - 1] - lo) <= bounds[k - 1] + 1e-4 * max(1.0, abs(lo)), (b, k, g["la"][k - 1], lo, bounds[k - 1])
+    # the kernel's decision follows from its own statistic, exactly
+    j_own, fragile = gpu_own_jstar(g["la"], log_thr, Ke, acc.mode)
+    if not fragile:
+        assert g["j"] == j_own, (b, g["j"], j_own)
+    # the oracle's decisions up to and including its first rejection are the ones that matter
+    jo = d["jstar"]
+    near = False
+    for k in range(1, min(jo, Ke) + 1):
+        v = min(0.0, d["log_alpha"][k - 1]) if acc.mode == 1 else d["log_alpha"][k - 1]
+        near |= abs(v - log_thr[k - 1]) < BAND + bounds[k - 1]
+    if g["j"] != jo:
+        assert near, (b, g["j"], jo, d["log_alpha"], log_thr, bounds)
+        return False
+    assert g["t_new"] == g["t_oracle"], (b, g["t_new"], g["t_oracle"])
+    assert np.max(np.abs(g["x_new"].reshape(-1) - g["x_oracle"].reshape(-1))) < 3 * tol_x, b
+    return True

@@ -12,7 +12,6 @@ from paper_2512_15773_b200 import binding, inputs
 from tests import helpers as hp
 
 pytestmark = pytest.mark.gpu
-BAND = 1e-3
 
 
 def test_serving_round_at_bench_size_sampled_environments():
@@ -33,25 +32,17 @@ def test_serving_round_at_bench_size_sampled_environments():
     h_j = np.zeros(B, dtype=np.int32)
     acc = hp.accept_t(sigma_scale=1.5)
     smp.round(dobs, B, K, acc, seed, dx, h_t, d_xt, d_mh, d_eps, d_la, h_j)
-    xt, mh, eps = d_xt.cpu().numpy(), d_mh.cpu().numpy(), d_eps.cpu().numpy()
+    xt, mh, eps, la = d_xt.cpu().numpy(), d_mh.cpu().numpy(), d_eps.cpu().numpy(), d_la.cpu().numpy()
     x_new = dx.cpu().numpy()
     checked = 0
-    for b in (0, 1, 2, 3, 100, 255):
+    envs = (0, 1, 2, 3, 100, 255)
+    for b in envs:
         xo, to, d = spec.spec_round(S, base, draft, noise, b, obs[b], x0[b].astype(np.float64).reshape(shape), int(t0s[b]), K,
                                     hp.oracle_accept(acc))
-        Ke = d["K_eff"]
-        for k in range(d["n_base"]):
-            assert hp.max_rel(eps[b, k], d["eps"][k].reshape(-1)) < 2e-2, (b, k)
-        near_tie = False
-        for k in range(1, Ke + 1):
-            assert np.max(np.abs(mh[b, k - 1] - d["mu_hat"][k].reshape(-1))) < 3e-3
-            lu = np.log(noise.u(b, t0s[b] - k + 1))
-            near_tie |= abs(d["log_alpha"][k - 1] - lu) < BAND + 0.02 * abs(d["log_alpha"][k - 1])
-        if not near_tie:
-            assert h_j[b] == d["jstar"] and h_t[b] == to, (b, h_j[b], d["jstar"])
-            assert np.max(np.abs(x_new[b] - xo.reshape(-1))) < 1e-2
-            checked += 1
-    assert checked >= 3
+        g = dict(xt=xt[b], mh=mh[b], eps=eps[b], la=la[b], j=int(h_j[b]), t_new=int(h_t[b]), x_new=x_new[b],
+                 t_oracle=to, x_oracle=xo)
+        checked += hp.check_round_env(S, noise, hp.oracle_accept(acc), b, int(t0s[b]), K, d, g, 2e-2, 3e-3)
+    assert checked >= len(envs) - 1, checked
     smp.close()
 
 
@@ -97,4 +88,28 @@ def test_mid_size_batch_both_head_widths():
         for n in (0, 1, 7, 599, 1199):
             ref = net(x[n].astype(np.float64), int(tau[n]), obs[n])
             assert hp.max_rel(got[n], ref) < 2e-2, (which, n)
+    smp.close()
+
+
+def test_robomimic_unet_at_full_width_sampled_candidates():
+    """The conv UNet at the width the benchmark times (channels 256 / 512 / 1024, kernel-5 convolutions with
+    K = 5 C_in up to 7680 through the tensor-core GEMM's convolution addressing) and at its batch-32 row counts:
+    288 candidates = 5760 / 3456 / 2304 padded rows per level, several waves of row tiles with ragged tails.
+    A few candidates are recomputed by the oracle."""
+    wl = dict(inputs.WORKLOADS["robomimic_unet"], gamma=1.0)
+    N = 32 * 9
+    smp, S, base, draft = hp.setup(wl, max_B=N, max_K=1)
+    rng = np.random.default_rng(3)
+    x = rng.normal(size=(N, wl["H"], wl["A"])).astype(np.float32)
+    tau = rng.integers(0, 100, size=N).astype(np.int32)
+    tau[:2] = [99, 0]
+    obs = inputs.make_obs(8, N, wl["To"], wl["Do"])
+    dx = torch.tensor(x, device="cuda"); dobs = torch.tensor(obs, dtype=torch.float32, device="cuda")
+    out = torch.zeros_like(dx)
+    smp.denoise(binding.BASE, dx, tau, dobs, N, out)
+    got = out.cpu().numpy()
+    assert np.isfinite(got).all()
+    for n in (0, 1, 143, 287):
+        ref = base(x[n].astype(np.float64), int(tau[n]), obs[n])
+        assert hp.max_rel(got[n], ref) < 2e-2, n
     smp.close()

@@ -20,7 +20,7 @@
  * into its memory tokens (the query and output projections are applied once to the time / observation tokens
  * instead of to every token row) when H <= 16, (1 + obs_tokens) * heads <= 32, heads is even and d is 128, 256
  * or 512; TSDP_NO_FOLD, set before tsdp_load_weights, keeps the separate kernels.  Same function either way.
- * TSDP_NO_ASYNC_BCAST (read at every round) makes the cluster kernel hand its stages over with plain distributed-
+ * TSDP_NO_ASYNC_BCAST (read by tsdp_init, like TSDP_NO_PDL) makes the cluster kernel hand its stages over with plain distributed-
  * shared-memory stores and a cluster barrier instead of st.async stores counted by mbarriers.
  * TSDP_GEMM_BN = 32 | 64 | 128 | 256 (read by tsdp_init) forces that tile width on every tensor-core GEMM whose
  * output width it divides -- a tuning aid; results do not depend on the tile width.
@@ -57,7 +57,7 @@ enum { TSDP_ARCH_GAUSS = 0, TSDP_ARCH_MLP = 1, TSDP_ARCH_XFMR = 2, TSDP_ARCH_DIT
         * is always accepted.  Takes no weights: tsdp_load_weights(TSDP_DRAFT) is not called. */
        TSDP_ARCH_FROZEN = 5 };
 enum { TSDP_BASE = 0, TSDP_DRAFT = 1, TSDP_SCHED = 2 };
-enum { TSDP_MAX_T = 1024, TSDP_MAX_K = 32 };
+enum { TSDP_MAX_T = 1024, TSDP_MAX_K = 32, TSDP_LATENCY_RING = 256 };
 
 /* One denoiser eps = M(x, t; obs).
  *   GAUSS: closed-form optimal denoiser of iid N(m0, s0^2) data (the 1-D Gaussian toy); no sizes.
@@ -130,6 +130,13 @@ typedef struct {
                                the base forward that supplies them)                            */
   uint64_t hist_drafted[TSDP_MAX_T], hist_tested[TSDP_MAX_T], hist_accepted[TSDP_MAX_T];
                             /* per timestep of the drafted transition                          */
+  /* Device time (CUDA events on the caller's stream, copies included) of the last calls of
+   * tsdp_sample_chunk / tsdp_sample_chunk_host / tsdp_serve since the last reset, kept in a ring of
+   * TSDP_LATENCY_RING entries: nearest-rank median and 99th percentile in milliseconds, and how
+   * many calls they are taken over (0: no call yet, percentiles are 0).  With one environment per
+   * call this is the per-chunk latency the paper's Table 5 reports. */
+  double call_ms_p50, call_ms_p99;
+  uint64_t call_ms_samples;
 } tsdp_stats_t;
 
 /* Create a context on cfg->device: allocates every workspace for (max_B, max_K).  *out is set only on
@@ -270,6 +277,19 @@ int tsdp_process_reward(tsdp_ctx* ctx, float R_final, int T_max, int dt, float* 
 int tsdp_distill_loss(tsdp_ctx* ctx, const float* d_x0, const float* d_obs, int N, uint64_t seed, float lambda1,
                       float lambda2, double* h_out);
 
+/* One gradient step of that objective on the drafter, the base model frozen (Sec. 3.2, "Draft Model Training": only
+ * the drafter's parameters are updated).  Built for the closed-form Gaussian drafter (draft.arch = TSDP_ARCH_GAUSS,
+ * parameters theta = (m0, s0), m^(x, t) = sqrt(1 - abar)(x - sqrt(abar) m0) / (abar s0^2 + 1 - abar)), whose gradient
+ * is analytic; the base model may be any architecture.  Same draws (t_n, eps_n) as tsdp_distill_loss.  On the device:
+ * noising, the base forward, the per-sample gradient terms, their reduction and  theta <- theta - lr dL/dtheta.
+ * h_out[7] (HOST, double) = {L_pred, L_norm, L (all before the step), dL/dm0, dL/ds0, m0, s0 after the step}.
+ * The new parameters are in force for every later call (rounds captured in graphs are captured again).  lr = 0
+ * evaluates the gradient only.  Backward passes through the transformer / UNet drafters are not built.
+ * Uses the round's work buffers: call between chunks.  Synchronous.
+ * Errors: ARG (N, null pointers, a drafter that is not TSDP_ARCH_GAUSS, clip > 0, lr < 0), STATE, CUDA. */
+int tsdp_distill_step(tsdp_ctx* ctx, const float* d_x0, const float* d_obs, int N, uint64_t seed, float lambda1,
+                      float lambda2, float lr, double* h_out);
+
 /* Copy the counters accumulated since the last reset (synchronises the device). */
 int tsdp_stats(tsdp_ctx* ctx, tsdp_stats_t* out);
 int tsdp_reset_stats(tsdp_ctx* ctx);
@@ -306,8 +326,9 @@ int tsdp_profile_read(tsdp_ctx* ctx, double* ms, double* flop, uint64_t* launche
  * parameters: under 64 KiB) is a fixed array inside the library image; every GPU that loads the
  * library holds it until the process exits.  Capacity: B <= TSDP_STATIC_MAX_B, T <= TSDP_STATIC_MAX_T,
  * K <= TSDP_MAX_K; larger sizes return TSDP_ERR_TOO_LARGE and print the limits to stderr.
- * The first call on a device looks up the array's device address; make that first call before any
- * stream capture begins.  All calls share the one array, which still holds the previous call's
+ * The first call on a device looks up the array's device address.  Every call copies its small
+ * inputs to the device, reads the results back and waits for `cuda_stream`, so it must not be made
+ * while that stream is being captured into a graph.  All calls share the one array, which still holds the previous call's
  * values on entry (the function clears what must start at zero itself); two calls whose GPU work
  * overlaps -- different streams or threads -- race on it.  Synchronous: returns after `cuda_stream`
  * has finished the work.

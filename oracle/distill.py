@@ -46,3 +46,48 @@ def distill_loss(sched, base, drafter, x0s, obs, seed, lambda1=1.0, lambda2=1.0,
     L_pred = float(np.mean(preds))
     L_norm = float(np.mean(norms)) if norms else 0.0
     return L_pred, L_norm, lambda1 * L_pred + lambda2 * L_norm, (float(np.mean(accs)) if accs else 1.0)
+
+
+def gauss_distill_grad(sched, base, m0, s0, x0s, obs, seed, lambda1=1.0, lambda2=1.0):
+    """Gradient of L = lambda1 L_pred + lambda2 L_norm with respect to the parameters theta = (m0, s0) of the
+    closed-form Gaussian drafter  m^(x, t) = sqrt(1 - abar)(x - sqrt(abar) m0) / (abar s0^2 + 1 - abar), the base
+    model frozen (Sec. 3.2, "Draft Model Training": only theta is updated).  Same draws as distill_loss.
+
+    With v = abar s0^2 + 1 - abar:
+        d m^ / d m0 = -sqrt(1 - abar) sqrt(abar) / v,
+        d m^ / d s0 = -sqrt(1 - abar) (x - sqrt(abar) m0) 2 abar s0 / v^2,
+    and, the posterior mean being affine in the network output (no clipping),
+        (mu^ - mu) / sigma_t = -c_t (m^ - m),   c_t = c_x0(t) sqrt(1 - abar_t) / (sqrt(abar_t) sigma_t),
+    so  dL/dtheta = sum_n (lambda1 / N + [t_n >= 1] lambda2 c_{t_n}^2 / N_1) 2 <m^_n - m_n, d m^_n / d theta>,
+    N_1 the number of samples with t_n >= 1.  Returns (L_pred, L_norm, L, dL/dm0, dL/ds0)."""
+    N = len(x0s)
+    rows = []
+    for n, x0 in enumerate(x0s):
+        t = min(sched.T - 1, int(philox.uniform(seed, n, 0) * sched.T))
+        eps = philox.x_init(seed, n, x0.size).reshape(x0.shape)
+        ab = sched.abar[t]
+        x_t = np.sqrt(ab) * np.asarray(x0, dtype=np.float64) + np.sqrt(1.0 - ab) * eps
+        m = base(x_t, t, None if obs is None else obs[n])
+        v = ab * s0 * s0 + 1.0 - ab
+        mh = np.sqrt(1.0 - ab) * (x_t - np.sqrt(ab) * m0) / v
+        dm = -np.sqrt(1.0 - ab) * np.sqrt(ab) / v * np.ones_like(x_t)
+        ds = -np.sqrt(1.0 - ab) * (x_t - np.sqrt(ab) * m0) * 2.0 * ab * s0 / (v * v)
+        r = mh - m
+        c2 = 0.0
+        if t >= 1:
+            c_t = sched.c_x0[t] * np.sqrt(1.0 - ab) / (np.sqrt(ab) * sched.sigma[t])
+            c2 = c_t * c_t
+        rows.append((float(np.sum(r * r)), c2, t >= 1, 2.0 * float(np.sum(r * dm)), 2.0 * float(np.sum(r * ds))))
+    N1 = sum(1 for r in rows if r[2])
+    L_pred = sum(r[0] for r in rows) / N
+    L_norm = sum(r[0] * r[1] for r in rows) / N1 if N1 else 0.0
+    gm = sum((lambda1 / N + (lambda2 * r[1] / N1 if r[2] else 0.0)) * r[3] for r in rows)
+    gs = sum((lambda1 / N + (lambda2 * r[1] / N1 if r[2] else 0.0)) * r[4] for r in rows)
+    return L_pred, L_norm, lambda1 * L_pred + lambda2 * L_norm, gm, gs
+
+
+def gauss_distill_step(sched, base, m0, s0, x0s, obs, seed, lambda1=1.0, lambda2=1.0, lr=0.1):
+    """One plain gradient step theta <- theta - lr dL/dtheta.  Returns (L_pred, L_norm, L, dL/dm0, dL/ds0, m0', s0');
+    the losses are those before the step."""
+    Lp, Ln, L, gm, gs = gauss_distill_grad(sched, base, m0, s0, x0s, obs, seed, lambda1, lambda2)
+    return Lp, Ln, L, gm, gs, m0 - lr * gm, s0 - lr * gs

@@ -16,7 +16,7 @@ EXPORTS = ["tsdp_init", "tsdp_destroy", "tsdp_strerror", "tsdp_last_error", "tsd
            "tsdp_load_weights", "tsdp_set_schedule", "tsdp_sample_chunk", "tsdp_sample_chunk_host",
            "tsdp_round", "tsdp_denoise", "tsdp_gemm", "tsdp_gemm_timed", "tsdp_stats", "tsdp_reset_stats",
            "tsdp_kernel_launches", "tsdp_profile", "tsdp_profile_read", "tsdp_verify_commit_static", "tsdp_set_scheduler", "tsdp_set_progress",
-           "tsdp_sched_eval", "tsdp_serve", "tsdp_request_counts", "tsdp_process_reward", "tsdp_distill_loss"]
+           "tsdp_sched_eval", "tsdp_serve", "tsdp_request_counts", "tsdp_process_reward", "tsdp_distill_loss", "tsdp_distill_step"]
 PROF_FAMILIES = ["gemm", "layernorm", "attention", "embed_head", "round", "small_net", "gemm_draft", "drafter_cluster", "accept", "verifier_cluster"]
 
 
@@ -41,7 +41,8 @@ class StatsT(C.Structure):
                 ("drafts_accepted", C.c_uint64), ("rejections", C.c_uint64), ("bonus_steps", C.c_uint64),
                 ("steps_advanced", C.c_uint64), ("draft_rounds", C.c_uint64), ("nfe", C.c_double),
                 ("hist_drafted", C.c_uint64 * TSDP_MAX_T), ("hist_tested", C.c_uint64 * TSDP_MAX_T),
-                ("hist_accepted", C.c_uint64 * TSDP_MAX_T)]
+                ("hist_accepted", C.c_uint64 * TSDP_MAX_T), ("call_ms_p50", C.c_double), ("call_ms_p99", C.c_double),
+                ("call_ms_samples", C.c_uint64)]
 
 
 class TsdpError(RuntimeError):
@@ -84,15 +85,13 @@ def load_library():
     lib.tsdp_sched_eval.argtypes = [vp, fp, fp, fp, i, fp, vp]
     lib.tsdp_request_counts.argtypes = [vp, vp, i]
     lib.tsdp_distill_loss.argtypes = [vp, fp, fp, i, u64, C.c_float, C.c_float, vp]
+    lib.tsdp_distill_step.argtypes = [vp, fp, fp, i, u64, C.c_float, C.c_float, C.c_float, vp]
     lib.tsdp_process_reward.argtypes = [vp, C.c_float, i, i, fp, i]
     lib.tsdp_stats.argtypes = [vp, C.POINTER(StatsT)]
     lib.tsdp_reset_stats.argtypes = [vp]
     lib.tsdp_kernel_launches.argtypes = [vp]; lib.tsdp_kernel_launches.restype = u64
     lib.tsdp_profile.argtypes = [vp, i]
     lib.tsdp_profile_read.argtypes = [vp, fp, fp, fp]
-    for n in EXPORTS:
-        if getattr(lib, n).restype is C.c_int:
-            pass
     _lib = lib
     return lib
 
@@ -229,6 +228,13 @@ class Sampler:
         out = np.zeros(4, dtype=np.float64)
         self._check(self.lib.tsdp_distill_loss(self.h, _ptr(d_x0), _ptr(d_obs), N, seed, lambda1, lambda2, out.ctypes.data),
                     "tsdp_distill_loss")
+        return tuple(float(v) for v in out)
+
+    def distill_step(self, d_x0, d_obs, N, seed, lambda1=1.0, lambda2=1.0, lr=0.1):
+        """One gradient step on the Gaussian drafter: (L_pred, L_norm, L, dL/dm0, dL/ds0, m0', s0')."""
+        out = np.zeros(7, dtype=np.float64)
+        self._check(self.lib.tsdp_distill_step(self.h, _ptr(d_x0), _ptr(d_obs), N, seed, lambda1, lambda2, lr, out.ctypes.data),
+                    "tsdp_distill_step")
         return tuple(float(v) for v in out)
 
     def request_counts(self, n):

@@ -3,6 +3,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -104,7 +105,8 @@ struct tsdp_ctx {
   std::vector<int> sched_K;
   std::vector<tsdp_accept_t> sched_acc;
   // graphs and tensor maps
-  std::map<std::tuple<int, int>, cudaGraphExec_t> graphs;
+  struct GraphRec { cudaGraphExec_t exec; int launches; };
+  std::map<std::tuple<int, int>, GraphRec> graphs;
   std::map<std::tuple<const void*, int, int, int, int, int, int>, CUtensorMap> maps;
   EncodeTiledFn encode = nullptr;
   cudaStream_t cap_stream = nullptr;
@@ -116,11 +118,18 @@ struct tsdp_ctx {
   float *progress = nullptr, *sched_dbg = nullptr;
   int* item_counts = nullptr;        // per request: drafts proposed, drafts accepted, rounds, reverse steps taken
   float* reward = nullptr;
+  float *distill_theta = nullptr, *distill_terms = nullptr;   // Gaussian-drafter distillation step: (m0, s0), per-sample terms
+  double* distill_res = nullptr;
   int items_last = 0;                // requests of the last chunk call
   std::vector<void*> sched_allocs;
   cudaStream_t side_stream = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  // device time of the last chunk calls (ring buffer behind the latency percentiles of tsdp_stats)
+  cudaEvent_t ev_chunk0 = nullptr, ev_chunk1 = nullptr;
+  std::vector<float> lat_ring;
+  size_t lat_pos = 0, lat_n = 0;
   bool pdl = true;                            // programmatic dependent launch between the kernels of a round
+  bool async_bcast = true;                    // cluster kernel: st.async + mbarrier stage hand-over (TSDP_NO_ASYNC_BCAST unset)
   bool dc_ok = false;
   int dc_smem = 0, dc_max_clusters = 0;
   bool dc_resident = false;
@@ -962,7 +971,7 @@ int launch_cluster_forward(tsdp_ctx* c, int which, int mode, int B, int K, cudaS
   P.kq_time = n.fold_kq_time; P.ut_time = n.fold_ut_time; P.c_time = n.fold_c_time;
   P.kq_obs = n.fold_kq_obs; P.ut_obs = n.fold_ut_obs; P.c_obs = n.fold_c_obs;
   P.status = c->status;
-  P.async_bcast = getenv("TSDP_NO_ASYNC_BCAST") == nullptr ? 1 : 0;
+  P.async_bcast = c->async_bcast ? 1 : 0;
   P.S = c->S;
   P.xt = c->xt; P.xs_b = (long long)(c->cfg.max_K + 1) * c->D;
   P.muhat = c->muhat; P.ms_b = (long long)(c->cfg.max_K > 0 ? c->cfg.max_K : 1) * c->D;
@@ -1049,8 +1058,6 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
   return TSDP_OK;
 }
 
-struct GraphRec { cudaGraphExec_t exec; int launches; };
-
 int run_round(tsdp_ctx* c, int B, int K, cudaStream_t s) {
   if (!c->cfg.use_graph || c->prof_on) {
     c->launches_per_round_tmp = 0;
@@ -1058,7 +1065,6 @@ int run_round(tsdp_ctx* c, int B, int K, cudaStream_t s) {
     c->launches += c->launches_per_round_tmp;
     return r;
   }
-  static std::map<cudaGraphExec_t, int> launch_counts;
   auto key = std::make_tuple(B, K);
   auto it = c->graphs.find(key);
   if (it == c->graphs.end()) {
@@ -1074,11 +1080,10 @@ int run_round(tsdp_ctx* c, int B, int K, cudaStream_t s) {
     cudaGraphExec_t exec = nullptr;
     CU_TRY(c, cudaGraphInstantiate(&exec, graph, 0));
     cudaGraphDestroy(graph);
-    launch_counts[exec] = c->launches_per_round_tmp;
-    it = c->graphs.emplace(key, exec).first;
+    it = c->graphs.emplace(key, tsdp_ctx::GraphRec{exec, c->launches_per_round_tmp}).first;
   }
-  CU_TRY(c, cudaGraphLaunch(it->second, s));
-  c->launches += launch_counts[it->second];
+  CU_TRY(c, cudaGraphLaunch(it->second.exec, s));
+  c->launches += it->second.launches;
   return TSDP_OK;
 }
 
@@ -1164,6 +1169,7 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   c->cfg = *cfg;
   c->D = cfg->H * cfg->A;
   c->pdl = getenv("TSDP_NO_PDL") == nullptr;
+  c->async_bcast = getenv("TSDP_NO_ASYNC_BCAST") == nullptr;
   if (const char* fb = getenv("TSDP_GEMM_BN")) {      // tuning aid: one tile width for every GEMM it divides
     const int v = atoi(fb);
     if (v == 32 || v == 64 || v == 128 || v == 256) c->force_bn = v;
@@ -1234,6 +1240,9 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   st |= dev_alloc(c, c->allocs, &c->sched_dbg, B * 8);
   st |= dev_alloc(c, c->allocs, &c->item_counts, (size_t)B * 4);
   st |= dev_alloc(c, c->allocs, &c->reward, B);
+  st |= dev_alloc(c, c->allocs, &c->distill_theta, 2);
+  st |= dev_alloc(c, c->allocs, &c->distill_terms, 5 * B);
+  st |= dev_alloc(c, c->allocs, &c->distill_res, 8);
   if (st) return fail(TSDP_ERR_CUDA);
   INIT_TRY(cudaHostAlloc(reinterpret_cast<void**>(&c->host_done), sizeof(int), cudaHostAllocMapped));
   *c->host_done = 0;
@@ -1242,6 +1251,9 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   INIT_TRY(cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking));
   INIT_TRY(cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
   INIT_TRY(cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming));
+  INIT_TRY(cudaEventCreate(&c->ev_chunk0));
+  INIT_TRY(cudaEventCreate(&c->ev_chunk1));
+  c->lat_ring.assign(TSDP_LATENCY_RING, 0.f);
 
   // transformer workspaces, sized for the larger of (base over all candidates, drafter over B)
   size_t rows_d = 0, rows_4d = 0, mem_rows_d = 0;
@@ -1346,7 +1358,7 @@ void tsdp_destroy(tsdp_ctx* c) {
   if (!c) return;
   cudaSetDevice(c->cfg.device);
   cudaDeviceSynchronize();
-  for (auto& g : c->graphs) cudaGraphExecDestroy(g.second);
+  for (auto& g : c->graphs) cudaGraphExecDestroy(g.second.exec);
   for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
   for (void* p : c->allocs) cudaFree(p);
   for (int w = 0; w < 2; ++w)
@@ -1357,6 +1369,8 @@ void tsdp_destroy(tsdp_ctx* c) {
   if (c->side_stream) cudaStreamDestroy(c->side_stream);
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
   if (c->ev_join) cudaEventDestroy(c->ev_join);
+  if (c->ev_chunk0) cudaEventDestroy(c->ev_chunk0);
+  if (c->ev_chunk1) cudaEventDestroy(c->ev_chunk1);
   for (void* p : c->sched_allocs) cudaFree(p);
   delete c;
 }
@@ -1402,7 +1416,7 @@ int tsdp_load_weights(tsdp_ctx* c, int which, const float* blob, size_t n) {
   net.L.clear();
   net.loaded = false;
   // graphs captured with the old pointers are stale
-  for (auto& g : c->graphs) cudaGraphExecDestroy(g.second);
+  for (auto& g : c->graphs) cudaGraphExecDestroy(g.second.exec);
   c->graphs.clear();
   c->maps.clear();
 
@@ -1792,7 +1806,7 @@ int tsdp_set_scheduler(tsdp_ctx* c, int enable) {
   CU_TRY(c, cudaSetDevice(c->cfg.device));
   CU_TRY(c, cudaDeviceSynchronize());
   // captured rounds carry the pointer to the per-environment parameters (or null): capture again
-  for (auto& g : c->graphs) cudaGraphExecDestroy(g.second);
+  for (auto& g : c->graphs) cudaGraphExecDestroy(g.second.exec);
   c->graphs.clear();
   c->sched_on = enable != 0;
   return TSDP_OK;
@@ -1861,7 +1875,7 @@ static int ensure_items(tsdp_ctx* c, size_t N) {
   if (dmax) st |= alloc_bytes(c, c->allocs, &c->memtok, std::max((size_t)cfg.T, N * To) * dmax * (cfg.precision == 0 ? 4 : 2));
   if (st) return TSDP_ERR_CUDA;
   c->items_cap = N;
-  for (auto& g : c->graphs) cudaGraphExecDestroy(g.second);
+  for (auto& g : c->graphs) cudaGraphExecDestroy(g.second.exec);
   c->graphs.clear();
   c->maps.clear();
   return TSDP_OK;
@@ -1879,6 +1893,7 @@ static int sample_chunk_impl(tsdp_ctx* c, const float* obs, bool obs_on_host, in
   const int D = c->D, T = c->cfg.T;
   int r;
   if ((r = ensure_items(c, (size_t)N))) return r;
+  CU_TRY(c, cudaEventRecord(c->ev_chunk0, s));
   if (obs_n)
     CU_TRY(c, cudaMemcpyAsync(c->obs, obs, obs_n * sizeof(float), obs_on_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, s));
   CU_TRY(c, cudaMemcpyAsync(c->seed, &seed, sizeof(seed), cudaMemcpyHostToDevice, s));
@@ -1923,7 +1938,16 @@ static int sample_chunk_impl(tsdp_ctx* c, const float* obs, bool obs_on_host, in
   }
   CU_TRY(c, cudaMemcpyAsync(actions, c->actions, (size_t)N * D * sizeof(float),
                             actions_on_host ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice, s));
+  CU_TRY(c, cudaEventRecord(c->ev_chunk1, s));
   CU_TRY(c, cudaStreamSynchronize(s));
+  {   // device time of this call, copies included, into the latency ring
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, c->ev_chunk0, c->ev_chunk1) == cudaSuccess) {
+      c->lat_ring[c->lat_pos] = ms;
+      c->lat_pos = (c->lat_pos + 1) % c->lat_ring.size();
+      if (c->lat_n < c->lat_ring.size()) c->lat_n++;
+    }
+  }
   return check_status(c);
 }
 
@@ -2071,6 +2095,46 @@ int tsdp_distill_loss(tsdp_ctx* c, const float* d_x0, const float* d_obs, int N,
   return TSDP_OK;
 }
 
+int tsdp_distill_step(tsdp_ctx* c, const float* d_x0, const float* d_obs, int N, uint64_t seed, float lambda1, float lambda2,
+                      float lr, double* h_out) {
+  if (!c || !d_x0 || !h_out || N < 1 || N > c->cfg.max_B || c->cfg.draft.arch != TSDP_ARCH_GAUSS || c->cfg.clip > 0.f ||
+      !(lr >= 0.f))
+    return TSDP_ERR_ARG;
+  const size_t obs_n = (size_t)N * c->cfg.obs_tokens * c->cfg.obs_dim;
+  if (obs_n > 0 && !d_obs) return TSDP_ERR_ARG;
+  if (!c->net[0].loaded || !c->net[1].loaded) return TSDP_ERR_STATE;
+  CU_TRY(c, cudaSetDevice(c->cfg.device));
+  cudaStream_t s = nullptr;
+  const int D = c->D;
+  const long long xs_b = (long long)(c->cfg.max_K + 1) * D;
+  Net& dn = c->net[TSDP_DRAFT];
+  int r;
+  if ((r = ensure_items(c, (size_t)N))) return r;
+  if (obs_n) CU_TRY(c, cudaMemcpyAsync(c->obs, d_obs, obs_n * sizeof(float), cudaMemcpyDeviceToDevice, s));
+  CU_TRY(c, cudaMemcpyAsync(c->seed, &seed, sizeof(seed), cudaMemcpyHostToDevice, s));
+  const float theta[2] = {dn.m0, dn.s0};
+  CU_TRY(c, cudaMemcpyAsync(c->distill_theta, theta, sizeof(theta), cudaMemcpyHostToDevice, s));
+  distill_noise_kernel<<<N, 128, 0, s>>>(c->S, d_x0, c->xt, xs_b, c->t, D, c->seed);
+  CU_TRY(c, cudaGetLastError());
+  c->launches_per_round_tmp = 1;
+  if ((r = prepare_obs(c, c->net[TSDP_BASE], N, s))) return r;
+  CandMap cb{c->xt, xs_b, c->eps, xs_b, c->t, 1, 0, nullptr};
+  if ((r = forward(c, c->net[TSDP_BASE], cb, N, s))) return r;
+  distill_gauss_grad_kernel<<<N, 128, 0, s>>>(c->S, c->xt, xs_b, c->eps, xs_b, c->t, D, c->distill_theta, c->distill_terms);
+  distill_gauss_update_kernel<<<1, 256, 0, s>>>(c->distill_terms, N, lambda1, lambda2, lr, c->distill_theta, c->distill_res);
+  CU_TRY(c, cudaGetLastError());
+  c->launches += c->launches_per_round_tmp + 2;
+  CU_TRY(c, cudaMemcpyAsync(h_out, c->distill_res, sizeof(double) * 7, cudaMemcpyDeviceToHost, s));
+  CU_TRY(c, cudaStreamSynchronize(s));
+  if ((r = check_status(c))) return r;
+  // the drafter's parameters travel to its kernels by value: adopt the new ones and drop rounds captured with the old
+  dn.m0 = (float)h_out[5];
+  dn.s0 = (float)h_out[6];
+  for (auto& g : c->graphs) cudaGraphExecDestroy(g.second.exec);
+  c->graphs.clear();
+  return TSDP_OK;
+}
+
 int tsdp_gemm(tsdp_ctx* c, const void* d_A, const void* d_W, const float* d_bias, int M, int N, int K, int epi,
               void* d_out, void* stream) {
   if (!c || !d_A || !d_W || !d_out || M < 1 || N < 1 || K < 1 || epi < 0 || epi > 3) return TSDP_ERR_ARG;
@@ -2119,7 +2183,8 @@ int tsdp_stats(tsdp_ctx* c, tsdp_stats_t* out) {
   if (!c || !out) return TSDP_ERR_ARG;
   CU_TRY(c, cudaSetDevice(c->cfg.device));
   CU_TRY(c, cudaDeviceSynchronize());
-  static DevStats ds;
+  std::vector<DevStats> staging(1);
+  DevStats& ds = staging[0];
   CU_TRY(c, cudaMemcpy(&ds, c->stats, sizeof(DevStats), cudaMemcpyDeviceToHost));
   memset(out, 0, sizeof(*out));
   out->chunks = ds.chunks_done;
@@ -2135,6 +2200,14 @@ int tsdp_stats(tsdp_ctx* c, tsdp_stats_t* out) {
   out->draft_rounds = ds.draft_rounds;
   out->nfe = (double)ds.env_rounds + (double)c->cfg.draft_nfe * (double)ds.draft_evals;
   if (c->cfg.draft.arch == TSDP_ARCH_FROZEN) out->nfe = (double)ds.env_rounds + (double)ds.draft_rounds;
+  out->call_ms_samples = c->lat_n;
+  if (c->lat_n > 0) {   // nearest-rank percentiles over the ring
+    std::vector<float> v(c->lat_ring.begin(), c->lat_ring.begin() + c->lat_n);
+    std::sort(v.begin(), v.end());
+    auto pct = [&](double q) { size_t i = (size_t)std::ceil(q * v.size()); return (double)v[i > 0 ? i - 1 : 0]; };
+    out->call_ms_p50 = pct(0.50);
+    out->call_ms_p99 = pct(0.99);
+  }
   for (int i = 0; i < TSDP_MAX_T; ++i) {
     out->hist_drafted[i] = ds.hist_drafted[i];
     out->hist_tested[i] = ds.hist_tested[i];
@@ -2150,6 +2223,7 @@ int tsdp_reset_stats(tsdp_ctx* c) {
   CU_TRY(c, cudaMemset(c->stats, 0, sizeof(DevStats)));
   c->rounds = 0;
   c->launches = 0;
+  c->lat_pos = c->lat_n = 0;
   return TSDP_OK;
 }
 

@@ -512,3 +512,33 @@ def test_argument_errors_on_device():
     smp.sample_chunk(obs, 2, 4, hp.accept_t(), 0, out)
     assert torch.isfinite(out).all()
     smp.close()
+
+
+def test_call_latency_ring_percentiles():
+    """tsdp_stats reports the median and 99th percentile of the device time of the last chunk calls; checked against
+    CUDA events recorded around the same calls on the same stream."""
+    wl = dict(inputs.WORKLOADS["toy_mlp"])
+    smp, *_ = hp.setup(wl, max_B=2, max_K=4)
+    obs = torch.tensor(inputs.make_obs(4, 2, wl["To"], wl["Do"]), dtype=torch.float32, device="cuda")
+    out = torch.zeros(2, wl["H"], wl["A"], device="cuda")
+    smp.sample_chunk(obs, 2, 4, hp.accept_t(), 1, out)
+    smp.reset_stats()
+    assert smp.stats()["call_ms_samples"] == 0
+    n, ms = 7, []
+    for i in range(n):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        smp.sample_chunk(obs, 2, 4 if i else 0, hp.accept_t(), 10 + i, out)      # the first call is vanilla: the slowest
+        e1.record()
+        torch.cuda.synchronize()
+        ms.append(e0.elapsed_time(e1))
+    st = smp.stats()
+    assert st["call_ms_samples"] == n
+    assert 0 < st["call_ms_p50"] <= st["call_ms_p99"] <= max(ms) * 1.05
+    assert abs(st["call_ms_p50"] - float(np.median(ms))) < 0.25 * float(np.median(ms)) + 0.05
+    assert st["call_ms_p99"] > 1.5 * st["call_ms_p50"]                           # the K = 0 call stands out
+    # the ring keeps the last TSDP_LATENCY_RING calls only
+    for i in range(260):
+        smp.sample_chunk(obs, 2, 4, hp.accept_t(), 100 + i, out)
+    assert smp.stats()["call_ms_samples"] == 256
+    smp.close()

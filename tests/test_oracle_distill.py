@@ -50,3 +50,44 @@ def test_loss_is_the_weighted_sum_and_the_acceptance_is_the_gaussian_overlap():
         pdf = lambda m: np.exp(-0.5 * (z - m) ** 2) / math.sqrt(2 * math.pi)
         overlap = np.trapezoid(np.minimum(pdf(0.0), pdf(d)), z)
         assert abs(overlap - math.erfc(d / (2 * math.sqrt(2)))) < 1e-6
+
+
+# ----------------------------------------------------------------------------- the distillation step (Gaussian drafter)
+def _gauss_pair(m, s):
+    return nets.make_denoiser(inputs.make_gauss_params(m, s), S)
+
+
+def test_gauss_gradient_matches_finite_differences_of_the_pinned_loss():
+    base = _gauss_pair(0.7, 0.5)
+    x0s = np.random.default_rng(5).normal(0.7, 0.5, size=(96, 4, 2))
+    m, s, l1, l2, seed = 0.95, 0.4, 1.5, 0.25, 17
+    Lp, Ln, L, gm, gs = distill.gauss_distill_grad(S, base, m, s, x0s, None, seed, l1, l2)
+    ref = distill.distill_loss(S, base, _gauss_pair(m, s), x0s, None, seed, l1, l2)
+    assert abs(Lp - ref[0]) < 1e-12 * max(1, ref[0]) and abs(Ln - ref[1]) < 1e-10 * max(1, ref[1]) and abs(L - ref[2]) < 1e-10 * max(1, ref[2])
+    h = 1e-6
+    f = lambda mm, ss: distill.distill_loss(S, base, _gauss_pair(mm, ss), x0s, None, seed, l1, l2)[2]
+    fd_m = (f(m + h, s) - f(m - h, s)) / (2 * h)
+    fd_s = (f(m, s + h) - f(m, s - h)) / (2 * h)
+    assert abs(gm - fd_m) < 1e-6 * max(1.0, abs(fd_m)) and abs(gs - fd_s) < 1e-6 * max(1.0, abs(fd_s))
+    assert abs(gm) > 1e-3 and abs(gs) > 1e-3
+    # each term alone (a dropped weight or a wrong c_t would survive a test of the sum only at one (lambda1, lambda2))
+    for a, b in ((1.0, 0.0), (0.0, 1.0)):
+        g = distill.gauss_distill_grad(S, base, m, s, x0s, None, seed, a, b)
+        fa = lambda mm, ss: distill.distill_loss(S, base, _gauss_pair(mm, ss), x0s, None, seed, a, b)[2]
+        assert abs(g[3] - (fa(m + h, s) - fa(m - h, s)) / (2 * h)) < 1e-6 * max(1.0, abs(g[3]))
+        assert abs(g[4] - (fa(m, s + h) - fa(m, s - h)) / (2 * h)) < 1e-6 * max(1.0, abs(g[4]))
+
+
+def test_gauss_distillation_descends_to_the_base_parameters():
+    """The base's own parameters are a fixed point (zero loss, zero gradient); small steps decrease L monotonically
+    and carry (m0, s0) to the base's."""
+    base = _gauss_pair(0.7, 0.5)
+    x0s = np.random.default_rng(6).normal(0.7, 0.5, size=(128, 1, 1))
+    out = distill.gauss_distill_grad(S, base, 0.7, 0.5, x0s, None, 3)
+    assert out[2] < 1e-24 and abs(out[3]) < 1e-12 and abs(out[4]) < 1e-12
+    m, s, last = 0.95, 0.4, None
+    for it in range(400):
+        Lp, Ln, L, gm, gs, m, s = distill.gauss_distill_step(S, base, m, s, x0s, None, 3, 1.0, 1.0, lr=0.02)
+        assert last is None or L <= last * (1 + 1e-12)
+        last = L
+    assert abs(m - 0.7) < 5e-3 and abs(s - 0.5) < 5e-3 and last < 1e-3

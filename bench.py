@@ -142,6 +142,98 @@ def make_sampler(wl, B, device, use_graph=1):
     return smp
 
 
+def gemm_traffic_record():
+    """Measured DRAM bytes per GEMM launch, from the tracked ncu summary -- valid only for the kernel source it was
+    taken with: the summary names the sha256 prefix of gemm_tcgen05.cuh, and a different source gives null."""
+    import hashlib
+    import re
+    prof = os.path.join(ROOT, "profiles", "gemm_tcgen05_serving_shapes.md")
+    src = os.path.join(ROOT, "paper_2512_15773_b200", "csrc", "gemm_tcgen05.cuh")
+    try:
+        txt = open(prof).read()
+        sha = hashlib.sha256(open(src, "rb").read()).hexdigest()[:16]
+        m = re.search(r"traffic_bytes_per_launch:\s*([0-9.eE+]+)\s+kernel_source_sha256_16:\s*([0-9a-f]{16})\s+captured:\s*(\S+)", txt)
+        if m and m.group(2) == sha:
+            return float(m.group(1)), f"ncu dram read+write bytes per launch, {os.path.basename(prof)}, captured {m.group(3)}"
+        return None, "the GEMM kernel changed since the ncu counters in profiles/ were taken" if m else "no ncu record"
+    except OSError:
+        return None, "no ncu record"
+
+
+def family_rooflines(prof, peaks):
+    """Two tensor rooflines from one event-timed step: the GEMM kernel alone, and the whole verification forward
+    (base-model GEMM flops over base-model GEMM + LayerNorm + attention + embedding / head time)."""
+    g = prof["gemm"]
+    fam_ms = {k: round(v["ms"], 3) for k, v in prof.items() if v["launches"]}
+    tot_ms = sum(v["ms"] for v in prof.values())
+    if not g["launches"] or g["ms"] <= 0:
+        return None, None, fam_ms, tot_ms
+    ach = g["flop"] / (g["ms"] * 1e-3) / 1e12
+    r1 = dict(bound="tensor", kernel="gemm_tcgen05_kernel", achieved=ach, peak=peaks["bf16_sustained"], unit="TFLOP/s",
+              frac=ach / peaks["bf16_sustained"], frac_of_burst=ach / peaks["bf16_burst"],
+              peak_source=f"bf16_tflops_sustained of {peaks['source']}", traffic=None, launches_timed=g["launches"],
+              avg_launch_us=1e3 * g["ms"] / g["launches"], share_of_kernel_time=g["ms"] / tot_ms, family_ms=fam_ms,
+              flops_counted="2 M N K over the rows each launch really processed (live candidates x tokens)")
+    fwd_ms = sum(prof[k]["ms"] for k in ("gemm", "layernorm", "attention", "embed_head"))
+    a2 = g["flop"] / (fwd_ms * 1e-3) / 1e12
+    r2 = dict(bound="tensor", kernel="verification forward: GEMM + LayerNorm + attention + embed/head kernels of the base model",
+              achieved=a2, unit="TFLOP/s", peak=peaks["bf16_sustained"], frac=a2 / peaks["bf16_sustained"],
+              peak_burst=peaks["bf16_burst"], frac_of_burst=a2 / peaks["bf16_burst"],
+              peak_source=f"bf16_tflops_sustained / bf16_tflops of {peaks['source']}", forward_ms=fwd_ms,
+              note="GEMM flops only (attention flops not counted) over all base-model kernel time")
+    return r1, r2, fam_ms, tot_ms
+
+
+def side_record(name, B, K, local, acc, n_warm, n_timed, peaks, vanilla_steps=2, profile=True, drafter=None):
+    """Compact record of another named configuration: speculative and vanilla timing, acceptance, GEMM roofline."""
+    import torch
+    from paper_2512_15773_b200 import inputs
+    wl = workload_spec(name, B)
+    wl["K"] = K
+    wl.pop("schedule", None)
+    if drafter == "frozen":
+        wl["draft"] = dict(arch="frozen")
+    smp = make_sampler(wl, B, local)
+    obs = torch.tensor(inputs.make_obs(5, B, wl["To"], wl["Do"]).astype(np.float32), device="cuda")
+    out = torch.zeros(B, wl["H"], wl["A"], device="cuda")
+    time_steps(smp, obs, out, B, K, acc, list(range(n_warm)))
+    smp.reset_stats()
+    ts = time_steps(smp, obs, out, B, K, acc, list(range(100, 100 + n_timed)))
+    st = smp.stats()
+    n_chunks = B * n_timed
+    rec = dict(workload=f"{name} B={B} K={K}", steps=n_timed, p50_step_ms=float(np.median(ts)),
+               chunks_per_s=B / (float(np.median(ts)) / 1e3),
+               accepted_denoise_steps_per_s=st["drafts_accepted"] / (sum(ts) / 1e3),
+               acceptance=st["drafts_accepted"] / max(st["draft_evals"], 1),
+               base_forwards_per_chunk=st["env_rounds"] / n_chunks, drafts_per_chunk=st["draft_evals"] / n_chunks,
+               nfe_per_chunk=st["nfe"] / n_chunks, lib_call_ms_p50=st["call_ms_p50"], lib_call_ms_p99=st["call_ms_p99"],
+               useful_row_fraction=(st["base_evals"] / st["cand_computed"]) if st["cand_computed"] else None,
+               dense_row_fraction=(st["base_evals"] / st["cand_dense"]) if st["cand_dense"] else None)
+    if B == 1:
+        rec["p50_chunk_ms"] = rec["p50_step_ms"]
+        rec["p99_chunk_ms"] = float(np.percentile(ts, 99))
+    if profile:
+        smp.profile(1)
+        time_steps(smp, obs, out, B, K, acc, [100])
+        pr = smp.profile_read()
+        smp.profile(0)
+        r1, r2, fam_ms, _ = family_rooflines(pr, peaks)
+        rec["family_ms"] = fam_ms
+        if r1 and wl["precision"] == 1:
+            rec["roofline"] = {k: r1[k] for k in ("achieved", "frac", "frac_of_burst", "launches_timed", "avg_launch_us", "unit")}
+            rec["roofline_verify_forward"] = {k: r2[k] for k in ("achieved", "frac", "frac_of_burst", "forward_ms")}
+    if vanilla_steps:
+        time_steps(smp, obs, out, B, 0, acc, [0])
+        tv = time_steps(smp, obs, out, B, 0, acc, list(range(vanilla_steps)))
+        rec["vanilla_p50_step_ms"] = float(np.median(tv))
+        rec["vanilla_chunks_per_s"] = B / (float(np.median(tv)) / 1e3)
+        rec["speedup_vs_vanilla"] = float(np.median(tv)) / rec["p50_step_ms"]
+    smp.close()
+    del smp
+    torch.cuda.empty_cache()
+    return rec
+
+
 def time_steps(smp, d_obs, out, B, K, acc, seeds, host=False, h_obs=None, h_out=None):
     """Device time of each step (CUDA events on the stream the library launches on: the default one)."""
     import torch
@@ -163,6 +255,10 @@ def run_ours(args):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.gpus != world:
+        # one process per GPU: N > 1 needs the torchrun launch, which sets WORLD_SIZE; never silently run fewer ranks
+        raise SystemExit(f"bench.py --gpus {args.gpus} was started with WORLD_SIZE={world}: launch it as "
+                         f"python -m torch.distributed.run --nnodes=1 --nproc-per-node {args.gpus} bench.py --gpus {args.gpus} ...")
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
@@ -236,25 +332,22 @@ def run_ours(args):
         time_steps(smp, d_obs, out, B, K, acc, [rank_seed(7, rank, 0)])
         prof = smp.profile_read()
         smp.profile(0)
+        r1, r2, fam_ms, tot_ms = family_rooflines(prof, peaks)
         g = prof["gemm"]
-        fam_ms = {k: round(v["ms"], 3) for k, v in prof.items() if v["launches"]}
-        tot_ms = sum(v["ms"] for v in prof.values())
-        if wl["precision"] == 1 and g["launches"] and g["ms"] > 0.2 * tot_ms:
-            ach = g["flop"] / (g["ms"] * 1e-3) / 1e12
-            result["roofline"] = dict(bound="tensor", kernel="gemm_tcgen05_kernel", achieved=ach,
-                                      peak=peaks["bf16_sustained"], unit="TFLOP/s", frac=ach / peaks["bf16_sustained"],
-                                      peak_source=f"bf16_tflops_sustained of {peaks['source']}", traffic=None,
-                                      launches_timed=g["launches"], avg_launch_us=1e3 * g["ms"] / g["launches"],
-                                      share_of_kernel_time=g["ms"] / tot_ms, family_ms=fam_ms)
+        if wl["precision"] == 1 and r1 and g["ms"] > 0.2 * tot_ms:
+            result["roofline"] = r1
+            result["roofline_verify_forward"] = r2
             if args.workload == "serving_xfmr" and B == 256:
-                # ncu DRAM bytes (read + write) of the four GEMM shapes a base block launches (qkv, attention
-                # projection -- bf16 store --, MLP up, MLP down; the cross-attention projections are folded into its
-                # memory tokens) at K = 10 (45056 rows), averaged per launch: profiles/gemm_tcgen05_serving_shapes.md.
-                # Rounds with a smaller K launch proportionally fewer rows.
-                result["roofline"]["traffic"] = 170.5e6
-                result["roofline"]["traffic_note"] = ("mean DRAM bytes per launch over the 4 GEMM shapes of a block at "
-                                                      "45056 rows (ncu: 126.6, 49.7, 173.5, 332.3 MB); algorithmic "
-                                                      "operand+output bytes average 221e6, the difference stays in L2")
+                tr, note = gemm_traffic_record()
+                result["roofline"]["traffic"] = tr
+                result["roofline"]["traffic_note"] = note
+        else:
+            # batch-1 style workloads run in the persistent cluster kernels (or the toy CUDA-core networks): a chain
+            # of dependent stages on a few SMs, bound by latency, not by a throughput roof
+            top = max(prof.items(), key=lambda kv: kv[1]["ms"])[0] if prof else None
+            result["roofline"] = dict(bound="alu", kernel=top, achieved=None, peak=None, unit="TFLOP/s", frac=None,
+                                      traffic=None, family_ms=fam_ms,
+                                      note="latency-bound chain of small dependent stages; no throughput roofline applies")
         a = prof.get("accept")
         if a and a["launches"]:
             # fused acceptance / commit kernel: bytes it must move per launch (candidates, drafter means, base
@@ -270,13 +363,6 @@ def run_ours(args):
                                              unit="GB/s", frac=gbs / peaks["hbm_gbs"],
                                              avg_launch_us=1e3 * a["ms"] / a["launches"],
                                              note="working set of a few MB: launch-latency-bound, not bandwidth-bound")
-        else:
-            # batch-1 style workloads run in the persistent cluster kernels (or the toy CUDA-core networks): a chain
-            # of dependent stages on a few SMs, bound by latency, not by a throughput roof
-            top = max(prof.items(), key=lambda kv: kv[1]["ms"])[0] if prof else None
-            result["roofline"] = dict(bound="alu", kernel=top, achieved=None, peak=None, unit="TFLOP/s", frac=None,
-                                      traffic=None, family_ms=fam_ms,
-                                      note="latency-bound chain of small dependent stages; no throughput roofline applies")
         # ---- continuous batching: 4 B requests through the same B slots (finished slots refill at once)
         cont = None
         if wl["precision"] == 1 and args.workload == "serving_xfmr":
@@ -336,8 +422,26 @@ def run_ours(args):
                                                acceptance=st2["drafts_accepted"] / max(st2["draft_evals"], 1),
                                                rounds_per_chunk=st2["env_rounds"] / 64, nfe_per_chunk=st2["nfe"] / 64)
             s2.close()
+        # ---- the other named configurations, each as a compact record (same library, same timing method)
+        others = None
+        if args.configs and world == 1:
+            others = {}
+            # free this workload's context first: the largest configuration wants the memory
+            smp.close()
+            torch.cuda.empty_cache()
+            for k2 in (2, 4):
+                others[f"pusht_xfmr_B1_K{k2}"] = side_record("pusht_xfmr", 1, k2, local, acc, 6, 32, peaks, vanilla_steps=0, profile=False)
+            others["robomimic_unet_B1_K8"] = side_record("robomimic_unet", 1, 8, local, acc, 3, 12, peaks, vanilla_steps=3)
+            others["robomimic_unet_B32_K8"] = side_record("robomimic_unet", 32, 8, local, acc, 3, 6, peaks, vanilla_steps=2)
+            others["robomimic_unet_B32_K8_frozen_target_drafts"] = side_record("robomimic_unet", 32, 8, local, acc, 3, 6, peaks,
+                                                                                 vanilla_steps=0, profile=False, drafter="frozen")
+            others["vla_dit_B64_K16"] = side_record("vla_dit", 64, 16, local, acc, 1, 2, peaks, vanilla_steps=1)
         cpu = cpu_baseline(wl, budget_s=args.cpu_seconds) if world == 1 else None
+        cand = reduce_sum([st["base_evals"], st["cand_computed"], st["cand_dense"]], 1)
         result.update(
+            useful_row_fraction=(cand[0] / cand[1]) if cand[1] else None,
+            dense_row_fraction=(cand[0] / cand[2]) if cand[2] else None,
+            lib_call_ms_p50=st["call_ms_p50"], lib_call_ms_p99=st["call_ms_p99"], other_configs=others,
             accepted_denoise_steps_per_s=acc_steps / (total_ms / 1e3),
             p50_step_ms=float(np.median(per_step)),
             acceptance=acc_steps / max(drafted, 1.0), base_forwards_per_chunk=env_rounds / chunks_total,
@@ -348,6 +452,9 @@ def run_ours(args):
                                  f"seeded 3-state Markov K/sigma schedule)" if args.workload == "serving_xfmr"
                         else f"{args.workload} B={B} K={K}",
                         global_batch=B * world, K_max=K, T=wl["T"], gamma=wl.get("gamma"),
+                        sampler=("likelihood-ratio test with the schedule's sigma-scale 1.5 / 2.0 in two of its three states: "
+                                 "those rounds widen the test and are NOT lossless (only sigma-scale 1 keeps the law of "
+                                 "vanilla DDPM)") if "schedule" in wl else "lossless: likelihood-ratio test, sigma-scale 1",
                         l2="per-step working set (activations of all candidates) exceeds the 126 MB L2; no explicit flush"
                         if B * (K + 1) * wl["H"] * wl["base"].get("d", 0) * 16 > 126e6 else
                         "working set fits L2 by design (weights are reused across rounds); no explicit flush",
@@ -445,6 +552,8 @@ def main():
                     help="net: the workload's drafter network; frozen: no drafter, drafts reuse the base output at the round's start")
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
     ap.add_argument("--no-latency", dest="latency", action="store_false")
+    ap.add_argument("--no-configs", dest="configs", action="store_false",
+                    help="skip the compact records of the other named configurations (other_configs)")
     ap.add_argument("--only-timed", action="store_true",
                     help="run warm-up and the timed region only (for a profiler's launch list)")
     args = ap.parse_args()

@@ -137,6 +137,12 @@ typedef struct {
    * call this is the per-chunk latency the paper's Table 5 reports. */
   double call_ms_p50, call_ms_p99;
   uint64_t call_ms_samples;
+  /* Candidate latents the verification forwards covered.  cand_dense: what the dense layout B x (K+1) per round
+   * amounts to; cand_computed: what was really evaluated -- each round first lists the candidates that are still
+   * needed (unfinished environments, draft slots up to K_eff, the bonus slot) and the layer-by-layer forwards run
+   * on that list only (TSDP_NO_COMPACT, read by tsdp_init, or more than 4096 environments per call: dense).
+   * Rounds verified by the cluster kernel count in cand_dense only. */
+  uint64_t cand_dense, cand_computed;
 } tsdp_stats_t;
 
 /* Create a context on cfg->device: allocates every workspace for (max_B, max_K).  *out is set only on
@@ -221,7 +227,8 @@ int tsdp_sample_chunk_host(tsdp_ctx* ctx, const float* h_obs, int B, int K, cons
 /* One speculative round from a given state, with every intermediate exposed (test interface).
  *   d_x [B, D] in/out: current latents;  h_t [B] in/out: their timesteps (HOST).
  * Optional outputs (null to skip): d_xtilde [B, K+1, D] candidates (slot 0 = input latent),
- * d_muhat [B, K, D] drafter means, d_eps [B, K+1, D] base outputs, d_logalpha [B, K],
+ * d_muhat [B, K, D] drafter means, d_eps [B, K+1, D] base outputs, d_logalpha [B, K] (entries of draft
+ * slots beyond an environment's window K_eff = min(K, t) are unspecified in the first three, 0 in the last),
  * h_jstar [B] (HOST; first rejected step, K_eff+1 if none, -1 if the environment was finished).
  * Synchronous. */
 int tsdp_round(tsdp_ctx* ctx, const float* d_obs, int B, int K, const tsdp_accept_t* accept, uint64_t seed,
@@ -302,10 +309,12 @@ uint64_t tsdp_kernel_launches(const tsdp_ctx* ctx);
  * stream.  Families: 0 GEMMs of the base model (tcgen05 or check-mode), 1 LayerNorm, 2 attention,
  * 3 embed/head/memory tokens, 4 draft-step kernel, 5 MLP / Gaussian denoiser, 6 GEMMs
  * of the drafter, 7 the persistent cluster drafter, 8 the fused
- * acceptance / commit kernel, 9 the cluster kernel as verifier.  tsdp_profile(ctx, 0|1)
+ * acceptance / commit kernel, 9 the cluster kernel as verifier, 10 / 11 / 12 the drafter's LayerNorm / attention /
+ * embedding-head kernels (families 1-3 hold the base model's only).  A GEMM's flops count the rows it really
+ * processed (the live candidates of the round's plan).  tsdp_profile(ctx, 0|1)
  * clears the record.  tsdp_profile_read fills three arrays of TSDP_PROF_FAMILIES entries: summed
  * milliseconds, summed algorithmic flops (2*M*N*K per GEMM launch, 0 elsewhere) and launch counts. */
-enum { TSDP_PROF_FAMILIES = 10 };
+enum { TSDP_PROF_FAMILIES = 13 };
 int tsdp_profile(tsdp_ctx* ctx, int enable);
 int tsdp_profile_read(tsdp_ctx* ctx, double* ms, double* flop, uint64_t* launches);
 

@@ -17,7 +17,8 @@ EXPORTS = ["tsdp_init", "tsdp_destroy", "tsdp_strerror", "tsdp_last_error", "tsd
            "tsdp_round", "tsdp_denoise", "tsdp_gemm", "tsdp_gemm_timed", "tsdp_stats", "tsdp_reset_stats",
            "tsdp_kernel_launches", "tsdp_profile", "tsdp_profile_read", "tsdp_verify_commit_static", "tsdp_set_scheduler", "tsdp_set_progress",
            "tsdp_sched_eval", "tsdp_serve", "tsdp_request_counts", "tsdp_process_reward", "tsdp_distill_loss", "tsdp_distill_step"]
-PROF_FAMILIES = ["gemm", "layernorm", "attention", "embed_head", "round", "small_net", "gemm_draft", "drafter_cluster", "accept", "verifier_cluster"]
+PROF_FAMILIES = ["gemm", "layernorm", "attention", "embed_head", "round", "small_net", "gemm_draft", "drafter_cluster", "accept", "verifier_cluster",
+                 "layernorm_draft", "attention_draft", "embed_head_draft"]
 
 
 class NetT(C.Structure):
@@ -42,7 +43,7 @@ class StatsT(C.Structure):
                 ("steps_advanced", C.c_uint64), ("draft_rounds", C.c_uint64), ("nfe", C.c_double),
                 ("hist_drafted", C.c_uint64 * TSDP_MAX_T), ("hist_tested", C.c_uint64 * TSDP_MAX_T),
                 ("hist_accepted", C.c_uint64 * TSDP_MAX_T), ("call_ms_p50", C.c_double), ("call_ms_p99", C.c_double),
-                ("call_ms_samples", C.c_uint64)]
+                ("call_ms_samples", C.c_uint64), ("cand_dense", C.c_uint64), ("cand_computed", C.c_uint64)]
 
 
 class TsdpError(RuntimeError):

@@ -110,17 +110,39 @@ __device__ __forceinline__ float gelu_tanh(float v) {
 }
 __device__ __forceinline__ float silu(float v) { return v / (1.0f + __expf(-v)); }
 
-// Which candidate rows a forward pass covers: candidate n = (env b = n / C, slot c = n % C) reads its
-// latent at xin + b*x_stride_b + c*D, is evaluated at timestep clamp(t[b] - koff - c, 0, T-1) and
-// writes eps at eout + b*e_stride_b + c*D.  b is a slot of the batch; which request (environment-chunk)
-// the slot is working on is item[b].
+// Which candidate rows a forward pass covers.  Dense form (list == null): candidate n = (env b = n / C, slot
+// c = n % C).  Compacted form: candidate n = (b, c) = (list[n] >> 6, list[n] & 63), and only the first *n_live
+// entries exist -- the round's plan (round_plan_kernel) lists the candidates that are still needed, so that finished
+// environments and draft slots beyond an environment's window cost nothing.  Either way the candidate reads its
+// latent at xin + b*x_stride_b + c*D, is evaluated at timestep clamp(t[b] - koff - c, 0, T-1) and writes eps at
+// eout + b*e_stride_b + c*D.  b is a slot of the batch; which request (environment-chunk) the slot is working on
+// is item[b].
 struct CandMap {
   const float* xin;  long long x_stride_b;
   float* eout;       long long e_stride_b;
   const int* t;      int C;  int koff;
   const int* item;   // slot b currently serves request item[b] (its observation, its noise streams); null: b
+  const int* list;   // compacted candidate list (null: dense)
+  const int* n_live; // number of entries of `list` in use (device word written earlier in the stream)
 };
 __device__ __forceinline__ int item_of(const int* item, int b) { return item ? item[b] : b; }
+__device__ __forceinline__ void cand_decode(const CandMap& cm, int n, int& b, int& c) {
+  if (cm.list) { const int v = cm.list[n]; b = v >> 6; c = v & 63; }
+  else { b = n / cm.C; c = n % cm.C; }
+}
+// Candidates this pass really has (n_static is what the launch was sized for).
+__device__ __forceinline__ int cand_count(const CandMap& cm, int n_static) {
+  return cm.n_live ? min(*cm.n_live, n_static) : n_static;
+}
+// The same for kernels that only see rows: rows = *n * mul + add, never more than the launch was sized for.
+struct LiveRows {
+  const int* n;  int mul;  int add;
+};
+__device__ __forceinline__ int live_rows(const LiveRows& lv, int rows_static) {
+  if (lv.n == nullptr) return rows_static;
+  const int v = *lv.n * lv.mul + lv.add;
+  return v < 0 ? 0 : (v < rows_static ? v : rows_static);
+}
 
 // Per-round speculative parameters (the scheduler's action space, Sec. 3.3: draft steps, acceptance
 // threshold, sigma scale).
@@ -153,7 +175,7 @@ __device__ __forceinline__ int env_draft_cap(const EnvParams* envp, int env, int
 // Device-side counters behind tsdp_stats.
 struct DevStats {
   unsigned long long env_rounds, base_evals, draft_evals, drafts_tested, drafts_accepted, rejections,
-      bonus_steps, steps_advanced, chunks_done, draft_rounds;
+      bonus_steps, steps_advanced, chunks_done, draft_rounds, cand_computed, draft_computed;
   unsigned long long hist_drafted[1024], hist_tested[1024], hist_accepted[1024];
 };
 

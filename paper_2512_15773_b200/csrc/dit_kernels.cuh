@@ -17,8 +17,9 @@ __global__ void silu_inplace_kernel(float* __restrict__ x, long long n) {
 }
 
 __device__ __forceinline__ int row_tau(const CandMap& cm, int row, int H, int Tsteps) {
-  const int n = row / H;
-  int tau = cm.t[n / cm.C] - cm.koff - (n % cm.C);
+  int b, c;
+  cand_decode(cm, row / H, b, c);
+  const int tau = cm.t[b] - cm.koff - c;
   return max(0, min(Tsteps - 1, tau));
 }
 
@@ -32,7 +33,7 @@ __global__ void ln_mod_kernel(const float* __restrict__ h, const float* __restri
   constexpr int d = VEC * 128;
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
-  if (row >= M) return;
+  if (row >= M || row / H >= cand_count(cm, M / H)) return;
   float4 v[VEC];
   float s = 0.f;
 #pragma unroll
@@ -69,7 +70,7 @@ __global__ void head_mod_kernel(const float* __restrict__ h, const float* __rest
   constexpr int d = VEC * 128;
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
-  if (row >= M) return;
+  if (row >= M || row / H >= cand_count(cm, M / H)) return;
   float4 v[VEC];
   float s = 0.f;
 #pragma unroll
@@ -95,7 +96,8 @@ __global__ void head_mod_kernel(const float* __restrict__ h, const float* __rest
     v[j].z = v[j].z * rstd * (1.0f + sc.z) + sh.z; v[j].w = v[j].w * rstd * (1.0f + sc.w) + sh.w;
   }
   const int n = row / H, i = row % H;
-  const int b = n / cm.C, c = n % cm.C;
+  int b, c;
+  cand_decode(cm, n, b, c);
   float* o = cm.eout + b * cm.e_stride_b + (long long)c * H * A + (long long)i * A;
   for (int a = 0; a < A; ++a) {
     float acc = 0.f;
@@ -122,8 +124,9 @@ __global__ void cross_attn_ctx_simt_kernel(const T* __restrict__ q, T* __restric
   extern __shared__ float sm_ctx[];                       // per warp: Tc scores
   const int wpb = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = blockIdx.x * wpb + warp;
-  if (row >= M) return;
-  const int n = row / H, b = n / cm.C;
+  if (row >= M || row / H >= cand_count(cm, M / H)) return;
+  int b, c_unused;
+  cand_decode(cm, row / H, b, c_unused);
   const int dh = d / heads;
   const T* kvb = kv + (size_t)item_of(cm.item, b) * Tc * ld_kv + kv_off;
   float* sc = sm_ctx + (size_t)warp * Tc;
@@ -167,7 +170,7 @@ template <int DH>
 __global__ void __launch_bounds__(CX_WARPS * 32)
 cross_attn_ctx_mma_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out,
                           const __nv_bfloat16* __restrict__ kv, long long ld_kv, int kv_off, CandMap cm, int rows_per_slot,
-                          int d, int heads, int Tc) {
+                          int d, int heads, int Tc, const int* __restrict__ slot_start, int H) {
   pdl_trigger();
   pdl_wait();
   extern __shared__ __align__(16) uint8_t cx_raw[];
@@ -175,8 +178,21 @@ cross_attn_ctx_mma_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __
   constexpr int CX_U = 1;      // query tiles a warp processes together (2 costs more in occupancy than it saves in shared-memory reads)
   __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(cx_raw);
   __nv_bfloat16* Vs = Ks + (size_t)Tc * P;
-  const int b = blockIdx.x / heads, hd = blockIdx.x % heads;
+  int b = blockIdx.x / heads;
+  const int hd = blockIdx.x % heads;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, tg = lane & 3;
+  // Rows of group b.  Dense layout: slot b owns [b * rows_per_slot, +rows_per_slot).  Compacted candidate list
+  // with slot_start: slot b's candidates are the list entries slot_start[b] .. slot_start[b + 1] - 1, H rows each.
+  // Compacted list without slot_start (one candidate per slot, C = 1): group b is list entry b, slot list[b] >> 6.
+  size_t row0 = (size_t)b * rows_per_slot;
+  if (slot_start != nullptr) {
+    row0 = (size_t)slot_start[b] * H;
+    rows_per_slot = (slot_start[b + 1] - slot_start[b]) * H;
+    if (rows_per_slot <= 0) return;
+  } else if (cm.list != nullptr) {
+    if (b >= cand_count(cm, (int)(gridDim.x / heads))) return;
+    b = cm.list[b] >> 6;
+  }
   const __nv_bfloat16* kvb = kv + (size_t)item_of(cm.item, b) * Tc * ld_kv + kv_off + hd * DH;
   constexpr int VPR = DH / 8;
   for (int i = threadIdx.x; i < Tc * VPR; i += blockDim.x) {
@@ -186,7 +202,6 @@ cross_attn_ctx_mma_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __
   }
   __syncthreads();
   const float scale = rsqrtf((float)DH);
-  const size_t row0 = (size_t)b * rows_per_slot;
   // A warp works on CX_U query tiles at a time, so that every key / value fragment read from shared
   // memory feeds CX_U tensor-core instructions.
   for (int pt = warp; pt * (16 * CX_U) < rows_per_slot; pt += CX_WARPS) {

@@ -19,14 +19,19 @@ __global__ void draft_tail_kernel(float* __restrict__ h, const float* __restrict
                                   const uint64_t* __restrict__ seedp, const EnvParams* __restrict__ envp,
                                   const int* __restrict__ item, const float* __restrict__ W_in, const float* __restrict__ b_in,
                                   const float* __restrict__ pos, const float* __restrict__ ln1_g, const float* __restrict__ ln1_b,
-                                  T* __restrict__ a_out, int embed_next, int M, int H, int A) {
+                                  T* __restrict__ a_out, int embed_next, int M, int H, int A,
+                                  const int* __restrict__ order, const int* __restrict__ n_live) {
   pdl_trigger();
   pdl_wait();
   constexpr int d = VEC * 128;
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= M) return;
-  const int b = row / H, l = row % H;
+  // rows n*H .. n*H+H-1 of the drafter's activations belong to slot b = n, or, when the drafter runs on the
+  // round's compacted slot order, to slot order[n] >> 6 (only the first *n_live entries are drafting at step k)
+  const int n = row / H, l = row % H;
+  if (n_live != nullptr && n >= *n_live) return;
+  const int b = order != nullptr ? (order[n] >> 6) : n;
   const int D = H * A;
   float4 v[VEC];
   head_ln_row<VEC>(h + (size_t)row * d, lnf_g, lnf_b, v, lane);

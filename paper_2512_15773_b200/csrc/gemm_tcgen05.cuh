@@ -206,11 +206,15 @@ struct GemmArgs {
   // is the 5 conv_c elements starting at tensor row m, so k-block kb is tensor rows m + tap, columns
   // [c0, c0 + 64) with tap = (64 kb) / conv_c, c0 = (64 kb) % conv_c; conv_c is a multiple of 64.
   int conv_c;
+  // Rows that really exist when the forward runs on a compacted candidate list: min(M, *live.n * live.mul + live.add)
+  // (live.n null: M).  The tensor maps keep their full extent; tiles beyond the live rows are simply not visited.
+  LiveRows live;
+  const int* list;      // EPI_GATE with a compacted list: candidate n of a row is (list[n] >> 6, list[n] & 63)
 };
 
 __device__ __forceinline__ const float* gate_row(const GemmArgs& g, int row) {
   const int n = row / g.H;
-  int tau = g.t[n / g.C] - g.koff - (n % g.C);
+  int tau = g.list ? g.t[g.list[n] >> 6] - g.koff - (g.list[n] & 63) : g.t[n / g.C] - g.koff - (n % g.C);
   tau = max(0, min(g.Tsteps - 1, tau));
   return g.gate + (size_t)tau * g.gate_ld;
 }
@@ -280,9 +284,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - ptx::smem_u32(smem_raw)));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tiles_m = (g.M + GEMM_BM - 1) / GEMM_BM;
   const int tiles_n = g.N / BN;
-  const int n_tiles = tiles_m * tiles_n;
   const int kblocks = g.K / GEMM_BK;
 
   if (threadIdx.x == 0) {
@@ -300,7 +302,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_ptr;
   bool ok = true;
-  pdl_wait();      // operands, bias and the output belong to earlier kernels of the stream
+  pdl_wait();      // operands, bias, the output and the live-row count belong to earlier kernels of the stream
+  const int M = live_rows(g.live, g.M);
+  const int tiles_m = (M + GEMM_BM - 1) / GEMM_BM;
+  const int n_tiles = tiles_m * tiles_n;
 
   if (warp == 0) {
     if (lane == 0) {
@@ -396,7 +401,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               for (int i = 0; i < 32; ++i) f[i] = ptx::gelu_fast(f[i]);
             }
             if (EPI == EPI_GATE) {
-              const int grow = min(tm * GEMM_BM + r, g.M - 1);     // rows past M are clipped by the TMA store
+              const int grow = min(tm * GEMM_BM + r, M - 1);       // rows past the live ones only reach rows nobody reads
               const float4* gp = reinterpret_cast<const float4*>(gate_row(g, grow) + col);
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
@@ -447,7 +452,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           uint32_t v[16];
           ptx::tmem_ld16(taddr + (uint32_t)c, v);
           ptx::tmem_ld_wait();
-          if (row < g.M) epilogue_store16<EPI>(g, row, tn * BN + half * COLS + c, v);
+          if (row < M) epilogue_store16<EPI>(g, row, tn * BN + half * COLS + c, v);
         }
         ptx::tc_fence_before();
         __syncwarp();

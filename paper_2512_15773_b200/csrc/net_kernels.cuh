@@ -18,6 +18,8 @@ gemm_simt_kernel(const float* __restrict__ A, const float* __restrict__ W, GemmA
   __shared__ float As[16][65], Ws[16][65];
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
   const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+  g.M = live_rows(g.live, g.M);
+  if (m0 >= g.M) return;
   float acc[4][4] = {};
   for (int k0 = 0; k0 < g.K; k0 += 16) {
     for (int i = threadIdx.x; i < 64 * 16; i += 256) {
@@ -65,7 +67,9 @@ __global__ void embed_kernel(CandMap cm, const float* __restrict__ W_in, const f
   pdl_wait();
   const int row = blockIdx.x;
   const int n = row / H, i = row % H;
-  const int b = n / cm.C, c = n % cm.C;
+  if (n >= cand_count(cm, gridDim.x / H)) return;
+  int b, c;
+  cand_decode(cm, n, b, c);
   const float* x = cm.xin + b * cm.x_stride_b + (long long)c * H * A + (long long)i * A;
   for (int col = threadIdx.x; col < d; col += blockDim.x) {
     float v = b_in[col] + pos[i * d + col];
@@ -112,13 +116,13 @@ __device__ __forceinline__ void store4(__nv_bfloat16* o, float a, float b, float
 
 template <typename T, int VEC>
 __global__ void ln_kernel(const float* __restrict__ h, const float* __restrict__ gam, const float* __restrict__ bet,
-                          T* __restrict__ out, int M) {
+                          T* __restrict__ out, int M, LiveRows lv) {
   pdl_trigger();
   pdl_wait();
   constexpr int d = VEC * 128;
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
-  if (row >= M) return;
+  if (row >= live_rows(lv, M)) return;
   float4 v[VEC];
   float s = 0.f;
 #pragma unroll
@@ -204,7 +208,9 @@ __global__ void embed_ln_kernel(CandMap cm, const float* __restrict__ W_in, cons
   const int lane = threadIdx.x & 31;
   if (row >= M) return;
   const int n = row / H, i = row % H;
-  const int b = n / cm.C, c = n % cm.C;
+  if (n >= cand_count(cm, M / H)) return;
+  int b, c;
+  cand_decode(cm, n, b, c);
   const float* x = cm.xin + b * cm.x_stride_b + (long long)c * H * A + (long long)i * A;
   embed_ln_row<T, VEC>([&](int a) { return x[a]; }, A, W_in, b_in, pos + (size_t)i * d, h + (size_t)row * d, gam, bet,
                        out + (size_t)row * d, lane);
@@ -216,9 +222,10 @@ __global__ void embed_ln_kernel(CandMap cm, const float* __restrict__ W_in, cons
 // ------------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void self_attn_kernel(const T* __restrict__ qkv, T* __restrict__ out, int n_cand, int H, int d,
-                                 int heads, int causal) {
+                                 int heads, int causal, LiveRows lv) {
   pdl_trigger();
   pdl_wait();
+  n_cand = live_rows(lv, n_cand);
   extern __shared__ float sm[];
   const int dh = d / heads;
   const int wpb = blockDim.x >> 5;
@@ -282,7 +289,9 @@ __global__ void cross_attn_kernel(const T* __restrict__ q, T* __restrict__ out, 
   const int lane = threadIdx.x & 31;
   if (row >= M) return;
   const int n = row / H;
-  const int b = n / cm.C, c = n % cm.C;
+  if (n >= cand_count(cm, M / H)) return;
+  int b, c;
+  cand_decode(cm, n, b, c);
   int tau = cm.t[b] - cm.koff - c;
   tau = max(0, min(Tsteps - 1, tau));
   const int dh = d / heads;
@@ -352,9 +361,10 @@ constexpr int SA_WARPS = 4;
 template <int DH>
 __global__ void __launch_bounds__(SA_WARPS * 32)
 self_attn_mma_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ out, int n_cand, int H, int d,
-                     int heads, int causal) {
+                     int heads, int causal, LiveRows lv) {
   pdl_trigger();
   pdl_wait();
+  n_cand = live_rows(lv, n_cand);
   constexpr int KS = DH / 16;        // k-steps of Q K^T
   constexpr int NO = DH / 8;         // n-tiles of the output
   constexpr int LDS = DH + 8;        // staging row pitch (elements); keeps 16-byte alignment
@@ -477,9 +487,10 @@ self_attn_mma_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __res
 template <int DH>
 __global__ void __launch_bounds__((DH > 64 ? 2 : 4) * 32)
 self_attn_tile_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ out, int n_cand, int H, int d,
-                      int heads, int causal) {
+                      int heads, int causal, LiveRows lv) {
   pdl_trigger();
   pdl_wait();
+  n_cand = live_rows(lv, n_cand);
   constexpr int TW = DH > 64 ? 2 : 4;
   constexpr int KS = DH / 16, NO = DH / 8, P = DH + 8, VPR = DH / 8;
   __shared__ __align__(16) __nv_bfloat16 sm[TW][3][16 * P];
@@ -603,13 +614,14 @@ self_attn_tile_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __re
 template <int DH>
 __global__ void __launch_bounds__(128)
 self_attn_staged_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ out, int n_cand, int H, int d,
-                        int heads, int causal) {
+                        int heads, int causal, LiveRows lv) {
   pdl_trigger();
   pdl_wait();
   constexpr int KS = DH / 16, NO = DH / 8, P = DH + 8, VPR = DH / 8;
   __shared__ __align__(16) __nv_bfloat16 Ks[64 * P], Vs[64 * P];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, tg = lane & 3;
   const int n = blockIdx.x / heads, hd = blockIdx.x % heads;
+  if (n >= live_rows(lv, n_cand)) return;
   const size_t ld = (size_t)3 * d;
   const __nv_bfloat16* base = qkv + (size_t)n * H * ld + (size_t)hd * DH;
   for (int i = threadIdx.x; i < 64 * VPR; i += blockDim.x) {
@@ -731,11 +743,14 @@ cross_attn_group_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __re
   // a group works on CA_ROWS consecutive query rows of its (candidate, head): more groups in flight than
   // one per (candidate, head) would give, at the price of re-reading the few keys / values from cache
   const int row_chunks = (H + CA_ROWS - 1) / CA_ROWS;
+  n_cand = cand_count(cm, n_cand);
+  if (n_cand <= 0) return;
   const bool live = gid_raw < n_cand * heads * row_chunks;
   const int gid_c = live ? gid_raw : n_cand * heads * row_chunks - 1;
   const int rc = gid_c % row_chunks, gid = gid_c / row_chunks;
   const int n = gid / heads, hd = gid % heads;
-  const int b = n / cm.C, c = n % cm.C;
+  int b, c;
+  cand_decode(cm, n, b, c);
   int tau = cm.t[b] - cm.koff - c;
   tau = max(0, min(Tsteps - 1, tau));
   const size_t ldkv = (size_t)L * 2 * d;
@@ -854,10 +869,12 @@ __global__ void head_kernel(const float* __restrict__ h, const float* __restrict
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= M) return;
+  const int n = row / H, i = row % H;
+  if (n >= cand_count(cm, M / H)) return;
   float4 v[VEC];
   head_ln_row<VEC>(h + (size_t)row * d, gam, bet, v, lane);
-  const int n = row / H, i = row % H;
-  const int b = n / cm.C, c = n % cm.C;
+  int b, c;
+  cand_decode(cm, n, b, c);
   float* o = cm.eout + b * cm.e_stride_b + (long long)c * H * A + (long long)i * A;
   for (int a = 0; a < A; ++a) {
     const float e = head_out<VEC>(v, W_outT + (size_t)a * d, b_out[a], lane);
@@ -885,7 +902,9 @@ __global__ void mlp_forward_kernel(MlpWeights w, CandMap cm, const float* __rest
   pdl_wait();
   extern __shared__ float sm[];
   const int n = blockIdx.x;
-  const int b = n / cm.C, c = n % cm.C;
+  if (n >= cand_count(cm, gridDim.x)) return;
+  int b, c;
+  cand_decode(cm, n, b, c);
   int tau = cm.t[b] - cm.koff - c;
   tau = max(0, min(Tsteps - 1, tau));
   int maxw = 0;
@@ -922,7 +941,9 @@ __global__ void gauss_forward_kernel(DdpmTables S, float m0, float s0, CandMap c
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (long long)n_cand * D) return;
   const int n = (int)(idx / D), i = (int)(idx % D);
-  const int b = n / cm.C, c = n % cm.C;
+  if (n >= cand_count(cm, n_cand)) return;
+  int b, c;
+  cand_decode(cm, n, b, c);
   int tau = cm.t[b] - cm.koff - c;
   tau = max(0, min(S.T - 1, tau));
   const float sab = S.sqrt_ab[tau], s1 = S.sqrt_1mab[tau];

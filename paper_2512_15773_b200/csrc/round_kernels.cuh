@@ -7,6 +7,9 @@
 
 namespace tsdp {
 
+constexpr int TSDP_PLAN_MAXK = 32;      // = TSDP_MAX_K of the C ABI
+
+
 // x_T ~ N(0, I), t = T-1 for every environment.  xt holds the round's candidate latents
 // [B, Kmax+1, D]; slot 0 is the current latent x.
 __global__ void init_chunk_kernel(float* __restrict__ xt, long long xs_b, int* __restrict__ t, int B, int D,
@@ -28,6 +31,110 @@ __global__ void init_chunk_kernel(float* __restrict__ xt, long long xs_b, int* _
     t[b] = T - 1;
     item[b] = b;                         // slot b starts on request b; further requests are taken from queue_head on
     if (b == 0) { *round_idx = 0; *n_done = 0; *queue_head = B; }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Plan of a round (first kernel of the round): which candidates the base model must evaluate and which slots the
+// drafter must run at each draft step, as dense lists, so that finished environments, draft slots beyond an
+// environment's window K_eff = min(K, scheduler cap, t) (Sec. 3.2: drafting stops at K or at t = 0) and an unused
+// bonus slot cost no network rows.
+//   live_list[0 .. *live_n)       : (b << 6) | c for b ascending, c = 0 .. n_base(b) - 1,
+//                                   n_base = K_eff + 1 if the bonus step can be taken (or K_eff = 0), else K_eff
+//   slot_start[b], slot_start[B]  : first list entry of slot b / the total (a slot's candidates are contiguous)
+//   order[0 .. dn[1])             : (b << 6) of the drafting slots, longest window first (stable in b), so that the
+//                                   slots drafting at step k are the prefix order[0 .. dn[k])
+//   dn[k], k = 1..K               : slots with K_eff >= k
+// One block of PLAN_THREADS threads; B <= PLAN_MAX_B.
+// ------------------------------------------------------------------------------------------------
+constexpr int PLAN_THREADS = 1024;
+constexpr int PLAN_MAX_B = 4096;
+constexpr int PLAN_PER_THREAD = PLAN_MAX_B / PLAN_THREADS;
+
+__global__ void __launch_bounds__(PLAN_THREADS)
+round_plan_kernel(const int* __restrict__ t, int B, int K, const RoundParams* __restrict__ sched, int n_sched,
+                  const int* __restrict__ round_idx, const EnvParams* __restrict__ envp, const int* __restrict__ item,
+                  int Tsteps, int* __restrict__ live_n, int* __restrict__ live_list, int* __restrict__ slot_start,
+                  int* __restrict__ order, int* __restrict__ dn, DevStats* __restrict__ stats) {
+  pdl_trigger();
+  pdl_wait();
+  __shared__ signed char s_ke[PLAN_MAX_B];          // K_eff of each slot, -1: finished
+  __shared__ int s_warp[PLAN_THREADS / 32];
+  __shared__ int s_hist[TSDP_PLAN_MAXK + 2];        // slots with K_eff == k
+  __shared__ int s_base[TSDP_PLAN_MAXK + 2];        // first position in `order` of the slots with K_eff == k
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int bonus = sched[min(*round_idx, n_sched - 1)].bonus;
+  if (tid < TSDP_PLAN_MAXK + 2) s_hist[tid] = 0;
+  __syncthreads();
+  // ---- per slot: K_eff and the number of candidates the base model must see
+  int nb[PLAN_PER_THREAD], mine = 0;
+#pragma unroll
+  for (int j = 0; j < PLAN_PER_THREAD; ++j) {
+    const int b = tid * PLAN_PER_THREAD + j;
+    int ke = -1, n = 0;
+    if (b < B) {
+      const int tb = t[b];
+      if (tb >= 0) {
+        ke = min(env_draft_cap(envp, item_of(item, b), tb, K, Tsteps), tb);
+        n = (bonus || ke == 0) ? ke + 1 : ke;
+        if (ke > 0) atomicAdd(&s_hist[ke], 1);
+      }
+      s_ke[b] = (signed char)ke;
+    }
+    nb[j] = n; mine += n;
+  }
+  // ---- exclusive scan of the candidate counts over the slots
+  int incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  if (lane == 31) s_warp[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int w = s_warp[lane];
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, w, o);
+      if (lane >= o) w += v;
+    }
+    s_warp[lane] = w;                               // inclusive over warps
+  }
+  __syncthreads();
+  int start = incl - mine + (warp > 0 ? s_warp[warp - 1] : 0);
+  const int total = s_warp[PLAN_THREADS / 32 - 1];
+#pragma unroll
+  for (int j = 0; j < PLAN_PER_THREAD; ++j) {
+    const int b = tid * PLAN_PER_THREAD + j;
+    if (b < B) {
+      slot_start[b] = start;
+      for (int c = 0; c < nb[j]; ++c) live_list[start + c] = (b << 6) | c;
+      start += nb[j];
+    }
+  }
+  // ---- draft order: counting sort by K_eff, longest first; dn[k] = slots with K_eff >= k
+  if (tid == 0) {
+    slot_start[B] = total;
+    *live_n = total;
+    int run = 0, drafts = 0;
+    for (int k = K; k >= 1; --k) { s_base[k] = run; run += s_hist[k]; dn[k] = run; drafts += run; }
+    dn[0] = B;
+    atomicAdd(&stats->cand_computed, (unsigned long long)total);
+    atomicAdd(&stats->draft_computed, (unsigned long long)drafts);
+  }
+  __syncthreads();
+  // warp w places the slots whose K_eff is w + 1 (K <= 32 = the number of warps), in slot order
+  const int k = warp + 1;
+  if (k <= K) {
+    int pos = s_base[k];
+    for (int b0 = 0; b0 < B; b0 += 32) {
+      const int b = b0 + lane;
+      const bool hit = b < B && s_ke[b] == k;
+      const unsigned m = __ballot_sync(0xffffffffu, hit);
+      if (hit) order[pos + __popc(m & ((1u << lane) - 1u))] = b << 6;
+      pos += __popc(m);
+    }
   }
 }
 

@@ -138,6 +138,18 @@ struct tsdp_ctx {
   int cv_smem = 0, cv_max_clusters = 0;
   uint64_t rounds = 0, launches = 0;
   int launches_per_round_tmp = 0;
+  // plan of a round (round_plan_kernel): compacted candidate list of the verification forward, slot order and
+  // per-step counts of the drafter; `compact` off: every forward runs on the dense B x (K+1) layout
+  bool compact = true;
+  int *plan_live_n = nullptr, *plan_list = nullptr, *plan_slot_start = nullptr, *plan_order = nullptr, *plan_dn = nullptr;
+  // live-row information of the forward pass being enqueued (set by forward(), read by the launch helpers)
+  const int* live_n = nullptr;
+  const int* live_slot_start = nullptr;
+  int live_static = 0;
+  // while profiling: host copies of the plan's counts, so that a GEMM's flops are those of the rows it really processed
+  int prof_plan_live = -1, prof_plan_dn[TSDP_MAX_K + 2] = {};
+  int prof_live_count = -1;                   // live candidates of the forward being enqueued (-1: unknown, use the dense count)
+  uint64_t cand_static = 0;                   // candidates the dense layout would have evaluated since the last reset
   // optional per-kernel-family timing with CUDA events (plain launches, no graph)
   bool prof_on = false;
   int prof_gemm_cat = 0;                      // 0 while the base model runs, 6 while the drafter runs
@@ -194,6 +206,7 @@ void launch_kernel(tsdp_ctx* c, void (*kern)(P...), dim3 grid, dim3 block, size_
 constexpr size_t PROF_CAP = 60000;
 void prof_begin(tsdp_ctx* c, cudaStream_t s, int cat, double flop) {
   if (!c->prof_on || c->prof_cat.size() >= PROF_CAP) return;
+  if (c->prof_gemm_cat == 6 && cat >= 1 && cat <= 3) cat += 9;      // the drafter's LayerNorm / attention / embedding-head kernels
   cudaEvent_t a, b;
   if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) return;
   c->prof_ev.push_back(a); c->prof_ev.push_back(b);
@@ -204,6 +217,9 @@ void prof_end(tsdp_ctx* c, cudaStream_t s) {
   if (!c->prof_on || c->prof_ev.empty() || c->prof_ev.size() != 2 * c->prof_cat.size()) return;
   cudaEventRecord(c->prof_ev.back(), s);
 }
+
+// Live-row descriptor for a kernel whose launch was sized for `per` rows per candidate of the current forward.
+LiveRows live_desc(const tsdp_ctx* c, int per, int add = 0) { return LiveRows{c->live_n, per, add}; }
 
 // (C_in, C_out) of the residual blocks of the conv UNet in execution order: two per level down, two in the
 // middle, two per level up (the first of which takes the concatenation [upsampled | skip]).
@@ -299,12 +315,20 @@ int get_map(tsdp_ctx* c, const void* ptr, int esz, int rows, int cols, int ld, i
   return TSDP_OK;
 }
 
+// Rows a GEMM of the forward being enqueued really processes, as far as the host knows (profiling mode reads the
+// round's plan back); otherwise the dense count.
+int gemm_rows_known(const tsdp_ctx* c, const GemmArgs& g) {
+  if (g.live.n == nullptr || c->prof_live_count < 0) return g.M;
+  const int v = c->prof_live_count * g.live.mul + g.live.add;
+  return v < 0 ? 0 : (v < g.M ? v : g.M);
+}
+
 template <int BN, int EPI>
 int launch_tc(tsdp_ctx* c, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const GemmArgs& g,
               cudaStream_t s) {
   const int tiles = ((g.M + GEMM_BM - 1) / GEMM_BM) * (g.N / BN);
   const int grid = tiles < c->num_sms ? tiles : c->num_sms;
-  prof_begin(c, s, c->prof_gemm_cat, 2.0 * g.M * g.N * g.K);
+  prof_begin(c, s, c->prof_gemm_cat, 2.0 * gemm_rows_known(c, g) * g.N * g.K);
   TSDP_LAUNCH(c, (gemm_tcgen05_kernel<BN, EPI>), grid, GEMM_THREADS, gemm_smem_bytes(BN), s, ma, mb, mc, g);
   prof_end(c, s);
   c->launches_per_round_tmp++;
@@ -362,17 +386,24 @@ struct GateSpec {
 int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, int N, int K, int epi, void* out,
          int ldo, cudaStream_t s, const GateSpec* gs = nullptr, int conv_c = 0) {
   if (M <= 0) return TSDP_OK;
-  GemmArgs g{M, N, K, bias, out, ldo, c->status, nullptr, 0, nullptr, 1, 0, 1, 1, conv_c > 0 ? conv_c : K, conv_c};
+  GemmArgs g{M, N, K, bias, out, ldo, c->status, nullptr, 0, nullptr, 1, 0, 1, 1, conv_c > 0 ? conv_c : K, conv_c,
+             LiveRows{nullptr, 0, 0}, nullptr};
   if (epi == EPI_GATE) {
     if (!gs) return TSDP_ERR_ARG;
     g.gate = gs->gate; g.gate_ld = gs->gate_ld; g.t = gs->cm->t; g.C = gs->cm->C; g.koff = gs->cm->koff; g.H = gs->H;
-    g.Tsteps = gs->Tsteps;
+    g.Tsteps = gs->Tsteps; g.list = gs->cm->list;
+  }
+  if (c->live_n != nullptr && c->live_static > 0) {
+    // rows per candidate of this GEMM: M = n rows_per (token rows), or n rows_per - 4 (a convolution over padded tensors)
+    const int n = c->live_static;
+    if (M % n == 0) g.live = LiveRows{c->live_n, M / n, 0};
+    else if ((M + 4) % n == 0) g.live = LiveRows{c->live_n, (M + 4) / n, -4};
   }
   if (c->cfg.precision == 0) {
     dim3 grid((N + 63) / 64, (M + 63) / 64);
     const float* a = reinterpret_cast<const float*>(A);
     const float* w = reinterpret_cast<const float*>(W);
-    prof_begin(c, s, c->prof_gemm_cat, 2.0 * M * N * K);
+    prof_begin(c, s, c->prof_gemm_cat, 2.0 * gemm_rows_known(c, g) * N * K);
     switch (epi) {
       case EPI_GELU: TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_GELU>), grid, 256, 0, s, a, w, g); break;
       case EPI_RESID: TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_RESID>), grid, 256, 0, s, a, w, g); break;
@@ -416,7 +447,7 @@ int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, in
 // fp32 CUDA-core GEMM whatever the precision mode: the timestep-conditioning tables built at weight load.
 int gemm_f32(tsdp_ctx* c, const float* A, const float* W, const float* bias, int M, int N, int K, int epi, float* out,
              cudaStream_t s) {
-  GemmArgs g{M, N, K, bias, out, N, c->status, nullptr, 0, nullptr, 1, 0, 1, 1, K, 0};
+  GemmArgs g{M, N, K, bias, out, N, c->status, nullptr, 0, nullptr, 1, 0, 1, 1, K, 0, LiveRows{nullptr, 0, 0}, nullptr};
   dim3 grid((N + 63) / 64, (M + 63) / 64);
   if (epi == EPI_MISH) TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_MISH>), grid, 256, 0, s, A, W, g);
   else if (epi == EPI_SILU) TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_SILU>), grid, 256, 0, s, A, W, g);
@@ -432,14 +463,14 @@ int ln_launch(tsdp_ctx* c, const float* h, const float* g, const float* b, T* ou
   const int grid = (M + wpb - 1) / wpb;
   prof_begin(c, s, 1, 0.0);
   switch (d / 128) {
-    case 1: TSDP_LAUNCH(c, (ln_kernel<T, 1>), grid, wpb * 32, 0, s, h, g, b, out, M); break;
-    case 2: TSDP_LAUNCH(c, (ln_kernel<T, 2>), grid, wpb * 32, 0, s, h, g, b, out, M); break;
-    case 3: TSDP_LAUNCH(c, (ln_kernel<T, 3>), grid, wpb * 32, 0, s, h, g, b, out, M); break;
-    case 4: TSDP_LAUNCH(c, (ln_kernel<T, 4>), grid, wpb * 32, 0, s, h, g, b, out, M); break;
-    case 5: TSDP_LAUNCH(c, (ln_kernel<T, 5>), grid, wpb * 32, 0, s, h, g, b, out, M); break;
-    case 6: TSDP_LAUNCH(c, (ln_kernel<T, 6>), grid, wpb * 32, 0, s, h, g, b, out, M); break;
-    case 7: TSDP_LAUNCH(c, (ln_kernel<T, 7>), grid, wpb * 32, 0, s, h, g, b, out, M); break;
-    default: TSDP_LAUNCH(c, (ln_kernel<T, 8>), grid, wpb * 32, 0, s, h, g, b, out, M); break;
+    case 1: TSDP_LAUNCH(c, (ln_kernel<T, 1>), grid, wpb * 32, 0, s, h, g, b, out, M, live_desc(c, c->cfg.H)); break;
+    case 2: TSDP_LAUNCH(c, (ln_kernel<T, 2>), grid, wpb * 32, 0, s, h, g, b, out, M, live_desc(c, c->cfg.H)); break;
+    case 3: TSDP_LAUNCH(c, (ln_kernel<T, 3>), grid, wpb * 32, 0, s, h, g, b, out, M, live_desc(c, c->cfg.H)); break;
+    case 4: TSDP_LAUNCH(c, (ln_kernel<T, 4>), grid, wpb * 32, 0, s, h, g, b, out, M, live_desc(c, c->cfg.H)); break;
+    case 5: TSDP_LAUNCH(c, (ln_kernel<T, 5>), grid, wpb * 32, 0, s, h, g, b, out, M, live_desc(c, c->cfg.H)); break;
+    case 6: TSDP_LAUNCH(c, (ln_kernel<T, 6>), grid, wpb * 32, 0, s, h, g, b, out, M, live_desc(c, c->cfg.H)); break;
+    case 7: TSDP_LAUNCH(c, (ln_kernel<T, 7>), grid, wpb * 32, 0, s, h, g, b, out, M, live_desc(c, c->cfg.H)); break;
+    default: TSDP_LAUNCH(c, (ln_kernel<T, 8>), grid, wpb * 32, 0, s, h, g, b, out, M, live_desc(c, c->cfg.H)); break;
   }
   prof_end(c, s);
   c->launches_per_round_tmp++;
@@ -475,33 +506,34 @@ template <typename T>
 int self_attn_launch(tsdp_ctx* c, const T* qkv, T* out, int n_cand, int H, int d, int heads, cudaStream_t s,
                      int causal = 1) {
   const int dh = d / heads;
+  const LiveRows lv = live_desc(c, 1);
   prof_begin(c, s, 2, 0.0);
   if constexpr (std::is_same<T, __nv_bfloat16>::value) {
     const int QT = (H + 15) / 16;
     const int grid = (n_cand * heads * QT + SA_WARPS - 1) / SA_WARPS;
     if (H > 16 && (dh == 32 || dh == 64 || dh == 128)) {     // several query tiles share a head's K/V: stage them once
       const int g2 = n_cand * heads;
-      if (dh == 32) TSDP_LAUNCH(c, (self_attn_staged_kernel<32>), g2, 128, 0, s, qkv, out, n_cand, H, d, heads, causal);
-      else if (dh == 64) TSDP_LAUNCH(c, (self_attn_staged_kernel<64>), g2, 128, 0, s, qkv, out, n_cand, H, d, heads, causal);
-      else TSDP_LAUNCH(c, (self_attn_staged_kernel<128>), g2, 128, 0, s, qkv, out, n_cand, H, d, heads, causal);
+      if (dh == 32) TSDP_LAUNCH(c, (self_attn_staged_kernel<32>), g2, 128, 0, s, qkv, out, n_cand, H, d, heads, causal, lv);
+      else if (dh == 64) TSDP_LAUNCH(c, (self_attn_staged_kernel<64>), g2, 128, 0, s, qkv, out, n_cand, H, d, heads, causal, lv);
+      else TSDP_LAUNCH(c, (self_attn_staged_kernel<128>), g2, 128, 0, s, qkv, out, n_cand, H, d, heads, causal, lv);
     } else if (H <= 16 && (dh == 32 || dh == 64 || dh == 128)) {   // one 16-row tile: operands staged per warp
       const int tw = dh > 64 ? 2 : 4, g3 = (n_cand * heads + tw - 1) / tw;
-      if (dh == 32) TSDP_LAUNCH(c, (self_attn_tile_kernel<32>), g3, tw * 32, 0, s, qkv, out, n_cand, H, d, heads, causal);
-      else if (dh == 64) TSDP_LAUNCH(c, (self_attn_tile_kernel<64>), g3, tw * 32, 0, s, qkv, out, n_cand, H, d, heads, causal);
-      else TSDP_LAUNCH(c, (self_attn_tile_kernel<128>), g3, tw * 32, 0, s, qkv, out, n_cand, H, d, heads, causal);
+      if (dh == 32) TSDP_LAUNCH(c, (self_attn_tile_kernel<32>), g3, tw * 32, 0, s, qkv, out, n_cand, H, d, heads, causal, lv);
+      else if (dh == 64) TSDP_LAUNCH(c, (self_attn_tile_kernel<64>), g3, tw * 32, 0, s, qkv, out, n_cand, H, d, heads, causal, lv);
+      else TSDP_LAUNCH(c, (self_attn_tile_kernel<128>), g3, tw * 32, 0, s, qkv, out, n_cand, H, d, heads, causal, lv);
     } else
     switch (dh) {
-      case 32: TSDP_LAUNCH(c, (self_attn_mma_kernel<32>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads, causal); break;
-      case 64: TSDP_LAUNCH(c, (self_attn_mma_kernel<64>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads, causal); break;
-      case 96: TSDP_LAUNCH(c, (self_attn_mma_kernel<96>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads, causal); break;
-      default: TSDP_LAUNCH(c, (self_attn_mma_kernel<128>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads, causal); break;
+      case 32: TSDP_LAUNCH(c, (self_attn_mma_kernel<32>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads, causal, lv); break;
+      case 64: TSDP_LAUNCH(c, (self_attn_mma_kernel<64>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads, causal, lv); break;
+      case 96: TSDP_LAUNCH(c, (self_attn_mma_kernel<96>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads, causal, lv); break;
+      default: TSDP_LAUNCH(c, (self_attn_mma_kernel<128>), grid, SA_WARPS * 32, 0, s, qkv, out, n_cand, H, d, heads, causal, lv); break;
     }
   } else {
     const size_t per_warp = (size_t)(H * dh + 2 * H * (dh + 1)) * sizeof(float);
     int wpb = (int)((200 * 1024) / per_warp);      // the opt-in shared-memory limit set at init
     wpb = wpb > 4 ? 4 : (wpb < 1 ? 1 : wpb);
     const size_t smem = (size_t)wpb * per_warp;
-    TSDP_LAUNCH(c, (self_attn_kernel<T>), (n_cand * heads + wpb - 1) / wpb, wpb * 32, smem, s, qkv, out, n_cand, H, d, heads, causal);
+    TSDP_LAUNCH(c, (self_attn_kernel<T>), (n_cand * heads + wpb - 1) / wpb, wpb * 32, smem, s, qkv, out, n_cand, H, d, heads, causal, lv);
   }
   prof_end(c, s);
   c->launches_per_round_tmp++;
@@ -633,7 +665,8 @@ int xfmr_forward_t(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStrea
 
 // Head of the drafter, the draft step and the next step's embedding + LayerNorm in one launch (draft_tail.cuh).
 template <typename T>
-int draft_tail_launch(tsdp_ctx* c, Net& n, int B, int k, int K, bool embed_next, cudaStream_t s) {
+int draft_tail_launch(tsdp_ctx* c, Net& n, int B, int k, int K, bool embed_next, cudaStream_t s, const int* order,
+                      const int* n_live) {
   const int H = c->cfg.H, A = c->cfg.A, D = c->D, M = B * H, d = n.cfg.d;
   const long long xs_b = (long long)(c->cfg.max_K + 1) * D, ms_b = (long long)(c->cfg.max_K > 0 ? c->cfg.max_K : 1) * D;
   const int wpb = 8, grid = (M + wpb - 1) / wpb;
@@ -642,7 +675,7 @@ int draft_tail_launch(tsdp_ctx* c, Net& n, int B, int k, int K, bool embed_next,
   prof_begin(c, s, 4, 0.0);
 #define DT_CASE(V) TSDP_LAUNCH(c, (draft_tail_kernel<T, V>), grid, wpb * 32, 0, s, c->h, n.lnf_g, n.lnf_b, n.W_outT, n.b_out, c->S, c->xt, xs_b, \
                                c->muhat, ms_b, c->eps_d, c->t, k, K, c->cfg.T, c->seed, c->sched_on ? c->envp : nullptr, c->item, n.W_in, n.b_in,   \
-                               n.pos, w0.ln1_g, w0.ln1_b, a, embed_next ? 1 : 0, M, H, A)
+                               n.pos, w0.ln1_g, w0.ln1_b, a, embed_next ? 1 : 0, M, H, A, order, n_live)
   switch (d / 128) {
     case 1: DT_CASE(1); break; case 2: DT_CASE(2); break; case 3: DT_CASE(3); break; case 4: DT_CASE(4); break;
     case 5: DT_CASE(5); break; case 6: DT_CASE(6); break; case 7: DT_CASE(7); break; default: DT_CASE(8); break;
@@ -700,7 +733,7 @@ int cross_attn_ctx_launch(tsdp_ctx* c, const Net& n, const T* q2, T* out, const 
   if constexpr (std::is_same<T, __nv_bfloat16>::value) {
     if (Tc % 16 == 0 && (dh == 32 || dh == 64 || dh == 128) && n_cand % cm.C == 0) {
       const int slots = n_cand / cm.C, rows = cm.C * H;
-#define CX_CASE(DH) TSDP_LAUNCH(c, (cross_attn_ctx_mma_kernel<DH>), slots * heads, CX_WARPS * 32, cx_smem_bytes<DH>(Tc), s, q2, out, kv, ld_kv, layer * 2 * d, cm, rows, d, heads, Tc)
+#define CX_CASE(DH) TSDP_LAUNCH(c, (cross_attn_ctx_mma_kernel<DH>), slots * heads, CX_WARPS * 32, cx_smem_bytes<DH>(Tc), s, q2, out, kv, ld_kv, layer * 2 * d, cm, rows, d, heads, Tc, c->live_slot_start, H)
       if (dh == 32) CX_CASE(32); else if (dh == 64) CX_CASE(64); else CX_CASE(128);
 #undef CX_CASE
       done = true;
@@ -827,7 +860,7 @@ int unet_forward_t(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStrea
       const long long tot = (long long)n_cand * (L / 2) * C;
       prof_begin(c, s, 3, 0.0);
       TSDP_LAUNCH(c, (unet_pool_kernel<T>), (unsigned)((tot + 255) / 256), 256, 0, s, P(n.uw.CAT[lv]), Ccat, Cup, P(n.uw.P[lv]),
-                  n_cand, L / 2, C);
+                  n_cand, L / 2, C, live_desc(c, 1));
       prof_end(c, s);
       c->launches_per_round_tmp++;
       CU_TRY(c, cudaGetLastError());
@@ -846,7 +879,7 @@ int unet_forward_t(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStrea
     const int L = H >> lv, C = ch << lv, Cup = ch << (lv + 1), Ccat = Cup + C;
     const long long tot = (long long)n_cand * L * Cup;
     prof_begin(c, s, 3, 0.0);
-    TSDP_LAUNCH(c, (unet_upsample_kernel<T>), (unsigned)((tot + 255) / 256), 256, 0, s, cur, P(n.uw.CAT[lv]), Ccat, n_cand, L, Cup);
+    TSDP_LAUNCH(c, (unet_upsample_kernel<T>), (unsigned)((tot + 255) / 256), 256, 0, s, cur, P(n.uw.CAT[lv]), Ccat, n_cand, L, Cup, live_desc(c, 1));
     prof_end(c, s);
     c->launches_per_round_tmp++;
     CU_TRY(c, cudaGetLastError());
@@ -885,8 +918,21 @@ int prepare_obs(tsdp_ctx* c, Net& n, int B, cudaStream_t s) {
   return c->cfg.precision == 0 ? xfmr_prepare_obs_t<float>(c, n, B, s) : xfmr_prepare_obs_t<__nv_bfloat16>(c, n, B, s);
 }
 
-int forward(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStream_t s) {
+int forward_arch(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStream_t s);
+
+// One network forward over the candidates of `cm`.  With a compacted list the launches are still sized for n_cand
+// (the dense count, so that a captured graph stays valid) and every kernel reads the live count from the device.
+int forward(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStream_t s, const int* slot_start = nullptr) {
   if (n_cand <= 0) return TSDP_OK;
+  c->live_n = cm.n_live;
+  c->live_static = n_cand;
+  c->live_slot_start = cm.list ? slot_start : nullptr;
+  const int r = forward_arch(c, n, cm, n_cand, s);
+  c->live_n = nullptr; c->live_static = 0; c->live_slot_start = nullptr;
+  return r;
+}
+
+int forward_arch(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStream_t s) {
   const int D = c->D;
   switch (n.cfg.arch) {
     case TSDP_ARCH_GAUSS: {
@@ -1001,8 +1047,28 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
   const long long xs_b = (long long)(c->cfg.max_K + 1) * D, ms_b = (long long)(c->cfg.max_K > 0 ? c->cfg.max_K : 1) * D;
   int r;
   const bool cluster_draft = K > 0 && use_cluster_drafter(c, B);
-  if (cluster_draft && (r = launch_cluster_forward(c, TSDP_DRAFT, 0, B, K, s))) return r;
+  const bool cluster_verify = use_cluster_verifier(c, B, K);
   const bool frozen_draft = c->net[TSDP_DRAFT].cfg.arch == TSDP_ARCH_FROZEN;
+  // Plan of the round: the layer-by-layer forwards then run on the live candidates only.  Not needed when both sides
+  // run in the cluster kernels (small batches), which skip finished slots themselves.
+  const bool layered_draft = K > 0 && !cluster_draft && (!frozen_draft || !use_cluster_verifier(c, B, 0));
+  const bool compact = c->compact && B <= PLAN_MAX_B && (layered_draft || !cluster_verify);
+  if (compact) {
+    prof_begin(c, s, 4, 0.0);
+    TSDP_LAUNCH(c, (round_plan_kernel), 1, PLAN_THREADS, 0, s, c->t, B, K, c->sched, TSDP_MAX_T + 1, c->round_idx,
+                c->sched_on ? c->envp : nullptr, c->item, c->cfg.T, c->plan_live_n, c->plan_list, c->plan_slot_start,
+                c->plan_order, c->plan_dn, c->stats);
+    prof_end(c, s);
+    c->launches_per_round_tmp++;
+    CU_TRY(c, cudaGetLastError());
+    if (c->prof_on) {      // plain launches, no capture: the counts can be read back for the flop accounting
+      CU_TRY(c, cudaStreamSynchronize(s));
+      CU_TRY(c, cudaMemcpy(&c->prof_plan_live, c->plan_live_n, sizeof(int), cudaMemcpyDeviceToHost));
+      CU_TRY(c, cudaMemcpy(c->prof_plan_dn, c->plan_dn, sizeof(int) * (TSDP_MAX_K + 2), cudaMemcpyDeviceToHost));
+    }
+  }
+  const bool counts_known = compact && c->prof_on;
+  if (cluster_draft && (r = launch_cluster_forward(c, TSDP_DRAFT, 0, B, K, s))) return r;
   const float* eps_hat = c->eps_d;        // where the draft step finds eps^ of slot b: eps_hat + b * eps_hat_b
   long long eps_hat_b = D;
   if (frozen_draft && K > 0) {
@@ -1011,24 +1077,31 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
       if ((r = launch_cluster_forward(c, TSDP_BASE, 1, B, 0, s))) return r;
       eps_hat = c->eps; eps_hat_b = xs_b;
     } else {
-      CandMap c0{c->xt, xs_b, c->eps_d, (long long)D, c->t, 1, 0, c->item};
-      if ((r = forward(c, c->net[TSDP_BASE], c0, B, s))) return r;
+      CandMap c0{c->xt, xs_b, c->eps_d, (long long)D, c->t, 1, 0, c->item, compact ? c->plan_order : nullptr,
+                 compact ? c->plan_dn + 1 : nullptr};      // the slots that draft at all
+      c->prof_live_count = counts_known ? c->prof_plan_dn[1] : -1;
+      r = forward(c, c->net[TSDP_BASE], c0, B, s);
+      c->prof_live_count = -1;
+      if (r) return r;
     }
   }
   // transformer drafter, layer by layer: its head, the draft step and the next step's embedding are one kernel
   const bool fused_tail = c->net[TSDP_DRAFT].cfg.arch == TSDP_ARCH_XFMR && c->cfg.A <= 32;
   for (int k = 1; k <= K && !cluster_draft; ++k) {
-    CandMap cm{c->xt + (long long)(k - 1) * D, xs_b, c->eps_d, (long long)D, c->t, 1, k - 1, c->item};
+    CandMap cm{c->xt + (long long)(k - 1) * D, xs_b, c->eps_d, (long long)D, c->t, 1, k - 1, c->item,
+               compact ? c->plan_order : nullptr, compact ? c->plan_dn + k : nullptr};     // the slots still drafting at step k
     c->prof_gemm_cat = 6;
     c->xf_skip_embed = fused_tail && k > 1;
     c->xf_skip_head = fused_tail;
+    c->prof_live_count = counts_known ? c->prof_plan_dn[k] : -1;
     r = frozen_draft ? TSDP_OK : forward(c, c->net[TSDP_DRAFT], cm, B, s);
+    c->prof_live_count = -1;
     c->prof_gemm_cat = 0;
     c->xf_skip_embed = c->xf_skip_head = false;
     if (r) return r;
     if (fused_tail) {
-      r = c->cfg.precision == 0 ? draft_tail_launch<float>(c, c->net[TSDP_DRAFT], B, k, K, k < K, s)
-                                : draft_tail_launch<__nv_bfloat16>(c, c->net[TSDP_DRAFT], B, k, K, k < K, s);
+      r = c->cfg.precision == 0 ? draft_tail_launch<float>(c, c->net[TSDP_DRAFT], B, k, K, k < K, s, cm.list, cm.n_live)
+                                : draft_tail_launch<__nv_bfloat16>(c, c->net[TSDP_DRAFT], B, k, K, k < K, s, cm.list, cm.n_live);
       if (r) return r;
       continue;
     }
@@ -1039,10 +1112,16 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
     c->launches_per_round_tmp++;
     CU_TRY(c, cudaGetLastError());
   }
-  CandMap cv{c->xt, xs_b, c->eps, xs_b, c->t, K + 1, 0, c->item};
-  if (use_cluster_verifier(c, B, K)) {
+  CandMap cv{c->xt, xs_b, c->eps, xs_b, c->t, K + 1, 0, c->item, compact ? c->plan_list : nullptr,
+             compact ? c->plan_live_n : nullptr};
+  if (cluster_verify) {
     if ((r = launch_cluster_forward(c, TSDP_BASE, 1, B, K, s))) return r;
-  } else if ((r = forward(c, c->net[TSDP_BASE], cv, B * (K + 1), s))) return r;
+  } else {
+    c->prof_live_count = counts_known ? c->prof_plan_live : -1;
+    r = forward(c, c->net[TSDP_BASE], cv, B * (K + 1), s, c->plan_slot_start);
+    c->prof_live_count = -1;
+    if (r) return r;
+  }
   int warps = K < 1 ? 1 : K;
   if (warps < 4) warps = 4;
   if (warps > 16) warps = 16;
@@ -1059,6 +1138,7 @@ int enqueue_round(tsdp_ctx* c, int B, int K, cudaStream_t s, bool dbg) {
 }
 
 int run_round(tsdp_ctx* c, int B, int K, cudaStream_t s) {
+  c->cand_static += (uint64_t)B * (K + 1);
   if (!c->cfg.use_graph || c->prof_on) {
     c->launches_per_round_tmp = 0;
     int r = enqueue_round(c, B, K, s, false);
@@ -1170,6 +1250,7 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   c->D = cfg->H * cfg->A;
   c->pdl = getenv("TSDP_NO_PDL") == nullptr;
   c->async_bcast = getenv("TSDP_NO_ASYNC_BCAST") == nullptr;
+  c->compact = getenv("TSDP_NO_COMPACT") == nullptr;
   if (const char* fb = getenv("TSDP_GEMM_BN")) {      // tuning aid: one tile width for every GEMM it divides
     const int v = atoi(fb);
     if (v == 32 || v == 64 || v == 128 || v == 256) c->force_bn = v;
@@ -1240,6 +1321,11 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   st |= dev_alloc(c, c->allocs, &c->sched_dbg, B * 8);
   st |= dev_alloc(c, c->allocs, &c->item_counts, (size_t)B * 4);
   st |= dev_alloc(c, c->allocs, &c->reward, B);
+  st |= dev_alloc(c, c->allocs, &c->plan_live_n, 1);
+  st |= dev_alloc(c, c->allocs, &c->plan_list, B * K1);
+  st |= dev_alloc(c, c->allocs, &c->plan_slot_start, B + 1);
+  st |= dev_alloc(c, c->allocs, &c->plan_order, B);
+  st |= dev_alloc(c, c->allocs, &c->plan_dn, TSDP_MAX_K + 2);
   st |= dev_alloc(c, c->allocs, &c->distill_theta, 2);
   st |= dev_alloc(c, c->allocs, &c->distill_terms, 5 * B);
   st |= dev_alloc(c, c->allocs, &c->distill_res, 8);
@@ -2002,6 +2088,7 @@ int tsdp_round(tsdp_ctx* c, const float* d_obs, int B, int K, const tsdp_accept_
   if ((r = prepare_obs(c, c->net[TSDP_DRAFT], B, s))) return r;
   if ((r = enqueue_round(c, B, K, s, true))) return r;
   c->launches += c->launches_per_round_tmp;
+  c->cand_static += (uint64_t)B * (K + 1);
   c->rounds++;
   // candidates and drafter means are still intact except slot 0, which now holds the new latent
   if (d_xtilde) {
@@ -2198,6 +2285,8 @@ int tsdp_stats(tsdp_ctx* c, tsdp_stats_t* out) {
   out->bonus_steps = ds.bonus_steps;
   out->steps_advanced = ds.steps_advanced;
   out->draft_rounds = ds.draft_rounds;
+  out->cand_dense = c->cand_static;
+  out->cand_computed = ds.cand_computed > 0 || c->compact ? ds.cand_computed : c->cand_static;
   out->nfe = (double)ds.env_rounds + (double)c->cfg.draft_nfe * (double)ds.draft_evals;
   if (c->cfg.draft.arch == TSDP_ARCH_FROZEN) out->nfe = (double)ds.env_rounds + (double)ds.draft_rounds;
   out->call_ms_samples = c->lat_n;
@@ -2223,6 +2312,7 @@ int tsdp_reset_stats(tsdp_ctx* c) {
   CU_TRY(c, cudaMemset(c->stats, 0, sizeof(DevStats)));
   c->rounds = 0;
   c->launches = 0;
+  c->cand_static = 0;
   c->lat_pos = c->lat_n = 0;
   return TSDP_OK;
 }

@@ -32,7 +32,9 @@ __global__ void unet_embed_kernel(CandMap cm, const float* __restrict__ W_in, co
   pdl_wait();
   const int row = blockIdx.x;                      // n * H + l
   const int n = row / H, l = row % H;
-  const int b = n / cm.C, c = n % cm.C;
+  if (n >= cand_count(cm, gridDim.x / H)) return;
+  int b, c;
+  cand_decode(cm, n, b, c);
   const float* x = cm.xin + b * cm.x_stride_b + (long long)c * H * A + (long long)l * A;
   T* o = X + ((size_t)n * (H + 4) + l + 2) * C;
   for (int col = threadIdx.x; col < C; col += blockDim.x) {
@@ -58,6 +60,7 @@ gn_mish_kernel(const float* __restrict__ Y, const float* __restrict__ gam, const
   pdl_wait();
   __shared__ float red[2][8];
   const int n = blockIdx.x / groups, grp = blockIdx.x % groups;
+  if (n >= cand_count(cm, gridDim.x / groups)) return;
   const int Cg = C / groups, Lp = L + 4;
   const int cnt = L * Cg;
   const float* y0 = Y + (size_t)n * Lp * C + (size_t)grp * Cg;
@@ -75,8 +78,9 @@ gn_mish_kernel(const float* __restrict__ Y, const float* __restrict__ gam, const
   const float rstd = rsqrtf(fmaxf(tq / cnt - mean * mean, 0.f) + 1e-5f);
   const float *ft = nullptr, *fo = nullptr;
   if (film_time) {
-    const int b = n / cm.C;
-    int tau = cm.t[b] - cm.koff - (n % cm.C);
+    int b, cc;
+    cand_decode(cm, n, b, cc);
+    int tau = cm.t[b] - cm.koff - cc;
     tau = max(0, min(Tsteps - 1, tau));
     ft = film_time + (size_t)tau * F + foff;
     fo = film_obs + (size_t)item_of(cm.item, b) * F + foff;
@@ -96,9 +100,10 @@ gn_mish_kernel(const float* __restrict__ Y, const float* __restrict__ gam, const
 // 2:1 mean pooling along the sequence: dst[n, l + 2, c] = (src[n, 2l + 2, soff + c] + src[n, 2l + 3, soff + c]) / 2.
 template <typename T>
 __global__ void unet_pool_kernel(const T* __restrict__ src, int src_pitch, int soff, T* __restrict__ dst, int n_cand,
-                                 int L_dst, int C) {
+                                 int L_dst, int C, LiveRows lv) {
   pdl_trigger();
   pdl_wait();
+  n_cand = live_rows(lv, n_cand);
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (long long)n_cand * L_dst * C) return;
   const int c = (int)(idx % C), l = (int)((idx / C) % L_dst), n = (int)(idx / ((long long)C * L_dst));
@@ -109,9 +114,10 @@ __global__ void unet_pool_kernel(const T* __restrict__ src, int src_pitch, int s
 // 2x repetition along the sequence into channels [0, C) of a wider tensor: dst[n, l + 2, c] = src[n, l/2 + 2, c].
 template <typename T>
 __global__ void unet_upsample_kernel(const T* __restrict__ src, T* __restrict__ dst, int dst_pitch, int n_cand, int L_dst,
-                                     int C) {
+                                     int C, LiveRows lv) {
   pdl_trigger();
   pdl_wait();
+  n_cand = live_rows(lv, n_cand);
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (long long)n_cand * L_dst * C) return;
   const int c = (int)(idx % C), l = (int)((idx / C) % L_dst), n = (int)(idx / ((long long)C * L_dst));
@@ -128,7 +134,9 @@ __global__ void unet_head_kernel(const T* __restrict__ X, const float* __restric
   const int lane = threadIdx.x & 31;
   if (row >= M) return;
   const int n = row / H, l = row % H;
-  const int b = n / cm.C, c = n % cm.C;
+  if (n >= cand_count(cm, M / H)) return;
+  int b, c;
+  cand_decode(cm, n, b, c);
   const T* x = X + ((size_t)n * (H + 4) + l + 2) * C;
   float* o = cm.eout + b * cm.e_stride_b + (long long)c * H * A + (long long)l * A;
   for (int a = 0; a < A; ++a) {

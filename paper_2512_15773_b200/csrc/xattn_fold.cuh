@@ -187,9 +187,11 @@ xattn_fold_kernel(float* __restrict__ x, const __nv_bfloat16* __restrict__ delta
   float* sS = reinterpret_cast<float*>(sU + (size_t)(NKH / 2) * LDU);      // [4][16][XF_MAXN]
   __nv_bfloat16* sP = reinterpret_cast<__nv_bfloat16*>(sS + 4 * 16 * XF_MAXN);
   const int n = blockIdx.x;
+  if (n >= cand_count(cm, gridDim.x)) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, tg = lane & 3;
-  const int b = n / cm.C, cnd = n % cm.C;
+  int b, cnd;
+  cand_decode(cm, n, b, cnd);
   int tau = cm.t[b] - cm.koff - cnd;
   tau = max(0, min(Tsteps - 1, tau));
   const int item = item_of(cm.item, b);

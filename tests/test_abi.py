@@ -30,7 +30,7 @@ def test_struct_layouts_match_the_header():
     assert ctypes.sizeof(binding.NetT) == 20
     assert ctypes.sizeof(binding.ConfigT) == 2 * 20 + 16 * 4
     assert ctypes.sizeof(binding.AcceptT) == 16
-    assert ctypes.sizeof(binding.StatsT) == 11 * 8 + 8 + 3 * 8 * 1024 + 3 * 8
+    assert ctypes.sizeof(binding.StatsT) == 11 * 8 + 8 + 3 * 8 * 1024 + 5 * 8
 
 
 def test_weight_counts_match_the_packer(lib):

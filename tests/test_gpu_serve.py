@@ -85,3 +85,53 @@ def test_serve_with_obs_beyond_max_b():
     small.serve(dobs, N, slots, K, hp.accept_t(), 5, out)
     assert torch.equal(out, ref)
     big.close(); small.close()
+
+
+@pytest.mark.parametrize("arch", ["xfmr_bf16", "xfmr_fp32", "dit_bf16", "unet_bf16", "mlp_fp32"])
+def test_compacted_rounds_give_the_same_bits_as_dense_rounds(arch, monkeypatch):
+    """Each round lists the candidates that are still needed and the layer-by-layer forwards run on that list only.
+    Rows are computed independently of one another, so the chunk must come out bit for bit as from the dense
+    B x (K+1) layout (TSDP_NO_COMPACT), with the same counters, while fewer candidates are evaluated -- exactly as many
+    as the acceptance kernel counts as useful base evaluations."""
+    if arch == "xfmr_bf16":
+        wl = hp.small_xfmr_workload(1, d=256, heads=4, layers=2, dd=128, dlayers=2, H=16, A=7, To=2, Do=16, gamma=0.05)
+    elif arch == "xfmr_fp32":
+        wl = hp.small_xfmr_workload(0, d=128, heads=4, layers=1, dd=128, dlayers=1, H=16, A=7, To=2, Do=16, gamma=0.05)
+    elif arch == "dit_bf16":
+        wl = dict(H=10, A=4, To=16, Do=8, T=100, precision=1, gamma=0.05,
+                  base=dict(arch="dit", layers=2, d=128, heads=4), draft=dict(arch="dit", layers=1, d=128, heads=2))
+    elif arch == "unet_bf16":
+        wl = dict(H=16, A=10, To=2, Do=24, T=100, precision=1, gamma=0.05,
+                  base=dict(arch="unet", layers=2, d=128, heads=8, temb=32), draft=dict(arch="xfmr", layers=1, d=128, heads=4))
+    else:
+        wl = dict(inputs.WORKLOADS["toy_mlp"])
+    B, K, seed = 37, 6, 3
+    Ks, Ss = inputs.markov_schedule(1, 60)
+    Ks = [min(k, K) for k in Ks]
+    res = []
+    for dense in (True, False):
+        if dense:
+            monkeypatch.setenv("TSDP_NO_COMPACT", "1")
+        else:
+            monkeypatch.delenv("TSDP_NO_COMPACT")
+        smp, *_ = hp.setup(wl, max_B=B, max_K=K, drafter=1, verifier=1)
+        smp.set_schedule(Ks, [hp.accept_t(sigma_scale=s, bonus=(i % 3 != 0)) for i, s in enumerate(Ss)])
+        obs = torch.tensor(inputs.make_obs(11, B, wl["To"], wl["Do"]), dtype=torch.float32, device="cuda")
+        out = torch.zeros(B, wl["H"], wl["A"], device="cuda")
+        smp.reset_stats()
+        smp.sample_chunk(obs, B, K, hp.accept_t(), seed, out)
+        st = smp.stats()
+        # continuous batching on top: slots refill while others are still mid-chunk
+        N = 3 * B + 5
+        obs2 = torch.tensor(inputs.make_obs(12, N, wl["To"], wl["Do"]), dtype=torch.float32, device="cuda")
+        out2 = torch.zeros(N, wl["H"], wl["A"], device="cuda")
+        smp.serve(obs2, N, B, K, hp.accept_t(), seed + 1, out2)
+        res.append((out.clone(), out2.clone(), st))
+        smp.close()
+    (o_d, o2_d, st_d), (o_c, o2_c, st_c) = res
+    assert torch.equal(o_d, o_c) and torch.equal(o2_d, o2_c)
+    for k in ("env_rounds", "base_evals", "draft_evals", "drafts_accepted", "rejections", "bonus_steps", "steps_advanced", "rounds"):
+        assert st_d[k] == st_c[k], k
+    assert np.array_equal(st_d["hist_accepted"], st_c["hist_accepted"])
+    assert st_d["cand_computed"] == st_d["cand_dense"] == st_c["cand_dense"]
+    assert st_c["cand_computed"] == st_c["base_evals"] < st_c["cand_dense"]

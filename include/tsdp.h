@@ -247,6 +247,14 @@ int tsdp_denoise(tsdp_ctx* ctx, int which, const float* d_x, const int* h_tau, c
 int tsdp_gemm(tsdp_ctx* ctx, const void* d_A, const void* d_W, const float* d_bias, int M, int N, int K,
               int epi, void* d_out, void* cuda_stream);
 
+/* Exercise the time-out path of the tensor-core GEMM without hanging anything (test interface, precision 1).  Every
+ * wait inside the kernel is bounded; normally the bound (about a second) is never reached.  After this call the NEXT
+ * tsdp_gemm launch runs with the bound set to `wait_cycles` SM clock cycles (1e3 .. 2e9) and with one operand tile
+ * withheld from CTA 0: that CTA's waits run out, it records TSDP_ERR_TIMEOUT, drains its copies, frees its tensor
+ * memory and returns, while the other CTAs finish normally.  tsdp_gemm then returns TSDP_ERR_TIMEOUT (its output is
+ * incomplete), the status word is cleared, and the context stays usable.  One-shot.  Errors: ARG. */
+int tsdp_debug_arm_gemm_timeout(tsdp_ctx* ctx, long long wait_cycles);
+
 /* The same GEMM launched `reps` times back to back between one pair of CUDA events on `cuda_stream`
  * (after one untimed launch); *h_ms (HOST) receives the mean device time of one launch in milliseconds.
  * With EPI 2 the output accumulates over the launches.  Measurement interface; synchronous. */

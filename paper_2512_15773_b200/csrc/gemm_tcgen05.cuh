@@ -64,20 +64,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait: false when the barrier did not flip within GEMM_WAIT_CYCLES.
-__device__ __forceinline__ bool mbar_wait_thread(uint32_t bar, uint32_t parity) {
+// Bounded wait: false when the barrier did not flip within `limit` SM clock cycles.
+__device__ __forceinline__ bool mbar_wait_thread(uint32_t bar, uint32_t parity, long long limit = GEMM_WAIT_CYCLES) {
   for (int i = 0; i < 128; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (clock64() - t0 > GEMM_WAIT_CYCLES) return false;
+    if (clock64() - t0 > limit) return false;
   }
 }
 // The same for a whole converged warp; the outcome is made uniform so that no lane leaves a
 // .sync.aligned section alone.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity) {
-  return __all_sync(0xffffffffu, mbar_wait_thread(bar, parity)) != 0;
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, long long limit = GEMM_WAIT_CYCLES) {
+  return __all_sync(0xffffffffu, mbar_wait_thread(bar, parity, limit)) != 0;
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
@@ -210,6 +210,11 @@ struct GemmArgs {
   // (live.n null: M).  The tensor maps keep their full extent; tiles beyond the live rows are simply not visited.
   LiveRows live;
   const int* list;      // EPI_GATE with a compacted list: candidate n of a row is (list[n] >> 6, list[n] & 63)
+  long long wait_cycles;  // limit of every mbarrier wait in SM clock cycles (0: GEMM_WAIT_CYCLES, about a second)
+  // Test of the time-out path (host-armed, one launch): CTA 0's producer leaves out the operand loads of its very
+  // first pipeline stage, so the waits that depend on that stage run out, the CTA reports TSDP_ERR_TIMEOUT through
+  // `status`, drains and returns; every other CTA finishes its tiles as usual.
+  int withhold_first_stage;
 };
 
 __device__ __forceinline__ const float* gate_row(const GemmArgs& g, int row) {
@@ -302,6 +307,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_ptr;
   bool ok = true;
+  const long long wlim = g.wait_cycles > 0 ? g.wait_cycles : GEMM_WAIT_CYCLES;
   pdl_wait();      // operands, bias, the output and the live-row count belong to earlier kernels of the stream
   const int M = live_rows(g.live, g.M);
   const int tiles_m = (M + GEMM_BM - 1) / GEMM_BM;
@@ -313,13 +319,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         const int tm = tile / tiles_n, tn = tile % tiles_n;
         for (int kb = 0; kb < kblocks; ++kb) {
-          if (!ptx::mbar_wait_thread(empty_bar(stage), phase ^ 1u)) { ok = false; break; }
-          ptx::mbar_expect_tx(full_bar(stage), STAGE_BYTES);
-          const uint32_t sa = base + stage * STAGE_BYTES;
-          const int kcol = kb * GEMM_BK;
-          const int ax = g.conv_c ? kcol % g.conv_c : kcol, ay = tm * GEMM_BM + (g.conv_c ? kcol / g.conv_c : 0);
-          ptx::tma_load_2d(sa, &tmA, ax, ay, full_bar(stage));
-          ptx::tma_load_2d(sa + A_BYTES, &tmB, kb * GEMM_BK, tn * BN, full_bar(stage));
+          if (!ptx::mbar_wait_thread(empty_bar(stage), phase ^ 1u, wlim)) { ok = false; break; }
+          if (!(g.withhold_first_stage && blockIdx.x == 0 && tile == 0 && kb == 0)) {
+            ptx::mbar_expect_tx(full_bar(stage), STAGE_BYTES);
+            const uint32_t sa = base + stage * STAGE_BYTES;
+            const int kcol = kb * GEMM_BK;
+            const int ax = g.conv_c ? kcol % g.conv_c : kcol, ay = tm * GEMM_BM + (g.conv_c ? kcol / g.conv_c : 0);
+            ptx::tma_load_2d(sa, &tmA, ax, ay, full_bar(stage));
+            ptx::tma_load_2d(sa + A_BYTES, &tmB, kb * GEMM_BK, tn * BN, full_bar(stage));
+          }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -329,11 +337,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       int stage = 0; uint32_t phase = 0; int it = 0;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
         const int as = it & 1; const uint32_t aphase = (it >> 1) & 1;
-        if (!ptx::mbar_wait_thread(tempty_bar(as), aphase ^ 1u)) { ok = false; break; }
+        if (!ptx::mbar_wait_thread(tempty_bar(as), aphase ^ 1u, wlim)) { ok = false; break; }
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(as * BN);
         for (int kb = 0; kb < kblocks; ++kb) {
-          if (!ptx::mbar_wait_thread(full_bar(stage), phase)) { ok = false; break; }
+          if (!ptx::mbar_wait_thread(full_bar(stage), phase, wlim)) { ok = false; break; }
           ptx::tc_fence_after();
           const uint32_t sa = base + stage * STAGE_BYTES;
           const uint64_t da = umma_desc_sw128(sa), db = umma_desc_sw128(sa + A_BYTES);
@@ -368,7 +376,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const int tm = tile / tiles_n, tn = tile % tiles_n;
         const int as = it & 1; const uint32_t aphase = (it >> 1) & 1;
         // all four warps of this half agree on the outcome, so none is left alone at a named barrier
-        ok = ptx::named_bar_and(bar_id, 128, ptx::mbar_wait_warp(tfull_bar(as), aphase));
+        ok = ptx::named_bar_and(bar_id, 128, ptx::mbar_wait_warp(tfull_bar(as), aphase, wlim));
         if (!ok) break;
         ptx::tc_fence_after();
         const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * BN + half * COLS);
@@ -443,7 +451,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
         const int tm = tile / tiles_n, tn = tile % tiles_n;
         const int as = it & 1; const uint32_t aphase = (it >> 1) & 1;
-        if (!ptx::mbar_wait_warp(tfull_bar(as), aphase)) { ok = false; break; }
+        if (!ptx::mbar_wait_warp(tfull_bar(as), aphase, wlim)) { ok = false; break; }
         ptx::tc_fence_after();
         const int row = tm * GEMM_BM + quad * 32 + lane;
         const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * BN + half * COLS);

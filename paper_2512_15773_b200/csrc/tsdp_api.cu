@@ -149,6 +149,8 @@ struct tsdp_ctx {
   // while profiling: host copies of the plan's counts, so that a GEMM's flops are those of the rows it really processed
   int prof_plan_live = -1, prof_plan_dn[TSDP_MAX_K + 2] = {};
   int prof_live_count = -1;                   // live candidates of the forward being enqueued (-1: unknown, use the dense count)
+  bool dbg_armed = false, dbg_in_test_gemm = false;   // tsdp_debug_arm_gemm_timeout
+  long long dbg_wait_cycles = 0;
   uint64_t cand_static = 0;                   // candidates the dense layout would have evaluated since the last reset
   // optional per-kernel-family timing with CUDA events (plain launches, no graph)
   bool prof_on = false;
@@ -387,7 +389,12 @@ int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, in
          int ldo, cudaStream_t s, const GateSpec* gs = nullptr, int conv_c = 0) {
   if (M <= 0) return TSDP_OK;
   GemmArgs g{M, N, K, bias, out, ldo, c->status, nullptr, 0, nullptr, 1, 0, 1, 1, conv_c > 0 ? conv_c : K, conv_c,
-             LiveRows{nullptr, 0, 0}, nullptr};
+             LiveRows{nullptr, 0, 0}, nullptr, 0, 0};
+  if (c->dbg_armed && c->dbg_in_test_gemm && c->cfg.precision == 1) {      // one launch: see tsdp_debug_arm_gemm_timeout
+    g.wait_cycles = c->dbg_wait_cycles;
+    g.withhold_first_stage = 1;
+    c->dbg_armed = false;
+  }
   if (epi == EPI_GATE) {
     if (!gs) return TSDP_ERR_ARG;
     g.gate = gs->gate; g.gate_ld = gs->gate_ld; g.t = gs->cm->t; g.C = gs->cm->C; g.koff = gs->cm->koff; g.H = gs->H;
@@ -447,7 +454,7 @@ int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, in
 // fp32 CUDA-core GEMM whatever the precision mode: the timestep-conditioning tables built at weight load.
 int gemm_f32(tsdp_ctx* c, const float* A, const float* W, const float* bias, int M, int N, int K, int epi, float* out,
              cudaStream_t s) {
-  GemmArgs g{M, N, K, bias, out, N, c->status, nullptr, 0, nullptr, 1, 0, 1, 1, K, 0, LiveRows{nullptr, 0, 0}, nullptr};
+  GemmArgs g{M, N, K, bias, out, N, c->status, nullptr, 0, nullptr, 1, 0, 1, 1, K, 0, LiveRows{nullptr, 0, 0}, nullptr, 0, 0};
   dim3 grid((N + 63) / 64, (M + 63) / 64);
   if (epi == EPI_MISH) TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_MISH>), grid, 256, 0, s, A, W, g);
   else if (epi == EPI_SILU) TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_SILU>), grid, 256, 0, s, A, W, g);
@@ -2229,13 +2236,22 @@ int tsdp_gemm(tsdp_ctx* c, const void* d_A, const void* d_W, const float* d_bias
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   if (c->cfg.precision == 0 && epi == EPI_STORE) epi = EPI_F32;
   c->launches_per_round_tmp = 0;
+  c->dbg_in_test_gemm = true;
   int r = gemm(c, d_A, d_W, d_bias, M, N, K, epi, d_out, N, s);
+  c->dbg_in_test_gemm = false;
   c->launches += c->launches_per_round_tmp;
   if (r) return r;
   CU_TRY(c, cudaStreamSynchronize(s));
   // test interface: operands are caller-owned and may be freed, so their tensor maps are not kept
   c->maps.clear();
   return check_status(c);
+}
+
+int tsdp_debug_arm_gemm_timeout(tsdp_ctx* c, long long wait_cycles) {
+  if (!c || wait_cycles < 1000 || wait_cycles > 2000000000ll || c->cfg.precision != 1) return TSDP_ERR_ARG;
+  c->dbg_armed = true;
+  c->dbg_wait_cycles = wait_cycles;
+  return TSDP_OK;
 }
 
 int tsdp_gemm_timed(tsdp_ctx* c, const void* d_A, const void* d_W, const float* d_bias, int M, int N, int K, int epi,

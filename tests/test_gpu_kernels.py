@@ -177,3 +177,31 @@ def test_unet_denoiser(precision, tol, shape):
     ref = np.stack([base(x[n].astype(np.float64), int(tau[n]), obs[n]) for n in range(N)])
     assert hp.max_rel(out2.cpu().numpy(), ref) < tol
     smp.close()
+
+
+def test_gemm_bounded_wait_runs_out_and_the_context_recovers():
+    """Failure detection without a fault: one CTA of the tensor-core GEMM is starved of an operand tile (a barrier
+    that nothing completes) with the wait limit lowered to about a millisecond.  The kernel must return by giving up
+    its waits, the call must report TSDP_ERR_TIMEOUT, the status word must be cleared, and the next ordinary calls on
+    the same context must pass their parity checks."""
+    import time
+    wl = hp.small_xfmr_workload(1)
+    smp, *_ = hp.setup(wl, max_B=1, max_K=1)
+    rng = np.random.default_rng(5)
+    _gemm_case(smp, 4000, 512, 512, 0, rng)                       # healthy before
+    M, N, K = 4000, 512, 512
+    dA = torch.zeros(M, K, dtype=torch.bfloat16, device="cuda"); dW = torch.zeros(N, K, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(M, N, dtype=torch.bfloat16, device="cuda")
+    smp.arm_gemm_timeout(2_000_000)                               # about 1 ms of SM clock
+    t0 = time.perf_counter()
+    with pytest.raises(binding.TsdpError) as e:
+        smp.gemm(dA, dW, None, M, N, K, 0, out)
+    assert e.value.status == 5                                    # TSDP_ERR_TIMEOUT
+    assert time.perf_counter() - t0 < 5.0                         # gave up after milliseconds, not after the default second per wait
+    # one-shot and cleared: the same context works again, every epilogue
+    for epi in (0, 1, 2, 3):
+        _gemm_case(smp, 4000, 512, 512, epi, rng)
+    _gemm_case(smp, 129, 64, 512, 2, rng)
+    with pytest.raises(binding.TsdpError):
+        smp.arm_gemm_timeout(10)                                  # below the accepted range
+    smp.close()

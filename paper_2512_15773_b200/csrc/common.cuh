@@ -98,6 +98,118 @@ __device__ __forceinline__ float warp_max(float v) {
   return v;
 }
 
+// ---- warp-level tensor-core helpers (mma.sync m16n8k16 bf16, ldmatrix) shared by the attention kernels
+__device__ __forceinline__ void mma_bf16_16816(float c[4], const uint32_t a[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 h2 = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&h2);
+}
+
+// Four 8x8 b16 matrices from shared memory: lanes 8i..8i+7 give the 16-byte row addresses of matrix i.
+// Plain: lane l receives M[l/4][2(l%4) .. +1] -- the B fragment of a [n][k] (K-major) tile.
+// Transposed: lane l receives M[2(l%4) .. +1][l/4] -- the B fragment of a [k][n] tile (values V of attention).
+__device__ __forceinline__ void ldmatrix_x4(uint32_t r[4], const void* smem_row) {
+  const uint32_t a = (uint32_t)__cvta_generic_to_shared(smem_row);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t r[4], const void* smem_row) {
+  const uint32_t a = (uint32_t)__cvta_generic_to_shared(smem_row);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+
+// Attention of one (candidate, head) with at most 16 tokens by one warp, operands already in shared memory:
+// sQ, sK, sV are [16][DH + 8] bf16 tiles (rows past H zero).  S = Q K^T and O = P V on mma.sync m16n8k16 (Q with
+// 4-byte loads, K through ldmatrix, V through ldmatrix.trans), softmax in the accumulator registers.  The
+// normalised output tile overwrites sQ.  Used by self_attn_tile_kernel and by the fused QKV epilogue of the
+// tensor-core GEMM, which therefore produce the same bits.
+template <int DH>
+__device__ __forceinline__ void attn16_from_smem(__nv_bfloat16* sQ, const __nv_bfloat16* sK, const __nv_bfloat16* sV, int H,
+                                                 int causal, int lane) {
+  constexpr int KS = DH / 16, NO = DH / 8, P = DH + 8;
+  const int g = lane >> 2, tg = lane & 3;
+  uint32_t qa[KS][4];
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks) {
+    const __nv_bfloat16* q0 = sQ + g * P + ks * 16 + 2 * tg;
+    qa[ks][0] = *reinterpret_cast<const uint32_t*>(q0);
+    qa[ks][1] = *reinterpret_cast<const uint32_t*>(q0 + 8 * P);
+    qa[ks][2] = *reinterpret_cast<const uint32_t*>(q0 + 8);
+    qa[ks][3] = *reinterpret_cast<const uint32_t*>(q0 + 8 * P + 8);
+  }
+  const int nkt = causal ? 2 : (H + 7) >> 3;
+  float s[2][4];
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+    s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+    if (nt < nkt) {
+#pragma unroll
+      for (int ks = 0; ks < KS; ks += 2) {
+        uint32_t b[4];
+        ldmatrix_x4(b, sK + (nt * 8 + (lane & 7)) * P + ks * 16 + 8 * (lane >> 3));
+        mma_bf16_16816(s[nt], qa[ks], b[0], b[1]);
+        mma_bf16_16816(s[nt], qa[ks + 1], b[2], b[3]);
+      }
+    }
+  }
+  const float scale = rsqrtf((float)DH);
+  const int r0 = g, r1 = g + 8;
+  float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+    if (nt < nkt) {
+      const int col = nt * 8 + 2 * tg;
+      const int lim0 = causal ? r0 : H, lim1 = causal ? r1 : H;
+      s[nt][0] = (col <= lim0 && col < H) ? s[nt][0] * scale : -INFINITY;
+      s[nt][1] = (col + 1 <= lim0 && col + 1 < H) ? s[nt][1] * scale : -INFINITY;
+      s[nt][2] = (col <= lim1 && col < H) ? s[nt][2] * scale : -INFINITY;
+      s[nt][3] = (col + 1 <= lim1 && col + 1 < H) ? s[nt][3] * scale : -INFINITY;
+      m0 = fmaxf(m0, fmaxf(s[nt][0], s[nt][1]));
+      m1 = fmaxf(m1, fmaxf(s[nt][2], s[nt][3]));
+    }
+  }
+  m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 1)); m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 2));
+  m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 1)); m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 2));
+  // rows beyond H have no visible key: keep the arithmetic finite, their output is never stored
+  if (m0 == -INFINITY) m0 = 0.f;
+  if (m1 == -INFINITY) m1 = 0.f;
+  float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+    if (nt < nkt) {
+      s[nt][0] = __expf(s[nt][0] - m0); s[nt][1] = __expf(s[nt][1] - m0);
+      s[nt][2] = __expf(s[nt][2] - m1); s[nt][3] = __expf(s[nt][3] - m1);
+      l0 += s[nt][0] + s[nt][1]; l1 += s[nt][2] + s[nt][3];
+    }
+  }
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+  l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+  const float inv0 = l0 > 0.f ? 1.0f / l0 : 0.f, inv1 = l1 > 0.f ? 1.0f / l1 : 0.f;
+  uint32_t pa[4];
+  pa[0] = pack_bf16(s[0][0], s[0][1]); pa[1] = pack_bf16(s[0][2], s[0][3]);
+  pa[2] = pack_bf16(s[1][0], s[1][1]); pa[3] = pack_bf16(s[1][2], s[1][3]);
+  __syncwarp();                                   // every lane has its Q fragments: the Q rows become the output tile
+#pragma unroll
+  for (int no = 0; no < NO; no += 2) {
+    float o0[4] = {0.f, 0.f, 0.f, 0.f}, o1[4] = {0.f, 0.f, 0.f, 0.f};
+    uint32_t b[4];
+    ldmatrix_x4_trans(b, sV + ((lane & 7) + 8 * ((lane >> 3) & 1)) * P + no * 8 + 8 * (lane >> 4));
+    mma_bf16_16816(o0, pa, b[0], b[1]);
+    mma_bf16_16816(o1, pa, b[2], b[3]);
+    const int col = no * 8 + 2 * tg;
+    *reinterpret_cast<uint32_t*>(sQ + g * P + col) = pack_bf16(o0[0] * inv0, o0[1] * inv0);
+    *reinterpret_cast<uint32_t*>(sQ + (g + 8) * P + col) = pack_bf16(o0[2] * inv1, o0[3] * inv1);
+    *reinterpret_cast<uint32_t*>(sQ + g * P + col + 8) = pack_bf16(o1[0] * inv0, o1[1] * inv0);
+    *reinterpret_cast<uint32_t*>(sQ + (g + 8) * P + col + 8) = pack_bf16(o1[2] * inv1, o1[3] * inv1);
+  }
+}
+
 __device__ __forceinline__ float to_f(float v) { return v; }
 __device__ __forceinline__ float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
 template <typename T> __device__ __forceinline__ T from_f(float v);

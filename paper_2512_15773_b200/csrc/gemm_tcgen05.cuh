@@ -28,7 +28,11 @@ namespace tsdp {
 // EPI_GATE: fp32 out += gate[tau(row), col] * (acc + bias), the gated residual of an adaptive-LayerNorm block.
 // EPI_SILU: fp32 store of SiLU(acc + bias); CUDA-core GEMM only (conditioning tables built at load).
 // EPI_MISH: as EPI_SILU with Mish.
-enum { EPI_STORE = 0, EPI_GELU = 1, EPI_RESID = 2, EPI_F32 = 3, EPI_GATE = 4, EPI_SILU = 5, EPI_MISH = 6 };
+// EPI_ATTN: the QKV projection with the self-attention fused into its epilogue (tensor-core kernel only, BN = 192):
+//           output tile column block tn = head tn's [Q | K | V] (64 columns each, weights stored in that order), a
+//           128-row tile = 8 candidates of 16 tokens; the epilogue runs the 16-token attention of each (candidate,
+//           head) from shared memory and writes only the attention output, bf16 [M, d] at columns [64 tn, +64).
+enum { EPI_STORE = 0, EPI_GELU = 1, EPI_RESID = 2, EPI_F32 = 3, EPI_GATE = 4, EPI_SILU = 5, EPI_MISH = 6, EPI_ATTN = 7 };
 
 constexpr int GEMM_BM = 128;
 constexpr int GEMM_BK = 64;
@@ -36,12 +40,18 @@ constexpr int GEMM_THREADS = 320;
 constexpr int GEMM_EPI_WARPS = 8;
 constexpr long long GEMM_WAIT_CYCLES = 2000000000ll;   // about one second of SM clock
 
-__host__ __device__ constexpr int gemm_stages(int BN) { return BN >= 256 ? 4 : (BN >= 128 ? 6 : 8); }
+__host__ __device__ constexpr int gemm_stages(int BN) { return BN >= 192 ? 4 : (BN >= 128 ? 6 : 8); }
 __host__ __device__ constexpr int gemm_stage_bytes(int BN) { return GEMM_BM * GEMM_BK * 2 + BN * GEMM_BK * 2; }
 constexpr int GEMM_STAGING_BYTES = 2 * 128 * 128;   // one 128-row x 128-byte chunk per column half
-__host__ __device__ constexpr bool gemm_tma_epilogue(int BN) { return BN >= 128; }
+constexpr int GEMM_ATTN_BN = 192;                   // [Q | K | V] of one 64-wide head
+constexpr int GEMM_ATTN_P = 64 + 8;                 // row pitch (elements) of the staged Q / K / V tiles
+constexpr int GEMM_ATTN_STAGING_BYTES = 8 * 3 * 16 * GEMM_ATTN_P * 2;   // 8 candidates x {Q, K, V} x 16 rows
+__host__ __device__ constexpr bool gemm_tma_epilogue(int BN) { return BN >= 128 && BN != GEMM_ATTN_BN; }
+__host__ __device__ constexpr int gemm_epi_smem_bytes(int BN) {
+  return BN == GEMM_ATTN_BN ? GEMM_ATTN_STAGING_BYTES : (gemm_tma_epilogue(BN) ? GEMM_STAGING_BYTES : 0);
+}
 __host__ __device__ constexpr int gemm_smem_bytes(int BN) {
-  return gemm_stages(BN) * gemm_stage_bytes(BN) + (gemm_tma_epilogue(BN) ? GEMM_STAGING_BYTES : 0) + 1024 + 256;
+  return gemm_stages(BN) * gemm_stage_bytes(BN) + gemm_epi_smem_bytes(BN) + 1024 + 256;
 }
 
 namespace ptx {
@@ -215,6 +225,7 @@ struct GemmArgs {
   // first pipeline stage, so the waits that depend on that stage run out, the CTA reports TSDP_ERR_TIMEOUT through
   // `status`, drains and returns; every other CTA finishes its tiles as usual.
   int withhold_first_stage;
+  int causal;           // EPI_ATTN: causal mask of the fused 16-token self-attention
 };
 
 __device__ __forceinline__ const float* gate_row(const GemmArgs& g, int row) {
@@ -270,16 +281,18 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   constexpr int STAGES = gemm_stages(BN);
   constexpr int A_BYTES = GEMM_BM * GEMM_BK * 2;
   constexpr int STAGE_BYTES = gemm_stage_bytes(BN);
-  constexpr uint32_t TMEM_COLS = (2 * BN < 32) ? 32 : 2 * BN;
+  constexpr int ACC = BN == GEMM_ATTN_BN ? 256 : BN;          // column distance of the two accumulator buffers
+  constexpr uint32_t TMEM_COLS = (2 * ACC < 32) ? 32 : 2 * ACC;  // a power of two
   constexpr uint32_t IDESC = umma_idesc_bf16(BN);
-  static_assert(BN == 32 || BN == 64 || BN == 128 || BN == 256, "BN");
+  static_assert(BN == 32 || BN == 64 || BN == 128 || BN == 256 || BN == GEMM_ATTN_BN, "BN");
+  static_assert((EPI == EPI_ATTN) == (BN == GEMM_ATTN_BN), "the fused attention epilogue has its own tile width");
 
   extern __shared__ uint8_t smem_raw[];
   pdl_trigger();
   const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   constexpr bool TMA_EPI = gemm_tma_epilogue(BN);
   const uint32_t staging = base + STAGES * STAGE_BYTES;    // 1024-byte aligned: every stage is a multiple of 1 KB
-  const uint32_t bar0 = staging + (TMA_EPI ? GEMM_STAGING_BYTES : 0);   // full[STAGES], empty[STAGES], tfull[2], tempty[2]
+  const uint32_t bar0 = staging + gemm_epi_smem_bytes(BN);   // full[STAGES], empty[STAGES], tfull[2], tempty[2]
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
   auto tfull_bar = [&](int s) { return bar0 + 8u * (2 * STAGES + s); };
@@ -339,7 +352,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const int as = it & 1; const uint32_t aphase = (it >> 1) & 1;
         if (!ptx::mbar_wait_thread(tempty_bar(as), aphase ^ 1u, wlim)) { ok = false; break; }
         ptx::tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(as * BN);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(as * ACC);
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!ptx::mbar_wait_thread(full_bar(stage), phase, wlim)) { ok = false; break; }
           ptx::tc_fence_after();
@@ -361,7 +374,67 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const int half = ew >> 2;                // which half of the tile's columns
     constexpr int COLS = BN / 2;
     int it = 0;
-    if constexpr (TMA_EPI) {
+    if constexpr (EPI == EPI_ATTN) {
+      // Rows 32 quad .. +31 of the tile are two candidates (16 tokens each); the two warps of a quadrant each bring
+      // half of the 192 columns of those rows from tensor memory to shared memory (bias added, bf16), then each runs
+      // the attention of one of the two candidates.  Only the two warps of a quadrant ever touch its staging area.
+      constexpr int P = GEMM_ATTN_P;
+      __nv_bfloat16* att = reinterpret_cast<__nv_bfloat16*>(smem_raw + (staging - ptx::smem_u32(smem_raw)));
+      const int pair_bar = 1 + quad;
+      const int r_tile = quad * 32 + lane;                    // this lane's row of the tile
+      const int cand_l = r_tile >> 4, r_l = r_tile & 15;      // candidate (0..7) and token of that row
+      const int cand_w = 2 * quad + half;                     // the candidate this warp attends for
+      for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
+        const int tm = tile / tiles_n, tn = tile % tiles_n;
+        const int as = it & 1; const uint32_t aphase = (it >> 1) & 1;
+        // both warps of the quadrant agree on the outcome; the barrier also orders the previous tile's reads of the
+        // staging area before this tile's writes
+        ok = ptx::named_bar_and(pair_bar, 64, ptx::mbar_wait_warp(tfull_bar(as), aphase, wlim));
+        if (!ok) break;
+        ptx::tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * ACC + half * 96);
+#pragma unroll
+        for (int part = 0; part < 3; ++part) {
+          uint32_t v[32];
+          ptx::tmem_ld32(taddr + (uint32_t)(part * 32), v);
+          ptx::tmem_ld_wait();
+          if (part == 2) {                                    // accumulator fully read: hand it back
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(tempty_bar(as));
+          }
+          const int col = half * 96 + part * 32;              // column inside the head's [Q | K | V]
+          float f[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]);
+          if (g.bias) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const float4 bb = __ldg(reinterpret_cast<const float4*>(g.bias + tn * BN + col) + i);
+              f[4 * i] += bb.x; f[4 * i + 1] += bb.y; f[4 * i + 2] += bb.z; f[4 * i + 3] += bb.w;
+            }
+          }
+          __nv_bfloat16* dst = att + ((size_t)(cand_l * 3 + (col >> 6)) * 16 + r_l) * P + (col & 63);
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            *reinterpret_cast<uint4*>(dst + 8 * j) =
+                make_uint4(pack_bf16x2(f[8 * j], f[8 * j + 1]), pack_bf16x2(f[8 * j + 2], f[8 * j + 3]),
+                           pack_bf16x2(f[8 * j + 4], f[8 * j + 5]), pack_bf16x2(f[8 * j + 6], f[8 * j + 7]));
+        }
+        ptx::named_bar_sync(pair_bar, 64);                    // the quadrant's Q, K, V tiles are complete
+        __nv_bfloat16* sQ = att + (size_t)(cand_w * 3) * 16 * P;
+        attn16_from_smem<64>(sQ, sQ + 16 * P, sQ + 32 * P, 16, g.causal, lane);
+        __syncwarp();
+        const int row0 = tm * GEMM_BM + cand_w * 16;
+        __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(g.out) + (size_t)row0 * g.ldo + tn * 64;
+#pragma unroll
+        for (int i = lane; i < 16 * 8; i += 32) {
+          const int r = i >> 3, v8 = i & 7;
+          if (row0 + r < M)
+            *reinterpret_cast<uint4*>(o + (size_t)r * g.ldo + v8 * 8) = *reinterpret_cast<const uint4*>(sQ + r * P + v8 * 8);
+        }
+      }
+    } else if constexpr (TMA_EPI) {
       // Output element size, columns per 128-byte chunk, chunks per half tile.
       constexpr int ESZ = (EPI == EPI_STORE || EPI == EPI_GELU) ? 2 : 4;
       constexpr int CW = 128 / ESZ;
@@ -379,7 +452,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         ok = ptx::named_bar_and(bar_id, 128, ptx::mbar_wait_warp(tfull_bar(as), aphase, wlim));
         if (!ok) break;
         ptx::tc_fence_after();
-        const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * BN + half * COLS);
+        const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * ACC + half * COLS);
 #pragma unroll 1
         for (int ch = 0; ch < NCH; ++ch) {
 #pragma unroll
@@ -454,7 +527,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (!ptx::mbar_wait_warp(tfull_bar(as), aphase, wlim)) { ok = false; break; }
         ptx::tc_fence_after();
         const int row = tm * GEMM_BM + quad * 32 + lane;
-        const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * BN + half * COLS);
+        const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * ACC + half * COLS);
 #pragma unroll 1
         for (int c = 0; c < COLS; c += 16) {
           uint32_t v[16];

@@ -39,6 +39,10 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 struct XfmrLayer {
   float *ln1_g, *ln1_b, *bqkv, *bo, *ln2_g, *ln2_b, *bq2, *bo2, *ln3_g, *ln3_b, *b1, *b2;
   void *Wqkv, *Wo, *Wq2, *Wo2, *W1, *W2;      // [out, in], bf16 or fp32 by precision
+  // decoder transformer, bf16, 64-wide heads, H = 16: the QKV projection again with its output features ordered
+  // head by head, [Q_h | K_h | V_h] (64 each), for the GEMM whose epilogue runs the self-attention (null: not built)
+  void* Wqkv_hm = nullptr;
+  float* bqkv_hm = nullptr;
 };
 
 struct Net {
@@ -389,7 +393,7 @@ int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, in
          int ldo, cudaStream_t s, const GateSpec* gs = nullptr, int conv_c = 0) {
   if (M <= 0) return TSDP_OK;
   GemmArgs g{M, N, K, bias, out, ldo, c->status, nullptr, 0, nullptr, 1, 0, 1, 1, conv_c > 0 ? conv_c : K, conv_c,
-             LiveRows{nullptr, 0, 0}, nullptr, 0, 0};
+             LiveRows{nullptr, 0, 0}, nullptr, 0, 0, 0};
   if (c->dbg_armed && c->dbg_in_test_gemm && c->cfg.precision == 1) {      // one launch: see tsdp_debug_arm_gemm_timeout
     g.wait_cycles = c->dbg_wait_cycles;
     g.withhold_first_stage = 1;
@@ -454,7 +458,7 @@ int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, in
 // fp32 CUDA-core GEMM whatever the precision mode: the timestep-conditioning tables built at weight load.
 int gemm_f32(tsdp_ctx* c, const float* A, const float* W, const float* bias, int M, int N, int K, int epi, float* out,
              cudaStream_t s) {
-  GemmArgs g{M, N, K, bias, out, N, c->status, nullptr, 0, nullptr, 1, 0, 1, 1, K, 0, LiveRows{nullptr, 0, 0}, nullptr, 0, 0};
+  GemmArgs g{M, N, K, bias, out, N, c->status, nullptr, 0, nullptr, 1, 0, 1, 1, K, 0, LiveRows{nullptr, 0, 0}, nullptr, 0, 0, 0};
   dim3 grid((N + 63) / 64, (M + 63) / 64);
   if (epi == EPI_MISH) TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_MISH>), grid, 256, 0, s, A, W, g);
   else if (epi == EPI_SILU) TSDP_LAUNCH(c, (gemm_simt_kernel<EPI_SILU>), grid, 256, 0, s, A, W, g);
@@ -575,6 +579,32 @@ int cross_attn_launch(tsdp_ctx* c, const Net& n, const T* q2, T* out, const Cand
   return TSDP_OK;
 }
 
+// Whether the QKV projection and the causal self-attention of this net run as one tensor-core kernel (EPI_ATTN).
+bool fused_attn_ok(const tsdp_config_t& cfg, const tsdp_net_t& net) {
+  return cfg.precision == 1 && net.arch == TSDP_ARCH_XFMR && cfg.H == 16 && net.heads > 0 && net.d / net.heads == 64 &&
+         getenv("TSDP_NO_FUSED_ATTN") == nullptr;
+}
+
+// a [M, d] -> attention output [M, d]: QKV projection (head-major weights) with the 16-token causal self-attention in
+// the GEMM's epilogue.  M is a multiple of 16 (whole candidates).
+int gemm_qkv_attn(tsdp_ctx* c, const void* A, const XfmrLayer& w, int M, int d, void* out, cudaStream_t s) {
+  const int N = 3 * d, K = d, BN = GEMM_ATTN_BN;
+  GemmArgs g{M, N, K, w.bqkv_hm, out, d, c->status, nullptr, 0, nullptr, 1, 0, 1, 1, K, 0, LiveRows{nullptr, 0, 0}, nullptr, 0, 0, 1};
+  if (c->live_n != nullptr && c->live_static > 0 && M % c->live_static == 0) g.live = LiveRows{c->live_n, M / c->live_static, 0};
+  CUtensorMap ma, mb;
+  int r;
+  if ((r = get_map(c, A, 2, M, K, K, GEMM_BK, GEMM_BM, &ma)) != TSDP_OK) return r;
+  if ((r = get_map(c, w.Wqkv_hm, 2, N, K, K, GEMM_BK, BN, &mb)) != TSDP_OK) return r;
+  const int tiles = ((M + GEMM_BM - 1) / GEMM_BM) * (N / BN);
+  const int grid = tiles < c->num_sms ? tiles : c->num_sms;
+  prof_begin(c, s, c->prof_gemm_cat, 2.0 * gemm_rows_known(c, g) * N * K);
+  TSDP_LAUNCH(c, (gemm_tcgen05_kernel<GEMM_ATTN_BN, EPI_ATTN>), grid, GEMM_THREADS, gemm_smem_bytes(BN), s, ma, mb, ma, g);
+  prof_end(c, s);
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  return TSDP_OK;
+}
+
 // Whether the cross-attention sub-block of this net runs folded into its memory tokens (xattn_fold.cuh).
 bool xfold_ok(const tsdp_config_t& cfg, const tsdp_net_t& net) {
   if (cfg.precision != 1 || net.arch != TSDP_ARCH_XFMR || getenv("TSDP_NO_FOLD") != nullptr) return false;
@@ -647,8 +677,15 @@ int xfmr_forward_t(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStrea
   for (int l = 0; l < L; ++l) {
     const XfmrLayer& w = n.L[l];
     if (l > 0 && (r = ln_launch<T>(c, c->h, w.ln1_g, w.ln1_b, a, M, d, s))) return r;
-    if ((r = gemm(c, a, w.Wqkv, w.bqkv, M, 3 * d, d, out_epi, qkv, 3 * d, s))) return r;
-    if ((r = self_attn_launch<T>(c, qkv, a, n_cand, H, d, heads, s))) return r;
+    if (w.Wqkv_hm != nullptr && std::is_same<T, __nv_bfloat16>::value) {
+      // QKV projection and self-attention in one kernel: q, k, v never reach memory.  Its output goes to q2 (the
+      // kernel reads `a` while it writes) and is then the operand of the attention projection.
+      if ((r = gemm_qkv_attn(c, a, w, M, d, q2, s))) return r;
+      std::swap(a, q2);
+    } else {
+      if ((r = gemm(c, a, w.Wqkv, w.bqkv, M, 3 * d, d, out_epi, qkv, 3 * d, s))) return r;
+      if ((r = self_attn_launch<T>(c, qkv, a, n_cand, H, d, heads, s))) return r;
+    }
     if (n.fold) {
       // the attention projection leaves as bf16; the fold kernel adds it to the stream, does the cross-attention
       // sub-block and the LayerNorm in front of the MLP
@@ -1378,6 +1415,8 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
     INIT_TRY(set_smem_attr_all<128>());
     INIT_TRY(set_smem_attr_all<64>());
     INIT_TRY(set_smem_attr_all<32>());
+    INIT_TRY(cudaFuncSetAttribute(gemm_tcgen05_kernel<GEMM_ATTN_BN, EPI_ATTN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  gemm_smem_bytes(GEMM_ATTN_BN)));
   }
   for (int which = 0; which < 2; ++which) {
     const tsdp_net_t& nn = which == TSDP_BASE ? cfg->base : cfg->draft;
@@ -1782,6 +1821,20 @@ int tsdp_load_weights(tsdp_ctx* c, int which, const float* blob, size_t n) {
       if ((r = up_f32(&w.ln1_g, d))) return r;
       if ((r = up_f32(&w.ln1_b, d))) return r;
       if ((r = up_wT(&w.Wqkv, cur, d, 3 * d))) return r;
+      if (fused_attn_ok(cfg, net.cfg)) {      // the same matrix and bias, output features head-major
+        const size_t heads = net.cfg.heads;
+        std::vector<float> wp(d * 3 * d), bp(3 * d);
+        const float* bsrc = cur + d * 3 * d;
+        for (size_t o = 0; o < 3 * d; ++o) {
+          const size_t which = o / d, hd = (o % d) / 64, cc = o % 64, on = hd * 192 + which * 64 + cc;
+          for (size_t i = 0; i < d; ++i) wp[i * 3 * d + on] = cur[i * 3 * d + o];
+          bp[on] = bsrc[o];
+        }
+        (void)heads;
+        if ((r = up_wT(&w.Wqkv_hm, wp.data(), d, 3 * d))) return r;
+        if (dev_alloc(c, net.allocs, &w.bqkv_hm, 3 * d)) return TSDP_ERR_CUDA;
+        CU_TRY(c, cudaMemcpy(w.bqkv_hm, bp.data(), 3 * d * sizeof(float), cudaMemcpyHostToDevice));
+      }
       cur += d * 3 * d;
       if ((r = up_f32(&w.bqkv, 3 * d))) return r;
       if ((r = up_wT(&w.Wo, cur, d, d))) return r;

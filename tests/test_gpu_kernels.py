@@ -205,3 +205,32 @@ def test_gemm_bounded_wait_runs_out_and_the_context_recovers():
     with pytest.raises(binding.TsdpError):
         smp.arm_gemm_timeout(10)                                  # below the accepted range
     smp.close()
+
+
+def test_fused_qkv_attention_equals_the_separate_kernels(monkeypatch):
+    """With 64-wide heads and 16-token chunks the QKV projection and the causal self-attention are one tensor-core
+    kernel (the attention runs in the GEMM's epilogue on the tile it has just produced).  It shares the attention
+    arithmetic with the stand-alone kernel, so the denoiser output must be bit-identical with the fusion switched off;
+    both are then held to the oracle.  301 candidates: 37 full 128-row tiles and a ragged one."""
+    wl = dict(inputs.WORKLOADS["pusht_xfmr"], precision=1, gamma=1.0)
+    N = 301
+    rng = np.random.default_rng(4)
+    x = rng.normal(size=(N, wl["H"], wl["A"])).astype(np.float32)
+    tau = rng.integers(0, 100, size=N).astype(np.int32)
+    obs = inputs.make_obs(6, N, wl["To"], wl["Do"])
+    outs = []
+    for fused in (True, False):
+        if not fused:
+            monkeypatch.setenv("TSDP_NO_FUSED_ATTN", "1")
+        smp, S, base, draft = hp.setup(wl, max_B=N, max_K=1)
+        dx = torch.tensor(x, device="cuda"); dobs = torch.tensor(obs, dtype=torch.float32, device="cuda")
+        out = torch.zeros_like(dx)
+        smp.denoise(binding.BASE, dx, tau, dobs, N, out)
+        outs.append(out.clone())
+        if fused:
+            got = out.cpu().numpy()
+            for n in (0, 7, 8, 127, 300):
+                ref = base(x[n].astype(np.float64), int(tau[n]), obs[n])
+                assert hp.max_rel(got[n], ref) < 2e-2, n
+        smp.close()
+    assert torch.equal(outs[0], outs[1])

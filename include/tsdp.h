@@ -242,7 +242,10 @@ int tsdp_denoise(tsdp_ctx* ctx, int which, const float* d_x, const int* h_tau, c
 
 /* C[M,N] = A[M,K] W[N,K]^T + bias through the context's GEMM (tcgen05 in precision 1, where d_A, d_W
  * are bf16 and K % 64 == 0, N % 32 == 0; CUDA cores in precision 0, where they are fp32).
- * epi: 0 store (bf16 / fp32 by precision), 1 GELU then store, 2 d_out fp32 += result, 3 store fp32.
+ * epi: 0 store (bf16 / fp32 by precision), 1 GELU then store, 2 d_out fp32 += result, 3 store fp32,
+ * 4 (precision 1, N = 3K, K % 64 = 0, M % 16 = 0) the fused QKV projection + causal self-attention over chunks of
+ *   16 rows with 64-wide heads: W rows (output features) ordered head by head, [Q_h | K_h | V_h] of 64 each; d_out is
+ *   the attention output, bf16 [M, K].
  * Test interface; synchronous. */
 int tsdp_gemm(tsdp_ctx* ctx, const void* d_A, const void* d_W, const float* d_bias, int M, int N, int K,
               int epi, void* d_out, void* cuda_stream);

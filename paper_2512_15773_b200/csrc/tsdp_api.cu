@@ -605,6 +605,13 @@ int gemm_qkv_attn(tsdp_ctx* c, const void* A, const XfmrLayer& w, int M, int d, 
   return TSDP_OK;
 }
 
+int gemm_qkv_attn_raw(tsdp_ctx* c, const void* A, const void* W_hm, const float* b_hm, int M, int d, void* out, cudaStream_t s) {
+  XfmrLayer w{};
+  w.Wqkv_hm = const_cast<void*>(W_hm);
+  w.bqkv_hm = const_cast<float*>(b_hm);
+  return gemm_qkv_attn(c, A, w, M, d, out, s);
+}
+
 // Whether the cross-attention sub-block of this net runs folded into its memory tokens (xattn_fold.cuh).
 bool xfold_ok(const tsdp_config_t& cfg, const tsdp_net_t& net) {
   if (cfg.precision != 1 || net.arch != TSDP_ARCH_XFMR || getenv("TSDP_NO_FOLD") != nullptr) return false;
@@ -2284,13 +2291,14 @@ int tsdp_distill_step(tsdp_ctx* c, const float* d_x0, const float* d_obs, int N,
 
 int tsdp_gemm(tsdp_ctx* c, const void* d_A, const void* d_W, const float* d_bias, int M, int N, int K, int epi,
               void* d_out, void* stream) {
-  if (!c || !d_A || !d_W || !d_out || M < 1 || N < 1 || K < 1 || epi < 0 || epi > 3) return TSDP_ERR_ARG;
+  if (!c || !d_A || !d_W || !d_out || M < 1 || N < 1 || K < 1 || epi < 0 || epi > 4) return TSDP_ERR_ARG;
+  if (epi == 4 && (c->cfg.precision != 1 || N != 3 * K || K % 64 != 0 || M % 16 != 0)) return TSDP_ERR_ARG;
   CU_TRY(c, cudaSetDevice(c->cfg.device));
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   if (c->cfg.precision == 0 && epi == EPI_STORE) epi = EPI_F32;
   c->launches_per_round_tmp = 0;
   c->dbg_in_test_gemm = true;
-  int r = gemm(c, d_A, d_W, d_bias, M, N, K, epi, d_out, N, s);
+  int r = epi == 4 ? gemm_qkv_attn_raw(c, d_A, d_W, d_bias, M, K, d_out, s) : gemm(c, d_A, d_W, d_bias, M, N, K, epi, d_out, N, s);
   c->dbg_in_test_gemm = false;
   c->launches += c->launches_per_round_tmp;
   if (r) return r;
@@ -2309,18 +2317,23 @@ int tsdp_debug_arm_gemm_timeout(tsdp_ctx* c, long long wait_cycles) {
 
 int tsdp_gemm_timed(tsdp_ctx* c, const void* d_A, const void* d_W, const float* d_bias, int M, int N, int K, int epi,
                     void* d_out, int reps, float* h_ms, void* stream) {
-  if (!c || !d_A || !d_W || !d_out || !h_ms || M < 1 || N < 1 || K < 1 || epi < 0 || epi > 3 || reps < 1)
+  if (!c || !d_A || !d_W || !d_out || !h_ms || M < 1 || N < 1 || K < 1 || epi < 0 || epi > 4 || reps < 1)
     return TSDP_ERR_ARG;
+  if (epi == 4 && (c->cfg.precision != 1 || N != 3 * K || K % 64 != 0 || M % 16 != 0)) return TSDP_ERR_ARG;
   CU_TRY(c, cudaSetDevice(c->cfg.device));
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  cudaStream_t s_ = s;
   if (c->cfg.precision == 0 && epi == EPI_STORE) epi = EPI_F32;
+  auto one = [&]() {
+    return epi == 4 ? gemm_qkv_attn_raw(c, d_A, d_W, d_bias, M, K, d_out, s_) : gemm(c, d_A, d_W, d_bias, M, N, K, epi, d_out, N, s_);
+  };
   cudaEvent_t e0, e1;
   CU_TRY(c, cudaEventCreate(&e0));
   CU_TRY(c, cudaEventCreate(&e1));
   c->launches_per_round_tmp = 0;
-  int r = gemm(c, d_A, d_W, d_bias, M, N, K, epi, d_out, N, s);     // builds the tensor maps, warms up
+  int r = one();     // builds the tensor maps, warms up
   cudaEventRecord(e0, s);
-  for (int i = 0; i < reps && r == TSDP_OK; ++i) r = gemm(c, d_A, d_W, d_bias, M, N, K, epi, d_out, N, s);
+  for (int i = 0; i < reps && r == TSDP_OK; ++i) r = one();
   cudaEventRecord(e1, s);
   c->launches += c->launches_per_round_tmp;
   cudaError_t e = cudaStreamSynchronize(s);

@@ -234,3 +234,28 @@ def test_fused_qkv_attention_equals_the_separate_kernels(monkeypatch):
                 assert hp.max_rel(got[n], ref) < 2e-2, n
         smp.close()
     assert torch.equal(outs[0], outs[1])
+
+
+def test_fused_qkv_attention_kernel_against_fp64():
+    """tsdp_gemm, epilogue 4: projection with head-major output features [Q_h | K_h | V_h] and the causal attention
+    of every 16-row chunk, against the definition in fp64 (softmax(Q K^T / 8) V per head, q / k / v rounded to bf16
+    as the kernel keeps them)."""
+    wl = hp.small_xfmr_workload(1)
+    smp, *_ = hp.setup(wl, max_B=1, max_K=1)
+    rng = np.random.default_rng(7)
+    for M, d in ((16, 64), (2000, 256), (6544, 512)):
+        heads = d // 64
+        A = inputs.bf16_round(rng.normal(size=(M, d)))
+        W = inputs.bf16_round(rng.normal(size=(3 * d, d)) / np.sqrt(d))
+        bias = rng.normal(size=3 * d).astype(np.float32)
+        qkv = inputs.bf16_round(A @ W.T + bias.astype(np.float64)).reshape(M // 16, 16, heads, 3, 64)
+        q, k, v = qkv[:, :, :, 0], qkv[:, :, :, 1], qkv[:, :, :, 2]                     # [chunk, token, head, 64]
+        s = np.einsum("cihe,cjhe->chij", q, k) / 8.0
+        s = np.where(np.tril(np.ones((16, 16), dtype=bool)), s, -np.inf)
+        p = np.exp(s - s.max(-1, keepdims=True)); p /= p.sum(-1, keepdims=True)
+        ref = np.einsum("chij,cjhe->cihe", p, v).reshape(M, d)
+        out = torch.zeros(M, d, dtype=torch.bfloat16, device="cuda")
+        smp.gemm(torch.tensor(A, dtype=torch.bfloat16, device="cuda"), torch.tensor(W, dtype=torch.bfloat16, device="cuda"),
+                 torch.tensor(bias, device="cuda"), M, 3 * d, d, 4, out)
+        assert hp.max_rel(out.float().cpu().numpy().astype(np.float64), ref) < 1.5e-2, (M, d)
+    smp.close()

@@ -53,6 +53,14 @@ __host__ __device__ constexpr int gemm_epi_smem_bytes(int BN) {
 __host__ __device__ constexpr int gemm_smem_bytes(int BN) {
   return gemm_stages(BN) * gemm_stage_bytes(BN) + gemm_epi_smem_bytes(BN) + 1024 + 256;
 }
+// CTA-pair form (CG = 2, tcgen05 cta_group::2): a 256 x BN tile on two SMs.  Each CTA stages its own 128 rows of A and
+// HALF of the W tile, so a stage is smaller and the ring deeper.
+constexpr int GEMM_PAIR_STAGES = 6;
+__host__ __device__ constexpr int gemm_stage_bytes_cg(int BN, int CG) { return GEMM_BM * GEMM_BK * 2 + (BN / CG) * GEMM_BK * 2; }
+__host__ __device__ constexpr int gemm_stages_cg(int BN, int CG) { return CG == 2 ? GEMM_PAIR_STAGES : gemm_stages(BN); }
+__host__ __device__ constexpr int gemm_smem_bytes_cg(int BN, int CG) {
+  return gemm_stages_cg(BN, CG) * gemm_stage_bytes_cg(BN, CG) + gemm_epi_smem_bytes(BN) + 1024 + 256;
+}
 
 namespace ptx {
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -102,6 +110,46 @@ __device__ __forceinline__ void tmem_relinquish() {
 }
 __device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t ncols) {
   asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(ncols) : "memory");
+}
+// ---- CTA-pair (cta_group::2) forms.  The two CTAs of a cluster of 2 act as one tensor-core unit: the leader (cluster
+// rank 0) issues the MMAs, which read A from each CTA's own shared memory and one half of the B tile from each.
+__device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t mapa_rank(uint32_t addr, uint32_t rank) {
+  uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank)); return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load whose completion is counted on a barrier that may live in the peer CTA (no multicast: each CTA fetches its own tiles)
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar_cluster_addr) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t addr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(ncols) : "memory");
+}
+// arrive on the barrier at this shared-memory offset in BOTH CTAs of the pair once the MMAs issued so far are done
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -189,8 +237,8 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
 }
 
 // Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M = 128, N = BN.
-__host__ __device__ constexpr uint32_t umma_idesc_bf16(int BN) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(GEMM_BM >> 4) << 24);
+__host__ __device__ constexpr uint32_t umma_idesc_bf16(int BN, int M = GEMM_BM) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -274,16 +322,24 @@ __device__ __forceinline__ void epilogue_store16(const GemmArgs& g, int row, int
   }
 }
 
-template <int BN, int EPI>
+// CG = 1: one CTA per 128 x BN tile.  CG = 2: launched in clusters of two CTAs that share a 256 x BN tile (cta_group::2):
+// CTA `rank` owns rows [128 rank, +128) of the tile and stages rows [rank BN/2, +BN/2) of the W tile; the leader's MMA
+// warp issues for both; stage and accumulator hand-over barriers are signalled in both CTAs by multicast commits, the
+// stage-full and accumulator-empty barriers live in the leader and are signalled from both CTAs.  Per flop each SM
+// pulls a third fewer operand bytes from the L2, which is what bounds the 128 x 256 form at K = 512.
+template <int BN, int EPI, int CG = 1>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmC, GemmArgs g) {
-  constexpr int STAGES = gemm_stages(BN);
+  constexpr int STAGES = gemm_stages_cg(BN, CG);
   constexpr int A_BYTES = GEMM_BM * GEMM_BK * 2;
-  constexpr int STAGE_BYTES = gemm_stage_bytes(BN);
+  constexpr int B_ROWS = BN / CG;                      // rows of the W tile this CTA stages
+  constexpr int STAGE_BYTES = gemm_stage_bytes_cg(BN, CG);
+  static_assert(CG == 1 || CG == 2, "CG");
+  static_assert(CG == 1 || BN == 256 || BN == GEMM_ATTN_BN, "pair form: wide tiles only");
   constexpr int ACC = BN == GEMM_ATTN_BN ? 256 : BN;          // column distance of the two accumulator buffers
   constexpr uint32_t TMEM_COLS = (2 * ACC < 32) ? 32 : 2 * ACC;  // a power of two
-  constexpr uint32_t IDESC = umma_idesc_bf16(BN);
+  constexpr uint32_t IDESC = umma_idesc_bf16(BN, GEMM_BM * CG);
   static_assert(BN == 32 || BN == 64 || BN == 128 || BN == 256 || BN == GEMM_ATTN_BN, "BN");
   static_assert((EPI == EPI_ATTN) == (BN == GEMM_ATTN_BN), "the fused attention epilogue has its own tile width");
 
@@ -304,51 +360,67 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tiles_n = g.N / BN;
   const int kblocks = g.K / GEMM_BK;
+  const uint32_t rank = CG == 2 ? ptx::cluster_rank() : 0u;     // 0: the pair's leader
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(full_bar(s), 1); ptx::mbar_init(empty_bar(s), 1); }
-    for (int s = 0; s < 2; ++s) { ptx::mbar_init(tfull_bar(s), 1); ptx::mbar_init(tempty_bar(s), GEMM_EPI_WARPS); }
+    for (int s = 0; s < 2; ++s) { ptx::mbar_init(tfull_bar(s), 1); ptx::mbar_init(tempty_bar(s), GEMM_EPI_WARPS * CG); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    ptx::tmem_alloc(tmem_slot, TMEM_COLS);
-    ptx::tmem_relinquish();
+    if (CG == 2) { ptx::tmem_alloc_pair(tmem_slot, TMEM_COLS); ptx::tmem_relinquish_pair(); }
+    else { ptx::tmem_alloc(tmem_slot, TMEM_COLS); ptx::tmem_relinquish(); }
   }
   ptx::tc_fence_before();
   __syncthreads();
+  if (CG == 2) ptx::cluster_sync_all();      // the peer's barriers exist before anything is signalled across the pair
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_ptr;
   bool ok = true;
   const long long wlim = g.wait_cycles > 0 ? g.wait_cycles : GEMM_WAIT_CYCLES;
   pdl_wait();      // operands, bias, the output and the live-row count belong to earlier kernels of the stream
   const int M = live_rows(g.live, g.M);
-  const int tiles_m = (M + GEMM_BM - 1) / GEMM_BM;
+  const int tiles_m = (M + GEMM_BM * CG - 1) / (GEMM_BM * CG);     // tiles of 128 CG rows
   const int n_tiles = tiles_m * tiles_n;
+  const int tile0 = blockIdx.x / CG, tile_step = gridDim.x / CG;      // both CTAs of a pair walk the same tiles
+  // an epilogue warp hands accumulator buffer `as` back: the barrier that the MMA warp waits on lives in the leader
+  auto release_acc = [&](int as) {
+    if (CG == 2 && rank != 0) ptx::mbar_arrive_cluster(ptx::mapa_rank(tempty_bar(as), 0));
+    else ptx::mbar_arrive(tempty_bar(as));
+  };
 
   if (warp == 0) {
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-        const int tm = tile / tiles_n, tn = tile % tiles_n;
+      for (int tile = tile0; tile < n_tiles && ok; tile += tile_step) {
+        const int tm = (tile / tiles_n) * CG + (int)rank, tn = tile % tiles_n;
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!ptx::mbar_wait_thread(empty_bar(stage), phase ^ 1u, wlim)) { ok = false; break; }
           if (!(g.withhold_first_stage && blockIdx.x == 0 && tile == 0 && kb == 0)) {
-            ptx::mbar_expect_tx(full_bar(stage), STAGE_BYTES);
             const uint32_t sa = base + stage * STAGE_BYTES;
             const int kcol = kb * GEMM_BK;
             const int ax = g.conv_c ? kcol % g.conv_c : kcol, ay = tm * GEMM_BM + (g.conv_c ? kcol / g.conv_c : 0);
-            ptx::tma_load_2d(sa, &tmA, ax, ay, full_bar(stage));
-            ptx::tma_load_2d(sa + A_BYTES, &tmB, kb * GEMM_BK, tn * BN, full_bar(stage));
+            if (CG == 2) {
+              // the leader's barrier counts the bytes of both CTAs' loads of this stage
+              if (rank == 0) ptx::mbar_expect_tx(full_bar(stage), STAGE_BYTES * 2);
+              const uint32_t fb = ptx::mapa_rank(full_bar(stage), 0);
+              ptx::tma_load_2d_pair(sa, &tmA, ax, ay, fb);
+              ptx::tma_load_2d_pair(sa + A_BYTES, &tmB, kb * GEMM_BK, tn * BN + (int)rank * B_ROWS, fb);
+            } else {
+              ptx::mbar_expect_tx(full_bar(stage), STAGE_BYTES);
+              ptx::tma_load_2d(sa, &tmA, ax, ay, full_bar(stage));
+              ptx::tma_load_2d(sa + A_BYTES, &tmB, kb * GEMM_BK, tn * BN, full_bar(stage));
+            }
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    if (lane == 0 && rank == 0) {      // in a pair only the leader issues
       int stage = 0; uint32_t phase = 0; int it = 0;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
+      for (int tile = tile0; tile < n_tiles && ok; tile += tile_step, ++it) {
         const int as = it & 1; const uint32_t aphase = (it >> 1) & 1;
         if (!ptx::mbar_wait_thread(tempty_bar(as), aphase ^ 1u, wlim)) { ok = false; break; }
         ptx::tc_fence_after();
@@ -359,13 +431,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           const uint32_t sa = base + stage * STAGE_BYTES;
           const uint64_t da = umma_desc_sw128(sa), db = umma_desc_sw128(sa + A_BYTES);
 #pragma unroll
-          for (int k = 0; k < GEMM_BK / 16; ++k)
-            ptx::tc_mma_bf16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), IDESC, (kb | k) ? 1u : 0u);
-          ptx::tc_commit(empty_bar(stage));
+          for (int k = 0; k < GEMM_BK / 16; ++k) {
+            if (CG == 2) ptx::tc_mma_bf16_pair(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), IDESC, (kb | k) ? 1u : 0u);
+            else ptx::tc_mma_bf16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), IDESC, (kb | k) ? 1u : 0u);
+          }
+          if (CG == 2) ptx::tc_commit_pair(empty_bar(stage)); else ptx::tc_commit(empty_bar(stage));
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        ptx::tc_commit(tfull_bar(as));
+        if (CG == 2) ptx::tc_commit_pair(tfull_bar(as)); else ptx::tc_commit(tfull_bar(as));
       }
     }
   } else {
@@ -384,8 +458,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int r_tile = quad * 32 + lane;                    // this lane's row of the tile
       const int cand_l = r_tile >> 4, r_l = r_tile & 15;      // candidate (0..7) and token of that row
       const int cand_w = 2 * quad + half;                     // the candidate this warp attends for
-      for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
-        const int tm = tile / tiles_n, tn = tile % tiles_n;
+      for (int tile = tile0; tile < n_tiles; tile += tile_step, ++it) {
+        const int tm = (tile / tiles_n) * CG + (int)rank, tn = tile % tiles_n;
         const int as = it & 1; const uint32_t aphase = (it >> 1) & 1;
         // both warps of the quadrant agree on the outcome; the barrier also orders the previous tile's reads of the
         // staging area before this tile's writes
@@ -401,7 +475,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           if (part == 2) {                                    // accumulator fully read: hand it back
             ptx::tc_fence_before();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(tempty_bar(as));
+            if (lane == 0) release_acc(as);
           }
           const int col = half * 96 + part * 32;              // column inside the head's [Q | K | V]
           float f[32];
@@ -445,8 +519,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const uint32_t sw = (uint32_t)(r & 7);
       const bool issuer = (quad == 0 && lane == 0);
       const int bar_id = 1 + half;
-      for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
-        const int tm = tile / tiles_n, tn = tile % tiles_n;
+      for (int tile = tile0; tile < n_tiles; tile += tile_step, ++it) {
+        const int tm = (tile / tiles_n) * CG + (int)rank, tn = tile % tiles_n;
         const int as = it & 1; const uint32_t aphase = (it >> 1) & 1;
         // all four warps of this half agree on the outcome, so none is left alone at a named barrier
         ok = ptx::named_bar_and(bar_id, 128, ptx::mbar_wait_warp(tfull_bar(as), aphase, wlim));
@@ -464,7 +538,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             if (ch == NCH - 1 && part == CW / 32 - 1) {            // accumulator fully read: hand it back
               ptx::tc_fence_before();
               __syncwarp();
-              if (lane == 0) ptx::mbar_arrive(tempty_bar(as));
+              if (lane == 0) release_acc(as);
             }
             const int col = tn * BN + half * COLS + col_t;
             float f[32];
@@ -521,8 +595,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       }
       if (issuer) ptx::bulk_wait_read0();
     } else {
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
-        const int tm = tile / tiles_n, tn = tile % tiles_n;
+      for (int tile = tile0; tile < n_tiles && ok; tile += tile_step, ++it) {
+        const int tm = (tile / tiles_n) * CG + (int)rank, tn = tile % tiles_n;
         const int as = it & 1; const uint32_t aphase = (it >> 1) & 1;
         if (!ptx::mbar_wait_warp(tfull_bar(as), aphase, wlim)) { ok = false; break; }
         ptx::tc_fence_after();
@@ -537,7 +611,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
         ptx::tc_fence_before();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(tempty_bar(as));
+        if (lane == 0) release_acc(as);
       }
     }
   }
@@ -549,8 +623,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   }
   ptx::tc_fence_before();
   __syncthreads();
+  if (CG == 2) ptx::cluster_sync_all();      // neither CTA leaves while its peer may still signal or read it
   ptx::tc_fence_after();
-  if (warp == 1) ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+  if (warp == 1) {
+    if (CG == 2) ptx::tmem_dealloc_pair(tmem_base, TMEM_COLS);
+    else ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+  }
 }
 
 }  // namespace tsdp

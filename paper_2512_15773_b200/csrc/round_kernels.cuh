@@ -179,6 +179,26 @@ __global__ void draft_step_kernel(DdpmTables S, float* __restrict__ xt, long lon
   }
 }
 
+// Four consecutive latent values starting at element 4q: one 16-byte load when D is a multiple of 4 (every row of
+// the round's buffers then starts on a 16-byte boundary), element by element with a bounds check otherwise.
+__device__ __forceinline__ void load_quad(const float* __restrict__ p, int q, int D, bool vec, float v[4]) {
+  if (vec) {
+    const float4 t = *reinterpret_cast<const float4*>(p + 4 * q);
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+  } else {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) v[j] = 4 * q + j < D ? p[4 * q + j] : 0.f;
+  }
+}
+__device__ __forceinline__ void store_quad(float* __restrict__ p, int q, int D, bool vec, const float v[4]) {
+  if (vec) *reinterpret_cast<float4*>(p + 4 * q) = make_float4(v[0], v[1], v[2], v[3]);
+  else {
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if (4 * q + j < D) p[4 * q + j] = v[j];
+  }
+}
+
 // Fused verification tail, one block per environment, one warp per drafted step.
 //   warp k-1 (k = 1..K_eff): mu_k = posterior mean of (x~_{k-1}, eps_{k-1}) at tau = t-k+1;
 //       d = (mu^_k - mu_k) / (s sigma_tau);  log alpha = -1/2 |d|^2 - <d, xi_tau>   (Sec. 3.2)
@@ -221,20 +241,27 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
   const float* xb = xt + b * xs_b;
   const float* mb = muhat + b * ms_b;
   const float* eb = eps + b * es_b;
+  // 16-byte loads when every row of the three buffers is 16-byte aligned
+  const bool vec = (D & 3) == 0 && (xs_b & 3) == 0 && (ms_b & 3) == 0 && (es_b & 3) == 0 &&
+                   ((reinterpret_cast<uintptr_t>(xt) | reinterpret_cast<uintptr_t>(muhat) | reinterpret_cast<uintptr_t>(eps) |
+                     reinterpret_cast<uintptr_t>(actions)) & 15) == 0;
 
   for (int k = warp + 1; k <= K_eff; k += (blockDim.x >> 5)) {
     const int tau = tb - k + 1;
     const float inv = 1.0f / (rp.sigma_scale * S.sigma[tau]);
     float s1 = 0.f, s2 = 0.f, d2 = 0.f;
     for (int q = lane; q < nq; q += 32) {
-      float z[4];
+      float z[4], xv[4], ev[4], mv[4];
       normal4(seed, (uint32_t)env, STREAM_XI, (uint32_t)tau, (uint32_t)q, z);
+      load_quad(xb + (long long)(k - 1) * D, q, D, vec, xv);
+      load_quad(eb + (long long)(k - 1) * D, q, D, vec, ev);
+      load_quad(mb + (long long)(k - 1) * D, q, D, vec, mv);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int i = 4 * q + j;
         if (i < D) {
-          const float mu = posterior_mean(S, xb[(long long)(k - 1) * D + i], eb[(long long)(k - 1) * D + i], tau);
-          const float delta = mb[(long long)(k - 1) * D + i] - mu;
+          const float mu = posterior_mean(S, xv[j], ev[j], tau);
+          const float delta = mv[j] - mu;
           const float d = delta * inv;
           s1 += d * d; s2 += d * z[j]; d2 += delta * delta;
         }
@@ -274,36 +301,32 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
     // e <e, xi> = Delta <Delta, xi> / |Delta|^2 = Delta * S2 / (S1 * s * sigma)
     const float coef = 2.0f * s_s2[j - 1] / (s_s1[j - 1] * rp.sigma_scale * sig);
     for (int q = threadIdx.x; q < nq; q += blockDim.x) {
-      float z[4];
+      float z[4], xv[4], ev[4], mv[4], ov[4] = {0.f, 0.f, 0.f, 0.f};
       normal4(seed, (uint32_t)env, STREAM_XI, (uint32_t)tau, (uint32_t)q, z);
+      load_quad(xb + (long long)(j - 1) * D, q, D, vec, xv);
+      load_quad(eb + (long long)(j - 1) * D, q, D, vec, ev);
+      load_quad(mb + (long long)(j - 1) * D, q, D, vec, mv);
 #pragma unroll
       for (int jj = 0; jj < 4; ++jj) {
-        const int i = 4 * q + jj;
-        if (i < D) {
-          const float mu = posterior_mean(S, xb[(long long)(j - 1) * D + i], eb[(long long)(j - 1) * D + i], tau);
-          const float delta = mb[(long long)(j - 1) * D + i] - mu;
-          const float v = mu + sig * (z[jj] - coef * delta);
-          xo[i] = v;
-          if (t_new < 0) actions[(long long)env * D + i] = v;
-        }
+        const float mu = posterior_mean(S, xv[jj], ev[jj], tau);
+        const float delta = mv[jj] - mu;
+        ov[jj] = mu + sig * (z[jj] - coef * delta);
       }
+      store_quad(xo, q, D, vec, ov);
+      if (t_new < 0) store_quad(actions + (long long)env * D, q, D, vec, ov);
     }
   } else if (bonus) {
     const int tau = tb - K_eff;
     const float sig = S.sigma[tau];
     for (int q = threadIdx.x; q < nq; q += blockDim.x) {
-      float z[4] = {0.f, 0.f, 0.f, 0.f};
+      float z[4] = {0.f, 0.f, 0.f, 0.f}, xv[4], ev[4], ov[4];
       if (tau > 0) normal4(seed, (uint32_t)env, STREAM_XI, (uint32_t)tau, (uint32_t)q, z);
+      load_quad(xb + (long long)K_eff * D, q, D, vec, xv);
+      load_quad(eb + (long long)K_eff * D, q, D, vec, ev);
 #pragma unroll
-      for (int jj = 0; jj < 4; ++jj) {
-        const int i = 4 * q + jj;
-        if (i < D) {
-          const float mu = posterior_mean(S, xb[(long long)K_eff * D + i], eb[(long long)K_eff * D + i], tau);
-          const float v = ddpm_sample(mu, sig, z[jj]);
-          xo[i] = v;
-          if (t_new < 0) actions[(long long)env * D + i] = v;
-        }
-      }
+      for (int jj = 0; jj < 4; ++jj) ov[jj] = ddpm_sample(posterior_mean(S, xv[jj], ev[jj], tau), sig, z[jj]);
+      store_quad(xo, q, D, vec, ov);
+      if (t_new < 0) store_quad(actions + (long long)env * D, q, D, vec, ov);
     }
   } else {
     for (int i = threadIdx.x; i < D; i += blockDim.x) {
@@ -312,25 +335,26 @@ __global__ void accept_kernel(DdpmTables S, float* __restrict__ xt, long long xs
       if (t_new < 0) actions[(long long)env * D + i] = v;
     }
   }
-  if (threadIdx.x == 0) {
-    t[b] = t_new;
+  if (threadIdx.x < 32) {      // statistics: the lanes of warp 0 issue the independent atomics side by side
     const int n_acc = min(j - 1, K_eff);
     const int n_tested = min(j, K_eff);
-    atomicAdd(&stats->env_rounds, 1ull);
-    atomicAdd(&stats->base_evals, (unsigned long long)((rp.bonus || K_eff == 0) ? K_eff + 1 : K_eff));
-    atomicAdd(&stats->draft_evals, (unsigned long long)K_eff);
-    atomicAdd(&stats->draft_rounds, K_eff > 0 ? 1ull : 0ull);
-    atomicAdd(&stats->drafts_tested, (unsigned long long)n_tested);
-    atomicAdd(&stats->drafts_accepted, (unsigned long long)n_acc);
-    atomicAdd(&stats->rejections, rejected ? 1ull : 0ull);
-    atomicAdd(&stats->bonus_steps, bonus ? 1ull : 0ull);
-    atomicAdd(&stats->steps_advanced, (unsigned long long)adv);
-    for (int k = 1; k <= K_eff; ++k) {
+    const unsigned long long vals[9] = {1ull, (unsigned long long)((rp.bonus || K_eff == 0) ? K_eff + 1 : K_eff),
+                                        (unsigned long long)K_eff, (unsigned long long)n_tested, (unsigned long long)n_acc,
+                                        rejected ? 1ull : 0ull, bonus ? 1ull : 0ull, (unsigned long long)adv, K_eff > 0 ? 1ull : 0ull};
+    unsigned long long* ctr[9] = {&stats->env_rounds, &stats->base_evals, &stats->draft_evals, &stats->drafts_tested,
+                                  &stats->drafts_accepted, &stats->rejections, &stats->bonus_steps, &stats->steps_advanced,
+                                  &stats->draft_rounds};
+    if (threadIdx.x < 9 && vals[threadIdx.x] != 0ull) atomicAdd(ctr[threadIdx.x], vals[threadIdx.x]);
+    for (int k = 1 + (int)threadIdx.x; k <= K_eff; k += 32) {
       const int tau = tb - k + 1;
       atomicAdd(&stats->hist_drafted[tau], 1ull);
       if (k <= n_tested) atomicAdd(&stats->hist_tested[tau], 1ull);
       if (k <= n_acc) atomicAdd(&stats->hist_accepted[tau], 1ull);
     }
+  }
+  if (threadIdx.x == 0) {
+    t[b] = t_new;
+    const int n_acc = min(j - 1, K_eff);
     if (item_counts) {                     // a request occupies one slot at a time: no atomics needed
       int* ic = item_counts + 4 * (long long)env;
       ic[0] += K_eff; ic[1] += n_acc; ic[2] += 1; ic[3] += adv;

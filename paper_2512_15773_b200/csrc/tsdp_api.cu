@@ -153,6 +153,9 @@ struct tsdp_ctx {
   // while profiling: host copies of the plan's counts, so that a GEMM's flops are those of the rows it really processed
   int prof_plan_live = -1, prof_plan_dn[TSDP_MAX_K + 2] = {};
   int prof_live_count = -1;                   // live candidates of the forward being enqueued (-1: unknown, use the dense count)
+  // CTA-pair GEMM (cta_group::2): clusters of two CTAs that fit the device at once (0: not usable), and whether it is used
+  int pair_clusters = 0, pair_clusters_attn = 0;
+  int pair_mode = 0;                          // TSDP_GEMM_PAIR: 0 never, 1 when the tile count fills the pairs, 2 always
   bool dbg_armed = false, dbg_in_test_gemm = false;   // tsdp_debug_arm_gemm_timeout
   long long dbg_wait_cycles = 0;
   uint64_t cand_static = 0;                   // candidates the dense layout would have evaluated since the last reset
@@ -205,6 +208,20 @@ void launch_kernel(tsdp_ctx* c, void (*kern)(P...), dim3 grid, dim3 block, size_
   cfg.attrs = at;
   cfg.numAttrs = c->pdl ? 1 : 0;
   cudaLaunchKernelEx(&cfg, kern, std::forward<A>(args)...);   // a failure is read by cudaGetLastError at the call site
+}
+// The same for a kernel that runs in clusters of `cluster` CTAs along x.
+template <typename... P, typename... A>
+void launch_kernel_cluster(tsdp_ctx* c, void (*kern)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, int cluster, A&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = cluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = c->pdl ? 2 : 1;
+  cudaLaunchKernelEx(&cfg, kern, std::forward<A>(args)...);
 }
 #define TSDP_LAUNCH(ctx, kern, grid, block, smem, stream, ...) \
   launch_kernel(ctx, kern, dim3(grid), dim3(block), (size_t)(smem), stream, __VA_ARGS__)
@@ -342,6 +359,38 @@ int launch_tc(tsdp_ctx* c, const CUtensorMap& ma, const CUtensorMap& mb, const C
   return TSDP_OK;
 }
 
+// 256 x 256 tiles on CTA pairs (cta_group::2); `mb` is the W map with a box of 128 rows (each CTA stages half a tile).
+template <int EPI>
+int launch_tc_pair(tsdp_ctx* c, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const GemmArgs& g,
+                   cudaStream_t s) {
+  const int tiles = ((g.M + 2 * GEMM_BM - 1) / (2 * GEMM_BM)) * (g.N / 256);
+  const int pairs = tiles < c->pair_clusters ? tiles : c->pair_clusters;
+  prof_begin(c, s, c->prof_gemm_cat, 2.0 * gemm_rows_known(c, g) * g.N * g.K);
+  launch_kernel_cluster(c, gemm_tcgen05_kernel<256, EPI, 2>, dim3(2 * pairs), dim3(GEMM_THREADS), (size_t)gemm_smem_bytes_cg(256, 2), s, 2,
+                        ma, mb, mc, g);
+  prof_end(c, s);
+  c->launches_per_round_tmp++;
+  CU_TRY(c, cudaGetLastError());
+  return TSDP_OK;
+}
+int launch_tc_pair_epi(tsdp_ctx* c, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const GemmArgs& g,
+                       int epi, cudaStream_t s) {
+  switch (epi) {
+    case EPI_STORE: return launch_tc_pair<EPI_STORE>(c, ma, mb, mc, g, s);
+    case EPI_GELU: return launch_tc_pair<EPI_GELU>(c, ma, mb, mc, g, s);
+    case EPI_RESID: return launch_tc_pair<EPI_RESID>(c, ma, mb, mc, g, s);
+    case EPI_GATE: return launch_tc_pair<EPI_GATE>(c, ma, mb, mc, g, s);
+    default: return launch_tc_pair<EPI_F32>(c, ma, mb, mc, g, s);
+  }
+}
+// Whether a GEMM of M rows and N columns runs on CTA pairs: wide outputs, and enough 256 x 256 tiles to occupy the pairs.
+bool use_pair_gemm(const tsdp_ctx* c, int M, int N) {
+  if (c->pair_mode == 0 || c->pair_clusters < 1 || N % 256 != 0) return false;
+  if (c->pair_mode == 2) return true;
+  const long long tiles = (long long)((M + 255) / 256) * (N / 256);
+  return tiles * 5 >= (long long)c->pair_clusters * 4;
+}
+
 template <int BN>
 int launch_tc_epi(tsdp_ctx* c, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const GemmArgs& g,
                   int epi, cudaStream_t s) {
@@ -430,14 +479,15 @@ int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, in
     c->last_error = "tensor-core GEMM needs K % 64 == 0 and N % 32 == 0";
     return TSDP_ERR_ARG;
   }
-  const int BN = (c->force_bn > 0 && N % c->force_bn == 0) ? c->force_bn : pick_bn(M, N, c->num_sms);
+  const bool pair = c->force_bn == 0 && use_pair_gemm(c, M, N);
+  const int BN = pair ? 256 : ((c->force_bn > 0 && N % c->force_bn == 0) ? c->force_bn : pick_bn(M, N, c->num_sms));
   CUtensorMap ma, mb, mc;
   int r;
   if (conv_c > 0) {      // kernel-5 convolution: A is the padded tensor [M + 4, conv_c] itself
     if (conv_c % GEMM_BK != 0 || K != 5 * conv_c) return TSDP_ERR_ARG;
     if ((r = get_map(c, A, 2, M + 4, conv_c, conv_c, GEMM_BK, GEMM_BM, &ma)) != TSDP_OK) return r;
   } else if ((r = get_map(c, A, 2, M, K, K, GEMM_BK, GEMM_BM, &ma)) != TSDP_OK) return r;
-  if ((r = get_map(c, W, 2, N, K, K, GEMM_BK, BN, &mb)) != TSDP_OK) return r;
+  if ((r = get_map(c, W, 2, N, K, K, GEMM_BK, pair ? BN / 2 : BN, &mb)) != TSDP_OK) return r;
   mc = ma;
   if (gemm_tma_epilogue(BN)) {   // the epilogue hands 128-row x 128-byte chunks to TMA
     const int esz = (epi == EPI_STORE || epi == EPI_GELU) ? 2 : 4;
@@ -447,6 +497,7 @@ int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, in
     }
     if ((r = get_map(c, out, esz, M, N, ldo, 128 / esz, GEMM_BM, &mc)) != TSDP_OK) return r;
   }
+  if (pair) return launch_tc_pair_epi(c, ma, mb, mc, g, epi, s);
   switch (BN) {
     case 256: return launch_tc_epi<256>(c, ma, mb, mc, g, epi, s);
     case 128: return launch_tc_epi<128>(c, ma, mb, mc, g, epi, s);
@@ -594,11 +645,19 @@ int gemm_qkv_attn(tsdp_ctx* c, const void* A, const XfmrLayer& w, int M, int d, 
   CUtensorMap ma, mb;
   int r;
   if ((r = get_map(c, A, 2, M, K, K, GEMM_BK, GEMM_BM, &ma)) != TSDP_OK) return r;
-  if ((r = get_map(c, w.Wqkv_hm, 2, N, K, K, GEMM_BK, BN, &mb)) != TSDP_OK) return r;
-  const int tiles = ((M + GEMM_BM - 1) / GEMM_BM) * (N / BN);
-  const int grid = tiles < c->num_sms ? tiles : c->num_sms;
+  const long long ptiles = (long long)((M + 255) / 256) * (N / BN);
+  const bool pair = c->pair_mode != 0 && c->pair_clusters_attn >= 1 && (c->pair_mode == 2 || ptiles * 5 >= (long long)c->pair_clusters_attn * 4);
+  if ((r = get_map(c, w.Wqkv_hm, 2, N, K, K, GEMM_BK, pair ? BN / 2 : BN, &mb)) != TSDP_OK) return r;
   prof_begin(c, s, c->prof_gemm_cat, 2.0 * gemm_rows_known(c, g) * N * K);
-  TSDP_LAUNCH(c, (gemm_tcgen05_kernel<GEMM_ATTN_BN, EPI_ATTN>), grid, GEMM_THREADS, gemm_smem_bytes(BN), s, ma, mb, ma, g);
+  if (pair) {
+    const int pairs = ptiles < c->pair_clusters_attn ? (int)ptiles : c->pair_clusters_attn;
+    launch_kernel_cluster(c, gemm_tcgen05_kernel<GEMM_ATTN_BN, EPI_ATTN, 2>, dim3(2 * pairs), dim3(GEMM_THREADS),
+                          (size_t)gemm_smem_bytes_cg(BN, 2), s, 2, ma, mb, ma, g);
+  } else {
+    const int tiles = ((M + GEMM_BM - 1) / GEMM_BM) * (N / BN);
+    const int grid = tiles < c->num_sms ? tiles : c->num_sms;
+    TSDP_LAUNCH(c, (gemm_tcgen05_kernel<GEMM_ATTN_BN, EPI_ATTN>), grid, GEMM_THREADS, gemm_smem_bytes(BN), s, ma, mb, ma, g);
+  }
   prof_end(c, s);
   c->launches_per_round_tmp++;
   CU_TRY(c, cudaGetLastError());
@@ -1424,6 +1483,26 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
     INIT_TRY(set_smem_attr_all<32>());
     INIT_TRY(cudaFuncSetAttribute(gemm_tcgen05_kernel<GEMM_ATTN_BN, EPI_ATTN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   gemm_smem_bytes(GEMM_ATTN_BN)));
+    if (const char* pm = getenv("TSDP_GEMM_PAIR")) c->pair_mode = atoi(pm);
+    if (c->pair_mode != 0) {      // CTA-pair kernels: shared-memory opt-in and how many clusters of 2 the device holds at once
+      const void* fns[6] = {(const void*)gemm_tcgen05_kernel<256, EPI_STORE, 2>, (const void*)gemm_tcgen05_kernel<256, EPI_GELU, 2>,
+                            (const void*)gemm_tcgen05_kernel<256, EPI_RESID, 2>, (const void*)gemm_tcgen05_kernel<256, EPI_GATE, 2>,
+                            (const void*)gemm_tcgen05_kernel<256, EPI_F32, 2>, (const void*)gemm_tcgen05_kernel<GEMM_ATTN_BN, EPI_ATTN, 2>};
+      for (int i = 0; i < 6; ++i) {
+        const int smem = i < 5 ? gemm_smem_bytes_cg(256, 2) : gemm_smem_bytes_cg(GEMM_ATTN_BN, 2);
+        INIT_TRY(cudaFuncSetAttribute(fns[i], cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        if (i != 0 && i != 5) continue;
+        cudaLaunchConfig_t lc{};
+        lc.gridDim = dim3(2 * c->num_sms); lc.blockDim = dim3(GEMM_THREADS); lc.dynamicSmemBytes = (size_t)smem;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        lc.attrs = at; lc.numAttrs = 1;
+        int ncl = 0;
+        if (cudaOccupancyMaxActiveClusters(&ncl, fns[i], &lc) != cudaSuccess) { cudaGetLastError(); ncl = 0; }
+        if (i == 0) c->pair_clusters = ncl; else c->pair_clusters_attn = ncl;
+      }
+    }
   }
   for (int which = 0; which < 2; ++which) {
     const tsdp_net_t& nn = which == TSDP_BASE ? cfg->base : cfg->draft;

@@ -22,6 +22,9 @@
  * or 512; TSDP_NO_FOLD, set before tsdp_load_weights, keeps the separate kernels.  Same function either way.
  * TSDP_NO_ASYNC_BCAST (read by tsdp_init, like TSDP_NO_PDL) makes the cluster kernel hand its stages over with plain distributed-
  * shared-memory stores and a cluster barrier instead of st.async stores counted by mbarriers.
+ * TSDP_GEMM_PAIR = 0 | 1 | 2 (read by tsdp_init; default 1) selects the two-CTA form of the tensor-core GEMM
+ * (tcgen05 cta_group::2, 256 x 256 tiles on clusters of two CTAs): never / for long reductions with enough tiles /
+ * wherever the output width allows -- a tuning aid; results do not depend on it.
  * TSDP_GEMM_BN = 32 | 64 | 128 | 256 (read by tsdp_init) forces that tile width on every tensor-core GEMM whose
  * output width it divides -- a tuning aid; results do not depend on the tile width.
  * Every function returns a tsdp_status; nothing throws or aborts.  A context is not re-entrant: one

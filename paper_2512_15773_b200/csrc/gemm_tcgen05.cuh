@@ -55,11 +55,16 @@ __host__ __device__ constexpr int gemm_smem_bytes(int BN) {
 }
 // CTA-pair form (CG = 2, tcgen05 cta_group::2): a 256 x BN tile on two SMs.  Each CTA stages its own 128 rows of A and
 // HALF of the W tile, so a stage is smaller and the ring deeper.
-constexpr int GEMM_PAIR_STAGES = 6;
+// The smaller stages also leave room for two staging chunks per column half, so that the epilogue does not have to
+// wait for its previous TMA store (which queues behind the operand loads) before it fills the next chunk.
 __host__ __device__ constexpr int gemm_stage_bytes_cg(int BN, int CG) { return GEMM_BM * GEMM_BK * 2 + (BN / CG) * GEMM_BK * 2; }
-__host__ __device__ constexpr int gemm_stages_cg(int BN, int CG) { return CG == 2 ? GEMM_PAIR_STAGES : gemm_stages(BN); }
+__host__ __device__ constexpr int gemm_stages_cg(int BN, int CG) { return CG == 2 ? (BN == GEMM_ATTN_BN ? 6 : 5) : gemm_stages(BN); }
+__host__ __device__ constexpr int gemm_staging_bufs(int CG) { return CG == 2 ? 2 : 1; }      // per column half
+__host__ __device__ constexpr int gemm_epi_smem_bytes_cg(int BN, int CG) {
+  return gemm_tma_epilogue(BN) ? GEMM_STAGING_BYTES * gemm_staging_bufs(CG) : gemm_epi_smem_bytes(BN);
+}
 __host__ __device__ constexpr int gemm_smem_bytes_cg(int BN, int CG) {
-  return gemm_stages_cg(BN, CG) * gemm_stage_bytes_cg(BN, CG) + gemm_epi_smem_bytes(BN) + 1024 + 256;
+  return gemm_stages_cg(BN, CG) * gemm_stage_bytes_cg(BN, CG) + gemm_epi_smem_bytes_cg(BN, CG) + 1024 + 256;
 }
 
 namespace ptx {
@@ -191,6 +196,7 @@ __device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, int x,
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
@@ -348,7 +354,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   constexpr bool TMA_EPI = gemm_tma_epilogue(BN);
   const uint32_t staging = base + STAGES * STAGE_BYTES;    // 1024-byte aligned: every stage is a multiple of 1 KB
-  const uint32_t bar0 = staging + gemm_epi_smem_bytes(BN);   // full[STAGES], empty[STAGES], tfull[2], tempty[2]
+  const uint32_t bar0 = staging + gemm_epi_smem_bytes_cg(BN, CG);   // full[STAGES], empty[STAGES], tfull[2], tempty[2]
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
   auto tfull_bar = [&](int s) { return bar0 + 8u * (2 * STAGES + s); };
@@ -513,9 +519,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       constexpr int ESZ = (EPI == EPI_STORE || EPI == EPI_GELU) ? 2 : 4;
       constexpr int CW = 128 / ESZ;
       constexpr int NCH = COLS / CW;
-      const uint32_t stg = staging + (uint32_t)half * (GEMM_STAGING_BYTES / 2);
+      // NB chunk buffers per column half, used in turn; a buffer is refilled once the store issued NB chunks ago has
+      // read it (NB = 1: the previous one)
+      constexpr int NB = gemm_staging_bufs(CG);
+      const uint32_t stg0 = staging + (uint32_t)half * (uint32_t)(NB * (GEMM_STAGING_BYTES / 2));
+      int chunk_no = 0;
       const int r = quad * 32 + lane;        // row of the tile this thread owns
-      const uint32_t row_addr = stg + (uint32_t)r * 128u;
       const uint32_t sw = (uint32_t)(r & 7);
       const bool issuer = (quad == 0 && lane == 0);
       const int bar_id = 1 + half;
@@ -528,7 +537,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         ptx::tc_fence_after();
         const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * ACC + half * COLS);
 #pragma unroll 1
-        for (int ch = 0; ch < NCH; ++ch) {
+        for (int ch = 0; ch < NCH; ++ch, ++chunk_no) {
+          const uint32_t stg = stg0 + (uint32_t)(chunk_no % NB) * (uint32_t)(GEMM_STAGING_BYTES / 2);
+          const uint32_t row_addr = stg + (uint32_t)r * 128u;
 #pragma unroll
           for (int part = 0; part < CW / 32; ++part) {
             uint32_t v[32];
@@ -564,8 +575,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 f[4 * i] *= gg.x; f[4 * i + 1] *= gg.y; f[4 * i + 2] *= gg.z; f[4 * i + 3] *= gg.w;
               }
             }
-            if (part == 0) {   // the previous chunk's TMA store must have drained the staging buffer
-              if (issuer) ptx::bulk_wait_read0();
+            if (part == 0) {   // the TMA store that last used this staging buffer must have read it
+              if (issuer) { if (NB == 2) ptx::bulk_wait_read1(); else ptx::bulk_wait_read0(); }
               ptx::named_bar_sync(bar_id, 128);
             }
             if (ESZ == 2) {

@@ -155,7 +155,7 @@ struct tsdp_ctx {
   int prof_live_count = -1;                   // live candidates of the forward being enqueued (-1: unknown, use the dense count)
   // CTA-pair GEMM (cta_group::2): clusters of two CTAs that fit the device at once (0: not usable), and whether it is used
   int pair_clusters = 0, pair_clusters_attn = 0;
-  int pair_mode = 0;                          // TSDP_GEMM_PAIR: 0 never, 1 when the tile count fills the pairs, 2 always
+  int pair_mode = 1;                          // TSDP_GEMM_PAIR: 0 never, 1 (default) by shape (use_pair_gemm), 2 wherever it applies
   bool dbg_armed = false, dbg_in_test_gemm = false;   // tsdp_debug_arm_gemm_timeout
   long long dbg_wait_cycles = 0;
   uint64_t cand_static = 0;                   // candidates the dense layout would have evaluated since the last reset
@@ -383,12 +383,15 @@ int launch_tc_pair_epi(tsdp_ctx* c, const CUtensorMap& ma, const CUtensorMap& mb
     default: return launch_tc_pair<EPI_F32>(c, ma, mb, mc, g, s);
   }
 }
-// Whether a GEMM of M rows and N columns runs on CTA pairs: wide outputs, and enough 256 x 256 tiles to occupy the pairs.
-bool use_pair_gemm(const tsdp_ctx* c, int M, int N) {
+// Whether a GEMM runs on CTA pairs: wide outputs, enough 256 x 256 tiles to occupy the pairs, and a long reduction.
+// Measured (45 056 - 54 400 rows): with K >= 1024 the pair form is 5 - 12 % faster on every shape (1.28 -> 1.43 PFLOP/s
+// at N 3072, K 1024); at K = 512 a tile has only 8 k-blocks, the epilogue and the hand-overs weigh as much as the
+// mainloop, and the two forms tie or the single-CTA one wins by a few per cent.
+bool use_pair_gemm(const tsdp_ctx* c, int M, int N, int K) {
   if (c->pair_mode == 0 || c->pair_clusters < 1 || N % 256 != 0) return false;
   if (c->pair_mode == 2) return true;
   const long long tiles = (long long)((M + 255) / 256) * (N / 256);
-  return tiles * 5 >= (long long)c->pair_clusters * 4;
+  return K >= 1024 && tiles * 5 >= (long long)c->pair_clusters * 4;
 }
 
 template <int BN>
@@ -479,7 +482,7 @@ int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, in
     c->last_error = "tensor-core GEMM needs K % 64 == 0 and N % 32 == 0";
     return TSDP_ERR_ARG;
   }
-  const bool pair = c->force_bn == 0 && use_pair_gemm(c, M, N);
+  const bool pair = c->force_bn == 0 && use_pair_gemm(c, M, N, K);
   const int BN = pair ? 256 : ((c->force_bn > 0 && N % c->force_bn == 0) ? c->force_bn : pick_bn(M, N, c->num_sms));
   CUtensorMap ma, mb, mc;
   int r;
@@ -646,7 +649,7 @@ int gemm_qkv_attn(tsdp_ctx* c, const void* A, const XfmrLayer& w, int M, int d, 
   int r;
   if ((r = get_map(c, A, 2, M, K, K, GEMM_BK, GEMM_BM, &ma)) != TSDP_OK) return r;
   const long long ptiles = (long long)((M + 255) / 256) * (N / BN);
-  const bool pair = c->pair_mode != 0 && c->pair_clusters_attn >= 1 && (c->pair_mode == 2 || ptiles * 5 >= (long long)c->pair_clusters_attn * 4);
+  const bool pair = c->pair_mode == 2 && c->pair_clusters_attn >= 1;      // K = d <= 1024 here: the single-CTA form is as fast
   if ((r = get_map(c, w.Wqkv_hm, 2, N, K, K, GEMM_BK, pair ? BN / 2 : BN, &mb)) != TSDP_OK) return r;
   prof_begin(c, s, c->prof_gemm_cat, 2.0 * gemm_rows_known(c, g) * N * K);
   if (pair) {
@@ -1502,6 +1505,9 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
         if (cudaOccupancyMaxActiveClusters(&ncl, fns[i], &lc) != cudaSuccess) { cudaGetLastError(); ncl = 0; }
         if (i == 0) c->pair_clusters = ncl; else c->pair_clusters_attn = ncl;
       }
+      if (getenv("TSDP_VERBOSE"))
+        fprintf(stderr, "tsdp_init: CTA-pair GEMM mode %d, %d / %d co-resident clusters of 2\n", c->pair_mode, c->pair_clusters,
+                c->pair_clusters_attn);
     }
   }
   for (int which = 0; which < 2; ++which) {

@@ -259,3 +259,31 @@ def test_fused_qkv_attention_kernel_against_fp64():
                  torch.tensor(bias, device="cuda"), M, 3 * d, d, 4, out)
         assert hp.max_rel(out.float().cpu().numpy().astype(np.float64), ref) < 1.5e-2, (M, d)
     smp.close()
+
+
+def test_gemm_pair_form_gives_the_same_bits_as_the_single_cta_form(monkeypatch):
+    """The two-CTA form of the tensor-core GEMM (tcgen05 cta_group::2: 256 x 256 tiles on clusters of two CTAs, each
+    staging half of the W tile) accumulates every output element in the same order as the single-CTA form, so every
+    epilogue must return identical bits; both are held to fp64 elsewhere.  Ragged M, odd and even numbers of
+    128-row blocks, short and long reductions."""
+    wl = hp.small_xfmr_workload(1)
+    shapes = [(129, 256, 64), (1000, 512, 128), (5000, 256, 1024), (33000, 1024, 512), (8200, 768, 2048)]
+    outs = {}
+    for mode in ("0", "2"):
+        monkeypatch.setenv("TSDP_GEMM_PAIR", mode)
+        smp, *_ = hp.setup(wl, max_B=1, max_K=1)
+        g = torch.Generator(device="cuda").manual_seed(3)
+        res = []
+        for (M, N, K) in shapes:
+            A = torch.randn(M, K, device="cuda", generator=g).to(torch.bfloat16)
+            W = (torch.randn(N, K, device="cuda", generator=g) / np.sqrt(K)).to(torch.bfloat16)
+            bias = torch.randn(N, device="cuda", generator=g)
+            for epi in (0, 1, 2, 3):
+                out = (torch.zeros(M, N, dtype=torch.bfloat16, device="cuda") if epi in (0, 1)
+                       else torch.full((M, N), 0.25, device="cuda"))
+                smp.gemm(A, W, bias, M, N, K, epi, out)
+                res.append(out.clone())
+        outs[mode] = res
+        smp.close()
+    for a, b in zip(outs["0"], outs["2"]):
+        assert torch.equal(a, b)

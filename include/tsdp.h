@@ -49,7 +49,8 @@ typedef enum {
   TSDP_ERR_TIMEOUT = 5,     /* a bounded wait inside a kernel expired                      */
   TSDP_ERR_NAN = 6,         /* non-finite value in a weight blob                           */
   TSDP_ERR_UNSUPPORTED = 7, /* architecture not built                                      */
-  TSDP_ERR_TOO_LARGE = 8    /* size beyond the capacity of tsdp_verify_commit_static       */
+  TSDP_ERR_TOO_LARGE = 8,   /* size beyond the capacity of tsdp_verify_commit_static       */
+  TSDP_ERR_OVERRUN = 9      /* tsdp_debug_check_guards found a buffer overrun              */
 } tsdp_status;
 
 enum { TSDP_ARCH_GAUSS = 0, TSDP_ARCH_MLP = 1, TSDP_ARCH_XFMR = 2, TSDP_ARCH_DIT = 3, TSDP_ARCH_UNET = 4,
@@ -252,6 +253,13 @@ int tsdp_denoise(tsdp_ctx* ctx, int which, const float* d_x, const int* h_tau, c
  * Test interface; synchronous. */
 int tsdp_gemm(tsdp_ctx* ctx, const void* d_A, const void* d_W, const float* d_bias, int M, int N, int K,
               int epi, void* d_out, void* cuda_stream);
+
+/* Memory check without a memory checker (test interface).  Every device buffer a context owns -- round state, network
+ * workspaces, weights, tables, plans -- is followed by 256 guard bytes holding a pattern.  This call waits for the
+ * device and verifies all of them: TSDP_OK, or TSDP_ERR_OVERRUN if some kernel wrote past the end of a buffer
+ * (tsdp_last_error names its size).  *h_checked (may be null) receives the number of buffers verified.
+ * Errors: ARG, CUDA, OVERRUN. */
+int tsdp_debug_check_guards(tsdp_ctx* ctx, int* h_checked);
 
 /* Exercise the time-out path of the tensor-core GEMM without hanging anything (test interface, precision 1).  Every
  * wait inside the kernel is bounded; normally the bound (about a second) is never reached.  After this call the NEXT

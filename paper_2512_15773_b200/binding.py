@@ -16,7 +16,7 @@ EXPORTS = ["tsdp_init", "tsdp_destroy", "tsdp_strerror", "tsdp_last_error", "tsd
            "tsdp_load_weights", "tsdp_set_schedule", "tsdp_sample_chunk", "tsdp_sample_chunk_host",
            "tsdp_round", "tsdp_denoise", "tsdp_gemm", "tsdp_gemm_timed", "tsdp_stats", "tsdp_reset_stats",
            "tsdp_kernel_launches", "tsdp_profile", "tsdp_profile_read", "tsdp_verify_commit_static", "tsdp_set_scheduler", "tsdp_set_progress",
-           "tsdp_sched_eval", "tsdp_serve", "tsdp_request_counts", "tsdp_process_reward", "tsdp_distill_loss", "tsdp_distill_step", "tsdp_debug_arm_gemm_timeout"]
+           "tsdp_sched_eval", "tsdp_serve", "tsdp_request_counts", "tsdp_process_reward", "tsdp_distill_loss", "tsdp_distill_step", "tsdp_debug_arm_gemm_timeout", "tsdp_debug_check_guards"]
 PROF_FAMILIES = ["gemm", "layernorm", "attention", "embed_head", "round", "small_net", "gemm_draft", "drafter_cluster", "accept", "verifier_cluster",
                  "layernorm_draft", "attention_draft", "embed_head_draft"]
 
@@ -88,6 +88,7 @@ def load_library():
     lib.tsdp_distill_loss.argtypes = [vp, fp, fp, i, u64, C.c_float, C.c_float, vp]
     lib.tsdp_distill_step.argtypes = [vp, fp, fp, i, u64, C.c_float, C.c_float, C.c_float, vp]
     lib.tsdp_debug_arm_gemm_timeout.argtypes = [vp, C.c_longlong]
+    lib.tsdp_debug_check_guards.argtypes = [vp, C.POINTER(C.c_int)]
     lib.tsdp_process_reward.argtypes = [vp, C.c_float, i, i, fp, i]
     lib.tsdp_stats.argtypes = [vp, C.POINTER(StatsT)]
     lib.tsdp_reset_stats.argtypes = [vp]
@@ -275,6 +276,12 @@ class Sampler:
     def gemm(self, d_A, d_W, d_bias, M, N, K, epi, d_out, stream=0):
         self._check(self.lib.tsdp_gemm(self.h, _ptr(d_A), _ptr(d_W), _ptr(d_bias), M, N, K, epi, _ptr(d_out),
                                        stream), "tsdp_gemm")
+
+    def check_guards(self):
+        """Verify the guard bytes behind every device buffer of the context; returns how many were checked."""
+        n = C.c_int(0)
+        self._check(self.lib.tsdp_debug_check_guards(self.h, C.byref(n)), "tsdp_debug_check_guards")
+        return n.value
 
     def arm_gemm_timeout(self, wait_cycles):
         self._check(self.lib.tsdp_debug_arm_gemm_timeout(self.h, int(wait_cycles)), "tsdp_debug_arm_gemm_timeout")

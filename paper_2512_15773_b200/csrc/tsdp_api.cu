@@ -112,6 +112,7 @@ struct tsdp_ctx {
   struct GraphRec { cudaGraphExec_t exec; int launches; };
   std::map<std::tuple<int, int>, GraphRec> graphs;
   std::map<std::tuple<const void*, int, int, int, int, int, int>, CUtensorMap> maps;
+  std::map<void*, size_t> guards;             // device buffer -> its size: the guard bytes sit right behind it
   EncodeTiledFn encode = nullptr;
   cudaStream_t cap_stream = nullptr;
   // persistent cluster drafter: usable for this configuration, shared memory per CTA, clusters that fit the GPU
@@ -181,14 +182,26 @@ namespace {
     }                                                                                             \
   } while (0)
 
+// Every device buffer of a context is followed by a 256-byte guard filled with a pattern; tsdp_debug_check_guards
+// verifies that no kernel wrote past a buffer's end (the stand-in for a memory checker on the kernels' index math).
+constexpr size_t GUARD_BYTES = 256;
+constexpr int GUARD_PATTERN = 0xA5;
+
 template <typename T>
 int dev_alloc(tsdp_ctx* c, std::vector<void*>& pool, T** p, size_t n) {
   void* q = nullptr;
-  CU_TRY(c, cudaMalloc(&q, n * sizeof(T) + 256));
-  CU_TRY(c, cudaMemset(q, 0, n * sizeof(T) + 256));
+  const size_t bytes = (n * sizeof(T) + 15) / 16 * 16;
+  CU_TRY(c, cudaMalloc(&q, bytes + GUARD_BYTES));
+  CU_TRY(c, cudaMemset(q, 0, bytes));
+  CU_TRY(c, cudaMemset(static_cast<uint8_t*>(q) + bytes, GUARD_PATTERN, GUARD_BYTES));
   pool.push_back(q);
+  c->guards[q] = bytes;
   *p = reinterpret_cast<T*>(q);
   return TSDP_OK;
+}
+void dev_free_pool(tsdp_ctx* c, std::vector<void*>& pool) {
+  for (void* q : pool) { c->guards.erase(q); cudaFree(q); }
+  pool.clear();
 }
 
 int alloc_bytes(tsdp_ctx* c, std::vector<void*>& pool, void** p, size_t bytes) {
@@ -1333,6 +1346,7 @@ const char* tsdp_strerror(int st) {
     case TSDP_ERR_NAN: return "non-finite value in weights";
     case TSDP_ERR_UNSUPPORTED: return "architecture not built";
     case TSDP_ERR_TOO_LARGE: return "size exceeds the capacity of the built-in scratch array";
+    case TSDP_ERR_OVERRUN: return "a kernel wrote past the end of a device buffer";
   }
   return "unknown status";
 }
@@ -1584,9 +1598,8 @@ void tsdp_destroy(tsdp_ctx* c) {
   cudaDeviceSynchronize();
   for (auto& g : c->graphs) cudaGraphExecDestroy(g.second.exec);
   for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
-  for (void* p : c->allocs) cudaFree(p);
-  for (int w = 0; w < 2; ++w)
-    for (void* p : c->net[w].allocs) cudaFree(p);
+  dev_free_pool(c, c->allocs);
+  for (int w = 0; w < 2; ++w) dev_free_pool(c, c->net[w].allocs);
   if (c->host_done) cudaFreeHost(c->host_done);
   if (c->sched_host) cudaFreeHost(c->sched_host);
   if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
@@ -1595,7 +1608,7 @@ void tsdp_destroy(tsdp_ctx* c) {
   if (c->ev_join) cudaEventDestroy(c->ev_join);
   if (c->ev_chunk0) cudaEventDestroy(c->ev_chunk0);
   if (c->ev_chunk1) cudaEventDestroy(c->ev_chunk1);
-  for (void* p : c->sched_allocs) cudaFree(p);
+  dev_free_pool(c, c->sched_allocs);
   delete c;
 }
 
@@ -1604,8 +1617,7 @@ static int load_sched_weights(tsdp_ctx* c, const float* blob, size_t n) {
   for (size_t i = 0; i < n; ++i)
     if (!std::isfinite(blob[i])) return TSDP_ERR_NAN;
   CU_TRY(c, cudaDeviceSynchronize());
-  for (void* p : c->sched_allocs) cudaFree(p);
-  c->sched_allocs.clear();
+  dev_free_pool(c, c->sched_allocs);
   c->sched_loaded = false;
   float* d = nullptr;
   if (dev_alloc(c, c->sched_allocs, &d, n)) return TSDP_ERR_CUDA;
@@ -1635,8 +1647,7 @@ int tsdp_load_weights(tsdp_ctx* c, int which, const float* blob, size_t n) {
   for (size_t i = 0; i < n; ++i)
     if (!std::isfinite(blob[i])) return TSDP_ERR_NAN;
   CU_TRY(c, cudaDeviceSynchronize());
-  for (void* p : net.allocs) cudaFree(p);
-  net.allocs.clear();
+  dev_free_pool(c, net.allocs);
   net.L.clear();
   net.loaded = false;
   // graphs captured with the old pointers are stale
@@ -1783,7 +1794,7 @@ int tsdp_load_weights(tsdp_ctx* c, int which, const float* blob, size_t n) {
     st |= dev_alloc(c, tmp_pool, &d_w2, 4 * dt * dt); st |= dev_alloc(c, tmp_pool, &d_b2, dt);
     st |= dev_alloc(c, tmp_pool, &d_wf, F * dt); st |= dev_alloc(c, tmp_pool, &d_bf, F);
     st |= dev_alloc(c, tmp_pool, &d_hid, (size_t)T * 4 * dt); st |= dev_alloc(c, tmp_pool, &d_tv, (size_t)T * dt);
-    auto free_tmp = [&]() { for (void* q : tmp_pool) cudaFree(q); };
+    auto free_tmp = [&]() { dev_free_pool(c, tmp_pool); };
     if (st) { free_tmp(); return TSDP_ERR_CUDA; }
     cudaMemcpy(d_w1, wt1T.data(), wt1T.size() * 4, cudaMemcpyHostToDevice); cudaMemcpy(d_b1, bt1, 4 * dt * 4, cudaMemcpyHostToDevice);
     cudaMemcpy(d_w2, wt2T.data(), wt2T.size() * 4, cudaMemcpyHostToDevice); cudaMemcpy(d_b2, bt2, dt * 4, cudaMemcpyHostToDevice);
@@ -1881,7 +1892,7 @@ int tsdp_load_weights(tsdp_ctx* c, int which, const float* blob, size_t n) {
     st |= dev_alloc(c, tmp_pool, &d_w2, d * d); st |= dev_alloc(c, tmp_pool, &d_b2, d);
     st |= dev_alloc(c, tmp_pool, &d_wm, mod_ld * d); st |= dev_alloc(c, tmp_pool, &d_bm, mod_ld);
     st |= dev_alloc(c, tmp_pool, &d_hid, (size_t)T * d); st |= dev_alloc(c, tmp_pool, &d_c, (size_t)T * d);
-    auto free_tmp = [&]() { for (void* q : tmp_pool) cudaFree(q); };
+    auto free_tmp = [&]() { dev_free_pool(c, tmp_pool); };
     if (st) { free_tmp(); return TSDP_ERR_CUDA; }
     cudaMemcpy(d_w1, wt1T.data(), d * d * 4, cudaMemcpyHostToDevice); cudaMemcpy(d_b1, bt1, d * 4, cudaMemcpyHostToDevice);
     cudaMemcpy(d_w2, wt2T.data(), d * d * 4, cudaMemcpyHostToDevice); cudaMemcpy(d_b2, bt2, d * 4, cudaMemcpyHostToDevice);
@@ -2391,6 +2402,27 @@ int tsdp_gemm(tsdp_ctx* c, const void* d_A, const void* d_W, const float* d_bias
   // test interface: operands are caller-owned and may be freed, so their tensor maps are not kept
   c->maps.clear();
   return check_status(c);
+}
+
+int tsdp_debug_check_guards(tsdp_ctx* c, int* h_checked) {
+  if (!c) return TSDP_ERR_ARG;
+  CU_TRY(c, cudaSetDevice(c->cfg.device));
+  CU_TRY(c, cudaDeviceSynchronize());
+  uint8_t tail[GUARD_BYTES];
+  int n = 0;
+  for (const auto& g : c->guards) {
+    CU_TRY(c, cudaMemcpy(tail, static_cast<const uint8_t*>(g.first) + g.second, GUARD_BYTES, cudaMemcpyDeviceToHost));
+    for (size_t i = 0; i < GUARD_BYTES; ++i)
+      if (tail[i] != GUARD_PATTERN) {
+        c->last_error = "guard bytes behind a device buffer of " + std::to_string(g.second) + " bytes were overwritten (offset " +
+                        std::to_string(i) + ")";
+        if (h_checked) *h_checked = n;
+        return TSDP_ERR_OVERRUN;
+      }
+    ++n;
+  }
+  if (h_checked) *h_checked = n;
+  return TSDP_OK;
 }
 
 int tsdp_debug_arm_gemm_timeout(tsdp_ctx* c, long long wait_cycles) {

@@ -135,3 +135,31 @@ def test_compacted_rounds_give_the_same_bits_as_dense_rounds(arch, monkeypatch):
     assert np.array_equal(st_d["hist_accepted"], st_c["hist_accepted"])
     assert st_d["cand_computed"] == st_d["cand_dense"] == st_c["cand_dense"]
     assert st_c["cand_computed"] == st_c["base_evals"] < st_c["cand_dense"]
+
+
+def test_no_kernel_writes_past_a_buffer():
+    """Every device buffer of a context is followed by guard bytes; after whole chunks on every architecture pairing
+    (ragged batch sizes, compacted rounds, continuous batching with buffers that had to grow, the cluster kernels at
+    batch 1) all guards must be intact."""
+    cases = [
+        (hp.small_xfmr_workload(1, d=256, heads=4, layers=2, dd=128, dlayers=2, H=16, A=7, To=2, Do=16, gamma=0.05), 37, 6),
+        (hp.small_xfmr_workload(1, d=128, heads=4, layers=2, dd=128, dlayers=1, H=7, A=3, To=3, Do=5, gamma=0.05), 5, 4),
+        (dict(inputs.WORKLOADS["pusht_xfmr"], precision=1), 1, 8),
+        (dict(H=10, A=4, To=16, Do=8, T=100, precision=1, gamma=0.05,
+              base=dict(arch="dit", layers=2, d=128, heads=4), draft=dict(arch="dit", layers=1, d=128, heads=2)), 9, 5),
+        (dict(H=16, A=10, To=2, Do=24, T=100, precision=1, gamma=0.05,
+              base=dict(arch="unet", layers=2, d=128, heads=8, temb=32), draft=dict(arch="xfmr", layers=1, d=128, heads=4)), 11, 5),
+        (dict(inputs.WORKLOADS["toy_mlp"]), 3, 4),
+    ]
+    for wl, B, K in cases:
+        smp, *_ = hp.setup(wl, max_B=B, max_K=K)
+        obs = torch.tensor(inputs.make_obs(11, B, wl["To"], wl["Do"]), dtype=torch.float32, device="cuda")
+        out = torch.zeros(B, wl["H"], wl["A"], device="cuda")
+        smp.sample_chunk(obs, B, K, hp.accept_t(), 3, out)
+        N = 2 * B + 3
+        obs2 = torch.tensor(inputs.make_obs(12, N, wl["To"], wl["Do"]), dtype=torch.float32, device="cuda")
+        out2 = torch.zeros(N, wl["H"], wl["A"], device="cuda")
+        smp.serve(obs2, N, B, K, hp.accept_t(bonus=0), 4, out2)
+        assert smp.check_guards() >= 20
+        assert torch.isfinite(out).all() and torch.isfinite(out2).all()
+        smp.close()

@@ -113,3 +113,55 @@ def test_robomimic_unet_at_full_width_sampled_candidates():
         ref = base(x[n].astype(np.float64), int(tau[n]), obs[n])
         assert hp.max_rel(got[n], ref) < 2e-2, n
     smp.close()
+
+
+def _round_sampled(wl, B, K, seed, t0s, envs, acc=None):
+    """One round at full width from random states; the listed environments are recomputed by the oracle."""
+    acc = acc or hp.accept_t()
+    smp, S, base, draft = hp.setup(wl, max_B=B, max_K=K)
+    D = wl["H"] * wl["A"]; shape = (wl["H"], wl["A"])
+    obs = inputs.make_obs(50, B, wl["To"], wl["Do"])
+    noise = spec.PhiloxNoise(seed)
+    rng = np.random.default_rng(seed)
+    x0 = rng.normal(size=(B, D)).astype(np.float32)
+    dx = torch.tensor(x0, device="cuda"); dobs = torch.tensor(obs, dtype=torch.float32, device="cuda")
+    h_t = np.array(t0s, dtype=np.int32)
+    d_xt = torch.zeros(B, K + 1, D, device="cuda"); d_mh = torch.zeros(B, K, D, device="cuda")
+    d_eps = torch.zeros(B, K + 1, D, device="cuda"); d_la = torch.zeros(B, K, device="cuda")
+    h_j = np.zeros(B, dtype=np.int32)
+    smp.round(dobs, B, K, acc, seed, dx, h_t, d_xt, d_mh, d_eps, d_la, h_j)
+    xt, mh, eps, la = d_xt.cpu().numpy(), d_mh.cpu().numpy(), d_eps.cpu().numpy(), d_la.cpu().numpy()
+    x_new = dx.cpu().numpy()
+    checked = 0
+    for b in envs:
+        xo, to, d = spec.spec_round(S, base, draft, noise, b, obs[b], x0[b].astype(np.float64).reshape(shape), int(t0s[b]), K,
+                                    hp.oracle_accept(acc))
+        g = dict(xt=xt[b], mh=mh[b], eps=eps[b], la=la[b], j=int(h_j[b]), t_new=int(h_t[b]), x_new=x_new[b],
+                 t_oracle=to, x_oracle=xo)
+        checked += hp.check_round_env(S, noise, hp.oracle_accept(acc), b, int(t0s[b]), K, d, g, 2e-2, 3e-3)
+    assert smp.check_guards() > 0
+    smp.close()
+    return checked
+
+
+def test_vla_shaped_round_at_full_width_sampled_environments():
+    """A whole speculative round of the VLA-scale pairing at full width (d = 1024 / 512, 50 tokens, 256 context tokens,
+    K = 16; two base blocks and one drafter block so that the oracle stays affordable): compacted candidate list with a
+    finished environment and short windows in it, the two-CTA GEMM on the K >= 1024 shapes, context cross-attention
+    grouped by slot through the plan's slot offsets."""
+    wl = dict(inputs.WORKLOADS["vla_dit"])
+    wl["base"] = dict(wl["base"], layers=2); wl["draft"] = dict(wl["draft"], layers=1)
+    B, K = 12, 16
+    t0s = [99, 50, 7, 0, -1, 30, 3, 99, 12, 64, 1, 80]
+    checked = _round_sampled(wl, B, K, 17, t0s, envs=(0, 2, 3))
+    assert checked >= 2
+
+
+def test_robomimic_shaped_round_at_full_width_sampled_environments():
+    """The conv UNet at its real channel widths verified against the 4-block transformer drafter's drafts, one round,
+    ragged windows and a finished environment; two environments through the oracle."""
+    wl = dict(inputs.WORKLOADS["robomimic_unet"])
+    B, K = 10, 8
+    t0s = [99, 40, 3, -1, 0, 70, 5, 99, 20, 1]
+    checked = _round_sampled(wl, B, K, 23, t0s, envs=(1, 2))
+    assert checked >= 1

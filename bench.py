@@ -436,6 +436,10 @@ def run_ours(args):
             others["robomimic_unet_B32_K8_frozen_target_drafts"] = side_record("robomimic_unet", 32, 8, local, acc, 3, 6, peaks,
                                                                                  vanilla_steps=0, profile=False, drafter="frozen")
             others["vla_dit_B64_K16"] = side_record("vla_dit", 64, 16, local, acc, 1, 2, peaks, vanilla_steps=1)
+            others["vla_dit_B64_K16_frozen_target_drafts"] = side_record("vla_dit", 64, 16, local, acc, 1, 2, peaks, vanilla_steps=0,
+                                                                           profile=False, drafter="frozen")
+            others["serving_xfmr_B256_K10_frozen_target_drafts"] = side_record("serving_xfmr", 256, 10, local, acc, 2, 4, peaks,
+                                                                                 vanilla_steps=0, profile=False, drafter="frozen")
         cpu = cpu_baseline(wl, budget_s=args.cpu_seconds) if world == 1 else None
         cand = reduce_sum([st["base_evals"], st["cand_computed"], st["cand_dense"]], 1)
         result.update(

@@ -18,9 +18,12 @@ Pin status (what checks each part against something other than itself):
                         first-rejection enumeration, drafter==base == vanilla,
                         KS test against the analytic marginal of the sampler.
   nets.py     parity unpinned against the paper (its trained networks and exact
-              layer layout are not published); pinned only by structural
-              invariants (causality, zero-weight behaviour, a hand-computed
-              1-token case) -- see the function headers.
+              layer layout are not published); the wiring of the library's own
+              architecture definition IS pinned: attention against a library routine
+              (scale, head partition, causal mask), a decoder block, an adaptive-LayerNorm
+              block and a 2-level conv UNet element by element in plain loops, the
+              modulation slices and FiLM halves through closed forms, plus structural
+              invariants (causality, zero-weight behaviour) -- tests/test_oracle_nets*.py.
   sched.py    parity unpinned against the paper (Sec. 3.3 names the three input streams, the
               separate encoders, the aggregating MLP and the five outputs, but no sizes, weights
               or ranges); pinned by structure: zero network, output ranges, stream separation,
@@ -30,6 +33,9 @@ Pin status (what checks each part against something other than itself):
   distill.py  pinned  : zero for equal networks, the closed form for a constant output offset
                         (with the printed values c_50 = 0.2145, c_1 = 1.735 of the linear schedule),
                         linearity in (lambda1, lambda2), the Gaussian-overlap integral.
+                        Gradient step on the Gaussian drafter: central finite differences of that
+                        loss (each term alone and the sum), zero gradient at the base's parameters,
+                        monotone descent to them.
   spec.FrozenTargetDraft  parity unpinned against the prior work that Sec. 2.2 cites (only named
               there); pinned by: first draft exact, K = 1 == vanilla, the Gaussian chain's marginal.
   sigma_scale parity unpinned against the paper (formula not given there).

@@ -1,14 +1,15 @@
 """The denoisers eps = M(x, tau; obs) in numpy fp64: closed-form Gaussian toy, MLP, transformer, DiT,
 conv UNet.
 
-The paper states only the block counts ("DP consists of 8 Transformer blocks while the drafter
-contains only one", Sec. 4) and that the drafter has the same input-output interface and shares
-the encoder and scheduler (Sec. 3.2 "Draft Model Training").  Everything below that is more
+The paper gives only the block counts (eight transformer blocks for the base policy, a single one for
+the drafter, Sec. 4) and says that the drafter has the same input-output interface and shares the
+encoder and scheduler (Sec. 3.2 "Draft Model Training").  Everything below that is more
 specific than that is this library's own architecture definition; parity with the paper's trained
-networks is UNPINNED (no weights or layer layout are published).  The pins that exist are
-structural: causality of self-attention (bidirectionality for the adaLN transformer, whose
-blocks reduce to the identity with zero gates), independence of candidates, zero-head => zero output,
-and the closed-form Gaussian denoiser against the analytic posterior mean.
+networks is UNPINNED (no weights or layer layout are published).  What is pinned is the wiring of that
+definition: attention against a library routine and plain-loop restatements of a decoder block, an
+adaptive-LayerNorm block and a 2-level UNet, closed forms for the modulation slices and the FiLM halves,
+and structural invariants (causality, bidirectionality of the adaLN transformer, independence of candidates,
+zero-head => zero output, the closed-form Gaussian denoiser against the analytic posterior mean).
 
 Parameters are dicts of float64 arrays produced by the seeded input generators; a linear layer
 y = x W + b stores W as [in, out].

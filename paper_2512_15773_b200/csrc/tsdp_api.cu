@@ -1925,7 +1925,6 @@ int tsdp_load_weights(tsdp_ctx* c, int which, const float* blob, size_t n) {
       if ((r = up_f32(&w.ln1_b, d))) return r;
       if ((r = up_wT(&w.Wqkv, cur, d, 3 * d))) return r;
       if (fused_attn_ok(cfg, net.cfg)) {      // the same matrix and bias, output features head-major
-        const size_t heads = net.cfg.heads;
         std::vector<float> wp(d * 3 * d), bp(3 * d);
         const float* bsrc = cur + d * 3 * d;
         for (size_t o = 0; o < 3 * d; ++o) {
@@ -1933,7 +1932,6 @@ int tsdp_load_weights(tsdp_ctx* c, int which, const float* blob, size_t n) {
           for (size_t i = 0; i < d; ++i) wp[i * 3 * d + on] = cur[i * 3 * d + o];
           bp[on] = bsrc[o];
         }
-        (void)heads;
         if ((r = up_wT(&w.Wqkv_hm, wp.data(), d, 3 * d))) return r;
         if (dev_alloc(c, net.allocs, &w.bqkv_hm, 3 * d)) return TSDP_ERR_CUDA;
         CU_TRY(c, cudaMemcpy(w.bqkv_hm, bp.data(), 3 * d * sizeof(float), cudaMemcpyHostToDevice));

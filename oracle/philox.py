@@ -1,7 +1,7 @@
 """Philox4x32-10 counter-based generator and the noise/uniform streams built on it.
 
-The paper fixes seeds but names no generator (Sec. 4 "fixed seeds"; Sec. 3.2 says the
-rollout "retains the random noise realizations").  The reading used here: every random
+The paper fixes seeds but names no generator (Sec. 4 runs with fixed seeds; Sec. 3.2 keeps the
+noise realisations of the drafter's rollout for the verification).  The reading used here: every random
 number is a pure function of (seed, environment, stream, timestep, element), never of
 the round structure, so a draft at timestep tau and a base step at tau draw the same
 xi_tau.  Generator: Philox4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw, SC'11),

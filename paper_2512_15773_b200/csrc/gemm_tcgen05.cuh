@@ -1,7 +1,7 @@
 // bf16 GEMM for sm_100a:  C[M,N] = A[M,K] * W[N,K]^T (+ bias, activation, residual), fp32 accumulate.
 //
-// This is the dense contraction of the verification forward (Sec. 3.2, "evaluating the frozen
-// target model on all elements of C in a single batched forward pass"): every linear layer of the
+// This is the dense contraction of the verification forward (Sec. 3.2, "Verification of Speculative
+// Drafts": the frozen base model sees every candidate of the set C in one batched pass): every linear layer of the
 // base transformer applied to all (K+1)*B candidate latents at once.
 //
 // Structure (one persistent CTA per SM, 128 x BN output tiles, BK = 64):

@@ -23,6 +23,7 @@
 #include "drafter_cluster.cuh"
 #include "sched_kernel.cuh"
 #include "dit_kernels.cuh"
+#include "ctx_attn_tcgen05.cuh"
 #include "unet_kernels.cuh"
 #include "xattn_fold.cuh"
 #include "draft_tail.cuh"
@@ -134,6 +135,7 @@ struct tsdp_ctx {
   std::vector<float> lat_ring;
   size_t lat_pos = 0, lat_n = 0;
   bool pdl = true;                            // programmatic dependent launch between the kernels of a round
+  int tc_attn = 1;                            // context cross-attention on tcgen05: 0 never (TSDP_NO_TC_ATTN), 1 large groups, 2 always (TSDP_TC_ATTN=2)
   bool async_bcast = true;                    // cluster kernel: st.async + mbarrier stage hand-over (TSDP_NO_ASYNC_BCAST unset)
   bool dc_ok = false;
   int dc_smem = 0, dc_max_clusters = 0;
@@ -854,8 +856,28 @@ int cross_attn_ctx_launch(tsdp_ctx* c, const Net& n, const T* q2, T* out, const 
   const int dh = d / heads, M = n_cand * H;
   const long long ld_kv = (long long)L * 2 * d;
   const T* kv = reinterpret_cast<const T*>(n.kv_obs);
-  prof_begin(c, s, 2, 0.0);
   bool done = false;
+  if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+    // 64-wide heads and groups of at least two 128-row tiles (the verification forward: all candidates of a slot share
+    // the keys / values a CTA fetched): both products on the 5th-generation tensor cores (ctx_attn_tcgen05.cuh).
+    // Measured on the VLA-scale workload: 7 % less attention time than the mma.sync kernel there, but slower for the
+    // drafter's single 50-row group per CTA, where fetching and re-laying-out K / V dominates; tc_attn = 2 forces it.
+    if (c->tc_attn && (cm.C * H >= 256 || c->tc_attn == 2) && dh == 64 && Tc % 32 == 0 && Tc <= 256 && n_cand % cm.C == 0 && d % 8 == 0) {
+      const int slots = n_cand / cm.C, rows = cm.C * H;
+      CUtensorMap mq, mkv;
+      int r;
+      if ((r = get_map(c, q2, 2, M, d, d, 64, 128, &mq)) != TSDP_OK) return r;
+      if ((r = get_map(c, kv, 2, (int)(c->items_cap * (size_t)Tc), L * 2 * d, L * 2 * d, 64, Tc, &mkv)) != TSDP_OK) return r;
+      prof_begin(c, s, 2, 0.0);
+      TSDP_LAUNCH(c, (cross_attn_ctx_tc_kernel), slots * heads, CXT_THREADS, CXT_SMEM_BYTES, s, mq, mkv, reinterpret_cast<__nv_bfloat16*>(out),
+                  layer * 2 * d, cm, rows, d, heads, Tc, c->live_slot_start, H, c->status);
+      prof_end(c, s);
+      c->launches_per_round_tmp++;
+      CU_TRY(c, cudaGetLastError());
+      return TSDP_OK;
+    }
+  }
+  prof_begin(c, s, 2, 0.0);
   if constexpr (std::is_same<T, __nv_bfloat16>::value) {
     if (Tc % 16 == 0 && (dh == 32 || dh == 64 || dh == 128) && n_cand % cm.C == 0) {
       const int slots = n_cand / cm.C, rows = cm.C * H;
@@ -1378,6 +1400,7 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   c->pdl = getenv("TSDP_NO_PDL") == nullptr;
   c->async_bcast = getenv("TSDP_NO_ASYNC_BCAST") == nullptr;
   c->compact = getenv("TSDP_NO_COMPACT") == nullptr;
+  c->tc_attn = getenv("TSDP_NO_TC_ATTN") != nullptr ? 0 : (getenv("TSDP_TC_ATTN") != nullptr ? atoi(getenv("TSDP_TC_ATTN")) : 1);
   if (const char* fb = getenv("TSDP_GEMM_BN")) {      // tuning aid: one tile width for every GEMM it divides
     const int v = atoi(fb);
     if (v == 32 || v == 64 || v == 128 || v == 256) c->force_bn = v;
@@ -1555,6 +1578,7 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   INIT_TRY(cudaFuncSetAttribute(cross_attn_ctx_mma_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, cx_smem_bytes<32>(256)));
   INIT_TRY(cudaFuncSetAttribute(cross_attn_ctx_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, cx_smem_bytes<64>(256)));
   INIT_TRY(cudaFuncSetAttribute(cross_attn_ctx_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, cx_smem_bytes<128>(256)));
+  INIT_TRY(cudaFuncSetAttribute(cross_attn_ctx_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, CXT_SMEM_BYTES));
   INIT_TRY(cudaFuncSetAttribute(xfold_build_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
   INIT_TRY(cudaFuncSetAttribute(xattn_fold_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)xf_smem_bytes(128, XF_MAXN)));
   INIT_TRY(cudaFuncSetAttribute(xattn_fold_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)xf_smem_bytes(256, XF_MAXN)));

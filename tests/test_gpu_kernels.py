@@ -119,19 +119,26 @@ def test_transformer_denoiser_bf16_without_the_cross_attention_fold(shape, monke
 
 
 @pytest.mark.parametrize("precision,tol", [(0, 1e-4), (1, 2e-2)])
-@pytest.mark.parametrize("shape", ["small", "wide"])
-def test_dit_denoiser(precision, tol, shape):
+@pytest.mark.parametrize("shape", ["small", "wide", "tc"])
+def test_dit_denoiser(precision, tol, shape, monkeypatch):
     """Adaptive-LayerNorm transformer against the oracle: gated residual epilogue, modulated LayerNorm,
     bidirectional self-attention, cross-attention to the context tokens."""
     rng = np.random.default_rng(3)
+    if shape == "tc":
+        monkeypatch.setenv("TSDP_TC_ATTN", "2")      # single-candidate groups too (the default keeps those on mma.sync)
     if shape == "small":
         # 7 tokens, 12 context tokens (not a multiple of 16: the scalar context attention), head width 32
         wl = dict(H=7, A=3, To=12, Do=5, T=100, precision=precision, gamma=1.0,
                   base=dict(arch="dit", layers=2, d=128, heads=4), draft=dict(arch="dit", layers=1, d=256, heads=2))
-    else:
+    elif shape == "wide":
         # 50 tokens, 48 context tokens (tensor-core context attention over a ragged 64-key chunk), head widths 64 / 128
         wl = dict(H=50, A=14, To=48, Do=24, T=100, precision=precision, gamma=1.0,
                   base=dict(arch="dit", layers=2, d=256, heads=4), draft=dict(arch="dit", layers=1, d=128, heads=1))
+    else:
+        # 64-wide heads and 96 context tokens: in bf16 the context attention runs on tcgen05 (S = Q K^T and O = P V in
+        # tensor memory, one and a half 64-key atoms)
+        wl = dict(H=50, A=14, To=96, Do=24, T=100, precision=precision, gamma=1.0,
+                  base=dict(arch="dit", layers=2, d=256, heads=4), draft=dict(arch="dit", layers=1, d=512, heads=8))
     N = 9
     smp, S, base, draft = hp.setup(wl, max_B=N, max_K=1)
     x = rng.normal(size=(N, wl["H"], wl["A"])).astype(np.float32)

@@ -7,11 +7,12 @@
 // re-laid out in shared memory as V^T so that both products take K-major operands.  Then, per tile of 128 query rows:
 //   TMA      Q tile [128 x 64] -> shared memory (double-buffered, the next tile is fetched during this one)
 //   MMA 1    S = Q K^T      [128 x Tc], fp32, in tensor memory                      (tcgen05.mma, one issuing thread)
-//   softmax  thread r of warps 0-3 owns query row r: two passes over its Tc scores straight from tensor memory
-//            (tcgen05.ld), p = exp2((s - max) log2(e) / sqrt(dh)), row sum kept in a register, P as bf16 into shared
-//            memory in the 128-byte-swizzled K-major layout the second product reads
+//   softmax  two threads per query row (warps w and w + 4 share tensor-memory lane quadrant w and split the Tc
+//            columns): two passes over the scores straight from tensor memory (tcgen05.ld), row maximum and row sum
+//            exchanged through shared memory, p = exp2((s - max) log2(e) / sqrt(dh)), P as bf16 into shared memory
+//            in the 128-byte-swizzled K-major layout the second product reads
 //   MMA 2    O = P V        [128 x 64], fp32, in tensor memory
-//   epilogue the same thread reads its row of O, scales by 1 / row sum, stores 128 bytes of bf16.
+//   epilogue the same two threads read half a row of O each, scale by 1 / row sum, store 64 bytes of bf16 each.
 // No online softmax: all Tc <= 256 scores of a row are in tensor memory at once.  Rows past the group's end are
 // computed on whatever the tile fetched (other rows of the buffer, or zeros past its end) and never stored.
 // Every mbarrier wait is bounded; on expiry the CTA records TSDP_ERR_TIMEOUT (5) in `status`, frees its tensor
@@ -22,13 +23,14 @@
 
 namespace tsdp {
 
-constexpr int CXT_THREADS = 160;                 // warps 0-3: softmax / epilogue (row = thread), warp 4: TMA + MMA issue
+constexpr int CXT_THREADS = 288;                 // warps 0-7: softmax / epilogue (two threads per row), warp 8: TMA + MMA issue
 constexpr int CXT_Q_BYTES = 128 * 128;           // one Q tile: 128 rows x 64 bf16
 constexpr int CXT_OFF_K = 2 * CXT_Q_BYTES;       // keys [Tc x 64], up to 32 KB
 constexpr int CXT_OFF_VT = CXT_OFF_K + 256 * 128;        // V^T as Tc/64 atoms of [64 x 64]
 constexpr int CXT_OFF_P = CXT_OFF_VT + 256 * 128;        // P as Tc/64 atoms of [128 x 64]; first used as the V staging tile
 constexpr int CXT_OFF_BAR = CXT_OFF_P + 4 * CXT_Q_BYTES;
-constexpr int CXT_SMEM_BYTES = CXT_OFF_BAR + 128 + 1024;  // + alignment slack
+constexpr int CXT_OFF_X = CXT_OFF_BAR + 128;              // row maxima and row sums of the two column halves: float [2][2][128]
+constexpr int CXT_SMEM_BYTES = CXT_OFF_X + 2048 + 1024;   // + alignment slack
 
 __global__ void __launch_bounds__(CXT_THREADS, 1)
 cross_attn_ctx_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKV,
@@ -44,11 +46,11 @@ cross_attn_ctx_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     ptx::mbar_init(bar_kv, 1); ptx::mbar_init(bar_q0, 1); ptx::mbar_init(bar_q0 + 8, 1);
-    ptx::mbar_init(bar_s, 1); ptx::mbar_init(bar_p, 128); ptx::mbar_init(bar_o, 1); ptx::mbar_init(bar_or, 128);
+    ptx::mbar_init(bar_s, 1); ptx::mbar_init(bar_p, 256); ptx::mbar_init(bar_o, 1); ptx::mbar_init(bar_or, 256);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 4) { ptx::tmem_alloc(tmem_slot, 512); ptx::tmem_relinquish(); }
+  if (warp == 8) { ptx::tmem_alloc(tmem_slot, 512); ptx::tmem_relinquish(); }
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
@@ -75,7 +77,7 @@ cross_attn_ctx_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
 
   if (n_tiles > 0) {
     // ---- keys, values (into the staging tile) and the first Q tile
-    if (warp == 4 && lane == 0) {
+    if (warp == 8 && lane == 0) {
       const int y = item_of(cm.item, b) * Tc;
       ptx::mbar_expect_tx(bar_kv, 2 * kv_bytes);
       ptx::tma_load_2d(sK, &tmKV, kv_off + hd * 64, y, bar_kv);
@@ -106,7 +108,7 @@ cross_attn_ctx_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
   }
 
   if (ok && n_tiles > 0) {
-    if (warp == 4) {
+    if (warp == 8) {
       if (lane == 0) {
         const uint32_t idesc1 = umma_idesc_bf16(Tc, 128), idesc2 = umma_idesc_bf16(64, 128);
         for (int i = 0; i < n_tiles; ++i) {
@@ -134,66 +136,71 @@ cross_attn_ctx_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         }
       }
     } else {
-      const int r = warp * 32 + lane;                       // query row of the tile; tensor-memory lane
-      const uint32_t t_s = tmem_base + ((uint32_t)(warp * 32) << 16);
+      const int quad = warp & 3, half = warp >> 2;          // tensor-memory lane quadrant; which half of the columns
+      const int r = quad * 32 + lane;                       // query row of the tile; tensor-memory lane
+      const uint32_t t_s = tmem_base + ((uint32_t)(quad * 32) << 16);
       const float c = 1.4426950408889634f * 0.125f;         // log2(e) / sqrt(64)
       uint8_t* prow = gbase + CXT_OFF_P + r * 128;
       const uint32_t sw = (uint32_t)(r & 7);
+      float* xmax = reinterpret_cast<float*>(gbase + CXT_OFF_X);       // [2][128]
+      float* xsum = xmax + 256;                                       // [2][128]
+      const int cbeg = half * (Tc / 2), cend = cbeg + Tc / 2;           // Tc / 2 is a multiple of 16
+      const int pair_bar = 1 + quad;                                  // the two warps of a quadrant
       for (int i = 0; i < n_tiles; ++i) {
-        if (!ptx::mbar_wait_warp(bar_s, (uint32_t)(i & 1))) { ok = false; break; }
+        ok = ptx::named_bar_and(pair_bar, 64, ptx::mbar_wait_warp(bar_s, (uint32_t)(i & 1)));
+        if (!ok) break;
         ptx::tc_fence_after();
         float mx = -INFINITY;
-        for (int c0 = 0; c0 < Tc; c0 += 32) {
-          uint32_t v[32];
-          ptx::tmem_ld32(t_s + (uint32_t)c0, v);
+        for (int c0 = cbeg; c0 < cend; c0 += 16) {
+          uint32_t v[16];
+          ptx::tmem_ld16(t_s + (uint32_t)c0, v);
           ptx::tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(v[j]));
+          for (int j = 0; j < 16; ++j) mx = fmaxf(mx, __uint_as_float(v[j]));
         }
+        xmax[half * 128 + r] = mx;
+        ptx::named_bar_sync(pair_bar, 64);
+        mx = fmaxf(mx, xmax[(half ^ 1) * 128 + r]);
         const float mc = mx * c;
         float sum = 0.f;
-        for (int c0 = 0; c0 < Tc; c0 += 32) {
-          uint32_t v[32];
-          ptx::tmem_ld32(t_s + (uint32_t)c0, v);
+        for (int c0 = cbeg; c0 < cend; c0 += 16) {
+          uint32_t v[16];
+          ptx::tmem_ld16(t_s + (uint32_t)c0, v);
           ptx::tmem_ld_wait();
-          float p[32];
+          float p[16];
 #pragma unroll
-          for (int j = 0; j < 32; ++j) { p[j] = exp2f(__fmaf_rn(__uint_as_float(v[j]), c, -mc)); sum += p[j]; }
+          for (int j = 0; j < 16; ++j) { p[j] = exp2f(__fmaf_rn(__uint_as_float(v[j]), c, -mc)); sum += p[j]; }
           uint8_t* dst = prow + (c0 >> 6) * CXT_Q_BYTES;
           const uint32_t ch0 = (uint32_t)((c0 & 63) >> 3);
 #pragma unroll
-          for (int j = 0; j < 4; ++j)
+          for (int j = 0; j < 2; ++j)
             *reinterpret_cast<uint4*>(dst + (((ch0 + j) ^ sw) << 4)) =
                 make_uint4(pack_bf16x2(p[8 * j], p[8 * j + 1]), pack_bf16x2(p[8 * j + 2], p[8 * j + 3]),
                            pack_bf16x2(p[8 * j + 4], p[8 * j + 5]), pack_bf16x2(p[8 * j + 6], p[8 * j + 7]));
         }
+        xsum[half * 128 + r] = sum;
         ptx::fence_async_smem();                            // P is read by the tensor core (async proxy)
         ptx::tc_fence_before();                             // and the scores have been read: S may be overwritten
         ptx::mbar_arrive(bar_p);
-        if (!ptx::mbar_wait_warp(bar_o, (uint32_t)(i & 1))) { ok = false; break; }
+        ok = ptx::named_bar_and(pair_bar, 64, ptx::mbar_wait_warp(bar_o, (uint32_t)(i & 1)));     // also publishes the partner's row sum
+        if (!ok) break;
         ptx::tc_fence_after();
-        uint32_t o0[32], o1[32];
-        ptx::tmem_ld32(t_s + 256u, o0);
-        ptx::tmem_ld32(t_s + 288u, o1);
+        sum += xsum[(half ^ 1) * 128 + r];
+        uint32_t o0[32];
+        ptx::tmem_ld32(t_s + 256u + (uint32_t)(half * 32), o0);
         ptx::tmem_ld_wait();
         ptx::tc_fence_before();
         ptx::mbar_arrive(bar_or);                           // O may be overwritten by the next tile's second product
         const int row = i * 128 + r;
         if (row < rows) {
           const float inv = 1.0f / sum;
-          uint4* o = reinterpret_cast<uint4*>(out + (size_t)(row0 + row) * d + hd * 64);
+          uint4* o = reinterpret_cast<uint4*>(out + (size_t)(row0 + row) * d + hd * 64 + half * 32);
 #pragma unroll
           for (int j = 0; j < 4; ++j)
             o[j] = make_uint4(pack_bf16x2(__uint_as_float(o0[8 * j]) * inv, __uint_as_float(o0[8 * j + 1]) * inv),
                               pack_bf16x2(__uint_as_float(o0[8 * j + 2]) * inv, __uint_as_float(o0[8 * j + 3]) * inv),
                               pack_bf16x2(__uint_as_float(o0[8 * j + 4]) * inv, __uint_as_float(o0[8 * j + 5]) * inv),
                               pack_bf16x2(__uint_as_float(o0[8 * j + 6]) * inv, __uint_as_float(o0[8 * j + 7]) * inv));
-#pragma unroll
-          for (int j = 0; j < 4; ++j)
-            o[4 + j] = make_uint4(pack_bf16x2(__uint_as_float(o1[8 * j]) * inv, __uint_as_float(o1[8 * j + 1]) * inv),
-                                  pack_bf16x2(__uint_as_float(o1[8 * j + 2]) * inv, __uint_as_float(o1[8 * j + 3]) * inv),
-                                  pack_bf16x2(__uint_as_float(o1[8 * j + 4]) * inv, __uint_as_float(o1[8 * j + 5]) * inv),
-                                  pack_bf16x2(__uint_as_float(o1[8 * j + 6]) * inv, __uint_as_float(o1[8 * j + 7]) * inv));
         }
       }
     }
@@ -206,7 +213,7 @@ cross_attn_ctx_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
-  if (warp == 4) ptx::tmem_dealloc(tmem_base, 512);
+  if (warp == 8) ptx::tmem_dealloc(tmem_base, 512);
 }
 
 }  // namespace tsdp

@@ -27,6 +27,13 @@
  * wherever the output width allows -- a tuning aid; results do not depend on it.
  * TSDP_GEMM_BN = 32 | 64 | 128 | 256 (read by tsdp_init) forces that tile width on every tensor-core GEMM whose
  * output width it divides -- a tuning aid; results do not depend on the tile width.
+ * Further switches, all read by tsdp_init unless stated, none of which changes what is computed (they select between
+ * kernels that are tested against the same reference): TSDP_NO_COMPACT runs every round on the dense candidate
+ * layout instead of the list of live candidates; TSDP_NO_FUSED_ATTN (read at every forward) keeps the 16-token
+ * self-attention as a kernel of its own instead of the QKV projection's epilogue; TSDP_NO_TC_ATTN keeps the context
+ * cross-attention of TSDP_ARCH_DIT on the mma.sync kernel, TSDP_TC_ATTN=2 puts it on the tcgen05 kernel for every
+ * group size (default: groups of at least 256 query rows, 64-wide heads, obs_tokens a multiple of 32 and <= 256);
+ * TSDP_VERBOSE prints the kernels' occupancy figures once per tsdp_load_weights.
  * Every function returns a tsdp_status; nothing throws or aborts.  A context is not re-entrant: one
  * call at a time.  There is no CPU fallback: without a CUDA device tsdp_init fails with TSDP_ERR_CUDA.
  */

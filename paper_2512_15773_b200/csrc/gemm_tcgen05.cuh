@@ -50,8 +50,12 @@ __host__ __device__ constexpr bool gemm_tma_epilogue(int BN) { return BN >= 128 
 __host__ __device__ constexpr int gemm_epi_smem_bytes(int BN) {
   return BN == GEMM_ATTN_BN ? GEMM_ATTN_STAGING_BYTES : (gemm_tma_epilogue(BN) ? GEMM_STAGING_BYTES : 0);
 }
+// The tile's bias values, staged once per tile (one tile ahead of their use) so that no epilogue warp waits on a
+// global load between its tensor-memory reads: 128 floats per column half, or one copy of the head's 192 per
+// row quadrant in the fused-attention kernel (whose warps only synchronise quadrant by quadrant).
+__host__ __device__ constexpr int gemm_bias_smem_bytes(int BN) { return BN == GEMM_ATTN_BN ? 4 * GEMM_ATTN_BN * 4 : 2 * 128 * 4; }
 __host__ __device__ constexpr int gemm_smem_bytes(int BN) {
-  return gemm_stages(BN) * gemm_stage_bytes(BN) + gemm_epi_smem_bytes(BN) + 1024 + 256;
+  return gemm_stages(BN) * gemm_stage_bytes(BN) + gemm_epi_smem_bytes(BN) + 1024 + 256 + gemm_bias_smem_bytes(BN);
 }
 // CTA-pair form (CG = 2, tcgen05 cta_group::2): a 256 x BN tile on two SMs.  Each CTA stages its own 128 rows of A and
 // HALF of the W tile, so a stage is smaller and the ring deeper.
@@ -64,7 +68,7 @@ __host__ __device__ constexpr int gemm_epi_smem_bytes_cg(int BN, int CG) {
   return gemm_tma_epilogue(BN) ? GEMM_STAGING_BYTES * gemm_staging_bufs(CG) : gemm_epi_smem_bytes(BN);
 }
 __host__ __device__ constexpr int gemm_smem_bytes_cg(int BN, int CG) {
-  return gemm_stages_cg(BN, CG) * gemm_stage_bytes_cg(BN, CG) + gemm_epi_smem_bytes_cg(BN, CG) + 1024 + 256;
+  return gemm_stages_cg(BN, CG) * gemm_stage_bytes_cg(BN, CG) + gemm_epi_smem_bytes_cg(BN, CG) + 1024 + 256 + gemm_bias_smem_bytes(BN);
 }
 
 namespace ptx {
@@ -227,6 +231,15 @@ __device__ __forceinline__ float gelu_fast(float x) {
   const float t = tanh_fast(__fmul_rn(0.7978845608028654f, __fmaf_rn(0.044715f, x3, x)));
   return __fmul_rn(__fmul_rn(0.5f, x), __fadd_rn(1.0f, t));
 }
+// Two values at a time on the packed fp32 pipe: every operation is the per-component round-to-nearest one of
+// gelu_fast, so the bits are the same.
+__device__ __forceinline__ float2 gelu_fast2(float2 x) {
+  const float2 x3 = __fmul2_rn(__fmul2_rn(x, x), x);
+  const float2 u = __fmul2_rn(make_float2(0.7978845608028654f, 0.7978845608028654f),
+                              __ffma2_rn(make_float2(0.044715f, 0.044715f), x3, x));
+  const float2 t = make_float2(tanh_fast(u.x), tanh_fast(u.y));
+  return __fmul2_rn(__fmul2_rn(make_float2(0.5f, 0.5f), x), __fadd2_rn(make_float2(1.0f, 1.0f), t));
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 }  // namespace ptx
 
@@ -289,13 +302,14 @@ __device__ __forceinline__ const float* gate_row(const GemmArgs& g, int row) {
   return g.gate + (size_t)tau * g.gate_ld;
 }
 
+// `bias16`: the 16 bias values of these columns (fetched by the caller before it waited for the accumulator).
 template <int EPI>
-__device__ __forceinline__ void epilogue_store16(const GemmArgs& g, int row, int col, const uint32_t v[16]) {
+__device__ __forceinline__ void epilogue_store16(const GemmArgs& g, int row, int col, const uint32_t v[16], const float* bias16) {
   float f[16];
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
     f[i] = __uint_as_float(v[i]);
-    if (g.bias) f[i] += __ldg(g.bias + col + i);
+    if (g.bias) f[i] += bias16[i];
     if (EPI == EPI_GELU) f[i] = ptx::gelu_fast(f[i]);
   }
   if (EPI == EPI_GATE) {
@@ -362,6 +376,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const uint32_t tmem_slot = bar0 + 8u * (2 * STAGES + 4);
   volatile uint32_t* tmem_slot_ptr =
       reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - ptx::smem_u32(smem_raw)));
+  float* sbias = reinterpret_cast<float*>(smem_raw + (bar0 + 256u - ptx::smem_u32(smem_raw)));    // behind the barriers
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tiles_n = g.N / BN;
@@ -464,11 +479,27 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int r_tile = quad * 32 + lane;                    // this lane's row of the tile
       const int cand_l = r_tile >> 4, r_l = r_tile & 15;      // candidate (0..7) and token of that row
       const int cand_w = 2 * quad + half;                     // the candidate this warp attends for
+      // the quadrant's copy of the head's bias: thread j of the pair brings values j, j + 64, j + 128, one tile ahead
+      float* sb = sbias + quad * GEMM_ATTN_BN;
+      const int bj = half * 32 + lane;
+      float bnx[3] = {0.f, 0.f, 0.f};
+      if (g.bias && tile0 < n_tiles) {
+#pragma unroll
+        for (int u = 0; u < 3; ++u) bnx[u] = __ldg(g.bias + (tile0 % tiles_n) * BN + bj + 64 * u);
+      }
       for (int tile = tile0; tile < n_tiles; tile += tile_step, ++it) {
         const int tm = (tile / tiles_n) * CG + (int)rank, tn = tile % tiles_n;
         const int as = it & 1; const uint32_t aphase = (it >> 1) & 1;
+        if (g.bias) {      // the previous tile's reads of `sb` lie before its staging barrier
+#pragma unroll
+          for (int u = 0; u < 3; ++u) sb[bj + 64 * u] = bnx[u];
+          if (tile + tile_step < n_tiles) {
+#pragma unroll
+            for (int u = 0; u < 3; ++u) bnx[u] = __ldg(g.bias + ((tile + tile_step) % tiles_n) * BN + bj + 64 * u);
+          }
+        }
         // both warps of the quadrant agree on the outcome; the barrier also orders the previous tile's reads of the
-        // staging area before this tile's writes
+        // staging area before this tile's writes, and publishes `sb`
         ok = ptx::named_bar_and(pair_bar, 64, ptx::mbar_wait_warp(tfull_bar(as), aphase, wlim));
         if (!ok) break;
         ptx::tc_fence_after();
@@ -490,8 +521,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           if (g.bias) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-              const float4 bb = __ldg(reinterpret_cast<const float4*>(g.bias + tn * BN + col) + i);
-              f[4 * i] += bb.x; f[4 * i + 1] += bb.y; f[4 * i + 2] += bb.z; f[4 * i + 3] += bb.w;
+              const float4 bb = reinterpret_cast<const float4*>(sb + col)[i];
+              const float2 lo = __fadd2_rn(make_float2(f[4 * i], f[4 * i + 1]), make_float2(bb.x, bb.y));
+              const float2 hi = __fadd2_rn(make_float2(f[4 * i + 2], f[4 * i + 3]), make_float2(bb.z, bb.w));
+              f[4 * i] = lo.x; f[4 * i + 1] = lo.y; f[4 * i + 2] = hi.x; f[4 * i + 3] = hi.y;
             }
           }
           __nv_bfloat16* dst = att + ((size_t)(cand_l * 3 + (col >> 6)) * 16 + r_l) * P + (col & 63);
@@ -528,10 +561,30 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const uint32_t sw = (uint32_t)(r & 7);
       const bool issuer = (quad == 0 && lane == 0);
       const int bar_id = 1 + half;
+      // this half's bias values of a tile: thread r brings value r, one tile ahead of its use
+      float* sb = sbias + half * 128;
+      const bool bias_lane = g.bias != nullptr && r < COLS;
+      float bias_next = 0.f;
+      if (bias_lane && tile0 < n_tiles) bias_next = __ldg(g.bias + (tile0 % tiles_n) * BN + half * COLS + r);
+      constexpr int NPART = COLS / 32;       // 32-column parts of this half
       for (int tile = tile0; tile < n_tiles; tile += tile_step, ++it) {
         const int tm = (tile / tiles_n) * CG + (int)rank, tn = tile % tiles_n;
         const int as = it & 1; const uint32_t aphase = (it >> 1) & 1;
-        // all four warps of this half agree on the outcome, so none is left alone at a named barrier
+        if (bias_lane) {         // the previous tile's reads of `sb` lie before its last staging barrier
+          sb[r] = bias_next;
+          if (tile + tile_step < n_tiles) bias_next = __ldg(g.bias + ((tile + tile_step) % tiles_n) * BN + half * COLS + r);
+        }
+        // the row's gate values of the first part, in flight while the accumulator is awaited
+        float4 gq[8];
+        const float* gate_base = nullptr;
+        if (EPI == EPI_GATE) {
+          const int grow = min(tm * GEMM_BM + r, M - 1);       // rows past the live ones only reach rows nobody reads
+          gate_base = gate_row(g, grow) + tn * BN + half * COLS;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) gq[i] = __ldg(reinterpret_cast<const float4*>(gate_base) + i);
+        }
+        // all four warps of this half agree on the outcome, so none is left alone at a named barrier (which also
+        // publishes `sb`)
         ok = ptx::named_bar_and(bar_id, 128, ptx::mbar_wait_warp(tfull_bar(as), aphase, wlim));
         if (!ok) break;
         ptx::tc_fence_after();
@@ -544,6 +597,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           for (int part = 0; part < CW / 32; ++part) {
             uint32_t v[32];
             const int col_t = ch * CW + part * 32;                 // column inside this half
+            float4 gn[8];                                          // the next part's gate values: in flight during this one
+            if (EPI == EPI_GATE && col_t + 32 < COLS) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i) gn[i] = __ldg(reinterpret_cast<const float4*>(gate_base + col_t + 32) + i);
+            }
             ptx::tmem_ld32(taddr + (uint32_t)col_t, v);
             ptx::tmem_ld_wait();
             if (ch == NCH - 1 && part == CW / 32 - 1) {            // accumulator fully read: hand it back
@@ -551,30 +609,35 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               __syncwarp();
               if (lane == 0) release_acc(as);
             }
-            const int col = tn * BN + half * COLS + col_t;
-            float f[32];
+            float2 f2[16];
 #pragma unroll
-            for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]);
+            for (int i = 0; i < 16; ++i) f2[i] = make_float2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
             if (g.bias) {
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
-                const float4 bb = __ldg(reinterpret_cast<const float4*>(g.bias + col) + i);
-                f[4 * i] += bb.x; f[4 * i + 1] += bb.y; f[4 * i + 2] += bb.z; f[4 * i + 3] += bb.w;
+                const float4 bb = reinterpret_cast<const float4*>(sb + col_t)[i];
+                f2[2 * i] = __fadd2_rn(f2[2 * i], make_float2(bb.x, bb.y));
+                f2[2 * i + 1] = __fadd2_rn(f2[2 * i + 1], make_float2(bb.z, bb.w));
               }
             }
             if (EPI == EPI_GELU) {
 #pragma unroll
-              for (int i = 0; i < 32; ++i) f[i] = ptx::gelu_fast(f[i]);
+              for (int i = 0; i < 16; ++i) f2[i] = ptx::gelu_fast2(f2[i]);
             }
             if (EPI == EPI_GATE) {
-              const int grow = min(tm * GEMM_BM + r, M - 1);       // rows past the live ones only reach rows nobody reads
-              const float4* gp = reinterpret_cast<const float4*>(gate_row(g, grow) + col);
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
-                const float4 gg = __ldg(gp + i);
-                f[4 * i] *= gg.x; f[4 * i + 1] *= gg.y; f[4 * i + 2] *= gg.z; f[4 * i + 3] *= gg.w;
+                f2[2 * i] = __fmul2_rn(f2[2 * i], make_float2(gq[i].x, gq[i].y));
+                f2[2 * i + 1] = __fmul2_rn(f2[2 * i + 1], make_float2(gq[i].z, gq[i].w));
+              }
+              if (col_t + 32 < COLS) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) gq[i] = gn[i];
               }
             }
+            float f[32];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) { f[2 * i] = f2[i].x; f[2 * i + 1] = f2[i].y; }
             if (part == 0) {   // the TMA store that last used this staging buffer must have read it
               if (issuer) { if (NB == 2) ptx::bulk_wait_read1(); else ptx::bulk_wait_read0(); }
               ptx::named_bar_sync(bar_id, 128);
@@ -609,16 +672,24 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       for (int tile = tile0; tile < n_tiles && ok; tile += tile_step, ++it) {
         const int tm = (tile / tiles_n) * CG + (int)rank, tn = tile % tiles_n;
         const int as = it & 1; const uint32_t aphase = (it >> 1) & 1;
+        float bv[COLS];          // this half's bias values (narrow tiles: at most 32), fetched while the accumulator is awaited
+        if (g.bias) {
+#pragma unroll
+          for (int i = 0; i < COLS / 4; ++i) {
+            const float4 bb = __ldg(reinterpret_cast<const float4*>(g.bias + tn * BN + half * COLS) + i);
+            bv[4 * i] = bb.x; bv[4 * i + 1] = bb.y; bv[4 * i + 2] = bb.z; bv[4 * i + 3] = bb.w;
+          }
+        }
         if (!ptx::mbar_wait_warp(tfull_bar(as), aphase, wlim)) { ok = false; break; }
         ptx::tc_fence_after();
         const int row = tm * GEMM_BM + quad * 32 + lane;
         const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * ACC + half * COLS);
-#pragma unroll 1
+#pragma unroll
         for (int c = 0; c < COLS; c += 16) {
           uint32_t v[16];
           ptx::tmem_ld16(taddr + (uint32_t)c, v);
           ptx::tmem_ld_wait();
-          if (row < M) epilogue_store16<EPI>(g, row, tn * BN + half * COLS + c, v);
+          if (row < M) epilogue_store16<EPI>(g, row, tn * BN + half * COLS + c, v, bv + c);
         }
         ptx::tc_fence_before();
         __syncwarp();

@@ -9,6 +9,8 @@ pass where each operand was written by the previous kernel.  Prints one line per
 line with the flop-weighted total of the six plain shapes, and the total of the four kernels the decoder
 transformer really launches per block (QKV projection with the self-attention in its epilogue, the bf16
 attention projection, MLP up, MLP down: the cross-attention projections are folded into its memory tokens).
+With --library each plain shape is also timed as torch.mm (the vendor library's bf16 GEMM, no bias, no epilogue) on
+the same operands: context for what the shape itself allows, not a path of the sampler.
 """
 import argparse
 import json
@@ -30,6 +32,7 @@ def main():
     ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--K", type=int, default=-1)
     ap.add_argument("--reps", type=int, default=20)
+    ap.add_argument("--library", action="store_true", help="also time torch.mm on the same operands")
     args = ap.parse_args()
     wl = dict(inputs.WORKLOADS[args.workload])
     B = args.batch or wl["B"]
@@ -50,9 +53,24 @@ def main():
         flop = 2.0 * M * N * Kd
         io = M * Kd * 2 + N * Kd * 2 + (M * Kd * 2 if epi == 4 else M * N * (2 if epi in (0, 1) else (8 if epi == 2 else 4)))
         rows.append(dict(name=name, M=M, N=N, K=Kd, epi=epi, us=1e3 * ms, tflops=flop / ms / 1e9, gbs=io / ms / 1e6))
+        if args.library and epi != 4:
+            Wt = W.t()
+            lib_out = torch.empty(M, N, device="cuda", dtype=torch.bfloat16)
+            for _ in range(3):
+                torch.mm(A, Wt, out=lib_out)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(args.reps):
+                torch.mm(A, Wt, out=lib_out)
+            e1.record()
+            torch.cuda.synchronize()
+            lib_ms = e0.elapsed_time(e1) / args.reps
+            rows[-1].update(library_us=1e3 * lib_ms, library_tflops=flop / lib_ms / 1e9)
         tot_ms += ms; tot_flop += flop
         print(f"{name:10s} M={M:6d} N={N:5d} K={Kd:5d} epi={epi}  {1e3 * ms:8.1f} us  {flop / ms / 1e9:7.1f} TFLOP/s"
-              f"  {io / ms / 1e6:7.0f} GB/s (A + W + out bytes)")
+              f"  {io / ms / 1e6:7.0f} GB/s (A + W + out bytes)"
+              + (f"   torch.mm {rows[-1]['library_us']:8.1f} us {rows[-1]['library_tflops']:7.1f} TFLOP/s" if "library_us" in rows[-1] else ""))
     # what the decoder transformer launches per block: fused QKV + attention, the bf16 attention projection, the MLP pair
     four = [r for r in rows if r["name"] in ("qkv_attn", "attn_out_bf16", "mlp_up", "mlp_down")]
     rows_all, rows = rows, [r for r in rows if r["name"] not in ("qkv_attn", "attn_out_bf16")]

@@ -693,7 +693,7 @@ int gemm_qkv_attn_raw(tsdp_ctx* c, const void* A, const void* W_hm, const float*
 bool xfold_ok(const tsdp_config_t& cfg, const tsdp_net_t& net) {
   if (cfg.precision != 1 || net.arch != TSDP_ARCH_XFMR || getenv("TSDP_NO_FOLD") != nullptr) return false;
   const int NK = 1 + cfg.obs_tokens, d = net.d, heads = net.heads;
-  if (heads < 2 || heads % 2 || d % heads) return false;
+  if (heads < 2 || heads > 16 || heads % 2 || d % heads) return false;      // one (row, head) of the softmax per thread
   const int dh = d / heads;
   return cfg.H <= 16 && NK <= XF_MAXNK && NK * heads <= XF_MAXN && (d == 128 || d == 256 || d == 512) &&
          dh % 8 == 0 && dh <= 128 && xfold_build_smem(d, dh) <= 200 * 1024;

@@ -142,10 +142,11 @@ __device__ __forceinline__ void xf_cp_commit() { asm volatile("cp.async.commit_g
 template <int N>
 __device__ __forceinline__ void xf_cp_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// Shared memory of one block: xhat [16][D+8] bf16 | kq rows [NKH][D+8] bf16, later the warps' output tiles
-// [warps][16][D/16+8] fp32 | u rows [NKH/2][D+8] words | partial scores [4][16][32] fp32 | P [16][40] bf16.
+// Shared memory of one block: xhat [16][D+8] bf16 | kq rows [NKH][D+8] bf16 (both dead after the scores: the product
+// P . U [16][D+8] fp32 is then laid over the two) | u rows [NKH/2][D+8] words | partial scores [4][16][32] fp32 |
+// P [16][40] bf16.
 __host__ __device__ constexpr size_t xf_region_bytes(int D, int nkh) {
-  const size_t k = (size_t)nkh * (D + 8) * 2, t = (size_t)XF_WARPS * 16 * (D / (2 * XF_WARPS) + 8) * 4;
+  const size_t k = (size_t)nkh * (D + 8) * 2, t = (size_t)16 * (D + 8) * 2;     // xhat + region >= [16][D+8] fp32
   return k > t ? k : t;
 }
 __host__ __device__ constexpr size_t xf_smem_bytes(int D, int nkh) {
@@ -159,9 +160,10 @@ __host__ __device__ constexpr size_t xf_smem_bytes(int D, int nkh) {
 //   1  xhat = LayerNorm without affine of the candidate's rows, bf16, into shared memory (warp w: rows 2w, 2w+1)
 //   2  partial scores: warp w covers a quarter of the D input columns for two of the 8-wide score tiles
 //   3  softmax over the memory tokens per (row, head) -> P [16 x 32] bf16
-//   4  warp w: output columns [w D/8, (w+1) D/8) = P . U + bo2, staged through shared memory so that the
-//      residual stream is read and written in full 16-byte lanes along its rows, in place
-//   5  the LayerNorm in front of the MLP, from the updated rows still in registers -> ln3_out (bf16)
+//   4  warp w: output columns [w D/8, (w+1) D/8) of P . U for all 16 rows -> shared memory (fp32)
+//   5  warp w again owns rows 2w, 2w+1, whose residual values (stream + delta) are still in its registers from
+//      phase 1: adds the product and bo2, writes the stream back in full 16-byte lanes, and applies the LayerNorm in
+//      front of the MLP with warp-level statistics -> ln3_out (bf16)
 // `delta` is the output of the self-attention projection (bf16, bias included), which this kernel adds to the
 // residual stream before anything else: that GEMM then writes 2 bytes per element instead of doing an fp32
 // read-modify-write of the stream.
@@ -176,8 +178,6 @@ xattn_fold_kernel(float* __restrict__ x, const __nv_bfloat16* __restrict__ delta
   constexpr int LDU = D + 8;               // words per row of the u rows
   constexpr int LDP = XF_MAXN + 8;
   constexpr int V = D / 128;
-  constexpr int HW = D / (2 * XF_WARPS);   // output columns of a warp per half
-  constexpr int LDT = HW + 8;
   extern __shared__ __align__(16) unsigned char xf_smem[];
   const int NK = 1 + To, NKH = NK * heads;
   __nv_bfloat16* sA = reinterpret_cast<__nv_bfloat16*>(xf_smem);
@@ -226,6 +226,21 @@ xattn_fold_kernel(float* __restrict__ x, const __nv_bfloat16* __restrict__ delta
 
   // ---- 1: LayerNorm statistics, normalised rows to shared memory
   for (int i = threadIdx.x; i < 16 * LDP / 2; i += XF_THREADS) reinterpret_cast<uint32_t*>(sP)[i] = 0u;
+  float4 xr[2][V];                             // rows 2 warp, 2 warp + 1 of the stream with delta added: kept until phase 5
+  // the score constants this thread needs in phase 3: in flight from here on
+  float cst[XF_MAXNK];
+  {
+    const int h = threadIdx.x % heads;
+#pragma unroll
+    for (int j = 0; j < XF_MAXNK; ++j) {
+      cst[j] = 0.f;
+      if (j < NK && threadIdx.x < 16 * heads) {
+        const float* cp = (j == 0 ? tb.c_time + (size_t)tau * L * heads : tb.c_obs + ((size_t)item * To + (j - 1)) * L * heads) +
+                          (size_t)layer * heads;
+        cst[j] = __ldg(cp + h);
+      }
+    }
+  }
   {                                            // two rows per warp: all of their loads are in flight together
     float4 v[2][V];
 #pragma unroll
@@ -244,7 +259,7 @@ xattn_fold_kernel(float* __restrict__ x, const __nv_bfloat16* __restrict__ delta
 #pragma unroll
     for (int rr = 0; rr < 2; ++rr)
 #pragma unroll
-      for (int j = 0; j < V; ++j) xf_add_bf16x4(v[rr][j], dv[rr][j]);
+      for (int j = 0; j < V; ++j) { xf_add_bf16x4(v[rr][j], dv[rr][j]); xr[rr][j] = v[rr][j]; }
 #pragma unroll
     for (int rr = 0; rr < 2; ++rr) {
       const int r = 2 * warp + rr;
@@ -317,17 +332,12 @@ xattn_fold_kernel(float* __restrict__ x, const __nv_bfloat16* __restrict__ delta
   __syncthreads();
 
   // ---- 3: softmax over the NK memory tokens for every (row, head)
-  for (int idx = threadIdx.x; idx < 16 * heads; idx += XF_THREADS) {
+  if (threadIdx.x < 16 * heads) {              // heads <= 16: one (row, head) per thread
+    const int idx = threadIdx.x;
     const int r = idx / heads, h = idx % heads;
     float s[XF_MAXNK];
 #pragma unroll
-    for (int j = 0; j < XF_MAXNK; ++j) {
-      if (j < NK) {
-        const float* cp = (j == 0 ? tb.c_time + (size_t)tau * L * heads : tb.c_obs + ((size_t)item * To + (j - 1)) * L * heads) +
-                          (size_t)layer * heads;
-        s[j] = __ldg(cp + h);
-      }
-    }
+    for (int j = 0; j < XF_MAXNK; ++j) s[j] = cst[j];
     float m = -INFINITY;
 #pragma unroll
     for (int j = 0; j < XF_MAXNK; ++j) {
@@ -348,9 +358,12 @@ xattn_fold_kernel(float* __restrict__ x, const __nv_bfloat16* __restrict__ delta
       if (j < NK) sP[r * LDP + j * heads + h] = __float2bfloat16_rn(s[j] * inv);
   }
   xf_cp_wait<0>();                             // this thread's u chunks have landed
-  __syncthreads();                             // also: every warp is done with the kq rows, whose memory the tiles reuse
+  __syncthreads();                             // also: every warp is done with the normalised rows and the kq rows, whose memory the product reuses
 
-  // ---- 4: P . U + bo2 into the residual stream
+  // ---- 4: P . U for all 16 rows, warp w the output columns [w D/8, (w+1) D/8), into shared memory over the
+  //         (now dead) normalised rows and kq rows
+  constexpr int LDO = D + 8;                   // fp32 words per row of the product
+  float* sO = reinterpret_cast<float*>(xf_smem);
   {
     uint32_t pa[2][4];
 #pragma unroll
@@ -372,89 +385,67 @@ xattn_fold_kernel(float* __restrict__ x, const __nv_bfloat16* __restrict__ delta
         ulive[k2][rg] = 2 * pr < NKH ? 0xffffffffu : 0u;
         pu[k2][rg] = sU + (size_t)min(pr, NKH / 2 - 1) * LDU + g;
       }
-    float* tile = reinterpret_cast<float*>(region) + (size_t)warp * 16 * LDT;
-    constexpr int LPR = HW / 4;              // lanes per tile row in the row-wise pass
-    constexpr int RPI = 32 / LPR;            // rows per instruction
-    constexpr int NI = 16 / RPI;
-    const int rr0 = lane / LPR, c4 = (lane % LPR) * 4;
-    float4 xn[2][NI];                        // the updated rows of this lane, kept for the LayerNorm that follows
+    const int o_base = warp * (D / XF_WARPS);
 #pragma unroll
-    for (int half = 0; half < 2; ++half) {
-      const int o_base = warp * (D / XF_WARPS) + half * HW;
-      uint2 dl[NI];
+    for (int nt = 0; nt < D / (8 * XF_WARPS); ++nt) {
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int i = 0; i < NI; ++i) {
-        const int r = min(i * RPI + rr0, H - 1);
-        xn[half][i] = *reinterpret_cast<const float4*>(xc + (size_t)r * D + o_base + c4);
-        dl[i] = *reinterpret_cast<const uint2*>(dc + (size_t)r * D + o_base + c4);
-      }
-      const float4 bb = __ldg(reinterpret_cast<const float4*>(bo2 + o_base + c4));
-#pragma unroll
-      for (int nt = 0; nt < HW / 8; ++nt) {
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int k2 = 0; k2 < 2; ++k2)
-          if (16 * k2 < NKH)
-            mma_bf16_16816(acc, pa[k2], pu[k2][0][o_base + 8 * nt] & ulive[k2][0], pu[k2][1][o_base + 8 * nt] & ulive[k2][1]);
-        *reinterpret_cast<float2*>(tile + g * LDT + 8 * nt + 2 * tg) = make_float2(acc[0], acc[1]);
-        *reinterpret_cast<float2*>(tile + (g + 8) * LDT + 8 * nt + 2 * tg) = make_float2(acc[2], acc[3]);
-      }
-      __syncwarp();
-#pragma unroll
-      for (int i = 0; i < NI; ++i) {
-        const int r = i * RPI + rr0;
-        const float4 t = *reinterpret_cast<const float4*>(tile + r * LDT + c4);
-        xf_add_bf16x4(xn[half][i], dl[i]);
-        xn[half][i].x += t.x + bb.x; xn[half][i].y += t.y + bb.y; xn[half][i].z += t.z + bb.z; xn[half][i].w += t.w + bb.w;
-        if (r < H) *reinterpret_cast<float4*>(xc + (size_t)r * D + o_base + c4) = xn[half][i];
-      }
-      __syncwarp();
+      for (int k2 = 0; k2 < 2; ++k2)
+        if (16 * k2 < NKH)
+          mma_bf16_16816(acc, pa[k2], pu[k2][0][o_base + 8 * nt] & ulive[k2][0], pu[k2][1][o_base + 8 * nt] & ulive[k2][1]);
+      *reinterpret_cast<float2*>(sO + g * LDO + o_base + 8 * nt + 2 * tg) = make_float2(acc[0], acc[1]);
+      *reinterpret_cast<float2*>(sO + (g + 8) * LDO + o_base + 8 * nt + 2 * tg) = make_float2(acc[2], acc[3]);
     }
+  }
+  // bo2 of this lane's columns: in flight across the barrier
+  float4 bb[V];
+#pragma unroll
+  for (int j = 0; j < V; ++j) bb[j] = __ldg(reinterpret_cast<const float4*>(bo2) + j * 32 + lane);
+  __syncthreads();
 
-    // ---- 5: LayerNorm of the updated rows (the block's third LayerNorm), bf16, for the MLP that follows.
-    //         Row r's D values sit in LPR lanes of each of the 8 warps: lane group -> warp partial -> block.
-    float* part = sS;                          // [XF_WARPS][16] partial sums, then [16] means / rstds behind them
-    float* stat = sS + XF_WARPS * 16;
+  // ---- 5: rows 2 warp, 2 warp + 1: stream + delta (registers) + product + bo2 -> the stream; LayerNorm -> ln3_out
+  {
 #pragma unroll
-    for (int pass = 0; pass < 2; ++pass) {
+    for (int rr = 0; rr < 2; ++rr) {
+      const int r = 2 * warp + rr;
 #pragma unroll
-      for (int i = 0; i < NI; ++i) {
-        const int r = i * RPI + rr0;
-        float a = 0.f;
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          const float4 e = xn[half][i];
-          if (pass == 0) a += (e.x + e.y) + (e.z + e.w);
-          else { const float m = stat[r]; a += (e.x - m) * (e.x - m) + (e.y - m) * (e.y - m) + (e.z - m) * (e.z - m) + (e.w - m) * (e.w - m); }
-        }
-#pragma unroll
-        for (int o = LPR / 2; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-        if (lane % LPR == 0) part[warp * 16 + r] = a;
+      for (int j = 0; j < V; ++j) {
+        const float4 t = *reinterpret_cast<const float4*>(sO + r * LDO + (j * 32 + lane) * 4);
+        float4& e = xr[rr][j];
+        e.x += t.x + bb[j].x; e.y += t.y + bb[j].y; e.z += t.z + bb[j].z; e.w += t.w + bb[j].w;
+        if (r < H) reinterpret_cast<float4*>(xc + (size_t)r * D)[j * 32 + lane] = e;
       }
-      __syncthreads();
-      if (threadIdx.x < 16) {
-        float a = 0.f;
+    }
+    float4 gg[V], be[V];
 #pragma unroll
-        for (int w = 0; w < XF_WARPS; ++w) a += part[w * 16 + threadIdx.x];
-        stat[pass * 16 + threadIdx.x] = pass == 0 ? a / D : rsqrtf(a / D + 1e-5f);
-      }
-      __syncthreads();
+    for (int j = 0; j < V; ++j) {
+      gg[j] = __ldg(reinterpret_cast<const float4*>(ln3_g) + j * 32 + lane);
+      be[j] = __ldg(reinterpret_cast<const float4*>(ln3_b) + j * 32 + lane);
     }
     __nv_bfloat16* oc = ln3_out + (size_t)n * H * D;
 #pragma unroll
-    for (int half = 0; half < 2; ++half) {
-      const int col = warp * (D / XF_WARPS) + half * HW + c4;
-      const float4 gg = __ldg(reinterpret_cast<const float4*>(ln3_g + col)), be = __ldg(reinterpret_cast<const float4*>(ln3_b + col));
+    for (int rr = 0; rr < 2; ++rr) {
+      const int r = 2 * warp + rr;
+      float sm = 0.f;
 #pragma unroll
-      for (int i = 0; i < NI; ++i) {
-        const int r = i * RPI + rr0;
-        if (r < H) {
-          const float m = stat[r], rs = stat[16 + r];
-          const float4 e = xn[half][i];
+      for (int j = 0; j < V; ++j) sm += (xr[rr][j].x + xr[rr][j].y) + (xr[rr][j].z + xr[rr][j].w);
+      const float mean = warp_sum(sm) / D;
+      float q = 0.f;
+#pragma unroll
+      for (int j = 0; j < V; ++j) {
+        float4& e = xr[rr][j];
+        e.x -= mean; e.y -= mean; e.z -= mean; e.w -= mean;
+        q += (e.x * e.x + e.y * e.y) + (e.z * e.z + e.w * e.w);
+      }
+      const float rs = rsqrtf(warp_sum(q) / D + 1e-5f);
+      if (r < H) {
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+          const float4 e = xr[rr][j];
           uint2 o2;
-          o2.x = pack_bf16((e.x - m) * rs * gg.x + be.x, (e.y - m) * rs * gg.y + be.y);
-          o2.y = pack_bf16((e.z - m) * rs * gg.z + be.z, (e.w - m) * rs * gg.w + be.w);
-          *reinterpret_cast<uint2*>(oc + (size_t)r * D + col) = o2;
+          o2.x = pack_bf16(e.x * rs * gg[j].x + be[j].x, e.y * rs * gg[j].y + be[j].y);
+          o2.y = pack_bf16(e.z * rs * gg[j].z + be[j].z, e.w * rs * gg[j].w + be[j].w);
+          reinterpret_cast<uint2*>(oc + (size_t)r * D)[j * 32 + lane] = o2;
         }
       }
     }

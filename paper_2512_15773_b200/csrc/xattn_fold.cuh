@@ -138,6 +138,11 @@ __device__ __forceinline__ void xf_add_bf16x4(float4& a, const uint2 d) {
   const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&d.y));
   a.x += lo.x; a.y += lo.y; a.z += hi.x; a.w += hi.y;
 }
+// fp32 arithmetic two values at a time (packed fp32 pipe; each component rounded as the scalar operation would be)
+__device__ __forceinline__ float2 xf_lo(const float4& a) { return make_float2(a.x, a.y); }
+__device__ __forceinline__ float2 xf_hi(const float4& a) { return make_float2(a.z, a.w); }
+__device__ __forceinline__ float4 xf_join(float2 lo, float2 hi) { return make_float4(lo.x, lo.y, hi.x, hi.y); }
+__device__ __forceinline__ float2 xf_dup(float v) { return make_float2(v, v); }
 __device__ __forceinline__ void xf_cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void xf_cp_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
@@ -263,23 +268,26 @@ xattn_fold_kernel(float* __restrict__ x, const __nv_bfloat16* __restrict__ delta
 #pragma unroll
     for (int rr = 0; rr < 2; ++rr) {
       const int r = 2 * warp + rr;
-      float s = 0.f;
+      float2 s2 = make_float2(0.f, 0.f);
 #pragma unroll
-      for (int j = 0; j < V; ++j) s += v[rr][j].x + v[rr][j].y + v[rr][j].z + v[rr][j].w;
-      const float mean = warp_sum(s) / D;
-      float q = 0.f;
+      for (int j = 0; j < V; ++j) s2 = __fadd2_rn(s2, __fadd2_rn(xf_lo(v[rr][j]), xf_hi(v[rr][j])));
+      const float mean = warp_sum(s2.x + s2.y) / D;
+      const float2 nm = xf_dup(-mean);
+      float2 q2 = make_float2(0.f, 0.f);
+      float2 lo[V], hi[V];
 #pragma unroll
       for (int j = 0; j < V; ++j) {
-        float4& e = v[rr][j];
-        e.x -= mean; e.y -= mean; e.z -= mean; e.w -= mean;
-        q += e.x * e.x + e.y * e.y + e.z * e.z + e.w * e.w;
+        lo[j] = __fadd2_rn(xf_lo(v[rr][j]), nm); hi[j] = __fadd2_rn(xf_hi(v[rr][j]), nm);
+        q2 = __ffma2_rn(lo[j], lo[j], q2); q2 = __ffma2_rn(hi[j], hi[j], q2);
       }
-      const float rstd = r < H ? rsqrtf(warp_sum(q) / D + 1e-5f) : 0.f;      // rows past H enter the products as zeros
+      const float rstd = r < H ? rsqrtf(warp_sum(q2.x + q2.y) / D + 1e-5f) : 0.f;      // rows past H enter the products as zeros
+      const float2 rs2 = xf_dup(rstd);
 #pragma unroll
       for (int j = 0; j < V; ++j) {
+        const float2 a = __fmul2_rn(lo[j], rs2), b = __fmul2_rn(hi[j], rs2);
         uint2 pk2;
-        pk2.x = pack_bf16(v[rr][j].x * rstd, v[rr][j].y * rstd);
-        pk2.y = pack_bf16(v[rr][j].z * rstd, v[rr][j].w * rstd);
+        pk2.x = pack_bf16(a.x, a.y);
+        pk2.y = pack_bf16(b.x, b.y);
         *reinterpret_cast<uint2*>(sA + r * LDA + (j * 32 + lane) * 4) = pk2;
       }
     }
@@ -288,38 +296,26 @@ xattn_fold_kernel(float* __restrict__ x, const __nv_bfloat16* __restrict__ delta
   __syncthreads();
 
   // ---- 2: scores.  Warp w takes quarter (w & 3) of the D input columns and the score tiles 2 (w >> 2), 2 (w >> 2) + 1;
-  //         the four partial sums of a score are added in a fixed order in phase 3 (no atomics: same bits every run)
+  //         the four partial sums of a score are added in a fixed order in phase 3 (no atomics: same bits every run).
+  //         Score columns past the last (token, head) are computed on a repeated row and never read.
   {
     constexpr int KSW = D / 64;
     const int kq4 = warp & 3, nh = warp >> 2;
-    const __nv_bfloat16* pk[2];
-    uint32_t live[2];
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      const int nt = 2 * nh + u;
-      live[u] = 8 * nt + g < NKH ? 0xffffffffu : 0u;           // rows past the last (token, head) read row NKH-1, masked
-      pk[u] = sK + (size_t)min(8 * nt + g, NKH - 1) * LDA + kq4 * (D / 4) + 2 * tg;
-    }
     float sc[2][4];
 #pragma unroll
     for (int u = 0; u < 2; ++u) { sc[u][0] = sc[u][1] = sc[u][2] = sc[u][3] = 0.f; }
     if (16 * nh < NKH) {
+      // ldmatrix addresses: A rows l & 15 at column 8 (l >> 4); B rows 16 nh + (l & 7) + 8 (l >> 4) at column 8 ((l >> 3) & 1)
+      const __nv_bfloat16* pa_l = sA + (lane & 15) * LDA + kq4 * (D / 4) + 8 * (lane >> 4);
+      const __nv_bfloat16* pb_l = sK + (size_t)min(16 * nh + (lane & 7) + 8 * (lane >> 4), NKH - 1) * LDA + kq4 * (D / 4) +
+                                  8 * ((lane >> 3) & 1);
 #pragma unroll
       for (int kk = 0; kk < KSW; ++kk) {
-        uint32_t a[4];
-        const __nv_bfloat16* ar = sA + g * LDA + (kq4 * KSW + kk) * 16 + 2 * tg;
-        a[0] = *reinterpret_cast<const uint32_t*>(ar);
-        a[1] = *reinterpret_cast<const uint32_t*>(ar + 8 * LDA);
-        a[2] = *reinterpret_cast<const uint32_t*>(ar + 8);
-        a[3] = *reinterpret_cast<const uint32_t*>(ar + 8 * LDA + 8);
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          if (8 * (2 * nh + u) < NKH) {
-            const uint32_t b0 = *reinterpret_cast<const uint32_t*>(pk[u] + kk * 16) & live[u];
-            const uint32_t b1 = *reinterpret_cast<const uint32_t*>(pk[u] + kk * 16 + 8) & live[u];
-            mma_bf16_16816(sc[u], a, b0, b1);
-          }
-        }
+        uint32_t a[4], b[4];
+        ldmatrix_x4(a, pa_l + kk * 16);
+        ldmatrix_x4(b, pb_l + kk * 16);
+        mma_bf16_16816(sc[0], a, b[0], b[1]);
+        mma_bf16_16816(sc[1], a, b[2], b[3]);
       }
     }
 #pragma unroll
@@ -367,13 +363,7 @@ xattn_fold_kernel(float* __restrict__ x, const __nv_bfloat16* __restrict__ delta
   {
     uint32_t pa[2][4];
 #pragma unroll
-    for (int k2 = 0; k2 < 2; ++k2) {
-      const __nv_bfloat16* ar = sP + g * LDP + k2 * 16 + 2 * tg;
-      pa[k2][0] = *reinterpret_cast<const uint32_t*>(ar);
-      pa[k2][1] = *reinterpret_cast<const uint32_t*>(ar + 8 * LDP);
-      pa[k2][2] = *reinterpret_cast<const uint32_t*>(ar + 8);
-      pa[k2][3] = *reinterpret_cast<const uint32_t*>(ar + 8 * LDP + 8);
-    }
+    for (int k2 = 0; k2 < 2; ++k2) ldmatrix_x4(pa[k2], sP + (lane & 15) * LDP + k2 * 16 + 8 * (lane >> 4));
     // B fragment (k2, rg) of a lane: memory-token/head pair row 8 k2 + 4 rg + tg of the u rows
     const uint32_t* pu[2][2];
     uint32_t ulive[2][2];
@@ -412,7 +402,7 @@ xattn_fold_kernel(float* __restrict__ x, const __nv_bfloat16* __restrict__ delta
       for (int j = 0; j < V; ++j) {
         const float4 t = *reinterpret_cast<const float4*>(sO + r * LDO + (j * 32 + lane) * 4);
         float4& e = xr[rr][j];
-        e.x += t.x + bb[j].x; e.y += t.y + bb[j].y; e.z += t.z + bb[j].z; e.w += t.w + bb[j].w;
+        e = xf_join(__fadd2_rn(xf_lo(e), __fadd2_rn(xf_lo(t), xf_lo(bb[j]))), __fadd2_rn(xf_hi(e), __fadd2_rn(xf_hi(t), xf_hi(bb[j]))));
         if (r < H) reinterpret_cast<float4*>(xc + (size_t)r * D)[j * 32 + lane] = e;
       }
     }
@@ -426,25 +416,27 @@ xattn_fold_kernel(float* __restrict__ x, const __nv_bfloat16* __restrict__ delta
 #pragma unroll
     for (int rr = 0; rr < 2; ++rr) {
       const int r = 2 * warp + rr;
-      float sm = 0.f;
+      float2 s2 = make_float2(0.f, 0.f);
 #pragma unroll
-      for (int j = 0; j < V; ++j) sm += (xr[rr][j].x + xr[rr][j].y) + (xr[rr][j].z + xr[rr][j].w);
-      const float mean = warp_sum(sm) / D;
-      float q = 0.f;
+      for (int j = 0; j < V; ++j) s2 = __fadd2_rn(s2, __fadd2_rn(xf_lo(xr[rr][j]), xf_hi(xr[rr][j])));
+      const float mean = warp_sum(s2.x + s2.y) / D;
+      const float2 nm = xf_dup(-mean);
+      float2 q2 = make_float2(0.f, 0.f);
+      float2 lo[V], hi[V];
 #pragma unroll
       for (int j = 0; j < V; ++j) {
-        float4& e = xr[rr][j];
-        e.x -= mean; e.y -= mean; e.z -= mean; e.w -= mean;
-        q += (e.x * e.x + e.y * e.y) + (e.z * e.z + e.w * e.w);
+        lo[j] = __fadd2_rn(xf_lo(xr[rr][j]), nm); hi[j] = __fadd2_rn(xf_hi(xr[rr][j]), nm);
+        q2 = __ffma2_rn(lo[j], lo[j], q2); q2 = __ffma2_rn(hi[j], hi[j], q2);
       }
-      const float rs = rsqrtf(warp_sum(q) / D + 1e-5f);
+      const float2 rs2 = xf_dup(rsqrtf(warp_sum(q2.x + q2.y) / D + 1e-5f));
       if (r < H) {
 #pragma unroll
         for (int j = 0; j < V; ++j) {
-          const float4 e = xr[rr][j];
+          const float2 a = __ffma2_rn(__fmul2_rn(lo[j], rs2), xf_lo(gg[j]), xf_lo(be[j]));
+          const float2 b = __ffma2_rn(__fmul2_rn(hi[j], rs2), xf_hi(gg[j]), xf_hi(be[j]));
           uint2 o2;
-          o2.x = pack_bf16(e.x * rs * gg[j].x + be[j].x, e.y * rs * gg[j].y + be[j].y);
-          o2.y = pack_bf16(e.z * rs * gg[j].z + be[j].z, e.w * rs * gg[j].w + be[j].w);
+          o2.x = pack_bf16(a.x, a.y);
+          o2.y = pack_bf16(b.x, b.y);
           reinterpret_cast<uint2*>(oc + (size_t)r * D)[j * 32 + lane] = o2;
         }
       }

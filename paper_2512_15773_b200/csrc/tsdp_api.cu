@@ -860,8 +860,9 @@ int cross_attn_ctx_launch(tsdp_ctx* c, const Net& n, const T* q2, T* out, const 
   if constexpr (std::is_same<T, __nv_bfloat16>::value) {
     // 64-wide heads and groups of at least two 128-row tiles (the verification forward: all candidates of a slot share
     // the keys / values a CTA fetched): both products on the 5th-generation tensor cores (ctx_attn_tcgen05.cuh).
-    // Measured on the VLA-scale workload: 7 % less attention time than the mma.sync kernel there, but slower for the
-    // drafter's single 50-row group per CTA, where fetching and re-laying-out K / V dominates; tc_attn = 2 forces it.
+    // Measured on the VLA-scale workload: a quarter less attention time than the mma.sync kernel there (55 vs 75 ms of
+    // the step), but no faster for the drafter's single 50-row group per CTA, where fetching and re-laying-out K / V
+    // dominates; tc_attn = 2 forces it.
     if (c->tc_attn && (cm.C * H >= 256 || c->tc_attn == 2) && dh == 64 && Tc % 32 == 0 && Tc <= 256 && n_cand % cm.C == 0 && d % 8 == 0) {
       const int slots = n_cand / cm.C, rows = cm.C * H;
       CUtensorMap mq, mkv;

@@ -121,15 +121,67 @@ __host__ __device__ inline DcSmem dc_smem_plan(int d, int layers, int A, bool re
 // Y[16, n_slice] = X[16, KD] * Wslice[n_slice, KD]^T.  Work units are (8-column tile, K part): with
 // fewer tiles than warps the K range is split and the parts are summed through shared memory.
 // `emit(row, col, v)` receives 8 adjacent columns (col a multiple of 8) of the finished slice.
-template <int KD, typename Emit>
-__device__ __forceinline__ void dc_linear(const __nv_bfloat16* X, int px, const __nv_bfloat16* W, int PW, int n_slice,
-                                          float* red, Emit emit) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int g = lane >> 2, tg = lane & 3;
-  const int n_tiles = n_slice >> 3;      // PW: row pitch of W (KD + 8 in shared memory, KD in global memory)
+__host__ __device__ constexpr int dc_ksplit(int KD, int n_tiles) {
   int ksplit = 1;
   while (n_tiles * ksplit * 2 <= DC_WARPS && (KD / 32) % (ksplit * 2) == 0) ksplit *= 2;     // parts of whole 32-k blocks
-  const int units = n_tiles * ksplit;
+  return ksplit;
+}
+template <int KD, int NSLICE, typename Emit>
+__device__ __forceinline__ void dc_linear(const __nv_bfloat16* X, int px, const __nv_bfloat16* W, int PW, float* red, Emit emit) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, tg = lane & 3;
+  constexpr int n_tiles = NSLICE >> 3;      // PW: row pitch of W (KD + 8 in shared memory, KD in global memory)
+  constexpr int ksplit = dc_ksplit(KD, n_tiles);
+  constexpr int units = n_tiles * ksplit;
+  if constexpr (ksplit == 1) {
+    // No K split: a warp owns whole tiles (tiles warp, warp + 8, ...), so it finishes them on its own and the warps
+    // run through the layer without meeting; one block barrier at the end.  All of a warp's tiles go through the k
+    // loop together -- the activations are read once and the weight loads of every tile are in flight at the same
+    // time -- then each is finished in turn: fragment to the warp's 16 x 8 patch of `red`, lanes 0..15 emit one row
+    // each (same sums in the same order as the split path with one part).
+    constexpr int TPW = (n_tiles + DC_WARPS - 1) / DC_WARPS;
+    float* r = red + (size_t)warp * (DC_ROWS * 8);
+    float c[TPW][4];
+#pragma unroll
+    for (int t = 0; t < TPW; ++t) { c[t][0] = c[t][1] = c[t][2] = c[t][3] = 0.f; }
+    const __nv_bfloat16* x0 = X + (size_t)g * px;
+    const __nv_bfloat16* x1 = X + (size_t)(g + 8) * px;
+#pragma unroll 8
+    for (int ks = 0; ks < KD / 16; ks += 2) {
+      const int k = ks * 16 + 8 * tg;
+      const uint4 xa = *reinterpret_cast<const uint4*>(x0 + k);
+      const uint4 xb = *reinterpret_cast<const uint4*>(x1 + k);
+      const uint32_t a1[4] = {xa.x, xb.x, xa.y, xb.y}, a2[4] = {xa.z, xb.z, xa.w, xb.w};
+      uint4 wv[TPW];
+#pragma unroll
+      for (int t = 0; t < TPW; ++t) {
+        const int nt = min(warp + t * DC_WARPS, n_tiles - 1);          // past the last tile: recomputed, not emitted
+        wv[t] = *reinterpret_cast<const uint4*>(W + (size_t)(nt * 8 + g) * PW + k);
+      }
+#pragma unroll
+      for (int t = 0; t < TPW; ++t) {
+        mma_bf16_16816(c[t], a1, wv[t].x, wv[t].y);
+        mma_bf16_16816(c[t], a2, wv[t].z, wv[t].w);
+      }
+    }
+#pragma unroll
+    for (int t = 0; t < TPW; ++t) {
+      const int nt = warp + t * DC_WARPS;
+      if (nt < n_tiles) {                                               // warp-uniform
+        r[g * 8 + 2 * tg] = c[t][0]; r[g * 8 + 2 * tg + 1] = c[t][1];
+        r[(g + 8) * 8 + 2 * tg] = c[t][2]; r[(g + 8) * 8 + 2 * tg + 1] = c[t][3];
+        __syncwarp();
+        if (lane < DC_ROWS) {
+          const float4* rp = reinterpret_cast<const float4*>(r + lane * 8);
+          const float4 lo = rp[0], hi = rp[1];
+          float v[8] = {0.f + lo.x, 0.f + lo.y, 0.f + lo.z, 0.f + lo.w, 0.f + hi.x, 0.f + hi.y, 0.f + hi.z, 0.f + hi.w};
+          emit(lane, nt * 8, v);
+        }
+        __syncwarp();
+      }
+    }
+    __syncthreads();
+  } else {
   for (int u0 = 0; u0 < units; u0 += DC_WARPS) {
     const int u = u0 + warp;
     if (u < units) {
@@ -144,7 +196,7 @@ __device__ __forceinline__ void dc_linear(const __nv_bfloat16* X, int px, const 
       // inside the block of 32 that A and B share, so the sum is unchanged while every load is one full
       // 16-byte access (four times fewer loads than the natural fragment layout; it matters most when the
       // weights come from the L2).
-#pragma unroll 4
+#pragma unroll 8
       for (int ks = ks0; ks < ks1; ks += 2) {
         const int k = ks * 16 + 8 * tg;
         const uint4 xa = *reinterpret_cast<const uint4*>(x0 + k);
@@ -177,6 +229,7 @@ __device__ __forceinline__ void dc_linear(const __nv_bfloat16* X, int px, const 
       emit(row, tile * 8, v);
     }
     __syncthreads();
+  }
   }
 }
 
@@ -519,7 +572,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
       dc_layernorm<d>(h, W.ln1_g, W.ln1_b, a, PA);
       __syncthreads();
       stage_begin(DC_ROWS * 3 * d * 2);
-      dc_linear<d>(a, PA, w_ptr(l, 0), PWD, NS_3D, red, [&](int row, int col, float* v) {
+      dc_linear<d, NS_3D>(a, PA, w_ptr(l, 0), PWD, red, [&](int row, int col, float* v) {
         const int cg_ = rank * NS_3D + col;
         const float4 b0 = *reinterpret_cast<const float4*>(W.bqkv + col), b1 = *(reinterpret_cast<const float4*>(W.bqkv + col) + 1);
         v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
@@ -568,7 +621,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         asm volatile("cp.async.commit_group;" ::: "memory");
       }
       stage_begin(DC_ROWS * d * 4);
-      dc_linear<d>(a, PA, w_ptr(l, 1), PWD, NS_D, red, [&](int row, int col, float* v) {
+      dc_linear<d, NS_D>(a, PA, w_ptr(l, 1), PWD, red, [&](int row, int col, float* v) {
         const int cg_ = rank * NS_D + col;
         const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
         const float4 h0 = hp[0], h1 = hp[1];
@@ -598,7 +651,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         for (int i = threadIdx.x; i < DC_ROWS * DC_PU / 2; i += DC_THREADS) reinterpret_cast<uint32_t*>(sP)[i] = 0u;
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         __syncthreads();
-        dc_linear<d>(a, PA, q2, PA, 16, red, [&](int row, int col, float* v) {
+        dc_linear<d, 16>(a, PA, q2, PA, red, [&](int row, int col, float* v) {
 #pragma unroll
           for (int j = 0; j < 8; ++j) sS[row * 16 + col + j] = v[j];
         });
@@ -625,7 +678,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         }
         __syncthreads();
         const float* bo2_full = pb + 6 * d + 11 * d / DC_CS;
-        dc_linear<32>(sP, DC_PU, qkv, DC_PU, d, red, [&](int row, int col, float* v) {
+        dc_linear<32, d>(sP, DC_PU, qkv, DC_PU, red, [&](int row, int col, float* v) {
           float4* hp4 = reinterpret_cast<float4*>(h + row * d + col);
           const float4 b0 = *reinterpret_cast<const float4*>(bo2_full + col), b1 = *(reinterpret_cast<const float4*>(bo2_full + col) + 1);
           float4 h0 = hp4[0], h1 = hp4[1];
@@ -638,7 +691,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
       dc_layernorm<d>(h, W.ln2_g, W.ln2_b, a, PA);
       __syncthreads();
       stage_begin(DC_ROWS * d * 2);
-      dc_linear<d>(a, PA, w_ptr(l, 2), PWD, NS_D, red, [&](int row, int col, float* v) {
+      dc_linear<d, NS_D>(a, PA, w_ptr(l, 2), PWD, red, [&](int row, int col, float* v) {
         const int cg_ = rank * NS_D + col;
         const float4 b0 = *reinterpret_cast<const float4*>(W.bq2 + col), b1 = *(reinterpret_cast<const float4*>(W.bq2 + col) + 1);
         v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
@@ -649,7 +702,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
       dc_attention<d, false>(q2, PA, nullptr, 0, skv + (size_t)(resident ? l : 0) * DC_MAX_NK * 2 * d, NK, a, PA, P.heads, H);
       __syncthreads();
       stage_begin(DC_ROWS * d * 4);
-      dc_linear<d>(a, PA, w_ptr(l, 3), PWD, NS_D, red, [&](int row, int col, float* v) {
+      dc_linear<d, NS_D>(a, PA, w_ptr(l, 3), PWD, red, [&](int row, int col, float* v) {
         const int cg_ = rank * NS_D + col;
         const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
         const float4 h0 = hp[0], h1 = hp[1];
@@ -665,7 +718,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
       dc_layernorm<d>(h, W.ln3_g, W.ln3_b, a, PA);
       __syncthreads();
       stage_begin(DC_ROWS * 4 * d * 2);
-      dc_linear<d>(a, PA, w_ptr(l, 4), PWD, NS_4D, red, [&](int row, int col, float* v) {
+      dc_linear<d, NS_4D>(a, PA, w_ptr(l, 4), PWD, red, [&](int row, int col, float* v) {
         const int cg_ = rank * NS_4D + col;
         const float4 b0 = *reinterpret_cast<const float4*>(W.b1 + col), b1 = *(reinterpret_cast<const float4*>(W.b1 + col) + 1);
         v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
@@ -677,7 +730,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
       });
       stage_end();
       stage_begin(DC_ROWS * d * 4);
-      dc_linear<4 * d>(f, PF, w_ptr(l, 5), PW4, NS_D, red, [&](int row, int col, float* v) {
+      dc_linear<4 * d, NS_D>(f, PF, w_ptr(l, 5), PW4, red, [&](int row, int col, float* v) {
         const int cg_ = rank * NS_D + col;
         const float4* hp = reinterpret_cast<const float4*>(h + row * d + cg_);
         const float4 h0 = hp[0], h1 = hp[1];

@@ -590,7 +590,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
       if (P.fold) {
         // the memory tokens' folded tables of this block start their way into shared memory now (the qkv buffer
         // is free until the next block, the q2 buffer is not used at all): kq rows with their constant in the
-        // row padding -> q2 buffer; u transposed to [output column][token, head] -> qkv buffer, pad columns zero
+        // row padding -> q2 buffer; u rows as they are stored (head pairs in one word) -> qkv buffer
         const int heads = P.heads, hp = heads >> 1, NKH = NK * heads;
         const size_t tok_stride = (size_t)L * heads * d, lay = (size_t)l * heads * d;
         for (int i = threadIdx.x; i < NKH * (d / 8); i += DC_THREADS) {
@@ -606,17 +606,13 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
                              (size_t)l * heads + hh;
           dc_cp_async<4>(q2 + n * PA + d, src);
         }
-        uint32_t* sU = reinterpret_cast<uint32_t*>(qkv);                    // [d][DC_PU / 2] words
-        for (int i = threadIdx.x; i < (NKH / 2) * d; i += DC_THREADS) {
-          const int pr = i / d, o = i - pr * d;
+        uint32_t* sU = reinterpret_cast<uint32_t*>(qkv);                    // [NKH / 2][d + 8] words: word (pair row, o) = u of heads 2q, 2q+1 at output column o
+        for (int i = threadIdx.x; i < (NKH / 2) * (d / 4); i += DC_THREADS) {
+          const int pr = i / (d / 4), ch = i - pr * (d / 4);
           const int j = pr / hp, q = pr - j * hp;
           const __nv_bfloat16* src = (j == 0 ? P.ut_time + (size_t)tau * tok_stride : P.ut_obs + ((size_t)env * P.To + (j - 1)) * tok_stride) +
-                                     lay + ((size_t)q * d + o) * 2;
-          dc_cp_async<4>(sU + o * (DC_PU / 2) + pr, src);
-        }
-        for (int i = threadIdx.x; i < d * (16 - NKH / 2); i += DC_THREADS) {
-          const int o = i / (16 - NKH / 2), w = NKH / 2 + i % (16 - NKH / 2);
-          sU[o * (DC_PU / 2) + w] = 0u;
+                                     lay + (size_t)q * d * 2 + ch * 8;
+          dc_cp_async<16>(sU + pr * (d + 8) + ch * 4, src);
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
       }
@@ -678,14 +674,49 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         }
         __syncthreads();
         const float* bo2_full = pb + 6 * d + 11 * d / DC_CS;
-        dc_linear<32, d>(sP, DC_PU, qkv, DC_PU, red, [&](int row, int col, float* v) {
-          float4* hp4 = reinterpret_cast<float4*>(h + row * d + col);
-          const float4 b0 = *reinterpret_cast<const float4*>(bo2_full + col), b1 = *(reinterpret_cast<const float4*>(bo2_full + col) + 1);
-          float4 h0 = hp4[0], h1 = hp4[1];
-          h0.x += v[0] + b0.x; h0.y += v[1] + b0.y; h0.z += v[2] + b0.z; h0.w += v[3] + b0.w;
-          h1.x += v[4] + b1.x; h1.y += v[5] + b1.y; h1.z += v[6] + b1.z; h1.w += v[7] + b1.w;
-          hp4[0] = h0; hp4[1] = h1;
-        });
+        {
+          // out = P . u: warp w the output columns [w d/8, (w+1) d/8), every row; a word of the u rows is one B
+          // fragment register (k = heads 2q, 2q+1 of a memory token), so nothing is transposed.  Each 16 x 8 tile
+          // leaves through the warp's patch of `red`: lanes 0..15 add one row each into the stream (own replica).
+          const int g = lane >> 2, tg = lane & 3;
+          const uint32_t* sU = reinterpret_cast<const uint32_t*>(qkv);
+          uint32_t pa[2][4];
+#pragma unroll
+          for (int k2 = 0; k2 < 2; ++k2) ldmatrix_x4(pa[k2], sP + (lane & 15) * DC_PU + k2 * 16 + 8 * (lane >> 4));
+          const uint32_t* pu[2][2];
+          uint32_t ulive[2][2];
+#pragma unroll
+          for (int k2 = 0; k2 < 2; ++k2)
+#pragma unroll
+            for (int rg = 0; rg < 2; ++rg) {
+              const int pr = 8 * k2 + 4 * rg + tg;
+              ulive[k2][rg] = 2 * pr < NKH ? 0xffffffffu : 0u;
+              pu[k2][rg] = sU + (size_t)min(pr, NKH / 2 - 1) * (d + 8) + g;
+            }
+          float* r = red + (size_t)warp * (DC_ROWS * 8);
+#pragma unroll
+          for (int nt = 0; nt < d / 64; ++nt) {
+            const int col = warp * (d / 8) + nt * 8;
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int k2 = 0; k2 < 2; ++k2)
+              if (16 * k2 < NKH) mma_bf16_16816(acc, pa[k2], pu[k2][0][col] & ulive[k2][0], pu[k2][1][col] & ulive[k2][1]);
+            r[g * 8 + 2 * tg] = acc[0]; r[g * 8 + 2 * tg + 1] = acc[1];
+            r[(g + 8) * 8 + 2 * tg] = acc[2]; r[(g + 8) * 8 + 2 * tg + 1] = acc[3];
+            __syncwarp();
+            if (lane < DC_ROWS) {
+              const float4* rp = reinterpret_cast<const float4*>(r + lane * 8);
+              const float4 v0 = rp[0], v1 = rp[1];
+              float4* hp4 = reinterpret_cast<float4*>(h + lane * d + col);
+              const float4 b0 = *reinterpret_cast<const float4*>(bo2_full + col), b1 = *(reinterpret_cast<const float4*>(bo2_full + col) + 1);
+              float4 h0 = hp4[0], h1 = hp4[1];
+              h0.x += v0.x + b0.x; h0.y += v0.y + b0.y; h0.z += v0.z + b0.z; h0.w += v0.w + b0.w;
+              h1.x += v1.x + b1.x; h1.y += v1.y + b1.y; h1.z += v1.z + b1.z; h1.w += v1.w + b1.w;
+              hp4[0] = h0; hp4[1] = h1;
+            }
+            __syncwarp();
+          }
+        }
         __syncthreads();
       } else {
       dc_layernorm<d>(h, W.ln2_g, W.ln2_b, a, PA);

@@ -437,7 +437,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
     const uint32_t la = ptx::smem_u32(local_ptr);
     if (use_async) {
       const uint32_t lb = bar_addr[stage_no & 1u];
-#pragma unroll 1
+#pragma unroll
       for (uint32_t r = 0; r < DC_CS; ++r) dc_st_async16(dc_mapa(la, r), v, dc_mapa(lb, r));
     } else {
 #pragma unroll 1
@@ -676,8 +676,7 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
         const float* bo2_full = pb + 6 * d + 11 * d / DC_CS;
         {
           // out = P . u: warp w the output columns [w d/8, (w+1) d/8), every row; a word of the u rows is one B
-          // fragment register (k = heads 2q, 2q+1 of a memory token), so nothing is transposed.  Each 16 x 8 tile
-          // leaves through the warp's patch of `red`: lanes 0..15 add one row each into the stream (own replica).
+          // fragment register (k = heads 2q, 2q+1 of a memory token), so nothing is transposed.
           const int g = lane >> 2, tg = lane & 3;
           const uint32_t* sU = reinterpret_cast<const uint32_t*>(qkv);
           uint32_t pa[2][4];
@@ -693,7 +692,6 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
               ulive[k2][rg] = 2 * pr < NKH ? 0xffffffffu : 0u;
               pu[k2][rg] = sU + (size_t)min(pr, NKH / 2 - 1) * (d + 8) + g;
             }
-          float* r = red + (size_t)warp * (DC_ROWS * 8);
 #pragma unroll
           for (int nt = 0; nt < d / 64; ++nt) {
             const int col = warp * (d / 8) + nt * 8;
@@ -701,20 +699,13 @@ drafter_cluster_kernel(const __grid_constant__ DcParams P) {
 #pragma unroll
             for (int k2 = 0; k2 < 2; ++k2)
               if (16 * k2 < NKH) mma_bf16_16816(acc, pa[k2], pu[k2][0][col] & ulive[k2][0], pu[k2][1][col] & ulive[k2][1]);
-            r[g * 8 + 2 * tg] = acc[0]; r[g * 8 + 2 * tg + 1] = acc[1];
-            r[(g + 8) * 8 + 2 * tg] = acc[2]; r[(g + 8) * 8 + 2 * tg + 1] = acc[3];
-            __syncwarp();
-            if (lane < DC_ROWS) {
-              const float4* rp = reinterpret_cast<const float4*>(r + lane * 8);
-              const float4 v0 = rp[0], v1 = rp[1];
-              float4* hp4 = reinterpret_cast<float4*>(h + lane * d + col);
-              const float4 b0 = *reinterpret_cast<const float4*>(bo2_full + col), b1 = *(reinterpret_cast<const float4*>(bo2_full + col) + 1);
-              float4 h0 = hp4[0], h1 = hp4[1];
-              h0.x += v0.x + b0.x; h0.y += v0.y + b0.y; h0.z += v0.z + b0.z; h0.w += v0.w + b0.w;
-              h1.x += v1.x + b1.x; h1.y += v1.y + b1.y; h1.z += v1.z + b1.z; h1.w += v1.w + b1.w;
-              hp4[0] = h0; hp4[1] = h1;
-            }
-            __syncwarp();
+            // every CTA updates its own replica of the stream: straight from the fragment, two columns per lane and row
+            const float2 b2 = *reinterpret_cast<const float2*>(bo2_full + col + 2 * tg);
+            float2* h0 = reinterpret_cast<float2*>(h + g * d + col + 2 * tg);
+            float2* h1 = reinterpret_cast<float2*>(h + (g + 8) * d + col + 2 * tg);
+            float2 a0 = *h0, a1 = *h1;
+            a0.x += acc[0] + b2.x; a0.y += acc[1] + b2.y; a1.x += acc[2] + b2.x; a1.y += acc[3] + b2.y;
+            *h0 = a0; *h1 = a1;
           }
         }
         __syncthreads();

@@ -293,6 +293,13 @@ struct GemmArgs {
   // `status`, drains and returns; every other CTA finishes its tiles as usual.
   int withhold_first_stage;
   int causal;           // EPI_ATTN: causal mask of the fused 16-token self-attention
+  // Split reduction (narrow tiles with the plain-store epilogue, EPI_F32 only; 0 or 1: off): the k-blocks of every
+  // tile are cut into `ksplit` contiguous parts, each a work unit of its own whose partial sums go to the buffer
+  // out + part * split_stride (elements); the bias goes into part 0.  The consumer adds the parts in a fixed order,
+  // so the result does not depend on which CTA ran which part.  For deep reductions over few rows (the convolutions
+  // of a small batch), where the tiles alone occupy a fraction of the SMs.
+  int ksplit;
+  long long split_stride;
 };
 
 __device__ __forceinline__ const float* gate_row(const GemmArgs& g, int row) {
@@ -304,12 +311,13 @@ __device__ __forceinline__ const float* gate_row(const GemmArgs& g, int row) {
 
 // `bias16`: the 16 bias values of these columns (fetched by the caller before it waited for the accumulator).
 template <int EPI>
-__device__ __forceinline__ void epilogue_store16(const GemmArgs& g, int row, int col, const uint32_t v[16], const float* bias16) {
+__device__ __forceinline__ void epilogue_store16(const GemmArgs& g, int row, int col, const uint32_t v[16], const float* bias16,
+                                                 bool add_bias = true, size_t out_off = 0) {
   float f[16];
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
     f[i] = __uint_as_float(v[i]);
-    if (g.bias) f[i] += bias16[i];
+    if (g.bias && add_bias) f[i] += bias16[i];
     if (EPI == EPI_GELU) f[i] = ptx::gelu_fast(f[i]);
   }
   if (EPI == EPI_GATE) {
@@ -329,7 +337,7 @@ __device__ __forceinline__ void epilogue_store16(const GemmArgs& g, int row, int
     reinterpret_cast<uint4*>(o)[0] = p[0];
     reinterpret_cast<uint4*>(o)[1] = p[1];
   } else {
-    float* o = reinterpret_cast<float*>(g.out) + (size_t)row * g.ldo + col;
+    float* o = reinterpret_cast<float*>(g.out) + out_off + (size_t)row * g.ldo + col;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       float4 r = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
@@ -403,7 +411,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   pdl_wait();      // operands, bias, the output and the live-row count belong to earlier kernels of the stream
   const int M = live_rows(g.live, g.M);
   const int tiles_m = (M + GEMM_BM * CG - 1) / (GEMM_BM * CG);     // tiles of 128 CG rows
-  const int n_tiles = tiles_m * tiles_n;
+  const int S = g.ksplit > 1 ? g.ksplit : 1;                       // parts of the reduction (plain-store epilogue only)
+  const int n_tiles = tiles_m * tiles_n * S;                       // work units: (tile, part), part fastest
   const int tile0 = blockIdx.x / CG, tile_step = gridDim.x / CG;      // both CTAs of a pair walk the same tiles
   // an epilogue warp hands accumulator buffer `as` back: the barrier that the MMA warp waits on lives in the leader
   auto release_acc = [&](int as) {
@@ -414,11 +423,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   if (warp == 0) {
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
-      for (int tile = tile0; tile < n_tiles && ok; tile += tile_step) {
+      for (int unit = tile0; unit < n_tiles && ok; unit += tile_step) {
+        const int tile = unit / S, part = unit - tile * S;
         const int tm = (tile / tiles_n) * CG + (int)rank, tn = tile % tiles_n;
-        for (int kb = 0; kb < kblocks; ++kb) {
+        const int kb0 = part * kblocks / S, kb1 = (part + 1) * kblocks / S;
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!ptx::mbar_wait_thread(empty_bar(stage), phase ^ 1u, wlim)) { ok = false; break; }
-          if (!(g.withhold_first_stage && blockIdx.x == 0 && tile == 0 && kb == 0)) {
+          if (!(g.withhold_first_stage && blockIdx.x == 0 && unit == 0 && kb == 0)) {
             const uint32_t sa = base + stage * STAGE_BYTES;
             const int kcol = kb * GEMM_BK;
             const int ax = g.conv_c ? kcol % g.conv_c : kcol, ay = tm * GEMM_BM + (g.conv_c ? kcol / g.conv_c : 0);
@@ -441,20 +452,22 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   } else if (warp == 1) {
     if (lane == 0 && rank == 0) {      // in a pair only the leader issues
       int stage = 0; uint32_t phase = 0; int it = 0;
-      for (int tile = tile0; tile < n_tiles && ok; tile += tile_step, ++it) {
+      for (int unit = tile0; unit < n_tiles && ok; unit += tile_step, ++it) {
+        const int part = unit % S;
+        const int kb0 = part * kblocks / S, kb1 = (part + 1) * kblocks / S;
         const int as = it & 1; const uint32_t aphase = (it >> 1) & 1;
         if (!ptx::mbar_wait_thread(tempty_bar(as), aphase ^ 1u, wlim)) { ok = false; break; }
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(as * ACC);
-        for (int kb = 0; kb < kblocks; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!ptx::mbar_wait_thread(full_bar(stage), phase, wlim)) { ok = false; break; }
           ptx::tc_fence_after();
           const uint32_t sa = base + stage * STAGE_BYTES;
           const uint64_t da = umma_desc_sw128(sa), db = umma_desc_sw128(sa + A_BYTES);
 #pragma unroll
           for (int k = 0; k < GEMM_BK / 16; ++k) {
-            if (CG == 2) ptx::tc_mma_bf16_pair(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), IDESC, (kb | k) ? 1u : 0u);
-            else ptx::tc_mma_bf16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), IDESC, (kb | k) ? 1u : 0u);
+            if (CG == 2) ptx::tc_mma_bf16_pair(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), IDESC, (kb > kb0 || k) ? 1u : 0u);
+            else ptx::tc_mma_bf16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), IDESC, (kb > kb0 || k) ? 1u : 0u);
           }
           if (CG == 2) ptx::tc_commit_pair(empty_bar(stage)); else ptx::tc_commit(empty_bar(stage));
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -669,7 +682,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       }
       if (issuer) ptx::bulk_wait_read0();
     } else {
-      for (int tile = tile0; tile < n_tiles && ok; tile += tile_step, ++it) {
+      for (int unit = tile0; unit < n_tiles && ok; unit += tile_step, ++it) {
+        const int tile = unit / S, part = unit - tile * S;
         const int tm = (tile / tiles_n) * CG + (int)rank, tn = tile % tiles_n;
         const int as = it & 1; const uint32_t aphase = (it >> 1) & 1;
         float bv[COLS];          // this half's bias values (narrow tiles: at most 32), fetched while the accumulator is awaited
@@ -689,7 +703,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           uint32_t v[16];
           ptx::tmem_ld16(taddr + (uint32_t)c, v);
           ptx::tmem_ld_wait();
-          if (row < M) epilogue_store16<EPI>(g, row, tn * BN + half * COLS + c, v, bv + c);
+          if (row < M) epilogue_store16<EPI>(g, row, tn * BN + half * COLS + c, v, bv + c, part == 0, (size_t)part * (size_t)g.split_stride);
         }
         ptx::tc_fence_before();
         __syncwarp();

@@ -76,7 +76,7 @@ struct Net {
   // UNET activations (zero-padded channels-last tensors, see unet_kernels.cuh), allocated at init
   struct UWs { void *X0 = nullptr, *E = nullptr, *M1 = nullptr, *M2 = nullptr, *HB = nullptr;
                void *TMP[4] = {}, *D[4] = {}, *CAT[4] = {}, *P[4] = {}, *U1[4] = {}, *U2[4] = {};
-               float *Y = nullptr, *R = nullptr; } uw;
+               float *Y = nullptr, *R = nullptr; size_t Y_cap = 0; } uw;
   std::vector<void*> allocs;
 };
 
@@ -364,7 +364,7 @@ int gemm_rows_known(const tsdp_ctx* c, const GemmArgs& g) {
 template <int BN, int EPI>
 int launch_tc(tsdp_ctx* c, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const GemmArgs& g,
               cudaStream_t s) {
-  const int tiles = ((g.M + GEMM_BM - 1) / GEMM_BM) * (g.N / BN);
+  const int tiles = ((g.M + GEMM_BM - 1) / GEMM_BM) * (g.N / BN) * (g.ksplit > 1 ? g.ksplit : 1);
   const int grid = tiles < c->num_sms ? tiles : c->num_sms;
   prof_begin(c, s, c->prof_gemm_cat, 2.0 * gemm_rows_known(c, g) * g.N * g.K);
   TSDP_LAUNCH(c, (gemm_tcgen05_kernel<BN, EPI>), grid, GEMM_THREADS, gemm_smem_bytes(BN), s, ma, mb, mc, g);
@@ -451,13 +451,30 @@ int pick_bn(int M, int N, int num_sms) {
   return 0;
 }
 
+// Parts into which the reduction of a convolution GEMM [M x N x K] -> fp32 is split (1: not at all).  With a small batch
+// the deep levels of the UNet are a handful of narrow tiles (16 - 32 CTAs) that each walk 80 - 160 k-blocks one after the
+// other: cutting the k range puts those k-blocks on otherwise idle SMs, each part writes its partial sums to a buffer
+// of its own and the GroupNorm kernel that consumes them adds the parts in order (same bits whatever ran where; a
+// function of the launch shape only).  Parts of at least 4 k-blocks, at most 8 parts, no more units than SMs, and
+// only where the tiles use the plain-store epilogue (widths below 128).
+int conv_ksplit(const tsdp_ctx* c, int M, int N, int K, size_t cap_elems) {
+  if (c->cfg.precision == 0 || M <= 0 || K % GEMM_BK != 0 || N % 32 != 0) return 1;
+  if (c->force_bn == 0 && use_pair_gemm(c, M, N, K)) return 1;
+  const int BN = (c->force_bn > 0 && N % c->force_bn == 0) ? c->force_bn : pick_bn(M, N, c->num_sms);
+  if (gemm_tma_epilogue(BN)) return 1;
+  const int tiles = ((M + GEMM_BM - 1) / GEMM_BM) * (N / BN), kblocks = K / GEMM_BK;
+  int S = 1;
+  while (S < 8 && tiles * S * 2 <= c->num_sms && kblocks / (S * 2) >= 4 && (size_t)(S * 2) * (size_t)(M + 4) * (size_t)N <= cap_elems) S *= 2;
+  return S;
+}
+
 // Gate of an adaptive-LayerNorm residual (EPI_GATE): gate vectors and the row -> timestep map.
 struct GateSpec {
   const float* gate; int gate_ld; const CandMap* cm; int H, Tsteps;
 };
 
 int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, int N, int K, int epi, void* out,
-         int ldo, cudaStream_t s, const GateSpec* gs = nullptr, int conv_c = 0) {
+         int ldo, cudaStream_t s, const GateSpec* gs = nullptr, int conv_c = 0, int ksplit = 1, long long split_stride = 0) {
   if (M <= 0) return TSDP_OK;
   GemmArgs g{M, N, K, bias, out, ldo, c->status, nullptr, 0, nullptr, 1, 0, 1, 1, conv_c > 0 ? conv_c : K, conv_c,
              LiveRows{nullptr, 0, 0}, nullptr, 0, 0, 0};
@@ -499,6 +516,10 @@ int gemm(tsdp_ctx* c, const void* A, const void* W, const float* bias, int M, in
   }
   const bool pair = c->force_bn == 0 && use_pair_gemm(c, M, N, K);
   const int BN = pair ? 256 : ((c->force_bn > 0 && N % c->force_bn == 0) ? c->force_bn : pick_bn(M, N, c->num_sms));
+  if (ksplit > 1) {      // see conv_ksplit: narrow tiles with the plain-store epilogue only
+    if (pair || gemm_tma_epilogue(BN) || epi != EPI_F32 || ksplit > K / GEMM_BK) return TSDP_ERR_ARG;
+    g.ksplit = ksplit; g.split_stride = split_stride;
+  }
   CUtensorMap ma, mb, mc;
   int r;
   if (conv_c > 0) {      // kernel-5 convolution: A is the padded tensor [M + 4, conv_c] itself
@@ -962,11 +983,12 @@ int dit_prepare_ctx_t(tsdp_ctx* c, Net& n, int B, cudaStream_t s) {
 // ------------------------------------------------------------------------------------------ conv UNet
 template <typename T>
 int unet_gn(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, const float* gam, const float* bet, int foff, const T* res_t,
-            int res_pitch, const float* res_f, T* dst, int dst_pitch, int coff, int L, int C, cudaStream_t s) {
+            int res_pitch, const float* res_f, T* dst, int dst_pitch, int coff, int L, int C, cudaStream_t s, int n_split = 1,
+            long long split_stride = 0) {
   prof_begin(c, s, 1, 0.0);
   TSDP_LAUNCH(c, (gn_mish_kernel<T>), n_cand * n.cfg.heads, 256, 0, s, n.uw.Y, gam, bet, n.cfg.heads,
               foff >= 0 ? n.film_time : nullptr, n.film_obs, n.F, foff >= 0 ? foff : 0, cm, c->cfg.T, res_t, res_pitch, res_f, dst,
-              dst_pitch, coff, L, C);
+              dst_pitch, coff, L, C, n_split, split_stride);
   prof_end(c, s);
   c->launches_per_round_tmp++;
   CU_TRY(c, cudaGetLastError());
@@ -979,14 +1001,16 @@ int unet_resblock(tsdp_ctx* c, Net& n, const Net::UBlock& b, const CandMap& cm, 
                   int dst_pitch, int coff, int L, cudaStream_t s) {
   const int rows = n_cand * (L + 4);
   int r;
-  if ((r = gemm(c, xin, b.W1, b.b1, rows - 4, b.cout, 5 * b.cin, EPI_F32, n.uw.Y, b.cout, s, nullptr, b.cin))) return r;
-  if ((r = unet_gn<T>(c, n, cm, n_cand, b.g1, b.be1, b.foff, nullptr, 0, nullptr, tmp, b.cout, 0, L, b.cout, s))) return r;
-  if ((r = gemm(c, tmp, b.W2, b.b2, rows - 4, b.cout, 5 * b.cout, EPI_F32, n.uw.Y, b.cout, s, nullptr, b.cout))) return r;
+  const long long ystr = (long long)rows * b.cout;      // distance of the partial-sum buffers of a split reduction
+  const int s1 = conv_ksplit(c, rows - 4, b.cout, 5 * b.cin, n.uw.Y_cap), s2 = conv_ksplit(c, rows - 4, b.cout, 5 * b.cout, n.uw.Y_cap);
+  if ((r = gemm(c, xin, b.W1, b.b1, rows - 4, b.cout, 5 * b.cin, EPI_F32, n.uw.Y, b.cout, s, nullptr, b.cin, s1, ystr))) return r;
+  if ((r = unet_gn<T>(c, n, cm, n_cand, b.g1, b.be1, b.foff, nullptr, 0, nullptr, tmp, b.cout, 0, L, b.cout, s, s1, ystr))) return r;
+  if ((r = gemm(c, tmp, b.W2, b.b2, rows - 4, b.cout, 5 * b.cout, EPI_F32, n.uw.Y, b.cout, s, nullptr, b.cout, s2, ystr))) return r;
   if (b.Wr) {
     if ((r = gemm(c, xin, b.Wr, b.br, rows, b.cout, b.cin, EPI_F32, n.uw.R, b.cout, s))) return r;
-    return unet_gn<T>(c, n, cm, n_cand, b.g2, b.be2, -1, nullptr, 0, n.uw.R, dst, dst_pitch, coff, L, b.cout, s);
+    return unet_gn<T>(c, n, cm, n_cand, b.g2, b.be2, -1, nullptr, 0, n.uw.R, dst, dst_pitch, coff, L, b.cout, s, s2, ystr);
   }
-  return unet_gn<T>(c, n, cm, n_cand, b.g2, b.be2, -1, xin, b.cin, nullptr, dst, dst_pitch, coff, L, b.cout, s);
+  return unet_gn<T>(c, n, cm, n_cand, b.g2, b.be2, -1, xin, b.cin, nullptr, dst, dst_pitch, coff, L, b.cout, s, s2, ystr);
 }
 
 template <typename T>
@@ -1037,8 +1061,10 @@ int unet_forward_t(tsdp_ctx* c, Net& n, const CandMap& cm, int n_cand, cudaStrea
     cur = P(n.uw.U2[lv]);
   }
   const int rows = n_cand * (H + 4);
-  if ((r = gemm(c, cur, n.Wh, n.bh, rows - 4, ch, 5 * ch, EPI_F32, n.uw.Y, ch, s, nullptr, ch))) return r;
-  if ((r = unet_gn<T>(c, n, cm, n_cand, n.gh, n.beh, -1, nullptr, 0, nullptr, P(n.uw.HB), ch, 0, H, ch, s))) return r;
+  const long long ystr = (long long)rows * ch;
+  const int sh = conv_ksplit(c, rows - 4, ch, 5 * ch, n.uw.Y_cap);
+  if ((r = gemm(c, cur, n.Wh, n.bh, rows - 4, ch, 5 * ch, EPI_F32, n.uw.Y, ch, s, nullptr, ch, sh, ystr))) return r;
+  if ((r = unet_gn<T>(c, n, cm, n_cand, n.gh, n.beh, -1, nullptr, 0, nullptr, P(n.uw.HB), ch, 0, H, ch, s, sh, ystr))) return r;
   prof_begin(c, s, 3, 0.0);
   TSDP_LAUNCH(c, (unet_head_kernel<T>), (n_cand * H + 7) / 8, 256, 0, s, P(n.uw.HB), n.W_outT, n.b_out, cm, n_cand * H, H, A, ch);
   prof_end(c, s);
@@ -1607,7 +1633,8 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
         e |= pad(&n.uw.U1[lv], lv, ch << lv); e |= pad(&n.uw.U2[lv], lv, ch << lv);
       }
     }
-    e |= dev_alloc(c, c->allocs, &n.uw.Y, nc * (cfg->H + 4) * (ch << last));
+    n.uw.Y_cap = 4 * nc * (cfg->H + 4) * (ch << last);      // room for the partial sums of a split reduction (conv_ksplit)
+    e |= dev_alloc(c, c->allocs, &n.uw.Y, n.uw.Y_cap);
     e |= dev_alloc(c, c->allocs, &n.uw.R, nc * (cfg->H + 4) * (ch << last));
     if (e) return fail(TSDP_ERR_CUDA);
   }

@@ -55,18 +55,25 @@ __global__ void __launch_bounds__(256)
 gn_mish_kernel(const float* __restrict__ Y, const float* __restrict__ gam, const float* __restrict__ bet, int groups,
                const float* __restrict__ film_time, const float* __restrict__ film_obs, int F, int foff, CandMap cm,
                int Tsteps, const T* __restrict__ res_t, int res_pitch, const float* __restrict__ res_f,
-               T* __restrict__ dst, int dst_pitch, int coff, int L, int C) {
+               T* __restrict__ dst, int dst_pitch, int coff, int L, int C, int n_split, long long split_stride) {
   pdl_trigger();
   pdl_wait();
   __shared__ float red[2][8];
+  // Y may arrive as n_split partial sums of the convolution's reduction, split_stride elements apart: added here in
+  // the order of the parts, whichever CTA produced which
+  auto y_at = [&](size_t idx) {
+    float v = Y[idx];
+    for (int sp = 1; sp < n_split; ++sp) v += Y[idx + (size_t)sp * (size_t)split_stride];
+    return v;
+  };
   const int n = blockIdx.x / groups, grp = blockIdx.x % groups;
   if (n >= cand_count(cm, gridDim.x / groups)) return;
   const int Cg = C / groups, Lp = L + 4;
   const int cnt = L * Cg;
-  const float* y0 = Y + (size_t)n * Lp * C + (size_t)grp * Cg;
+  const size_t y0 = (size_t)n * Lp * C + (size_t)grp * Cg;
   float s = 0.f, q = 0.f;
   for (int i = threadIdx.x; i < cnt; i += blockDim.x) {
-    const float v = y0[(size_t)(i / Cg) * C + (i % Cg)];
+    const float v = y_at(y0 + (size_t)(i / Cg) * C + (i % Cg));
     s += v; q += v * v;
   }
   s = warp_sum(s); q = warp_sum(q);
@@ -87,7 +94,7 @@ gn_mish_kernel(const float* __restrict__ Y, const float* __restrict__ gam, const
   }
   for (int i = threadIdx.x; i < cnt; i += blockDim.x) {
     const int l = i / Cg, c = grp * Cg + (i % Cg);
-    float v = (Y[((size_t)n * Lp + l) * C + c] - mean) * rstd * gam[c] + bet[c];
+    float v = (y_at(((size_t)n * Lp + l) * C + c) - mean) * rstd * gam[c] + bet[c];
     v = mish_f(v);
     if (ft) v = (ft[c] + fo[c]) * v + (ft[C + c] + fo[C + c]);
     const size_t prow = (size_t)n * Lp + l + 2;

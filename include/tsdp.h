@@ -33,6 +33,9 @@
  * self-attention as a kernel of its own instead of the QKV projection's epilogue; TSDP_NO_TC_ATTN keeps the context
  * cross-attention of TSDP_ARCH_DIT on the mma.sync kernel, TSDP_TC_ATTN=2 puts it on the tcgen05 kernel for every
  * group size (default: groups of at least 256 query rows, 64-wide heads, obs_tokens a multiple of 32 and <= 256);
+ * TSDP_NO_KSPLIT keeps the convolution GEMMs of TSDP_ARCH_UNET from splitting their reduction over idle SMs at small
+ * batch (the split changes the order of the fp32 sums, so the last bits of a result depend on it; for a given
+ * batch shape the result is the same on every run);
  * TSDP_VERBOSE prints the kernels' occupancy figures once per tsdp_load_weights.
  * Every function returns a tsdp_status; nothing throws or aborts.  A context is not re-entrant: one
  * call at a time.  There is no CPU fallback: without a CUDA device tsdp_init fails with TSDP_ERR_CUDA.

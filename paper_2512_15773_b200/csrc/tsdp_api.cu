@@ -138,6 +138,7 @@ struct tsdp_ctx {
   int tc_attn = 1;                            // context cross-attention on tcgen05: 0 never (TSDP_NO_TC_ATTN), 1 large groups, 2 always (TSDP_TC_ATTN=2)
   bool async_bcast = true;                    // cluster kernel: st.async + mbarrier stage hand-over (TSDP_NO_ASYNC_BCAST unset)
   bool dc_ok = false;
+  bool no_ksplit = false;                      // TSDP_NO_KSPLIT: convolution GEMMs never split their reduction
   int dc_smem = 0, dc_max_clusters = 0;
   bool dc_resident = false;
   // the same cluster kernel running the BASE model's verification forward (small batches of small transformers)
@@ -458,7 +459,7 @@ int pick_bn(int M, int N, int num_sms) {
 // function of the launch shape only).  Parts of at least 4 k-blocks, at most 8 parts, no more units than SMs, and
 // only where the tiles use the plain-store epilogue (widths below 128).
 int conv_ksplit(const tsdp_ctx* c, int M, int N, int K, size_t cap_elems) {
-  if (c->cfg.precision == 0 || M <= 0 || K % GEMM_BK != 0 || N % 32 != 0) return 1;
+  if (c->no_ksplit || c->cfg.precision == 0 || M <= 0 || K % GEMM_BK != 0 || N % 32 != 0) return 1;
   if (c->force_bn == 0 && use_pair_gemm(c, M, N, K)) return 1;
   const int BN = (c->force_bn > 0 && N % c->force_bn == 0) ? c->force_bn : pick_bn(M, N, c->num_sms);
   if (gemm_tma_epilogue(BN)) return 1;
@@ -1427,6 +1428,7 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   c->pdl = getenv("TSDP_NO_PDL") == nullptr;
   c->async_bcast = getenv("TSDP_NO_ASYNC_BCAST") == nullptr;
   c->compact = getenv("TSDP_NO_COMPACT") == nullptr;
+  c->no_ksplit = getenv("TSDP_NO_KSPLIT") != nullptr;
   c->tc_attn = getenv("TSDP_NO_TC_ATTN") != nullptr ? 0 : (getenv("TSDP_TC_ATTN") != nullptr ? atoi(getenv("TSDP_TC_ATTN")) : 1);
   if (const char* fb = getenv("TSDP_GEMM_BN")) {      // tuning aid: one tile width for every GEMM it divides
     const int v = atoi(fb);

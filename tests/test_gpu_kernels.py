@@ -186,6 +186,36 @@ def test_unet_denoiser(precision, tol, shape):
     smp.close()
 
 
+def test_unet_split_reduction_is_reproducible_and_matches_the_unsplit_sums(monkeypatch):
+    """At small batch the convolution GEMMs cut their reduction into parts that run on otherwise idle SMs; the
+    GroupNorm kernel adds the partial sums in a fixed order.  So two runs must agree bit for bit, and against the
+    same forward with the split switched off (other summation order) the difference must stay at rounding level."""
+    wl = dict(H=16, A=10, To=2, Do=24, T=100, precision=1, gamma=1.0,
+              base=dict(arch="unet", layers=3, d=128, heads=8, temb=64), draft=dict(arch="xfmr", layers=1, d=128, heads=4))
+    rng = np.random.default_rng(9)
+    N = 3
+    x = rng.normal(size=(N, wl["H"], wl["A"])).astype(np.float32)
+    tau = np.array([5, 50, 99], dtype=np.int32)
+    obs = inputs.make_obs(6, N, wl["To"], wl["Do"])
+    outs = []
+    for split in (True, True, False):
+        if split:
+            monkeypatch.delenv("TSDP_NO_KSPLIT", raising=False)
+        else:
+            monkeypatch.setenv("TSDP_NO_KSPLIT", "1")
+        smp, S, base, draft = hp.setup(wl, max_B=N, max_K=1)
+        dx = torch.tensor(x, device="cuda"); dobs = torch.tensor(obs, dtype=torch.float32, device="cuda")
+        out = torch.zeros_like(dx)
+        smp.denoise(binding.BASE, dx, tau, dobs, N, out)
+        launches = smp.kernel_launches()
+        outs.append(out.cpu().numpy().copy())
+        smp.close()
+    assert np.array_equal(outs[0], outs[1])                       # same split, same bits
+    ref = np.stack([base(x[n].astype(np.float64), int(tau[n]), obs[n]) for n in range(N)])
+    assert hp.max_rel(outs[0], ref) < 2e-2 and hp.max_rel(outs[2], ref) < 2e-2
+    assert hp.max_rel(outs[0], outs[2]) < 2e-2 and not np.array_equal(outs[0], outs[2])   # the split really was taken
+
+
 def test_gemm_bounded_wait_runs_out_and_the_context_recovers():
     """Failure detection without a fault: one CTA of the tensor-core GEMM is starved of an operand tile (a barrier
     that nothing completes) with the wait limit lowered to about a millisecond.  The kernel must return by giving up

@@ -207,7 +207,6 @@ def test_unet_split_reduction_is_reproducible_and_matches_the_unsplit_sums(monke
         dx = torch.tensor(x, device="cuda"); dobs = torch.tensor(obs, dtype=torch.float32, device="cuda")
         out = torch.zeros_like(dx)
         smp.denoise(binding.BASE, dx, tau, dobs, N, out)
-        launches = smp.kernel_launches()
         outs.append(out.cpu().numpy().copy())
         smp.close()
     assert np.array_equal(outs[0], outs[1])                       # same split, same bits

@@ -115,6 +115,29 @@ def test_robomimic_unet_at_full_width_sampled_candidates():
     smp.close()
 
 
+def test_robomimic_unet_at_full_width_batch_one_split_reduction():
+    """The same UNet at the row counts of a batch-1 round (9 candidates = 180 / 108 / 72 padded rows per level): every
+    level is one or two row tiles, so the convolution GEMMs split their K = 1280 .. 7680 reductions into parts that
+    run on otherwise idle SMs and the GroupNorm kernel adds the partial sums.  Every candidate against the oracle."""
+    wl = dict(inputs.WORKLOADS["robomimic_unet"], gamma=1.0)
+    N = 9
+    smp, S, base, draft = hp.setup(wl, max_B=N, max_K=1)
+    rng = np.random.default_rng(13)
+    x = rng.normal(size=(N, wl["H"], wl["A"])).astype(np.float32)
+    tau = rng.integers(0, 100, size=N).astype(np.int32)
+    tau[:2] = [99, 0]
+    obs = inputs.make_obs(9, N, wl["To"], wl["Do"])
+    dx = torch.tensor(x, device="cuda"); dobs = torch.tensor(obs, dtype=torch.float32, device="cuda")
+    out = torch.zeros_like(dx)
+    smp.denoise(binding.BASE, dx, tau, dobs, N, out)
+    got = out.cpu().numpy()
+    assert np.isfinite(got).all()
+    for n in (0, 1, 4, 8):
+        ref = base(x[n].astype(np.float64), int(tau[n]), obs[n])
+        assert hp.max_rel(got[n], ref) < 2e-2, n
+    smp.close()
+
+
 def _round_sampled(wl, B, K, seed, t0s, envs, acc=None):
     """One round at full width from random states; the listed environments are recomputed by the oracle."""
     acc = acc or hp.accept_t()

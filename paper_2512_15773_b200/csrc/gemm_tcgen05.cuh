@@ -18,7 +18,8 @@
 //               columns store straight from registers.  The second accumulator buffer lets the
 //               next tile's MMAs overlap this tile's epilogue.
 // Every mbarrier wait is bounded: on expiry the kernel records TSDP_ERR_TIMEOUT in `status`, drains,
-// frees its TMEM and returns.  No cluster launch, no multicast.
+// frees its TMEM and returns.  This form is launched without clusters; the CTA-pair form further down runs in clusters
+// of two.  No operand load is multicast in either: every CTA fetches its own tiles.
 #pragma once
 #include <cuda.h>
 #include "common.cuh"

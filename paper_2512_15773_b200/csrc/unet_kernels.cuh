@@ -62,8 +62,13 @@ gn_mish_kernel(const float* __restrict__ Y, const float* __restrict__ gam, const
   // Y may arrive as n_split partial sums of the convolution's reduction, split_stride elements apart: added here in
   // the order of the parts, whichever CTA produced which
   auto y_at = [&](size_t idx) {
-    float v = Y[idx];
-    for (int sp = 1; sp < n_split; ++sp) v += Y[idx + (size_t)sp * (size_t)split_stride];
+    if (n_split <= 1) return Y[idx];
+    float part[8];                               // at most 8 parts: all loads in flight together, added in order
+#pragma unroll
+    for (int sp = 0; sp < 8; ++sp) part[sp] = sp < n_split ? Y[idx + (size_t)sp * (size_t)split_stride] : 0.f;
+    float v = part[0];
+#pragma unroll
+    for (int sp = 1; sp < 8; ++sp) if (sp < n_split) v += part[sp];
     return v;
   };
   const int n = blockIdx.x / groups, grp = blockIdx.x % groups;

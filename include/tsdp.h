@@ -228,7 +228,10 @@ int tsdp_sample_chunk(tsdp_ctx* ctx, const float* d_obs, int B, int K, const tsd
  * DEVICE) are worked through `slots` <= max_B batch slots.  A slot whose request reaches t = -1 takes the
  * next waiting request inside the acceptance kernel (fresh x_T, t = T-1), so no slot idles while work
  * remains.  Request i draws the noise streams of environment i: its chunk equals the one
- * tsdp_sample_chunk returns for environment i of a batch of N with the same seed.  Per-request buffers grow
+ * tsdp_sample_chunk returns for environment i of a batch of N with the same seed -- bit for bit when both calls run
+ * the same kernels with sums in the same order (the networks are evaluated row by row); where the kernel choice or a
+ * split reduction depends on the number of slots (cluster kernels at small batches, TSDP_ARCH_UNET convolutions at
+ * small batches) the two agree to rounding only.  Per-request buffers grow
  * on demand (the only call besides tsdp_init / tsdp_load_weights that may allocate).  With a per-round
  * schedule the round index counts batched rounds of the whole call.  Errors as tsdp_sample_chunk. */
 int tsdp_serve(tsdp_ctx* ctx, const float* d_obs, int N, int slots, int K, const tsdp_accept_t* accept,

@@ -36,6 +36,8 @@
  * TSDP_NO_KSPLIT keeps the convolution GEMMs of TSDP_ARCH_UNET from splitting their reduction over idle SMs at small
  * batch (the split changes the order of the fp32 sums, so the last bits of a result depend on it; for a given
  * batch shape the result is the same on every run);
+ * TSDP_NO_AUX_STREAM keeps the 1x1 residual convolutions of TSDP_ARCH_UNET on the caller's stream instead of a second
+ * stream of the context beside the block's two kernel-5 convolutions (inside the round's CUDA graph: a parallel branch);
  * TSDP_VERBOSE prints the kernels' occupancy figures once per tsdp_load_weights.
  * Every function returns a tsdp_status; nothing throws or aborts.  A context is not re-entrant: one
  * call at a time.  There is no CPU fallback: without a CUDA device tsdp_init fails with TSDP_ERR_CUDA.

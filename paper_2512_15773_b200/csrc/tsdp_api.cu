@@ -130,6 +130,11 @@ struct tsdp_ctx {
   std::vector<void*> sched_allocs;
   cudaStream_t side_stream = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  // second stream of a forward: the 1x1 residual convolution of a UNet block runs beside the block's two kernel-5
+  // convolutions (it only needs the block's input) and joins in front of the block's last GroupNorm
+  cudaStream_t aux_stream = nullptr;
+  cudaEvent_t ev_aux_fork = nullptr, ev_aux_join = nullptr;
+  bool aux_on = true;                          // TSDP_NO_AUX_STREAM: everything on one stream
   // device time of the last chunk calls (ring buffer behind the latency percentiles of tsdp_stats)
   cudaEvent_t ev_chunk0 = nullptr, ev_chunk1 = nullptr;
   std::vector<float> lat_ring;
@@ -1004,11 +1009,19 @@ int unet_resblock(tsdp_ctx* c, Net& n, const Net::UBlock& b, const CandMap& cm, 
   int r;
   const long long ystr = (long long)rows * b.cout;      // distance of the partial-sum buffers of a split reduction
   const int s1 = conv_ksplit(c, rows - 4, b.cout, 5 * b.cin, n.uw.Y_cap), s2 = conv_ksplit(c, rows - 4, b.cout, 5 * b.cout, n.uw.Y_cap);
+  const bool fork = b.Wr != nullptr && c->aux_on && !c->prof_on;      // (per-launch timing keeps one stream)
+  if (fork) {      // the residual projection only needs xin: beside the two convolutions, on the second stream
+    CU_TRY(c, cudaEventRecord(c->ev_aux_fork, s));
+    CU_TRY(c, cudaStreamWaitEvent(c->aux_stream, c->ev_aux_fork, 0));
+    if ((r = gemm(c, xin, b.Wr, b.br, rows, b.cout, b.cin, EPI_F32, n.uw.R, b.cout, c->aux_stream))) return r;
+    CU_TRY(c, cudaEventRecord(c->ev_aux_join, c->aux_stream));
+  }
   if ((r = gemm(c, xin, b.W1, b.b1, rows - 4, b.cout, 5 * b.cin, EPI_F32, n.uw.Y, b.cout, s, nullptr, b.cin, s1, ystr))) return r;
   if ((r = unet_gn<T>(c, n, cm, n_cand, b.g1, b.be1, b.foff, nullptr, 0, nullptr, tmp, b.cout, 0, L, b.cout, s, s1, ystr))) return r;
   if ((r = gemm(c, tmp, b.W2, b.b2, rows - 4, b.cout, 5 * b.cout, EPI_F32, n.uw.Y, b.cout, s, nullptr, b.cout, s2, ystr))) return r;
   if (b.Wr) {
-    if ((r = gemm(c, xin, b.Wr, b.br, rows, b.cout, b.cin, EPI_F32, n.uw.R, b.cout, s))) return r;
+    if (fork) CU_TRY(c, cudaStreamWaitEvent(s, c->ev_aux_join, 0));
+    else if ((r = gemm(c, xin, b.Wr, b.br, rows, b.cout, b.cin, EPI_F32, n.uw.R, b.cout, s))) return r;
     return unet_gn<T>(c, n, cm, n_cand, b.g2, b.be2, -1, nullptr, 0, n.uw.R, dst, dst_pitch, coff, L, b.cout, s, s2, ystr);
   }
   return unet_gn<T>(c, n, cm, n_cand, b.g2, b.be2, -1, xin, b.cin, nullptr, dst, dst_pitch, coff, L, b.cout, s, s2, ystr);
@@ -1516,6 +1529,10 @@ int tsdp_init(const tsdp_config_t* cfg, tsdp_ctx** out) {
   INIT_TRY(cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking));
   INIT_TRY(cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
   INIT_TRY(cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming));
+  INIT_TRY(cudaStreamCreateWithFlags(&c->aux_stream, cudaStreamNonBlocking));
+  INIT_TRY(cudaEventCreateWithFlags(&c->ev_aux_fork, cudaEventDisableTiming));
+  INIT_TRY(cudaEventCreateWithFlags(&c->ev_aux_join, cudaEventDisableTiming));
+  c->aux_on = getenv("TSDP_NO_AUX_STREAM") == nullptr;
   INIT_TRY(cudaEventCreate(&c->ev_chunk0));
   INIT_TRY(cudaEventCreate(&c->ev_chunk1));
   c->lat_ring.assign(TSDP_LATENCY_RING, 0.f);
@@ -1660,6 +1677,9 @@ void tsdp_destroy(tsdp_ctx* c) {
   if (c->side_stream) cudaStreamDestroy(c->side_stream);
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
   if (c->ev_join) cudaEventDestroy(c->ev_join);
+  if (c->ev_aux_fork) cudaEventDestroy(c->ev_aux_fork);
+  if (c->ev_aux_join) cudaEventDestroy(c->ev_aux_join);
+  if (c->aux_stream) cudaStreamDestroy(c->aux_stream);
   if (c->ev_chunk0) cudaEventDestroy(c->ev_chunk0);
   if (c->ev_chunk1) cudaEventDestroy(c->ev_chunk1);
   dev_free_pool(c, c->sched_allocs);
